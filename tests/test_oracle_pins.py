@@ -1,0 +1,460 @@
+"""CPU pins for the oracle: each function is checked against something other than itself.
+
+Pins used: values printed in the figures of Appendix B (tests/golden), operator matrices
+built cell by cell with a brute-force owner search, closed forms (R after B = k * identity),
+library routines on the unpartitioned tensor (numpy.pad, scipy correlate2d, a plain matmul),
+and a hand-evaluated worked case for the order of the adjoint halo sums.
+"""
+
+import itertools
+import os
+
+import numpy as np
+import pytest
+from scipy.signal import correlate2d
+
+import oracle
+from oracle import Partition
+from paper_2006_03108_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# --------------------------------------------------------------------------
+# Appendix B figures
+# --------------------------------------------------------------------------
+
+def _load_appendix_b():
+    cases, cur = [], None
+    for line in open(os.path.join(GOLDEN, "appendix_b_halo_1d.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        tok = line.split()
+        if tok[0] == "case":
+            cur = dict(name=tok[1], workers=[])
+            cur.update({k: int(v) for k, v in (t.split("=") for t in tok[2:])})
+            cases.append(cur)
+        else:
+            kv = dict(t.split("=") for t in tok[2:])
+            rng = lambda s: tuple(int(v) for v in s.split(":"))
+            pair = lambda s: tuple(int(v) for v in s.split(","))
+            cur["workers"].append(dict(inp=rng(kv["in"]), out=rng(kv["out"]), halo=pair(kv["halo"]),
+                                       unused=pair(kv["unused"]), view=kv["view"].split(",")))
+    return cases
+
+
+APPENDIX_B = _load_appendix_b()
+
+
+@pytest.mark.parametrize("case", APPENDIX_B, ids=[c["name"] for c in APPENDIX_B])
+def test_halo_geometry_matches_appendix_b_figures(case):
+    got = oracle.halo_widths_1d(case["n"], case["p"], case["kernel"], case["stride"],
+                                case["dilation"], case["pad_lo"], case["pad_hi"])
+    assert len(got) == len(case["workers"]) == case["p"]
+    for g, w in zip(got, case["workers"]):
+        assert (g["in_start"], g["in_start"] + g["in_size"]) == w["inp"]
+        assert (g["out_start"], g["out_start"] + g["out_size"]) == w["out"]
+        assert (g["halo_lo"], g["halo_hi"]) == w["halo"]
+        assert (g["unused_lo"], g["unused_hi"]) == w["unused"]
+
+
+@pytest.mark.parametrize("case", APPENDIX_B, ids=[c["name"] for c in APPENDIX_B])
+@pytest.mark.parametrize("form", ["definition", "sequence"])
+def test_halo_fwd_reproduces_appendix_b_views(case, form):
+    """With x[g] = g + 1 the exchanged padded rows must show the indices the figures print."""
+    ws = case["workers"]
+    part = Partition((case["n"],), (case["p"],), [[w["halo"][0] for w in ws]], [[w["halo"][1] for w in ws]])
+    x = np.arange(1, case["n"] + 1, dtype=np.float32)
+    shards = oracle.scatter_global(part, x, fill=lambda w: np.full(part.padded_shape(w), 77.0))
+    H = oracle.halo_fwd_definition if form == "definition" else oracle.halo_fwd_sequence
+    out = H(part, shards)
+    for w, o in zip(ws, out):
+        expect = [0.0 if v == "-" else float(int(v) + 1) for v in w["view"]]
+        # the figures of the pooling cases draw unused inputs too: they are part of the bulk
+        assert o.tolist() == expect
+
+
+def test_balanced_split_from_appendix_b():
+    assert oracle.balanced_split(11, 3)[1] == [4, 4, 3]
+    assert oracle.balanced_split(7, 3)[1] == [3, 2, 2]
+    assert oracle.balanced_split(10, 3)[1] == [4, 3, 3]
+    assert oracle.balanced_split(20, 6) == ([0, 4, 8, 11, 14, 17], [4, 4, 3, 3, 3, 3])
+    assert oracle.balanced_split(10, 6)[1] == [2, 2, 2, 2, 1, 1]
+
+
+def test_worker_numbering_is_row_major():
+    # Appendix B.2: workers 0,1 are the top row of a 2 x 2 partition, 2,3 the bottom row.
+    part = Partition((4, 4), (2, 2))
+    assert [part.coords(w) for w in range(4)] == [(0, 0), (0, 1), (1, 0), (1, 1)]
+    assert part.bulk_start(1) == (0, 2) and part.bulk_start(2) == (2, 0)
+
+
+# --------------------------------------------------------------------------
+# Broadcast / sum-reduce
+# --------------------------------------------------------------------------
+
+def test_broadcast_and_sumreduce_dense_matrices():
+    n, k = 5, 3
+    Bm = np.vstack([np.eye(n)] * k)                      # [I; I; I]
+    x = inputs.uniform_pm1((n,), 1)
+    got = np.concatenate(oracle.broadcast_fwd(x, k))
+    assert np.array_equal(got, (Bm @ x.astype(np.float64)).astype(np.float32))
+    ys = [inputs.integers((n,), 10 + i) for i in range(k)]
+    got = oracle.sumreduce_fwd(ys)
+    assert np.array_equal(got, (Bm.T @ np.concatenate(ys).astype(np.float64)).astype(np.float32))
+    # operator matrices from unit vectors are each other's transpose
+    MB = np.stack([np.concatenate(oracle.broadcast_fwd(e, k)) for e in np.eye(n, dtype=np.float32)], 1)
+    MR = np.stack([oracle.sumreduce_fwd(np.split(e, k)) for e in np.eye(n * k, dtype=np.float32)], 1)
+    assert np.array_equal(MB, Bm) and np.array_equal(MR, Bm.T)
+
+
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_reduce_after_broadcast_is_k_times_identity(k):
+    x = inputs.uniform_pm1((1000,), 2)
+    got = oracle.sumreduce_fwd(oracle.broadcast_fwd(x, k))
+    if k <= 2:
+        assert np.array_equal(got, x * np.float32(k))    # x + x is exact
+    # the left fold rounds the odd multiples (3x, 5x, ...): at most k-2 roundings of 2^-24 each
+    assert np.all(np.abs(got.astype(np.float64) - k * x.astype(np.float64))
+                  <= (k - 1) * 2.0 ** -24 * k * np.abs(x.astype(np.float64)))
+    xi = inputs.integers((1000,), 2)
+    assert np.array_equal(oracle.sumreduce_fwd(oracle.broadcast_fwd(xi, k)), xi * np.float32(k))
+
+
+def test_sumreduce_order_and_signed_zero():
+    # fixed worker order: ((a + b) + c), not (a + (b + c))
+    a, b, c = np.float32(1e8), np.float32(-1e8), np.float32(1.0)
+    assert oracle.sumreduce_fwd([np.array([a]), np.array([b]), np.array([c])])[0] == np.float32(1.0)
+    assert oracle.sumreduce_fwd([np.array([c]), np.array([a]), np.array([b])])[0] == np.float32(0.0)
+    # the fold starts from y_0, so k = 1 keeps -0.0
+    z = oracle.sumreduce_fwd([np.array([-0.0], dtype=np.float32)])
+    assert np.signbit(z[0])
+    x = inputs.uniform_pm1((7,), 3)
+    assert oracle.sumreduce_fwd([x]).tobytes() == x.tobytes()
+
+
+def test_broadcast_dot_test_closed_form():
+    # <Bx, y> = <x, sum_i y_i>
+    k, n = 4, 257
+    x = inputs.uniform_pm1((n,), 4)
+    ys = [inputs.uniform_pm1((n,), 20 + i) for i in range(k)]
+    r = oracle.adjoint_test_ratio(oracle.broadcast_fwd(x, k), ys, [x], [oracle.broadcast_adj(ys)])
+    assert r < 1e-6
+
+
+def test_adjoint_ratio_known_values():
+    x = [np.array([1.0, 2.0])]
+    assert oracle.adjoint_test_ratio(x, x, x, x) == 0.0          # F = I
+    # F = 2I claimed adjoint I: <Fx,y> = 2*5, <x,F*y> = 5, norms: |Fx||y| = 10, |x||F*y| = 5
+    Fx = [np.array([2.0, 4.0])]
+    assert oracle.adjoint_test_ratio(Fx, x, x, x) == pytest.approx(0.5)
+
+
+# --------------------------------------------------------------------------
+# Halo exchange: brute-force matrices
+# --------------------------------------------------------------------------
+
+HALO_CASES = [
+    # global shape, partition, hlo, hhi
+    ((11,), (3,), 2, 2),
+    ((7,), (1,), 1, 2),
+    ((10,), (4,), [[0, 1, 2, 1]], [[1, 0, 2, 0]]),
+    ((6, 6), (2, 2), 1, 1),
+    ((7, 5), (3, 2), (1, 2), (2, 1)),
+    ((9, 8), (2, 2), [[0, 4], [3, 0]], [[2, 0], [0, 3]]),      # Appendix B.2 style widths
+    ((5, 6, 7), (2, 1, 3), (1, 2, 1), (1, 0, 2)),
+    ((4, 4, 4), (2, 2, 2), 1, 1),
+    ((6, 4), (3, 1), 2, 2),                                   # bulk 2 = halo: both-side receivers
+    ((3, 3, 2, 4), (1, 1, 2, 2), (0, 0, 1, 1), (0, 0, 1, 1)),
+]
+HALO_IDS = ["1d", "1d_p1", "1d_asym", "2d", "2d_uneven", "2d_appB2", "3d_uneven", "3d_corner", "thin", "4d"]
+
+
+def _cells(part):
+    """Flat list of (worker, padded-local index) and the offset of each worker's block."""
+    cells, off = [], []
+    for w in range(part.num_workers):
+        off.append(len(cells))
+        for l in itertools.product(*[range(v) for v in part.padded_shape(w)]):
+            cells.append((w, l))
+    return cells, off
+
+
+def _brute_force_H_matrix(part):
+    """0/1 matrix of H built cell by cell: each ghost cell looks for the worker owning its
+    global index by testing every worker's bulk box."""
+    cells, off = _cells(part)
+    index = {c: i for i, c in enumerate(cells)}
+    M = np.zeros((len(cells), len(cells)))
+    for i, (w, l) in enumerate(cells):
+        st, sh = part.bulk_start(w), part.bulk_shape(w)
+        lo, _ = part.widths(w)
+        g = tuple(st[k] - lo[k] + l[k] for k in range(part.rank))
+        in_bulk = all(lo[k] <= l[k] < lo[k] + sh[k] for k in range(part.rank))
+        if in_bulk:
+            M[i, i] = 1.0
+            continue
+        for v in range(part.num_workers):
+            vs, vh = part.bulk_start(v), part.bulk_shape(v)
+            if all(vs[k] <= g[k] < vs[k] + vh[k] for k in range(part.rank)):
+                vlo, _ = part.widths(v)
+                M[i, index[(v, tuple(g[k] - vs[k] + vlo[k] for k in range(part.rank)))]] = 1.0
+                break
+    return M
+
+
+def _flatten(shards):
+    return np.concatenate([np.asarray(s).ravel() for s in shards])
+
+
+def _unflatten(part, v, dtype=np.float32):
+    out, o = [], 0
+    for w in range(part.num_workers):
+        n = int(np.prod(part.padded_shape(w)))
+        out.append(np.array(v[o:o + n], dtype=dtype).reshape(part.padded_shape(w)))
+        o += n
+    return out
+
+
+def _operator_matrix(part, op):
+    n = sum(int(np.prod(part.padded_shape(w))) for w in range(part.num_workers))
+    cols = []
+    for i in range(n):
+        e = np.zeros(n, dtype=np.float32)
+        e[i] = 1.0
+        cols.append(_flatten(op(part, _unflatten(part, e))))
+    return np.stack(cols, 1)
+
+
+@pytest.mark.parametrize("case", HALO_CASES, ids=HALO_IDS)
+def test_halo_matrices_match_brute_force_and_transpose(case):
+    part = Partition(*case)
+    M = _brute_force_H_matrix(part)
+    assert np.array_equal(_operator_matrix(part, oracle.halo_fwd_definition), M)
+    assert np.array_equal(_operator_matrix(part, oracle.halo_fwd_sequence), M)
+    assert np.array_equal(_operator_matrix(part, oracle.halo_adj_sequence), M.T)
+
+
+def _random_shards(part, seed, kind="uniform"):
+    out = []
+    for w in range(part.num_workers):
+        gen = inputs.uniform_pm1 if kind == "uniform" else inputs.integers
+        out.append(gen(part.padded_shape(w), seed * 1000 + w))
+    return out
+
+
+@pytest.mark.parametrize("case", HALO_CASES, ids=HALO_IDS)
+def test_halo_forms_agree_bitwise_and_match_numpy_pad(case):
+    part = Partition(*case)
+    x = _random_shards(part, 5)                      # garbage in the ghosts
+    a = oracle.halo_fwd_definition(part, x)
+    b = oracle.halo_fwd_sequence(part, x)
+    g = oracle.assemble_global(part, x)
+    for w in range(part.num_workers):
+        assert a[w].tobytes() == b[w].tobytes()
+        # library pin: a window of the zero-padded global tensor
+        lo, hi = part.widths(w)
+        mlo, mhi = max(max(part.hlo[k]) for k in range(part.rank)), max(max(part.hhi[k]) for k in range(part.rank))
+        gp = np.pad(g, [(mlo, mhi)] * part.rank)
+        st, ps = part.bulk_start(w), part.padded_shape(w)
+        win = tuple(slice(st[k] - lo[k] + mlo, st[k] - lo[k] + mlo + ps[k]) for k in range(part.rank))
+        assert np.array_equal(a[w], gp[win])
+
+
+def test_halo_special_cases():
+    # a single worker: H only zeroes the ghosts
+    part = Partition((5, 4), (1, 1), 2, 1)
+    x = _random_shards(part, 6)
+    out = oracle.halo_fwd_sequence(part, x)[0]
+    ref = np.zeros_like(x[0])
+    ref[part.bulk_slices(0)] = x[0][part.bulk_slices(0)]
+    assert np.array_equal(out, ref)
+    # zero widths: H and H* are the identity
+    part = Partition((5, 4), (2, 2), 0, 0)
+    x = _random_shards(part, 7)
+    for op in (oracle.halo_fwd_definition, oracle.halo_fwd_sequence, oracle.halo_adj_sequence):
+        assert all(np.array_equal(a, b) for a, b in zip(op(part, x), x))
+
+
+@pytest.mark.parametrize("case", HALO_CASES, ids=HALO_IDS)
+def test_halo_adjoint_invariants(case):
+    part = Partition(*case)
+    M = _brute_force_H_matrix(part)
+    # integer-valued inputs: every summation order gives the same fp32 result
+    y = _random_shards(part, 8, "int")
+    got = oracle.halo_adj_sequence(part, y)
+    assert np.array_equal(_flatten(got), (M.T @ _flatten(y).astype(np.float64)).astype(np.float32))
+    # all ghosts are zero on exit
+    y = _random_shards(part, 9)
+    got = oracle.halo_adj_sequence(part, y)
+    for w in range(part.num_workers):
+        mask = np.ones(part.padded_shape(w), dtype=bool)
+        mask[part.bulk_slices(w)] = False
+        assert not got[w][mask].any()
+    # dot-product test
+    x = _random_shards(part, 10)
+    r = oracle.adjoint_test_ratio(oracle.halo_fwd_sequence(part, x), y, x, got)
+    assert r < 1e-6
+    # the sum over all cells is kept, up to what sits in exterior ghosts (dropped)
+    total = float(np.sum(M.T @ _flatten(y).astype(np.float64)))
+    assert float(np.sum(_flatten(got).astype(np.float64))) == pytest.approx(total, rel=1e-5, abs=1e-4)
+
+
+def test_halo_adjoint_order_worked_case():
+    """2 x 2 partition of a 2 x 2 tensor, width 1 everywhere: the single bulk cell of worker 0
+    receives from the ghosts of workers 1, 2 and 3.  The adjoint undoes dimension 1 first
+    (Appendix B.2: "adjoint of second phase" comes first), so
+        result = (own + w1's ghost) + (w2's ghost + w3's corner ghost),
+    evaluated here by hand in fp32 with values for which other orders differ."""
+    part = Partition((2, 2), (2, 2), 1, 1)
+    y = [np.zeros((3, 3), dtype=np.float32) for _ in range(4)]
+    own, g1, g2, g3 = np.float32(1.0), np.float32(1e8), np.float32(-1e8), np.float32(3.0)
+    y[0][1, 1] = own        # worker 0's bulk cell (global (0,0))
+    y[1][1, 0] = g1         # worker 1 (right of 0): its low ghost in dim 1
+    y[2][0, 1] = g2         # worker 2 (below 0): its low ghost in dim 0
+    y[3][0, 0] = g3         # worker 3 (diagonal): corner ghost
+    got = oracle.halo_adj_sequence(part, y)[0][1, 1]
+    expect = np.float32(np.float32(own + g1) + np.float32(g2 + g3))
+    assert got == expect == np.float32(0.0)
+    # a different association would not give this
+    assert np.float32(np.float32(np.float32(own + g1) + g2) + g3) == np.float32(3.0)
+
+
+def test_halo_adjoint_both_sides_low_first():
+    # 1-D, 3 workers, bulk 1, width 1: the middle cell receives from both neighbours, low first
+    part = Partition((3,), (3,), 1, 1)
+    y = [np.zeros(3, dtype=np.float32) for _ in range(3)]
+    y[1][1] = np.float32(1.0)
+    y[0][2] = np.float32(1e8)      # low neighbour's high ghost
+    y[2][0] = np.float32(-1e8)     # high neighbour's low ghost
+    got = oracle.halo_adj_sequence(part, y)[1][1]
+    assert got == np.float32(np.float32(np.float32(1.0) + np.float32(1e8)) + np.float32(-1e8)) == np.float32(0.0)
+
+
+def test_appendix_b2_unbalanced_2d_exchange():
+    """Appendix B.2 in words: 2 x 2 partition; workers 0 and 2 need nothing from 1 and 3 but
+    give them width 3; workers 0,1 need width 2 from 2,3; workers 2,3 need width 4 from 0,1."""
+    part = Partition((9, 8), (2, 2), [[0, 4], [0, 3]], [[2, 0], [0, 0]])
+    g = np.arange(72, dtype=np.float32).reshape(9, 8) + 1
+    x = oracle.scatter_global(part, g, fill=lambda w: np.full(part.padded_shape(w), -5.0))
+    a = oracle.halo_fwd_sequence(part, x)
+    assert a[0].shape == (5 + 2, 4) and a[1].shape == (5 + 2, 4 + 3)
+    assert a[2].shape == (4 + 4, 4) and a[3].shape == (4 + 4, 4 + 3)
+    assert np.array_equal(a[3], g[1:9, 1:8])          # rows 5-4.., cols 4-3..: a plain window
+    assert np.array_equal(a[1], g[0:7, 1:8])
+    assert np.array_equal(a[0], g[0:7, 0:4]) and np.array_equal(a[2], g[1:9, 0:4])
+
+
+# --------------------------------------------------------------------------
+# Convolution layer
+# --------------------------------------------------------------------------
+
+CONV_PARTS = [(1, 1, 1, 1), (1, 1, 2, 2), (1, 1, 3, 2), (1, 1, 1, 4)]
+
+
+def _conv_problem(pshape, shape=(2, 3, 12, 13), k=(5, 5), seed=11):
+    part = Partition(shape, pshape, (0, 0, k[0] // 2, k[1] // 2), (0, 0, k[0] // 2, k[1] // 2))
+    xg = inputs.normal(shape, seed)
+    w = inputs.normal((shape[1],) + k, seed + 1, 0.1)
+    return part, xg, w
+
+
+@pytest.mark.parametrize("pshape", CONV_PARTS)
+def test_conv_fwd_matches_scipy_on_global_tensor(pshape):
+    part, xg, w = _conv_problem(pshape)
+    bias = inputs.normal((xg.shape[1],), 13)
+    x = oracle.scatter_global(part, xg, fill=lambda wk: np.full(part.padded_shape(wk), 9.0))
+    y = oracle.assemble_global(Partition(xg.shape, pshape), oracle.conv_fwd(part, x, w, bias))
+    for n in range(xg.shape[0]):
+        for c in range(xg.shape[1]):
+            ref = correlate2d(xg[n, c].astype(np.float64), w[c].astype(np.float64), mode="same") + float(bias[c])
+            assert np.allclose(y[n, c], ref, rtol=0, atol=2e-6)
+
+
+@pytest.mark.parametrize("pshape", CONV_PARTS)
+def test_conv_adj_is_transpose_and_matches_stepwise_form(pshape):
+    part, xg, w = _conv_problem(pshape, shape=(1, 2, 7, 6), k=(5, 3))
+    ypart = Partition(xg.shape, pshape)
+    dyg = inputs.normal(xg.shape, 14)
+    dy = oracle.scatter_global(ypart, dyg)
+    dx = oracle.conv_adj(part, dy, w)
+    # library pin: the adjoint of a same-size correlation is the same-size convolution,
+    # i.e. correlation with the kernel rotated by 180 degrees
+    dxg = oracle.assemble_global(part, dx)
+    for c in range(xg.shape[1]):
+        ref = correlate2d(dyg[0, c].astype(np.float64), w[c, ::-1, ::-1].astype(np.float64), mode="same")
+        assert np.allclose(dxg[0, c], ref, rtol=0, atol=2e-6)
+    # ghosts are zero
+    for wk in range(part.num_workers):
+        mask = np.ones(part.padded_shape(wk), dtype=bool)
+        mask[part.bulk_slices(wk)] = False
+        assert not dx[wk][mask].any()
+    # step-by-step algorithm (local adjoint into padded shards, then H*)
+    dx2 = oracle.conv_adj_scatter_then_halo(part, dy, w)
+    for a, b in zip(dx, dx2):
+        assert np.allclose(a, b, rtol=0, atol=5e-6)
+    # dot-product test <Conv x, dy> = <x, Conv* dy> on the bulk
+    x = oracle.scatter_global(part, xg)
+    y = oracle.conv_fwd(part, x, w)
+    assert oracle.adjoint_test_ratio(y, dy, x, dx) < 1e-6
+
+
+def test_conv_unit_impulse_orientation():
+    # cross-correlation: an impulse at (i0, j0) puts w[a, b] at output (i0 - a + ph, j0 - b + pw)
+    part, _, w = _conv_problem((1, 1, 2, 2), shape=(1, 1, 8, 8))
+    xg = np.zeros((1, 1, 8, 8), dtype=np.float32)
+    xg[0, 0, 4, 3] = 1.0
+    y = oracle.assemble_global(Partition(xg.shape, part.pshape), oracle.conv_fwd(part, oracle.scatter_global(part, xg), w))
+    for a in range(5):
+        for b in range(5):
+            assert y[0, 0, 4 - a + 2, 3 - b + 2] == w[0, a, b]
+
+
+# --------------------------------------------------------------------------
+# Affine layer
+# --------------------------------------------------------------------------
+
+def _affine_problem(nb, nfi, nfo, pfo, pfi, seed, integer=False):
+    if integer:
+        xg = inputs.integers((nb, nfi), seed)
+        wg = inputs.integers((nfo, nfi), seed + 1)
+    else:
+        xg = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(inputs.normal((nb, nfi), seed)))
+        wg = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(inputs.normal((nfo, nfi), seed + 1, nfi ** -0.5)))
+    xs = np.split(xg, pfi, axis=1)
+    ws = [blk for row in np.split(wg, pfo, axis=0) for blk in np.split(row, pfi, axis=1)]
+    return xg, wg, xs, ws
+
+
+@pytest.mark.parametrize("pfo,pfi", [(1, 1), (2, 2), (4, 2), (1, 4)])
+def test_affine_matches_plain_matmul(pfo, pfi):
+    xg, wg, xs, ws = _affine_problem(6, 16, 8, pfo, pfi, 21, integer=True)
+    bias = inputs.integers((8,), 23)
+    y = np.concatenate(oracle.affine_fwd(xs, ws, pfo, pfi, np.split(bias, pfo)), axis=1)
+    assert np.array_equal(y, xg @ wg.T + bias[None, :])            # integers: exact, bias once
+    dyg = inputs.integers((6, 8), 24)
+    dx = np.concatenate(oracle.affine_adj(np.split(dyg, pfo, axis=1), ws, pfo, pfi), axis=1)
+    assert np.array_equal(dx, dyg @ wg)
+
+
+def test_affine_bf16_inputs_against_fp64_and_dot_test():
+    pfo = pfi = 2
+    xg, wg, xs, ws = _affine_problem(8, 64, 32, pfo, pfi, 25)
+    y = oracle.affine_fwd(xs, ws, pfo, pfi)
+    ref = xg.astype(np.float64) @ wg.astype(np.float64).T
+    assert np.allclose(np.concatenate(y, axis=1), ref, rtol=1e-6, atol=1e-6)
+    dyg = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(inputs.normal((8, 32), 26)))
+    dys = np.split(dyg, pfo, axis=1)
+    dx = oracle.affine_adj(dys, ws, pfo, pfi)
+    assert np.allclose(np.concatenate(dx, axis=1), dyg.astype(np.float64) @ wg.astype(np.float64), rtol=1e-6, atol=1e-6)
+    assert oracle.adjoint_test_ratio(y, dys, xs, dx) < 1e-6
+
+
+def test_bf16_helpers_round_to_nearest_even():
+    # 1 + 2^-8 is a tie between 1.0 (even mantissa) and 1 + 2^-7: goes to 1.0
+    a = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -2.5, 0.0], dtype=np.float32)
+    bits = inputs.f32_to_bf16_bits(a)
+    assert bits.tolist() == [0x3F80, 0x3F82, 0xC020, 0x0000]
+    assert oracle.bf16_bits_to_f64(bits).tolist() == [1.0, 1.0 + 2.0 ** -6, -2.5, 0.0]
+    assert inputs.bf16_bits_to_f32(bits).tolist() == [1.0, 1.0 + 2.0 ** -6, -2.5, 0.0]
