@@ -1,0 +1,204 @@
+/*
+ * distdl.h -- C ABI of the linear data-movement operators of Hewett & Grady,
+ * "A Linear Algebraic Approach to Model Parallelism in Deep Learning", and of
+ * the two distributed layers built from them, for P virtual workers whose
+ * shards all live in the memory of one GPU (sm_100a).
+ *
+ * General conventions
+ *   - Every data buffer is DEVICE memory owned by the caller.  Arrays of
+ *     pointers (`void *const *`) and arrays of shapes are HOST arrays; they are
+ *     read during the call and need not outlive it.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Operator calls validate on the host, enqueue their kernels on
+ *     that stream and return without synchronising.
+ *   - Every function returns a distdl_status_t.  On any error nothing is
+ *     launched; distdl_last_error() gives a thread-local message.  No function
+ *     aborts, throws or traps on the device.
+ *   - Every data pointer must be 16-byte aligned (DISTDL_ERR_ALIGNMENT).
+ *   - Workers are numbered by the row-major index of their partition
+ *     coordinate, last dimension fastest (Appendix B.2: in a 2 x 2 partition
+ *     workers 0,1 are the top row, 2,3 the bottom row).
+ *   - A shard is one contiguous row-major array of the padded shape
+ *     bulk[k] + halo_lo[k] + halo_hi[k]; the bulk (the part the worker owns,
+ *     Section 3 "Halo exchange") starts at index halo_lo[k] in each dimension.
+ *   - The library allocates device memory only inside distdl_partition_create*
+ *     (a few KB of plan tables, freed by distdl_partition_destroy).
+ */
+#ifndef DISTDL_H
+#define DISTDL_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DISTDL_OK = 0,
+    DISTDL_ERR_INVALID_ARG = 1, /* NULL pointer, bad count, forbidden aliasing           */
+    DISTDL_ERR_SHAPE = 2,       /* shapes / partition / halo widths inconsistent          */
+    DISTDL_ERR_ALIGNMENT = 3,   /* a data pointer is not 16-byte aligned                  */
+    DISTDL_ERR_UNSUPPORTED = 4, /* valid request outside what is implemented              */
+    DISTDL_ERR_CUDA = 5,        /* a CUDA runtime call failed (message has the detail)    */
+    DISTDL_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out (affine kernels)    */
+    DISTDL_ERR_NOMEM = 7
+} distdl_status_t;
+
+typedef enum { DISTDL_F32 = 0, DISTDL_BF16 = 1 } distdl_dtype_t;
+
+#define DISTDL_MAX_RANK 5
+#define DISTDL_MAX_WORKERS 256
+
+typedef struct distdl_partition distdl_partition_t; /* opaque, immutable after create */
+
+/* ------------------------------------------------------------------------
+ * Partition and halo geometry (host planner).
+ *
+ * Section 4: a rank-d tensor is partitioned along each dimension by a d-length
+ * partition vector of worker counts.  Section 3 / Appendix B: each extent is
+ * split evenly (n = q*p + r, the first r workers get q+1 -- the rule read from
+ * the index lists of Figs. B1-B4) and every side of every dimension of every
+ * worker may carry its own ghost width.
+ *
+ * distdl_partition_create: the same width halo_lo[k] / halo_hi[k] on the low /
+ *   high side of dimension k for every worker (NULL = all zero).  Ghosts on the
+ *   tensor's own boundary exist too and stand for zero padding (Fig. B1).
+ * distdl_partition_create_general: halo_lo[k] / halo_hi[k] point to
+ *   partition_shape[k] widths, one per worker coordinate along dimension k
+ *   (the unbalanced halos of Figs. B2-B4 and Appendix B.2).
+ *
+ * rank 1..DISTDL_MAX_RANK; product of partition_shape <= DISTDL_MAX_WORKERS;
+ * global_shape[k] >= partition_shape[k]; a ghost may not be wider than the
+ * adjacent worker's bulk (the paper assumes data from directly adjacent
+ * workers only) -> DISTDL_ERR_SHAPE.  The plan tables are uploaded with a
+ * synchronous copy on the current device.  *out is written only on success.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_partition_create(int32_t rank, const int64_t *global_shape,
+                                        const int32_t *partition_shape,
+                                        const int32_t *halo_lo, const int32_t *halo_hi,
+                                        distdl_dtype_t dtype, distdl_partition_t **out);
+distdl_status_t distdl_partition_create_general(int32_t rank, const int64_t *global_shape,
+                                                const int32_t *partition_shape,
+                                                const int32_t *const *halo_lo,
+                                                const int32_t *const *halo_hi,
+                                                distdl_dtype_t dtype, distdl_partition_t **out);
+void distdl_partition_destroy(distdl_partition_t *p); /* NULL is allowed */
+int32_t distdl_partition_num_workers(const distdl_partition_t *p); /* -1 if p is NULL */
+
+/* Extents of one worker's shard; each output array has `rank` entries and may be NULL. */
+distdl_status_t distdl_partition_shard_extents(const distdl_partition_t *p, int32_t worker,
+                                               int64_t *bulk_start, int64_t *bulk_shape,
+                                               int64_t *padded_shape, int32_t *halo_lo,
+                                               int32_t *halo_hi);
+
+/* Size of the host-built plan of H (adjoint = 0) or H* (adjoint != 0): number of boxes (one per
+ * shard and neighbour direction), number of thread-block tiles, and the algorithmic bytes of one
+ * application of the in-place method (H: every interior ghost cell read once from its owner and
+ * every ghost cell written once; H*: every receiving bulk cell read and written once, every
+ * interior ghost read once, every ghost cleared once).  Host only; outputs may be NULL. */
+distdl_status_t distdl_partition_halo_stats(const distdl_partition_t *p, int32_t adjoint,
+                                            int64_t *boxes, int64_t *tiles, int64_t *bytes);
+
+/* Halo widths of a 1-D sliding kernel (Section 3: "determined by the minimum and maximum global
+ * indices of the worker's output tensor and the size, stride, dilation, and padding parameters of
+ * the kernel"; worked cases: Figs. B1-B4).  Input length n and the output length
+ * floor((n + pad_lo + pad_hi - dilation*(kernel-1) - 1)/stride) + 1 are both split evenly over p
+ * workers.  Host only.  Each output array has p entries and may be NULL: halo widths, and the
+ * count of owned inputs at either end that the worker's outputs never read. */
+distdl_status_t distdl_halo_widths_1d(int64_t n, int32_t p, int32_t kernel, int32_t stride,
+                                      int32_t dilation, int32_t pad_lo, int32_t pad_hi,
+                                      int32_t *halo_lo, int32_t *halo_hi,
+                                      int32_t *unused_lo, int32_t *unused_hi);
+
+/* ------------------------------------------------------------------------
+ * Broadcast B and sum-reduce R = B* (Section 3, "Broadcast", "Sum-reduce").
+ *
+ * broadcast_fwd:  dst[i][e] = src[e], i < k          (B = k copies)
+ * sumreduce_fwd:  dst[e] = ((src[0][e] + src[1][e]) + ...) + src[k-1][e]
+ *                 in the arithmetic of `t`, fixed worker order, starting from src[0]
+ *                 (k = 1 is an exact copy).
+ * broadcast_adj == sumreduce_fwd, sumreduce_adj == broadcast_fwd (R = B*, R* = B).
+ *
+ * n = elements per realisation (n = 0 is a no-op), 1 <= k.  In broadcast a dst[i] equal to
+ * src is the in-place form (identity copy, skipped); any other overlap between buffers is not
+ * detected and gives undefined results.  In sum-reduce dst may equal src[0] only.
+ * F32 and BF16 are supported by the copies; the sums support F32 (BF16: UNSUPPORTED).
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_broadcast_fwd(const void *src, void *const *dst, int32_t k, int64_t n,
+                                     distdl_dtype_t t, void *stream);
+distdl_status_t distdl_broadcast_adj(const void *const *dy, void *dx, int32_t k, int64_t n,
+                                     distdl_dtype_t t, void *stream);
+distdl_status_t distdl_sumreduce_fwd(const void *const *src, void *dst, int32_t k, int64_t n,
+                                     distdl_dtype_t t, void *stream);
+distdl_status_t distdl_sumreduce_adj(const void *dy, void *const *dx, int32_t k, int64_t n,
+                                     distdl_dtype_t t, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Halo exchange H and its adjoint H* (Section 3, "Halo exchange": the H and H* operator
+ * sequences; Appendix B.2), in place on the P padded shards.
+ *
+ * halo_fwd: every ghost cell <- the bulk cell with the same global index (owned by a
+ *   neighbouring worker), or +0 where that index lies outside the tensor.  Bulk cells are
+ *   not written; previous ghost contents are never read.
+ * halo_adj: every bulk cell that some neighbour holds ghost copies of <- itself plus those
+ *   copies, summed in the nested order of H* (dimension d-1 undone first, so the sum is
+ *   grouped by dimension 0 outermost; within a dimension: own, low neighbour, high neighbour);
+ *   then every ghost cell <- 0.  F32 only.
+ * shards[w] = device pointer of worker w's padded shard, w < P (host array).
+ * Shards must not overlap one another.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_halo_fwd(const distdl_partition_t *p, void *const *shards, void *stream);
+distdl_status_t distdl_halo_adj(const distdl_partition_t *p, void *const *shards, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Distributed convolution layer, feature-space partition only (Section 4, "Sparse layers":
+ * forward / adjoint convolution algorithms and the closing remark that the broadcasts and
+ * reductions drop out when only the feature space is partitioned).
+ *
+ * p: rank-4 NCHW F32 partition of shape 1 x 1 x Ph x Pw whose halo widths are (kh-1)/2 rows and
+ *    (kw-1)/2 columns on every side (else DISTDL_ERR_SHAPE).  Depthwise, centred, stride 1,
+ *    kh = kw in {3, 5, 7} (else DISTDL_ERR_UNSUPPORTED).
+ * conv_fwd = H then the local cross-correlation, fused: y[n,c,i,j] = bias[c] +
+ *    sum_{a,b} w[c,a,b] * x[n,c,i+a-ph,j+b-pw] over the GLOBAL tensor with zeros outside.
+ *    x[w]: padded shards (only their bulk is read; ghost storage is neither read for its value
+ *    nor written).  y[w]: bulk-shaped shards (no ghosts).  w: [C,kh,kw] F32.  bias: [C] or NULL.
+ * conv_adj = local adjoint then H*, fused: dx[n,c,p,q] = sum_{a,b} w[c,a,b] *
+ *    dy[n,c,p-a+ph,q-b+pw] (zeros outside), written to the bulk of the padded shards dx[w],
+ *    whose ghosts are set to zero.  dy[w]: bulk-shaped shards.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_conv_fwd(const distdl_partition_t *p, const void *const *x, const void *w,
+                                const void *bias, int32_t kh, int32_t kw, void *const *y,
+                                void *stream);
+distdl_status_t distdl_conv_adj(const distdl_partition_t *p, const void *const *dy, const void *w,
+                                int32_t kh, int32_t kw, void *const *dx, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Distributed affine layer on a Pfo x Pfi worker grid (Section 4, "Dense layers": forward and
+ * adjoint affine algorithms).
+ *
+ * affine_fwd: x^_{ij} <- B x_j (along grid columns); y^_{ij} <- x^_{ij} W_{ij}^T (+ b_i on
+ *   column j = 0 only: the "one Pfo x 1 subset"); y_i <- R over j = 0..Pfi-1 in order.
+ * affine_adj: dy^_{ij} <- B dy_i (along grid rows); dx^_{ij} <- dy^_{ij} W_{ij};
+ *   dx_j <- R over i = 0..Pfo-1 in order.  (dW, db are not computed.)
+ * x[j]  BF16 [nb, nfi/Pfi]      w[i*Pfi+j]  BF16 [nfo/Pfo, nfi/Pfi]  (row-major)
+ * y[i]  F32  [nb, nfo/Pfo]      bias[i] F32 [nfo/Pfo] or bias == NULL
+ * dy[i] BF16 [nb, nfo/Pfo]      dx[j] F32 [nb, nfi/Pfi]
+ * The contraction runs on the tensor cores with fp32 accumulation; the sums of R continue in the
+ * same fp32 accumulator in the stated order.  nfi % Pfi == 0, nfo % Pfo == 0; the per-worker
+ * block sizes must be multiples of 64 and nb a multiple of 8, nb <= 256 per call
+ * (else DISTDL_ERR_UNSUPPORTED).
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                  const void *const *x, const void *const *w,
+                                  const void *const *bias, void *const *y, void *stream);
+distdl_status_t distdl_affine_adj(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                  const void *const *dy, const void *const *w, void *const *dx,
+                                  void *stream);
+
+/* Thread-local message of the last error returned on this thread ("" if none). */
+const char *distdl_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DISTDL_H */

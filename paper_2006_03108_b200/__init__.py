@@ -1,0 +1,250 @@
+"""Thin Python binding of the C-ABI library (include/distdl.h).
+
+Argument marshalling only: tensors are turned into device pointers and sizes, every step of
+every operator runs in the CUDA kernels of libdistdl.so.  There is no CPU or PyTorch fallback:
+if the library is missing or a call fails, an exception is raised.
+
+PyTorch is used by callers for device memory and streams; this module only reads
+`tensor.data_ptr()` and the current stream handle.
+"""
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdistdl.so")
+
+F32 = 0
+BF16 = 1
+MAX_RANK = 5
+
+STATUS_NAMES = {
+    0: "DISTDL_OK", 1: "DISTDL_ERR_INVALID_ARG", 2: "DISTDL_ERR_SHAPE", 3: "DISTDL_ERR_ALIGNMENT",
+    4: "DISTDL_ERR_UNSUPPORTED", 5: "DISTDL_ERR_CUDA", 6: "DISTDL_ERR_TIMEOUT", 7: "DISTDL_ERR_NOMEM",
+}
+
+
+class DistdlError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__("%s: %s" % (STATUS_NAMES.get(status, status), message))
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """Loads libdistdl.so (once) and declares the prototypes."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "libdistdl.so is not built: run `python -m paper_2006_03108_b200.build` "
+            "(there is no fallback path)")
+    L = ctypes.CDLL(LIB_PATH)
+    c_i32, c_i64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
+    pi32, pi64, pvp = ctypes.POINTER(c_i32), ctypes.POINTER(c_i64), ctypes.POINTER(vp)
+    ppi32 = ctypes.POINTER(pi32)
+    L.distdl_last_error.restype = ctypes.c_char_p
+    L.distdl_last_error.argtypes = []
+    L.distdl_partition_create.argtypes = [c_i32, pi64, pi32, pi32, pi32, c_i32, pvp]
+    L.distdl_partition_create_general.argtypes = [c_i32, pi64, pi32, ppi32, ppi32, c_i32, pvp]
+    L.distdl_partition_destroy.argtypes = [vp]
+    L.distdl_partition_destroy.restype = None
+    L.distdl_partition_num_workers.argtypes = [vp]
+    L.distdl_partition_shard_extents.argtypes = [vp, c_i32, pi64, pi64, pi64, pi32, pi32]
+    L.distdl_partition_halo_stats.argtypes = [vp, c_i32, pi64, pi64, pi64]
+    L.distdl_halo_widths_1d.argtypes = [c_i64, c_i32, c_i32, c_i32, c_i32, c_i32, c_i32, pi32, pi32, pi32, pi32]
+    L.distdl_broadcast_fwd.argtypes = [vp, pvp, c_i32, c_i64, c_i32, vp]
+    L.distdl_sumreduce_adj.argtypes = [vp, pvp, c_i32, c_i64, c_i32, vp]
+    L.distdl_sumreduce_fwd.argtypes = [pvp, vp, c_i32, c_i64, c_i32, vp]
+    L.distdl_broadcast_adj.argtypes = [pvp, vp, c_i32, c_i64, c_i32, vp]
+    L.distdl_halo_fwd.argtypes = [vp, pvp, vp]
+    L.distdl_halo_adj.argtypes = [vp, pvp, vp]
+    L.distdl_conv_fwd.argtypes = [vp, pvp, vp, vp, c_i32, c_i32, pvp, vp]
+    L.distdl_conv_adj.argtypes = [vp, pvp, vp, c_i32, c_i32, pvp, vp]
+    if hasattr(L, "distdl_affine_fwd"):
+        L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
+        L.distdl_affine_adj.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, vp]
+    _lib = L
+    return L
+
+
+def _check(status):
+    if status != 0:
+        raise DistdlError(status, lib().distdl_last_error().decode())
+
+
+def _ptr(t):
+    """Device (or host) address of a tensor-like, or of a raw int."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _ptr_array(ts):
+    arr = (ctypes.c_void_p * len(ts))()
+    for i, t in enumerate(ts):
+        arr[i] = _ptr(t)
+    return arr
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("unsupported dtype %s" % t.dtype)
+
+
+class Partition:
+    """Handle of a distdl_partition_t (see distdl_partition_create in include/distdl.h)."""
+
+    def __init__(self, global_shape, partition_shape, halo_lo=None, halo_hi=None, dtype=F32):
+        L = lib()
+        rank = len(global_shape)
+        if len(partition_shape) != rank:
+            raise ValueError("global_shape and partition_shape differ in rank")
+        self.rank = rank
+        self.global_shape = tuple(int(v) for v in global_shape)
+        self.partition_shape = tuple(int(v) for v in partition_shape)
+        self._h = ctypes.c_void_p()
+        gs = (ctypes.c_int64 * rank)(*self.global_shape)
+        ps = (ctypes.c_int32 * rank)(*self.partition_shape)
+
+        def general(h):
+            return h is not None and any(isinstance(v, (list, tuple)) for v in h)
+
+        if general(halo_lo) or general(halo_hi):
+            keep = []
+
+            def rows(h):
+                out = (ctypes.POINTER(ctypes.c_int32) * rank)()
+                for k in range(rank):
+                    hk = 0 if h is None else h[k]
+                    vals = list(hk) if isinstance(hk, (list, tuple)) else [int(hk)] * self.partition_shape[k]
+                    if len(vals) != self.partition_shape[k]:
+                        raise ValueError("halo width list %d has the wrong length" % k)
+                    a = (ctypes.c_int32 * len(vals))(*vals)
+                    keep.append(a)
+                    out[k] = ctypes.cast(a, ctypes.POINTER(ctypes.c_int32))
+                return out
+
+            _check(L.distdl_partition_create_general(rank, gs, ps, rows(halo_lo), rows(halo_hi), dtype,
+                                                     ctypes.byref(self._h)))
+        else:
+            lo = None if halo_lo is None else (ctypes.c_int32 * rank)(*[int(v) for v in halo_lo])
+            hi = None if halo_hi is None else (ctypes.c_int32 * rank)(*[int(v) for v in halo_hi])
+            _check(L.distdl_partition_create(rank, gs, ps, lo, hi, dtype, ctypes.byref(self._h)))
+        self.dtype = dtype
+        self.num_workers = L.distdl_partition_num_workers(self._h)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def shard_extents(self, worker):
+        """(bulk_start, bulk_shape, padded_shape, halo_lo, halo_hi) of one worker, as tuples."""
+        r = self.rank
+        a, b, c = (ctypes.c_int64 * r)(), (ctypes.c_int64 * r)(), (ctypes.c_int64 * r)()
+        lo, hi = (ctypes.c_int32 * r)(), (ctypes.c_int32 * r)()
+        _check(lib().distdl_partition_shard_extents(self._h, worker, a, b, c, lo, hi))
+        return tuple(a), tuple(b), tuple(c), tuple(lo), tuple(hi)
+
+    def padded_shape(self, worker):
+        return self.shard_extents(worker)[2]
+
+    def bulk_shape(self, worker):
+        return self.shard_extents(worker)[1]
+
+    def halo_stats(self, adjoint=False):
+        """(boxes, tiles, algorithmic bytes) of the H (or H*) plan."""
+        a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+        _check(lib().distdl_partition_halo_stats(self._h, 1 if adjoint else 0, ctypes.byref(a),
+                                                 ctypes.byref(b), ctypes.byref(c)))
+        return a.value, b.value, c.value
+
+    def close(self):
+        if self._h:
+            lib().distdl_partition_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def partition_create(global_shape, partition_shape, halo_lo=None, halo_hi=None, dtype=F32):
+    return Partition(global_shape, partition_shape, halo_lo, halo_hi, dtype)
+
+
+def halo_widths_1d(n, p, kernel, stride=1, dilation=1, pad_lo=0, pad_hi=0):
+    """Per-worker (halo_lo, halo_hi, unused_lo, unused_hi) lists of a 1-D sliding kernel."""
+    arrs = [(ctypes.c_int32 * p)() for _ in range(4)]
+    _check(lib().distdl_halo_widths_1d(n, p, kernel, stride, dilation, pad_lo, pad_hi, *arrs))
+    return tuple(list(a) for a in arrs)
+
+
+def broadcast_fwd(src, dsts, stream=None):
+    _check(lib().distdl_broadcast_fwd(_ptr(src), _ptr_array(dsts), len(dsts), src.numel(), _dtype_code(src),
+                                      _stream(stream)))
+
+
+def sumreduce_adj(dy, dxs, stream=None):
+    _check(lib().distdl_sumreduce_adj(_ptr(dy), _ptr_array(dxs), len(dxs), dy.numel(), _dtype_code(dy),
+                                      _stream(stream)))
+
+
+def sumreduce_fwd(srcs, dst, stream=None):
+    _check(lib().distdl_sumreduce_fwd(_ptr_array(srcs), _ptr(dst), len(srcs), dst.numel(), _dtype_code(dst),
+                                      _stream(stream)))
+
+
+def broadcast_adj(dys, dx, stream=None):
+    _check(lib().distdl_broadcast_adj(_ptr_array(dys), _ptr(dx), len(dys), dx.numel(), _dtype_code(dx),
+                                      _stream(stream)))
+
+
+def halo_fwd(part, shards, stream=None):
+    _check(lib().distdl_halo_fwd(part.handle, _ptr_array(shards), _stream(stream)))
+
+
+def halo_adj(part, shards, stream=None):
+    _check(lib().distdl_halo_adj(part.handle, _ptr_array(shards), _stream(stream)))
+
+
+def conv_fwd(part, x, w, bias, y, stream=None):
+    kh, kw = int(w.shape[-2]), int(w.shape[-1])
+    _check(lib().distdl_conv_fwd(part.handle, _ptr_array(x), _ptr(w), _ptr(bias), kh, kw, _ptr_array(y),
+                                 _stream(stream)))
+
+
+def conv_adj(part, dy, w, dx, stream=None):
+    kh, kw = int(w.shape[-2]), int(w.shape[-1])
+    _check(lib().distdl_conv_adj(part.handle, _ptr_array(dy), _ptr(w), kh, kw, _ptr_array(dx), _stream(stream)))
+
+
+def affine_fwd(nb, nfi, nfo, pfo, pfi, x, w, bias, y, stream=None):
+    b = None if bias is None else _ptr_array(bias)
+    _check(lib().distdl_affine_fwd(nb, nfi, nfo, pfo, pfi, _ptr_array(x), _ptr_array(w), b, _ptr_array(y),
+                                   _stream(stream)))
+
+
+def affine_adj(nb, nfi, nfo, pfo, pfi, dy, w, dx, stream=None):
+    _check(lib().distdl_affine_adj(nb, nfi, nfo, pfo, pfi, _ptr_array(dy), _ptr_array(w), _ptr_array(dx),
+                                   _stream(stream)))

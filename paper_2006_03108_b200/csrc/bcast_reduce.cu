@@ -1,0 +1,196 @@
+// Broadcast B (k copies of one realisation) and sum-reduce R = B* (fixed-order sum of k
+// realisations).  Section 3, "Broadcast" and "Sum-reduce and all-reduce".
+//
+// Both are pure streaming kernels: every input byte is read once and every output byte written
+// once with 16-byte accesses, several independent loads in flight per thread.
+#include <algorithm>
+
+#include "common.h"
+
+namespace distdl {
+
+constexpr int kMaxFan = 16;         // destinations (B) or sources (R) handled by one launch
+constexpr int kStreamThreads = 256;
+constexpr int kUnroll = 4;          // 16-byte vectors per thread per step
+
+struct FanPointers {
+    void *p[kMaxFan];
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// coherent variant: the buffer may also be written by this kernel (in-place fold)
+__device__ __forceinline__ uint4 ld_stream_coherent(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4 *p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// dst[j][i] = src[i] for j < k; nvec 16-byte vectors, then `tail` trailing bytes.
+__global__ void __launch_bounds__(kStreamThreads)
+broadcast_kernel(const uint4 *__restrict__ src, const __grid_constant__ FanPointers dst, int k, size_t nvec, int tail) {
+    const size_t stride = (size_t)gridDim.x * kStreamThreads;
+    size_t i = (size_t)blockIdx.x * kStreamThreads + threadIdx.x;
+    for (; i + (kUnroll - 1) * stride < nvec; i += kUnroll * stride) {
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u] = ld_stream(src + i + u * stride);
+        for (int j = 0; j < k; ++j) {
+            uint4 *d = reinterpret_cast<uint4 *>(dst.p[j]);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) st_stream(d + i + u * stride, v[u]);
+        }
+    }
+    for (; i < nvec; i += stride) {
+        const uint4 v = ld_stream(src + i);
+        for (int j = 0; j < k; ++j) st_stream(reinterpret_cast<uint4 *>(dst.p[j]) + i, v);
+    }
+    if (blockIdx.x == 0 && (int)threadIdx.x < tail) {
+        const unsigned char b = reinterpret_cast<const unsigned char *>(src + nvec)[threadIdx.x];
+        for (int j = 0; j < k; ++j) (reinterpret_cast<unsigned char *>(reinterpret_cast<uint4 *>(dst.p[j]) + nvec))[threadIdx.x] = b;
+    }
+}
+
+__device__ __forceinline__ uint4 add_f32x4(uint4 a, uint4 b) {
+    uint4 r;
+    r.x = __float_as_uint(__fadd_rn(__uint_as_float(a.x), __uint_as_float(b.x)));
+    r.y = __float_as_uint(__fadd_rn(__uint_as_float(a.y), __uint_as_float(b.y)));
+    r.z = __float_as_uint(__fadd_rn(__uint_as_float(a.z), __uint_as_float(b.z)));
+    r.w = __float_as_uint(__fadd_rn(__uint_as_float(a.w), __uint_as_float(b.w)));
+    return r;
+}
+
+// dst[i] = ((src[0][i] + src[1][i]) + ...) + src[k-1][i]   (fp32, left fold in source order)
+template <int K>
+__global__ void __launch_bounds__(kStreamThreads)
+sumreduce_kernel(const __grid_constant__ FanPointers src, float *__restrict__ dst, int k_runtime, size_t nvec, int tail) {
+    const int k = K > 0 ? K : k_runtime;
+    const size_t stride = (size_t)gridDim.x * kStreamThreads;
+    for (size_t i = (size_t)blockIdx.x * kStreamThreads + threadIdx.x; i < nvec; i += stride) {
+        uint4 v[K > 0 ? K : kMaxFan];
+#pragma unroll
+        for (int j = 0; j < (K > 0 ? K : kMaxFan); ++j)
+            if (j < k) v[j] = ld_stream_coherent(reinterpret_cast<const uint4 *>(src.p[j]) + i);
+        uint4 acc = v[0];
+#pragma unroll
+        for (int j = 1; j < (K > 0 ? K : kMaxFan); ++j)
+            if (j < k) acc = add_f32x4(acc, v[j]);
+        st_stream(reinterpret_cast<uint4 *>(dst) + i, acc);
+    }
+    if (blockIdx.x == 0 && (int)threadIdx.x < tail) {
+        const size_t e = nvec * 4 + threadIdx.x;
+        float acc = reinterpret_cast<const float *>(src.p[0])[e];
+        for (int j = 1; j < k; ++j) acc = __fadd_rn(acc, reinterpret_cast<const float *>(src.p[j])[e]);
+        dst[e] = acc;
+    }
+}
+
+static int stream_grid(size_t nvec, int per_thread) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const size_t want = (nvec + (size_t)kStreamThreads * per_thread - 1) / ((size_t)kStreamThreads * per_thread);
+    const size_t cap = (size_t)sms * 8;   // 8 resident blocks of 256 threads per SM
+    return (int)std::max<size_t>(1, std::min(want, cap));
+}
+
+static distdl_status_t broadcast_impl(const void *src, void *const *dst, int32_t k, int64_t n, distdl_dtype_t t,
+                                      void *stream, const char *what) {
+    clear_error();
+    if (!src || !dst) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (k < 1 || n < 0) return fail(DISTDL_ERR_INVALID_ARG, "%s: k = %d, n = %lld", what, k, (long long)n);
+    if (t != DISTDL_F32 && t != DISTDL_BF16) return fail(DISTDL_ERR_INVALID_ARG, "%s: bad dtype", what);
+    if (!aligned16(src)) return fail(DISTDL_ERR_ALIGNMENT, "%s: src is not 16-byte aligned", what);
+    for (int32_t j = 0; j < k; ++j) {
+        if (!dst[j]) return fail(DISTDL_ERR_INVALID_ARG, "%s: destination %d is NULL", what, j);
+        if (!aligned16(dst[j])) return fail(DISTDL_ERR_ALIGNMENT, "%s: destination %d is not 16-byte aligned", what, j);
+    }
+    if (n == 0) return DISTDL_OK;
+    const size_t bytes = (size_t)n * elem_size(t);
+    const size_t nvec = bytes / 16;
+    const int tail = (int)(bytes % 16);
+    const int grid = stream_grid(nvec, kUnroll);
+    // destinations in groups of kMaxFan; a destination equal to the source is the in-place form
+    FanPointers fp;
+    int filled = 0;
+    for (int32_t j = 0; j <= k; ++j) {
+        if (j < k && dst[j] != src) fp.p[filled++] = dst[j];
+        if (filled == kMaxFan || (j == k && filled > 0)) {
+            for (int r = filled; r < kMaxFan; ++r) fp.p[r] = nullptr;
+            broadcast_kernel<<<grid, kStreamThreads, 0, (cudaStream_t)stream>>>((const uint4 *)src, fp, filled, nvec, tail);
+            DISTDL_CUDA_CHECK(cudaGetLastError());
+            filled = 0;
+        }
+    }
+    return DISTDL_OK;
+}
+
+template <int K>
+static void launch_sum(const FanPointers &fp, float *dst, int k, size_t nvec, int tail, int grid, cudaStream_t s) {
+    sumreduce_kernel<K><<<grid, kStreamThreads, 0, s>>>(fp, dst, k, nvec, tail);
+}
+
+static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t k, int64_t n, distdl_dtype_t t,
+                                      void *stream, const char *what) {
+    clear_error();
+    if (!src || !dst) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (k < 1 || n < 0) return fail(DISTDL_ERR_INVALID_ARG, "%s: k = %d, n = %lld", what, k, (long long)n);
+    if (t == DISTDL_BF16) return fail(DISTDL_ERR_UNSUPPORTED, "%s: BF16 sums are not implemented", what);
+    if (t != DISTDL_F32) return fail(DISTDL_ERR_INVALID_ARG, "%s: bad dtype", what);
+    if (!aligned16(dst)) return fail(DISTDL_ERR_ALIGNMENT, "%s: dst is not 16-byte aligned", what);
+    for (int32_t j = 0; j < k; ++j) {
+        if (!src[j]) return fail(DISTDL_ERR_INVALID_ARG, "%s: source %d is NULL", what, j);
+        if (!aligned16(src[j])) return fail(DISTDL_ERR_ALIGNMENT, "%s: source %d is not 16-byte aligned", what, j);
+        if (j > 0 && src[j] == dst) return fail(DISTDL_ERR_INVALID_ARG, "%s: dst may alias source 0 only", what);
+    }
+    if (n == 0) return DISTDL_OK;
+    const size_t nvec = (size_t)n / 4;
+    const int tail = (int)(n % 4);
+    const int grid = stream_grid(nvec, 1);
+    // sources in groups of kMaxFan; later groups continue the fold from dst, which keeps the order
+    int32_t done = 0;
+    while (done < k) {
+        FanPointers fp;
+        int filled = 0;
+        if (done > 0) fp.p[filled++] = dst;
+        while (filled < kMaxFan && done < k) fp.p[filled++] = const_cast<void *>(src[done++]);
+        for (int r = filled; r < kMaxFan; ++r) fp.p[r] = nullptr;
+        cudaStream_t s = (cudaStream_t)stream;
+        switch (filled) {
+            case 1: launch_sum<1>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
+            case 2: launch_sum<2>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
+            case 4: launch_sum<4>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
+            case 8: launch_sum<8>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
+            default: launch_sum<0>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
+        }
+        DISTDL_CUDA_CHECK(cudaGetLastError());
+    }
+    return DISTDL_OK;
+}
+
+}  // namespace distdl
+
+extern "C" distdl_status_t distdl_broadcast_fwd(const void *src, void *const *dst, int32_t k, int64_t n,
+                                                distdl_dtype_t t, void *stream) {
+    return distdl::broadcast_impl(src, dst, k, n, t, stream, "broadcast_fwd");
+}
+extern "C" distdl_status_t distdl_sumreduce_adj(const void *dy, void *const *dx, int32_t k, int64_t n,
+                                                distdl_dtype_t t, void *stream) {
+    return distdl::broadcast_impl(dy, dx, k, n, t, stream, "sumreduce_adj");
+}
+extern "C" distdl_status_t distdl_sumreduce_fwd(const void *const *src, void *dst, int32_t k, int64_t n,
+                                                distdl_dtype_t t, void *stream) {
+    return distdl::sumreduce_impl(src, dst, k, n, t, stream, "sumreduce_fwd");
+}
+extern "C" distdl_status_t distdl_broadcast_adj(const void *const *dy, void *dx, int32_t k, int64_t n,
+                                                distdl_dtype_t t, void *stream) {
+    return distdl::sumreduce_impl(dy, dx, k, n, t, stream, "broadcast_adj");
+}

@@ -1,0 +1,130 @@
+// Shared host-side helpers of the library: error reporting and the partition object.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "distdl.h"
+
+namespace distdl {
+
+// Records a thread-local message and returns `code`.
+distdl_status_t fail(distdl_status_t code, const char *fmt, ...);
+void clear_error();
+
+#define DISTDL_CUDA_CHECK(expr)                                                          \
+    do {                                                                                 \
+        cudaError_t e__ = (expr);                                                        \
+        if (e__ != cudaSuccess)                                                          \
+            return ::distdl::fail(DISTDL_ERR_CUDA, "%s failed: %s", #expr,               \
+                                  cudaGetErrorString(e__));                              \
+    } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int elem_size(distdl_dtype_t t) { return t == DISTDL_F32 ? 4 : 2; }
+
+// ---------------------------------------------------------------------------------------------
+// Device-side plan tables of the halo kernels.
+//
+// A *box* is a rectangular set of cells of one destination shard together with the list of
+// source boxes (same shape, possibly in other shards) whose values are combined into it.
+// A box with no source is cleared; a box with one source is a copy; a box with several sources
+// is the nested sum of H*.  A *tile* is a contiguous range of a box's flattened index space;
+// one thread block processes one tile.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxBoxDims = DISTDL_MAX_RANK;
+constexpr int kMaxLevels = DISTDL_MAX_RANK;   // nesting depth of the H* sum
+constexpr int kMaxSources = 32;               // sources of one box (2^5, or 3^3 for thin shards)
+
+struct HaloSource {
+    int32_t shard;                 // shard the source cells live in
+    int32_t close;                 // how many nesting levels are folded after adding this source
+    int32_t clear_after;           // 1: source cells are set to zero once read (ghost sources)
+    int32_t pad_;
+    int64_t offset;                // element offset of the box origin inside the shard
+    int64_t stride[kMaxBoxDims];   // element stride per box dimension (innermost last)
+};
+
+struct HaloBox {
+    int32_t dst_shard;
+    int32_t ndim;                  // box dimensions kept after dropping extent-1 dimensions
+    int32_t nsrc;
+    int32_t src_begin;             // index of the first source in the source table
+    int32_t vec;                   // 1: every offset, stride and extent allows 16-byte accesses
+    int32_t levels;                // nesting levels of the sum (>= 1)
+    int32_t shape[kMaxBoxDims];    // extents; innermost in units of `vec ? 16 bytes : elements`
+    int32_t pad_;
+    int64_t dst_offset;
+    int64_t dst_stride[kMaxBoxDims];
+};
+
+struct HaloTile {
+    int32_t box;
+    uint32_t first;                // first flattened unit of the tile
+    uint32_t count;                // units in the tile
+};
+
+struct HaloPlanHost {
+    std::vector<HaloBox> boxes;
+    std::vector<HaloSource> sources;
+    std::vector<HaloTile> tiles;
+    int64_t algorithmic_bytes = 0; // bytes read + written by the in-place method
+};
+
+struct HaloPlanDevice {
+    HaloBox *boxes = nullptr;
+    HaloSource *sources = nullptr;
+    HaloTile *tiles = nullptr;
+    int32_t num_tiles = 0;
+};
+
+}  // namespace distdl
+
+// The opaque partition object of the C ABI.
+struct distdl_partition {
+    int32_t rank = 0;
+    distdl_dtype_t dtype = DISTDL_F32;
+    int32_t num_workers = 0;
+    int device = 0;
+    int64_t global_shape[DISTDL_MAX_RANK] = {0};
+    int32_t pshape[DISTDL_MAX_RANK] = {0};
+    // per dimension, per worker coordinate along that dimension
+    std::vector<int64_t> start[DISTDL_MAX_RANK];
+    std::vector<int64_t> size[DISTDL_MAX_RANK];
+    std::vector<int32_t> hlo[DISTDL_MAX_RANK];
+    std::vector<int32_t> hhi[DISTDL_MAX_RANK];
+
+    distdl::HaloPlanHost fwd_host, adj_host;
+    distdl::HaloPlanDevice fwd_dev, adj_dev;
+    void *device_block = nullptr;   // one allocation holding all device tables
+
+    void coords(int32_t worker, int32_t *c) const {
+        for (int k = rank - 1; k >= 0; --k) {
+            c[k] = worker % pshape[k];
+            worker /= pshape[k];
+        }
+    }
+    int32_t worker_of(const int32_t *c) const {
+        int32_t w = 0;
+        for (int k = 0; k < rank; ++k) w = w * pshape[k] + c[k];
+        return w;
+    }
+    int64_t padded_extent(int k, int32_t c) const { return size[k][c] + hlo[k][c] + hhi[k][c]; }
+    int64_t shard_elems(int32_t worker) const {
+        int32_t c[DISTDL_MAX_RANK];
+        coords(worker, c);
+        int64_t n = 1;
+        for (int k = 0; k < rank; ++k) n *= padded_extent(k, c[k]);
+        return n;
+    }
+};
+
+namespace distdl {
+// Builds the forward (H) and adjoint (H*) box/tile lists of a partition (host only).
+distdl_status_t build_halo_plans(distdl_partition *p);
+// Checks every box of a plan: inside its shard, destination boxes pairwise disjoint.
+distdl_status_t validate_halo_plan(const distdl_partition *p, const HaloPlanHost &plan);
+}  // namespace distdl

@@ -1,0 +1,177 @@
+// Partition object of the C ABI: creation, queries, upload of the halo plan tables.
+#include <cstring>
+#include <new>
+
+#include "common.h"
+
+using namespace distdl;
+
+static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
+                                   const int32_t *const *hlo, const int32_t *const *hhi,
+                                   const int32_t *ulo, const int32_t *uhi, distdl_dtype_t dtype,
+                                   distdl_partition_t **out) {
+    clear_error();
+    if (!out) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: out is NULL");
+    if (rank < 1 || rank > DISTDL_MAX_RANK)
+        return fail(DISTDL_ERR_INVALID_ARG, "partition_create: rank %d outside 1..%d", rank, DISTDL_MAX_RANK);
+    if (!global_shape || !partition_shape) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: NULL shape");
+    if (dtype != DISTDL_F32 && dtype != DISTDL_BF16) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: bad dtype");
+    int64_t workers = 1;
+    for (int k = 0; k < rank; ++k) {
+        if (partition_shape[k] < 1) return fail(DISTDL_ERR_SHAPE, "partition_create: partition_shape[%d] < 1", k);
+        if (global_shape[k] < partition_shape[k])
+            return fail(DISTDL_ERR_SHAPE, "partition_create: global_shape[%d] smaller than the worker count", k);
+        workers *= partition_shape[k];
+        if (workers > DISTDL_MAX_WORKERS)
+            return fail(DISTDL_ERR_UNSUPPORTED, "partition_create: more than %d workers", DISTDL_MAX_WORKERS);
+    }
+    distdl_partition *p = new (std::nothrow) distdl_partition();
+    if (!p) return fail(DISTDL_ERR_NOMEM, "partition_create: out of host memory");
+    p->rank = rank;
+    p->dtype = dtype;
+    p->num_workers = (int32_t)workers;
+    for (int k = 0; k < rank; ++k) {
+        p->global_shape[k] = global_shape[k];
+        p->pshape[k] = partition_shape[k];
+        const int32_t pk = partition_shape[k];
+        const int64_t q = global_shape[k] / pk, r = global_shape[k] % pk;
+        int64_t at = 0;
+        for (int32_t c = 0; c < pk; ++c) {
+            const int64_t sz = q + (c < r ? 1 : 0);   // first r workers get one more
+            p->start[k].push_back(at);
+            p->size[k].push_back(sz);
+            at += sz;
+            const int32_t lo = hlo ? (hlo[k] ? hlo[k][c] : 0) : (ulo ? ulo[k] : 0);
+            const int32_t hi = hhi ? (hhi[k] ? hhi[k][c] : 0) : (uhi ? uhi[k] : 0);
+            if (lo < 0 || hi < 0) {
+                delete p;
+                return fail(DISTDL_ERR_SHAPE, "partition_create: negative halo width in dimension %d", k);
+            }
+            p->hlo[k].push_back(lo);
+            p->hhi[k].push_back(hi);
+        }
+        // a ghost may only hold cells of the directly adjacent worker
+        for (int32_t c = 0; c < pk; ++c) {
+            if (c > 0 && p->hlo[k][c] > p->size[k][c - 1]) {
+                delete p;
+                return fail(DISTDL_ERR_SHAPE, "partition_create: low halo of worker coordinate %d in dimension %d is wider than its neighbour's bulk", c, k);
+            }
+            if (c + 1 < pk && p->hhi[k][c] > p->size[k][c + 1]) {
+                delete p;
+                return fail(DISTDL_ERR_SHAPE, "partition_create: high halo of worker coordinate %d in dimension %d is wider than its neighbour's bulk", c, k);
+            }
+        }
+    }
+    for (int32_t w = 0; w < p->num_workers; ++w)
+        if (p->shard_elems(w) >= (int64_t)1 << 40) {
+            delete p;
+            return fail(DISTDL_ERR_UNSUPPORTED, "partition_create: shard too large");
+        }
+    distdl_status_t st = build_halo_plans(p);
+    if (st != DISTDL_OK) {
+        delete p;
+        return st;
+    }
+    // Upload.  Without a CUDA device the object stays host-only: geometry queries work, operator
+    // calls report DISTDL_ERR_CUDA.
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
+        cudaGetDevice(&p->device);
+        auto bytes_of = [](const HaloPlanHost &h, size_t *b, size_t *s, size_t *t) {
+            auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+            *b = up(h.boxes.size() * sizeof(HaloBox));
+            *s = up(h.sources.size() * sizeof(HaloSource));
+            *t = up(h.tiles.size() * sizeof(HaloTile));
+        };
+        size_t fbz, fsz, ftz, abz, asz, atz;
+        bytes_of(p->fwd_host, &fbz, &fsz, &ftz);
+        bytes_of(p->adj_host, &abz, &asz, &atz);
+        const size_t total = fbz + fsz + ftz + abz + asz + atz + 256;
+        cudaError_t e = cudaMalloc(&p->device_block, total);
+        if (e != cudaSuccess) {
+            delete p;
+            return fail(DISTDL_ERR_NOMEM, "partition_create: cudaMalloc(%zu) failed: %s", total, cudaGetErrorString(e));
+        }
+        char *at = (char *)p->device_block;
+        auto put = [&](const void *src, size_t n, size_t reserved) -> void * {
+            void *dst = at;
+            if (n && e == cudaSuccess) e = cudaMemcpy(dst, src, n, cudaMemcpyHostToDevice);
+            at += reserved;
+            return dst;
+        };
+        p->fwd_dev.boxes = (HaloBox *)put(p->fwd_host.boxes.data(), p->fwd_host.boxes.size() * sizeof(HaloBox), fbz);
+        p->fwd_dev.sources = (HaloSource *)put(p->fwd_host.sources.data(), p->fwd_host.sources.size() * sizeof(HaloSource), fsz);
+        p->fwd_dev.tiles = (HaloTile *)put(p->fwd_host.tiles.data(), p->fwd_host.tiles.size() * sizeof(HaloTile), ftz);
+        p->fwd_dev.num_tiles = (int32_t)p->fwd_host.tiles.size();
+        p->adj_dev.boxes = (HaloBox *)put(p->adj_host.boxes.data(), p->adj_host.boxes.size() * sizeof(HaloBox), abz);
+        p->adj_dev.sources = (HaloSource *)put(p->adj_host.sources.data(), p->adj_host.sources.size() * sizeof(HaloSource), asz);
+        p->adj_dev.tiles = (HaloTile *)put(p->adj_host.tiles.data(), p->adj_host.tiles.size() * sizeof(HaloTile), atz);
+        p->adj_dev.num_tiles = (int32_t)p->adj_host.tiles.size();
+        if (e != cudaSuccess) {
+            cudaFree(p->device_block);
+            delete p;
+            return fail(DISTDL_ERR_CUDA, "partition_create: upload failed: %s", cudaGetErrorString(e));
+        }
+    } else {
+        cudaGetLastError();
+    }
+    *out = p;
+    return DISTDL_OK;
+}
+
+extern "C" distdl_status_t distdl_partition_create(int32_t rank, const int64_t *global_shape,
+                                                   const int32_t *partition_shape, const int32_t *halo_lo,
+                                                   const int32_t *halo_hi, distdl_dtype_t dtype,
+                                                   distdl_partition_t **out) {
+    return create_impl(rank, global_shape, partition_shape, nullptr, nullptr, halo_lo, halo_hi, dtype, out);
+}
+
+extern "C" distdl_status_t distdl_partition_create_general(int32_t rank, const int64_t *global_shape,
+                                                           const int32_t *partition_shape,
+                                                           const int32_t *const *halo_lo,
+                                                           const int32_t *const *halo_hi, distdl_dtype_t dtype,
+                                                           distdl_partition_t **out) {
+    static const int32_t *const none[DISTDL_MAX_RANK] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    return create_impl(rank, global_shape, partition_shape, halo_lo ? halo_lo : none, halo_hi ? halo_hi : none,
+                       nullptr, nullptr, dtype, out);
+}
+
+extern "C" void distdl_partition_destroy(distdl_partition_t *p) {
+    if (!p) return;
+    if (p->device_block) cudaFree(p->device_block);
+    delete p;
+}
+
+extern "C" int32_t distdl_partition_num_workers(const distdl_partition_t *p) { return p ? p->num_workers : -1; }
+
+extern "C" distdl_status_t distdl_partition_shard_extents(const distdl_partition_t *p, int32_t worker,
+                                                          int64_t *bulk_start, int64_t *bulk_shape,
+                                                          int64_t *padded_shape, int32_t *halo_lo,
+                                                          int32_t *halo_hi) {
+    clear_error();
+    if (!p) return fail(DISTDL_ERR_INVALID_ARG, "shard_extents: partition is NULL");
+    if (worker < 0 || worker >= p->num_workers)
+        return fail(DISTDL_ERR_INVALID_ARG, "shard_extents: worker %d outside 0..%d", worker, p->num_workers - 1);
+    int32_t c[DISTDL_MAX_RANK];
+    p->coords(worker, c);
+    for (int k = 0; k < p->rank; ++k) {
+        if (bulk_start) bulk_start[k] = p->start[k][c[k]];
+        if (bulk_shape) bulk_shape[k] = p->size[k][c[k]];
+        if (padded_shape) padded_shape[k] = p->padded_extent(k, c[k]);
+        if (halo_lo) halo_lo[k] = p->hlo[k][c[k]];
+        if (halo_hi) halo_hi[k] = p->hhi[k][c[k]];
+    }
+    return DISTDL_OK;
+}
+
+// Plan statistics (host): number of boxes and tiles and the algorithmic bytes of one H or H*.
+extern "C" distdl_status_t distdl_partition_halo_stats(const distdl_partition_t *p, int32_t adjoint,
+                                                       int64_t *boxes, int64_t *tiles, int64_t *bytes) {
+    clear_error();
+    if (!p) return fail(DISTDL_ERR_INVALID_ARG, "halo_stats: partition is NULL");
+    const HaloPlanHost &h = adjoint ? p->adj_host : p->fwd_host;
+    if (boxes) *boxes = (int64_t)h.boxes.size();
+    if (tiles) *tiles = (int64_t)h.tiles.size();
+    if (bytes) *bytes = h.algorithmic_bytes;
+    return DISTDL_OK;
+}

@@ -1,0 +1,404 @@
+// Host planner: partition geometry (balanced split, per-side ghost widths) and the box / tile
+// lists that the halo kernels execute.  Section 3 "Halo exchange", Section 4 (partition vector),
+// Appendix B (worked geometry examples).
+#include <algorithm>
+#include <array>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.h"
+
+namespace distdl {
+
+static thread_local char g_error[512] = "";
+
+distdl_status_t fail(distdl_status_t code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+    return code;
+}
+void clear_error() { g_error[0] = 0; }
+
+}  // namespace distdl
+
+extern "C" const char *distdl_last_error(void) { return distdl::g_error; }
+
+using namespace distdl;
+
+// ---------------------------------------------------------------------------------------------
+// Balanced split and 1-D halo widths
+// ---------------------------------------------------------------------------------------------
+static void balanced_split(int64_t n, int32_t p, std::vector<int64_t> &start, std::vector<int64_t> &size) {
+    const int64_t q = n / p, r = n % p;
+    start.resize(p);
+    size.resize(p);
+    int64_t at = 0;
+    for (int32_t c = 0; c < p; ++c) {
+        size[c] = q + (c < r ? 1 : 0);
+        start[c] = at;
+        at += size[c];
+    }
+}
+
+extern "C" distdl_status_t distdl_halo_widths_1d(int64_t n, int32_t p, int32_t kernel, int32_t stride,
+                                                 int32_t dilation, int32_t pad_lo, int32_t pad_hi,
+                                                 int32_t *halo_lo, int32_t *halo_hi,
+                                                 int32_t *unused_lo, int32_t *unused_hi) {
+    clear_error();
+    if (n < 1 || p < 1 || kernel < 1 || stride < 1 || dilation < 1 || pad_lo < 0 || pad_hi < 0)
+        return fail(DISTDL_ERR_INVALID_ARG, "halo_widths_1d: non-positive argument");
+    const int64_t reach = (int64_t)dilation * (kernel - 1);
+    const int64_t span = n + pad_lo + pad_hi - reach - 1;
+    if (span < 0) return fail(DISTDL_ERR_SHAPE, "halo_widths_1d: kernel larger than padded input");
+    const int64_t m = span / stride + 1;
+    std::vector<int64_t> is, iz, os, oz;
+    balanced_split(n, p, is, iz);
+    balanced_split(m, p, os, oz);
+    for (int32_t c = 0; c < p; ++c) {
+        const int64_t own_first = is[c], own_last = is[c] + iz[c] - 1;
+        int64_t need_first = own_first, need_last = own_first - 1;   // empty range if no outputs
+        if (oz[c] > 0) {
+            need_first = os[c] * stride - pad_lo;
+            need_last = (os[c] + oz[c] - 1) * stride - pad_lo + reach;
+        }
+        const int64_t hl = std::max<int64_t>(0, own_first - need_first);
+        const int64_t hh = std::max<int64_t>(0, need_last - own_last);
+        const int64_t ul = std::max<int64_t>(0, std::min(need_first, own_last + 1) - own_first);
+        const int64_t uh = std::max<int64_t>(0, own_last - std::max(need_last, own_first - 1));
+        if (halo_lo) halo_lo[c] = (int32_t)hl;
+        if (halo_hi) halo_hi[c] = (int32_t)hh;
+        if (unused_lo) unused_lo[c] = (int32_t)ul;
+        if (unused_hi) unused_hi[c] = (int32_t)uh;
+    }
+    return DISTDL_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Box construction
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct Region {             // a rectangular set of cells of one shard, in padded-local indices
+    int32_t shard;
+    int64_t start[DISTDL_MAX_RANK];
+    int64_t extent[DISTDL_MAX_RANK];
+};
+
+struct PendingSource {
+    Region r;
+    int32_t close;
+    int32_t clear_after;
+};
+
+constexpr uint32_t kTileUnits = 2048;
+
+struct Builder {
+    const distdl_partition *p;
+    HaloPlanHost *plan;
+    std::vector<Region> dst_regions;   // for the disjointness check
+    int esize;
+
+    void strides_of(int32_t shard, int64_t *stride) const {
+        int32_t c[DISTDL_MAX_RANK];
+        p->coords(shard, c);
+        int64_t s = 1;
+        for (int k = p->rank - 1; k >= 0; --k) {
+            stride[k] = s;
+            s *= p->padded_extent(k, c[k]);
+        }
+    }
+    bool inside(const Region &r) const {
+        int32_t c[DISTDL_MAX_RANK];
+        p->coords(r.shard, c);
+        for (int k = 0; k < p->rank; ++k)
+            if (r.start[k] < 0 || r.extent[k] < 0 || r.start[k] + r.extent[k] > p->padded_extent(k, c[k]))
+                return false;
+        return true;
+    }
+
+    // Adds one box; `srcs` may be empty (clear).  Returns false on an internal inconsistency.
+    bool add(const Region &dst, const std::vector<PendingSource> &srcs, int levels) {
+        const int d = p->rank;
+        int64_t cells = 1;
+        for (int k = 0; k < d; ++k) cells *= dst.extent[k];
+        if (cells == 0) return true;
+        if (!inside(dst)) return false;
+        for (const auto &s : srcs) {
+            if (!inside(s.r)) return false;
+            for (int k = 0; k < d; ++k)
+                if (s.r.extent[k] != dst.extent[k]) return false;
+        }
+        if ((int)srcs.size() > kMaxSources) return false;
+        dst_regions.push_back(dst);
+
+        // element offsets and strides, all dimensions
+        int64_t dstride[DISTDL_MAX_RANK], doff = 0;
+        strides_of(dst.shard, dstride);
+        for (int k = 0; k < d; ++k) doff += dst.start[k] * dstride[k];
+        std::vector<std::array<int64_t, DISTDL_MAX_RANK>> sstride(srcs.size());
+        std::vector<int64_t> soff(srcs.size(), 0);
+        for (size_t j = 0; j < srcs.size(); ++j) {
+            strides_of(srcs[j].r.shard, sstride[j].data());
+            for (int k = 0; k < d; ++k) soff[j] += srcs[j].r.start[k] * sstride[j][k];
+        }
+        // drop extent-1 dimensions, merge dimensions that are contiguous everywhere
+        std::vector<int> keep;
+        for (int k = 0; k < d; ++k)
+            if (dst.extent[k] != 1) keep.push_back(k);
+        if (keep.empty()) keep.push_back(d - 1);
+        std::vector<int64_t> shape;
+        std::vector<int64_t> ds;
+        std::vector<std::vector<int64_t>> ss(srcs.size());
+        for (int k : keep) {
+            bool merged = false;
+            if (!shape.empty()) {
+                // previous kept dim (outer) merges with this one if outer stride == extent*stride
+                bool ok = ds.back() == dst.extent[k] * dstride[k];
+                for (size_t j = 0; j < srcs.size() && ok; ++j)
+                    ok = ss[j].back() == dst.extent[k] * sstride[j][k];
+                if (ok) {
+                    shape.back() *= dst.extent[k];
+                    ds.back() = dstride[k];
+                    for (size_t j = 0; j < srcs.size(); ++j) ss[j].back() = sstride[j][k];
+                    merged = true;
+                }
+            }
+            if (!merged) {
+                shape.push_back(dst.extent[k]);
+                ds.push_back(dstride[k]);
+                for (size_t j = 0; j < srcs.size(); ++j) ss[j].push_back(sstride[j][k]);
+            }
+        }
+        const int nd = (int)shape.size();
+        // 16-byte vector path: innermost dimension contiguous, everything a multiple of 16 bytes
+        const int64_t per = 16 / esize;
+        bool vec = ds[nd - 1] == 1 && shape[nd - 1] % per == 0 && doff % per == 0;
+        for (int i = 0; i + 1 < nd && vec; ++i) vec = ds[i] % per == 0;
+        for (size_t j = 0; j < srcs.size() && vec; ++j) {
+            vec = ss[j][nd - 1] == 1 && soff[j] % per == 0;
+            for (int i = 0; i + 1 < nd && vec; ++i) vec = ss[j][i] % per == 0;
+        }
+        const int64_t unit = vec ? per : 1;
+
+        HaloBox b;
+        memset(&b, 0, sizeof(b));
+        b.dst_shard = dst.shard;
+        b.ndim = nd;
+        b.nsrc = (int32_t)srcs.size();
+        b.src_begin = (int32_t)plan->sources.size();
+        b.vec = vec ? 1 : 0;
+        b.levels = std::max(levels, 1);
+        b.dst_offset = doff / unit;
+        int64_t units = 1;
+        for (int i = 0; i < nd; ++i) {
+            int64_t e = shape[i];
+            if (i == nd - 1) e /= unit;
+            if (e > INT32_MAX) return false;
+            b.shape[i] = (int32_t)e;
+            b.dst_stride[i] = (i == nd - 1) ? ds[i] : ds[i] / unit;
+            units *= e;
+        }
+        if (units >= (int64_t)UINT32_MAX) return false;
+        for (size_t j = 0; j < srcs.size(); ++j) {
+            HaloSource s;
+            memset(&s, 0, sizeof(s));
+            s.shard = srcs[j].r.shard;
+            s.close = srcs[j].close;
+            s.clear_after = srcs[j].clear_after;
+            s.offset = soff[j] / unit;
+            for (int i = 0; i < nd; ++i) s.stride[i] = (i == nd - 1) ? ss[j][i] : ss[j][i] / unit;
+            plan->sources.push_back(s);
+        }
+        const int32_t box_id = (int32_t)plan->boxes.size();
+        plan->boxes.push_back(b);
+        for (int64_t at = 0; at < units; at += kTileUnits) {
+            HaloTile t;
+            t.box = box_id;
+            t.first = (uint32_t)at;
+            t.count = (uint32_t)std::min<int64_t>(kTileUnits, units - at);
+            plan->tiles.push_back(t);
+        }
+        // algorithmic traffic: destination written once; every source read once; cleared sources
+        // written once; the destination's own previous value is source 0 of a sum (counted there).
+        int64_t bytes = cells * esize;
+        for (const auto &s : srcs) bytes += cells * esize * (1 + (s.clear_after ? 1 : 0));
+        plan->algorithmic_bytes += bytes;
+        return true;
+    }
+
+    bool destinations_disjoint() const {
+        const int d = p->rank;
+        for (size_t a = 0; a < dst_regions.size(); ++a)
+            for (size_t b = a + 1; b < dst_regions.size(); ++b) {
+                const Region &x = dst_regions[a], &y = dst_regions[b];
+                if (x.shard != y.shard) continue;
+                bool overlap = true;
+                for (int k = 0; k < d && overlap; ++k)
+                    overlap = x.start[k] < y.start[k] + y.extent[k] && y.start[k] < x.start[k] + x.extent[k];
+                if (overlap) return false;
+            }
+        return true;
+    }
+};
+
+// Iterates over {-1,0,+1}^d in row-major order of (delta + 1).
+inline bool next_delta(int *delta, int d) {
+    for (int k = d - 1; k >= 0; --k) {
+        if (delta[k] < 1) {
+            ++delta[k];
+            return true;
+        }
+        delta[k] = -1;
+    }
+    return false;
+}
+
+}  // namespace
+
+namespace distdl {
+
+distdl_status_t build_halo_plans(distdl_partition *p) {
+    const int d = p->rank;
+    const int esize = elem_size(p->dtype);
+
+    // ---------------- forward: one box per (shard, direction) ----------------
+    Builder fb{p, &p->fwd_host, {}, esize};
+    // exterior-ghost clear boxes are shared by the adjoint plan
+    Builder ab{p, &p->adj_host, {}, esize};
+    for (int32_t w = 0; w < p->num_workers; ++w) {
+        int32_t c[DISTDL_MAX_RANK];
+        p->coords(w, c);
+        int delta[DISTDL_MAX_RANK];
+        for (int k = 0; k < d; ++k) delta[k] = -1;
+        do {
+            bool centre = true, has_neighbour = true;
+            for (int k = 0; k < d; ++k) {
+                if (delta[k] != 0) centre = false;
+                const int32_t nc = c[k] + delta[k];
+                if (nc < 0 || nc >= p->pshape[k]) has_neighbour = false;
+            }
+            if (centre) continue;
+            Region dst;
+            dst.shard = w;
+            int32_t nc[DISTDL_MAX_RANK];
+            for (int k = 0; k < d; ++k) {
+                const int64_t hl = p->hlo[k][c[k]], b = p->size[k][c[k]], hh = p->hhi[k][c[k]];
+                dst.start[k] = delta[k] < 0 ? 0 : (delta[k] == 0 ? hl : hl + b);
+                dst.extent[k] = delta[k] < 0 ? hl : (delta[k] == 0 ? b : hh);
+                nc[k] = c[k] + delta[k];
+            }
+            std::vector<PendingSource> srcs;
+            if (has_neighbour) {
+                PendingSource s;
+                s.r.shard = p->worker_of(nc);
+                s.close = 0;
+                s.clear_after = 0;
+                for (int k = 0; k < d; ++k) {
+                    const int64_t nhl = p->hlo[k][nc[k]], nb = p->size[k][nc[k]];
+                    s.r.extent[k] = dst.extent[k];
+                    // low ghost <- the last cells of the low neighbour's bulk; high ghost <- the
+                    // first cells of the high neighbour's bulk; otherwise the same bulk range
+                    s.r.start[k] = delta[k] < 0 ? nhl + nb - dst.extent[k] : nhl;
+                }
+                srcs.push_back(s);
+                if (!fb.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: forward box out of range");
+            } else {
+                if (!fb.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
+                if (!ab.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
+            }
+        } while (next_delta(delta, d));
+    }
+    if (!fb.destinations_disjoint()) return fail(DISTDL_ERR_SHAPE, "halo plan: forward boxes overlap");
+
+    // ---------------- adjoint: receiving bulk boxes with their nested sources ----------------
+    for (int32_t w = 0; w < p->num_workers; ++w) {
+        int32_t c[DISTDL_MAX_RANK];
+        p->coords(w, c);
+        // per dimension: up to three segments of the bulk with (from_lo, from_hi) flags
+        struct Seg { int64_t s0, s1; bool from_lo, from_hi; };
+        std::vector<Seg> segs[DISTDL_MAX_RANK];
+        for (int k = 0; k < d; ++k) {
+            const int64_t b = p->size[k][c[k]];
+            const int64_t wl = c[k] > 0 ? p->hhi[k][c[k] - 1] : 0;                  // low neighbour's high ghost
+            const int64_t wh = c[k] + 1 < p->pshape[k] ? p->hlo[k][c[k] + 1] : 0;   // high neighbour's low ghost
+            int64_t cuts[4] = {0, wl, b - wh, b};
+            std::sort(cuts, cuts + 4);
+            for (int i = 0; i < 3; ++i) {
+                if (cuts[i] == cuts[i + 1]) continue;
+                Seg s{cuts[i], cuts[i + 1], cuts[i] < wl, cuts[i] >= b - wh};
+                segs[k].push_back(s);
+            }
+        }
+        std::vector<size_t> pick(d, 0);
+        while (true) {
+            bool any = false;
+            for (int k = 0; k < d; ++k) any = any || segs[k][pick[k]].from_lo || segs[k][pick[k]].from_hi;
+            if (any) {
+                Region dst;
+                dst.shard = w;
+                std::vector<int> options[DISTDL_MAX_RANK];
+                std::vector<int> active;   // dimensions with more than one option, outermost first
+                for (int k = 0; k < d; ++k) {
+                    const Seg &s = segs[k][pick[k]];
+                    dst.start[k] = p->hlo[k][c[k]] + s.s0;
+                    dst.extent[k] = s.s1 - s.s0;
+                    options[k].push_back(0);
+                    if (s.from_lo) options[k].push_back(-1);   // low neighbour first,
+                    if (s.from_hi) options[k].push_back(+1);   // then high
+                    if (options[k].size() > 1) active.push_back(k);
+                }
+                const int levels = (int)active.size();
+                std::vector<PendingSource> srcs;
+                std::vector<size_t> o(d, 0);
+                while (true) {
+                    PendingSource s;
+                    int32_t nc[DISTDL_MAX_RANK];
+                    bool self = true;
+                    for (int k = 0; k < d; ++k) {
+                        nc[k] = c[k] + options[k][o[k]];
+                        if (options[k][o[k]] != 0) self = false;
+                    }
+                    s.r.shard = p->worker_of(nc);
+                    s.clear_after = self ? 0 : 1;
+                    for (int k = 0; k < d; ++k) {
+                        // same global index, expressed in the neighbour's padded-local index
+                        const int64_t g = p->start[k][c[k]] + segs[k][pick[k]].s0;
+                        s.r.start[k] = g - p->start[k][nc[k]] + p->hlo[k][nc[k]];
+                        s.r.extent[k] = dst.extent[k];
+                    }
+                    // levels folded after this term: trailing active dimensions at their last option
+                    int close = 0;
+                    for (int i = levels - 1; i >= 1; --i) {
+                        const int k = active[i];
+                        if (o[k] + 1 == options[k].size()) ++close; else break;
+                    }
+                    s.close = close;
+                    srcs.push_back(s);
+                    int k = d - 1;
+                    for (; k >= 0; --k) {
+                        if (o[k] + 1 < options[k].size()) { ++o[k]; break; }
+                        o[k] = 0;
+                    }
+                    if (k < 0) break;
+                }
+                if ((int)srcs.size() > kMaxSources)
+                    return fail(DISTDL_ERR_UNSUPPORTED, "halo plan: a bulk cell receives from more than %d ghosts", kMaxSources);
+                if (!ab.add(dst, srcs, levels)) return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint box out of range");
+            }
+            int k = d - 1;
+            for (; k >= 0; --k) {
+                if (pick[k] + 1 < segs[k].size()) { ++pick[k]; break; }
+                pick[k] = 0;
+            }
+            if (k < 0) break;
+        }
+    }
+    if (!ab.destinations_disjoint()) return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint boxes overlap");
+    return DISTDL_OK;
+}
+
+}  // namespace distdl

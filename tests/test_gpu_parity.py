@@ -1,0 +1,270 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Copies (B, H) and fixed-order sums (R, H*) must be bit-exact; the convolution is
+compared within a bound derived from its 25-term fp32 accumulation."""
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2006_03108_b200 as distdl
+from paper_2006_03108_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def host(t):
+    return t.detach().cpu().numpy()
+
+
+def same_bits(a, b):
+    a, b = np.ascontiguousarray(a), np.ascontiguousarray(b)
+    return a.shape == b.shape and a.tobytes() == b.tobytes()
+
+
+def make_partitions(case):
+    gshape, pshape, hlo, hhi = case
+    return oracle.Partition(gshape, pshape, hlo, hhi), distdl.Partition(gshape, pshape, _w(hlo, len(gshape)), _w(hhi, len(gshape)))
+
+
+def _w(h, rank):
+    return [h] * rank if isinstance(h, int) else list(h)
+
+
+def random_shards(opart, seed, kind="uniform"):
+    gen = inputs.uniform_pm1 if kind == "uniform" else inputs.integers
+    return [gen(opart.padded_shape(w), seed * 1000 + w) for w in range(opart.num_workers)]
+
+
+# --------------------------------------------------------------------------
+# Broadcast / sum-reduce
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1000, 4099, 1 << 20, (1 << 22) + 5])
+@pytest.mark.parametrize("k", [1, 2, 3, 8, 19])
+def test_broadcast_bit_exact(n, k):
+    x = inputs.uniform_pm1((n,), n + k)
+    src = dev(x)
+    dsts = [torch.full((n + 8,), 7.0, device=DEV)[:n] for _ in range(k)]
+    distdl.broadcast_fwd(src, dsts)
+    torch.cuda.synchronize()
+    ref = oracle.broadcast_fwd(x, k)
+    for d, r in zip(dsts, ref):
+        assert same_bits(host(d), r)
+
+
+def test_broadcast_bf16_and_in_place():
+    x = inputs.f32_to_bf16_bits(inputs.normal((12345,), 3))
+    src = dev(x.view(np.int16)).view(torch.bfloat16)
+    dsts = [src] + [torch.zeros_like(src) for _ in range(3)]
+    distdl.broadcast_fwd(src, dsts)
+    torch.cuda.synchronize()
+    for d in dsts:
+        assert same_bits(host(d.view(torch.int16)).view(np.uint16), x)
+
+
+@pytest.mark.parametrize("n", [1, 5, 1000, 4099, (1 << 21) + 3])
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 8, 16, 17, 35])
+def test_sumreduce_bit_exact(n, k):
+    parts = [inputs.uniform_pm1((n,), 100 * k + i) * np.float32(10.0 ** (i % 5)) for i in range(k)]
+    srcs = [dev(p) for p in parts]
+    dst = torch.empty(n, device=DEV)
+    distdl.sumreduce_fwd(srcs, dst)
+    torch.cuda.synchronize()
+    assert same_bits(host(dst), oracle.sumreduce_fwd(parts))
+    # adjoint names are the same operators
+    dst2 = torch.empty(n, device=DEV)
+    distdl.broadcast_adj(srcs, dst2)
+    torch.cuda.synchronize()
+    assert same_bits(host(dst2), host(dst))
+
+
+def test_sumreduce_signed_zero_and_in_place():
+    a = np.array([-0.0, 1e8, 1.0, -0.0, 5.0], dtype=np.float32)
+    b = np.array([-0.0, -1e8, 1e8, 0.0, 5.0], dtype=np.float32)
+    c = np.array([-0.0, 1.0, -1e8, -0.0, 5.0], dtype=np.float32)
+    srcs = [dev(a), dev(b), dev(c)]
+    distdl.sumreduce_fwd(srcs, srcs[0])          # dst aliases source 0
+    torch.cuda.synchronize()
+    assert same_bits(host(srcs[0]), oracle.sumreduce_fwd([a, b, c]))
+    one = dev(a)
+    out = torch.empty_like(one)
+    distdl.sumreduce_fwd([one], out)             # k = 1 keeps -0.0
+    torch.cuda.synchronize()
+    assert same_bits(host(out), a)
+
+
+def test_reduce_after_broadcast_and_dot_test():
+    k, n = 8, 100003
+    x = inputs.uniform_pm1((n,), 7)
+    ys = [inputs.uniform_pm1((n,), 70 + i) for i in range(k)]
+    copies = [torch.empty(n, device=DEV) for _ in range(k)]
+    distdl.broadcast_fwd(dev(x), copies)
+    back = torch.empty(n, device=DEV)
+    distdl.sumreduce_fwd(copies, back)
+    bsy = torch.empty(n, device=DEV)
+    distdl.broadcast_adj([dev(y) for y in ys], bsy)
+    torch.cuda.synchronize()
+    assert same_bits(host(back), oracle.sumreduce_fwd(oracle.broadcast_fwd(x, k)))
+    assert np.allclose(host(back), 8 * x, rtol=1e-6, atol=0)
+    r = oracle.adjoint_test_ratio([host(c) for c in copies], ys, [x], [host(bsy)])
+    assert r < 1e-5
+
+
+# --------------------------------------------------------------------------
+# Halo exchange
+# --------------------------------------------------------------------------
+
+HALO_CASES = [
+    ((11,), (3,), 2, 2),
+    ((7,), (1,), 1, 2),
+    ((10,), (4,), [[0, 1, 2, 1]], [[1, 0, 2, 0]]),
+    ((6, 6), (2, 2), 1, 1),
+    ((7, 5), (3, 2), (1, 2), (2, 1)),
+    ((9, 8), (2, 2), [[0, 4], [3, 0]], [[2, 0], [0, 3]]),
+    ((9, 8), (2, 2), [[0, 4], [0, 3]], [[2, 0], [0, 0]]),      # Appendix B.2 widths
+    ((5, 6, 7), (2, 1, 3), (1, 2, 1), (1, 0, 2)),
+    ((4, 4, 4), (2, 2, 2), 1, 1),
+    ((6, 4), (3, 1), 2, 2),                                   # thin: a cell receives from both sides
+    ((3, 3, 3), (3, 3, 3), 1, 1),                             # 27 sources per cell
+    ((3, 3, 2, 4), (1, 1, 2, 2), (0, 0, 1, 1), (0, 0, 1, 1)),
+    ((4, 5, 6, 4, 6), (2, 1, 2, 1, 2), (1, 0, 1, 1, 2), (0, 1, 1, 0, 1)),
+    ((256, 256), (2, 2), 1, 1),                               # the small 2-D configuration
+    ((70, 66, 72), (2, 2, 2), 4, 4),                          # 16-byte paths, several tiles
+    ((67, 61, 68), (3, 2, 2), (2, 4, 4), (3, 4, 4)),          # uneven split, mixed alignment
+    ((2, 3, 40, 44), (1, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2)),
+]
+
+
+@pytest.mark.parametrize("case", HALO_CASES, ids=[str(c[0]) + str(c[1]) for c in HALO_CASES])
+def test_halo_fwd_and_adj_bit_exact(case):
+    opart, gpart = make_partitions(case)
+    for w in range(opart.num_workers):
+        assert gpart.padded_shape(w) == opart.padded_shape(w)
+    x = random_shards(opart, 11)                         # ghosts hold garbage on entry
+    xs = [dev(a) for a in x]
+    distdl.halo_fwd(gpart, xs)
+    torch.cuda.synchronize()
+    ref = oracle.halo_fwd_sequence(opart, x)
+    for w in range(opart.num_workers):
+        assert same_bits(host(xs[w]), ref[w]), "H differs on worker %d" % w
+    y = random_shards(opart, 12)
+    ys = [dev(a) for a in y]
+    distdl.halo_adj(gpart, ys)
+    torch.cuda.synchronize()
+    refa = oracle.halo_adj_sequence(opart, y)
+    for w in range(opart.num_workers):
+        assert same_bits(host(ys[w]), refa[w]), "H* differs on worker %d" % w
+    # the adjoint (dot-product) test on the GPU results, fp64 inner products over every cell
+    r = oracle.adjoint_test_ratio([host(t) for t in xs], y, x, [host(t) for t in ys])
+    assert r < 1e-5
+
+
+def test_halo_adj_order_sensitive_values():
+    """Values of very different magnitude: any other summation order changes the bits."""
+    case = ((12, 12, 12), (2, 2, 2), 2, 2)
+    opart, gpart = make_partitions(case)
+    y = []
+    for w in range(opart.num_workers):
+        a = inputs.uniform_pm1(opart.padded_shape(w), 900 + w)
+        scale = np.float32(10.0) ** inputs.integers(opart.padded_shape(w), 950 + w, -6, 7)
+        y.append((a * scale).astype(np.float32))
+    ys = [dev(a) for a in y]
+    distdl.halo_adj(gpart, ys)
+    torch.cuda.synchronize()
+    ref = oracle.halo_adj_sequence(opart, y)
+    for w in range(opart.num_workers):
+        assert same_bits(host(ys[w]), ref[w])
+
+
+def test_halo_bf16_copies():
+    case = ((20, 24), (2, 2), 2, 2)
+    opart = oracle.Partition(*case)
+    gpart = distdl.Partition(case[0], case[1], [2, 2], [2, 2], dtype=distdl.BF16)
+    x = [inputs.f32_to_bf16_bits(a) for a in random_shards(opart, 13)]
+    xs = [dev(a.view(np.int16)).view(torch.bfloat16) for a in x]
+    distdl.halo_fwd(gpart, xs)
+    torch.cuda.synchronize()
+    ref = oracle.halo_fwd_definition(opart, x)            # copies of bit patterns
+    for w in range(opart.num_workers):
+        assert same_bits(host(xs[w].view(torch.int16)).view(np.uint16), ref[w])
+
+
+# --------------------------------------------------------------------------
+# Convolution layer
+# --------------------------------------------------------------------------
+
+CONV_CASES = [
+    # global NCHW, partition, kernel
+    ((1, 2, 12, 13), (1, 1, 1, 1), 5),
+    ((2, 3, 12, 13), (1, 1, 2, 2), 5),
+    ((1, 2, 17, 19), (1, 1, 3, 2), 3),
+    ((1, 2, 23, 29), (1, 1, 2, 3), 7),
+    ((2, 2, 150, 300), (1, 1, 2, 2), 5),     # partial tiles in both directions
+    ((1, 3, 140, 264), (1, 1, 2, 2), 5),     # 16-byte aligned rows
+    ((1, 2, 130, 520), (1, 1, 1, 2), 3),
+    ((1, 1, 64, 1040), (1, 1, 1, 4), 7),
+]
+
+
+def _abs_bound(opart, x, w):
+    """sum |w||x| per output: the scale of the rounding error of the K*K-term fp32 accumulation,
+    |fl(sum) - exact| <= K*K * 2^-24 * sum |w||x| to first order."""
+    return oracle.conv_fwd(opart, [np.abs(a) for a in x], np.abs(w))
+
+
+@pytest.mark.parametrize("case", CONV_CASES, ids=[str(c) for c in CONV_CASES])
+def test_conv_fwd_and_adj(case):
+    gshape, pshape, k = case
+    h = k // 2
+    hl = (0, 0, h, h)
+    opart = oracle.Partition(gshape, pshape, hl, hl)
+    obulk = oracle.Partition(gshape, pshape, 0, 0)
+    gpart = distdl.Partition(gshape, pshape, hl, hl)
+    xg = inputs.normal(gshape, 31)
+    w = inputs.normal((gshape[1], k, k), 32, 0.1)
+    bias = inputs.normal((gshape[1],), 33)
+    x = oracle.scatter_global(opart, xg, fill=lambda wk: np.full(opart.padded_shape(wk), 1e30, dtype=np.float32))
+    xs = [dev(a) for a in x]
+    ys = [torch.full(obulk.padded_shape(wk), -7.0, device=DEV) for wk in range(opart.num_workers)]
+    distdl.conv_fwd(gpart, xs, dev(w), dev(bias), ys)
+    torch.cuda.synchronize()
+    ref = oracle.conv_fwd(opart, x, w, bias)
+    bound = _abs_bound(opart, x, w)
+    eps = (k * k + 1) * 2.0 ** -24
+    for wk in range(opart.num_workers):
+        got = host(ys[wk])
+        assert np.all(np.abs(got.astype(np.float64) - ref[wk]) <= eps * (bound[wk] + np.abs(bias)[None, :, None, None]) + 1e-30)
+        assert same_bits(host(xs[wk]), x[wk])            # x, ghosts included, is left untouched
+    num = np.sqrt(sum(float(np.sum((host(a).astype(np.float64) - b) ** 2)) for a, b in zip(ys, ref)))
+    den = np.sqrt(sum(float(np.sum(b.astype(np.float64) ** 2)) for b in ref))
+    assert num / den < 1e-6
+
+    # adjoint
+    dyg = inputs.normal(gshape, 34)
+    dy = oracle.scatter_global(obulk, dyg)
+    dys = [dev(a) for a in dy]
+    dxs = [torch.full(opart.padded_shape(wk), 3.0, device=DEV) for wk in range(opart.num_workers)]
+    distdl.conv_adj(gpart, dys, dev(w), dxs)
+    torch.cuda.synchronize()
+    refa = oracle.conv_adj(opart, dy, w)
+    bounda = oracle.conv_adj(opart, [np.abs(a) for a in dy], np.abs(w))
+    for wk in range(opart.num_workers):
+        got = host(dxs[wk])
+        assert np.all(np.abs(got.astype(np.float64) - refa[wk]) <= k * k * 2.0 ** -24 * bounda[wk] + 1e-30)
+        mask = np.ones(opart.padded_shape(wk), dtype=bool)
+        mask[opart.bulk_slices(wk)] = False
+        assert not got[mask].any()                       # ghosts of dx are zero, as H* leaves them
+    # dot-product test of the fused pair (bias is not part of the linear operator)
+    y0 = [torch.empty_like(t) for t in ys]
+    distdl.conv_fwd(gpart, xs, dev(w), None, y0)
+    torch.cuda.synchronize()
+    xb = oracle.scatter_global(opart, xg)                # zero ghosts: the inner product is over the bulk
+    r = oracle.adjoint_test_ratio([host(t) for t in y0], dy, xb, [host(t) for t in dxs])
+    assert r < 1e-5
