@@ -39,33 +39,42 @@ constexpr int kMaxBoxDims = DISTDL_MAX_RANK;
 constexpr int kMaxLevels = DISTDL_MAX_RANK;   // nesting depth of the H* sum
 constexpr int kMaxSources = 32;               // sources of one box (2^5, or 3^3 for thin shards)
 
+// Offsets and strides are in *units* (16-byte vectors when `vec`, elements otherwise) and fit in
+// 32 bits (a shard holds fewer than 2^31 elements).
 struct HaloSource {
     int32_t shard;                 // shard the source cells live in
     int32_t close;                 // how many nesting levels are folded after adding this source
     int32_t clear_after;           // 1: source cells are set to zero once read (ghost sources)
-    int32_t pad_;
-    int64_t offset;                // element offset of the box origin inside the shard
-    int64_t stride[kMaxBoxDims];   // element stride per box dimension (innermost last)
+    uint32_t offset;               // unit offset of the box origin inside the shard
+    uint32_t stride[kMaxBoxDims];  // unit stride per box dimension (innermost last)
+    uint32_t pad_[3];
 };
+static_assert(sizeof(HaloSource) == 48, "HaloSource layout");
 
 struct HaloBox {
     int32_t dst_shard;
     int32_t ndim;                  // box dimensions kept after dropping extent-1 dimensions
-    int32_t nsrc;
-    int32_t src_begin;             // index of the first source in the source table
     int32_t vec;                   // 1: every offset, stride and extent allows 16-byte accesses
     int32_t levels;                // nesting levels of the sum (>= 1)
-    int32_t shape[kMaxBoxDims];    // extents; innermost in units of `vec ? 16 bytes : elements`
-    int32_t pad_;
-    int64_t dst_offset;
-    int64_t dst_stride[kMaxBoxDims];
+    int32_t balanced;              // 1: every nesting level has exactly two terms (nsrc = 2^levels)
+    uint32_t dst_offset;
+    uint32_t shape[kMaxBoxDims];   // extents in units
+    uint32_t magic[kMaxBoxDims];   // n / shape[k] == umulhi(n, magic[k]) >> shift[k] for n < 2^31
+    uint32_t shift[kMaxBoxDims];
+    uint32_t dst_stride[kMaxBoxDims];
+    uint32_t pad_[6];
 };
+static_assert(sizeof(HaloBox) == 128, "HaloBox layout");
 
 struct HaloTile {
     int32_t box;
+    int32_t src_begin;             // index of the box's first source in the source table
+    int32_t nsrc;                  // 0: clear, 1: copy, more: nested sum
     uint32_t first;                // first flattened unit of the tile
     uint32_t count;                // units in the tile
+    uint32_t pad_[3];
 };
+static_assert(sizeof(HaloTile) == 32, "HaloTile layout");
 
 struct HaloPlanHost {
     std::vector<HaloBox> boxes;

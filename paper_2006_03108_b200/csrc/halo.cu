@@ -1,5 +1,5 @@
-// Halo exchange H and adjoint halo exchange H* (Section 3, "Halo exchange") as one gather
-// kernel over a host-planned list of boxes.
+// Halo exchange H and adjoint halo exchange H* (Section 3, "Halo exchange") as gather kernels
+// over a host-planned list of boxes.
 //
 // The paper runs the exchange as d nested pack / exchange / unpack phases so that corner data
 // reaches its destination in d hops between distributed memories.  Here every shard sits in the
@@ -18,10 +18,10 @@ struct ShardPointers {
 
 constexpr int kHaloThreads = 256;
 
-__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+__device__ __forceinline__ float4 vadd(float4 a, float4 b) {
     return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
 }
-__device__ __forceinline__ float add4(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ float vadd(float a, float b) { return __fadd_rn(a, b); }
 
 template <typename T> __device__ __forceinline__ T zero_of();
 template <> __device__ __forceinline__ float4 zero_of<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
@@ -29,72 +29,151 @@ template <> __device__ __forceinline__ float zero_of<float>() { return 0.f; }
 template <> __device__ __forceinline__ uint4 zero_of<uint4>() { return make_uint4(0, 0, 0, 0); }
 template <> __device__ __forceinline__ unsigned short zero_of<unsigned short>() { return 0; }
 
-// Copy / clear of one tile with element type T (uint4 = 16 bytes, float, or unsigned short).
-template <typename T>
-__device__ __forceinline__ void run_copy_tile(const HaloBox &box, const HaloSource *src, const ShardPointers &sh,
-                                              uint32_t first, uint32_t count) {
-    T *dst = reinterpret_cast<T *>(sh.p[box.dst_shard]) + box.dst_offset;
-    const T *s0 = box.nsrc ? reinterpret_cast<const T *>(sh.p[src[0].shard]) + src[0].offset : nullptr;
-    const int nd = box.ndim;
-    for (uint32_t i = threadIdx.x; i < count; i += kHaloThreads) {
-        uint32_t rem = first + i;
-        int64_t doff = 0, soff = 0;
-        for (int k = nd - 1; k >= 0; --k) {
-            const uint32_t e = (uint32_t)box.shape[k];
-            const uint32_t q = rem / e, c = rem - q * e;
-            rem = q;
-            doff += (int64_t)c * box.dst_stride[k];
-            if (s0) soff += (int64_t)c * src[0].stride[k];
+// Coordinates of flattened unit n inside the box (innermost dimension last).
+__device__ __forceinline__ void decompose(const HaloBox &box, uint32_t n, uint32_t *coord) {
+#pragma unroll
+    for (int k = kMaxBoxDims - 1; k >= 1; --k) {
+        coord[k] = 0;
+        if (k < box.ndim) {
+            const uint32_t q = __umulhi(n, box.magic[k]) >> box.shift[k];
+            coord[k] = n - q * box.shape[k];
+            n = q;
         }
-        dst[doff] = s0 ? s0[soff] : zero_of<T>();
+    }
+    coord[0] = n;
+}
+
+__device__ __forceinline__ uint32_t dot_stride(const uint32_t *coord, const uint32_t *stride, int nd) {
+    uint32_t o = 0;
+#pragma unroll
+    for (int k = 0; k < kMaxBoxDims; ++k)
+        if (k < nd) o += coord[k] * stride[k];
+    return o;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Copy / clear tile (H, and the ghost clears of H*): T = uint4 (16 bytes), float, unsigned short.
+// Each thread keeps kCopyBatch independent loads in flight.
+// ---------------------------------------------------------------------------------------------
+constexpr int kCopyBatch = 4;
+
+template <typename T>
+__device__ __forceinline__ void run_copy_tile(const HaloBox &box, const HaloSource *src, int nsrc,
+                                              const ShardPointers &sh, uint32_t first, uint32_t count) {
+    T *dst = reinterpret_cast<T *>(sh.p[box.dst_shard]) + box.dst_offset;
+    const int nd = box.ndim;
+    if (nsrc == 0) {
+        for (uint32_t i = threadIdx.x; i < count; i += kHaloThreads) {
+            uint32_t c[kMaxBoxDims];
+            decompose(box, first + i, c);
+            dst[dot_stride(c, box.dst_stride, nd)] = zero_of<T>();
+        }
+        return;
+    }
+    const T *s0 = reinterpret_cast<const T *>(sh.p[src[0].shard]) + src[0].offset;
+    for (uint32_t base = threadIdx.x; base < count; base += kHaloThreads * kCopyBatch) {
+        T v[kCopyBatch];
+        uint32_t doff[kCopyBatch];
+#pragma unroll
+        for (int u = 0; u < kCopyBatch; ++u) {
+            const uint32_t i = base + u * kHaloThreads;
+            if (i < count) {
+                uint32_t c[kMaxBoxDims];
+                decompose(box, first + i, c);
+                doff[u] = dot_stride(c, box.dst_stride, nd);
+                v[u] = s0[dot_stride(c, src[0].stride, nd)];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kCopyBatch; ++u)
+            if (base + u * kHaloThreads < count) dst[doff[u]] = v[u];
     }
 }
 
-// Nested sum of one tile (H*): T is float4 or float.
-template <typename T>
-__device__ __forceinline__ void run_sum_tile(const HaloBox &box, const HaloSource *src, const ShardPointers &sh,
-                                             uint32_t first, uint32_t count) {
-    T *dst = reinterpret_cast<T *>(sh.p[box.dst_shard]) + box.dst_offset;
+// ---------------------------------------------------------------------------------------------
+// Nested sum of H*.  Balanced case (every level has two terms, NSRC = 2^levels): all loads are
+// issued first, then the ghost clears, then a fixed binary tree in source order -- which is the
+// left-to-right nested fold when each level has exactly two terms.
+// ---------------------------------------------------------------------------------------------
+// Orders the stores that follow after the arrival of `v`: a store issued to a line whose load is
+// still in flight stalls the memory pipeline badly (measured: 4x lower throughput), so every
+// store of a batch waits until the batch's sums -- and with them all of its loads -- are done.
+__device__ __forceinline__ void stores_after(const float4 &v) {
+    asm volatile("" ::"f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void stores_after(const float &v) { asm volatile("" ::"f"(v) : "memory"); }
+
+template <typename T, int NSRC>
+__device__ __forceinline__ void run_sum_tile_balanced(const HaloBox &box, const HaloSource *src,
+                                                      const ShardPointers &sh, uint32_t first, uint32_t count) {
+    constexpr int U = NSRC >= 8 ? 1 : (NSRC == 4 ? 2 : 4);   // units per thread per batch
     const int nd = box.ndim;
-    const int nsrc = box.nsrc;
-    const int top = box.levels - 1;
-    for (uint32_t i = threadIdx.x; i < count; i += kHaloThreads) {
-        uint32_t rem = first + i;
-        uint32_t coord[kMaxBoxDims];
+    T *base[NSRC];
 #pragma unroll
-        for (int k = kMaxBoxDims - 1; k >= 0; --k) {
-            coord[k] = 0;
-            if (k < nd) {
-                const uint32_t e = (uint32_t)box.shape[k];
-                const uint32_t q = rem / e;
-                coord[k] = rem - q * e;
-                rem = q;
+    for (int j = 0; j < NSRC; ++j) base[j] = reinterpret_cast<T *>(sh.p[src[j].shard]) + src[j].offset;
+    for (uint32_t b0 = threadIdx.x; b0 < count; b0 += kHaloThreads * U) {
+        T *ptr[U][NSRC];
+        T v[U][NSRC];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = b0 + u * kHaloThreads;
+            if (i < count) {
+                uint32_t c[kMaxBoxDims];
+                decompose(box, first + i, c);
+#pragma unroll
+                for (int j = 0; j < NSRC; ++j) {
+                    ptr[u][j] = base[j] + dot_stride(c, src[j].stride, nd);
+                    v[u][j] = *ptr[u][j];
+                }
             }
         }
-        int64_t doff = 0;
+        // fixed binary tree in source order
 #pragma unroll
-        for (int k = 0; k < kMaxBoxDims; ++k)
-            if (k < nd) doff += (int64_t)coord[k] * box.dst_stride[k];
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int width = 1; width < NSRC; width *= 2)
+#pragma unroll
+                for (int j = 0; j < NSRC; j += 2 * width) v[u][j] = vadd(v[u][j], v[u][j + width]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) stores_after(v[u][0]);
+        // source 0 is the receiving bulk cell itself; every other source is a ghost cell
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (b0 + u * kHaloThreads < count) {
+                *ptr[u][0] = v[u][0];
+#pragma unroll
+                for (int j = 1; j < NSRC; ++j) *ptr[u][j] = zero_of<T>();
+            }
+        }
+    }
+}
 
+// General case (a level with three terms, i.e. a shard thinner than its two neighbours' ghosts).
+template <typename T>
+__device__ __forceinline__ void run_sum_tile_general(const HaloBox &box, const HaloSource *src, int nsrc,
+                                                     const ShardPointers &sh, uint32_t first, uint32_t count) {
+    T *dst = reinterpret_cast<T *>(sh.p[box.dst_shard]) + box.dst_offset;
+    const int nd = box.ndim;
+    const int top = box.levels - 1;
+    for (uint32_t i = threadIdx.x; i < count; i += kHaloThreads) {
+        uint32_t c[kMaxBoxDims];
+        decompose(box, first + i, c);
         T acc[kMaxLevels];
+#pragma unroll
+        for (int l = 0; l < kMaxLevels; ++l) acc[l] = zero_of<T>();
         unsigned has = 0;
+#pragma unroll 4
         for (int j = 0; j < nsrc; ++j) {
             const HaloSource &s = src[j];
-            int64_t soff = s.offset;
-#pragma unroll
-            for (int k = 0; k < kMaxBoxDims; ++k)
-                if (k < nd) soff += (int64_t)coord[k] * s.stride[k];
-            T *sp = reinterpret_cast<T *>(sh.p[s.shard]) + soff;
-            const T v = *sp;
-            if (s.clear_after) *sp = zero_of<T>();
+            const T v = *(reinterpret_cast<const T *>(sh.p[s.shard]) + s.offset + dot_stride(c, s.stride, nd));
             // absent terms are skipped, never added as zero
-            acc[0] = (has & 1u) ? add4(acc[0], v) : v;
+            acc[0] = (has & 1u) ? vadd(acc[0], v) : v;
             has |= 1u;
             const int close = s.close;
 #pragma unroll
             for (int l = 0; l < kMaxLevels - 1; ++l) {
                 if (l < close) {
-                    acc[l + 1] = ((has >> (l + 1)) & 1u) ? add4(acc[l + 1], acc[l]) : acc[l];
+                    acc[l + 1] = ((has >> (l + 1)) & 1u) ? vadd(acc[l + 1], acc[l]) : acc[l];
                     has |= 2u << l;
                     has &= ~(1u << l);
                 }
@@ -104,45 +183,57 @@ __device__ __forceinline__ void run_sum_tile(const HaloBox &box, const HaloSourc
 #pragma unroll
         for (int l = 1; l < kMaxLevels; ++l)
             if (l == top) res = acc[l];
-        dst[doff] = res;
+        stores_after(res);
+        dst[dot_stride(c, box.dst_stride, nd)] = res;
+        for (int j = 0; j < nsrc; ++j) {
+            const HaloSource &s = src[j];
+            if (s.clear_after)
+                *(reinterpret_cast<T *>(sh.p[s.shard]) + s.offset + dot_stride(c, s.stride, nd)) = zero_of<T>();
+        }
     }
 }
 
-__global__ void __launch_bounds__(kHaloThreads)
+template <typename T>
+__device__ __forceinline__ void run_sum_tile(const HaloBox &box, const HaloSource *src, int nsrc,
+                                             const ShardPointers &sh, uint32_t first, uint32_t count) {
+    if (box.balanced && nsrc == 2) run_sum_tile_balanced<T, 2>(box, src, sh, first, count);
+    else if (box.balanced && nsrc == 4) run_sum_tile_balanced<T, 4>(box, src, sh, first, count);
+    else if (box.balanced && nsrc == 8) run_sum_tile_balanced<T, 8>(box, src, sh, first, count);
+    else run_sum_tile_general<T>(box, src, nsrc, sh, first, count);
+}
+
+// One thread block per tile.  SUMS = false: the forward plan (copies and clears only).
+template <bool SUMS>
+__global__ void __launch_bounds__(kHaloThreads, SUMS ? 2 : 4)
 halo_box_kernel(const HaloBox *__restrict__ boxes, const HaloSource *__restrict__ sources,
-                const HaloTile *__restrict__ tiles, int32_t num_tiles, int32_t elem_bytes,
+                const HaloTile *__restrict__ tiles, int32_t elem_bytes,
                 const __grid_constant__ ShardPointers sh) {
-    __shared__ HaloBox s_box;
-    __shared__ HaloSource s_src[kMaxSources];
-    __shared__ HaloTile s_tile;
-    for (int32_t t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-        __syncthreads();
-        if (threadIdx.x == 0) s_tile = tiles[t];
-        __syncthreads();
-        const HaloBox *gb = boxes + s_tile.box;
-        // cooperative copy of the descriptors (4-byte words)
-        {
-            const uint32_t *g = reinterpret_cast<const uint32_t *>(gb);
-            uint32_t *s = reinterpret_cast<uint32_t *>(&s_box);
-            for (uint32_t i = threadIdx.x; i < sizeof(HaloBox) / 4; i += kHaloThreads) s[i] = g[i];
+    __shared__ __align__(16) HaloBox s_box;
+    __shared__ __align__(16) HaloSource s_src[kMaxSources];
+    // every thread reads the (uniform) tile record; box and sources are staged in shared memory
+    const uint4 t0 = __ldg(reinterpret_cast<const uint4 *>(tiles + blockIdx.x));
+    const uint32_t count = __ldg(&tiles[blockIdx.x].count);
+    const int box_id = (int)t0.x, src_begin = (int)t0.y, nsrc = (int)t0.z;
+    const uint32_t first = t0.w;
+    {
+        const uint32_t *g = reinterpret_cast<const uint32_t *>(boxes + box_id);
+        uint32_t *s = reinterpret_cast<uint32_t *>(&s_box);
+        const uint32_t bw = sizeof(HaloBox) / 4, sw = (uint32_t)nsrc * (sizeof(HaloSource) / 4);
+        const uint32_t *gs = reinterpret_cast<const uint32_t *>(sources + src_begin);
+        uint32_t *ss = reinterpret_cast<uint32_t *>(s_src);
+        for (uint32_t i = threadIdx.x; i < bw + sw; i += kHaloThreads) {
+            if (i < bw) s[i] = __ldg(g + i);
+            else ss[i - bw] = __ldg(gs + (i - bw));
         }
-        __syncthreads();
-        {
-            const uint32_t *g = reinterpret_cast<const uint32_t *>(sources + s_box.src_begin);
-            uint32_t *s = reinterpret_cast<uint32_t *>(s_src);
-            const uint32_t words = (uint32_t)s_box.nsrc * (sizeof(HaloSource) / 4);
-            for (uint32_t i = threadIdx.x; i < words; i += kHaloThreads) s[i] = g[i];
-        }
-        __syncthreads();
-        const uint32_t first = s_tile.first, count = s_tile.count;
-        if (s_box.nsrc <= 1) {
-            if (s_box.vec) run_copy_tile<uint4>(s_box, s_src, sh, first, count);
-            else if (elem_bytes == 4) run_copy_tile<float>(s_box, s_src, sh, first, count);
-            else run_copy_tile<unsigned short>(s_box, s_src, sh, first, count);
-        } else {
-            if (s_box.vec) run_sum_tile<float4>(s_box, s_src, sh, first, count);
-            else run_sum_tile<float>(s_box, s_src, sh, first, count);
-        }
+    }
+    __syncthreads();
+    if (!SUMS || nsrc <= 1) {
+        if (s_box.vec) run_copy_tile<uint4>(s_box, s_src, nsrc, sh, first, count);
+        else if (elem_bytes == 4) run_copy_tile<float>(s_box, s_src, nsrc, sh, first, count);
+        else run_copy_tile<unsigned short>(s_box, s_src, nsrc, sh, first, count);
+    } else {
+        if (s_box.vec) run_sum_tile<float4>(s_box, s_src, nsrc, sh, first, count);
+        else run_sum_tile<float>(s_box, s_src, nsrc, sh, first, count);
     }
 }
 
@@ -170,8 +261,12 @@ static distdl_status_t launch(const distdl_partition *p, const HaloPlanDevice &p
     }
     for (int32_t w = p->num_workers; w < DISTDL_MAX_WORKERS; ++w) sh.p[w] = nullptr;
     if (plan.num_tiles == 0) return DISTDL_OK;
-    halo_box_kernel<<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(
-        plan.boxes, plan.sources, plan.tiles, plan.num_tiles, elem_size(p->dtype), sh);
+    if (adjoint)
+        halo_box_kernel<true><<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(
+            plan.boxes, plan.sources, plan.tiles, elem_size(p->dtype), sh);
+    else
+        halo_box_kernel<false><<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(
+            plan.boxes, plan.sources, plan.tiles, elem_size(p->dtype), sh);
     DISTDL_CUDA_CHECK(cudaGetLastError());
     return DISTDL_OK;
 }

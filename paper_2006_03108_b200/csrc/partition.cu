@@ -63,7 +63,7 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
         }
     }
     for (int32_t w = 0; w < p->num_workers; ++w)
-        if (p->shard_elems(w) >= (int64_t)1 << 40) {
+        if (p->shard_elems(w) >= (int64_t)1 << 31) {
             delete p;
             return fail(DISTDL_ERR_UNSUPPORTED, "partition_create: shard too large");
         }

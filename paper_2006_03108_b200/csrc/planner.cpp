@@ -94,7 +94,7 @@ struct PendingSource {
     int32_t clear_after;
 };
 
-constexpr uint32_t kTileUnits = 2048;
+constexpr uint32_t kTileUnits = 4096;
 
 struct Builder {
     const distdl_partition *p;
@@ -183,41 +183,73 @@ struct Builder {
             for (int i = 0; i + 1 < nd && vec; ++i) vec = ss[j][i] % per == 0;
         }
         const int64_t unit = vec ? per : 1;
+        // to units; a dimension whose extent becomes one unit carries no coordinate and is dropped
+        {
+            shape[nd - 1] /= unit;
+            for (int i = 0; i + 1 < nd; ++i) {
+                ds[i] /= unit;
+                for (size_t j = 0; j < srcs.size(); ++j) ss[j][i] /= unit;
+            }
+            doff /= unit;
+            for (size_t j = 0; j < srcs.size(); ++j) soff[j] /= unit;
+            int o = 0;
+            for (int i = 0; i < nd; ++i) {
+                if (shape[i] == 1 && !(o == 0 && i == nd - 1)) continue;
+                shape[o] = shape[i];
+                ds[o] = ds[i];
+                for (size_t j = 0; j < srcs.size(); ++j) ss[j][o] = ss[j][i];
+                ++o;
+            }
+            shape.resize(o);
+        }
+        const int nd_units = (int)shape.size();
 
         HaloBox b;
         memset(&b, 0, sizeof(b));
         b.dst_shard = dst.shard;
-        b.ndim = nd;
-        b.nsrc = (int32_t)srcs.size();
-        b.src_begin = (int32_t)plan->sources.size();
         b.vec = vec ? 1 : 0;
         b.levels = std::max(levels, 1);
-        b.dst_offset = doff / unit;
+        b.balanced = ((int64_t)srcs.size() == ((int64_t)1 << b.levels)) ? 1 : 0;
+        b.ndim = nd_units;
+        b.dst_offset = (uint32_t)doff;
         int64_t units = 1;
-        for (int i = 0; i < nd; ++i) {
-            int64_t e = shape[i];
-            if (i == nd - 1) e /= unit;
-            if (e > INT32_MAX) return false;
-            b.shape[i] = (int32_t)e;
-            b.dst_stride[i] = (i == nd - 1) ? ds[i] : ds[i] / unit;
+        for (int i = 0; i < nd_units; ++i) {
+            const int64_t e = shape[i];
+            if (e >= ((int64_t)1 << 31)) return false;
+            b.shape[i] = (uint32_t)e;
+            b.dst_stride[i] = (uint32_t)ds[i];
+            // exact division of any n < 2^31 by e >= 2: q = (n * magic) >> (31 + s) with
+            // s = ceil(log2 e), magic = ceil(2^(31+s) / e) < 2^32; evaluated as
+            // umulhi(n, magic) >> (s - 1).  (e = 1 only for a one-unit box, never divided by.)
+            if (e >= 2) {
+                int sft = 0;
+                while (((int64_t)1 << sft) < e) ++sft;
+                const unsigned __int128 num = (unsigned __int128)1 << (31 + sft);
+                b.magic[i] = (uint32_t)((num + (uint64_t)e - 1) / (uint64_t)e);
+                b.shift[i] = (uint32_t)(sft - 1);
+            }
             units *= e;
         }
-        if (units >= (int64_t)UINT32_MAX) return false;
+        if (units >= ((int64_t)1 << 31)) return false;
+        const int32_t src_begin = (int32_t)plan->sources.size();
         for (size_t j = 0; j < srcs.size(); ++j) {
             HaloSource s;
             memset(&s, 0, sizeof(s));
             s.shard = srcs[j].r.shard;
             s.close = srcs[j].close;
             s.clear_after = srcs[j].clear_after;
-            s.offset = soff[j] / unit;
-            for (int i = 0; i < nd; ++i) s.stride[i] = (i == nd - 1) ? ss[j][i] : ss[j][i] / unit;
+            s.offset = (uint32_t)soff[j];
+            for (int i = 0; i < nd_units; ++i) s.stride[i] = (uint32_t)ss[j][i];
             plan->sources.push_back(s);
         }
         const int32_t box_id = (int32_t)plan->boxes.size();
         plan->boxes.push_back(b);
         for (int64_t at = 0; at < units; at += kTileUnits) {
             HaloTile t;
+            memset(&t, 0, sizeof(t));
             t.box = box_id;
+            t.src_begin = src_begin;
+            t.nsrc = (int32_t)srcs.size();
             t.first = (uint32_t)at;
             t.count = (uint32_t)std::min<int64_t>(kTileUnits, units - at);
             plan->tiles.push_back(t);
