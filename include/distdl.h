@@ -184,9 +184,10 @@ distdl_status_t distdl_conv_adj(const distdl_partition_t *p, const void *const *
  * y[i]  F32  [nb, nfo/Pfo]      bias[i] F32 [nfo/Pfo] or bias == NULL
  * dy[i] BF16 [nb, nfo/Pfo]      dx[j] F32 [nb, nfi/Pfi]
  * The contraction runs on the tensor cores with fp32 accumulation; the sums of R continue in the
- * same fp32 accumulator in the stated order.  nfi % Pfi == 0, nfo % Pfo == 0; the per-worker
- * block sizes must be multiples of 64 and nb a multiple of 8, nb <= 256 per call
- * (else DISTDL_ERR_UNSUPPORTED).
+ * same fp32 accumulator in the stated order.  nfi % Pfi == 0, nfo % Pfo == 0 (else
+ * DISTDL_ERR_SHAPE); the per-worker block sizes nfi/Pfi and nfo/Pfo must be multiples of 128,
+ * Pfo, Pfi <= 8 and Pfo * Pfi <= 16 (else DISTDL_ERR_UNSUPPORTED); nb >= 1 is arbitrary.
+ * A launch whose device-side waits ran out reports through distdl_device_status().
  * ---------------------------------------------------------------------- */
 distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
                                   const void *const *x, const void *const *w,
@@ -194,6 +195,12 @@ distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t 
 distdl_status_t distdl_affine_adj(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
                                   const void *const *dy, const void *const *w, void *const *dx,
                                   void *stream);
+
+/* Synchronises `stream`, then reads and clears the device status word that the affine kernels set
+ * when one of their bounded waits (on a shared-memory barrier fed by TMA or by the tensor cores)
+ * ran out: DISTDL_ERR_TIMEOUT in that case (the outputs of that launch are then undefined),
+ * DISTDL_OK otherwise.  The only call of this library that blocks the host. */
+distdl_status_t distdl_device_status(void *stream);
 
 /* Thread-local message of the last error returned on this thread ("" if none). */
 const char *distdl_last_error(void);

@@ -64,9 +64,9 @@ def lib():
     L.distdl_halo_adj.argtypes = [vp, pvp, vp]
     L.distdl_conv_fwd.argtypes = [vp, pvp, vp, vp, c_i32, c_i32, pvp, vp]
     L.distdl_conv_adj.argtypes = [vp, pvp, vp, c_i32, c_i32, pvp, vp]
-    if hasattr(L, "distdl_affine_fwd"):
-        L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
-        L.distdl_affine_adj.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, vp]
+    L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
+    L.distdl_affine_adj.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, vp]
+    L.distdl_device_status.argtypes = [vp]
     _lib = L
     return L
 
@@ -248,3 +248,8 @@ def affine_fwd(nb, nfi, nfo, pfo, pfi, x, w, bias, y, stream=None):
 def affine_adj(nb, nfi, nfo, pfo, pfi, dy, w, dx, stream=None):
     _check(lib().distdl_affine_adj(nb, nfi, nfo, pfo, pfi, _ptr_array(dy), _ptr_array(w), _ptr_array(dx),
                                    _stream(stream)))
+
+
+def device_status(stream=None):
+    """Synchronises the stream and raises DistdlError(DISTDL_ERR_TIMEOUT) if an affine kernel gave up."""
+    _check(lib().distdl_device_status(_stream(stream)))

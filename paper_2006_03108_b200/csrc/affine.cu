@@ -1,0 +1,413 @@
+// Distributed affine layer on a Pfo x Pfi worker grid (Section 4, "Dense layers"): forward
+//   x^_{ij} <- B x_j ;  y^_{ij} <- x^_{ij} W_{ij}^T (+ b_i on column j = 0) ;  y_i <- R_j y^_{ij}
+// and adjoint (dx only)
+//   dy^_{ij} <- B dy_i ;  dx^_{ij} <- dy^_{ij} W_{ij} ;  dx_j <- R_i dx^_{ij}.
+//
+// All workers live in one device memory, so the broadcast is implicit (every thread block that
+// needs a block of x reads it through L2 -- no copy is materialised) and the sum-reduce is the
+// tensor-core accumulator itself: one thread block owns a 128 x 128 tile of the output and walks
+// through the workers of its grid row (forward) or grid column (adjoint) in worker order, so the
+// partial products y^_{ij} never exist in memory and the order of the sum is fixed.
+//
+// Kernel: warp-specialised, one TMA producer thread, one tcgen05.mma issuer thread, four epilogue
+// warps.  Operands are staged by TMA (128-byte swizzle) into a ring of shared-memory stages; the
+// fp32 accumulator lives in tensor memory and is read back with tcgen05.ld for the epilogue.
+// The forward contraction takes W as the K-major operand ([out, in] rows are contiguous in K =
+// in); the adjoint takes the same buffers as the MN-major operand, so no transposed copy of W is
+// ever made.  Every wait is bounded: if one runs out, the block records DISTDL_ERR_TIMEOUT in a
+// device status word, releases its tensor memory and returns.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "common.h"
+
+namespace distdl {
+
+constexpr int kTileM = 128;
+constexpr int kTileN = 128;
+constexpr int kBlockK = 64;                 // 64 bf16 = one 128-byte swizzle row
+constexpr int kStages = 6;
+constexpr int kStageABytes = kTileM * kBlockK * 2;   // 16 KB
+constexpr int kStageBBytes = kTileN * kBlockK * 2;   // 16 KB
+constexpr int kStageBytes = kStageABytes + kStageBBytes;
+constexpr int kAffineThreads = 192;         // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
+constexpr int kMaxMaps = 24;                // tensor maps passed as kernel parameters
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+
+__device__ int g_affine_status = 0;         // 0 = ok, otherwise DISTDL_ERR_TIMEOUT
+
+struct AffineParams {
+    CUtensorMap a_map[8];                   // activation blocks (x_j forward, dy_i adjoint)
+    CUtensorMap w_map[kMaxMaps - 8];        // weight blocks, worker order i * pfi + j
+    float *out[8];                          // output blocks (y_i forward, dx_j adjoint)
+    const float *bias[8];                   // forward only, may be all null
+    int32_t nb;                             // batch rows
+    int32_t pfo, pfi;
+    int32_t blk_out;                        // columns of one output block
+    int32_t blk_red;                        // length of the contraction inside one worker
+    int32_t nred;                           // workers summed over (pfi forward, pfo adjoint)
+    int32_t adjoint;
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t global_timer() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait: false if the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(&g_affine_status, (int)DISTDL_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Fields (bit positions): start address >> 4
+// [0,14), leading byte offset >> 4 [16,30), stride byte offset >> 4 [32,46), descriptor version 1
+// [46,48), layout type 2 = 128-byte swizzle [61,64).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor of kind::f16: D = fp32 [4,6) = 1, A = B = bf16 [7,10) = [10,13) = 1,
+// A major bit 15, B major bit 16 (0 = K-major, 1 = MN-major), N >> 3 in [17,23), M >> 4 in [24,29).
+__host__ __device__ constexpr uint32_t instr_desc(int m, int n, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(m >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel: grid.x = output tiles along the feature axis * row tiles (row tile fastest, so the
+// blocks that share a weight tile run together and the tile comes from DRAM once).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kAffineThreads, 1)
+affine_kernel(const __grid_constant__ AffineParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment: the 128-byte swizzle pattern is a function of address bits [7,10)
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *aligned = smem_raw + (base - raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kStages * kStageBytes);
+    const uint32_t bar_full = smem_u32(bars);                  // kStages barriers
+    const uint32_t bar_empty = bar_full + 8 * kStages;         // kStages barriers
+    const uint32_t bar_acc = bar_empty + 8 * kStages;          // accumulator complete
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row_tiles = (P.nb + kTileM - 1) / kTileM;
+    const int m0 = (blockIdx.x % row_tiles) * kTileM;
+    const int ntile = blockIdx.x / row_tiles;
+    const int tiles_per_block = P.blk_out / kTileN;
+    const int oblk = ntile / tiles_per_block;                  // output block (i forward, j adjoint)
+    const int n0 = (ntile % tiles_per_block) * kTileN;         // first output column inside the block
+    const int kblocks_per_worker = P.blk_red / kBlockK;
+    const int num_kblocks = P.nred * kblocks_per_worker;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        // 128 columns of tensor memory: one fp32 accumulator of 128 lanes x 128 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kblocks; ++kb) {
+                const int s = kb % kStages;
+                const uint32_t phase = (kb / kStages) & 1;
+                if (!mbar_wait(bar_empty + 8 * s, phase ^ 1, abort_flag)) break;
+                const int r = kb / kblocks_per_worker;          // worker along the reduction
+                const int k0 = (kb % kblocks_per_worker) * kBlockK;
+                const uint32_t sa = base + s * kStageBytes, sb = sa + kStageABytes;
+                mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+                // activations: box {64 k, 128 rows} of block r at (k0, m0)
+                tma_load_2d(sa, &P.a_map[r], k0, m0, bar_full + 8 * s);
+                if (!P.adjoint) {
+                    // W_{oblk, r}: rows = output features, K-major: box {64 k, 128 rows} at (k0, n0)
+                    tma_load_2d(sb, &P.w_map[oblk * P.pfi + r], k0, n0, bar_full + 8 * s);
+                } else {
+                    // W_{r, oblk}: rows = reduction index, MN-major: two boxes {64 n, 64 k}
+                    const CUtensorMap *wm = &P.w_map[r * P.pfi + oblk];
+                    tma_load_2d(sb, wm, n0, k0, bar_full + 8 * s);
+                    tma_load_2d(sb + kStageBBytes / 2, wm, n0 + 64, k0, bar_full + 8 * s);
+                }
+                ++issued;
+            }
+            if (*abort_flag) {
+                // give copies that are still in flight time to land before the block retires
+                const uint64_t t0 = global_timer();
+                while (global_timer() - t0 < 1000000ull) {}
+            }
+            (void)issued;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(kTileM, kTileN, P.adjoint ? 1 : 0);
+            bool ok = true;
+            for (int kb = 0; kb < num_kblocks && ok; ++kb) {
+                const int s = kb % kStages;
+                const uint32_t phase = (kb / kStages) & 1;
+                ok = mbar_wait(bar_full + 8 * s, phase, abort_flag);
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint32_t sa = base + s * kStageBytes, sb = sa + kStageABytes;
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k) {
+                    // A, K-major: 8-row groups 1024 bytes apart; step 32 bytes along K
+                    const uint64_t adesc = smem_desc(sa + k * 32, 16, 1024);
+                    uint64_t bdesc;
+                    if (!P.adjoint) bdesc = smem_desc(sb + k * 32, 16, 1024);
+                    // B, MN-major: 64-column atoms 8192 bytes apart (leading), 8-k groups 1024
+                    // bytes apart (stride); step 16 k-rows = 2048 bytes
+                    else bdesc = smem_desc(sb + k * 2048, kStageBBytes / 2, 1024);
+                    umma_bf16(tmem_acc, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
+                }
+                tcgen05_commit(bar_empty + 8 * s);     // frees the stage once these MMAs retire
+            }
+            if (ok) tcgen05_commit(bar_acc);           // accumulator complete
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int quarter = warp & 3;                  // tensor-memory lanes [32 q, 32 q + 32)
+        // warp-uniform outcome: tcgen05.ld below is a warp-collective instruction
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, abort_flag));
+        tcgen05_fence_after();
+        if (ok) {
+            const int row = m0 + quarter * 32 + lane;
+            float *out = P.out[oblk] + (size_t)row * P.blk_out + n0;
+            const float *bias = P.bias[oblk];
+#pragma unroll 1
+            for (int c = 0; c < kTileN; c += 32) {
+                uint32_t v[32];
+                const uint32_t taddr = tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                    "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                      "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                      "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row < P.nb) {
+#pragma unroll
+                    for (int q = 0; q < 32; q += 4) {
+                        float4 o;
+                        o.x = __uint_as_float(v[q + 0]);
+                        o.y = __uint_as_float(v[q + 1]);
+                        o.z = __uint_as_float(v[q + 2]);
+                        o.w = __uint_as_float(v[q + 3]);
+                        if (bias) {
+                            const float4 b = __ldg(reinterpret_cast<const float4 *>(bias + n0 + c + q));
+                            o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                        }
+                        *reinterpret_cast<float4 *>(out + c + q) = o;
+                    }
+                }
+            }
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kTileN) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)sym;
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows, cols]; box = {box_cols (inner), box_rows}; 128-byte swizzle.
+static bool make_map(CUtensorMap *m, const void *ptr, int64_t rows, int64_t cols, int box_cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                   const void *const *act, const void *const *w, const void *const *bias,
+                                   void *const *out, void *stream, bool adjoint, const char *what) {
+    clear_error();
+    if (!act || !w || !out) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (nb < 1 || nfi < 1 || nfo < 1 || pfo < 1 || pfi < 1)
+        return fail(DISTDL_ERR_INVALID_ARG, "%s: non-positive size", what);
+    if (nfi % pfi || nfo % pfo) return fail(DISTDL_ERR_SHAPE, "%s: features not divisible by the worker grid", what);
+    const int64_t bfi = nfi / pfi, bfo = nfo / pfo;
+    if (bfi % kTileN || bfo % kTileN)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: per-worker feature blocks must be multiples of %d", what, kTileN);
+    if (pfo > 8 || pfi > 8 || pfo * pfi > kMaxMaps - 8)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: worker grid larger than 8 per side or %d workers", what, kMaxMaps - 8);
+    if (nb > (1 << 20)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: batch too large", what);
+    const int nact = adjoint ? pfo : pfi, nout = adjoint ? pfi : pfo;
+    for (int i = 0; i < nact; ++i) {
+        if (!act[i]) return fail(DISTDL_ERR_INVALID_ARG, "%s: activation block %d is NULL", what, i);
+        if (!aligned16(act[i])) return fail(DISTDL_ERR_ALIGNMENT, "%s: activation block %d not 16-byte aligned", what, i);
+    }
+    for (int i = 0; i < nout; ++i) {
+        if (!out[i]) return fail(DISTDL_ERR_INVALID_ARG, "%s: output block %d is NULL", what, i);
+        if (!aligned16(out[i])) return fail(DISTDL_ERR_ALIGNMENT, "%s: output block %d not 16-byte aligned", what, i);
+        if (bias && bias[i] && !aligned16(bias[i])) return fail(DISTDL_ERR_ALIGNMENT, "%s: bias %d not 16-byte aligned", what, i);
+    }
+    for (int i = 0; i < pfo * pfi; ++i) {
+        if (!w[i]) return fail(DISTDL_ERR_INVALID_ARG, "%s: weight block %d is NULL", what, i);
+        if (!aligned16(w[i])) return fail(DISTDL_ERR_ALIGNMENT, "%s: weight block %d not 16-byte aligned", what, i);
+    }
+    if (!encode_fn()) return fail(DISTDL_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", what);
+
+    AffineParams P;
+    memset(&P, 0, sizeof(P));
+    const int64_t act_cols = adjoint ? bfo : bfi;
+    for (int i = 0; i < nact; ++i)
+        if (!make_map(&P.a_map[i], act[i], nb, act_cols, kBlockK, kTileM))
+            return fail(DISTDL_ERR_CUDA, "%s: tensor map of activation block %d failed", what, i);
+    for (int i = 0; i < pfo * pfi; ++i) {
+        // forward: box {64 along in-features (K), 128 out-feature rows}; adjoint: box {64 along
+        // in-features (N), 64 out-feature rows (K)} of the same row-major [bfo, bfi] block
+        const bool ok = adjoint ? make_map(&P.w_map[i], w[i], bfo, bfi, 64, kBlockK)
+                                : make_map(&P.w_map[i], w[i], bfo, bfi, kBlockK, kTileN);
+        if (!ok) return fail(DISTDL_ERR_CUDA, "%s: tensor map of weight block %d failed", what, i);
+    }
+    for (int i = 0; i < nout; ++i) {
+        P.out[i] = (float *)out[i];
+        P.bias[i] = (!adjoint && bias) ? (const float *)bias[i] : nullptr;
+    }
+    P.nb = (int32_t)nb;
+    P.pfo = pfo;
+    P.pfi = pfi;
+    P.blk_out = (int32_t)(adjoint ? bfi : bfo);
+    P.blk_red = (int32_t)(adjoint ? bfo : bfi);
+    P.nred = adjoint ? pfo : pfi;
+    P.adjoint = adjoint ? 1 : 0;
+
+    static bool configured = false;
+    if (!configured) {
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        configured = true;
+    }
+    const int64_t row_tiles = (nb + kTileM - 1) / kTileM;
+    const int64_t ntiles = (adjoint ? nfi : nfo) / kTileN;
+    affine_kernel<<<(unsigned)(row_tiles * ntiles), kAffineThreads, kSmemBytes, (cudaStream_t)stream>>>(P);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+}  // namespace distdl
+
+extern "C" distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                             const void *const *x, const void *const *w, const void *const *bias,
+                                             void *const *y, void *stream) {
+    return distdl::affine_impl(nb, nfi, nfo, pfo, pfi, x, w, bias, y, stream, false, "affine_fwd");
+}
+
+extern "C" distdl_status_t distdl_affine_adj(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                             const void *const *dy, const void *const *w, void *const *dx,
+                                             void *stream) {
+    return distdl::affine_impl(nb, nfi, nfo, pfo, pfi, dy, w, nullptr, dx, stream, true, "affine_adj");
+}
+
+extern "C" distdl_status_t distdl_device_status(void *stream) {
+    using namespace distdl;
+    clear_error();
+    DISTDL_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+    int st = 0;
+    DISTDL_CUDA_CHECK(cudaMemcpyFromSymbol(&st, g_affine_status, sizeof(int)));
+    if (st != 0) {
+        const int zero = 0;
+        DISTDL_CUDA_CHECK(cudaMemcpyToSymbol(g_affine_status, &zero, sizeof(int)));
+        return fail(DISTDL_ERR_TIMEOUT, "a bounded device-side wait of an affine kernel ran out");
+    }
+    return DISTDL_OK;
+}

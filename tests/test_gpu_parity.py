@@ -268,3 +268,80 @@ def test_conv_fwd_and_adj(case):
     xb = oracle.scatter_global(opart, xg)                # zero ghosts: the inner product is over the bulk
     r = oracle.adjoint_test_ratio([host(t) for t in y0], dy, xb, [host(t) for t in dxs])
     assert r < 1e-5
+
+
+# --------------------------------------------------------------------------
+# Affine layer
+# --------------------------------------------------------------------------
+
+AFFINE_CASES = [
+    # nb, nfi, nfo, pfo, pfi
+    (16, 256, 256, 2, 2),
+    (128, 128, 128, 1, 1),
+    (200, 512, 384, 3, 2),       # ragged batch (two row tiles, the second partly empty)
+    (256, 1024, 512, 4, 4),
+    (77, 256, 1024, 1, 2),
+    (300, 768, 256, 2, 1),
+]
+
+
+def _affine_inputs(nb, nfi, nfo, pfo, pfi, seed, integer=False):
+    if integer:
+        xg = inputs.integers((nb, nfi), seed, -3, 4)
+        wg = inputs.integers((nfo, nfi), seed + 1, -3, 4)
+        dyg = inputs.integers((nb, nfo), seed + 2, -3, 4)
+    else:
+        xg = inputs.normal((nb, nfi), seed)
+        wg = inputs.normal((nfo, nfi), seed + 1, nfi ** -0.5)
+        dyg = inputs.normal((nb, nfo), seed + 2)
+    xb, wb, dyb = (inputs.f32_to_bf16_bits(a) for a in (xg, wg, dyg))
+    xs = np.split(xb, pfi, axis=1)
+    ws = [blk for row in np.split(wb, pfo, axis=0) for blk in np.split(row, pfi, axis=1)]
+    dys = np.split(dyb, pfo, axis=1)
+    return xs, ws, dys
+
+
+def _bf16_dev(bits):
+    return dev(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+
+
+def _rel_errors(got, ref):
+    got = np.concatenate([g.astype(np.float64) for g in got], axis=1)
+    ref = np.concatenate([r.astype(np.float64) for r in ref], axis=1)
+    return np.max(np.abs(got - ref)) / np.max(np.abs(ref)), np.linalg.norm(got - ref) / np.linalg.norm(ref)
+
+
+@pytest.mark.parametrize("case", AFFINE_CASES, ids=[str(c) for c in AFFINE_CASES])
+@pytest.mark.parametrize("integer", [True, False], ids=["int", "normal"])
+def test_affine_fwd_and_adj(case, integer):
+    nb, nfi, nfo, pfo, pfi = case
+    xs, ws, dys = _affine_inputs(nb, nfi, nfo, pfo, pfi, 41, integer)
+    bias = np.split(inputs.integers((nfo,), 44) if integer else inputs.normal((nfo,), 44), pfo)
+    x_d, w_d, dy_d = [_bf16_dev(a) for a in xs], [_bf16_dev(a) for a in ws], [_bf16_dev(a) for a in dys]
+    b_d = [dev(b) for b in bias]
+    y_d = [torch.full((nb, nfo // pfo), -9.0, device=DEV) for _ in range(pfo)]
+    dx_d = [torch.full((nb, nfi // pfi), -9.0, device=DEV) for _ in range(pfi)]
+    distdl.affine_fwd(nb, nfi, nfo, pfo, pfi, x_d, w_d, b_d, y_d)
+    distdl.affine_adj(nb, nfi, nfo, pfo, pfi, dy_d, w_d, dx_d)
+    distdl.device_status()
+    xf = [oracle.bf16_bits_to_f64(a) for a in xs]
+    wf = [oracle.bf16_bits_to_f64(a) for a in ws]
+    dyf = [oracle.bf16_bits_to_f64(a) for a in dys]
+    y_ref = oracle.affine_fwd(xf, wf, pfo, pfi, bias)
+    dx_ref = oracle.affine_adj(dyf, wf, pfo, pfi)
+    y, dx = [host(t) for t in y_d], [host(t) for t in dx_d]
+    if integer:
+        # small integers: every product and partial sum is exact in fp32, any order
+        for a, b in zip(y + dx, y_ref + dx_ref):
+            assert np.array_equal(a, b)
+    else:
+        for got, ref in ((y, y_ref), (dx, dx_ref)):
+            emax, el2 = _rel_errors(got, ref)
+            assert emax < 2e-2 and el2 < 2e-2          # the stated bound
+            assert emax < 1e-4 and el2 < 1e-5          # what fp32 accumulation of exact products gives
+        # dot-product test of the pair (no bias: it is not part of the linear operator)
+        y0 = [torch.empty_like(t) for t in y_d]
+        distdl.affine_fwd(nb, nfi, nfo, pfo, pfi, x_d, w_d, None, y0)
+        distdl.device_status()
+        r = oracle.adjoint_test_ratio([host(t) for t in y0], dyf, xf, dx)
+        assert r < 1e-4
