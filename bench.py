@@ -59,7 +59,7 @@ def conv_algorithmic_bytes(part):
 class Workload:
     """All buffers of one step, resident on `dev`, and the eight operator calls."""
 
-    def __init__(self, dev):
+    def __init__(self, dev, small=False):
         import torch
         import paper_2006_03108_b200 as distdl
         self.torch, self.d, self.dev = torch, distdl, dev
@@ -69,7 +69,7 @@ class Workload:
         n = lambda *s: torch.randn(*s, device=dev, generator=g)
         # broadcast / sum-reduce: fp32 [4096, 4096], 8 workers
         self.k = 8
-        rows = 4096
+        rows = 1024 if small else 4096   # small: the reduced case for profiler captures
         self.b_src = u(rows, 4096)
         self.b_dst = [torch.empty(rows, 4096, device=dev) for _ in range(self.k)]
         self.r_src = [u(rows, 4096) for _ in range(self.k)]
@@ -80,7 +80,7 @@ class Workload:
         self.h_x = [u(*self.hpart.padded_shape(w)) for w in range(self.hpart.num_workers)]
         self.h_y = [u(*self.hpart.padded_shape(w)) for w in range(self.hpart.num_workers)]
         # conv: NCHW [16,16,1024,1024] over 1x1x4x4 workers, depthwise 5x5
-        nc = 16
+        nc = 4 if small else 16
         self.cpart = distdl.Partition((nc, 16, 1024, 1024), (1, 1, 4, 4), (0, 0, 2, 2), (0, 0, 2, 2))
         P = self.cpart.num_workers
         self.c_x = [n(*self.cpart.padded_shape(w)) for w in range(P)]
@@ -314,6 +314,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-op", default=None,
+                    help="run only this operator, three times, on a reduced case (for profiler captures) and exit")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -335,6 +337,19 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     warmup = max(args.warmup, 3)
     peaks = measured_peaks()
+
+    if args.profile_op:
+        wl = Workload(dev, small=True)
+        op = [o for o in wl.ops if o[0] == args.profile_op]
+        if not op:
+            raise SystemExit("unknown operator %r" % args.profile_op)
+        for _ in range(3):
+            op[0][1]()
+        torch.cuda.synchronize()
+        import paper_2006_03108_b200 as distdl
+        distdl.device_status()
+        print(json.dumps({"profile_op": args.profile_op, "algorithmic_bytes": op[0][2], "flops": op[0][3]}))
+        return
 
     wl = Workload(dev)
     nops = len(wl.ops)

@@ -21,6 +21,7 @@
 #include <cstring>
 
 #include "common.h"
+#include "tma.h"
 
 namespace distdl {
 
@@ -54,27 +55,6 @@ struct AffineParams {
 // ------------------------------------------------------------------------------------------
 // PTX wrappers
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint64_t global_timer() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
-}
 // Bounded wait: false if the limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -88,11 +68,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -162,8 +137,7 @@ affine_kernel(const __grid_constant__ AffineParams P) {
         }
         mbar_init(bar_acc, 1);
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_barrier_init();
     }
     if (warp == 1) {
         // 128 columns of tensor memory: one fp32 accumulator of 128 lanes x 128 columns
@@ -288,21 +262,7 @@ affine_kernel(const __grid_constant__ AffineParams P) {
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)sym;
-    }
-    return fn;
-}
+static EncodeTiledFn encode_fn() { return tensor_map_encoder(); }
 
 // Row-major bf16 matrix [rows, cols]; box = {box_cols (inner), box_rows}; 128-byte swizzle.
 static bool make_map(CUtensorMap *m, const void *ptr, int64_t rows, int64_t cols, int box_cols, int box_rows) {
@@ -398,6 +358,10 @@ extern "C" distdl_status_t distdl_affine_adj(int64_t nb, int64_t nfi, int64_t nf
     return distdl::affine_impl(nb, nfi, nfo, pfo, pfi, dy, w, nullptr, dx, stream, true, "affine_adj");
 }
 
+namespace distdl {
+int conv_take_status();   // conv.cu
+}
+
 extern "C" distdl_status_t distdl_device_status(void *stream) {
     using namespace distdl;
     clear_error();
@@ -407,7 +371,11 @@ extern "C" distdl_status_t distdl_device_status(void *stream) {
     if (st != 0) {
         const int zero = 0;
         DISTDL_CUDA_CHECK(cudaMemcpyToSymbol(g_affine_status, &zero, sizeof(int)));
-        return fail(DISTDL_ERR_TIMEOUT, "a bounded device-side wait of an affine kernel ran out");
     }
+    const int cst = conv_take_status();
+    if (cst < 0) return fail(DISTDL_ERR_CUDA, "device_status: reading the status word failed");
+    if (st != 0 || cst != 0)
+        return fail(DISTDL_ERR_TIMEOUT, "a bounded device-side wait of %s kernel ran out",
+                    st != 0 ? "an affine" : "a convolution");
     return DISTDL_OK;
 }

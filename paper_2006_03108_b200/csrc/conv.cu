@@ -10,6 +10,7 @@
 #include <cstring>
 
 #include "common.h"
+#include "tma.h"
 
 namespace distdl {
 
@@ -49,191 +50,539 @@ __device__ __forceinline__ void cp_async16(float *smem, const float *gmem) {
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
+// Packed fp32 pair arithmetic (two FMAs per instruction on sm_100).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ void cp_async4(float *smem, const float *gmem) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+struct ConvTile {
+    int shard, plane, r, c, bh, bw, i0, j0;
+    bool valid;
+};
+
+__device__ __forceinline__ ConvTile decode_tile(const ConvParams &P, int tile, int tiles_y, int planes) {
+    // tile id = ((shard * planes + plane) * tiles_x + tx) * tiles_y + ty : vertically adjacent tiles
+    // get adjacent ids, so the rows they share are still in L2 when the second one asks for them
+    ConvTile t;
+    const int ty = tile % tiles_y;
+    int rest = tile / tiles_y;
+    const int tx = rest % P.tiles_x;
+    rest /= P.tiles_x;
+    t.plane = rest % planes;
+    t.shard = rest / planes;
+    t.r = t.shard / P.pw_workers;
+    t.c = t.shard % P.pw_workers;
+    t.bh = P.bh[t.r];
+    t.bw = P.bw[t.c];
+    t.i0 = ty * kTileH;
+    t.j0 = tx * kTileW;
+    t.valid = t.i0 < t.bh && t.j0 < t.bw;
+    return t;
+}
+
 // K: kernel extent (odd).  ADJ: false = forward (padded x -> bulk-shaped y), true = adjoint
 // (bulk-shaped dy -> padded dx, rotated kernel, ghosts of dx cleared).
+//
+// Persistent blocks walk over the output tiles; the input tile of the next step is fetched with
+// cp.async into the second shared-memory buffer while the current one is being consumed.
 template <int K, bool ADJ>
-__global__ void __launch_bounds__(kConvThreads, 2)
-conv_depthwise_kernel(const __grid_constant__ ConvParams P) {
-    constexpr int PH = K / 2;                    // halo rows = halo columns
-    constexpr int PADL = ADJ ? ((PH + 3) / 4) * 4 : PH;   // shared-memory columns left of the first output
-    constexpr int WOFF = PADL - PH;              // first column a thread needs, relative to its float4 slot
-    constexpr int NV = (WOFF + K + 3 + 3) / 4;   // float4 loads per thread per input row
-    constexpr int PITCH = conv_pitch(K, ADJ);
-    extern __shared__ __align__(16) float tile[];   // [kTileH + K - 1][PITCH]
+struct ConvCfg {
+    static constexpr int PH = K / 2;                                   // halo rows = halo columns
+    static constexpr int PADL = ADJ ? ((PH + 3) / 4) * 4 : PH;         // tile columns left of the first output
+    static constexpr int WOFF = PADL - PH;                             // first column a thread needs in its slot
+    static constexpr int NV = (WOFF + K + 3 + 3) / 4;                  // float4 loads per thread per input row
+    static constexpr int PITCH = conv_pitch(K, ADJ);
+    static constexpr int ROWS = kTileH + K - 1;
+    static constexpr int IOFF = ADJ ? 0 : PH;                          // offset of the bulk in the input layout
+    static constexpr int OOFF = ADJ ? PH : 0;                          // offset of the bulk in the output layout
+    static constexpr int TILE_FLOATS = ROWS * PITCH;
+};
 
-    const int shard = blockIdx.z;
-    const int plane = blockIdx.y;
-    const int r = shard / P.pw_workers, c = shard % P.pw_workers;
-    const int bh = P.bh[r], bw = P.bw[c];
-    const int i0 = (blockIdx.x / P.tiles_x) * kTileH;
-    const int j0 = (blockIdx.x % P.tiles_x) * kTileW;
-    if (i0 >= bh || j0 >= bw) return;
-    const int ch = plane % P.channels;
-
-    // input layout of a shard with bulk (h, w): forward = padded (h + 2PH, w + 2PH), bulk at
-    // (PH, PH); adjoint = bulk-shaped.
-    constexpr int IOFF = ADJ ? 0 : PH;
-    // ---------------------------------------------------------------- stage the input tile
-    // shared column s  <->  bulk column j0 - PADL + s ;  shared row ry  <->  bulk row i0 - PH + ry
-    const int need_cols = min(kTileW, bw - j0) + PADL + PH;           // columns that can be read
+// Issues the asynchronous copies (and the direct zero stores) that fill `tile` for output tile t.
+template <int K, bool ADJ>
+__device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &t, float *tile) {
+    using C = ConvCfg<K, ADJ>;
+    if (!t.valid) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int need_cols = min(kTileW, t.bw - t.j0) + C::PADL + C::PH;
     const int nvec_row = (need_cols + 3) / 4;
-    const int need_rows = min(kTileH, bh - i0) + 2 * PH;
-    for (int idx = threadIdx.x; idx < need_rows * nvec_row; idx += kConvThreads) {
-        const int ry = idx / nvec_row, v = idx - ry * nvec_row;
-        float *dst = tile + ry * PITCH + 4 * v;
-        // resolve the row: which worker row owns bulk row i, or none (outside the tensor)
-        int i = i0 - PH + ry, rr = r;
+    const int need_rows = min(kTileH, t.bh - t.i0) + 2 * C::PH;
+    // vectors [v_lo, v_hi) of a row lie inside this worker column's bulk and are 16-byte aligned
+    const bool fast = ((t.bw + 2 * C::IOFF) % 4) == 0;   // row pitch keeps every row 16-byte aligned
+    const int first_col = t.j0 - C::PADL;                               // bulk column of tile column 0
+    int v_lo = first_col < 0 ? (-first_col + 3) / 4 : 0;
+    int v_hi = min(nvec_row, (t.bw - first_col) / 4);
+    if (!fast) v_lo = v_hi = 0;
+    for (int ry = warp; ry < need_rows; ry += kConvThreads / 32) {
+        // which worker row owns bulk row i (warp-uniform), or none: outside the tensor
+        int i = t.i0 - C::PH + ry, rr = t.r;
         bool row_ok = true;
         if (i < 0) {
-            rr = r - 1;
+            rr = t.r - 1;
             row_ok = rr >= 0;
             if (row_ok) i += P.bh[rr];
-        } else if (i >= bh) {
-            rr = r + 1;
+        } else if (i >= t.bh) {
+            rr = t.r + 1;
             row_ok = rr < P.ph_workers;
-            i -= bh;
+            i -= t.bh;
             if (row_ok) row_ok = i < P.bh[rr];
         }
+        float *srow = tile + ry * C::PITCH;
         if (!row_ok) {
-            *reinterpret_cast<float4 *>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int v = lane; v < nvec_row; v += 32)
+                *reinterpret_cast<float4 *>(srow + 4 * v) = make_float4(0.f, 0.f, 0.f, 0.f);
             continue;
         }
         const int rbh = P.bh[rr];
-        const int jfirst = j0 - PADL + 4 * v;        // bulk column of the vector's first element
-        // fast path: the four columns lie in this worker column's bulk and the address is aligned
-        const int pitch_c = bw + 2 * IOFF;
-        const size_t plane_c = (size_t)(rbh + 2 * IOFF) * pitch_c;
-        const float *row_c = P.in[rr * P.pw_workers + c] + plane * plane_c + (size_t)(i + IOFF) * pitch_c + IOFF;
-        if (jfirst >= 0 && jfirst + 3 < bw && ((reinterpret_cast<uintptr_t>(row_c + jfirst) & 15u) == 0)) {
-            cp_async16(dst, row_c + jfirst);
-            continue;
-        }
-        float vals[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            int j = jfirst + e, cc = c;
+        const int pitch_c = t.bw + 2 * C::IOFF;
+        const float *grow = P.in[rr * P.pw_workers + t.c] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_c +
+                            (size_t)(i + C::IOFF) * pitch_c + C::IOFF + first_col;
+        for (int v = v_lo + lane; v < v_hi; v += 32) cp_async16(srow + 4 * v, grow + 4 * v);
+        // edge columns: left of v_lo and right of v_hi, element by element (neighbour columns or zero)
+        const int n_left = 4 * v_lo, n_right = 4 * (nvec_row - v_hi);
+        for (int e = lane; e < n_left + n_right; e += 32) {
+            const int s = e < n_left ? e : 4 * v_hi + (e - n_left);
+            int j = first_col + s, cc = t.c;
             bool ok = true;
             if (j < 0) {
-                cc = c - 1;
+                cc = t.c - 1;
                 ok = cc >= 0;
-                if (ok) j += P.bw[cc];
-                if (ok) ok = j >= 0;
-            } else if (j >= bw) {
-                cc = c + 1;
+                if (ok) {
+                    j += P.bw[cc];
+                    ok = j >= 0;
+                }
+            } else if (j >= t.bw) {
+                cc = t.c + 1;
                 ok = cc < P.pw_workers;
-                j -= bw;
+                j -= t.bw;
                 if (ok) ok = j < P.bw[cc];
             }
-            float val = 0.f;
             if (ok) {
-                const int pitch_n = P.bw[cc] + 2 * IOFF;
-                const size_t plane_n = (size_t)(rbh + 2 * IOFF) * pitch_n;
-                val = __ldg(P.in[rr * P.pw_workers + cc] + plane * plane_n + (size_t)(i + IOFF) * pitch_n + IOFF + j);
+                const int pitch_n = P.bw[cc] + 2 * C::IOFF;
+                cp_async4(srow + s, P.in[rr * P.pw_workers + cc] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_n +
+                                        (size_t)(i + C::IOFF) * pitch_n + C::IOFF + j);
+            } else {
+                srow[s] = 0.f;
             }
-            vals[e] = val;
         }
-        *reinterpret_cast<float4 *>(dst) = make_float4(vals[0], vals[1], vals[2], vals[3]);
     }
+}
 
-    // ---------------------------------------------------------------- weights to registers
-    float wreg[K * K];
+// Register-tiled stencil of one staged tile: each thread produces 8 rows x 4 columns, two columns
+// per packed FMA.
+template <int K, bool ADJ>
+__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile) {
+    using C = ConvCfg<K, ADJ>;
+    if (!t.valid) return;
+    const int ch = t.plane % P.channels;
+    // weights as broadcast pairs (w, w); adjoint: kernel rotated by 180 degrees
+    uint64_t w2[K * K];
 #pragma unroll
-    for (int t = 0; t < K * K; ++t) {
-        // adjoint: kernel rotated by 180 degrees
-        wreg[t] = __ldg(P.w + (size_t)ch * K * K + (ADJ ? K * K - 1 - t : t));
+    for (int q = 0; q < K * K; ++q) {
+        const float w = __ldg(P.w + (size_t)ch * K * K + (ADJ ? K * K - 1 - q : q));
+        w2[q] = pack2(w, w);
     }
     const float b0 = (!ADJ && P.bias) ? __ldg(P.bias + ch) : 0.f;
 
-    // ---------------------------------------------------------------- clear the ghosts of dx
     if (ADJ) {
-        const int pitch_o = bw + 2 * PH;
-        float *oplane = P.out[shard] + (size_t)plane * (bh + 2 * PH) * pitch_o;
-        const int i1 = min(i0 + kTileH, bh), j1 = min(j0 + kTileW, bw);
-        // padded row / column ranges this block is responsible for (ring included at the edges)
-        const int R0 = i0 == 0 ? 0 : i0 + PH, R1 = i1 == bh ? bh + 2 * PH : i1 + PH;
-        const int C0 = j0 == 0 ? 0 : j0 + PH, C1 = j1 == bw ? bw + 2 * PH : j1 + PH;
+        // clear the part of the ghost ring of dx that borders this tile
+        const int pitch_o = t.bw + 2 * C::PH;
+        float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::PH) * pitch_o;
+        const int i1 = min(t.i0 + kTileH, t.bh), j1 = min(t.j0 + kTileW, t.bw);
+        const int R0 = t.i0 == 0 ? 0 : t.i0 + C::PH, R1 = i1 == t.bh ? t.bh + 2 * C::PH : i1 + C::PH;
+        const int C0 = t.j0 == 0 ? 0 : t.j0 + C::PH, C1 = j1 == t.bw ? t.bw + 2 * C::PH : j1 + C::PH;
         const int ncol = C1 - C0;
-        if (i0 == 0)
-            for (int t = threadIdx.x; t < PH * ncol; t += kConvThreads) oplane[(size_t)(t / ncol) * pitch_o + C0 + t % ncol] = 0.f;
-        if (i1 == bh)
-            for (int t = threadIdx.x; t < PH * ncol; t += kConvThreads) oplane[(size_t)(bh + PH + t / ncol) * pitch_o + C0 + t % ncol] = 0.f;
-        const int Rb0 = max(R0, PH), Rb1 = min(R1, bh + PH);   // rows of the bulk band
-        if (j0 == 0)
-            for (int t = threadIdx.x; t < (Rb1 - Rb0) * PH; t += kConvThreads) oplane[(size_t)(Rb0 + t / PH) * pitch_o + t % PH] = 0.f;
-        if (j1 == bw)
-            for (int t = threadIdx.x; t < (Rb1 - Rb0) * PH; t += kConvThreads) oplane[(size_t)(Rb0 + t / PH) * pitch_o + bw + PH + t % PH] = 0.f;
+        if (t.i0 == 0)
+            for (int q = threadIdx.x; q < C::PH * ncol; q += kConvThreads) oplane[(size_t)(q / ncol) * pitch_o + C0 + q % ncol] = 0.f;
+        if (i1 == t.bh)
+            for (int q = threadIdx.x; q < C::PH * ncol; q += kConvThreads)
+                oplane[(size_t)(t.bh + C::PH + q / ncol) * pitch_o + C0 + q % ncol] = 0.f;
+        const int Rb0 = max(R0, C::PH), Rb1 = min(R1, t.bh + C::PH);
+        if (t.j0 == 0)
+            for (int q = threadIdx.x; q < (Rb1 - Rb0) * C::PH; q += kConvThreads) oplane[(size_t)(Rb0 + q / C::PH) * pitch_o + q % C::PH] = 0.f;
+        if (j1 == t.bw)
+            for (int q = threadIdx.x; q < (Rb1 - Rb0) * C::PH; q += kConvThreads)
+                oplane[(size_t)(Rb0 + q / C::PH) * pitch_o + t.bw + C::PH + q % C::PH] = 0.f;
     }
 
-    cp_async_wait_all();
-    __syncthreads();
-
-    // ---------------------------------------------------------------- register-tiled stencil
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    float acc[kRowsPerThread][4];
+    uint64_t acc[kRowsPerThread][2];
 #pragma unroll
-    for (int a = 0; a < kRowsPerThread; ++a)
-#pragma unroll
-        for (int t = 0; t < 4; ++t) acc[a][t] = b0;
+    for (int a = 0; a < kRowsPerThread; ++a) acc[a][0] = acc[a][1] = pack2(b0, b0);
 
-    const float *trow = tile + (ty * kRowsPerThread) * PITCH + 4 * tx;
+    const float *trow = tile + (ty * kRowsPerThread) * C::PITCH + 4 * tx;
 #pragma unroll
     for (int ry = 0; ry < kRowsPerThread + K - 1; ++ry) {
-        float in[4 * NV];
+        float in[4 * C::NV];
 #pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const float4 q = *reinterpret_cast<const float4 *>(trow + ry * PITCH + 4 * v);
+        for (int v = 0; v < C::NV; ++v) {
+            const float4 q = *reinterpret_cast<const float4 *>(trow + ry * C::PITCH + 4 * v);
             in[4 * v + 0] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
         }
+        // pairs (in[s], in[s+1]) for every s a tap can start at
+        uint64_t pr[4 * C::NV - 1];
+#pragma unroll
+        for (int s2 = 0; s2 < 4 * C::NV - 1; ++s2) pr[s2] = pack2(in[s2], in[s2 + 1]);
 #pragma unroll
         for (int a = 0; a < K; ++a) {
             const int orow = ry - a;       // output row (within the thread's strip) fed by tap row a
             if (orow >= 0 && orow < kRowsPerThread) {
 #pragma unroll
-                for (int b = 0; b < K; ++b)
-#pragma unroll
-                    for (int t = 0; t < 4; ++t)
-                        acc[orow][t] = fmaf(wreg[a * K + b], in[WOFF + t + b], acc[orow][t]);
+                for (int b = 0; b < K; ++b) {
+                    acc[orow][0] = fma2(w2[a * K + b], pr[C::WOFF + b], acc[orow][0]);
+                    acc[orow][1] = fma2(w2[a * K + b], pr[C::WOFF + b + 2], acc[orow][1]);
+                }
             }
         }
     }
 
-    // ---------------------------------------------------------------- store
-    constexpr int OOFF = ADJ ? PH : 0;
-    const int pitch_o = bw + 2 * OOFF;
-    float *oplane = P.out[shard] + (size_t)plane * (bh + 2 * OOFF) * pitch_o;
-    const int jo = j0 + 4 * tx;
+    const int pitch_o = t.bw + 2 * C::OOFF;
+    float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::OOFF) * pitch_o;
+    const int jo = t.j0 + 4 * tx;
 #pragma unroll
     for (int a = 0; a < kRowsPerThread; ++a) {
-        const int io = i0 + ty * kRowsPerThread + a;
-        if (io >= bh || jo >= bw) continue;
-        float *o = oplane + (size_t)(io + OOFF) * pitch_o + OOFF + jo;
-        if (jo + 3 < bw && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-            *reinterpret_cast<float4 *>(o) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
-        } else if (jo + 3 < bw && (reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
-            *reinterpret_cast<float2 *>(o) = make_float2(acc[a][0], acc[a][1]);
-            *reinterpret_cast<float2 *>(o + 2) = make_float2(acc[a][2], acc[a][3]);
+        const int io = t.i0 + ty * kRowsPerThread + a;
+        if (io >= t.bh || jo >= t.bw) continue;
+        float o0, o1, o2, o3;
+        unpack2(acc[a][0], o0, o1);
+        unpack2(acc[a][1], o2, o3);
+        float *o = oplane + (size_t)(io + C::OOFF) * pitch_o + C::OOFF + jo;
+        if (jo + 3 < t.bw && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+            *reinterpret_cast<float4 *>(o) = make_float4(o0, o1, o2, o3);
+        } else if (jo + 3 < t.bw && (reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
+            *reinterpret_cast<float2 *>(o) = make_float2(o0, o1);
+            *reinterpret_cast<float2 *>(o + 2) = make_float2(o2, o3);
         } else {
+            const float ov[4] = {o0, o1, o2, o3};
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
-                if (jo + t < bw) o[t] = acc[a][t];
+            for (int q = 0; q < 4; ++q)
+                if (jo + q < t.bw) o[q] = ov[q];
         }
     }
 }
 
 template <int K, bool ADJ>
-static constexpr int conv_smem_bytes() {
-    return (kTileH + K - 1) * conv_pitch(K, ADJ) * (int)sizeof(float);
+__global__ void __launch_bounds__(kConvThreads, 2)
+conv_depthwise_kernel(const __grid_constant__ ConvParams P, int total_tiles, int tiles_y, int planes) {
+    using C = ConvCfg<K, ADJ>;
+    extern __shared__ __align__(16) float smem[];   // two tile buffers
+    int buf = 0;
+    int tile = blockIdx.x;
+    if (tile >= total_tiles) return;
+    ConvTile cur = decode_tile(P, tile, tiles_y, planes);
+    stage_tile<K, ADJ>(P, cur, smem);
+    cp_async_commit();
+    while (true) {
+        const int next = tile + gridDim.x;
+        const bool has_next = next < total_tiles;
+        ConvTile nxt = cur;
+        if (has_next) {
+            nxt = decode_tile(P, next, tiles_y, planes);
+            stage_tile<K, ADJ>(P, nxt, smem + (buf ^ 1) * C::TILE_FLOATS);
+        }
+        cp_async_commit();
+        cp_async_wait_group<1>();          // everything but the newest group: the current tile is here
+        __syncthreads();
+        compute_tile<K, ADJ>(P, cur, smem + buf * C::TILE_FLOATS);
+        __syncthreads();                   // the buffer may be refilled from now on
+        if (!has_next) break;
+        cur = nxt;
+        tile = next;
+        buf ^= 1;
+    }
+    cp_async_wait_group<0>();
+}
+
+// ---------------------------------------------------------------------------------------------
+// TMA variant (up to 16 workers, 16-byte aligned row pitch): the tile body is fetched by one
+// bulk tensor copy per tile from the shard's own storage; only the halo strips that come from
+// neighbouring shards (or are zero outside the tensor) are fetched cell by cell into a small side
+// buffer and patched into the tile before it is consumed.  Staging then costs a handful of
+// instructions per thread, which leaves the issue slots to the packed FMAs.
+// ---------------------------------------------------------------------------------------------
+constexpr int kConvTmaMaxWorkers = 16;
+constexpr uint64_t kConvWaitLimitNs = 2000000000ull;
+
+__device__ int g_conv_status = 0;
+
+struct ConvTmaParams {
+    ConvParams base;
+    CUtensorMap in_map[kConvTmaMaxWorkers];
+    int32_t total_tiles, tiles_y, planes;
+};
+
+template <int K, bool ADJ>
+struct ConvTmaCfg {
+    using C = ConvCfg<K, ADJ>;
+    static constexpr int TILE_STRIDE = ((C::TILE_FLOATS * 4 + 127) / 128) * 32;     // floats, 128-byte multiple
+    static constexpr int SIDE = 2 * C::PH * C::PITCH + 2 * C::PH * C::ROWS;         // patch cells, upper bound
+    static constexpr int SIDE_STRIDE = ((SIDE + 31) / 32) * 32;
+    static constexpr int BOX_BYTES = C::PITCH * C::ROWS * 4;
+    static constexpr int SMEM_BYTES = 2 * TILE_STRIDE * 4 + 2 * SIDE_STRIDE * 4 + 64 + 128;
+};
+
+// The halo strips of a tile: top / bottom rows and left / right columns that lie outside the
+// shard's own bulk.  Cell q of the list maps to tile coordinates (ry, s).
+struct PatchList {
+    int nT, nB, nL, nR, W, rowB, colL, colR, total;
+};
+
+template <int K, bool ADJ>
+__device__ __forceinline__ PatchList make_patch_list(const ConvTile &t) {
+    using C = ConvCfg<K, ADJ>;
+    PatchList p;
+    const int out_rows = min(kTileH, t.bh - t.i0), out_cols = min(kTileW, t.bw - t.j0);
+    p.W = out_cols + 2 * C::PH;                     // columns a strip spans, starting at colL
+    const int H = out_rows + 2 * C::PH;
+    p.colL = C::PADL - C::PH;
+    p.colR = C::PADL + out_cols;
+    p.rowB = C::PH + out_rows;
+    p.nT = (t.i0 == 0) ? C::PH * p.W : 0;
+    p.nB = (t.i0 + out_rows == t.bh) ? C::PH * p.W : 0;
+    p.nL = (t.j0 == 0) ? C::PH * H : 0;
+    p.nR = (t.j0 + out_cols == t.bw) ? C::PH * H : 0;
+    p.total = p.nT + p.nB + p.nL + p.nR;
+    return p;
 }
 
 template <int K, bool ADJ>
-static distdl_status_t launch_conv(const ConvParams &P, dim3 grid, cudaStream_t s) {
+__device__ __forceinline__ void patch_cell(const PatchList &p, int q, int &ry, int &s) {
+    constexpr int PH = ConvCfg<K, ADJ>::PH;
+    if (q < p.nT) {
+        ry = q / p.W;
+        s = p.colL + q % p.W;
+    } else if (q < p.nT + p.nB) {
+        q -= p.nT;
+        ry = p.rowB + q / p.W;
+        s = p.colL + q % p.W;
+    } else if (q < p.nT + p.nB + p.nL) {
+        q -= p.nT + p.nB;
+        ry = q / PH;
+        s = p.colL + q % PH;
+    } else {
+        q -= p.nT + p.nB + p.nL;
+        ry = q / PH;
+        s = p.colR + q % PH;
+    }
+}
+
+template <int K, bool ADJ>
+__device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const ConvTile &t, float *tile, float *side,
+                                               uint32_t bar) {
+    using C = ConvCfg<K, ADJ>;
+    using T = ConvTmaCfg<K, ADJ>;
+    const ConvParams &P = Q.base;
+    if (!t.valid) return;
+    if (threadIdx.x == 0) {
+        fence_proxy_async();     // earlier generic-proxy accesses to this buffer are ordered before the bulk copy
+        mbar_expect_tx(bar, T::BOX_BYTES);
+        // forward: padded coordinates (bulk column j sits at j + PH); adjoint: bulk coordinates
+        const int x = ADJ ? t.j0 - C::PADL : t.j0;
+        const int y = ADJ ? t.i0 - C::PH : t.i0;
+        tma_load_3d(smem_u32(tile), &Q.in_map[t.shard], x, y, t.plane, bar);
+    }
+    const PatchList pl = make_patch_list<K, ADJ>(t);
+    for (int q = threadIdx.x; q < pl.total; q += kConvThreads) {
+        int ry, s;
+        patch_cell<K, ADJ>(pl, q, ry, s);
+        int i = t.i0 - C::PH + ry, rr = t.r;
+        bool ok = true;
+        if (i < 0) {
+            rr = t.r - 1;
+            ok = rr >= 0;
+            if (ok) i += P.bh[rr];
+        } else if (i >= t.bh) {
+            rr = t.r + 1;
+            ok = rr < P.ph_workers;
+            i -= t.bh;
+            if (ok) ok = i < P.bh[rr];
+        }
+        int j = t.j0 - C::PADL + s, cc = t.c;
+        if (j < 0) {
+            cc = t.c - 1;
+            ok = ok && cc >= 0;
+            if (ok) {
+                j += P.bw[cc];
+                ok = j >= 0;
+            }
+        } else if (j >= t.bw) {
+            cc = t.c + 1;
+            ok = ok && cc < P.pw_workers;
+            j -= t.bw;
+            if (ok) ok = j < P.bw[cc];
+        }
+        if (ok) {
+            const int pitch_n = P.bw[cc] + 2 * C::IOFF;
+            cp_async4(side + q, P.in[rr * P.pw_workers + cc] + (size_t)t.plane * (P.bh[rr] + 2 * C::IOFF) * pitch_n +
+                                    (size_t)(i + C::IOFF) * pitch_n + C::IOFF + j);
+        } else {
+            side[q] = 0.f;
+        }
+    }
+}
+
+template <int K, bool ADJ>
+__global__ void __launch_bounds__(kConvThreads, 2)
+conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
+    using C = ConvCfg<K, ADJ>;
+    using T = ConvTmaCfg<K, ADJ>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    float *tiles = reinterpret_cast<float *>(smem_raw + (((raw + 127u) & ~127u) - raw));
+    float *sides = tiles + 2 * T::TILE_STRIDE;
+    const uint32_t bars = smem_u32(sides + 2 * T::SIDE_STRIDE);
+    if (threadIdx.x == 0) {
+        mbar_init(bars, 1);
+        mbar_init(bars + 8, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    int tile = blockIdx.x;
+    if (tile >= Q.total_tiles) return;
+    int buf = 0;
+    uint32_t phase0 = 0, phase1 = 0;          // parity of the next completion of each buffer's barrier
+    ConvTile cur = decode_tile(Q.base, tile, Q.tiles_y, Q.planes);
+    stage_tile_tma<K, ADJ>(Q, cur, tiles, sides, bars);
+    cp_async_commit();
+    while (true) {
+        const int next = tile + gridDim.x;
+        const bool has_next = next < Q.total_tiles;
+        ConvTile nxt = cur;
+        if (has_next) {
+            nxt = decode_tile(Q.base, next, Q.tiles_y, Q.planes);
+            stage_tile_tma<K, ADJ>(Q, nxt, tiles + (buf ^ 1) * T::TILE_STRIDE, sides + (buf ^ 1) * T::SIDE_STRIDE,
+                                   bars + 8 * (buf ^ 1));
+        }
+        cp_async_commit();
+        cp_async_wait_group<1>();
+        bool ok = true;
+        if (cur.valid) {
+            const uint32_t bar = bars + 8 * buf, parity = buf ? phase1 : phase0;
+            if (!mbar_try_wait(bar, parity)) {
+                const uint64_t t0 = global_timer();
+                while (!mbar_try_wait(bar, parity)) {
+                    if (global_timer() - t0 > kConvWaitLimitNs) {
+                        ok = false;
+                        break;
+                    }
+                }
+            }
+            if (buf) phase1 ^= 1; else phase0 ^= 1;
+        }
+        if (__syncthreads_or(!ok)) {
+            // the bulk copy never arrived: record it and leave (every thread takes this branch)
+            if (threadIdx.x == 0) {
+                atomicExch(&g_conv_status, (int)DISTDL_ERR_TIMEOUT);
+                const uint64_t t0 = global_timer();
+                while (global_timer() - t0 < 1000000ull) {}
+            }
+            break;
+        }
+        float *tl = tiles + buf * T::TILE_STRIDE;
+        if (cur.valid) {
+            const float *sd = sides + buf * T::SIDE_STRIDE;
+            const PatchList pl = make_patch_list<K, ADJ>(cur);
+            for (int q = threadIdx.x; q < pl.total; q += kConvThreads) {
+                int ry, s;
+                patch_cell<K, ADJ>(pl, q, ry, s);
+                tl[ry * C::PITCH + s] = sd[q];
+            }
+        }
+        __syncthreads();
+        compute_tile<K, ADJ>(Q.base, cur, tl);
+        __syncthreads();
+        if (!has_next) break;
+        cur = nxt;
+        tile = next;
+        buf ^= 1;
+    }
+    cp_async_wait_group<0>();
+}
+
+int conv_take_status() {
+    int st = 0;
+    if (cudaMemcpyFromSymbol(&st, g_conv_status, sizeof(int)) != cudaSuccess) return -1;
+    if (st != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_conv_status, &zero, sizeof(int));
+    }
+    return st;
+}
+
+template <int K, bool ADJ>
+static constexpr int conv_smem_bytes() {
+    return 2 * (kTileH + K - 1) * conv_pitch(K, ADJ) * (int)sizeof(float);
+}
+
+template <int K, bool ADJ>
+static distdl_status_t launch_conv(const ConvParams &P, int total_tiles, int tiles_y, int planes, cudaStream_t s) {
     constexpr int smem = conv_smem_bytes<K, ADJ>();
     static bool configured = false;
+    static int blocks = 0;
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_depthwise_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        int dev = 0, sms = 0, per_sm = 0;
+        DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
+        DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, conv_depthwise_kernel<K, ADJ>, kConvThreads, smem));
+        blocks = sms * (per_sm > 0 ? per_sm : 1);
         configured = true;
     }
-    conv_depthwise_kernel<K, ADJ><<<grid, kConvThreads, smem, s>>>(P);
+    const int grid = total_tiles < blocks ? total_tiles : blocks;
+    conv_depthwise_kernel<K, ADJ><<<grid, kConvThreads, smem, s>>>(P, total_tiles, tiles_y, planes);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+template <int K, bool ADJ>
+static distdl_status_t launch_conv_tma(const distdl_partition *p, ConvTmaParams &Q, const void *const *in, cudaStream_t s) {
+    using C = ConvCfg<K, ADJ>;
+    using T = ConvTmaCfg<K, ADJ>;
+    EncodeTiledFn enc = tensor_map_encoder();
+    const int64_t planes = Q.planes;
+    for (int32_t wk = 0; wk < p->num_workers; ++wk) {
+        const int r = wk / Q.base.pw_workers, c = wk % Q.base.pw_workers;
+        const cuuint64_t pitch = (cuuint64_t)(Q.base.bw[c] + 2 * C::IOFF), rows = (cuuint64_t)(Q.base.bh[r] + 2 * C::IOFF);
+        const cuuint64_t dims[3] = {pitch, rows, (cuuint64_t)planes};
+        const cuuint64_t strides[2] = {pitch * 4, pitch * rows * 4};
+        const cuuint32_t box[3] = {(cuuint32_t)C::PITCH, (cuuint32_t)C::ROWS, 1};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (enc(&Q.in_map[wk], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(in[wk]), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return fail(DISTDL_ERR_CUDA, "conv: tensor map of shard %d failed", wk);
+    }
+    static bool configured = false;
+    static int blocks = 0;
+    if (!configured) {
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_tma_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES));
+        int dev = 0, sms = 0, per_sm = 0;
+        DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
+        DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, conv_tma_kernel<K, ADJ>, kConvThreads, T::SMEM_BYTES));
+        blocks = sms * (per_sm > 0 ? per_sm : 1);
+        configured = true;
+    }
+    const int grid = Q.total_tiles < blocks ? Q.total_tiles : blocks;
+    conv_tma_kernel<K, ADJ><<<grid, kConvThreads, T::SMEM_BYTES, s>>>(Q);
     DISTDL_CUDA_CHECK(cudaGetLastError());
     return DISTDL_OK;
 }
@@ -257,7 +606,6 @@ static distdl_status_t conv_impl(const distdl_partition *p, const void *const *i
         }
     if (!aligned16(w) || (bias && !aligned16(bias))) return fail(DISTDL_ERR_ALIGNMENT, "%s: w / bias not 16-byte aligned", what);
     const int64_t planes = p->global_shape[0] * p->global_shape[1];
-    if (planes > 65535) return fail(DISTDL_ERR_UNSUPPORTED, "%s: N*C > 65535", what);
     ConvParams P;
     memset(&P, 0, sizeof(P));
     int64_t max_bh = 0, max_bw = 0;
@@ -282,16 +630,38 @@ static distdl_status_t conv_impl(const distdl_partition *p, const void *const *i
     P.channels = (int32_t)p->global_shape[1];
     P.tiles_x = (int32_t)((max_bw + kTileW - 1) / kTileW);
     const int tiles_y = (int)((max_bh + kTileH - 1) / kTileH);
-    dim3 grid((unsigned)(P.tiles_x * tiles_y), (unsigned)planes, (unsigned)p->num_workers);
+    const int64_t total = (int64_t)P.tiles_x * tiles_y * planes * p->num_workers;
+    if (total >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
     cudaStream_t s = (cudaStream_t)stream;
-    if (!adj) {
-        if (kh == 3) return launch_conv<3, false>(P, grid, s);
-        if (kh == 5) return launch_conv<5, false>(P, grid, s);
-        return launch_conv<7, false>(P, grid, s);
+    const int tt = (int)total, pl = (int)planes;
+    // TMA variant: few enough workers for the tensor maps to travel as kernel parameters, and a row
+    // pitch of whole 16-byte units in every shard's input layout
+    bool tma_ok = p->num_workers <= kConvTmaMaxWorkers && tensor_map_encoder() != nullptr;
+    for (int32_t c = 0; c < p->pshape[3] && tma_ok; ++c) tma_ok = ((P.bw[c] + (adj ? 0 : 2 * h)) % 4) == 0;
+    if (tma_ok) {
+        ConvTmaParams Q;
+        memset(&Q, 0, sizeof(Q));
+        Q.base = P;
+        Q.total_tiles = tt;
+        Q.tiles_y = tiles_y;
+        Q.planes = pl;
+        if (!adj) {
+            if (kh == 3) return launch_conv_tma<3, false>(p, Q, in, s);
+            if (kh == 5) return launch_conv_tma<5, false>(p, Q, in, s);
+            return launch_conv_tma<7, false>(p, Q, in, s);
+        }
+        if (kh == 3) return launch_conv_tma<3, true>(p, Q, in, s);
+        if (kh == 5) return launch_conv_tma<5, true>(p, Q, in, s);
+        return launch_conv_tma<7, true>(p, Q, in, s);
     }
-    if (kh == 3) return launch_conv<3, true>(P, grid, s);
-    if (kh == 5) return launch_conv<5, true>(P, grid, s);
-    return launch_conv<7, true>(P, grid, s);
+    if (!adj) {
+        if (kh == 3) return launch_conv<3, false>(P, tt, tiles_y, pl, s);
+        if (kh == 5) return launch_conv<5, false>(P, tt, tiles_y, pl, s);
+        return launch_conv<7, false>(P, tt, tiles_y, pl, s);
+    }
+    if (kh == 3) return launch_conv<3, true>(P, tt, tiles_y, pl, s);
+    if (kh == 5) return launch_conv<5, true>(P, tt, tiles_y, pl, s);
+    return launch_conv<7, true>(P, tt, tiles_y, pl, s);
 }
 
 }  // namespace distdl
