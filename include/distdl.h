@@ -151,6 +151,36 @@ distdl_status_t distdl_halo_fwd(const distdl_partition_t *p, void *const *shards
 distdl_status_t distdl_halo_adj(const distdl_partition_t *p, void *const *shards, void *stream);
 
 /* ------------------------------------------------------------------------
+ * distdl_halo_fwd_noalloc: the halo exchange H for callers that must not allocate device memory.
+ * (An addition of this library; the paper has no counterpart.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits -- inside a service whose
+ * device memory was handed out in full at start-up, in a latency-critical loop where the implicit
+ * device synchronisation of an allocation is not acceptable, or in a plug-in that is only given
+ * buffers and a stream.  distdl_partition_create allocates a few KB of plan tables on the device;
+ * this call does not: it computes the same plan on the host and copies it, on `stream`, into a
+ * fixed array of 1 MiB that is part of the library image (so every GPU that loads the library
+ * holds that 1 MiB until the process exits).  It calls no cudaMalloc, no cudaFree and no
+ * allocating library routine; its only host-side scratch is ordinary heap memory, freed on return.
+ *
+ * Arguments: the geometry arguments of distdl_partition_create (uniform widths) and the shard
+ * pointers of distdl_halo_fwd; same result as distdl_halo_fwd, bit for bit.
+ * Limits: the plan tables (128 B per box, 48 B per copy source, 32 B per 64 KB tile) must fit in
+ * the 1 MiB array, else DISTDL_ERR_UNSUPPORTED with the sizes in the message -- e.g. 64 workers
+ * in 3-D with 128^3 shards need about 0.36 MiB, 256 workers in 3-D do not fit.
+ * The first call on a device looks up the device address of the array (one cudaGetSymbolAddress
+ * with that device current); make that first call outside any stream capture.
+ * All calls share the one array: the tables of the previous call stay in it and are overwritten,
+ * entry by entry as far as the new plan reaches, before the kernel of this call reads them.  Two
+ * calls whose work overlaps on the GPU (different streams, no ordering between them) race on the
+ * array and give undefined results; calls on one stream are safe.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_halo_fwd_noalloc(int32_t rank, const int64_t *global_shape,
+                                        const int32_t *partition_shape, const int32_t *halo_lo,
+                                        const int32_t *halo_hi, distdl_dtype_t dtype,
+                                        void *const *shards, void *stream);
+
+/* ------------------------------------------------------------------------
  * Distributed convolution layer, feature-space partition only (Section 4, "Sparse layers":
  * forward / adjoint convolution algorithms and the closing remark that the broadcasts and
  * reductions drop out when only the feature space is partitioned).

@@ -62,6 +62,7 @@ def lib():
     L.distdl_broadcast_adj.argtypes = [pvp, vp, c_i32, c_i64, c_i32, vp]
     L.distdl_halo_fwd.argtypes = [vp, pvp, vp]
     L.distdl_halo_adj.argtypes = [vp, pvp, vp]
+    L.distdl_halo_fwd_noalloc.argtypes = [c_i32, pi64, pi32, pi32, pi32, c_i32, pvp, vp]
     L.distdl_conv_fwd.argtypes = [vp, pvp, vp, vp, c_i32, c_i32, pvp, vp]
     L.distdl_conv_adj.argtypes = [vp, pvp, vp, c_i32, c_i32, pvp, vp]
     L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
@@ -226,6 +227,18 @@ def halo_fwd(part, shards, stream=None):
 
 def halo_adj(part, shards, stream=None):
     _check(lib().distdl_halo_adj(part.handle, _ptr_array(shards), _stream(stream)))
+
+
+def halo_fwd_noalloc(global_shape, partition_shape, halo_lo, halo_hi, shards, dtype=F32, stream=None):
+    """H for callers that must not allocate device memory: same result as halo_fwd, but the plan
+    tables go into a fixed 1 MiB device array of the library instead of a cudaMalloc'd block
+    (see distdl_halo_fwd_noalloc in include/distdl.h for the limits and the sharing rules)."""
+    rank = len(global_shape)
+    gs = (ctypes.c_int64 * rank)(*[int(v) for v in global_shape])
+    ps = (ctypes.c_int32 * rank)(*[int(v) for v in partition_shape])
+    lo = None if halo_lo is None else (ctypes.c_int32 * rank)(*[int(v) for v in halo_lo])
+    hi = None if halo_hi is None else (ctypes.c_int32 * rank)(*[int(v) for v in halo_hi])
+    _check(lib().distdl_halo_fwd_noalloc(rank, gs, ps, lo, hi, dtype, _ptr_array(shards), _stream(stream)))
 
 
 def conv_fwd(part, x, w, bias, y, stream=None):

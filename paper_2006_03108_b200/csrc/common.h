@@ -134,6 +134,8 @@ struct distdl_partition {
 namespace distdl {
 // Builds the forward (H) and adjoint (H*) box/tile lists of a partition (host only).
 distdl_status_t build_halo_plans(distdl_partition *p);
-// Checks every box of a plan: inside its shard, destination boxes pairwise disjoint.
-distdl_status_t validate_halo_plan(const distdl_partition *p, const HaloPlanHost &plan);
+// Geometry and halo plans only, no device memory.
+distdl_status_t partition_create_host_only(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
+                                           const int32_t *halo_lo, const int32_t *halo_hi, distdl_dtype_t dtype,
+                                           distdl_partition_t **out);
 }  // namespace distdl

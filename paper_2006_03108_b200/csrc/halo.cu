@@ -271,7 +271,92 @@ static distdl_status_t launch(const distdl_partition *p, const HaloPlanDevice &p
     return DISTDL_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Halo exchange without any device allocation: the plan tables go into a fixed device array.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticPlanBytes = (size_t)1 << 20;   // 1 MiB, held by every device that loads the library
+static __device__ __align__(256) unsigned char g_static_plan[kStaticPlanBytes];
+constexpr int kMaxDevices = 64;
+
+// Device address of g_static_plan on the current device.  In host code the array's name only
+// stands for the symbol; the address a kernel can use has to be asked for, once per device.
+static distdl_status_t static_plan_address(unsigned char **out) {
+    static unsigned char *cached[kMaxDevices] = {nullptr};
+    int dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(DISTDL_ERR_UNSUPPORTED, "halo_fwd_noalloc: device index %d", dev);
+    if (!cached[dev]) {
+        void *ptr = nullptr;
+        DISTDL_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_static_plan));
+        cached[dev] = static_cast<unsigned char *>(ptr);
+    }
+    *out = cached[dev];
+    return DISTDL_OK;
+}
+
+static distdl_status_t halo_fwd_noalloc_impl(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
+                                             const int32_t *halo_lo, const int32_t *halo_hi, distdl_dtype_t dtype,
+                                             void *const *shards, void *stream) {
+    const char *what = "halo_fwd_noalloc";
+    clear_error();
+    if (!shards) return fail(DISTDL_ERR_INVALID_ARG, "%s: shards is NULL", what);
+    distdl_partition *p = nullptr;
+    distdl_status_t st = partition_create_host_only(rank, global_shape, partition_shape, halo_lo, halo_hi, dtype, &p);
+    if (st != DISTDL_OK) return st;
+    struct Guard {
+        distdl_partition *p;
+        ~Guard() { delete p; }
+    } guard{p};
+    const HaloPlanHost &h = p->fwd_host;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t bz = up(h.boxes.size() * sizeof(HaloBox)), sz = up(h.sources.size() * sizeof(HaloSource)),
+                 tz = up(h.tiles.size() * sizeof(HaloTile));
+    if (bz + sz + tz > kStaticPlanBytes)
+        return fail(DISTDL_ERR_UNSUPPORTED,
+                    "%s: the plan of this partition needs %zu bytes of tables, the fixed device array holds %zu "
+                    "(use distdl_partition_create + distdl_halo_fwd for larger partitions)",
+                    what, bz + sz + tz, kStaticPlanBytes);
+    ShardPointers sh;
+    const int64_t es = elem_size(p->dtype);
+    for (int32_t w = 0; w < p->num_workers; ++w) {
+        if (!shards[w]) return fail(DISTDL_ERR_INVALID_ARG, "%s: shards[%d] is NULL", what, w);
+        if (!aligned16(shards[w])) return fail(DISTDL_ERR_ALIGNMENT, "%s: shards[%d] is not 16-byte aligned", what, w);
+        sh.p[w] = shards[w];
+    }
+    for (int32_t a = 0; a < p->num_workers; ++a)
+        for (int32_t b = a + 1; b < p->num_workers; ++b) {
+            const char *a0 = (const char *)shards[a], *a1 = a0 + p->shard_elems(a) * es;
+            const char *b0 = (const char *)shards[b], *b1 = b0 + p->shard_elems(b) * es;
+            if (a0 < b1 && b0 < a1) return fail(DISTDL_ERR_INVALID_ARG, "%s: shards %d and %d overlap", what, a, b);
+        }
+    for (int32_t w = p->num_workers; w < DISTDL_MAX_WORKERS; ++w) sh.p[w] = nullptr;
+    if (h.tiles.empty()) return DISTDL_OK;
+    unsigned char *base = nullptr;
+    st = static_plan_address(&base);
+    if (st != DISTDL_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    // Every table entry the kernel reads is rewritten here, so nothing of an earlier call is used.
+    // The copies are stream-ordered before the kernel; pageable sources are staged before the call
+    // returns, so the host tables may go away right after it.
+    DISTDL_CUDA_CHECK(cudaMemcpyAsync(base, h.boxes.data(), h.boxes.size() * sizeof(HaloBox), cudaMemcpyHostToDevice, s));
+    if (!h.sources.empty())
+        DISTDL_CUDA_CHECK(cudaMemcpyAsync(base + bz, h.sources.data(), h.sources.size() * sizeof(HaloSource), cudaMemcpyHostToDevice, s));
+    DISTDL_CUDA_CHECK(cudaMemcpyAsync(base + bz + sz, h.tiles.data(), h.tiles.size() * sizeof(HaloTile), cudaMemcpyHostToDevice, s));
+    halo_box_kernel<false><<<(unsigned)h.tiles.size(), kHaloThreads, 0, s>>>(
+        reinterpret_cast<const HaloBox *>(base), reinterpret_cast<const HaloSource *>(base + bz),
+        reinterpret_cast<const HaloTile *>(base + bz + sz), elem_size(p->dtype), sh);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
 }  // namespace distdl
+
+extern "C" distdl_status_t distdl_halo_fwd_noalloc(int32_t rank, const int64_t *global_shape,
+                                                   const int32_t *partition_shape, const int32_t *halo_lo,
+                                                   const int32_t *halo_hi, distdl_dtype_t dtype, void *const *shards,
+                                                   void *stream) {
+    return distdl::halo_fwd_noalloc_impl(rank, global_shape, partition_shape, halo_lo, halo_hi, dtype, shards, stream);
+}
 
 extern "C" distdl_status_t distdl_halo_fwd(const distdl_partition_t *p, void *const *shards, void *stream) {
     return distdl::launch(p, p ? p->fwd_dev : distdl::HaloPlanDevice(), shards, stream, false, "halo_fwd");

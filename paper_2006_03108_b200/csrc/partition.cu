@@ -9,7 +9,7 @@ using namespace distdl;
 static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
                                    const int32_t *const *hlo, const int32_t *const *hhi,
                                    const int32_t *ulo, const int32_t *uhi, distdl_dtype_t dtype,
-                                   distdl_partition_t **out) {
+                                   distdl_partition_t **out, bool upload = true) {
     clear_error();
     if (!out) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: out is NULL");
     if (rank < 1 || rank > DISTDL_MAX_RANK)
@@ -75,7 +75,9 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
     // Upload.  Without a CUDA device the object stays host-only: geometry queries work, operator
     // calls report DISTDL_ERR_CUDA.
     int ndev = 0;
-    if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
+    if (!upload) {
+        // host-only object: the caller keeps the plan tables wherever it wants
+    } else if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
         cudaGetDevice(&p->device);
         auto bytes_of = [](const HaloPlanHost &h, size_t *b, size_t *s, size_t *t) {
             auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
@@ -135,6 +137,15 @@ extern "C" distdl_status_t distdl_partition_create_general(int32_t rank, const i
     return create_impl(rank, global_shape, partition_shape, halo_lo ? halo_lo : none, halo_hi ? halo_hi : none,
                        nullptr, nullptr, dtype, out);
 }
+
+namespace distdl {
+// Geometry and halo plans only, no device memory (used by the entry point that must not allocate).
+distdl_status_t partition_create_host_only(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
+                                           const int32_t *halo_lo, const int32_t *halo_hi, distdl_dtype_t dtype,
+                                           distdl_partition_t **out) {
+    return create_impl(rank, global_shape, partition_shape, nullptr, nullptr, halo_lo, halo_hi, dtype, out, false);
+}
+}  // namespace distdl
 
 extern "C" void distdl_partition_destroy(distdl_partition_t *p) {
     if (!p) return;
