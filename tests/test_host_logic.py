@@ -1,0 +1,138 @@
+"""CPU tests of the host side of the library: the shared object loads and exports every symbol the
+header declares, the planner's geometry and byte counts, and the error codes of the validation paths.
+No kernel is launched here."""
+
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2006_03108_b200 as distdl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "distdl.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(distdl_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(distdl.LIB_PATH)
+    names = _declared_symbols()
+    assert len(names) >= 19
+    for n in names:
+        assert hasattr(lib, n), "libdistdl.so does not export %s" % n
+
+
+APPENDIX_B = [
+    # n, p, kernel, stride, pad -> halo_lo, halo_hi, unused_lo, unused_hi   (Figs. B1-B4)
+    ((11, 3, 5, 1, 2), ([2, 2, 2], [2, 2, 2], [0, 0, 0], [0, 0, 0])),
+    ((11, 3, 5, 1, 0), ([0, 1, 3], [3, 1, 0], [0, 0, 0], [0, 0, 0])),
+    ((10, 3, 2, 2, 0), ([0, 0, 0], [0, 1, 0], [0, 0, 1], [0, 0, 0])),
+    ((20, 6, 2, 2, 0), ([0] * 6, [0, 0, 1, 2, 1, 0], [0, 0, 0, 1, 2, 1], [0] * 6)),
+]
+
+
+@pytest.mark.parametrize("args,expect", APPENDIX_B)
+def test_halo_widths_match_appendix_b_and_the_oracle(args, expect):
+    n, p, k, s, pad = args
+    got = distdl.halo_widths_1d(n, p, k, stride=s, pad_lo=pad, pad_hi=pad)
+    assert tuple(got) == expect
+    ref = oracle.halo_widths_1d(n, p, k, s, 1, pad, pad)
+    assert list(got[0]) == [r["halo_lo"] for r in ref] and list(got[1]) == [r["halo_hi"] for r in ref]
+    assert list(got[2]) == [r["unused_lo"] for r in ref] and list(got[3]) == [r["unused_hi"] for r in ref]
+
+
+@pytest.mark.parametrize("n,p,k,s,d,pl,ph", [(37, 5, 3, 2, 2, 1, 0), (64, 7, 4, 3, 1, 2, 2), (9, 9, 3, 1, 1, 1, 1), (50, 4, 7, 1, 3, 0, 5)])
+def test_halo_widths_random_cases_against_the_oracle(n, p, k, s, d, pl, ph):
+    got = distdl.halo_widths_1d(n, p, k, stride=s, dilation=d, pad_lo=pl, pad_hi=ph)
+    ref = oracle.halo_widths_1d(n, p, k, s, d, pl, ph)
+    for i, key in enumerate(["halo_lo", "halo_hi", "unused_lo", "unused_hi"]):
+        assert list(got[i]) == [r[key] for r in ref]
+
+
+def test_shard_extents_match_the_oracle_partition():
+    cases = [((11,), (3,), [2], [2]), ((67, 61, 68), (3, 2, 2), [2, 4, 4], [3, 4, 4]),
+             ((9, 8), (2, 2), [[0, 4], [0, 3]], [[2, 0], [0, 0]])]
+    for gs, ps, lo, hi in cases:
+        g = distdl.Partition(gs, ps, lo, hi)
+        o = oracle.Partition(gs, ps, lo, hi)
+        assert g.num_workers == o.num_workers
+        for w in range(o.num_workers):
+            st, bulk, padded, hl, hh = g.shard_extents(w)
+            assert st == o.bulk_start(w) and bulk == o.bulk_shape(w) and padded == o.padded_shape(w)
+            assert (hl, hh) == o.widths(w)
+
+
+def test_plan_bytes_of_the_baseline_configurations():
+    # 2-D: 4 shards of 130^2, width 1.  3-D: 64 shards of 136^3, width 4.
+    p1 = distdl.Partition((256, 256), (2, 2), (1, 1), (1, 1))
+    assert p1.halo_stats(False) == (32, 32, 12368)
+    assert p1.halo_stats(True)[2] == 20528
+    p3 = distdl.Partition((512,) * 3, (4,) * 3, (4,) * 3, (4,) * 3)
+    boxes, tiles, nbytes = p3.halo_stats(False)
+    assert boxes == 64 * 26 and nbytes == 186177536
+    assert p3.halo_stats(True)[2] == 330205184
+    # independent count: ghost cells written + interior ghost cells read (fp32)
+    ghost = 64 * (136 ** 3 - 128 ** 3)
+    interior = sum(np.prod([min(s + 132, 512) - max(s - 4, 0) for s in (a, b, c)]) - 128 ** 3
+                   for a in range(0, 512, 128) for b in range(0, 512, 128) for c in range(0, 512, 128))
+    assert nbytes == 4 * (ghost + int(interior))
+
+
+def _status(fn, *a, **k):
+    with pytest.raises(distdl.DistdlError) as e:
+        fn(*a, **k)
+    return e.value.status
+
+
+def test_partition_validation_errors():
+    assert _status(distdl.Partition, (4, 4), (8, 1)) == 2                       # fewer cells than workers
+    assert _status(distdl.Partition, (8, 8), (4, 1), (3, 0), (0, 0)) == 2        # ghost wider than the neighbour
+    assert _status(distdl.Partition, (8,) * 6, (1,) * 6) == 1                    # rank > 5
+    assert _status(distdl.Partition, (1024, 1024), (32, 32)) == 4                # > 256 workers
+    assert _status(distdl.Partition, (8, 8), (2, 2), (-1, 0), (0, 0)) == 2
+    assert _status(distdl.halo_widths_1d, 4, 2, 9) == 2                          # kernel larger than the input
+
+
+class _FakeTensor:
+    """Stands in for a device tensor: only the address and the size are looked at before launch."""
+
+    def __init__(self, addr, numel=16):
+        self._addr, self._n = addr, numel
+        import torch
+        self.dtype = torch.float32
+
+    def data_ptr(self):
+        return self._addr
+
+    def numel(self):
+        return self._n
+
+
+def test_operator_argument_validation_without_a_device():
+    ok, odd = _FakeTensor(0x10000), _FakeTensor(0x10004)
+    assert _status(distdl.broadcast_fwd, odd, [ok], stream=0) == 3               # alignment
+    assert _status(distdl.broadcast_fwd, ok, [odd], stream=0) == 3
+    assert _status(distdl.sumreduce_fwd, [ok, _FakeTensor(0)], ok, stream=0) == 1  # NULL source
+    assert _status(distdl.sumreduce_fwd, [_FakeTensor(0x20000), ok], ok, stream=0) == 1  # dst aliases source 1
+    part = distdl.Partition((8, 8), (2, 2), (1, 1), (1, 1))
+    import torch
+    if not torch.cuda.is_available():
+        # created without a device: geometry works, operators refuse
+        assert _status(distdl.halo_fwd, part, [ok] * 4, stream=0) == 5
+    lib = distdl.lib()
+    vp = ctypes.c_void_p
+    arr = (vp * 4)(0x10000, 0x20000, 0x30000, 0x40000)
+    assert lib.distdl_affine_fwd(16, 100, 128, 1, 1, arr, arr, None, arr, None) == 4   # block not a multiple of 128
+    assert lib.distdl_affine_fwd(16, 256, 256, 3, 1, arr, arr, None, arr, None) == 2   # not divisible by the grid
+    assert lib.distdl_conv_fwd(part.handle, arr, vp(0x50000), None, 3, 3, arr, None) == 2  # not a rank-4 partition
+    p4 = distdl.Partition((1, 2, 16, 16), (1, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2))
+    assert lib.distdl_conv_fwd(p4.handle, arr, vp(0x50000), None, 3, 3, arr, None) == 2    # widths do not match 3x3
+    assert lib.distdl_conv_fwd(p4.handle, arr, vp(0x50000), None, 4, 4, arr, None) == 4    # even kernel
+    assert lib.distdl_last_error().decode() != ""
