@@ -28,14 +28,8 @@ namespace distdl {
 constexpr int kTileM = 128;
 constexpr int kTileN = 128;
 constexpr int kBlockK = 64;                 // 64 bf16 = one 128-byte swizzle row
-constexpr int kStages = 6;
-constexpr int kStageABytes = kTileM * kBlockK * 2;   // 16 KB
-constexpr int kStageBBytes = kTileN * kBlockK * 2;   // 16 KB
-constexpr int kStageBytes = kStageABytes + kStageBBytes;
 constexpr int kAffineThreads = 192;         // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
 constexpr int kMaxMaps = 24;                // tensor maps passed as kernel parameters
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 
 __device__ int g_affine_status = 0;         // 0 = ok, otherwise DISTDL_ERR_TIMEOUT
 
@@ -55,17 +49,24 @@ struct AffineParams {
 // ------------------------------------------------------------------------------------------
 // PTX wrappers
 // ------------------------------------------------------------------------------------------
-// Bounded wait: false if the limit ran out or another role already gave up.
+// Bounded wait: false if the limit ran out or another role already gave up.  The limit is counted
+// in SM clock cycles (reading %globaltimer costs several hundred nanoseconds, which would serialise
+// the pipeline when it sits on the critical path of every k-block), and the clock is only looked
+// at once in a while.
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer();
-    while (true) {
+    long long t0 = 0;
+    for (unsigned spins = 0;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_timer() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            atomicExch(&g_affine_status, (int)DISTDL_ERR_TIMEOUT);
-            return false;
+        if ((spins & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicExch(&g_affine_status, (int)DISTDL_ERR_TIMEOUT);
+                return false;
+            }
         }
     }
 }
@@ -103,27 +104,86 @@ __host__ __device__ constexpr uint32_t instr_desc(int m, int n, int b_mn_major) 
 }
 
 // ------------------------------------------------------------------------------------------
-// Kernel: grid.x = output tiles along the feature axis * row tiles (row tile fastest, so the
-// blocks that share a weight tile run together and the tile comes from DRAM once).
+// Cluster helpers for the two-SM variant
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t bar_cluster_addr) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tcgen05_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;   // both blocks of the pair
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel.  PAIR = false: one thread block owns a 128 x 128 output tile (used when the batch fits
+// one 128-row tile).  PAIR = true: a cluster of two blocks owns a 256 x 128 tile; each block stages
+// its own 128 activation rows and its own half of the weight tile, one tcgen05.mma.cta_group::2
+// issued by the leader drives the tensor cores of both SMs and reads the weight halves from both
+// shared memories -- a quarter less shared-memory fill per flop, which buys a deeper ring.  The
+// leader's "full" barrier counts the bytes of both blocks' bulk copies; "empty" and "accumulator
+// ready" are signalled in both blocks at once by a multicast commit.
+//
+// The producer and the MMA issuer are single threads, so their loops are kept to a few dozen
+// instructions per k-block: counters advance incrementally (no divisions) and the shared-memory
+// descriptors are a precomputed base plus an offset.
+// Tiles are numbered row tile fastest, so blocks that share a weight tile run together.
+// ------------------------------------------------------------------------------------------
+template <bool PAIR>
+struct AffineCfg {
+    static constexpr int STAGES = PAIR ? 9 : 6;
+    static constexpr int A_BYTES = kTileM * kBlockK * 2;                       // 16 KB
+    static constexpr int B_BYTES = (PAIR ? kTileN / 2 : kTileN) * kBlockK * 2; // 8 or 16 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment*/ + 256 /*barriers*/;
+};
+
+template <bool PAIR>
 __global__ void __launch_bounds__(kAffineThreads, 1)
 affine_kernel(const __grid_constant__ AffineParams P) {
+    using C = AffineCfg<PAIR>;
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128-byte swizzle pattern is a function of address bits [7,10)
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *aligned = smem_raw + (base - raw);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kStages * kStageBytes);
-    const uint32_t bar_full = smem_u32(bars);                  // kStages barriers
-    const uint32_t bar_empty = bar_full + 8 * kStages;         // kStages barriers
-    const uint32_t bar_acc = bar_empty + 8 * kStages;          // accumulator complete
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 1);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + C::STAGES * C::STAGE_BYTES);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * C::STAGES;
+    const uint32_t bar_acc = bar_empty + 8 * C::STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * C::STAGES + 1);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row_tiles = (P.nb + kTileM - 1) / kTileM;
-    const int m0 = (blockIdx.x % row_tiles) * kTileM;
-    const int ntile = blockIdx.x / row_tiles;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0;         // 0 = leader of the pair
+    const int rows_per_tile = PAIR ? 2 * kTileM : kTileM;
+    const int tile = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int row_tiles = (P.nb + rows_per_tile - 1) / rows_per_tile;
+    const int m0 = (tile % row_tiles) * rows_per_tile + (int)rank * kTileM;   // this block's first row
+    const int ntile = tile / row_tiles;
     const int tiles_per_block = P.blk_out / kTileN;
     const int oblk = ntile / tiles_per_block;                  // output block (i forward, j adjoint)
     const int n0 = (ntile % tiles_per_block) * kTileN;         // first output column inside the block
@@ -131,83 +191,125 @@ affine_kernel(const __grid_constant__ AffineParams P) {
     const int num_kblocks = P.nred * kblocks_per_worker;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);      // the (leader's) producer arrives once, with the byte count
+            mbar_init(bar_empty + 8 * s, 1);     // one commit per use
         }
         mbar_init(bar_acc, 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        // 128 columns of tensor memory: one fp32 accumulator of 128 lanes x 128 columns
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        // 128 columns of tensor memory: one fp32 accumulator of 128 lanes x 128 columns per block
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tcgen05_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();    // both blocks' barriers exist before anyone signals them
+    else __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_acc = *tmem_slot;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            int issued = 0;
+            const CUtensorMap *amap = &P.a_map[0];
+            // forward: W_{oblk, r}, next worker = next map; adjoint: W_{r, oblk}, next worker = next grid row
+            const CUtensorMap *wmap = P.adjoint ? &P.w_map[oblk] : &P.w_map[oblk * P.pfi];
+            const int wstep = P.adjoint ? P.pfi : 1;
+            const int nb0 = n0 + (PAIR ? (int)rank * (kTileN / 2) : 0);   // this block's part of the weight tile
+            uint32_t s = 0, phase = 0, sa = base;
+            int k0 = 0, kin = 0;
             for (int kb = 0; kb < num_kblocks; ++kb) {
-                const int s = kb % kStages;
-                const uint32_t phase = (kb / kStages) & 1;
                 if (!mbar_wait(bar_empty + 8 * s, phase ^ 1, abort_flag)) break;
-                const int r = kb / kblocks_per_worker;          // worker along the reduction
-                const int k0 = (kb % kblocks_per_worker) * kBlockK;
-                const uint32_t sa = base + s * kStageBytes, sb = sa + kStageABytes;
-                mbar_expect_tx(bar_full + 8 * s, kStageBytes);
-                // activations: box {64 k, 128 rows} of block r at (k0, m0)
-                tma_load_2d(sa, &P.a_map[r], k0, m0, bar_full + 8 * s);
-                if (!P.adjoint) {
-                    // W_{oblk, r}: rows = output features, K-major: box {64 k, 128 rows} at (k0, n0)
-                    tma_load_2d(sb, &P.w_map[oblk * P.pfi + r], k0, n0, bar_full + 8 * s);
+                const uint32_t full = bar_full + 8 * s;
+                if (PAIR) {
+                    const uint32_t full_leader = map_to_cta(full, 0);
+                    if (rank == 0) mbar_expect_tx(full, 2 * C::STAGE_BYTES);      // both blocks' bytes
+                    tma_load_2d_pair(sa, amap, k0, m0, full_leader);
+                    if (!P.adjoint) tma_load_2d_pair(sa + C::A_BYTES, wmap, k0, nb0, full_leader);   // box {64 k, 64 rows}
+                    else tma_load_2d_pair(sa + C::A_BYTES, wmap, nb0, k0, full_leader);              // box {64 n, 64 k}
                 } else {
-                    // W_{r, oblk}: rows = reduction index, MN-major: two boxes {64 n, 64 k}
-                    const CUtensorMap *wm = &P.w_map[r * P.pfi + oblk];
-                    tma_load_2d(sb, wm, n0, k0, bar_full + 8 * s);
-                    tma_load_2d(sb + kStageBBytes / 2, wm, n0 + 64, k0, bar_full + 8 * s);
+                    mbar_expect_tx(full, C::STAGE_BYTES);
+                    tma_load_2d(sa, amap, k0, m0, full);                        // box {64 k, 128 rows}
+                    if (!P.adjoint) {
+                        tma_load_2d(sa + C::A_BYTES, wmap, k0, nb0, full);      // K-major: box {64 k, 128 rows}
+                    } else {                                                    // MN-major: two boxes {64 n, 64 k}
+                        tma_load_2d(sa + C::A_BYTES, wmap, nb0, k0, full);
+                        tma_load_2d(sa + C::A_BYTES + C::B_BYTES / 2, wmap, nb0 + 64, k0, full);
+                    }
                 }
-                ++issued;
+                k0 += kBlockK;
+                if (++kin == kblocks_per_worker) {      // next worker of the grid row / column, in order
+                    kin = 0;
+                    k0 = 0;
+                    ++amap;
+                    wmap += wstep;
+                }
+                sa += C::STAGE_BYTES;
+                if (++s == C::STAGES) {
+                    s = 0;
+                    sa = base;
+                    phase ^= 1;
+                }
             }
             if (*abort_flag) {
                 // give copies that are still in flight time to land before the block retires
                 const uint64_t t0 = global_timer();
                 while (global_timer() - t0 < 1000000ull) {}
             }
-            (void)issued;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc(kTileM, kTileN, P.adjoint ? 1 : 0);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc(PAIR ? 2 * kTileM : kTileM, kTileN, P.adjoint ? 1 : 0);
+            // A, K-major: 8-row groups 1024 bytes apart; a K step of 16 elements is 32 bytes.
+            // B forward, K-major: the same.  B adjoint, MN-major: 64-column atoms B_BYTES/2 apart
+            // (leading offset; one atom per block in the pair variant), 8-k groups 1024 bytes apart; a
+            // K step of 16 rows is 2048 bytes.  Descriptor addresses are in 16-byte units.
+            const uint64_t a0 = smem_desc(base, 16, 1024);
+            const uint64_t b0 = P.adjoint ? smem_desc(base + C::A_BYTES, PAIR ? C::B_BYTES : C::B_BYTES / 2, 1024)
+                                          : smem_desc(base + C::A_BYTES, 16, 1024);
+            const uint64_t bstep = P.adjoint ? (2048 >> 4) : (32 >> 4);
+            uint32_t s = 0, phase = 0;
+            uint64_t off = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kblocks && ok; ++kb) {
-                const int s = kb % kStages;
-                const uint32_t phase = (kb / kStages) & 1;
+            for (int kb = 0; kb < num_kblocks; ++kb) {
                 ok = mbar_wait(bar_full + 8 * s, phase, abort_flag);
                 if (!ok) break;
                 tcgen05_fence_after();
-                const uint32_t sa = base + s * kStageBytes, sb = sa + kStageABytes;
-#pragma unroll
-                for (int k = 0; k < kBlockK / 16; ++k) {
-                    // A, K-major: 8-row groups 1024 bytes apart; step 32 bytes along K
-                    const uint64_t adesc = smem_desc(sa + k * 32, 16, 1024);
-                    uint64_t bdesc;
-                    if (!P.adjoint) bdesc = smem_desc(sb + k * 32, 16, 1024);
-                    // B, MN-major: 64-column atoms 8192 bytes apart (leading), 8-k groups 1024
-                    // bytes apart (stride); step 16 k-rows = 2048 bytes
-                    else bdesc = smem_desc(sb + k * 2048, kStageBBytes / 2, 1024);
-                    umma_bf16(tmem_acc, adesc, bdesc, idesc, (kb | k) ? 1u : 0u);
+                const uint64_t a = a0 + off, b = b0 + off;
+                if (PAIR) {
+                    umma_bf16_pair(tmem_acc, a, b, idesc, kb ? 1u : 0u);
+                    umma_bf16_pair(tmem_acc, a + 2, b + bstep, idesc, 1u);
+                    umma_bf16_pair(tmem_acc, a + 4, b + 2 * bstep, idesc, 1u);
+                    umma_bf16_pair(tmem_acc, a + 6, b + 3 * bstep, idesc, 1u);
+                    tcgen05_commit_pair(bar_empty + 8 * s);     // frees the stage in both blocks
+                } else {
+                    umma_bf16(tmem_acc, a, b, idesc, kb ? 1u : 0u);
+                    umma_bf16(tmem_acc, a + 2, b + bstep, idesc, 1u);
+                    umma_bf16(tmem_acc, a + 4, b + 2 * bstep, idesc, 1u);
+                    umma_bf16(tmem_acc, a + 6, b + 3 * bstep, idesc, 1u);
+                    tcgen05_commit(bar_empty + 8 * s);          // frees the stage once these MMAs retire
                 }
-                tcgen05_commit(bar_empty + 8 * s);     // frees the stage once these MMAs retire
+                off += C::STAGE_BYTES >> 4;
+                if (++s == C::STAGES) {
+                    s = 0;
+                    off = 0;
+                    phase ^= 1;
+                }
             }
-            if (ok) tcgen05_commit(bar_acc);           // accumulator complete
+            if (ok) {                                           // accumulator complete
+                if (PAIR) tcgen05_commit_pair(bar_acc);
+                else tcgen05_commit(bar_acc);
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -251,11 +353,17 @@ affine_kernel(const __grid_constant__ AffineParams P) {
             }
         }
     }
+    // a block may not retire, or free its tensor memory, while its peer can still read its shared
+    // memory or signal its barriers
     tcgen05_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();
+    else __syncthreads();
     if (warp == 1) {
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kTileN) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kTileN) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kTileN) : "memory");
     }
 }
 
@@ -313,11 +421,14 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
     for (int i = 0; i < nact; ++i)
         if (!make_map(&P.a_map[i], act[i], nb, act_cols, kBlockK, kTileM))
             return fail(DISTDL_ERR_CUDA, "%s: tensor map of activation block %d failed", what, i);
+    // more than one 128-row tile of the batch: a pair of blocks shares each 256 x 128 output tile
+    const bool pair = nb > kTileM;
     for (int i = 0; i < pfo * pfi; ++i) {
-        // forward: box {64 along in-features (K), 128 out-feature rows}; adjoint: box {64 along
-        // in-features (N), 64 out-feature rows (K)} of the same row-major [bfo, bfi] block
+        // forward: box {64 along in-features (K), 128 out-feature rows} (64 rows per block of a pair);
+        // adjoint: box {64 along in-features (N), 64 out-feature rows (K)} of the same row-major
+        // [bfo, bfi] block
         const bool ok = adjoint ? make_map(&P.w_map[i], w[i], bfo, bfi, 64, kBlockK)
-                                : make_map(&P.w_map[i], w[i], bfo, bfi, kBlockK, kTileN);
+                                : make_map(&P.w_map[i], w[i], bfo, bfi, kBlockK, pair ? kTileN / 2 : kTileN);
         if (!ok) return fail(DISTDL_ERR_CUDA, "%s: tensor map of weight block %d failed", what, i);
     }
     for (int i = 0; i < nout; ++i) {
@@ -334,12 +445,34 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
 
     static bool configured = false;
     if (!configured) {
-        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               AffineCfg<false>::SMEM_BYTES));
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               AffineCfg<true>::SMEM_BYTES));
         configured = true;
     }
-    const int64_t row_tiles = (nb + kTileM - 1) / kTileM;
     const int64_t ntiles = (adjoint ? nfi : nfo) / kTileN;
-    affine_kernel<<<(unsigned)(row_tiles * ntiles), kAffineThreads, kSmemBytes, (cudaStream_t)stream>>>(P);
+    if (pair) {
+        const int64_t row_pairs = (nb + 2 * kTileM - 1) / (2 * kTileM);
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)(2 * row_pairs * ntiles));
+        cfg.blockDim = dim3(kAffineThreads);
+        cfg.dynamicSmemBytes = AffineCfg<true>::SMEM_BYTES;
+        cfg.stream = (cudaStream_t)stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        DISTDL_CUDA_CHECK(cudaLaunchKernelEx(&cfg, affine_kernel<true>, P));
+    } else {
+        const int64_t row_tiles = (nb + kTileM - 1) / kTileM;
+        affine_kernel<false><<<(unsigned)(row_tiles * ntiles), kAffineThreads, AffineCfg<false>::SMEM_BYTES,
+                               (cudaStream_t)stream>>>(P);
+    }
     DISTDL_CUDA_CHECK(cudaGetLastError());
     return DISTDL_OK;
 }
