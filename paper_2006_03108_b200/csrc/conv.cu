@@ -187,19 +187,19 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
 
 // Register-tiled stencil of one staged tile: each thread produces 8 rows x 4 columns, two columns
 // per packed FMA.
+// wk: the K*K weights of this tile's channel followed by its bias (global or shared memory).
 template <int K, bool ADJ>
-__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile) {
+__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile, const float *wk) {
     using C = ConvCfg<K, ADJ>;
     if (!t.valid) return;
-    const int ch = t.plane % P.channels;
     // weights as broadcast pairs (w, w); adjoint: kernel rotated by 180 degrees
     uint64_t w2[K * K];
 #pragma unroll
     for (int q = 0; q < K * K; ++q) {
-        const float w = __ldg(P.w + (size_t)ch * K * K + (ADJ ? K * K - 1 - q : q));
+        const float w = wk[ADJ ? K * K - 1 - q : q];
         w2[q] = pack2(w, w);
     }
-    const float b0 = (!ADJ && P.bias) ? __ldg(P.bias + ch) : 0.f;
+    const float b0 = ADJ ? 0.f : wk[K * K];
 
     if (ADJ) {
         // clear the part of the ghost ring of dx that borders this tile
@@ -283,6 +283,7 @@ __global__ void __launch_bounds__(kConvThreads, 2)
 conv_depthwise_kernel(const __grid_constant__ ConvParams P, int total_tiles, int tiles_y, int planes) {
     using C = ConvCfg<K, ADJ>;
     extern __shared__ __align__(16) float smem[];   // two tile buffers
+    __shared__ float wk[K * K + 1];
     int buf = 0;
     int tile = blockIdx.x;
     if (tile >= total_tiles) return;
@@ -299,8 +300,13 @@ conv_depthwise_kernel(const __grid_constant__ ConvParams P, int total_tiles, int
         }
         cp_async_commit();
         cp_async_wait_group<1>();          // everything but the newest group: the current tile is here
+        if (cur.valid && threadIdx.x <= K * K) {
+            const int ch = cur.plane % P.channels;
+            wk[threadIdx.x] = threadIdx.x < K * K ? __ldg(P.w + (size_t)ch * K * K + threadIdx.x)
+                                                  : (P.bias ? __ldg(P.bias + ch) : 0.f);
+        }
         __syncthreads();
-        compute_tile<K, ADJ>(P, cur, smem + buf * C::TILE_FLOATS);
+        compute_tile<K, ADJ>(P, cur, smem + buf * C::TILE_FLOATS, wk);
         __syncthreads();                   // the buffer may be refilled from now on
         if (!has_next) break;
         cur = nxt;
@@ -335,57 +341,48 @@ struct ConvTmaCfg {
     static constexpr int SIDE = 2 * C::PH * C::PITCH + 2 * C::PH * C::ROWS;         // patch cells, upper bound
     static constexpr int SIDE_STRIDE = ((SIDE + 31) / 32) * 32;
     static constexpr int BOX_BYTES = C::PITCH * C::ROWS * 4;
-    static constexpr int SMEM_BYTES = 2 * TILE_STRIDE * 4 + 2 * SIDE_STRIDE * 4 + 64 + 128;
+    static constexpr int WK_STRIDE = 64;                                            // K*K weights + bias, per buffer
+    static constexpr int SMEM_BYTES = 2 * TILE_STRIDE * 4 + 2 * SIDE_STRIDE * 4 + 2 * WK_STRIDE * 4 + 64 + 128;
 };
 
-// The halo strips of a tile: top / bottom rows and left / right columns that lie outside the
-// shard's own bulk.  Cell q of the list maps to tile coordinates (ry, s).
-struct PatchList {
-    int nT, nB, nL, nR, W, rowB, colL, colR, total;
-};
-
-template <int K, bool ADJ>
-__device__ __forceinline__ PatchList make_patch_list(const ConvTile &t) {
+// The halo strips of a tile -- top / bottom rows and left / right columns that lie outside the
+// shard's own bulk -- are enumerated by every thread the same way at staging and at patching
+// time: f(q, ry, s) gets the cell's slot q in the side buffer and its tile coordinates.
+template <int K, bool ADJ, typename F>
+__device__ __forceinline__ void for_each_patch_cell(const ConvTile &t, F f) {
     using C = ConvCfg<K, ADJ>;
-    PatchList p;
     const int out_rows = min(kTileH, t.bh - t.i0), out_cols = min(kTileW, t.bw - t.j0);
-    p.W = out_cols + 2 * C::PH;                     // columns a strip spans, starting at colL
-    const int H = out_rows + 2 * C::PH;
-    p.colL = C::PADL - C::PH;
-    p.colR = C::PADL + out_cols;
-    p.rowB = C::PH + out_rows;
-    p.nT = (t.i0 == 0) ? C::PH * p.W : 0;
-    p.nB = (t.i0 + out_rows == t.bh) ? C::PH * p.W : 0;
-    p.nL = (t.j0 == 0) ? C::PH * H : 0;
-    p.nR = (t.j0 + out_cols == t.bw) ? C::PH * H : 0;
-    p.total = p.nT + p.nB + p.nL + p.nR;
-    return p;
-}
-
-template <int K, bool ADJ>
-__device__ __forceinline__ void patch_cell(const PatchList &p, int q, int &ry, int &s) {
-    constexpr int PH = ConvCfg<K, ADJ>::PH;
-    if (q < p.nT) {
-        ry = q / p.W;
-        s = p.colL + q % p.W;
-    } else if (q < p.nT + p.nB) {
-        q -= p.nT;
-        ry = p.rowB + q / p.W;
-        s = p.colL + q % p.W;
-    } else if (q < p.nT + p.nB + p.nL) {
-        q -= p.nT + p.nB;
-        ry = q / PH;
-        s = p.colL + q % PH;
-    } else {
-        q -= p.nT + p.nB + p.nL;
-        ry = q / PH;
-        s = p.colR + q % PH;
+    const int W = out_cols + 2 * C::PH, H = out_rows + 2 * C::PH;
+    const int colL = C::PADL - C::PH, colR = C::PADL + out_cols, rowB = C::PH + out_rows;
+    int q0 = 0;
+    if (t.i0 == 0) {
+#pragma unroll
+        for (int r = 0; r < C::PH; ++r)
+            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, r, colL + s);
+        q0 += C::PH * W;
+    }
+    if (t.i0 + out_rows == t.bh) {
+#pragma unroll
+        for (int r = 0; r < C::PH; ++r)
+            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, rowB + r, colL + s);
+        q0 += C::PH * W;
+    }
+    if (t.j0 == 0) {
+        for (int ry = threadIdx.x; ry < H; ry += kConvThreads)
+#pragma unroll
+            for (int c = 0; c < C::PH; ++c) f(q0 + ry * C::PH + c, ry, colL + c);
+        q0 += C::PH * H;
+    }
+    if (t.j0 + out_cols == t.bw) {
+        for (int ry = threadIdx.x; ry < H; ry += kConvThreads)
+#pragma unroll
+            for (int c = 0; c < C::PH; ++c) f(q0 + ry * C::PH + c, ry, colR + c);
     }
 }
 
 template <int K, bool ADJ>
 __device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const ConvTile &t, float *tile, float *side,
-                                               uint32_t bar) {
+                                               float *wk, uint32_t bar) {
     using C = ConvCfg<K, ADJ>;
     using T = ConvTmaCfg<K, ADJ>;
     const ConvParams &P = Q.base;
@@ -398,10 +395,14 @@ __device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const Con
         const int y = ADJ ? t.i0 - C::PH : t.i0;
         tma_load_3d(smem_u32(tile), &Q.in_map[t.shard], x, y, t.plane, bar);
     }
-    const PatchList pl = make_patch_list<K, ADJ>(t);
-    for (int q = threadIdx.x; q < pl.total; q += kConvThreads) {
-        int ry, s;
-        patch_cell<K, ADJ>(pl, q, ry, s);
+    // this channel's weights and bias
+    if (threadIdx.x <= K * K) {
+        const int ch = t.plane % P.channels;
+        if (threadIdx.x < K * K) cp_async4(wk + threadIdx.x, P.w + (size_t)ch * K * K + threadIdx.x);
+        else if (P.bias) cp_async4(wk + K * K, P.bias + ch);
+        else wk[K * K] = 0.f;
+    }
+    for_each_patch_cell<K, ADJ>(t, [&](int q, int ry, int s) {
         int i = t.i0 - C::PH + ry, rr = t.r;
         bool ok = true;
         if (i < 0) {
@@ -435,7 +436,7 @@ __device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const Con
         } else {
             side[q] = 0.f;
         }
-    }
+    });
 }
 
 template <int K, bool ADJ>
@@ -447,7 +448,8 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
     const uint32_t raw = smem_u32(smem_raw);
     float *tiles = reinterpret_cast<float *>(smem_raw + (((raw + 127u) & ~127u) - raw));
     float *sides = tiles + 2 * T::TILE_STRIDE;
-    const uint32_t bars = smem_u32(sides + 2 * T::SIDE_STRIDE);
+    float *wks = sides + 2 * T::SIDE_STRIDE;
+    const uint32_t bars = smem_u32(wks + 2 * T::WK_STRIDE);
     if (threadIdx.x == 0) {
         mbar_init(bars, 1);
         mbar_init(bars + 8, 1);
@@ -460,7 +462,7 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
     int buf = 0;
     uint32_t phase0 = 0, phase1 = 0;          // parity of the next completion of each buffer's barrier
     ConvTile cur = decode_tile(Q.base, tile, Q.tiles_y, Q.planes);
-    stage_tile_tma<K, ADJ>(Q, cur, tiles, sides, bars);
+    stage_tile_tma<K, ADJ>(Q, cur, tiles, sides, wks, bars);
     cp_async_commit();
     while (true) {
         const int next = tile + gridDim.x;
@@ -469,7 +471,7 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
         if (has_next) {
             nxt = decode_tile(Q.base, next, Q.tiles_y, Q.planes);
             stage_tile_tma<K, ADJ>(Q, nxt, tiles + (buf ^ 1) * T::TILE_STRIDE, sides + (buf ^ 1) * T::SIDE_STRIDE,
-                                   bars + 8 * (buf ^ 1));
+                                   wks + (buf ^ 1) * T::WK_STRIDE, bars + 8 * (buf ^ 1));
         }
         cp_async_commit();
         cp_async_wait_group<1>();
@@ -499,15 +501,10 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
         float *tl = tiles + buf * T::TILE_STRIDE;
         if (cur.valid) {
             const float *sd = sides + buf * T::SIDE_STRIDE;
-            const PatchList pl = make_patch_list<K, ADJ>(cur);
-            for (int q = threadIdx.x; q < pl.total; q += kConvThreads) {
-                int ry, s;
-                patch_cell<K, ADJ>(pl, q, ry, s);
-                tl[ry * C::PITCH + s] = sd[q];
-            }
+            for_each_patch_cell<K, ADJ>(cur, [&](int q, int ry, int s) { tl[ry * C::PITCH + s] = sd[q]; });
         }
         __syncthreads();
-        compute_tile<K, ADJ>(Q.base, cur, tl);
+        compute_tile<K, ADJ>(Q.base, cur, tl, wks + buf * T::WK_STRIDE);
         __syncthreads();
         if (!has_next) break;
         cur = nxt;
