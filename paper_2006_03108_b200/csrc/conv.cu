@@ -15,10 +15,11 @@
 namespace distdl {
 
 constexpr int kConvMaxWorkers = 64;
-constexpr int kConvThreads = 256;
-constexpr int kTileH = 64;    // output rows per block
+constexpr int kConvThreads = 128;
+constexpr int kTileH = 32;    // output rows per block (8 thread rows x 4)
 constexpr int kTileW = 128;   // output columns per block
-constexpr int kRowsPerThread = 8;
+constexpr int kRowsPerThread = 4;   // each thread: 4 rows x 8 columns of outputs
+constexpr int kColsPerThread = 8;
 
 struct ConvParams {
     const float *in[kConvMaxWorkers];
@@ -33,14 +34,14 @@ struct ConvParams {
 };
 
 // Row pitch (floats) of the shared-memory tile: wide enough for the staged columns (outputs plus
-// PADL columns on the left and PH on the right, rounded up to whole float4s) and for the last
-// thread's float4 window.
+// PADL columns on the left and PH on the right, rounded up to whole float4s) and for the float4
+// window of the last thread across (8 outputs, K - 1 more inputs, WOFF floats of lead-in).
 __host__ __device__ constexpr int conv_pitch(int K, bool adj) {
     const int ph = K / 2;
     const int padl = adj ? ((ph + 3) / 4) * 4 : ph;
-    const int nv = (padl - ph + K + 3 + 3) / 4;
+    const int nf = ((padl - ph + kColsPerThread + K - 1 + 3) / 4) * 4;
     const int staged = ((kTileW + padl + ph + 3) / 4) * 4;
-    const int window = kTileW - 4 + 4 * nv;
+    const int window = kTileW - kColsPerThread + nf;
     return staged > window ? staged : window;
 }
 
@@ -107,7 +108,7 @@ struct ConvCfg {
     static constexpr int PH = K / 2;                                   // halo rows = halo columns
     static constexpr int PADL = ADJ ? ((PH + 3) / 4) * 4 : PH;         // tile columns left of the first output
     static constexpr int WOFF = PADL - PH;                             // first column a thread needs in its slot
-    static constexpr int NV = (WOFF + K + 3 + 3) / 4;                  // float4 loads per thread per input row
+    static constexpr int NF = ((WOFF + kColsPerThread + K - 1 + 3) / 4) * 4;   // floats a thread loads per input row
     static constexpr int PITCH = conv_pitch(K, ADJ);
     static constexpr int ROWS = kTileH + K - 1;
     static constexpr int IOFF = ADJ ? 0 : PH;                          // offset of the bulk in the input layout
@@ -185,21 +186,18 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
     }
 }
 
-// Register-tiled stencil of one staged tile: each thread produces 8 rows x 4 columns, two columns
-// per packed FMA.
-// wk: the K*K weights of this tile's channel followed by its bias (global or shared memory).
+// Register-tiled stencil of one staged tile: each thread produces 4 rows x 8 columns with packed
+// fp32 pair FMAs and no register shuffling.  A thread's input row arrives as aligned pairs
+// P[i] = (x[2i], x[2i+1]).  Taps whose first input index is even feed the output pairs (o0,o1),
+// (o2,o3), (o4,o5), (o6,o7) from P directly; taps whose first index is odd feed the shifted pairs
+// (o1,o2), (o3,o4), (o5,o6), again from aligned P, plus o0 and o7 as two scalar FMAs.  The two
+// sets of partial sums are added once at the end.
+// wk2: K*K weights as (w, w) pairs (already rotated for the adjoint), then the bias.
 template <int K, bool ADJ>
-__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile, const float *wk) {
+__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile, const float *wk2) {
     using C = ConvCfg<K, ADJ>;
     if (!t.valid) return;
-    // weights as broadcast pairs (w, w); adjoint: kernel rotated by 180 degrees
-    uint64_t w2[K * K];
-#pragma unroll
-    for (int q = 0; q < K * K; ++q) {
-        const float w = wk[ADJ ? K * K - 1 - q : q];
-        w2[q] = pack2(w, w);
-    }
-    const float b0 = ADJ ? 0.f : wk[K * K];
+    const float b0 = ADJ ? 0.f : wk2[2 * K * K];
 
     if (ADJ) {
         // clear the part of the ghost ring of dx that borders this tile
@@ -210,44 +208,69 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
         const int C0 = t.j0 == 0 ? 0 : t.j0 + C::PH, C1 = j1 == t.bw ? t.bw + 2 * C::PH : j1 + C::PH;
         const int ncol = C1 - C0;
         if (t.i0 == 0)
-            for (int q = threadIdx.x; q < C::PH * ncol; q += kConvThreads) oplane[(size_t)(q / ncol) * pitch_o + C0 + q % ncol] = 0.f;
+            for (int r = 0; r < C::PH; ++r)
+                for (int q = threadIdx.x; q < ncol; q += kConvThreads) oplane[(size_t)r * pitch_o + C0 + q] = 0.f;
         if (i1 == t.bh)
-            for (int q = threadIdx.x; q < C::PH * ncol; q += kConvThreads)
-                oplane[(size_t)(t.bh + C::PH + q / ncol) * pitch_o + C0 + q % ncol] = 0.f;
+            for (int r = 0; r < C::PH; ++r)
+                for (int q = threadIdx.x; q < ncol; q += kConvThreads) oplane[(size_t)(t.bh + C::PH + r) * pitch_o + C0 + q] = 0.f;
         const int Rb0 = max(R0, C::PH), Rb1 = min(R1, t.bh + C::PH);
         if (t.j0 == 0)
-            for (int q = threadIdx.x; q < (Rb1 - Rb0) * C::PH; q += kConvThreads) oplane[(size_t)(Rb0 + q / C::PH) * pitch_o + q % C::PH] = 0.f;
+            for (int q = threadIdx.x; q < Rb1 - Rb0; q += kConvThreads)
+#pragma unroll
+                for (int c = 0; c < C::PH; ++c) oplane[(size_t)(Rb0 + q) * pitch_o + c] = 0.f;
         if (j1 == t.bw)
-            for (int q = threadIdx.x; q < (Rb1 - Rb0) * C::PH; q += kConvThreads)
-                oplane[(size_t)(Rb0 + q / C::PH) * pitch_o + t.bw + C::PH + q % C::PH] = 0.f;
+            for (int q = threadIdx.x; q < Rb1 - Rb0; q += kConvThreads)
+#pragma unroll
+                for (int c = 0; c < C::PH; ++c) oplane[(size_t)(Rb0 + q) * pitch_o + t.bw + C::PH + c] = 0.f;
     }
 
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    uint64_t acc[kRowsPerThread][2];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    constexpr int NP = C::NF / 2;                      // aligned input pairs per row
+    uint64_t acc_e[kRowsPerThread][4];                 // (o0,o1) (o2,o3) (o4,o5) (o6,o7)
+    uint64_t acc_o[kRowsPerThread][3];                 // (o1,o2) (o3,o4) (o5,o6)
+    float acc_s[kRowsPerThread][2];                    // o0, o7 from the odd-aligned taps
 #pragma unroll
-    for (int a = 0; a < kRowsPerThread; ++a) acc[a][0] = acc[a][1] = pack2(b0, b0);
-
-    const float *trow = tile + (ty * kRowsPerThread) * C::PITCH + 4 * tx;
+    for (int r = 0; r < kRowsPerThread; ++r) {
 #pragma unroll
-    for (int ry = 0; ry < kRowsPerThread + K - 1; ++ry) {
-        float in[4 * C::NV];
+        for (int p2 = 0; p2 < 4; ++p2) acc_e[r][p2] = pack2(b0, b0);
 #pragma unroll
-        for (int v = 0; v < C::NV; ++v) {
-            const float4 q = *reinterpret_cast<const float4 *>(trow + ry * C::PITCH + 4 * v);
-            in[4 * v + 0] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
-        }
-        // pairs (in[s], in[s+1]) for every s a tap can start at
-        uint64_t pr[4 * C::NV - 1];
+        for (int p2 = 0; p2 < 3; ++p2) acc_o[r][p2] = 0ull;
+        acc_s[r][0] = acc_s[r][1] = 0.f;
+    }
+    const float *tbase = tile + (ty * kRowsPerThread) * C::PITCH + kColsPerThread * tx;
+    const uint64_t *wpairs = reinterpret_cast<const uint64_t *>(wk2);
 #pragma unroll
-        for (int s2 = 0; s2 < 4 * C::NV - 1; ++s2) pr[s2] = pack2(in[s2], in[s2 + 1]);
+    for (int a = 0; a < K; ++a) {
+        uint64_t wp[K];
 #pragma unroll
-        for (int a = 0; a < K; ++a) {
-            const int orow = ry - a;       // output row (within the thread's strip) fed by tap row a
-            if (orow >= 0 && orow < kRowsPerThread) {
+        for (int b = 0; b < K; ++b) wp[b] = wpairs[a * K + b];
 #pragma unroll
-                for (int b = 0; b < K; ++b) {
-                    acc[orow][0] = fma2(w2[a * K + b], pr[C::WOFF + b], acc[orow][0]);
-                    acc[orow][1] = fma2(w2[a * K + b], pr[C::WOFF + b + 2], acc[orow][1]);
+        for (int r = 0; r < kRowsPerThread; ++r) {
+            uint64_t Pr[NP];
+            const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(tbase + (r + a) * C::PITCH);
+#pragma unroll
+            for (int v = 0; v < NP / 2; ++v) {
+                const ulonglong2 q = src[v];
+                Pr[2 * v] = q.x;
+                Pr[2 * v + 1] = q.y;
+            }
+#pragma unroll
+            for (int b = 0; b < K; ++b) {
+                constexpr int dummy = 0;
+                (void)dummy;
+                const int j0 = C::WOFF + b;            // array index of the first input of output 0
+                if ((j0 & 1) == 0) {
+#pragma unroll
+                    for (int p2 = 0; p2 < 4; ++p2) acc_e[r][p2] = fma2(wp[b], Pr[j0 / 2 + p2], acc_e[r][p2]);
+                } else {
+#pragma unroll
+                    for (int p2 = 0; p2 < 3; ++p2) acc_o[r][p2] = fma2(wp[b], Pr[(j0 + 1) / 2 + p2], acc_o[r][p2]);
+                    float wlo, whi, xlo, xhi;
+                    unpack2(wp[b], wlo, whi);
+                    unpack2(Pr[(j0 - 1) / 2], xlo, xhi);              // x[j0] is the high half
+                    acc_s[r][0] = fmaf(wlo, xhi, acc_s[r][0]);
+                    unpack2(Pr[(j0 + 7) / 2], xlo, xhi);              // x[j0 + 7] is the low half
+                    acc_s[r][1] = fmaf(wlo, xlo, acc_s[r][1]);
                 }
             }
         }
@@ -255,35 +278,53 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
 
     const int pitch_o = t.bw + 2 * C::OOFF;
     float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::OOFF) * pitch_o;
-    const int jo = t.j0 + 4 * tx;
+    const int jo = t.j0 + kColsPerThread * tx;
 #pragma unroll
-    for (int a = 0; a < kRowsPerThread; ++a) {
-        const int io = t.i0 + ty * kRowsPerThread + a;
+    for (int r = 0; r < kRowsPerThread; ++r) {
+        const int io = t.i0 + ty * kRowsPerThread + r;
         if (io >= t.bh || jo >= t.bw) continue;
-        float o0, o1, o2, o3;
-        unpack2(acc[a][0], o0, o1);
-        unpack2(acc[a][1], o2, o3);
-        float *o = oplane + (size_t)(io + C::OOFF) * pitch_o + C::OOFF + jo;
-        if (jo + 3 < t.bw && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-            *reinterpret_cast<float4 *>(o) = make_float4(o0, o1, o2, o3);
-        } else if (jo + 3 < t.bw && (reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
-            *reinterpret_cast<float2 *>(o) = make_float2(o0, o1);
-            *reinterpret_cast<float2 *>(o + 2) = make_float2(o2, o3);
-        } else {
-            const float ov[4] = {o0, o1, o2, o3};
+        float e[8], o[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (jo + q < t.bw) o[q] = ov[q];
+        for (int p2 = 0; p2 < 4; ++p2) unpack2(acc_e[r][p2], e[2 * p2], e[2 * p2 + 1]);
+        o[0] = acc_s[r][0];
+        o[7] = acc_s[r][1];
+#pragma unroll
+        for (int p2 = 0; p2 < 3; ++p2) unpack2(acc_o[r][p2], o[2 * p2 + 1], o[2 * p2 + 2]);
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = e[q] + o[q];
+        float *dst = oplane + (size_t)(io + C::OOFF) * pitch_o + C::OOFF + jo;
+        if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+            *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4 *>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+        } else if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
+#pragma unroll
+            for (int q = 0; q < 8; q += 2) *reinterpret_cast<float2 *>(dst + q) = make_float2(v[q], v[q + 1]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (jo + q < t.bw) dst[q] = v[q];
         }
     }
 }
 
+// Fills the (w, w) pair table and the bias of one channel from raw weights (global or shared).
 template <int K, bool ADJ>
-__global__ void __launch_bounds__(kConvThreads, 2)
+__device__ __forceinline__ void fill_weight_pairs(float *wk2, const float *wraw, float bias) {
+    if (threadIdx.x < K * K) {
+        const float w = wraw[ADJ ? K * K - 1 - (int)threadIdx.x : (int)threadIdx.x];   // adjoint: rotated kernel
+        reinterpret_cast<float2 *>(wk2)[threadIdx.x] = make_float2(w, w);
+    } else if (threadIdx.x == K * K) {
+        wk2[2 * K * K] = bias;
+    }
+}
+
+template <int K, bool ADJ>
+__global__ void __launch_bounds__(kConvThreads, 4)
 conv_depthwise_kernel(const __grid_constant__ ConvParams P, int total_tiles, int tiles_y, int planes) {
     using C = ConvCfg<K, ADJ>;
     extern __shared__ __align__(16) float smem[];   // two tile buffers
-    __shared__ float wk[K * K + 1];
+    __shared__ __align__(16) float wk[2 * K * K + 2];
     int buf = 0;
     int tile = blockIdx.x;
     if (tile >= total_tiles) return;
@@ -300,10 +341,9 @@ conv_depthwise_kernel(const __grid_constant__ ConvParams P, int total_tiles, int
         }
         cp_async_commit();
         cp_async_wait_group<1>();          // everything but the newest group: the current tile is here
-        if (cur.valid && threadIdx.x <= K * K) {
+        if (cur.valid) {
             const int ch = cur.plane % P.channels;
-            wk[threadIdx.x] = threadIdx.x < K * K ? __ldg(P.w + (size_t)ch * K * K + threadIdx.x)
-                                                  : (P.bias ? __ldg(P.bias + ch) : 0.f);
+            fill_weight_pairs<K, ADJ>(wk, P.w + (size_t)ch * K * K, P.bias ? __ldg(P.bias + ch) : 0.f);
         }
         __syncthreads();
         compute_tile<K, ADJ>(P, cur, smem + buf * C::TILE_FLOATS, wk);
@@ -341,7 +381,7 @@ struct ConvTmaCfg {
     static constexpr int SIDE = 2 * C::PH * C::PITCH + 2 * C::PH * C::ROWS;         // patch cells, upper bound
     static constexpr int SIDE_STRIDE = ((SIDE + 31) / 32) * 32;
     static constexpr int BOX_BYTES = C::PITCH * C::ROWS * 4;
-    static constexpr int WK_STRIDE = 64;                                            // K*K weights + bias, per buffer
+    static constexpr int WK_STRIDE = 64 + 128;                                      // raw weights + bias, (w,w) pairs + bias
     static constexpr int SMEM_BYTES = 2 * TILE_STRIDE * 4 + 2 * SIDE_STRIDE * 4 + 2 * WK_STRIDE * 4 + 64 + 128;
 };
 
@@ -440,7 +480,7 @@ __device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const Con
 }
 
 template <int K, bool ADJ>
-__global__ void __launch_bounds__(kConvThreads, 2)
+__global__ void __launch_bounds__(kConvThreads, 4)
 conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
     using C = ConvCfg<K, ADJ>;
     using T = ConvTmaCfg<K, ADJ>;
@@ -499,12 +539,14 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
             break;
         }
         float *tl = tiles + buf * T::TILE_STRIDE;
+        float *wraw = wks + buf * T::WK_STRIDE;
         if (cur.valid) {
             const float *sd = sides + buf * T::SIDE_STRIDE;
             for_each_patch_cell<K, ADJ>(cur, [&](int q, int ry, int s) { tl[ry * C::PITCH + s] = sd[q]; });
+            fill_weight_pairs<K, ADJ>(wraw + 64, wraw, wraw[K * K]);
         }
         __syncthreads();
-        compute_tile<K, ADJ>(Q.base, cur, tl, wks + buf * T::WK_STRIDE);
+        compute_tile<K, ADJ>(Q.base, cur, tl, wraw + 64);
         __syncthreads();
         if (!has_next) break;
         cur = nxt;
