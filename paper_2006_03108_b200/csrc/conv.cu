@@ -79,17 +79,22 @@ struct ConvTile {
 };
 
 __device__ __forceinline__ ConvTile decode_tile(const ConvParams &P, int tile, int tiles_y, int planes) {
-    // tile id = ((shard * planes + plane) * tiles_x + tx) * tiles_y + ty : vertically adjacent tiles
-    // get adjacent ids, so the rows they share are still in L2 when the second one asks for them
+    // tile id = (((plane * Ph + r) * tiles_y + ty) * Pw + c) * tiles_x + tx : consecutive ids sweep
+    // one row of tiles of the global image from left to right across the worker columns, the next
+    // row of tiles follows.  Blocks that run together therefore work on neighbouring tiles, and the
+    // halo cells a tile takes from the shard next door sit in lines that the block working on that
+    // shard's edge tile has just brought into L2.
     ConvTile t;
-    const int ty = tile % tiles_y;
-    int rest = tile / tiles_y;
-    const int tx = rest % P.tiles_x;
-    rest /= P.tiles_x;
-    t.plane = rest % planes;
-    t.shard = rest / planes;
-    t.r = t.shard / P.pw_workers;
-    t.c = t.shard % P.pw_workers;
+    const int tx = tile % P.tiles_x;
+    int rest = tile / P.tiles_x;
+    t.c = rest % P.pw_workers;
+    rest /= P.pw_workers;
+    const int ty = rest % tiles_y;
+    rest /= tiles_y;
+    t.r = rest % P.ph_workers;
+    t.plane = rest / P.ph_workers;
+    (void)planes;
+    t.shard = t.r * P.pw_workers + t.c;
     t.bh = P.bh[t.r];
     t.bw = P.bw[t.c];
     t.i0 = ty * kTileH;
