@@ -36,10 +36,17 @@ struct ConvParams {
 // Row pitch (floats) of the shared-memory tile: wide enough for the staged columns (outputs plus
 // PADL columns on the left and PH on the right, rounded up to whole float4s) and for the float4
 // window of the last thread across (8 outputs, K - 1 more inputs, WOFF floats of lead-in).
+__host__ __device__ constexpr int conv_padl(int K, bool adj) {
+    // forward: the halo width; adjoint: the next multiple of four of twice the halo width, so that a
+    // thread whose eight outputs start two columns to the left (see compute_tile) still reads an
+    // aligned window
+    return adj ? ((2 * (K / 2) + 3) / 4) * 4 : K / 2;
+}
+__host__ __device__ constexpr int conv_woff(int K, bool adj) { return adj ? conv_padl(K, adj) - 2 * (K / 2) : 0; }
 __host__ __device__ constexpr int conv_pitch(int K, bool adj) {
     const int ph = K / 2;
-    const int padl = adj ? ((ph + 3) / 4) * 4 : ph;
-    const int nf = ((padl - ph + kColsPerThread + K - 1 + 3) / 4) * 4;
+    const int padl = conv_padl(K, adj);
+    const int nf = ((conv_woff(K, adj) + kColsPerThread + K - 1 + 3) / 4) * 4;
     const int staged = ((kTileW + padl + ph + 3) / 4) * 4;
     const int window = kTileW - kColsPerThread + nf;
     return staged > window ? staged : window;
@@ -111,8 +118,8 @@ __device__ __forceinline__ ConvTile decode_tile(const ConvParams &P, int tile, i
 template <int K, bool ADJ>
 struct ConvCfg {
     static constexpr int PH = K / 2;                                   // halo rows = halo columns
-    static constexpr int PADL = ADJ ? ((PH + 3) / 4) * 4 : PH;         // tile columns left of the first output
-    static constexpr int WOFF = PADL - PH;                             // first column a thread needs in its slot
+    static constexpr int PADL = conv_padl(K, ADJ);                     // tile column of bulk column j0
+    static constexpr int WOFF = conv_woff(K, ADJ);                     // first column a thread needs in its slot
     static constexpr int NF = ((WOFF + kColsPerThread + K - 1 + 3) / 4) * 4;   // floats a thread loads per input row
     static constexpr int PITCH = conv_pitch(K, ADJ);
     static constexpr int ROWS = kTileH + K - 1;
@@ -204,29 +211,39 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
     if (!t.valid) return;
     const float b0 = ADJ ? 0.f : wk2[2 * K * K];
 
+    // Adjoint: a thread's eight outputs start PH columns to the left of its slot, i.e. they are the
+    // padded columns j0 + 8 tx .. + 7 of dx -- 32-byte aligned stores, an aligned input window, and
+    // the left ghost columns come out of the main pass as zeros.  The last 2 PH padded columns of the
+    // shard (PH outputs and the right ghost) are done by a small extra pass of the last tile.
+    const bool last_tile_x = t.j0 + kTileW >= t.bw;
     if (ADJ) {
-        // clear the part of the ghost ring of dx that borders this tile
+        // top / bottom ghost rows above and below this tile's padded column range
         const int pitch_o = t.bw + 2 * C::PH;
         float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::PH) * pitch_o;
-        const int i1 = min(t.i0 + kTileH, t.bh), j1 = min(t.j0 + kTileW, t.bw);
-        const int R0 = t.i0 == 0 ? 0 : t.i0 + C::PH, R1 = i1 == t.bh ? t.bh + 2 * C::PH : i1 + C::PH;
-        const int C0 = t.j0 == 0 ? 0 : t.j0 + C::PH, C1 = j1 == t.bw ? t.bw + 2 * C::PH : j1 + C::PH;
-        const int ncol = C1 - C0;
+        const int c0 = t.j0, c1 = last_tile_x ? pitch_o : t.j0 + kTileW;
         if (t.i0 == 0)
             for (int r = 0; r < C::PH; ++r)
-                for (int q = threadIdx.x; q < ncol; q += kConvThreads) oplane[(size_t)r * pitch_o + C0 + q] = 0.f;
-        if (i1 == t.bh)
+                for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(size_t)r * pitch_o + q] = 0.f;
+        if (t.i0 + kTileH >= t.bh)
             for (int r = 0; r < C::PH; ++r)
-                for (int q = threadIdx.x; q < ncol; q += kConvThreads) oplane[(size_t)(t.bh + C::PH + r) * pitch_o + C0 + q] = 0.f;
-        const int Rb0 = max(R0, C::PH), Rb1 = min(R1, t.bh + C::PH);
-        if (t.j0 == 0)
-            for (int q = threadIdx.x; q < Rb1 - Rb0; q += kConvThreads)
+                for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(size_t)(t.bh + C::PH + r) * pitch_o + q] = 0.f;
+        if (last_tile_x) {
+            // padded columns bw .. bw + 2 PH - 1: outputs bw - PH .. bw - 1, then the right ghost
+            const int out_rows = min(kTileH, t.bh - t.i0);
+            for (int idx = threadIdx.x; idx < out_rows * 2 * C::PH; idx += kConvThreads) {
+                const int row = idx / (2 * C::PH), c = idx % (2 * C::PH);
+                const int ob = t.bw - C::PH + c;                        // bulk column of this output
+                float acc = 0.f;
+                if (ob < t.bw) {
+                    const float *src = tile + row * C::PITCH + (ob - C::PH - (t.j0 - C::PADL));
 #pragma unroll
-                for (int c = 0; c < C::PH; ++c) oplane[(size_t)(Rb0 + q) * pitch_o + c] = 0.f;
-        if (j1 == t.bw)
-            for (int q = threadIdx.x; q < Rb1 - Rb0; q += kConvThreads)
+                    for (int a = 0; a < K; ++a)
 #pragma unroll
-                for (int c = 0; c < C::PH; ++c) oplane[(size_t)(Rb0 + q) * pitch_o + t.bw + C::PH + c] = 0.f;
+                        for (int b = 0; b < K; ++b) acc = fmaf(wk2[2 * (a * K + b)], src[a * C::PITCH + b], acc);
+                }
+                oplane[(size_t)(t.i0 + row + C::PH) * pitch_o + t.bw + c] = acc;
+            }
+        }
     }
 
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
@@ -283,11 +300,13 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
 
     const int pitch_o = t.bw + 2 * C::OOFF;
     float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::OOFF) * pitch_o;
+    // column of the first output inside an output row: forward = bulk column, adjoint = padded column
     const int jo = t.j0 + kColsPerThread * tx;
+    const int jlim = t.bw;                      // forward: bulk width; adjoint: the main pass ends at padded column bw
 #pragma unroll
     for (int r = 0; r < kRowsPerThread; ++r) {
         const int io = t.i0 + ty * kRowsPerThread + r;
-        if (io >= t.bh || jo >= t.bw) continue;
+        if (io >= t.bh || jo >= jlim) continue;
         float e[8], o[8];
 #pragma unroll
         for (int p2 = 0; p2 < 4; ++p2) unpack2(acc_e[r][p2], e[2 * p2], e[2 * p2 + 1]);
@@ -298,17 +317,22 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
         float v[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) v[q] = e[q] + o[q];
-        float *dst = oplane + (size_t)(io + C::OOFF) * pitch_o + C::OOFF + jo;
-        if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        if (ADJ) {
+#pragma unroll
+            for (int q = 0; q < C::PH; ++q)
+                if (jo + q < C::PH) v[q] = 0.f;   // left ghost columns of dx
+        }
+        float *dst = oplane + (size_t)(io + C::OOFF) * pitch_o + jo;
+        if (jo + 7 < jlim && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
             *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
             *reinterpret_cast<float4 *>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
-        } else if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
+        } else if (jo + 7 < jlim && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
 #pragma unroll
             for (int q = 0; q < 8; q += 2) *reinterpret_cast<float2 *>(dst + q) = make_float2(v[q], v[q + 1]);
         } else {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-                if (jo + q < t.bw) dst[q] = v[q];
+                if (jo + q < jlim) dst[q] = v[q];
         }
     }
 }
@@ -397,19 +421,22 @@ template <int K, bool ADJ, typename F>
 __device__ __forceinline__ void for_each_patch_cell(const ConvTile &t, F f) {
     using C = ConvCfg<K, ADJ>;
     const int out_rows = min(kTileH, t.bh - t.i0), out_cols = min(kTileW, t.bw - t.j0);
-    const int W = out_cols + 2 * C::PH, H = out_rows + 2 * C::PH;
+    const int H = out_rows + 2 * C::PH;
     const int colL = C::PADL - C::PH, colR = C::PADL + out_cols, rowB = C::PH + out_rows;
+    // the row strips span every column the tile's threads read: in the adjoint the threads' outputs
+    // start PH columns further left, so their windows start at tile column WOFF = PADL - 2 PH
+    const int colS = C::WOFF, W = colR + C::PH - colS;
     int q0 = 0;
     if (t.i0 == 0) {
 #pragma unroll
         for (int r = 0; r < C::PH; ++r)
-            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, r, colL + s);
+            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, r, colS + s);
         q0 += C::PH * W;
     }
     if (t.i0 + out_rows == t.bh) {
 #pragma unroll
         for (int r = 0; r < C::PH; ++r)
-            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, rowB + r, colL + s);
+            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, rowB + r, colS + s);
         q0 += C::PH * W;
     }
     if (t.j0 == 0) {

@@ -71,6 +71,7 @@ def test_conv_full_size_on_sampled_planes():
     distdl.conv_adj(gpart, dys, dev(w), dxs)
     distdl.device_status()
     planes = [(0, 0), (3, 7), (9, 15), (15, 2), (15, 15)]
+    # tolerance: 25 FMA roundings + one add of the kernel's two partial sums + the oracle's rounding to fp32
     sub = (1, 1, 1024, 1024)
     op = oracle.Partition(sub, ps, (0, 0, 2, 2), (0, 0, 2, 2))
     ob = oracle.Partition(sub, ps)
@@ -83,9 +84,9 @@ def test_conv_full_size_on_sampled_planes():
         dxbound = oracle.conv_adj(op, [np.abs(a) for a in dy1], np.abs(w[c:c + 1]))
         for k in range(16):
             got = host(ys[k][n:n + 1, c:c + 1]).astype(np.float64)
-            assert np.all(np.abs(got - yref[k]) <= 25 * 2.0 ** -24 * ybound[k] + 1e-30)
+            assert np.all(np.abs(got - yref[k]) <= 27 * 2.0 ** -24 * ybound[k] + 1e-30)
             gotx = host(dxs[k][n:n + 1, c:c + 1])
-            assert np.all(np.abs(gotx.astype(np.float64) - dxref[k]) <= 25 * 2.0 ** -24 * dxbound[k] + 1e-30)
+            assert np.all(np.abs(gotx.astype(np.float64) - dxref[k]) <= 27 * 2.0 ** -24 * dxbound[k] + 1e-30)
             mask = np.ones(gotx.shape, dtype=bool)
             mask[op.bulk_slices(k)] = False
             assert not gotx[mask].any()
