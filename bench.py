@@ -451,9 +451,20 @@ def main():
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per launch from the committed ncu summaries under profiles/; null for a
-# kernel that changed since its counters were taken.
-NCU_TRAFFIC = {}
+# DRAM bytes (read + write) per launch from the committed ncu summaries under profiles/ (captures of
+# the quarter-size case are scaled by 4: traffic grows with the number of planes / rows); None for a
+# kernel whose counters were not meaningful (the broadcast's output was still in L2 when the short
+# capture ended) or that changed since its counters were taken.
+NCU_TRAFFIC = {
+    "broadcast_fwd": None,
+    "sumreduce_fwd": 4 * (134223104 + 5289728),
+    "halo_fwd": 203052544 + 117629440,
+    "halo_adj": 262138112 + 167800064,
+    "conv_fwd": 4 * (277907712 + 220590848),
+    "conv_adj": 4 * (272324864 + 230528256),
+    "affine_fwd": 138433536 + 4947200,
+    "affine_adj": 138455040 + 4109056,
+}
 
 if __name__ == "__main__":
     main()
