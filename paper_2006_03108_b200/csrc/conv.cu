@@ -228,20 +228,33 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
             for (int r = 0; r < C::PH; ++r)
                 for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(size_t)(t.bh + C::PH + r) * pitch_o + q] = 0.f;
         if (last_tile_x) {
-            // padded columns bw .. bw + 2 PH - 1: outputs bw - PH .. bw - 1, then the right ghost
+            // padded columns bw .. bw + 2 PH - 1: the outputs bw - PH .. bw - 1, then the right ghost.
+            // One thread per tile row (a single warp), so the other warps go straight to the main pass.
             const int out_rows = min(kTileH, t.bh - t.i0);
-            for (int idx = threadIdx.x; idx < out_rows * 2 * C::PH; idx += kConvThreads) {
-                const int row = idx / (2 * C::PH), c = idx % (2 * C::PH);
-                const int ob = t.bw - C::PH + c;                        // bulk column of this output
-                float acc = 0.f;
-                if (ob < t.bw) {
-                    const float *src = tile + row * C::PITCH + (ob - C::PH - (t.j0 - C::PADL));
+            if ((int)threadIdx.x < out_rows) {
+                const int row = threadIdx.x;
+                const float *src = tile + row * C::PITCH + (t.bw - 2 * C::PH - (t.j0 - C::PADL));
+                float acc[C::PH];
 #pragma unroll
-                    for (int a = 0; a < K; ++a)
+                for (int c = 0; c < C::PH; ++c) acc[c] = 0.f;
 #pragma unroll
-                        for (int b = 0; b < K; ++b) acc = fmaf(wk2[2 * (a * K + b)], src[a * C::PITCH + b], acc);
+                for (int a = 0; a < K; ++a) {
+                    float in[3 * C::PH];
+#pragma unroll
+                    for (int j = 0; j < 3 * C::PH; ++j) in[j] = src[a * C::PITCH + j];
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const float w = wk2[2 * (a * K + b)];
+#pragma unroll
+                        for (int c = 0; c < C::PH; ++c) acc[c] = fmaf(w, in[c + b], acc[c]);
+                    }
                 }
-                oplane[(size_t)(t.i0 + row + C::PH) * pitch_o + t.bw + c] = acc;
+                float *dst = oplane + (size_t)(t.i0 + row + C::PH) * pitch_o + t.bw;
+#pragma unroll
+                for (int c = 0; c < C::PH; ++c) {
+                    dst[c] = acc[c];
+                    dst[C::PH + c] = 0.f;
+                }
             }
         }
     }
