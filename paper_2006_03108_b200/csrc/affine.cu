@@ -368,6 +368,243 @@ affine_kernel(const __grid_constant__ AffineParams P) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Four-block variant: a cluster of two pairs owns a 256 x 256 output tile and splits the workers of
+// the reduction between the pairs (pair 0 takes the first half of the grid row / column, pair 1
+// the second half, each in worker order).  With tiles twice as wide every block of activations is
+// streamed through L2 by half as many pairs, and splitting the reduction keeps all SMs busy.
+//
+// Epilogue: pair 0 finishes output columns [0, 128) of the tile, pair 1 columns [128, 256).  Every
+// block spills its 128 x 256 fp32 accumulator to its own shared memory (the ring is free by then):
+// the half it keeps into `own`, the other half into `send`, which one bulk copy through
+// distributed shared memory moves into the `recv` buffer of the block with the same rows in the
+// other pair.  Each block then adds (first half of the workers) + (second half), adds the bias and
+// writes whole 512-byte row segments.
+// ------------------------------------------------------------------------------------------
+constexpr int kQuadThreads = 256;                           // warps 0/1: one lane each for TMA and MMA; all 8 in the epilogue
+constexpr int kQuadN = 256;                                 // output columns per cluster
+constexpr int kQuadStages = 7;
+constexpr int kQuadABytes = kTileM * kBlockK * 2;           // 16 KB: this block's 128 activation rows
+constexpr int kQuadBBytes = (kQuadN / 2) * kBlockK * 2;     // 16 KB: this block's half of the weight tile
+constexpr int kQuadStageBytes = kQuadABytes + kQuadBBytes;
+constexpr int kQuadSmemBytes = kQuadStages * kQuadStageBytes + 1024 + 256;
+constexpr int kQuadPitch = kQuadN / 2 + 4;                  // floats per row of an epilogue buffer; staggers rows over the banks
+constexpr int kQuadBufBytes = kTileM * kQuadPitch * 4;      // 67,584
+static_assert(3 * kQuadBufBytes <= kQuadStages * kQuadStageBytes, "epilogue buffers must fit in the ring");
+static_assert(kQuadBufBytes % 16 == 0, "bulk copies move multiples of 16 bytes");
+
+__device__ __forceinline__ void tcgen05_commit_mask(uint32_t bar, uint16_t mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+// shared memory of this block -> shared memory of another block of the cluster; the bytes are
+// counted on a barrier of the destination block
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster_addr, uint32_t src, uint32_t bytes, uint32_t bar_cluster_addr) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster_addr), "r"(src), "r"(bytes), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kQuadThreads, 1)
+affine_kernel_quad(const __grid_constant__ AffineParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *aligned = smem_raw + (base - raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kQuadStages * kQuadStageBytes);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * kQuadStages;
+    const uint32_t bar_acc = bar_empty + 8 * kQuadStages;
+    const uint32_t bar_recv = bar_acc + 8;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kQuadStages + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t crank = cluster_ctarank();        // 0..3
+    const uint32_t khalf = crank >> 1;               // which half of the reduction this pair takes
+    const uint32_t prank = crank & 1;                // 0 = leader of its pair
+    const uint32_t leader = crank & ~1u;
+    const int tile = (int)(blockIdx.x >> 2);
+    const int row_tiles = (P.nb + 2 * kTileM - 1) / (2 * kTileM);
+    const int m0 = (tile % row_tiles) * 2 * kTileM + (int)prank * kTileM;
+    const int ntile = tile / row_tiles;
+    const int tiles_per_block = P.blk_out / kQuadN;
+    const int oblk = ntile / tiles_per_block;
+    const int n0 = (ntile % tiles_per_block) * kQuadN;
+    const int kblocks_per_worker = P.blk_red / kBlockK;
+    const int workers = P.nred / 2;                  // workers summed by this pair
+    const int r0 = (int)khalf * workers;             // first of them
+    const int num_kblocks = workers * kblocks_per_worker;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kQuadStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        mbar_init(bar_recv, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        mbar_expect_tx(bar_recv, kQuadBufBytes);     // the other pair's half of this block's columns
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kQuadN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    cluster_sync_all();
+    tcgen05_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const CUtensorMap *amap = &P.a_map[r0];
+            const CUtensorMap *wmap = P.adjoint ? &P.w_map[r0 * P.pfi + oblk] : &P.w_map[oblk * P.pfi + r0];
+            const int wstep = P.adjoint ? P.pfi : 1;
+            const int nb0 = n0 + (int)prank * (kQuadN / 2);
+            uint32_t s = 0, phase = 0, sa = base;
+            int k0 = 0, kin = 0;
+            for (int kb = 0; kb < num_kblocks; ++kb) {
+                if (!mbar_wait(bar_empty + 8 * s, phase ^ 1, abort_flag)) break;
+                const uint32_t full = bar_full + 8 * s;
+                const uint32_t full_leader = map_to_cta(full, leader);
+                if (prank == 0) mbar_expect_tx(full, 2 * kQuadStageBytes);
+                tma_load_2d_pair(sa, amap, k0, m0, full_leader);
+                if (!P.adjoint) {
+                    tma_load_2d_pair(sa + kQuadABytes, wmap, k0, nb0, full_leader);                  // box {64 k, 128 rows}
+                } else {                                                                            // two boxes {64 n, 64 k}
+                    tma_load_2d_pair(sa + kQuadABytes, wmap, nb0, k0, full_leader);
+                    tma_load_2d_pair(sa + kQuadABytes + kQuadBBytes / 2, wmap, nb0 + 64, k0, full_leader);
+                }
+                k0 += kBlockK;
+                if (++kin == kblocks_per_worker) {
+                    kin = 0;
+                    k0 = 0;
+                    ++amap;
+                    wmap += wstep;
+                }
+                sa += kQuadStageBytes;
+                if (++s == kQuadStages) {
+                    s = 0;
+                    sa = base;
+                    phase ^= 1;
+                }
+            }
+            if (*abort_flag) {
+                const uint64_t t0 = global_timer();
+                while (global_timer() - t0 < 1000000ull) {}
+            }
+        }
+        __syncwarp();       // the other lanes sleep here instead of polling beside the producer
+    } else if (warp == 1) {
+        if (lane == 0 && prank == 0) {
+            const uint32_t idesc = instr_desc(2 * kTileM, kQuadN, P.adjoint ? 1 : 0);
+            const uint64_t a0 = smem_desc(base, 16, 1024);
+            const uint64_t b0 = P.adjoint ? smem_desc(base + kQuadABytes, kQuadBBytes / 2, 1024)
+                                          : smem_desc(base + kQuadABytes, 16, 1024);
+            const uint64_t bstep = P.adjoint ? (2048 >> 4) : (32 >> 4);
+            const uint16_t mask = (uint16_t)(3u << leader);       // the two blocks of this pair
+            uint32_t s = 0, phase = 0;
+            uint64_t off = 0;
+            bool ok = true;
+            for (int kb = 0; kb < num_kblocks; ++kb) {
+                ok = mbar_wait(bar_full + 8 * s, phase, abort_flag);
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint64_t a = a0 + off, b = b0 + off;
+                umma_bf16_pair(tmem_acc, a, b, idesc, kb ? 1u : 0u);
+                umma_bf16_pair(tmem_acc, a + 2, b + bstep, idesc, 1u);
+                umma_bf16_pair(tmem_acc, a + 4, b + 2 * bstep, idesc, 1u);
+                umma_bf16_pair(tmem_acc, a + 6, b + 3 * bstep, idesc, 1u);
+                tcgen05_commit_mask(bar_empty + 8 * s, mask);
+                off += kQuadStageBytes >> 4;
+                if (++s == kQuadStages) {
+                    s = 0;
+                    off = 0;
+                    phase ^= 1;
+                }
+            }
+            if (ok) tcgen05_commit_mask(bar_acc, mask);
+        }
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------------------------- epilogue, all warps
+    // this pair's accumulator is complete: its MMAs have retired, so the ring is free as well
+    const bool acc_ok = mbar_wait(bar_acc, 0, abort_flag);
+    const bool ok = __syncthreads_and(acc_ok) != 0;
+    tcgen05_fence_after();
+    tcgen05_fence_before();
+    cluster_sync_all();                      // ... in all four blocks: `recv` may be written from outside
+
+    const int quarter = warp & 3;            // tensor-memory lanes [32 q, 32 q + 32) belong to warps q and q + 4
+    const int chalf = warp >> 2;             // column half of the tile this warp spills
+    const uint32_t buf_own = base, buf_send = base + kQuadBufBytes, buf_recv = base + 2 * kQuadBufBytes;
+    if (ok) {
+        tcgen05_fence_after();
+        const uint32_t dst = ((uint32_t)chalf == khalf ? buf_own : buf_send) +
+                             (uint32_t)((quarter * 32 + lane) * kQuadPitch * 4);
+#pragma unroll 1
+        for (int c = 0; c < kQuadN / 2; c += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(chalf * (kQuadN / 2) + c), v);
+#pragma unroll
+            for (int q = 0; q < 32; q += 4)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c + q) * 4)), "r"(v[q]),
+                             "r"(v[q + 1]), "r"(v[q + 2]), "r"(v[q + 3]) : "memory");
+        }
+        fence_proxy_async();                 // the bulk copy below reads what was just written
+    }
+    __syncthreads();
+    if (ok && threadIdx.x == 0)
+        bulk_copy_to_cta(map_to_cta(buf_recv, crank ^ 2u), buf_send, kQuadBufBytes, map_to_cta(bar_recv, crank ^ 2u));
+    const bool got = ok && mbar_wait(bar_recv, 0, abort_flag);
+    if (got) {
+        const float *own = reinterpret_cast<const float *>(aligned);
+        const float *recv = reinterpret_cast<const float *>(aligned + 2 * kQuadBufBytes);
+        const int col = n0 + (int)khalf * (kQuadN / 2) + 4 * lane;     // column inside the output block
+        const float *bias = P.bias[oblk];
+        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (bias) b = __ldg(reinterpret_cast<const float4 *>(bias + col));
+        constexpr int kRowsPerWarp = kTileM / (kQuadThreads / 32);
+#pragma unroll 4
+        for (int i = 0; i < kRowsPerWarp; ++i) {
+            const int rloc = warp * kRowsPerWarp + i;
+            const int row = m0 + rloc;
+            if (row >= P.nb) break;
+            const float4 mine = *reinterpret_cast<const float4 *>(own + rloc * kQuadPitch + 4 * lane);
+            const float4 other = *reinterpret_cast<const float4 *>(recv + rloc * kQuadPitch + 4 * lane);
+            // (workers of the first half) + (workers of the second half), then the bias
+            float4 o;
+            o.x = (khalf == 0 ? mine.x + other.x : other.x + mine.x) + b.x;
+            o.y = (khalf == 0 ? mine.y + other.y : other.y + mine.y) + b.y;
+            o.z = (khalf == 0 ? mine.z + other.z : other.z + mine.z) + b.z;
+            o.w = (khalf == 0 ? mine.w + other.w : other.w + mine.w) + b.w;
+            *reinterpret_cast<float4 *>(P.out[oblk] + (size_t)row * P.blk_out + col) = o;
+        }
+    }
+    // nobody retires while its outgoing copy may still read its shared memory or a peer may signal
+    // its barriers; the peer's arrival here follows the end of that copy
+    tcgen05_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kQuadN) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 static EncodeTiledFn encode_fn() { return tensor_map_encoder(); }
@@ -423,12 +660,14 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
             return fail(DISTDL_ERR_CUDA, "%s: tensor map of activation block %d failed", what, i);
     // more than one 128-row tile of the batch: a pair of blocks shares each 256 x 128 output tile
     const bool pair = nb > kTileM;
+    // four-block variant: an even number of workers to sum over and output blocks of whole 256-column tiles
+    const bool quad = pair && ((adjoint ? pfo : pfi) % 2 == 0) && ((adjoint ? bfi : bfo) % kQuadN == 0);
     for (int i = 0; i < pfo * pfi; ++i) {
         // forward: box {64 along in-features (K), 128 out-feature rows} (64 rows per block of a pair);
         // adjoint: box {64 along in-features (N), 64 out-feature rows (K)} of the same row-major
         // [bfo, bfi] block
         const bool ok = adjoint ? make_map(&P.w_map[i], w[i], bfo, bfi, 64, kBlockK)
-                                : make_map(&P.w_map[i], w[i], bfo, bfi, kBlockK, pair ? kTileN / 2 : kTileN);
+                                : make_map(&P.w_map[i], w[i], bfo, bfi, kBlockK, quad ? kQuadN / 2 : (pair ? kTileN / 2 : kTileN));
         if (!ok) return fail(DISTDL_ERR_CUDA, "%s: tensor map of weight block %d failed", what, i);
     }
     for (int i = 0; i < nout; ++i) {
@@ -449,10 +688,28 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
                                                AffineCfg<false>::SMEM_BYTES));
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                AffineCfg<true>::SMEM_BYTES));
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel_quad, cudaFuncAttributeMaxDynamicSharedMemorySize, kQuadSmemBytes));
         configured = true;
     }
     const int64_t ntiles = (adjoint ? nfi : nfo) / kTileN;
-    if (pair) {
+    if (quad) {
+        const int64_t row_pairs = (nb + 2 * kTileM - 1) / (2 * kTileM);
+        const int64_t qtiles = (adjoint ? nfi : nfo) / kQuadN;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)(4 * row_pairs * qtiles));
+        cfg.blockDim = dim3(kQuadThreads);
+        cfg.dynamicSmemBytes = kQuadSmemBytes;
+        cfg.stream = (cudaStream_t)stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 4;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        DISTDL_CUDA_CHECK(cudaLaunchKernelEx(&cfg, affine_kernel_quad, P));
+    } else if (pair) {
         const int64_t row_pairs = (nb + 2 * kTileM - 1) / (2 * kTileM);
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));

@@ -286,6 +286,8 @@ AFFINE_CASES = [
     (256, 1024, 512, 4, 4),
     (77, 256, 1024, 1, 2),
     (300, 768, 256, 2, 1),
+    (300, 1024, 1024, 2, 4),     # 256-column tiles, reduction split between two pairs (both directions)
+    (520, 512, 768, 3, 2),       # forward splits the reduction, adjoint (three workers) does not
 ]
 
 
