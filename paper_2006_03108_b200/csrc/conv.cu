@@ -31,7 +31,28 @@ struct ConvParams {
     int32_t ph_workers, pw_workers;
     int32_t channels;
     int32_t tiles_x;
+    // n / d for the four divisors of the tile decoding (tiles_x, pw_workers, tiles_y, ph_workers):
+    // umulhi(n, magic) >> shift for any n < 2^31; magic = 0 stands for d = 1
+    uint32_t div_magic[4], div_shift[4];
 };
+
+// magic = ceil(2^(31+s) / d) with s = ceil(log2 d) is below 2^32 and divides every n < 2^31 exactly.
+inline void conv_set_divisor(ConvParams &P, int which, uint32_t d) {
+    if (d < 2) {
+        P.div_magic[which] = 0;
+        P.div_shift[which] = 0;
+        return;
+    }
+    uint32_t sh = 0;
+    while ((1u << sh) < d) ++sh;
+    const uint64_t num = (uint64_t)1 << (31 + sh);
+    P.div_magic[which] = (uint32_t)((num + d - 1) / d);
+    P.div_shift[which] = sh - 1;
+}
+__device__ __forceinline__ uint32_t conv_div(const ConvParams &P, int which, uint32_t n) {
+    const uint32_t m = P.div_magic[which];
+    return m ? __umulhi(n, m) >> P.div_shift[which] : n;
+}
 
 // Row pitch (floats) of the shared-memory tile: wide enough for the staged columns (outputs plus
 // PADL columns on the left and PH on the right, rounded up to whole float4s) and for the float4
@@ -49,7 +70,10 @@ __host__ __device__ constexpr int conv_pitch(int K, bool adj) {
     const int nf = ((conv_woff(K, adj) + kColsPerThread + K - 1 + 3) / 4) * 4;
     const int staged = ((kTileW + padl + ph + 3) / 4) * 4;
     const int window = kTileW - kColsPerThread + nf;
-    return staged > window ? staged : window;
+    const int p = staged > window ? staged : window;
+    // an odd number of float4s per row: 16-byte loads whose lanes walk down a column (the edge pass
+    // of the adjoint) then fall into eight different bank groups per quarter warp
+    return (p / 4) % 2 ? p : p + 4;
 }
 
 __device__ __forceinline__ void cp_async16(float *smem, const float *gmem) {
@@ -92,14 +116,19 @@ __device__ __forceinline__ ConvTile decode_tile(const ConvParams &P, int tile, i
     // halo cells a tile takes from the shard next door sit in lines that the block working on that
     // shard's edge tile has just brought into L2.
     ConvTile t;
-    const int tx = tile % P.tiles_x;
-    int rest = tile / P.tiles_x;
-    t.c = rest % P.pw_workers;
-    rest /= P.pw_workers;
-    const int ty = rest % tiles_y;
-    rest /= tiles_y;
-    t.r = rest % P.ph_workers;
-    t.plane = rest / P.ph_workers;
+    uint32_t rest = (uint32_t)tile, q;
+    q = conv_div(P, 0, rest);
+    const int tx = (int)(rest - q * (uint32_t)P.tiles_x);
+    rest = q;
+    q = conv_div(P, 1, rest);
+    t.c = (int)(rest - q * (uint32_t)P.pw_workers);
+    rest = q;
+    q = conv_div(P, 2, rest);
+    const int ty = (int)(rest - q * (uint32_t)tiles_y);
+    rest = q;
+    q = conv_div(P, 3, rest);
+    t.r = (int)(rest - q * (uint32_t)P.ph_workers);
+    t.plane = (int)q;
     (void)planes;
     t.shard = t.r * P.pw_workers + t.c;
     t.bh = P.bh[t.r];
@@ -219,41 +248,82 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
     if (ADJ) {
         // top / bottom ghost rows above and below this tile's padded column range
         const int pitch_o = t.bw + 2 * C::PH;
-        float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::PH) * pitch_o;
+        float *oplane = P.out[t.shard] + (uint32_t)t.plane * (uint32_t)(t.bh + 2 * C::PH) * (uint32_t)pitch_o;
         const int c0 = t.j0, c1 = last_tile_x ? pitch_o : t.j0 + kTileW;
         if (t.i0 == 0)
             for (int r = 0; r < C::PH; ++r)
-                for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(size_t)r * pitch_o + q] = 0.f;
+                for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[r * pitch_o + q] = 0.f;
         if (t.i0 + kTileH >= t.bh)
             for (int r = 0; r < C::PH; ++r)
-                for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(size_t)(t.bh + C::PH + r) * pitch_o + q] = 0.f;
+                for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(t.bh + C::PH + r) * pitch_o + q] = 0.f;
         if (last_tile_x) {
             // padded columns bw .. bw + 2 PH - 1: the outputs bw - PH .. bw - 1, then the right ghost.
             // One thread per tile row (a single warp), so the other warps go straight to the main pass.
             const int out_rows = min(kTileH, t.bh - t.i0);
             if ((int)threadIdx.x < out_rows) {
                 const int row = threadIdx.x;
-                const float *src = tile + row * C::PITCH + (t.bw - 2 * C::PH - (t.j0 - C::PADL));
+                const int first = t.bw - 2 * C::PH - (t.j0 - C::PADL);     // tile column of the window's first input
                 float acc[C::PH];
 #pragma unroll
                 for (int c = 0; c < C::PH; ++c) acc[c] = 0.f;
+                constexpr int LEAD = C::WOFF % 4;                          // first % 4 when bw is a multiple of four
+                if (((first - LEAD) & 3) == 0) {
+                    // aligned window: float4 loads (conflict-free down a column thanks to the odd pitch)
+                    constexpr int NV = (LEAD + 3 * C::PH + 3) / 4;
+                    const float4 *src = reinterpret_cast<const float4 *>(tile + row * C::PITCH + (first - LEAD));
 #pragma unroll
-                for (int a = 0; a < K; ++a) {
-                    float in[3 * C::PH];
+                    for (int a = 0; a < K; ++a) {
+                        float in[4 * NV];
 #pragma unroll
-                    for (int j = 0; j < 3 * C::PH; ++j) in[j] = src[a * C::PITCH + j];
+                        for (int v = 0; v < NV; ++v) {
+                            const float4 q = src[a * (C::PITCH / 4) + v];
+                            in[4 * v] = q.x;
+                            in[4 * v + 1] = q.y;
+                            in[4 * v + 2] = q.z;
+                            in[4 * v + 3] = q.w;
+                        }
 #pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        const float w = wk2[2 * (a * K + b)];
+                        for (int b = 0; b < K; ++b) {
+                            const float w = wk2[2 * (a * K + b)];
 #pragma unroll
-                        for (int c = 0; c < C::PH; ++c) acc[c] = fmaf(w, in[c + b], acc[c]);
+                            for (int c = 0; c < C::PH; ++c) acc[c] = fmaf(w, in[LEAD + c + b], acc[c]);
+                        }
+                    }
+                } else {
+                    const float *src = tile + row * C::PITCH + first;
+#pragma unroll
+                    for (int a = 0; a < K; ++a) {
+                        float in[3 * C::PH];
+#pragma unroll
+                        for (int j = 0; j < 3 * C::PH; ++j) in[j] = src[a * C::PITCH + j];
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            const float w = wk2[2 * (a * K + b)];
+#pragma unroll
+                            for (int c = 0; c < C::PH; ++c) acc[c] = fmaf(w, in[c + b], acc[c]);
+                        }
                     }
                 }
-                float *dst = oplane + (size_t)(t.i0 + row + C::PH) * pitch_o + t.bw;
+                float *dst = oplane + ((t.i0 + row + C::PH) * pitch_o + t.bw);
+                // every lane writes to another row, so each store instruction costs 32 separate
+                // memory requests: use as few and as wide stores as the alignment allows
+                float e[2 * C::PH];
 #pragma unroll
                 for (int c = 0; c < C::PH; ++c) {
-                    dst[c] = acc[c];
-                    dst[C::PH + c] = 0.f;
+                    e[c] = acc[c];
+                    e[C::PH + c] = 0.f;
+                }
+                const uintptr_t da = reinterpret_cast<uintptr_t>(dst);
+                if (C::PH % 2 == 0 && (da & 15u) == 0) {
+#pragma unroll
+                    for (int c = 0; c < 2 * C::PH; c += 4)
+                        *reinterpret_cast<float4 *>(dst + c) = make_float4(e[c], e[c + 1], e[c + 2], e[c + 3]);
+                } else if ((da & 7u) == 0) {
+#pragma unroll
+                    for (int c = 0; c < 2 * C::PH; c += 2) *reinterpret_cast<float2 *>(dst + c) = make_float2(e[c], e[c + 1]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 2 * C::PH; ++c) dst[c] = e[c];
                 }
             }
         }
@@ -311,8 +381,8 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
         }
     }
 
-    const int pitch_o = t.bw + 2 * C::OOFF;
-    float *oplane = P.out[t.shard] + (size_t)t.plane * (t.bh + 2 * C::OOFF) * pitch_o;
+    const uint32_t pitch_o = (uint32_t)(t.bw + 2 * C::OOFF);
+    float *oplane = P.out[t.shard] + (uint32_t)t.plane * (uint32_t)(t.bh + 2 * C::OOFF) * pitch_o;   // below 2^31 elements per shard
     // column of the first output inside an output row: forward = bulk column, adjoint = padded column
     const int jo = t.j0 + kColsPerThread * tx;
     const int jlim = t.bw;                      // forward: bulk width; adjoint: the main pass ends at padded column bw
@@ -335,8 +405,12 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
             for (int q = 0; q < C::PH; ++q)
                 if (jo + q < C::PH) v[q] = 0.f;   // left ghost columns of dx
         }
-        float *dst = oplane + (size_t)(io + C::OOFF) * pitch_o + jo;
-        if (jo + 7 < jlim && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        float *dst = oplane + ((uint32_t)(io + C::OOFF) * pitch_o + (uint32_t)jo);
+        if (jo + 7 < jlim && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+            // one 256-bit store: a half warp then writes 512 contiguous bytes of a row in one request
+            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+                         "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+        } else if (jo + 7 < jlim && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
             *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
             *reinterpret_cast<float4 *>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
         } else if (jo + 7 < jlim && (reinterpret_cast<uintptr_t>(dst) & 7u) == 0) {
@@ -515,9 +589,11 @@ __device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const Con
             if (ok) ok = j < P.bw[cc];
         }
         if (ok) {
-            const int pitch_n = P.bw[cc] + 2 * C::IOFF;
-            cp_async4(side + q, P.in[rr * P.pw_workers + cc] + (size_t)t.plane * (P.bh[rr] + 2 * C::IOFF) * pitch_n +
-                                    (size_t)(i + C::IOFF) * pitch_n + C::IOFF + j);
+            // a shard holds fewer than 2^31 elements: 32-bit offsets
+            const uint32_t pitch_n = (uint32_t)(P.bw[cc] + 2 * C::IOFF);
+            const uint32_t off = ((uint32_t)t.plane * (uint32_t)(P.bh[rr] + 2 * C::IOFF) + (uint32_t)(i + C::IOFF)) * pitch_n +
+                                 (uint32_t)(C::IOFF + j);
+            cp_async4(side + q, P.in[rr * P.pw_workers + cc] + off);
         } else {
             side[q] = 0.f;
         }
@@ -714,6 +790,10 @@ static distdl_status_t conv_impl(const distdl_partition *p, const void *const *i
     P.channels = (int32_t)p->global_shape[1];
     P.tiles_x = (int32_t)((max_bw + kTileW - 1) / kTileW);
     const int tiles_y = (int)((max_bh + kTileH - 1) / kTileH);
+    conv_set_divisor(P, 0, (uint32_t)P.tiles_x);
+    conv_set_divisor(P, 1, (uint32_t)P.pw_workers);
+    conv_set_divisor(P, 2, (uint32_t)tiles_y);
+    conv_set_divisor(P, 3, (uint32_t)P.ph_workers);
     const int64_t total = (int64_t)P.tiles_x * tiles_y * planes * p->num_workers;
     if (total >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
     cudaStream_t s = (cudaStream_t)stream;
