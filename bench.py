@@ -460,10 +460,10 @@ NCU_TRAFFIC = {
     "sumreduce_fwd": 4 * (134223104 + 5289728),
     "halo_fwd": 203052544 + 117629440,
     "halo_adj": 262138112 + 167800064,
-    "conv_fwd": 4 * (277907712 + 220590848),
-    "conv_adj": 4 * (272324864 + 230528256),
-    "affine_fwd": 138433536 + 4947200,
-    "affine_adj": 138455040 + 4109056,
+    "conv_fwd": 4 * (277898496 + 221322496),
+    "conv_adj": 4 * (269446656 + 227919872),
+    "affine_fwd": 138432256 + 4193024,
+    "affine_adj": 138448640 + 4337152,
 }
 
 if __name__ == "__main__":
