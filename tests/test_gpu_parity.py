@@ -69,6 +69,24 @@ def test_broadcast_bf16_and_in_place():
         assert same_bits(host(d.view(torch.int16)).view(np.uint16), x)
 
 
+@pytest.mark.parametrize("shift", [(0, 0), (4, 0), (0, 4), (4, 4)], ids=["32/32", "16/32", "32/16", "16/16"])
+def test_broadcast_alignment_paths(shift):
+    # source / destinations aligned to 32 bytes take 256-bit accesses, anything else 16-byte ones;
+    # the cells around every destination must stay untouched
+    n, k = 100003, 3
+    x = inputs.uniform_pm1((n,), 17)
+    s_off, d_off = shift
+    src = torch.zeros(n + 16, device=DEV)
+    src[s_off:s_off + n] = dev(x)
+    bufs = [torch.full((n + 16,), 7.0, device=DEV) for _ in range(k)]
+    distdl.broadcast_fwd(src[s_off:s_off + n], [b[d_off:d_off + n] for b in bufs])
+    torch.cuda.synchronize()
+    for b in bufs:
+        h = host(b)
+        assert same_bits(h[d_off:d_off + n], x)
+        assert np.all(h[:d_off] == 7.0) and np.all(h[d_off + n:] == 7.0)
+
+
 @pytest.mark.parametrize("n", [1, 5, 1000, 4099, (1 << 21) + 3])
 @pytest.mark.parametrize("k", [1, 2, 3, 4, 8, 16, 17, 35])
 def test_sumreduce_bit_exact(n, k):
