@@ -2,8 +2,8 @@
 
 TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, deliberately naive
 numpy restatement of what the operators compute (broadcast B, sum-reduce R = B*,
-halo exchange H, adjoint halo exchange H*, the distributed depthwise convolution
-and the distributed affine layer, each with its adjoint).  Nothing in the product
+halo exchange H, adjoint halo exchange H*, the distributed depthwise convolution,
+the distributed pooling layer and the distributed affine layer, each with its adjoint).  Nothing in the product
 package imports it; only the test-suite, the smoke check and the CPU-baseline leg
 of the benchmark may call it.  It shares no code, table or helper with the CUDA
 path and imports nothing but numpy.
@@ -37,4 +37,9 @@ from .layers import (  # noqa: F401
     affine_fwd,
     affine_adj,
     bf16_bits_to_f64,
+    pool_partition,
+    pool_fwd_global,
+    pool_adj_global,
+    pool_fwd,
+    pool_adj,
 )

@@ -1,4 +1,4 @@
-"""Oracle distributed layers: depthwise convolution and affine (Section 4).
+"""Oracle distributed layers: depthwise convolution, pooling and affine (Section 4).
 
 TEST INFRASTRUCTURE ONLY (see the package docstring).
 
@@ -168,3 +168,174 @@ def affine_adj(dy_parts, w_parts, pfo, pfi):
             partial.append(dyhat[i][j] @ wij)
         dx.append(sumreduce_fwd(partial).astype(np.float32))
     return dx
+
+
+# --------------------------------------------------------------------------
+# Distributed pooling layer (Section 4, "Sparse layers": pooling layers follow
+# the convolution algorithms without weights; Appendix B: unbalanced halos of
+# strided kernels)
+# --------------------------------------------------------------------------
+
+def pool_partition(global_shape, pshape, kernel, stride, pad):
+    """Partition of a rank-4 NCHW input whose ghost widths are those of a pooling kernel.
+
+    kernel = (kh, kw), stride = (sh, sw), pad = ((lo_h, hi_h), (lo_w, hi_w)).
+    Only the two feature dimensions may be partitioned.  The widths of every
+    worker follow from the range of inputs its block of the evenly split output
+    needs (Section 3; Figs. B1-B4).  Returns (partition, geometry) where
+    geometry[k] (k = 0 for H, 1 for W) is the list of per-worker-coordinate
+    dicts of `halo_widths_1d`.
+    """
+    from .partition import halo_widths_1d
+    assert len(global_shape) == 4 and pshape[0] == 1 and pshape[1] == 1
+    geo = [halo_widths_1d(global_shape[2 + k], pshape[2 + k], kernel[k], stride[k], 1, pad[k][0], pad[k][1])
+           for k in range(2)]
+    hlo = [0, 0] + [[g["halo_lo"] for g in geo[k]] for k in range(2)]
+    hhi = [0, 0] + [[g["halo_hi"] for g in geo[k]] for k in range(2)]
+    return Partition(global_shape, pshape, hlo, hhi), geo
+
+
+def _pool_windows(xg, kernel, stride, pad, fill):
+    """All windows of the padded global tensor: array [N, C, Ho, Wo, kh, kw] (fp64)."""
+    N, C, Hg, Wg = xg.shape
+    (kh, kw), (sh, sw) = kernel, stride
+    (plh, phh), (plw, phw) = pad
+    Ho = (Hg + plh + phh - kh) // sh + 1
+    Wo = (Wg + plw + phw - kw) // sw + 1
+    xp = np.full((N, C, Hg + plh + phh, Wg + plw + phw), fill, dtype=np.float64)
+    xp[:, :, plh:plh + Hg, plw:plw + Wg] = xg
+    win = np.empty((N, C, Ho, Wo, kh, kw), dtype=np.float64)
+    for a in range(kh):
+        for b in range(kw):
+            win[..., a, b] = xp[:, :, a:a + (Ho - 1) * sh + 1:sh, b:b + (Wo - 1) * sw + 1:sw]
+    return win
+
+
+def pool_fwd_global(xg, kernel, stride, pad, mode):
+    """The sequential pooling layer on the unpartitioned tensor.
+
+    mode "avg": y = mean over the kh x kw window of the zero-padded input (padding
+    cells count in the divisor), fp64 sum rounded once to fp32.
+    mode "max": y = largest value of the window, padding excluded (the window is
+    clipped to the tensor); also returns, per output, the position a*kw + b inside
+    the unclipped window of the first largest value in row-major window order.
+    Returns (y, argmax or None).
+    """
+    xg = np.asarray(xg)
+    kh, kw = kernel
+    if mode == "avg":
+        win = _pool_windows(xg.astype(np.float64), kernel, stride, pad, 0.0)
+        return (win.sum(axis=(4, 5)) / (kh * kw)).astype(np.float32), None
+    assert mode == "max"
+    win = _pool_windows(xg.astype(np.float64), kernel, stride, pad, -np.inf)
+    flat = win.reshape(win.shape[:4] + (kh * kw,))
+    arg = flat.argmax(axis=4)            # first occurrence of the maximum
+    return flat.max(axis=4).astype(np.float32), arg.astype(np.int32)
+
+
+def pool_adj_global(dyg, in_hw, kernel, stride, pad, mode, argmax=None):
+    """Adjoint of the pooling layer (for "max": of its Jacobian at the recorded argmax).
+
+    dx[p, q] = sum over the outputs (i, j) whose window holds (p, q) of
+    dy[i, j] / (kh*kw)  (avg), or of dy[i, j] where the recorded position of the
+    maximum is (p, q)  (max).  fp64 sums rounded once to fp32.
+    """
+    dyg = np.asarray(dyg, dtype=np.float64)
+    N, C, Ho, Wo = dyg.shape
+    (kh, kw), (sh, sw) = kernel, stride
+    (plh, phh), (plw, phw) = pad
+    Hg, Wg = in_hw
+    dxp = np.zeros((N, C, Hg + plh + phh, Wg + plw + phw), dtype=np.float64)
+    for a in range(kh):
+        for b in range(kw):
+            if mode == "avg":
+                contrib = dyg / (kh * kw)
+            else:
+                contrib = np.where(argmax == a * kw + b, dyg, 0.0)
+            dxp[:, :, a:a + (Ho - 1) * sh + 1:sh, b:b + (Wo - 1) * sw + 1:sw] += contrib
+    return dxp[:, :, plh:plh + Hg, plw:plw + Wg].astype(np.float32)
+
+
+def _pool_out_slices(geo, coords):
+    return tuple(slice(geo[k][coords[2 + k]]["out_start"],
+                       geo[k][coords[2 + k]]["out_start"] + geo[k][coords[2 + k]]["out_size"]) for k in range(2))
+
+
+def pool_fwd(part: Partition, geo, x_shards, kernel, stride, pad, mode):
+    """Distributed pooling, forward: y = Pool(H x), in the steps of the forward algorithm.
+
+    1. halo exchange on the padded input shards (ghosts on the tensor boundary
+       hold the implicit zero padding; for "max" they are excluded from the window),
+    2. every worker applies the sequential layer to its padded shard, starting at the
+       first input its outputs need (owned inputs before it are unused, Fig. B3).
+    Returns (y shards, argmax shards or None); worker c owns the c-th block of the
+    evenly split output.
+    """
+    from .primitives import halo_fwd_definition
+    xs = halo_fwd_definition(part, x_shards)
+    (kh, kw), (sh, sw) = kernel, stride
+    ys, args = [], []
+    for w in range(part.num_workers):
+        c = part.coords(w)
+        gh, gw = geo[0][c[2]], geo[1][c[3]]
+        st = part.bulk_start(w)
+        lo, _ = part.widths(w)
+        x = xs[w].astype(np.float64)
+        oh, ow = gh["out_size"], gw["out_size"]
+        # padded-local index of the first input of the first local output
+        i0 = gh["out_start"] * sh - pad[0][0] - (st[2] - lo[2])
+        j0 = gw["out_start"] * sw - pad[1][0] - (st[3] - lo[3])
+        assert oh == 0 or (i0 >= 0 and i0 + (oh - 1) * sh + kh <= x.shape[2])
+        assert ow == 0 or (j0 >= 0 and j0 + (ow - 1) * sw + kw <= x.shape[3])
+        win = np.empty(x.shape[:2] + (oh, ow, kh, kw), dtype=np.float64)
+        for a in range(kh):
+            for b in range(kw):
+                win[..., a, b] = x[:, :, i0 + a:i0 + a + max(oh - 1, 0) * sh + 1:sh,
+                                   j0 + b:j0 + b + max(ow - 1, 0) * sw + 1:sw] if oh and ow else 0.0
+        if mode == "avg":
+            ys.append((win.sum(axis=(4, 5)) / (kh * kw)).astype(np.float32))
+            args.append(None)
+        else:
+            # cells outside the tensor are not candidates
+            gi = (st[2] - lo[2]) + i0 + np.arange(oh)[:, None] * sh + np.arange(kh)[None, :]
+            gj = (st[3] - lo[3]) + j0 + np.arange(ow)[:, None] * sw + np.arange(kw)[None, :]
+            out_i = (gi < 0) | (gi >= part.global_shape[2])
+            out_j = (gj < 0) | (gj >= part.global_shape[3])
+            mask = out_i[:, None, :, None] | out_j[None, :, None, :]
+            win = np.where(mask[None, None], -np.inf, win)
+            flat = win.reshape(win.shape[:4] + (kh * kw,))
+            ys.append(flat.max(axis=4).astype(np.float32) if oh and ow else np.zeros(win.shape[:4], np.float32))
+            args.append(flat.argmax(axis=4).astype(np.int32) if oh and ow else np.zeros(win.shape[:4], np.int32))
+    return ys, (None if mode == "avg" else args)
+
+
+def pool_adj(part: Partition, geo, dy_shards, kernel, stride, pad, mode, arg_shards=None):
+    """Distributed pooling, adjoint: dx = H* Pool* dy, in the steps of the adjoint algorithm.
+
+    1. every worker applies the adjoint of its local layer: each cell of its padded
+       shard (ghosts included) receives the contributions of the worker's own outputs,
+    2. adjoint halo exchange: ghost contributions are added into the owners' bulk
+       and the ghosts are cleared.
+    Returns padded fp32 shards.  (Local sums in fp64, rounded to fp32 before H*, whose
+    sums are fp32 in the nested order -- the rounding points of the method.)
+    """
+    (kh, kw), (sh, sw) = kernel, stride
+    dxs = []
+    for w in range(part.num_workers):
+        c = part.coords(w)
+        gh, gw = geo[0][c[2]], geo[1][c[3]]
+        st = part.bulk_start(w)
+        lo, _ = part.widths(w)
+        pshape = part.padded_shape(w)
+        dx = np.zeros(pshape, dtype=np.float64)
+        oh, ow = gh["out_size"], gw["out_size"]
+        if oh and ow:
+            i0 = gh["out_start"] * sh - pad[0][0] - (st[2] - lo[2])
+            j0 = gw["out_start"] * sw - pad[1][0] - (st[3] - lo[3])
+            dy = np.asarray(dy_shards[w], dtype=np.float64)
+            for a in range(kh):
+                for b in range(kw):
+                    contrib = dy / (kh * kw) if mode == "avg" else np.where(arg_shards[w] == a * kw + b, dy, 0.0)
+                    dx[:, :, i0 + a:i0 + a + (oh - 1) * sh + 1:sh, j0 + b:j0 + b + (ow - 1) * sw + 1:sw] += contrib
+        dxs.append(dx.astype(np.float32))
+    return halo_adj_sequence(part, dxs)

@@ -458,3 +458,124 @@ def test_bf16_helpers_round_to_nearest_even():
     assert bits.tolist() == [0x3F80, 0x3F82, 0xC020, 0x0000]
     assert oracle.bf16_bits_to_f64(bits).tolist() == [1.0, 1.0 + 2.0 ** -6, -2.5, 0.0]
     assert inputs.bf16_bits_to_f32(bits).tolist() == [1.0, 1.0 + 2.0 ** -6, -2.5, 0.0]
+
+
+# --------------------------------------------------------------------------
+# Distributed pooling layer (Section 4 "Sparse layers" + Appendix B halos)
+# --------------------------------------------------------------------------
+
+POOL_CASES = [
+    # global shape, partition, kernel, stride, padding
+    ((2, 3, 11, 10), (1, 1, 3, 2), (2, 2), (2, 2), ((0, 0), (0, 0))),
+    ((1, 2, 20, 17), (1, 1, 6, 3), (3, 3), (2, 2), ((1, 1), (1, 1))),
+    ((1, 1, 12, 12), (1, 1, 2, 2), (3, 2), (1, 2), ((1, 0), (0, 1))),
+    ((1, 1, 1, 20), (1, 1, 1, 6), (1, 2), (1, 2), ((0, 0), (0, 0))),     # Fig. B4 along the last dimension
+    ((1, 1, 1, 10), (1, 1, 1, 3), (1, 2), (1, 2), ((0, 0), (0, 0))),     # Fig. B3
+    ((1, 2, 9, 9), (1, 1, 1, 1), (3, 3), (3, 3), ((0, 0), (0, 0))),
+]
+
+
+def _pool_setup(case, seed):
+    gs, ps, k, s, pad = case
+    part, geo = oracle.layers.pool_partition(gs, ps, k, s, pad)
+    xg = inputs.normal(gs, seed)
+    garbage = lambda w: inputs.normal(part.padded_shape(w), seed + 100 + w)
+    return part, geo, xg, oracle.scatter_global(part, xg, fill=garbage)
+
+
+def _out_block(geo, part, w):
+    c = part.coords(w)
+    return (slice(None), slice(None)) + tuple(
+        slice(geo[k][c[2 + k]]["out_start"], geo[k][c[2 + k]]["out_start"] + geo[k][c[2 + k]]["out_size"]) for k in range(2))
+
+
+@pytest.mark.parametrize("mode", ["avg", "max"])
+def test_pool_global_matches_library_routine(mode):
+    import torch
+    import torch.nn.functional as F
+    xg = inputs.normal((2, 3, 13, 14), 71)
+    t = torch.from_numpy(xg)
+    for k, s, p in [((3, 3), (2, 2), 1), ((2, 2), (2, 2), 0), ((3, 2), (1, 2), 0), ((5, 5), (3, 3), 2)]:
+        pad = ((p, p), (p, p))
+        y, arg = oracle.layers.pool_fwd_global(xg, k, s, pad, mode)
+        if mode == "avg":
+            ref = F.avg_pool2d(t, k, s, p).numpy()           # padding counts in the divisor by default
+            assert np.max(np.abs(y - ref)) <= 4 * 2.0 ** -24 * np.max(np.abs(xg))
+        else:
+            ref, idx = F.max_pool2d(t, k, s, p, return_indices=True)
+            assert np.array_equal(y, ref.numpy())
+            # position inside the window -> flat index into the input plane (no ties in random data)
+            Ho, Wo = y.shape[2:]
+            i = np.arange(Ho)[:, None] * s[0] - p + arg // k[1]
+            j = np.arange(Wo)[None, :] * s[1] - p + arg % k[1]
+            assert np.array_equal(i * xg.shape[3] + j, idx.numpy())
+
+
+def test_pool_max_takes_first_of_equal_values_and_skips_padding():
+    xg = np.zeros((1, 1, 4, 4), np.float32)
+    y, arg = oracle.layers.pool_fwd_global(xg, (2, 2), (2, 2), ((0, 0), (0, 0)), "max")
+    assert np.all(arg == 0)
+    xg = -np.ones((1, 1, 4, 4), np.float32)                   # padding must not win over negative data
+    y, arg = oracle.layers.pool_fwd_global(xg, (3, 3), (2, 2), ((1, 1), (1, 1)), "max")
+    assert np.all(y == -1.0) and arg[0, 0, 0, 0] == 4 and arg[0, 0, 1, 1] == 0
+
+
+@pytest.mark.parametrize("case", POOL_CASES, ids=[str(c[:2]) for c in POOL_CASES])
+@pytest.mark.parametrize("mode", ["avg", "max"])
+def test_pool_distributed_forward_equals_sequential_layer(case, mode):
+    gs, ps, k, s, pad = case
+    part, geo, xg, xs = _pool_setup(case, 5)
+    yg, ag = oracle.layers.pool_fwd_global(xg, k, s, pad, mode)
+    ys, ar = oracle.layers.pool_fwd(part, geo, xs, k, s, pad, mode)
+    for w in range(part.num_workers):
+        assert np.array_equal(ys[w], yg[_out_block(geo, part, w)])
+        if mode == "max":
+            assert np.array_equal(ar[w], ag[_out_block(geo, part, w)])
+
+
+@pytest.mark.parametrize("case", POOL_CASES, ids=[str(c[:2]) for c in POOL_CASES])
+@pytest.mark.parametrize("mode", ["avg", "max"])
+def test_pool_adjoint_is_transpose_and_partition_invariant(case, mode):
+    gs, ps, k, s, pad = case
+    part, geo, xg, xs = _pool_setup(case, 9)
+    yg, ag = oracle.layers.pool_fwd_global(xg, k, s, pad, mode)
+    dyg = inputs.integers(yg.shape, 33)
+    dxg = oracle.layers.pool_adj_global(dyg, gs[2:], k, s, pad, mode, ag)
+    # brute force: column e of the forward operator (for max: of its Jacobian) applied to dy
+    if np.prod(gs) <= 400:
+        for e in range(0, int(np.prod(gs)), 7):
+            if mode == "avg":
+                u = np.zeros(gs, np.float32)
+                u.reshape(-1)[e] = 1.0
+                col, _ = oracle.layers.pool_fwd_global(u, k, s, pad, "avg")
+                want = float(np.sum(col.astype(np.float64) * dyg))
+            else:
+                idx = np.unravel_index(e, gs)
+                Ho, Wo = yg.shape[2:]
+                i = np.arange(Ho)[:, None] * s[0] - pad[0][0] + ag[idx[0], idx[1]] // k[1]
+                j = np.arange(Wo)[None, :] * s[1] - pad[1][0] + ag[idx[0], idx[1]] % k[1]
+                want = float(np.sum(dyg[idx[0], idx[1]][(i == idx[2]) & (j == idx[3])]))
+            assert abs(float(dxg.reshape(-1)[e]) - want) <= 1e-6 * max(1.0, abs(want))
+    # the distributed adjoint (local adjoint, then H*) gives the same tensor for every partition
+    dys = [dyg[_out_block(geo, part, w)] for w in range(part.num_workers)]
+    ars = None if mode == "avg" else [ag[_out_block(geo, part, w)] for w in range(part.num_workers)]
+    dxs = oracle.layers.pool_adj(part, geo, dys, k, s, pad, mode, ars)
+    got = oracle.assemble_global(part, dxs)
+    assert np.max(np.abs(got - dxg)) <= 4 * 2.0 ** -24 * max(1.0, np.max(np.abs(dxg)))
+    for w in range(part.num_workers):                          # ghosts are zero on exit
+        g = dxs[w].copy()
+        g[part.bulk_slices(w)] = 0
+        assert not g.any()
+    if mode == "max":                                          # every dy lands in exactly one cell
+        assert np.sum(got.astype(np.float64)) == np.sum(dyg.astype(np.float64))
+
+
+@pytest.mark.parametrize("case", POOL_CASES[:4], ids=[str(c[:2]) for c in POOL_CASES[:4]])
+def test_pool_avg_dot_test(case):
+    gs, ps, k, s, pad = case
+    part, geo, xg, xs = _pool_setup(case, 21)
+    xs = oracle.scatter_global(part, xg)                       # the operator acts on the bulk; ghosts are overwritten
+    ys, _ = oracle.layers.pool_fwd(part, geo, xs, k, s, pad, "avg")
+    dys = [inputs.normal(y.shape, 40 + w) for w, y in enumerate(ys)]
+    dxs = oracle.layers.pool_adj(part, geo, dys, k, s, pad, "avg")
+    assert oracle.adjoint_test_ratio(ys, dys, xs, dxs) < 1e-6
