@@ -203,6 +203,37 @@ distdl_status_t distdl_conv_adj(const distdl_partition_t *p, const void *const *
                                 int32_t kh, int32_t kw, void *const *dx, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Distributed pooling layer, feature-space partition only (Section 4, "Sparse layers": pooling
+ * layers follow the convolution algorithms; Section 3 / Appendix B: for a strided kernel the halo
+ * widths differ from worker to worker and owned inputs may go unused, Figs. B2-B4).
+ *
+ * p: rank-4 NCHW F32 partition of shape 1 x 1 x Ph x Pw (at most 32 workers) made by
+ *    distdl_partition_create_general with, in each feature dimension, exactly the widths
+ *    distdl_halo_widths_1d gives for (kernel, stride, dilation 1, padding) -- else
+ *    DISTDL_ERR_SHAPE.  Kernel extents up to 16.  Worker (r, c) owns block r / c of the evenly
+ *    split output rows / columns.
+ * pool_fwd = H on x in place (its ghosts are overwritten), then the local layer:
+ *    AVG: y = mean of the kh x kw window of the zero-padded tensor (padding counts in the
+ *         divisor), summed in fp32 in row-major window order, times 1/(kh*kw);
+ *    MAX: y = largest value of the window clipped to the tensor; argmax (may be NULL) receives
+ *         a*kw + b of the first largest value in row-major order of the unclipped window.
+ *    x[w]: padded shards.  y[w], argmax[w]: [N, C, oh, ow] F32 / int32.
+ * pool_adj = adjoint of the local layer into every cell of the padded dx[w] (a cell sums, in
+ *    ascending output order and in fp32, dy/(kh*kw) over the local outputs whose window holds it;
+ *    for MAX: dy of the outputs whose recorded position is that cell), then H* on dx in place:
+ *    ghost contributions are added into the owners' bulk and the ghosts are cleared.
+ * ---------------------------------------------------------------------- */
+typedef enum { DISTDL_POOL_AVG = 0, DISTDL_POOL_MAX = 1 } distdl_pool_mode_t;
+distdl_status_t distdl_pool_fwd(const distdl_partition_t *p, void *const *x, int32_t kh, int32_t kw,
+                                int32_t sh, int32_t sw, int32_t pad_h_lo, int32_t pad_h_hi,
+                                int32_t pad_w_lo, int32_t pad_w_hi, int32_t mode, void *const *y,
+                                void *const *argmax, void *stream);
+distdl_status_t distdl_pool_adj(const distdl_partition_t *p, const void *const *dy,
+                                const void *const *argmax, int32_t kh, int32_t kw, int32_t sh,
+                                int32_t sw, int32_t pad_h_lo, int32_t pad_h_hi, int32_t pad_w_lo,
+                                int32_t pad_w_hi, int32_t mode, void *const *dx, void *stream);
+
+/* ------------------------------------------------------------------------
  * Distributed affine layer on a Pfo x Pfi worker grid (Section 4, "Dense layers": forward and
  * adjoint affine algorithms).
  *

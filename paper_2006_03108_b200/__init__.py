@@ -65,6 +65,8 @@ def lib():
     L.distdl_halo_fwd_noalloc.argtypes = [c_i32, pi64, pi32, pi32, pi32, c_i32, pvp, vp]
     L.distdl_conv_fwd.argtypes = [vp, pvp, vp, vp, c_i32, c_i32, pvp, vp]
     L.distdl_conv_adj.argtypes = [vp, pvp, vp, c_i32, c_i32, pvp, vp]
+    L.distdl_pool_fwd.argtypes = [vp, pvp] + [c_i32] * 9 + [pvp, pvp, vp]
+    L.distdl_pool_adj.argtypes = [vp, pvp, pvp] + [c_i32] * 9 + [pvp, vp]
     L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
     L.distdl_affine_adj.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, vp]
     L.distdl_device_status.argtypes = [vp]
@@ -250,6 +252,22 @@ def conv_fwd(part, x, w, bias, y, stream=None):
 def conv_adj(part, dy, w, dx, stream=None):
     kh, kw = int(w.shape[-2]), int(w.shape[-1])
     _check(lib().distdl_conv_adj(part.handle, _ptr_array(dy), _ptr(w), kh, kw, _ptr_array(dx), _stream(stream)))
+
+
+POOL_AVG, POOL_MAX = 0, 1
+
+
+def pool_fwd(part, x, kernel, stride, pad, mode, y, argmax=None, stream=None):
+    """kernel = (kh, kw), stride = (sh, sw), pad = ((lo_h, hi_h), (lo_w, hi_w)); x is updated in place by H."""
+    a = None if argmax is None else _ptr_array(argmax)
+    _check(lib().distdl_pool_fwd(part.handle, _ptr_array(x), kernel[0], kernel[1], stride[0], stride[1], pad[0][0],
+                                 pad[0][1], pad[1][0], pad[1][1], mode, _ptr_array(y), a, _stream(stream)))
+
+
+def pool_adj(part, dy, argmax, kernel, stride, pad, mode, dx, stream=None):
+    a = None if argmax is None else _ptr_array(argmax)
+    _check(lib().distdl_pool_adj(part.handle, _ptr_array(dy), a, kernel[0], kernel[1], stride[0], stride[1], pad[0][0],
+                                 pad[0][1], pad[1][0], pad[1][1], mode, _ptr_array(dx), _stream(stream)))
 
 
 def affine_fwd(nb, nfi, nfo, pfo, pfi, x, w, bias, y, stream=None):

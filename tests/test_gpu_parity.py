@@ -369,3 +369,87 @@ def test_affine_fwd_and_adj(case, integer):
         distdl.device_status()
         r = oracle.adjoint_test_ratio([host(t) for t in y0], dyf, xf, dx)
         assert r < 1e-4
+
+
+# --------------------------------------------------------------------------
+# Distributed pooling layer (unbalanced halos)
+# --------------------------------------------------------------------------
+
+POOL_CASES = [
+    # global shape, partition, kernel, stride, padding
+    ((2, 3, 11, 10), (1, 1, 3, 2), (2, 2), (2, 2), ((0, 0), (0, 0))),
+    ((1, 2, 20, 17), (1, 1, 6, 3), (3, 3), (2, 2), ((1, 1), (1, 1))),
+    ((1, 1, 12, 12), (1, 1, 2, 2), (3, 2), (1, 2), ((1, 0), (0, 1))),
+    ((1, 1, 1, 20), (1, 1, 1, 6), (1, 2), (1, 2), ((0, 0), (0, 0))),      # Fig. B4
+    ((2, 2, 130, 203), (1, 1, 4, 4), (3, 3), (2, 2), ((1, 1), (1, 1))),   # several thread-block tiles, ragged
+    ((1, 4, 97, 64), (1, 1, 2, 3), (5, 5), (3, 3), ((2, 2), (2, 2))),
+    ((1, 1, 64, 64), (1, 1, 1, 1), (2, 2), (2, 2), ((0, 0), (0, 0))),
+]
+
+
+def _pool_parts(case):
+    gs, ps, k, s, pad = case
+    opart, geo = oracle.pool_partition(gs, ps, k, s, pad)
+    gpart = distdl.Partition(gs, ps, [list(h) for h in opart.hlo], [list(h) for h in opart.hhi])
+    return opart, geo, gpart
+
+
+@pytest.mark.parametrize("case", POOL_CASES, ids=[str(c[:2]) for c in POOL_CASES])
+@pytest.mark.parametrize("mode", ["avg", "max"])
+def test_pool_fwd_and_adj(case, mode):
+    gs, ps, k, s, pad = case
+    opart, geo, gpart = _pool_parts(case)
+    code = distdl.POOL_AVG if mode == "avg" else distdl.POOL_MAX
+    xg = inputs.normal(gs, 61)
+    xs = oracle.scatter_global(opart, xg, fill=lambda w: inputs.normal(opart.padded_shape(w), 700 + w))   # garbage ghosts
+    ys_ref, arg_ref = oracle.pool_fwd(opart, geo, xs, k, s, pad, mode)
+    x_d = [dev(a) for a in xs]
+    y_d = [torch.full(tuple(y.shape), -9.0, device=DEV) for y in ys_ref]
+    a_d = [torch.full(tuple(y.shape), -1, dtype=torch.int32, device=DEV) for y in ys_ref] if mode == "max" else None
+    distdl.pool_fwd(gpart, x_d, k, s, pad, code, y_d, a_d)
+    torch.cuda.synchronize()
+    # the ghosts of x now hold what H puts there
+    for got, ref in zip(x_d, oracle.halo_fwd_definition(opart, xs)):
+        assert same_bits(host(got), ref)
+    for w, (got, ref) in enumerate(zip(y_d, ys_ref)):
+        if mode == "max":
+            assert same_bits(host(got), ref)
+            assert np.array_equal(host(a_d[w]), arg_ref[w])
+        else:
+            # fp32 sum of kh*kw terms and one multiplication against the fp64 sum rounded once
+            bound = (k[0] * k[1] + 2) * 2.0 ** -24 * np.max(np.abs(xg)) + 1e-30
+            assert got.shape == ref.shape and np.max(np.abs(host(got) - ref), initial=0.0) <= bound
+
+    dys = [inputs.normal(y.shape, 800 + w) for w, y in enumerate(ys_ref)]
+    dx_ref = oracle.pool_adj(opart, geo, dys, k, s, pad, mode, arg_ref)
+    dy_d = [dev(a) for a in dys]
+    arg_in = None if mode == "avg" else [dev(a) for a in arg_ref]
+    dx_d = [torch.full(tuple(opart.padded_shape(w)), 5.0, device=DEV) for w in range(opart.num_workers)]
+    distdl.pool_adj(gpart, dy_d, arg_in, k, s, pad, code, dx_d)
+    torch.cuda.synchronize()
+    dymax = max([float(np.max(np.abs(d), initial=0.0)) for d in dys])
+    terms = ((k[0] + s[0] - 1) // s[0]) * ((k[1] + s[1] - 1) // s[1])      # outputs whose window holds one cell
+    for w, (got, ref) in enumerate(zip(dx_d, dx_ref)):
+        g = host(got)
+        if mode == "max" and terms == 1:
+            assert same_bits(g, ref)                                       # pure routing, then the fixed-order H*
+        else:
+            assert np.max(np.abs(g - ref), initial=0.0) <= 4 * (terms + 2) * 2.0 ** -24 * dymax
+        ghosts = g.copy()
+        ghosts[opart.bulk_slices(w)] = 0
+        assert not ghosts.any()
+    if mode == "avg":
+        # dot-product test of the pair on the device results (the operator acts on the bulk of x)
+        x0 = oracle.scatter_global(opart, xg)
+        r = oracle.adjoint_test_ratio([host(t) for t in y_d], dys, x0, [host(t) for t in dx_d])
+        assert r < 1e-5
+
+
+def test_pool_rejects_partitions_with_other_widths():
+    gs, ps = (1, 1, 16, 16), (1, 1, 2, 2)
+    part = distdl.Partition(gs, ps, [0, 0, 1, 1], [0, 0, 1, 1])
+    x = [torch.zeros(tuple(part.padded_shape(w)), device=DEV) for w in range(4)]
+    y = [torch.zeros(1, 1, 4, 4, device=DEV) for _ in range(4)]
+    with pytest.raises(distdl.DistdlError) as e:
+        distdl.pool_fwd(part, x, (2, 2), (2, 2), ((0, 0), (0, 0)), distdl.POOL_AVG, y)
+    assert e.value.status == 2          # DISTDL_ERR_SHAPE
