@@ -120,6 +120,33 @@ class Workload:
         self.bytes_per_step = sum(o[2] for o in self.ops)
         self.launches_per_step = sum(o[4] for o in self.ops)
 
+        # Distributed pooling layer (3 x 3 max pooling, stride 2, padding 1: ghost widths (1, 0) per worker):
+        # timed on its own after the step, reported under "extra_ops", not part of `value`.
+        k, st, pad = (3, 3), (2, 2), ((1, 1), (1, 1))
+        gsp = (nc, 16, 1024, 1024)
+        hl, hh = [0, 0], [0, 0]
+        for dim in (2, 3):
+            lo, hi, _, _ = d.halo_widths_1d(gsp[dim], 4, k[dim - 2], st[dim - 2], 1, pad[dim - 2][0], pad[dim - 2][1])
+            hl.append(lo)
+            hh.append(hi)
+        self.ppart = d.Partition(gsp, (1, 1, 4, 4), hl, hh)
+        oh = ((gsp[2] + 2 - 3) // 2 + 1) // 4
+        P = self.ppart.num_workers
+        self.p_x = [n(*self.ppart.padded_shape(w)) for w in range(P)]
+        self.p_y = [torch.empty(nc, 16, oh, oh, device=dev) for _ in range(P)]
+        self.p_arg = [torch.zeros(nc, 16, oh, oh, dtype=torch.int32, device=dev) for _ in range(P)]
+        self.p_dy = [n(nc, 16, oh, oh) for _ in range(P)]
+        self.p_dx = [torch.empty(*self.ppart.padded_shape(w), device=dev) for w in range(P)]
+        out_b = sum(t.numel() for t in self.p_y) * 4
+        need_b = P * nc * 16 * ((oh - 1) * 2 + 3) ** 2 * 4
+        pad_b = sum(t.numel() for t in self.p_dx) * 4
+        self.extra_ops = [
+            ("pool_fwd", lambda: d.pool_fwd(self.ppart, self.p_x, k, st, pad, d.POOL_MAX, self.p_y, self.p_arg),
+             self.ppart.halo_stats(False)[2] + need_b + 2 * out_b, 0, 2, "hbm"),
+            ("pool_adj", lambda: d.pool_adj(self.ppart, self.p_dy, self.p_arg, k, st, pad, d.POOL_MAX, self.p_dx),
+             2 * out_b + pad_b + self.ppart.halo_stats(True)[2], 0, 2, "hbm"),
+        ]
+
     def _conv_outputs(self):
         gs = self.cpart.global_shape
         return gs[0] * gs[1] * gs[2] * gs[3]
@@ -340,7 +367,7 @@ def main():
 
     if args.profile_op:
         wl = Workload(dev, small=True)
-        op = [o for o in wl.ops if o[0] == args.profile_op]
+        op = [o for o in wl.ops + wl.extra_ops if o[0] == args.profile_op]
         if not op:
             raise SystemExit("unknown operator %r" % args.profile_op)
         for _ in range(3):
@@ -385,6 +412,28 @@ def main():
     ms_per_step = elapsed_ms / args.steps
     value = world * wl.bytes_per_step / (ms_per_step * 1e-3) / 1e9
 
+    # ---- the pooling layer, timed on its own (not part of the step or of `value`) ----
+    extra_ms = []
+    for name, call, _, _, _, _ in wl.extra_ops:
+        for _ in range(3):
+            call()
+        reps = 20
+        xe = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        torch.cuda.synchronize()
+        for r in range(reps):
+            xe[r].record()
+            call()
+            wl.ops[0][1]()          # 0.6 GB of other traffic between two launches (the inputs alone exceed L2 anyway)
+        xe[reps].record()
+        torch.cuda.synchronize()
+        b0 = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        for r in range(reps):
+            b0[r].record()
+            wl.ops[0][1]()
+        b0[reps].record()
+        torch.cuda.synchronize()
+        extra_ms.append((xe[0].elapsed_time(xe[reps]) - b0[0].elapsed_time(b0[reps])) / reps)
+
     # ---- end to end: inputs from pinned host memory, results back to the host, every step ----
     wl.e2e_setup()
     wl.e2e_step()
@@ -412,6 +461,10 @@ def main():
             if bound == "tensor":
                 entry["frac_tensor"] = round(flops / ms / 1e9 / peaks["bf16_sustained"], 4)
             ops[name] = entry
+        extra = {}
+        for (name, _, nbytes, _, _, bound), ms in zip(wl.extra_ops, extra_ms):
+            extra[name] = {"ms": round(ms, 5), "gbs": round(nbytes / ms / 1e6, 1), "bound": bound,
+                           "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm"], 4)}
         # dominant kernel = the launch with the largest share of the step
         top = max(range(nops), key=lambda i: per_op_ms[i])
         tname, _, tbytes, _, _, tbound = wl.ops[top]
@@ -435,6 +488,9 @@ def main():
             "halo_bcast_reduce": {"gbs": round(dm_bytes / dm_ms / 1e6, 1),
                                   "frac_of_hbm_peak": round(dm_bytes / dm_ms / 1e6 / peaks["hbm"], 4)},
             "ops": ops,
+            "extra_ops": {"note": "3x3 max pooling, stride 2, padding 1 on fp32 16x16x1024x1024 over 4x4 workers "
+                                  "(H + local kernel, local adjoint + H*); timed separately, not part of value",
+                          **extra},
             "roofline": roofline,
             "clocks": clocks,
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes,

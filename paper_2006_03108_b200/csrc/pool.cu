@@ -108,6 +108,186 @@ pool_adj_kernel(const __grid_constant__ PoolParams P, int tiles_x, int tiles_y) 
     S.out[((size_t)plane * S.ph + p) * S.pw + q] = acc;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Variants with the kernel and stride fixed at compile time (2 x 2 / 2 and 3 x 3 / 2, the pooling
+// layers of the usual networks): index arithmetic in shifts, and four outputs (forward) or cells
+// (adjoint) per thread, 32 columns apart, so that the lanes of a warp always touch neighbouring
+// addresses.  Same sums in the same order as the general kernels above.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPoolPerThread = 4;
+
+template <int KH, int KW, int SH, int SW, int MODE>
+__global__ void __launch_bounds__(kPoolThreadsX *kPoolThreadsY)
+pool_fwd_fixed(const __grid_constant__ PoolParams P, int tiles_x, int tiles_y) {
+    const PoolShard &S = P.s[blockIdx.y];
+    int rest = blockIdx.x;
+    const int tx = rest % tiles_x;
+    rest /= tiles_x;
+    const int ty = rest % tiles_y;
+    const int plane = rest / tiles_y;
+    const int jb = tx * kPoolThreadsX * kPoolPerThread + threadIdx.x, i = ty * kPoolThreadsY + threadIdx.y;
+    if (i >= S.oh) return;
+    const int r0 = S.i0 + i * SH;
+    const float *row = S.in + ((size_t)plane * S.ph + r0) * S.pw + S.j0;
+    float *orow = S.out + ((size_t)plane * S.oh + i) * S.ow;
+    int32_t *arow = (MODE == DISTDL_POOL_MAX && S.arg) ? S.arg + ((size_t)plane * S.oh + i) * S.ow : nullptr;
+    bool row_in[KH];
+#pragma unroll
+    for (int a = 0; a < KH; ++a) row_in[a] = S.g0h + r0 + a >= 0 && S.g0h + r0 + a < P.hg;
+    bool rows_inside = true;
+#pragma unroll
+    for (int a = 0; a < KH; ++a) rows_inside = rows_inside && row_in[a];
+#pragma unroll
+    for (int u = 0; u < kPoolPerThread; ++u) {
+        const int j = jb + u * kPoolThreadsX;
+        if (j >= S.ow) break;
+        const float *src = row + j * SW;
+        const int gj0 = S.g0w + S.j0 + j * SW;
+        float acc = 0.f;
+        int where = -1;
+        if (MODE == DISTDL_POOL_AVG) {
+#pragma unroll
+            for (int a = 0; a < KH; ++a)
+#pragma unroll
+                for (int b = 0; b < KW; ++b) acc = __fadd_rn(acc, src[a * S.pw + b]);
+            acc = __fmul_rn(acc, 1.0f / (float)(KH * KW));
+        } else if (rows_inside && gj0 >= 0 && gj0 + KW <= P.wg) {
+            // the whole window lies inside the tensor: no cell to exclude
+            acc = src[0];
+            where = 0;
+#pragma unroll
+            for (int a = 0; a < KH; ++a)
+#pragma unroll
+                for (int b = 0; b < KW; ++b) {
+                    if (a == 0 && b == 0) continue;
+                    const float v = src[a * S.pw + b];
+                    if (v > acc) {
+                        acc = v;
+                        where = a * KW + b;
+                    }
+                }
+        } else {
+#pragma unroll
+            for (int a = 0; a < KH; ++a)
+#pragma unroll
+                for (int b = 0; b < KW; ++b) {
+                    const float v = src[a * S.pw + b];
+                    if (row_in[a] && gj0 + b >= 0 && gj0 + b < P.wg && (where < 0 || v > acc)) {
+                        acc = v;
+                        where = a * KW + b;
+                    }
+                }
+        }
+        orow[j] = acc;
+        if (arow) arow[j] = where < 0 ? 0 : where;
+    }
+}
+
+// Adjoint: a thread owns the SH x SW cells {i0 + SH*gi + r, j0 + SW*gj + c}.  The outputs whose window holds
+// cell (r, c) of the group are (gi - t, gj - v) with window positions a = r + t*SH < KH, b = c + v*SW < KW, all
+// known at compile time; the thread loads the NI x NJ candidate outputs once and every cell picks its terms
+// (ascending output order = descending t, v).  tiles count groups: row group = first group + tile row, and so on.
+template <int KH, int KW, int SH, int SW, int MODE>
+__global__ void __launch_bounds__(kPoolThreadsX *kPoolThreadsY)
+pool_adj_fixed(const __grid_constant__ PoolParams P, int tiles_x, int tiles_y) {
+    const PoolShard &S = P.s[blockIdx.y];
+    int rest = blockIdx.x;
+    const int tx = rest % tiles_x;
+    rest /= tiles_x;
+    const int ty = rest % tiles_y;
+    const int plane = rest / tiles_y;
+    constexpr int NI = (KH + SH - 1) / SH, NJ = (KW + SW - 1) / SW;
+    // the first group holds padded row / column 0
+    const int gi = div_floor(-S.i0, SH) + ty * kPoolThreadsY + (int)threadIdx.y;
+    const int gjb = div_floor(-S.j0, SW) + tx * kPoolThreadsX * kPoolPerThread + (int)threadIdx.x;
+    const int p0 = S.i0 + gi * SH;
+    if (p0 >= S.ph) return;
+    const float *dy = S.in + (size_t)plane * S.oh * S.ow;
+    const int32_t *arg = MODE == DISTDL_POOL_MAX ? S.arg + (size_t)plane * S.oh * S.ow : nullptr;
+    float *oplane = S.out + (size_t)plane * S.ph * S.pw;
+#pragma unroll
+    for (int u = 0; u < kPoolPerThread; ++u) {
+        const int gj = gjb + u * kPoolThreadsX;
+        const int q0 = S.j0 + gj * SW;
+        if (q0 >= S.pw) break;
+        float g[NI][NJ];
+        int code[NI][NJ];          // MAX: recorded position, -1 for an absent output; AVG: 0 present, -1 absent
+        const bool interior = gi - (NI - 1) >= 0 && gi < S.oh && gj - (NJ - 1) >= 0 && gj < S.ow && p0 >= 0 &&
+                              p0 + SH <= S.ph && q0 >= 0 && q0 + SW <= S.pw;
+        if (interior) {
+            // every candidate output exists and every cell of the group lies in the shard: no tests, 32-bit offsets
+            const uint32_t o = (uint32_t)(gi * S.ow + gj);
+#pragma unroll
+            for (int t = 0; t < NI; ++t)
+#pragma unroll
+                for (int v = 0; v < NJ; ++v) {
+                    g[t][v] = dy[o - (uint32_t)(t * S.ow + v)];
+                    code[t][v] = MODE == DISTDL_POOL_MAX ? arg[o - (uint32_t)(t * S.ow + v)] : 0;
+                }
+            float *dst = oplane + (uint32_t)(p0 * S.pw + q0);
+#pragma unroll
+            for (int r = 0; r < SH; ++r)
+#pragma unroll
+                for (int c = 0; c < SW; ++c) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int t = NI - 1; t >= 0; --t)
+#pragma unroll
+                        for (int v = NJ - 1; v >= 0; --v) {
+                            if (r + t * SH >= KH || c + v * SW >= KW) continue;      // compile-time
+                            if (MODE == DISTDL_POOL_AVG) acc = __fadd_rn(acc, g[t][v]);
+                            else if (code[t][v] == (r + t * SH) * KW + (c + v * SW)) acc = __fadd_rn(acc, g[t][v]);
+                        }
+                    if (MODE == DISTDL_POOL_AVG) acc = __fmul_rn(acc, 1.0f / (float)(KH * KW));
+                    dst[r * S.pw + c] = acc;
+                }
+            continue;
+        }
+#pragma unroll
+        for (int t = 0; t < NI; ++t)
+#pragma unroll
+            for (int v = 0; v < NJ; ++v) {
+                const int i = gi - t, j = gj - v;
+                const bool in = i >= 0 && i < S.oh && j >= 0 && j < S.ow;
+                g[t][v] = in ? dy[i * S.ow + j] : 0.f;
+                code[t][v] = !in ? -1 : (MODE == DISTDL_POOL_MAX ? arg[i * S.ow + j] : 0);
+            }
+#pragma unroll
+        for (int r = 0; r < SH; ++r) {
+            const int p = p0 + r;
+            if (p < 0 || p >= S.ph) continue;
+#pragma unroll
+            for (int c = 0; c < SW; ++c) {
+                const int q = q0 + c;
+                if (q < 0 || q >= S.pw) continue;
+                float acc = 0.f;
+#pragma unroll
+                for (int t = NI - 1; t >= 0; --t)
+#pragma unroll
+                    for (int v = NJ - 1; v >= 0; --v) {
+                        if (r + t * SH >= KH || c + v * SW >= KW) continue;      // compile-time
+                        const bool take = MODE == DISTDL_POOL_AVG ? code[t][v] == 0
+                                                                  : code[t][v] == (r + t * SH) * KW + (c + v * SW);
+                        if (take) acc = __fadd_rn(acc, g[t][v]);
+                    }
+                if (MODE == DISTDL_POOL_AVG) acc = __fmul_rn(acc, 1.0f / (float)(KH * KW));
+                oplane[(size_t)p * S.pw + q] = acc;
+            }
+        }
+    }
+}
+
+template <int KH, int KW, int SH, int SW>
+static void launch_pool_fixed(const PoolParams &P, dim3 grid, dim3 block, int tiles_x, int tiles_y, bool adjoint, cudaStream_t s) {
+    if (!adjoint) {
+        if (P.mode == DISTDL_POOL_AVG) pool_fwd_fixed<KH, KW, SH, SW, DISTDL_POOL_AVG><<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+        else pool_fwd_fixed<KH, KW, SH, SW, DISTDL_POOL_MAX><<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+    } else {
+        if (P.mode == DISTDL_POOL_AVG) pool_adj_fixed<KH, KW, SH, SW, DISTDL_POOL_AVG><<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+        else pool_adj_fixed<KH, KW, SH, SW, DISTDL_POOL_MAX><<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+    }
+}
+
 struct PoolDim {
     std::vector<int64_t> out_start, out_size;
     std::vector<int32_t> hlo, hhi;
@@ -198,7 +378,15 @@ static distdl_status_t pool_impl(const distdl_partition *p, const void *const *i
         max_cols = std::max<int64_t>(max_cols, adjoint ? S.pw : S.ow);
     }
     cudaStream_t s = (cudaStream_t)stream;
-    const int tiles_x = (int)((max_cols + kPoolThreadsX - 1) / kPoolThreadsX);
+    // the compile-time variants handle four outputs / cells per thread along a row
+    const int fixed = (kh == 2 && kw == 2 && sh == 2 && sw == 2) ? 1 : (kh == 3 && kw == 3 && sh == 2 && sw == 2) ? 2 : 0;
+    const int per_thread = fixed ? kPoolPerThread : 1;
+    if (fixed && adjoint) {
+        // the compile-time adjoint walks groups of sh x sw cells; the group lattice starts up to one group before cell 0
+        max_rows = max_rows / sh + 2;
+        max_cols = max_cols / sw + 2;
+    }
+    const int tiles_x = (int)((max_cols + kPoolThreadsX * per_thread - 1) / (kPoolThreadsX * per_thread));
     const int tiles_y = (int)((max_rows + kPoolThreadsY - 1) / kPoolThreadsY);
     const int64_t blocks = (int64_t)tiles_x * tiles_y * P.planes;
     if (blocks >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
@@ -207,12 +395,15 @@ static distdl_status_t pool_impl(const distdl_partition *p, const void *const *i
         // H in place on the padded input, then the local layer
         st = distdl_halo_fwd(p, const_cast<void *const *>(reinterpret_cast<const void *const *>(in)), stream);
         if (st != DISTDL_OK) return st;
-        if (blocks > 0) pool_fwd_kernel<<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
-        DISTDL_CUDA_CHECK(cudaGetLastError());
-        return DISTDL_OK;
     }
-    if (blocks > 0) pool_adj_kernel<<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+    if (blocks > 0) {
+        if (fixed == 1) launch_pool_fixed<2, 2, 2, 2>(P, grid, block, tiles_x, tiles_y, adjoint, s);
+        else if (fixed == 2) launch_pool_fixed<3, 3, 2, 2>(P, grid, block, tiles_x, tiles_y, adjoint, s);
+        else if (!adjoint) pool_fwd_kernel<<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+        else pool_adj_kernel<<<grid, block, 0, s>>>(P, tiles_x, tiles_y);
+    }
     DISTDL_CUDA_CHECK(cudaGetLastError());
+    if (!adjoint) return DISTDL_OK;
     return distdl_halo_adj(p, out, stream);
 }
 
