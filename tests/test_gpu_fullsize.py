@@ -121,3 +121,45 @@ def test_affine_full_size():
         assert np.max(np.abs(g - r)) / np.max(np.abs(r)) < 2e-2
         assert np.linalg.norm(g - r) / np.linalg.norm(r) < 1e-4
     assert oracle.adjoint_test_ratio([host(t) for t in y], dyf, xf, [host(t) for t in dx]) < 1e-4
+
+
+def test_pool_full_size_on_sampled_planes():
+    # the configuration bench.py times: 3 x 3 max pooling, stride 2, padding 1, ghost widths (1, 0) per worker
+    gs, ps, k, s, pad = (16, 16, 1024, 1024), (1, 1, 4, 4), (3, 3), (2, 2), ((1, 1), (1, 1))
+    sub = (1, 1, 1024, 1024)
+    opart, geo = oracle.pool_partition(sub, ps, k, s, pad)
+    gpart = distdl.Partition(gs, ps, [list(h) for h in opart.hlo], [list(h) for h in opart.hhi])
+    g = torch.Generator(device=DEV)
+    g.manual_seed(7)
+    xs = [torch.randn(*gpart.padded_shape(w), device=DEV, generator=g) for w in range(16)]
+    ys = [torch.empty(16, 16, 128, 128, device=DEV) for _ in range(16)]
+    args = [torch.full((16, 16, 128, 128), -1, dtype=torch.int32, device=DEV) for _ in range(16)]
+    dys = [torch.randn(16, 16, 128, 128, device=DEV, generator=g) for _ in range(16)]
+    dxs = [torch.full(tuple(gpart.padded_shape(w)), 7.0, device=DEV) for w in range(16)]
+    x_before = {(n, c): [host(t[n:n + 1, c:c + 1]) for t in xs] for n, c in [(0, 0), (5, 11), (15, 15)]}
+    distdl.pool_fwd(gpart, xs, k, s, pad, distdl.POOL_MAX, ys, args)
+    distdl.pool_adj(gpart, dys, args, k, s, pad, distdl.POOL_MAX, dxs)
+    torch.cuda.synchronize()
+    for (n, c), x1 in x_before.items():
+        yref, aref = oracle.pool_fwd(opart, geo, x1, k, s, pad, "max")
+        dy1 = [host(t[n:n + 1, c:c + 1]) for t in dys]
+        dxref = oracle.pool_adj(opart, geo, dy1, k, s, pad, "max", aref)
+        for w in range(16):
+            assert host(ys[w][n:n + 1, c:c + 1]).tobytes() == yref[w].tobytes()
+            assert np.array_equal(host(args[w][n:n + 1, c:c + 1]), aref[w])
+            got = host(dxs[w][n:n + 1, c:c + 1])
+            # up to four routed values per cell summed in fp32, then the fixed-order sums of H*
+            assert np.max(np.abs(got - dxref[w])) <= 8 * 2.0 ** -24 * 4 * float(np.max(np.abs(dy1[w])))
+    # properties at full size: every recorded position is a window position, ghosts of dx are zero,
+    # and the adjoint routes all of dy (sum preserved up to fp32 rounding)
+    for w in range(16):
+        assert int(args[w].min()) >= 0 and int(args[w].max()) <= 8
+        lo, hi = opart.widths(w)
+        t = dxs[w]
+        if lo[2]:
+            assert float(t[:, :, :lo[2], :].abs().max()) == 0.0
+        if lo[3]:
+            assert float(t[:, :, :, :lo[3]].abs().max()) == 0.0
+    total_dx = sum(float(t.double().sum()) for t in dxs)
+    total_dy = sum(float(t.double().sum()) for t in dys)
+    assert abs(total_dx - total_dy) <= 1e-6 * sum(float(t.double().abs().sum()) for t in dys)
