@@ -2,7 +2,8 @@
 
 TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, deliberately naive
 numpy restatement of what the operators compute (broadcast B, sum-reduce R = B*,
-halo exchange H, adjoint halo exchange H*, the distributed depthwise convolution,
+halo exchange H, adjoint halo exchange H*, the generalized all-to-all with scatter and
+gather as special cases, all-reduce, the distributed depthwise convolution,
 the distributed pooling layer and the distributed affine layer, each with its adjoint).  Nothing in the product
 package imports it; only the test-suite, the smoke check and the CPU-baseline leg
 of the benchmark may call it.  It shares no code, table or helper with the CUDA
@@ -29,6 +30,9 @@ from .primitives import (  # noqa: F401
     adjoint_test_ratio,
     assemble_global,
     scatter_global,
+    repartition_fwd,
+    repartition_adj,
+    allreduce,
 )
 from .layers import (  # noqa: F401
     conv_fwd,

@@ -282,3 +282,37 @@ def adjoint_test_ratio(Fx, y, x, Fsy):
     if den == 0.0:
         return 0.0
     return abs(lhs - rhs) / den
+
+
+# --------------------------------------------------------------------------
+# Generalized all-to-all (repartition), scatter / gather, all-reduce
+# (Section 3, "Scatter and Gather", "Sum-reduce and all-reduce", "Generalized all-to-all")
+# --------------------------------------------------------------------------
+
+def repartition_fwd(src_part: Partition, dst_part: Partition, shards):
+    """Generalized all-to-all: the same tensor, re-cut from one partition to another.
+
+    Every cell of the tensor is moved from the worker that owns it in `src_part`
+    to the worker that owns it in `dst_part` (a block permutation whose blocks are
+    send-receive copies).  Written as its plain meaning: put the source blocks
+    together, cut along the destination partition.  Both partitions carry no ghosts.
+    A source partition of a single worker gives the scatter, a destination
+    partition of a single worker the gather.
+    """
+    assert src_part.global_shape == dst_part.global_shape
+    return scatter_global(dst_part, assemble_global(src_part, shards))
+
+
+def repartition_adj(src_part: Partition, dst_part: Partition, dy_shards):
+    """Adjoint of the generalized all-to-all.
+
+    The operator is a permutation of cells (every copy is a move), so its adjoint
+    is its inverse: the all-to-all back from `dst_part` to `src_part`.
+    """
+    return scatter_global(src_part, assemble_global(dst_part, dy_shards))
+
+
+def allreduce(parts):
+    """All-reduce = broadcast after sum-reduce (self-adjoint): every worker ends up with
+    the fixed-order sum of all k realisations."""
+    return broadcast_fwd(sumreduce_fwd(parts), len(parts))

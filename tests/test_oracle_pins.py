@@ -579,3 +579,74 @@ def test_pool_avg_dot_test(case):
     dys = [inputs.normal(y.shape, 40 + w) for w, y in enumerate(ys)]
     dxs = oracle.layers.pool_adj(part, geo, dys, k, s, pad, "avg")
     assert oracle.adjoint_test_ratio(ys, dys, xs, dxs) < 1e-6
+
+
+# --------------------------------------------------------------------------
+# Generalized all-to-all, scatter / gather, all-reduce (Section 3)
+# --------------------------------------------------------------------------
+
+REPART_CASES = [
+    # global shape, source partition, destination partition
+    ((7, 9), (2, 1), (1, 3)),
+    ((6, 10), (3, 2), (2, 5)),
+    ((5, 4, 6), (1, 2, 3), (5, 1, 1)),
+    ((12,), (1,), (5,)),            # scatter
+    ((12,), (4,), (1,)),            # gather
+    ((4, 6), (2, 2), (2, 2)),       # identity
+]
+
+
+@pytest.mark.parametrize("case", REPART_CASES, ids=[str(c) for c in REPART_CASES])
+def test_repartition_is_a_permutation_with_inverse_adjoint(case):
+    gs, sp, dp = case
+    src, dst = Partition(gs, sp), Partition(gs, dp)
+    n = int(np.prod(gs))
+    sizes_s = [int(np.prod(src.padded_shape(w))) for w in range(src.num_workers)]
+    sizes_d = [int(np.prod(dst.padded_shape(w))) for w in range(dst.num_workers)]
+    assert sum(sizes_s) == n and sum(sizes_d) == n
+
+    def apply(fn, a, b, vec, sizes):
+        parts, at = [], 0
+        for w, z in enumerate(sizes):
+            parts.append(vec[at:at + z].reshape(a.padded_shape(w)))
+            at += z
+        return np.concatenate([p.reshape(-1) for p in fn(a, b, parts)]) if fn is oracle.repartition_fwd else \
+            np.concatenate([p.reshape(-1) for p in fn(b, a, parts)])
+
+    eye = np.eye(n, dtype=np.float32)
+    F = np.stack([apply(oracle.repartition_fwd, src, dst, eye[e], sizes_s) for e in range(n)], axis=1)
+    A = np.stack([apply(oracle.repartition_adj, dst, src, eye[e], sizes_d) for e in range(n)], axis=1)
+    assert np.all(F.sum(axis=0) == 1) and np.all(F.sum(axis=1) == 1) and set(np.unique(F)) <= {0.0, 1.0}
+    assert np.array_equal(A, F.T)                       # adjoint = transpose
+    assert np.array_equal(A @ F, eye)                   # = inverse: the round trip is the identity
+
+
+def test_repartition_transpose_scatter_gather_against_numpy_splits():
+    g = inputs.uniform_pm1((8, 12), 3)
+    rows, cols = Partition((8, 12), (4, 1)), Partition((8, 12), (1, 3))
+    out = oracle.repartition_fwd(rows, cols, np.split(g, 4, axis=0))      # row blocks -> column blocks
+    for got, ref in zip(out, np.split(g, 3, axis=1)):
+        assert np.array_equal(got, ref)
+    one, many = Partition((10,), (1,)), Partition((10,), (3,))
+    v = inputs.uniform_pm1((10,), 4)
+    sc = oracle.repartition_fwd(one, many, [v])                            # scatter: blocks 4, 3, 3
+    assert [a.shape[0] for a in sc] == [4, 3, 3] and np.array_equal(np.concatenate(sc), v)
+    assert np.array_equal(oracle.repartition_fwd(many, one, sc)[0], v)     # gather
+
+
+def test_allreduce_is_symmetric_and_gives_every_worker_the_sum():
+    k, n = 3, 4
+    cols = []
+    for e in range(k * n):
+        u = np.zeros(k * n, np.float32)
+        u[e] = 1
+        cols.append(np.concatenate(oracle.allreduce([u[i * n:(i + 1) * n] for i in range(k)])))
+    M = np.stack(cols, axis=1)
+    assert np.array_equal(M, M.T)                                          # self-adjoint
+    assert np.array_equal(M, np.kron(np.ones((k, k), np.float32), np.eye(n, dtype=np.float32)))
+    parts = [inputs.uniform_pm1((1000,), 50 + i) for i in range(5)]
+    out = oracle.allreduce(parts)
+    ref = parts[0]
+    for p in parts[1:]:
+        ref = ref + p                                                      # fp32 left fold
+    assert all(o.tobytes() == ref.tobytes() for o in out)
