@@ -181,6 +181,41 @@ distdl_status_t distdl_halo_fwd_noalloc(int32_t rank, const int64_t *global_shap
                                         void *const *shards, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Generalized all-to-all, scatter / gather, all-reduce (Section 3, "Scatter and Gather",
+ * "Sum-reduce and all-reduce", "Generalized all-to-all").
+ *
+ * A repartition object describes one tensor under two Cartesian partitions without ghosts, both
+ * split evenly (src_partition_shape -> dst_partition_shape; at most DISTDL_MAX_WORKERS workers in
+ * both together).  The all-to-all moves every cell from the worker that owns it in the source
+ * partition to its owner in the destination partition: a block permutation whose blocks are
+ * send-receive copies, one per pair of workers whose blocks intersect.  A source partition of one
+ * worker is the scatter, a destination partition of one worker the gather.
+ *   repartition_fwd: dst[Pdst] <- src[Psrc]   (contiguous row-major blocks, bit copies)
+ *   repartition_adj: dx[Psrc] <- dy[Pdst]     (every copy is a move, so the adjoint is the
+ *                                              inverse: the all-to-all back)
+ * Outputs may overlap neither each other nor any input (DISTDL_ERR_INVALID_ARG).  F32 and BF16.
+ * repartition_shard_shape: extents of one worker's block (destination != 0: in the destination
+ * partition); `shape` has rank entries.
+ *
+ * allreduce: A = B R on k buffers of n elements in place: every buffer ends up holding
+ * ((b[0] + b[1]) + ...) + b[k-1] (F32, fixed order); self-adjoint.  Two launches.
+ * ---------------------------------------------------------------------- */
+typedef struct distdl_repartition distdl_repartition_t; /* opaque, immutable after create */
+distdl_status_t distdl_repartition_create(int32_t rank, const int64_t *global_shape,
+                                          const int32_t *src_partition_shape,
+                                          const int32_t *dst_partition_shape, distdl_dtype_t dtype,
+                                          distdl_repartition_t **out);
+void distdl_repartition_destroy(distdl_repartition_t *r); /* NULL is allowed */
+distdl_status_t distdl_repartition_shard_shape(const distdl_repartition_t *r, int32_t destination,
+                                               int32_t worker, int64_t *shape);
+distdl_status_t distdl_repartition_fwd(const distdl_repartition_t *r, const void *const *src,
+                                       void *const *dst, void *stream);
+distdl_status_t distdl_repartition_adj(const distdl_repartition_t *r, const void *const *dy,
+                                       void *const *dx, void *stream);
+distdl_status_t distdl_allreduce(void *const *bufs, int32_t k, int64_t n, distdl_dtype_t t,
+                                 void *stream);
+
+/* ------------------------------------------------------------------------
  * Distributed convolution layer, feature-space partition only (Section 4, "Sparse layers":
  * forward / adjoint convolution algorithms and the closing remark that the broadcasts and
  * reductions drop out when only the feature space is partitioned).

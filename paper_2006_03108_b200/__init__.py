@@ -65,6 +65,13 @@ def lib():
     L.distdl_halo_fwd_noalloc.argtypes = [c_i32, pi64, pi32, pi32, pi32, c_i32, pvp, vp]
     L.distdl_conv_fwd.argtypes = [vp, pvp, vp, vp, c_i32, c_i32, pvp, vp]
     L.distdl_conv_adj.argtypes = [vp, pvp, vp, c_i32, c_i32, pvp, vp]
+    L.distdl_repartition_create.argtypes = [c_i32, pi64, pi32, pi32, c_i32, pvp]
+    L.distdl_repartition_destroy.argtypes = [vp]
+    L.distdl_repartition_destroy.restype = None
+    L.distdl_repartition_shard_shape.argtypes = [vp, c_i32, c_i32, pi64]
+    L.distdl_repartition_fwd.argtypes = [vp, pvp, pvp, vp]
+    L.distdl_repartition_adj.argtypes = [vp, pvp, pvp, vp]
+    L.distdl_allreduce.argtypes = [pvp, c_i32, c_i64, c_i32, vp]
     L.distdl_pool_fwd.argtypes = [vp, pvp] + [c_i32] * 9 + [pvp, pvp, vp]
     L.distdl_pool_adj.argtypes = [vp, pvp, pvp] + [c_i32] * 9 + [pvp, vp]
     L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
@@ -252,6 +259,54 @@ def conv_fwd(part, x, w, bias, y, stream=None):
 def conv_adj(part, dy, w, dx, stream=None):
     kh, kw = int(w.shape[-2]), int(w.shape[-1])
     _check(lib().distdl_conv_adj(part.handle, _ptr_array(dy), _ptr(w), kh, kw, _ptr_array(dx), _stream(stream)))
+
+
+class Repartition:
+    """Handle of a distdl_repartition_t: one tensor under a source and a destination partition."""
+
+    def __init__(self, global_shape, src_partition_shape, dst_partition_shape, dtype=F32):
+        rank = len(global_shape)
+        if len(src_partition_shape) != rank or len(dst_partition_shape) != rank:
+            raise ValueError("shapes differ in rank")
+        self.rank = rank
+        self._h = ctypes.c_void_p()
+        gs = (ctypes.c_int64 * rank)(*[int(v) for v in global_shape])
+        sp = (ctypes.c_int32 * rank)(*[int(v) for v in src_partition_shape])
+        dp = (ctypes.c_int32 * rank)(*[int(v) for v in dst_partition_shape])
+        _check(lib().distdl_repartition_create(rank, gs, sp, dp, dtype, ctypes.byref(self._h)))
+        self.num_src = self.num_dst = 1
+        for a, b in zip(src_partition_shape, dst_partition_shape):
+            self.num_src *= int(a)
+            self.num_dst *= int(b)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def shard_shape(self, worker, destination=False):
+        out = (ctypes.c_int64 * self.rank)()
+        _check(lib().distdl_repartition_shard_shape(self._h, 1 if destination else 0, worker, out))
+        return tuple(out)
+
+    def __del__(self):
+        try:
+            if self._h:
+                lib().distdl_repartition_destroy(self._h)
+                self._h = ctypes.c_void_p()
+        except Exception:
+            pass
+
+
+def repartition_fwd(rep, src, dst, stream=None):
+    _check(lib().distdl_repartition_fwd(rep.handle, _ptr_array(src), _ptr_array(dst), _stream(stream)))
+
+
+def repartition_adj(rep, dy, dx, stream=None):
+    _check(lib().distdl_repartition_adj(rep.handle, _ptr_array(dy), _ptr_array(dx), _stream(stream)))
+
+
+def allreduce(bufs, stream=None):
+    _check(lib().distdl_allreduce(_ptr_array(bufs), len(bufs), bufs[0].numel(), _dtype_code(bufs[0]), _stream(stream)))
 
 
 POOL_AVG, POOL_MAX = 0, 1

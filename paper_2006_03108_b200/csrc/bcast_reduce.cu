@@ -259,3 +259,12 @@ extern "C" distdl_status_t distdl_broadcast_adj(const void *const *dy, void *dx,
                                                 distdl_dtype_t t, void *stream) {
     return distdl::sumreduce_impl(dy, dx, k, n, t, stream, "broadcast_adj");
 }
+
+extern "C" distdl_status_t distdl_allreduce(void *const *bufs, int32_t k, int64_t n, distdl_dtype_t t, void *stream) {
+    // A = B R: the fixed-order sum lands in bufs[0] (a sum may be written over its first source), then goes out
+    // to the other k - 1 buffers (the broadcast skips a destination equal to the source)
+    distdl_status_t st = distdl::sumreduce_impl(reinterpret_cast<const void *const *>(bufs), bufs ? bufs[0] : nullptr, k, n, t,
+                                                stream, "allreduce");
+    if (st != DISTDL_OK) return st;
+    return distdl::broadcast_impl(bufs[0], bufs, k, n, t, stream, "allreduce");
+}

@@ -131,7 +131,30 @@ struct distdl_partition {
     }
 };
 
+// The opaque object of the generalized all-to-all: the same tensor under two partitions without ghosts.
+struct distdl_repartition {
+    int32_t rank = 0;
+    distdl_dtype_t dtype = DISTDL_F32;
+    int device = 0;
+    int64_t global_shape[DISTDL_MAX_RANK] = {0};
+    int32_t src_pshape[DISTDL_MAX_RANK] = {0}, dst_pshape[DISTDL_MAX_RANK] = {0};
+    int32_t num_src = 0, num_dst = 0;
+    std::vector<int64_t> src_start[DISTDL_MAX_RANK], src_size[DISTDL_MAX_RANK];
+    std::vector<int64_t> dst_start[DISTDL_MAX_RANK], dst_size[DISTDL_MAX_RANK];
+    std::vector<int64_t> shard_elems;      // source workers first, then destination workers
+    distdl::HaloPlanHost fwd_host, adj_host;
+    distdl::HaloPlanDevice fwd_dev, adj_dev;
+    void *device_block = nullptr;
+};
+
 namespace distdl {
+// Box / tile lists of the all-to-all and of its adjoint (the all-to-all back).
+distdl_status_t build_repartition_plans(distdl_repartition *r);
+void split_evenly(int64_t n, int32_t p, std::vector<int64_t> &start, std::vector<int64_t> &size);
+// One device allocation holding the tables of two plans; host-only when there is no CUDA device
+// (*block stays nullptr).  Synchronous copies on the current device.
+distdl_status_t upload_plan_pair(const HaloPlanHost &a, const HaloPlanHost &b, HaloPlanDevice *da, HaloPlanDevice *db,
+                                 void **block, int *device, const char *what);
 // Builds the forward (H) and adjoint (H*) box/tile lists of a partition (host only).
 distdl_status_t build_halo_plans(distdl_partition *p);
 // Geometry and halo plans only, no device memory.

@@ -358,6 +358,60 @@ extern "C" distdl_status_t distdl_halo_fwd_noalloc(int32_t rank, const int64_t *
     return distdl::halo_fwd_noalloc_impl(rank, global_shape, partition_shape, halo_lo, halo_hi, dtype, shards, stream);
 }
 
+namespace distdl {
+// The all-to-all runs the copy path of the box kernel on the pointer table [source shards, destination shards].
+static distdl_status_t repartition_launch(const distdl_repartition *r, const void *const *from, void *const *to,
+                                          void *stream, bool adjoint, const char *what) {
+    clear_error();
+    if (!r || !from || !to) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (!r->device_block) return fail(DISTDL_ERR_CUDA, "%s: the object was created without a CUDA device", what);
+    // forward: from = source shards, to = destination shards; adjoint: from = destination shards, to = source shards
+    const int32_t nfrom = adjoint ? r->num_dst : r->num_src, nto = adjoint ? r->num_src : r->num_dst;
+    const int32_t from_base = adjoint ? r->num_src : 0, to_base = adjoint ? 0 : r->num_src;
+    ShardPointers sh;
+    for (int32_t w = 0; w < DISTDL_MAX_WORKERS; ++w) sh.p[w] = nullptr;
+    const int64_t es = elem_size(r->dtype);
+    for (int32_t w = 0; w < nfrom; ++w) {
+        if (!from[w]) return fail(DISTDL_ERR_INVALID_ARG, "%s: input shard %d is NULL", what, w);
+        if (!aligned16(from[w])) return fail(DISTDL_ERR_ALIGNMENT, "%s: input shard %d is not 16-byte aligned", what, w);
+        sh.p[from_base + w] = const_cast<void *>(from[w]);
+    }
+    for (int32_t w = 0; w < nto; ++w) {
+        if (!to[w]) return fail(DISTDL_ERR_INVALID_ARG, "%s: output shard %d is NULL", what, w);
+        if (!aligned16(to[w])) return fail(DISTDL_ERR_ALIGNMENT, "%s: output shard %d is not 16-byte aligned", what, w);
+        sh.p[to_base + w] = to[w];
+    }
+    // an output shard may overlap neither another output nor any input (the copy is not in place)
+    for (int32_t a = 0; a < nto; ++a) {
+        const char *a0 = (const char *)to[a], *a1 = a0 + r->shard_elems[to_base + a] * es;
+        for (int32_t b = a + 1; b < nto; ++b) {
+            const char *b0 = (const char *)to[b], *b1 = b0 + r->shard_elems[to_base + b] * es;
+            if (a0 < b1 && b0 < a1) return fail(DISTDL_ERR_INVALID_ARG, "%s: output shards %d and %d overlap", what, a, b);
+        }
+        for (int32_t b = 0; b < nfrom; ++b) {
+            const char *b0 = (const char *)from[b], *b1 = b0 + r->shard_elems[from_base + b] * es;
+            if (a0 < b1 && b0 < a1) return fail(DISTDL_ERR_INVALID_ARG, "%s: output shard %d overlaps input shard %d", what, a, b);
+        }
+    }
+    const HaloPlanDevice &plan = adjoint ? r->adj_dev : r->fwd_dev;
+    if (plan.num_tiles == 0) return DISTDL_OK;
+    halo_box_kernel<false><<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(plan.boxes, plan.sources, plan.tiles,
+                                                                                       elem_size(r->dtype), sh);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+}  // namespace distdl
+
+extern "C" distdl_status_t distdl_repartition_fwd(const distdl_repartition_t *r, const void *const *src, void *const *dst,
+                                                  void *stream) {
+    return distdl::repartition_launch(r, src, dst, stream, false, "repartition_fwd");
+}
+
+extern "C" distdl_status_t distdl_repartition_adj(const distdl_repartition_t *r, const void *const *dy, void *const *dx,
+                                                  void *stream) {
+    return distdl::repartition_launch(r, dy, dx, stream, true, "repartition_adj");
+}
+
 extern "C" distdl_status_t distdl_halo_fwd(const distdl_partition_t *p, void *const *shards, void *stream) {
     return distdl::launch(p, p ? p->fwd_dev : distdl::HaloPlanDevice(), shards, stream, false, "halo_fwd");
 }

@@ -6,6 +6,52 @@
 
 using namespace distdl;
 
+distdl_status_t distdl::upload_plan_pair(const HaloPlanHost &a, const HaloPlanHost &b, HaloPlanDevice *da, HaloPlanDevice *db,
+                                 void **block, int *device, const char *what) {
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) {
+        cudaGetLastError();
+        return DISTDL_OK;      // host-only object
+    }
+    cudaGetDevice(device);
+    auto bytes_of = [](const HaloPlanHost &h, size_t *bz, size_t *sz, size_t *tz) {
+        auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+        *bz = up(h.boxes.size() * sizeof(HaloBox));
+        *sz = up(h.sources.size() * sizeof(HaloSource));
+        *tz = up(h.tiles.size() * sizeof(HaloTile));
+    };
+    size_t fbz, fsz, ftz, abz, asz, atz;
+    bytes_of(a, &fbz, &fsz, &ftz);
+    bytes_of(b, &abz, &asz, &atz);
+    const size_t total = fbz + fsz + ftz + abz + asz + atz + 256;
+    cudaError_t e = cudaMalloc(block, total);
+    if (e != cudaSuccess) {
+        *block = nullptr;
+        return fail(DISTDL_ERR_NOMEM, "%s: cudaMalloc(%zu) failed: %s", what, total, cudaGetErrorString(e));
+    }
+    char *at = (char *)*block;
+    auto put = [&](const void *src, size_t n, size_t reserved) -> void * {
+        void *dst = at;
+        if (n && e == cudaSuccess) e = cudaMemcpy(dst, src, n, cudaMemcpyHostToDevice);
+        at += reserved;
+        return dst;
+    };
+    da->boxes = (HaloBox *)put(a.boxes.data(), a.boxes.size() * sizeof(HaloBox), fbz);
+    da->sources = (HaloSource *)put(a.sources.data(), a.sources.size() * sizeof(HaloSource), fsz);
+    da->tiles = (HaloTile *)put(a.tiles.data(), a.tiles.size() * sizeof(HaloTile), ftz);
+    da->num_tiles = (int32_t)a.tiles.size();
+    db->boxes = (HaloBox *)put(b.boxes.data(), b.boxes.size() * sizeof(HaloBox), abz);
+    db->sources = (HaloSource *)put(b.sources.data(), b.sources.size() * sizeof(HaloSource), asz);
+    db->tiles = (HaloTile *)put(b.tiles.data(), b.tiles.size() * sizeof(HaloTile), atz);
+    db->num_tiles = (int32_t)b.tiles.size();
+    if (e != cudaSuccess) {
+        cudaFree(*block);
+        *block = nullptr;
+        return fail(DISTDL_ERR_CUDA, "%s: upload failed: %s", what, cudaGetErrorString(e));
+    }
+    return DISTDL_OK;
+}
+
 static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
                                    const int32_t *const *hlo, const int32_t *const *hhi,
                                    const int32_t *ulo, const int32_t *uhi, distdl_dtype_t dtype,
@@ -74,48 +120,13 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
     }
     // Upload.  Without a CUDA device the object stays host-only: geometry queries work, operator
     // calls report DISTDL_ERR_CUDA.
-    int ndev = 0;
-    if (!upload) {
-        // host-only object: the caller keeps the plan tables wherever it wants
-    } else if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
-        cudaGetDevice(&p->device);
-        auto bytes_of = [](const HaloPlanHost &h, size_t *b, size_t *s, size_t *t) {
-            auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
-            *b = up(h.boxes.size() * sizeof(HaloBox));
-            *s = up(h.sources.size() * sizeof(HaloSource));
-            *t = up(h.tiles.size() * sizeof(HaloTile));
-        };
-        size_t fbz, fsz, ftz, abz, asz, atz;
-        bytes_of(p->fwd_host, &fbz, &fsz, &ftz);
-        bytes_of(p->adj_host, &abz, &asz, &atz);
-        const size_t total = fbz + fsz + ftz + abz + asz + atz + 256;
-        cudaError_t e = cudaMalloc(&p->device_block, total);
-        if (e != cudaSuccess) {
+    if (upload) {
+        st = upload_plan_pair(p->fwd_host, p->adj_host, &p->fwd_dev, &p->adj_dev, &p->device_block, &p->device,
+                              "partition_create");
+        if (st != DISTDL_OK) {
             delete p;
-            return fail(DISTDL_ERR_NOMEM, "partition_create: cudaMalloc(%zu) failed: %s", total, cudaGetErrorString(e));
+            return st;
         }
-        char *at = (char *)p->device_block;
-        auto put = [&](const void *src, size_t n, size_t reserved) -> void * {
-            void *dst = at;
-            if (n && e == cudaSuccess) e = cudaMemcpy(dst, src, n, cudaMemcpyHostToDevice);
-            at += reserved;
-            return dst;
-        };
-        p->fwd_dev.boxes = (HaloBox *)put(p->fwd_host.boxes.data(), p->fwd_host.boxes.size() * sizeof(HaloBox), fbz);
-        p->fwd_dev.sources = (HaloSource *)put(p->fwd_host.sources.data(), p->fwd_host.sources.size() * sizeof(HaloSource), fsz);
-        p->fwd_dev.tiles = (HaloTile *)put(p->fwd_host.tiles.data(), p->fwd_host.tiles.size() * sizeof(HaloTile), ftz);
-        p->fwd_dev.num_tiles = (int32_t)p->fwd_host.tiles.size();
-        p->adj_dev.boxes = (HaloBox *)put(p->adj_host.boxes.data(), p->adj_host.boxes.size() * sizeof(HaloBox), abz);
-        p->adj_dev.sources = (HaloSource *)put(p->adj_host.sources.data(), p->adj_host.sources.size() * sizeof(HaloSource), asz);
-        p->adj_dev.tiles = (HaloTile *)put(p->adj_host.tiles.data(), p->adj_host.tiles.size() * sizeof(HaloTile), atz);
-        p->adj_dev.num_tiles = (int32_t)p->adj_host.tiles.size();
-        if (e != cudaSuccess) {
-            cudaFree(p->device_block);
-            delete p;
-            return fail(DISTDL_ERR_CUDA, "partition_create: upload failed: %s", cudaGetErrorString(e));
-        }
-    } else {
-        cudaGetLastError();
     }
     *out = p;
     return DISTDL_OK;
@@ -184,5 +195,91 @@ extern "C" distdl_status_t distdl_partition_halo_stats(const distdl_partition_t 
     if (boxes) *boxes = (int64_t)h.boxes.size();
     if (tiles) *tiles = (int64_t)h.tiles.size();
     if (bytes) *bytes = h.algorithmic_bytes;
+    return DISTDL_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Generalized all-to-all
+// ---------------------------------------------------------------------------------------------
+extern "C" distdl_status_t distdl_repartition_create(int32_t rank, const int64_t *global_shape,
+                                                     const int32_t *src_partition_shape,
+                                                     const int32_t *dst_partition_shape, distdl_dtype_t dtype,
+                                                     distdl_repartition_t **out) {
+    clear_error();
+    if (!global_shape || !src_partition_shape || !dst_partition_shape || !out)
+        return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: NULL argument");
+    if (rank < 1 || rank > DISTDL_MAX_RANK) return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: rank %d", rank);
+    if (dtype != DISTDL_F32 && dtype != DISTDL_BF16) return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: bad dtype");
+    distdl_repartition *r = new distdl_repartition();
+    r->rank = rank;
+    r->dtype = dtype;
+    int64_t ns = 1, nd = 1;
+    for (int k = 0; k < rank; ++k) {
+        if (global_shape[k] < 1 || src_partition_shape[k] < 1 || dst_partition_shape[k] < 1 ||
+            src_partition_shape[k] > global_shape[k] || dst_partition_shape[k] > global_shape[k]) {
+            delete r;
+            return fail(DISTDL_ERR_SHAPE, "repartition_create: dimension %d: extent %lld, workers %d -> %d", k,
+                        (long long)global_shape[k], src_partition_shape[k], dst_partition_shape[k]);
+        }
+        r->global_shape[k] = global_shape[k];
+        r->src_pshape[k] = src_partition_shape[k];
+        r->dst_pshape[k] = dst_partition_shape[k];
+        ns *= src_partition_shape[k];
+        nd *= dst_partition_shape[k];
+        split_evenly(global_shape[k], src_partition_shape[k], r->src_start[k], r->src_size[k]);
+        split_evenly(global_shape[k], dst_partition_shape[k], r->dst_start[k], r->dst_size[k]);
+    }
+    if (ns + nd > DISTDL_MAX_WORKERS) {
+        delete r;
+        return fail(DISTDL_ERR_UNSUPPORTED, "repartition_create: %lld + %lld workers (at most %d together)", (long long)ns,
+                    (long long)nd, DISTDL_MAX_WORKERS);
+    }
+    r->num_src = (int32_t)ns;
+    r->num_dst = (int32_t)nd;
+    auto elems = [&](const int32_t *pshape, const std::vector<int64_t> *size, int32_t w) {
+        int64_t n = 1;
+        for (int k = rank - 1; k >= 0; --k) {
+            n *= size[k][w % pshape[k]];
+            w /= pshape[k];
+        }
+        return n;
+    };
+    for (int32_t w = 0; w < r->num_src; ++w) r->shard_elems.push_back(elems(r->src_pshape, r->src_size, w));
+    for (int32_t w = 0; w < r->num_dst; ++w) r->shard_elems.push_back(elems(r->dst_pshape, r->dst_size, w));
+    for (int64_t n : r->shard_elems)
+        if (n >= (int64_t)1 << 31) {
+            delete r;
+            return fail(DISTDL_ERR_UNSUPPORTED, "repartition_create: shard too large");
+        }
+    distdl_status_t st = build_repartition_plans(r);
+    if (st == DISTDL_OK)
+        st = upload_plan_pair(r->fwd_host, r->adj_host, &r->fwd_dev, &r->adj_dev, &r->device_block, &r->device,
+                              "repartition_create");
+    if (st != DISTDL_OK) {
+        delete r;
+        return st;
+    }
+    *out = r;
+    return DISTDL_OK;
+}
+
+extern "C" void distdl_repartition_destroy(distdl_repartition_t *r) {
+    if (!r) return;
+    if (r->device_block) cudaFree(r->device_block);
+    delete r;
+}
+
+extern "C" distdl_status_t distdl_repartition_shard_shape(const distdl_repartition_t *r, int32_t destination, int32_t worker,
+                                                          int64_t *shape) {
+    clear_error();
+    if (!r || !shape) return fail(DISTDL_ERR_INVALID_ARG, "repartition_shard_shape: NULL argument");
+    const int32_t *pshape = destination ? r->dst_pshape : r->src_pshape;
+    const std::vector<int64_t> *size = destination ? r->dst_size : r->src_size;
+    if (worker < 0 || worker >= (destination ? r->num_dst : r->num_src))
+        return fail(DISTDL_ERR_INVALID_ARG, "repartition_shard_shape: worker %d", worker);
+    for (int k = r->rank - 1; k >= 0; --k) {
+        shape[k] = size[k][worker % pshape[k]];
+        worker /= pshape[k];
+    }
     return DISTDL_OK;
 }

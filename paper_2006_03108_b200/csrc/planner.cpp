@@ -97,32 +97,40 @@ struct PendingSource {
 constexpr uint32_t kTileUnits = 4096;
 
 struct Builder {
-    const distdl_partition *p;
     HaloPlanHost *plan;
-    std::vector<Region> dst_regions;   // for the disjointness check
     int esize;
+    int rank;
+    std::vector<std::array<int64_t, DISTDL_MAX_RANK>> shard_shape;   // extents of every shard's array
+    std::vector<Region> dst_regions;                                   // for the disjointness check
+
+    Builder(const distdl_partition *p, HaloPlanHost *plan_, int esize_) : plan(plan_), esize(esize_), rank(p->rank) {
+        shard_shape.resize(p->num_workers);
+        for (int32_t w = 0; w < p->num_workers; ++w) {
+            int32_t c[DISTDL_MAX_RANK];
+            p->coords(w, c);
+            for (int k = 0; k < rank; ++k) shard_shape[w][k] = p->padded_extent(k, c[k]);
+        }
+    }
+    Builder(int rank_, std::vector<std::array<int64_t, DISTDL_MAX_RANK>> shapes, HaloPlanHost *plan_, int esize_)
+        : plan(plan_), esize(esize_), rank(rank_), shard_shape(std::move(shapes)) {}
 
     void strides_of(int32_t shard, int64_t *stride) const {
-        int32_t c[DISTDL_MAX_RANK];
-        p->coords(shard, c);
         int64_t s = 1;
-        for (int k = p->rank - 1; k >= 0; --k) {
+        for (int k = rank - 1; k >= 0; --k) {
             stride[k] = s;
-            s *= p->padded_extent(k, c[k]);
+            s *= shard_shape[shard][k];
         }
     }
     bool inside(const Region &r) const {
-        int32_t c[DISTDL_MAX_RANK];
-        p->coords(r.shard, c);
-        for (int k = 0; k < p->rank; ++k)
-            if (r.start[k] < 0 || r.extent[k] < 0 || r.start[k] + r.extent[k] > p->padded_extent(k, c[k]))
-                return false;
+        if (r.shard < 0 || r.shard >= (int32_t)shard_shape.size()) return false;
+        for (int k = 0; k < rank; ++k)
+            if (r.start[k] < 0 || r.extent[k] < 0 || r.start[k] + r.extent[k] > shard_shape[r.shard][k]) return false;
         return true;
     }
 
     // Adds one box; `srcs` may be empty (clear).  Returns false on an internal inconsistency.
     bool add(const Region &dst, const std::vector<PendingSource> &srcs, int levels) {
-        const int d = p->rank;
+        const int d = rank;
         int64_t cells = 1;
         for (int k = 0; k < d; ++k) cells *= dst.extent[k];
         if (cells == 0) return true;
@@ -263,7 +271,7 @@ struct Builder {
     }
 
     bool destinations_disjoint() const {
-        const int d = p->rank;
+        const int d = rank;
         for (size_t a = 0; a < dst_regions.size(); ++a)
             for (size_t b = a + 1; b < dst_regions.size(); ++b) {
                 const Region &x = dst_regions[a], &y = dst_regions[b];
@@ -298,9 +306,9 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
     const int esize = elem_size(p->dtype);
 
     // ---------------- forward: one box per (shard, direction) ----------------
-    Builder fb{p, &p->fwd_host, {}, esize};
+    Builder fb(p, &p->fwd_host, esize);
     // exterior-ghost clear boxes are shared by the adjoint plan
-    Builder ab{p, &p->adj_host, {}, esize};
+    Builder ab(p, &p->adj_host, esize);
     for (int32_t w = 0; w < p->num_workers; ++w) {
         int32_t c[DISTDL_MAX_RANK];
         p->coords(w, c);
@@ -431,6 +439,70 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
     }
     if (!ab.destinations_disjoint()) return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint boxes overlap");
     return DISTDL_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Generalized all-to-all: one copy box per pair (destination worker, source worker) whose blocks of
+// the tensor intersect.  Shards are numbered source workers first, then destination workers; the
+// adjoint plan is the same list with the roles of the two regions exchanged.
+// ---------------------------------------------------------------------------------------------
+distdl_status_t build_repartition_plans(distdl_repartition *r) {
+    const int d = r->rank;
+    const int esize = elem_size(r->dtype);
+    const int32_t ns = r->num_src, nd = r->num_dst;
+    std::vector<std::array<int64_t, DISTDL_MAX_RANK>> shapes(ns + nd);
+    auto coords = [&](const int32_t *pshape, int32_t w, int32_t *c) {
+        for (int k = d - 1; k >= 0; --k) {
+            c[k] = w % pshape[k];
+            w /= pshape[k];
+        }
+    };
+    for (int32_t w = 0; w < ns; ++w) {
+        int32_t c[DISTDL_MAX_RANK];
+        coords(r->src_pshape, w, c);
+        for (int k = 0; k < d; ++k) shapes[w][k] = r->src_size[k][c[k]];
+    }
+    for (int32_t w = 0; w < nd; ++w) {
+        int32_t c[DISTDL_MAX_RANK];
+        coords(r->dst_pshape, w, c);
+        for (int k = 0; k < d; ++k) shapes[ns + w][k] = r->dst_size[k][c[k]];
+    }
+    Builder fb(d, shapes, &r->fwd_host, esize), ab(d, shapes, &r->adj_host, esize);
+    for (int32_t wd = 0; wd < nd; ++wd) {
+        int32_t cd[DISTDL_MAX_RANK];
+        coords(r->dst_pshape, wd, cd);
+        for (int32_t ws = 0; ws < ns; ++ws) {
+            int32_t cs[DISTDL_MAX_RANK];
+            coords(r->src_pshape, ws, cs);
+            Region in_dst, in_src;
+            in_dst.shard = ns + wd;
+            in_src.shard = ws;
+            bool empty = false;
+            for (int k = 0; k < d; ++k) {
+                const int64_t s0 = r->src_start[k][cs[k]], s1 = s0 + r->src_size[k][cs[k]];
+                const int64_t d0 = r->dst_start[k][cd[k]], d1 = d0 + r->dst_size[k][cd[k]];
+                const int64_t lo = std::max(s0, d0), hi = std::min(s1, d1);
+                if (hi <= lo) {
+                    empty = true;
+                    break;
+                }
+                in_dst.start[k] = lo - d0;
+                in_src.start[k] = lo - s0;
+                in_dst.extent[k] = in_src.extent[k] = hi - lo;
+            }
+            if (empty) continue;
+            PendingSource from_src{in_src, 0, 0}, from_dst{in_dst, 0, 0};
+            if (!fb.add(in_dst, {from_src}, 1)) return fail(DISTDL_ERR_SHAPE, "repartition plan: box out of range");
+            if (!ab.add(in_src, {from_dst}, 1)) return fail(DISTDL_ERR_SHAPE, "repartition plan: box out of range");
+        }
+    }
+    if (!fb.destinations_disjoint() || !ab.destinations_disjoint())
+        return fail(DISTDL_ERR_SHAPE, "repartition plan: boxes overlap");
+    return DISTDL_OK;
+}
+
+void split_evenly(int64_t n, int32_t p, std::vector<int64_t> &start, std::vector<int64_t> &size) {
+    balanced_split(n, p, start, size);
 }
 
 }  // namespace distdl

@@ -453,3 +453,75 @@ def test_pool_rejects_partitions_with_other_widths():
     with pytest.raises(distdl.DistdlError) as e:
         distdl.pool_fwd(part, x, (2, 2), (2, 2), ((0, 0), (0, 0)), distdl.POOL_AVG, y)
     assert e.value.status == 2          # DISTDL_ERR_SHAPE
+
+
+# --------------------------------------------------------------------------
+# Generalized all-to-all, scatter / gather, all-reduce
+# --------------------------------------------------------------------------
+
+REPART_CASES = [
+    # global shape, source partition, destination partition
+    ((7, 9), (2, 1), (1, 3)),
+    ((64, 96), (4, 1), (1, 4)),                  # row blocks -> column blocks ("transpose")
+    ((5, 40, 68), (1, 2, 3), (5, 1, 1)),
+    ((1000003,), (1,), (7,)),                    # scatter
+    ((1000003,), (5,), (1,)),                    # gather
+    ((2, 3, 130, 260), (1, 1, 4, 4), (1, 1, 16, 1)),
+    ((33, 1025), (3, 5), (3, 5)),                # identity
+]
+
+
+@pytest.mark.parametrize("case", REPART_CASES, ids=[str(c) for c in REPART_CASES])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_repartition_fwd_and_adj_bit_exact(case, dtype):
+    gs, sp, dp = case
+    osrc, odst = oracle.Partition(gs, sp), oracle.Partition(gs, dp)
+    code = distdl.F32 if dtype == "f32" else distdl.BF16
+    rep = distdl.Repartition(gs, sp, dp, code)
+    if dtype == "f32":
+        g = inputs.uniform_pm1(gs, 91)
+        up = lambda a: dev(a)
+        down = lambda t: host(t)
+        empty = lambda shape: torch.full(tuple(shape), 3.0, device=DEV)
+    else:
+        g = inputs.f32_to_bf16_bits(inputs.uniform_pm1(gs, 91))
+        up = lambda a: dev(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+        down = lambda t: host(t.view(torch.int16)).view(np.uint16)
+        empty = lambda shape: torch.full(tuple(shape), 3.0, device=DEV, dtype=torch.bfloat16)
+    src = oracle.scatter_global(osrc, g)
+    for w in range(rep.num_src):
+        assert rep.shard_shape(w) == tuple(src[w].shape)
+    ref = oracle.repartition_fwd(osrc, odst, src)
+    out = [empty(a.shape) for a in ref]
+    distdl.repartition_fwd(rep, [up(a) for a in src], out)
+    torch.cuda.synchronize()
+    for w, (got, r) in enumerate(zip(out, ref)):
+        assert rep.shard_shape(w, destination=True) == tuple(r.shape)
+        assert same_bits(down(got), r)
+    back = [empty(a.shape) for a in src]
+    distdl.repartition_adj(rep, out, back)
+    torch.cuda.synchronize()
+    for got, r in zip(back, oracle.repartition_adj(osrc, odst, ref)):
+        assert same_bits(down(got), r)
+    for got, r in zip(back, src):                       # the adjoint of a permutation is its inverse
+        assert same_bits(down(got), r)
+
+
+def test_repartition_rejects_overlapping_buffers():
+    rep = distdl.Repartition((8, 8), (2, 1), (1, 2))
+    a = torch.zeros(64, device=DEV)
+    src = [a[:32].view(4, 8), a[32:].view(4, 8)]
+    with pytest.raises(distdl.DistdlError) as e:
+        distdl.repartition_fwd(rep, src, [a[:32].view(8, 4), torch.zeros(8, 4, device=DEV)])
+    assert e.value.status == 1          # DISTDL_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("k", [1, 2, 5, 8])
+def test_allreduce_bit_exact(k):
+    n = 100003
+    parts = [inputs.uniform_pm1((n,), 300 + i) for i in range(k)]
+    bufs = [dev(p) for p in parts]
+    distdl.allreduce(bufs)
+    torch.cuda.synchronize()
+    for got, ref in zip(bufs, oracle.allreduce(parts)):
+        assert same_bits(host(got), ref)
