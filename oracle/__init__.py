@@ -38,8 +38,10 @@ from .layers import (  # noqa: F401
     conv_fwd,
     conv_adj,
     conv_adj_scatter_then_halo,
+    conv_adj_params,
     affine_fwd,
     affine_adj,
+    affine_adj_params,
     bf16_bits_to_f64,
     pool_partition,
     pool_fwd_global,

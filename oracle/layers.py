@@ -117,6 +117,36 @@ def conv_adj_scatter_then_halo(part: Partition, dy_shards, w):
     return halo_adj_sequence(part, local)
 
 
+def conv_adj_params(part: Partition, x_shards, dy_shards, kh, kw):
+    """Parameter part of the adjoint convolution algorithm: (dw, db), depthwise kernel.
+
+    With the tensor partitioned over the feature space only, every worker holds
+    a copy of the kernel (w^ <- B w), so its local gradients are summed over the
+    workers (dw <- R dw^, db <- R db^, in worker order).  Step by step:
+      x <- H x            (the exchanged input saved by the forward pass)
+      dw^_k[c,a,b] = sum_{n,i,j} dy_k[n,c,i,j] * x_k[n,c,i+a,j+b]   (padded-local indices)
+      db^_k[c]     = sum_{n,i,j} dy_k[n,c,i,j]
+      dw = R_k dw^_k,  db = R_k db^_k
+    Local sums and the fold over workers in fp64, rounded once to fp32.
+    """
+    _check_conv_partition(part, kh, kw)
+    from .primitives import halo_fwd_sequence
+    xh = halo_fwd_sequence(part, x_shards)
+    dws, dbs = [], []
+    for wk in range(part.num_workers):
+        x = np.asarray(xh[wk], dtype=np.float64)
+        dy = np.asarray(dy_shards[wk], dtype=np.float64)
+        N, C, hb, wb = dy.shape
+        assert x.shape == (N, C, hb + kh - 1, wb + kw - 1)
+        dwk = np.zeros((C, kh, kw), dtype=np.float64)
+        for a in range(kh):
+            for b in range(kw):
+                dwk[:, a, b] = (dy * x[:, :, a:a + hb, b:b + wb]).sum(axis=(0, 2, 3))
+        dws.append(dwk)
+        dbs.append(dy.sum(axis=(0, 2, 3)))
+    return sumreduce_fwd(dws).astype(np.float32), sumreduce_fwd(dbs).astype(np.float32)
+
+
 # --------------------------------------------------------------------------
 # Distributed affine layer (Section 4, "Dense layers")
 # --------------------------------------------------------------------------
@@ -168,6 +198,28 @@ def affine_adj(dy_parts, w_parts, pfo, pfi):
             partial.append(dyhat[i][j] @ wij)
         dx.append(sumreduce_fwd(partial).astype(np.float32))
     return dx
+
+
+def affine_adj_params(dy_parts, x_parts, pfo, pfi):
+    """Parameter part of the adjoint affine algorithm: (dW, db).
+
+    dy^_{ij} <- B dy_i (along grid rows); worker (i, j) holds x^_{ij} = x_j from
+    the forward pass and applies [dAffine]* to dy^_{ij}:
+        dW_{ij}[o, f] = sum_b dy^_{ij}[b, o] * x^_{ij}[b, f]
+        db_{ij}[o]    = sum_b dy^_{ij}[b, o]      (only where the bias lives: j = 0)
+    The weights are distributed on P_w itself, so no reduction follows: the
+    result is one block per worker, in worker order i * P_fi + j, and one bias
+    gradient per grid row.  fp64 sums over b in ascending order, rounded once
+    to fp32.
+    """
+    dyhat = [broadcast_fwd(np.asarray(dy_parts[i], dtype=np.float64), pfi) for i in range(pfo)]
+    xhat = [broadcast_fwd(np.asarray(x_parts[j], dtype=np.float64), pfo) for j in range(pfi)]
+    dw, db = [], []
+    for i in range(pfo):
+        for j in range(pfi):
+            dw.append((dyhat[i][j].T @ xhat[j][i]).astype(np.float32))
+        db.append(dyhat[i][0].sum(axis=0).astype(np.float32))
+    return dw, db
 
 
 # --------------------------------------------------------------------------

@@ -650,3 +650,90 @@ def test_allreduce_is_symmetric_and_gives_every_worker_the_sum():
     for p in parts[1:]:
         ref = ref + p                                                      # fp32 left fold
     assert all(o.tobytes() == ref.tobytes() for o in out)
+
+
+# --------------------------------------------------------------------------
+# Parameter gradients of the two layers (adjoint algorithms of Section 4: dW, db / dw, db)
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("pfo,pfi", [(1, 1), (2, 2), (4, 2), (1, 4)])
+def test_affine_param_gradients_exact_on_integers_and_against_autograd(pfo, pfi):
+    import torch
+    nb, nfi, nfo = 6, 16, 8
+    xg, wg, xs, ws = _affine_problem(nb, nfi, nfo, pfo, pfi, 61, integer=True)
+    dyg = inputs.integers((nb, nfo), 63)
+    dw, db = oracle.affine_adj_params(np.split(dyg, pfo, axis=1), xs, pfo, pfi)
+    dwg = np.concatenate([np.concatenate(dw[i * pfi:(i + 1) * pfi], axis=1) for i in range(pfo)], axis=0)
+    # library routine on the unpartitioned operands: reverse-mode derivative of the framework's linear layer
+    W = torch.tensor(wg, dtype=torch.float64, requires_grad=True)
+    b = torch.zeros(nfo, dtype=torch.float64, requires_grad=True)
+    y = torch.nn.functional.linear(torch.tensor(xg, dtype=torch.float64), W, b)
+    y.backward(torch.tensor(dyg, dtype=torch.float64))
+    assert np.array_equal(dwg, W.grad.numpy().astype(np.float32))
+    assert np.array_equal(np.concatenate(db), b.grad.numpy().astype(np.float32))
+
+
+def test_affine_param_gradients_brute_force_columns_and_dot_test():
+    pfo, pfi, nb, nfi, nfo = 2, 2, 5, 8, 6
+    xg, wg, xs, ws = _affine_problem(nb, nfi, nfo, pfo, pfi, 65)
+    dyg = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(inputs.normal((nb, nfo), 66)))
+    dys = np.split(dyg, pfo, axis=1)
+    dw, db = oracle.affine_adj_params(dys, xs, pfo, pfi)
+    bo, bi = nfo // pfo, nfi // pfi
+    # the layer is linear in (W, b) for a fixed x: the gradient entry of one weight is <Affine(E; x), dy>
+    # with E the unit weight tensor -- evaluated through the (separately pinned) forward oracle
+    zero_w = [np.zeros((bo, bi), np.float32) for _ in range(pfo * pfi)]
+    for i, j, o, f in itertools.product(range(pfo), range(pfi), range(bo), range(bi)):
+        unit = [z.copy() for z in zero_w]
+        unit[i * pfi + j][o, f] = 1.0
+        y = oracle.affine_fwd(xs, unit, pfo, pfi)
+        ref = sum(float((a.astype(np.float64) * d).sum()) for a, d in zip(y, dys))
+        assert abs(float(dw[i * pfi + j][o, f]) - ref) <= 1e-6 * max(1.0, abs(ref))
+    for i, o in itertools.product(range(pfo), range(bo)):
+        unit_b = [np.zeros(bo, np.float32) for _ in range(pfo)]
+        unit_b[i][o] = 1.0
+        y = oracle.affine_fwd([np.zeros_like(x) for x in xs], zero_w, pfo, pfi, unit_b)
+        ref = sum(float((a.astype(np.float64) * d).sum()) for a, d in zip(y, dys))
+        assert abs(float(db[i][o]) - ref) <= 1e-6 * max(1.0, abs(ref))
+    # dot test in parameter space: <Affine(W, b; x), dy> = <W, dW> + <b, db>
+    bias = np.split(inputs.normal((nfo,), 67), pfo)
+    y = oracle.affine_fwd(xs, ws, pfo, pfi, bias)
+    assert oracle.adjoint_test_ratio(y, dys, list(ws) + bias, list(dw) + list(db)) < 1e-6
+
+
+@pytest.mark.parametrize("pshape", CONV_PARTS)
+def test_conv_param_gradients_against_autograd_and_partition_invariance(pshape):
+    import torch
+    part, xg, w = _conv_problem(pshape, shape=(2, 3, 12, 13), k=(5, 5), seed=71)
+    dyg = inputs.normal(xg.shape, 73)
+    x = oracle.scatter_global(part, xg, fill=lambda wk: np.full(part.padded_shape(wk), 7.0))   # garbage ghosts
+    dy = oracle.scatter_global(Partition(xg.shape, pshape), dyg)
+    dw, db = oracle.conv_adj_params(part, x, dy, 5, 5)
+    W = torch.tensor(w[:, None], dtype=torch.float64, requires_grad=True)
+    b = torch.zeros(xg.shape[1], dtype=torch.float64, requires_grad=True)
+    y = torch.nn.functional.conv2d(torch.tensor(xg, dtype=torch.float64), W, b, padding=2, groups=xg.shape[1])
+    y.backward(torch.tensor(dyg, dtype=torch.float64))
+    assert np.allclose(dw, W.grad.numpy()[:, 0], rtol=1e-6, atol=1e-5)
+    assert np.allclose(db, b.grad.numpy(), rtol=1e-6, atol=1e-5)
+    # same result for every partition, 1 x 1 included
+    one = Partition(xg.shape, (1, 1, 1, 1), (0, 0, 2, 2), (0, 0, 2, 2))
+    dw1, db1 = oracle.conv_adj_params(one, oracle.scatter_global(one, xg), [dyg], 5, 5)
+    assert np.allclose(dw, dw1, rtol=1e-6, atol=1e-5) and np.allclose(db, db1, rtol=1e-6, atol=1e-5)
+
+
+def test_conv_param_gradients_brute_force_taps_and_dot_test():
+    part, xg, w = _conv_problem((1, 1, 2, 2), shape=(1, 2, 7, 6), k=(5, 3), seed=75)
+    ypart = Partition(xg.shape, part.pshape)
+    dyg = inputs.normal(xg.shape, 77)
+    x, dy = oracle.scatter_global(part, xg), oracle.scatter_global(ypart, dyg)
+    dw, db = oracle.conv_adj_params(part, x, dy, 5, 3)
+    # linear in (w, b): the gradient of tap (c, a, b) is <Conv(E_cab; x), dy> through the forward oracle
+    for c, a, b in itertools.product(range(2), range(5), range(3)):
+        unit = np.zeros_like(w)
+        unit[c, a, b] = 1.0
+        y = oracle.conv_fwd(part, x, unit)
+        ref = sum(float((u.astype(np.float64) * v).sum()) for u, v in zip(y, dy))
+        assert abs(float(dw[c, a, b]) - ref) <= 2e-6 * max(1.0, abs(ref))
+    bias = inputs.normal((2,), 78)
+    y = oracle.conv_fwd(part, x, w, bias)
+    assert oracle.adjoint_test_ratio(y, dy, [w, bias], [dw, db]) < 1e-6
