@@ -147,6 +147,30 @@ class Workload:
              2 * out_b + pad_b + self.ppart.halo_stats(True)[2], 0, 2, "hbm"),
         ]
 
+        # Parameter gradients of the two layers (dw, db of the convolution; dW, db of the affine layer) on the
+        # step's own buffers, and the generalized all-to-all between a row and a column partition of a
+        # fp32 8192 x 8192 tensor (8 -> 8 workers); timed on their own like the pooling layer.
+        self.c_dw = torch.empty(16, 5, 5, device=dev)
+        self.c_db = torch.empty(16, device=dev)
+        self.c_ws = torch.empty(d.conv_adj_params_workspace(self.cpart, 5, 5), dtype=torch.uint8, device=dev)
+        self.a_dw = [torch.empty(blk, blk, device=dev) for _ in range(self.pf * self.pf)]
+        self.a_db = [torch.empty(blk, device=dev) for _ in range(self.pf)]
+        side2 = 4096 if small else 8192
+        self.rep = d.Repartition((side2, side2), (8, 1), (1, 8))
+        self.t_src = [u(side2 // 8, side2) for _ in range(8)]
+        self.t_dst = [torch.empty(side2, side2 // 8, device=dev) for _ in range(8)]
+        self.extra_ops += [
+            ("conv_adj_params", lambda: d.conv_adj_params(self.cpart, self.c_x, self.c_dy, (5, 5), self.c_dw, self.c_db,
+                                                          self.c_ws), conv_bytes, 2 * 25 * self._conv_outputs(), 2, "hbm"),
+            ("affine_adj_params", lambda: d.affine_adj_params(self.nb, self.nf, self.nf, self.pf, self.pf, self.a_dy,
+                                                              self.a_x, self.a_dw, self.a_db),
+             self.nf * self.nf * 4 + 2 * self.nb * self.nf * 2 + self.nf * 4, aff_flops, 2, "hbm"),
+            ("repartition_fwd", lambda: d.repartition_fwd(self.rep, self.t_src, self.t_dst), 2 * side2 * side2 * 4, 0, 1,
+             "hbm"),
+            ("repartition_adj", lambda: d.repartition_adj(self.rep, self.t_dst, self.t_src), 2 * side2 * side2 * 4, 0, 1,
+             "hbm"),
+        ]
+
     def _conv_outputs(self):
         gs = self.cpart.global_shape
         return gs[0] * gs[1] * gs[2] * gs[3]
@@ -412,7 +436,7 @@ def main():
     ms_per_step = elapsed_ms / args.steps
     value = world * wl.bytes_per_step / (ms_per_step * 1e-3) / 1e9
 
-    # ---- the pooling layer, timed on its own (not part of the step or of `value`) ----
+    # ---- the operators outside the step, each timed on its own (not part of `value`) ----
     extra_ms = []
     for name, call, _, _, _, _ in wl.extra_ops:
         for _ in range(3):
@@ -488,8 +512,10 @@ def main():
             "halo_bcast_reduce": {"gbs": round(dm_bytes / dm_ms / 1e6, 1),
                                   "frac_of_hbm_peak": round(dm_bytes / dm_ms / 1e6 / peaks["hbm"], 4)},
             "ops": ops,
-            "extra_ops": {"note": "3x3 max pooling, stride 2, padding 1 on fp32 16x16x1024x1024 over 4x4 workers "
-                                  "(H + local kernel, local adjoint + H*); timed separately, not part of value",
+            "extra_ops": {"note": "timed separately, not part of value: 3x3 max pooling, stride 2, padding 1 on fp32 "
+                                  "16x16x1024x1024 over 4x4 workers (H + local kernel, local adjoint + H*); parameter "
+                                  "gradients of the step's convolution (dw, db) and affine layer (dW, db); generalized "
+                                  "all-to-all of fp32 8192x8192 between 8 row blocks and 8 column blocks",
                           **extra},
             "roofline": roofline,
             "clocks": clocks,

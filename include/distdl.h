@@ -237,6 +237,28 @@ distdl_status_t distdl_conv_fwd(const distdl_partition_t *p, const void *const *
 distdl_status_t distdl_conv_adj(const distdl_partition_t *p, const void *const *dy, const void *w,
                                 int32_t kh, int32_t kw, void *const *dx, void *stream);
 
+
+/* Parameter gradients of the convolution layer (Section 4, "Sparse layers", adjoint convolution
+ * algorithm: dw^, db^ <- [dConv]*(dy^) on every worker, then dw <- R dw^, db <- R db^; with a
+ * feature-space partition every worker holds a copy of the kernel, so the sum runs over all workers).
+ *   dw[c,a,b] = sum over workers k and n,i,j of dy_k[n,c,i,j] * (H x)_k[n,c,i+a,j+b]   (padded-local i+a, j+b)
+ *             = sum_{n,i,j} dy[n,c,i,j] * x[n,c,i+a-ph,j+b-pw] on the global tensor, zeros outside;
+ *   db[c]     = sum_{n,i,j} dy[n,c,i,j].
+ * Same partition and kernel restrictions as conv_fwd.  x[w]: padded shards (only the bulk is read: the
+ * halo exchange is fused, ghost storage is not touched); dy[w]: bulk-shaped shards; dw: [C,kh,kw] F32;
+ * db: [C] F32 or NULL.  Sums are taken in fp32 in a fixed order that depends only on the shapes and
+ * on the device (number of SMs): per-thread running sums over a static set of tiles, a tree over the
+ * threads of a block, then the blocks' partial results in order -- the same bits on every run.
+ * workspace: device scratch of at least the size conv_adj_params_workspace reports (a few hundred
+ * KB), overwritten by the call; the caller may reuse it once the call's work on `stream` is done.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_conv_adj_params_workspace(const distdl_partition_t *p, int32_t kh, int32_t kw,
+                                                 int64_t *bytes);
+distdl_status_t distdl_conv_adj_params(const distdl_partition_t *p, const void *const *x,
+                                       const void *const *dy, int32_t kh, int32_t kw, void *dw,
+                                       void *db, void *workspace, int64_t workspace_bytes,
+                                       void *stream);
+
 /* ------------------------------------------------------------------------
  * Distributed pooling layer, feature-space partition only (Section 4, "Sparse layers": pooling
  * layers follow the convolution algorithms; Section 3 / Appendix B: for a strided kernel the halo
@@ -291,6 +313,19 @@ distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t 
 distdl_status_t distdl_affine_adj(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
                                   const void *const *dy, const void *const *w, void *const *dx,
                                   void *stream);
+
+/* Parameter gradients of the affine layer (Section 4, "Dense layers", adjoint affine algorithm:
+ * dW^, db^ <- [dAffine]*(dy^) with dy^_{ij} = dy_i and the x^_{ij} = x_j of the forward pass; the
+ * weights are distributed on the worker grid itself, so no reduction follows).
+ *   dw[i*Pfi+j]  F32 [nfo/Pfo, nfi/Pfi]   dW_{ij}[o,f] = sum_b dy_i[b,o] * x_j[b,f]
+ *   db[i]        F32 [nfo/Pfo] (db may be NULL)   db_i[o] = sum_b dy_i[b,o]   (bias lives on column j = 0)
+ * dy[i] BF16 [nb, nfo/Pfo], x[j] BF16 [nb, nfi/Pfi].  Tensor cores with fp32 accumulation over the
+ * batch in ascending order (dW); db in fp32, eight contiguous chunks of the batch added in order.
+ * Same shape restrictions as affine_fwd.  Bounded waits report through distdl_device_status().
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_affine_adj_params(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo,
+                                         int32_t pfi, const void *const *dy, const void *const *x,
+                                         void *const *dw, void *const *db, void *stream);
 
 /* Synchronises `stream`, then reads and clears the device status word that the affine kernels set
  * when one of their bounded waits (on a shared-memory barrier fed by TMA or by the tensor cores)

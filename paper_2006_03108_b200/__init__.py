@@ -76,6 +76,9 @@ def lib():
     L.distdl_pool_adj.argtypes = [vp, pvp, pvp] + [c_i32] * 9 + [pvp, vp]
     L.distdl_affine_fwd.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
     L.distdl_affine_adj.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, vp]
+    L.distdl_affine_adj_params.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
+    L.distdl_conv_adj_params_workspace.argtypes = [vp, c_i32, c_i32, pi64]
+    L.distdl_conv_adj_params.argtypes = [vp, pvp, pvp, c_i32, c_i32, vp, vp, vp, c_i64, vp]
     L.distdl_device_status.argtypes = [vp]
     _lib = L
     return L
@@ -334,6 +337,27 @@ def affine_fwd(nb, nfi, nfo, pfo, pfi, x, w, bias, y, stream=None):
 def affine_adj(nb, nfi, nfo, pfo, pfi, dy, w, dx, stream=None):
     _check(lib().distdl_affine_adj(nb, nfi, nfo, pfo, pfi, _ptr_array(dy), _ptr_array(w), _ptr_array(dx),
                                    _stream(stream)))
+
+
+def affine_adj_params(nb, nfi, nfo, pfo, pfi, dy, x, dw, db=None, stream=None):
+    """dW blocks (worker order i * pfi + j) and, if given, the db blocks of the adjoint affine algorithm."""
+    b = None if db is None else _ptr_array(db)
+    _check(lib().distdl_affine_adj_params(nb, nfi, nfo, pfo, pfi, _ptr_array(dy), _ptr_array(x), _ptr_array(dw), b,
+                                          _stream(stream)))
+
+
+def conv_adj_params_workspace(part, kh, kw):
+    """Bytes of device scratch conv_adj_params needs for this partition on the current device."""
+    n = ctypes.c_int64(0)
+    _check(lib().distdl_conv_adj_params_workspace(part.handle, kh, kw, ctypes.byref(n)))
+    return n.value
+
+
+def conv_adj_params(part, x, dy, kernel, dw, db, workspace, stream=None):
+    """dw [C, kh, kw] and db [C] (or None) of the adjoint convolution algorithm; workspace: a uint8 tensor."""
+    _check(lib().distdl_conv_adj_params(part.handle, _ptr_array(x), _ptr_array(dy), kernel[0], kernel[1], _ptr(dw),
+                                        _ptr(db), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                        _stream(stream)))
 
 
 def device_status(stream=None):

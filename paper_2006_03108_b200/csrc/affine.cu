@@ -605,6 +605,209 @@ affine_kernel_quad(const __grid_constant__ AffineParams P) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Parameter gradients of the adjoint affine algorithm (Section 4, "Dense layers"):
+//   dW_{ij} = dy^_{ij}^T x^_{ij}  with dy^_{ij} = dy_i (B along grid rows), x^_{ij} = x_j (B along grid
+//   columns, kept from the forward pass);  db_i = column sums of dy_i (the bias lives on grid column 0).
+// The weights are distributed over the worker grid itself, so nothing is reduced afterwards: each
+// thread block owns one 128 x 128 tile of one worker's dW block and contracts over the batch.
+// Both operands are MN-major for the tensor cores (dy_i is [nb, out] row-major: the M index is
+// contiguous; x_j is [nb, in]: the N index is contiguous), staged by TMA as 64 x 64 swizzled atoms.
+// The output (fp32, nfo x nfi) dominates the traffic, so up to three blocks share an SM and the
+// epilogue stages the tile in (swizzled) shared memory and hands it to TMA stores: whole 128-byte
+// lines leave the SM while the next block's loads and MMAs run.
+// ------------------------------------------------------------------------------------------
+constexpr int kDwThreads = 192;                              // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
+constexpr int kDwStages = 2;
+constexpr int kDwOperandBytes = 2 * 64 * kBlockK * 2;        // two 64 x 64 bf16 atoms = 16 KB
+constexpr int kDwStageBytes = 2 * kDwOperandBytes;           // A and B
+constexpr int kDwOutBytes = kTileM * kTileN * 4;             // 64 KB: the fp32 tile as four 128 x 32 boxes
+static_assert(kDwStages * kDwStageBytes == kDwOutBytes, "the epilogue reuses the ring");
+constexpr int kDwSmemBytes = kDwOutBytes + 1024 + 128;
+
+struct AffineDwParams {
+    CUtensorMap dy_map[8];                  // dy_i  [nb, bfo] bf16, box {64 out, 64 batch}
+    CUtensorMap x_map[8];                   // x_j   [nb, bfi] bf16, box {64 in, 64 batch}
+    CUtensorMap dw_map[kMaxMaps - 8];       // dW_ij [bfo, bfi] fp32, box {32 in, 128 out}
+    int32_t nb, pfi;
+    int32_t tiles_m, tiles_n;               // 128 x 128 tiles per worker block
+};
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int32_t c0, int32_t c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+
+__global__ void __launch_bounds__(kDwThreads, 3)
+affine_dw_kernel(const __grid_constant__ AffineDwParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *aligned = smem_raw + (base - raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kDwOutBytes);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * kDwStages;
+    const uint32_t bar_acc = bar_empty + 8 * kDwStages;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kDwStages + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // tile id: column tile fastest, then row tile, then worker j, then worker i
+    int rest = blockIdx.x;
+    const int tn = rest % P.tiles_n;
+    rest /= P.tiles_n;
+    const int tm = rest % P.tiles_m;
+    rest /= P.tiles_m;
+    const int wj = rest % P.pfi, wi = rest / P.pfi;
+    const int m0 = tm * kTileM, n0 = tn * kTileN;
+    const int num_kblocks = (P.nb + kBlockK - 1) / kBlockK;       // rows past nb are filled with zeros by TMA
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kDwStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const CUtensorMap *amap = &P.dy_map[wi], *bmap = &P.x_map[wj];
+            uint32_t s = 0, phase = 0;
+            for (int kb = 0; kb < num_kblocks; ++kb) {
+                if (!mbar_wait(bar_empty + 8 * s, phase ^ 1, abort_flag)) break;
+                const uint32_t full = bar_full + 8 * s, sa = base + s * kDwStageBytes;
+                mbar_expect_tx(full, kDwStageBytes);
+                const int k0 = kb * kBlockK;
+                tma_load_2d(sa, amap, m0, k0, full);                                   // atom: out features m0 .. m0 + 63
+                tma_load_2d(sa + kDwOperandBytes / 2, amap, m0 + 64, k0, full);
+                tma_load_2d(sa + kDwOperandBytes, bmap, n0, k0, full);                 // atom: in features n0 .. n0 + 63
+                tma_load_2d(sa + kDwOperandBytes + kDwOperandBytes / 2, bmap, n0 + 64, k0, full);
+                if (++s == kDwStages) {
+                    s = 0;
+                    phase ^= 1;
+                }
+            }
+            if (*abort_flag) {
+                const uint64_t t0 = global_timer();
+                while (global_timer() - t0 < 1000000ull) {}
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // both operands MN-major (bits 15 and 16): 64-wide atoms 8 KB apart (leading offset), groups of
+            // eight batch rows 1024 bytes apart (stride offset), a K step of 16 batch rows is 2048 bytes
+            const uint32_t idesc = instr_desc(kTileM, kTileN, 1) | (1u << 15);
+            uint32_t s = 0, phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < num_kblocks; ++kb) {
+                ok = mbar_wait(bar_full + 8 * s, phase, abort_flag);
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint32_t sa = base + s * kDwStageBytes;
+                const uint64_t a = smem_desc(sa, kDwOperandBytes / 2, 1024);
+                const uint64_t b = smem_desc(sa + kDwOperandBytes, kDwOperandBytes / 2, 1024);
+                constexpr uint64_t kstep = 2048 >> 4;
+                umma_bf16(tmem_acc, a, b, idesc, kb ? 1u : 0u);
+                umma_bf16(tmem_acc, a + kstep, b + kstep, idesc, 1u);
+                umma_bf16(tmem_acc, a + 2 * kstep, b + 2 * kstep, idesc, 1u);
+                umma_bf16(tmem_acc, a + 3 * kstep, b + 3 * kstep, idesc, 1u);
+                tcgen05_commit(bar_empty + 8 * s);
+                if (++s == kDwStages) {
+                    s = 0;
+                    phase ^= 1;
+                }
+            }
+            if (ok) tcgen05_commit(bar_acc);
+        }
+        __syncwarp();
+    } else {
+        // epilogue: the accumulator is complete, so every MMA has retired and the ring is free.
+        // Box q (columns 32 q .. 32 q + 31) is a 128 x 32 fp32 array of 128-byte rows with the 16-byte
+        // chunks of row r stored at chunk ^ (r & 7): the layout of a 128-byte-swizzled tensor map.
+        const int quarter = warp & 3;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, abort_flag));
+        tcgen05_fence_after();
+        if (ok) {
+            const int row = quarter * 32 + lane;
+#pragma unroll 1
+            for (int q = 0; q < kTileN / 32; ++q) {
+                uint32_t v[32];
+                tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(32 * q), v);
+                const uint32_t rowaddr = base + (uint32_t)q * (kTileM * 128) + (uint32_t)row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                 ::"r"(rowaddr + (uint32_t)((c ^ (row & 7)) << 4)), "r"(v[4 * c]), "r"(v[4 * c + 1]),
+                                   "r"(v[4 * c + 2]), "r"(v[4 * c + 3]) : "memory");
+            }
+            fence_proxy_async();
+        }
+        // the four epilogue warps meet, then one thread hands the tile to TMA
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ok && warp == 2 && lane == 0) {
+            const CUtensorMap *omap = &P.dw_map[wi * P.pfi + wj];
+#pragma unroll
+            for (int q = 0; q < kTileN / 32; ++q) tma_store_2d(omap, base + (uint32_t)q * (kTileM * 128), n0 + 32 * q, m0);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory read out before the block retires
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kTileN) : "memory");
+    }
+}
+
+// db_i[o] = sum over the batch of dy_i[b, o], fp32 sums of bf16 values in a fixed order: the batch is cut
+// into eight contiguous chunks (one per warp, rows ascending inside a chunk) and the chunk sums are
+// added in chunk order.  A block covers 64 columns of one dy block.
+struct AffineDbParams {
+    const uint16_t *dy[8];
+    float *db[8];
+    int32_t nb, bfo;
+};
+constexpr int kDbThreads = 256;
+__global__ void __launch_bounds__(kDbThreads) affine_db_kernel(const AffineDbParams P) {
+    __shared__ float part[kDbThreads / 32][64];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int col = blockIdx.x * 64 + 2 * lane;
+    const int i = blockIdx.y;
+    const int chunk = (P.nb + kDbThreads / 32 - 1) / (kDbThreads / 32);
+    const int b0 = warp * chunk, b1 = min(P.nb, b0 + chunk);
+    const uint16_t *src = P.dy[i] + col;
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+    for (int b = b0; b < b1; ++b) {
+        const uint32_t two = *reinterpret_cast<const uint32_t *>(src + (size_t)b * P.bfo);
+        s0 += __uint_as_float(two << 16);
+        s1 += __uint_as_float(two & 0xffff0000u);
+    }
+    part[warp][2 * lane] = s0;
+    part[warp][2 * lane + 1] = s1;
+    __syncthreads();
+    if (threadIdx.x < 64) {
+        float v = part[0][threadIdx.x];
+#pragma unroll
+        for (int w = 1; w < kDbThreads / 32; ++w) v += part[w][threadIdx.x];
+        P.db[i][blockIdx.x * 64 + threadIdx.x] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 static EncodeTiledFn encode_fn() { return tensor_map_encoder(); }
@@ -734,6 +937,83 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
     return DISTDL_OK;
 }
 
+static bool make_map_f32(CUtensorMap *m, const void *ptr, int64_t rows, int64_t cols, int box_cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                          const void *const *dy, const void *const *x, void *const *dw,
+                                          void *const *db, void *stream) {
+    const char *what = "affine_adj_params";
+    clear_error();
+    if (!dy || !x || !dw) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (nb < 1 || nfi < 1 || nfo < 1 || pfo < 1 || pfi < 1) return fail(DISTDL_ERR_INVALID_ARG, "%s: non-positive size", what);
+    if (nfi % pfi || nfo % pfo) return fail(DISTDL_ERR_SHAPE, "%s: features not divisible by the worker grid", what);
+    const int64_t bfi = nfi / pfi, bfo = nfo / pfo;
+    if (bfi % kTileN || bfo % kTileM)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: per-worker feature blocks must be multiples of %d", what, kTileN);
+    if (pfo > 8 || pfi > 8 || pfo * pfi > kMaxMaps - 8)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: worker grid larger than 8 per side or %d workers", what, kMaxMaps - 8);
+    if (nb > (1 << 20)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: batch too large", what);
+    for (int i = 0; i < pfo; ++i) {
+        if (!dy[i] || (db && !db[i])) return fail(DISTDL_ERR_INVALID_ARG, "%s: dy / db block %d is NULL", what, i);
+        if (!aligned16(dy[i]) || (db && !aligned16(db[i]))) return fail(DISTDL_ERR_ALIGNMENT, "%s: dy / db block %d not 16-byte aligned", what, i);
+    }
+    for (int j = 0; j < pfi; ++j) {
+        if (!x[j]) return fail(DISTDL_ERR_INVALID_ARG, "%s: x block %d is NULL", what, j);
+        if (!aligned16(x[j])) return fail(DISTDL_ERR_ALIGNMENT, "%s: x block %d not 16-byte aligned", what, j);
+    }
+    for (int i = 0; i < pfo * pfi; ++i) {
+        if (!dw[i]) return fail(DISTDL_ERR_INVALID_ARG, "%s: dW block %d is NULL", what, i);
+        if (!aligned16(dw[i])) return fail(DISTDL_ERR_ALIGNMENT, "%s: dW block %d not 16-byte aligned", what, i);
+    }
+    if (!encode_fn()) return fail(DISTDL_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", what);
+    const int64_t tiles = (bfo / kTileM) * (bfi / kTileN) * pfo * pfi;
+    if (tiles >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
+
+    AffineDwParams P;
+    memset(&P, 0, sizeof(P));
+    for (int i = 0; i < pfo; ++i)
+        if (!make_map(&P.dy_map[i], dy[i], nb, bfo, 64, kBlockK)) return fail(DISTDL_ERR_CUDA, "%s: tensor map of dy block %d failed", what, i);
+    for (int j = 0; j < pfi; ++j)
+        if (!make_map(&P.x_map[j], x[j], nb, bfi, 64, kBlockK)) return fail(DISTDL_ERR_CUDA, "%s: tensor map of x block %d failed", what, j);
+    for (int i = 0; i < pfo * pfi; ++i)
+        if (!make_map_f32(&P.dw_map[i], dw[i], bfo, bfi, 32, kTileM)) return fail(DISTDL_ERR_CUDA, "%s: tensor map of dW block %d failed", what, i);
+    P.nb = (int32_t)nb;
+    P.pfi = pfi;
+    P.tiles_m = (int32_t)(bfo / kTileM);
+    P.tiles_n = (int32_t)(bfi / kTileN);
+    static bool configured = false;
+    if (!configured) {
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemBytes));
+        configured = true;
+    }
+    affine_dw_kernel<<<(unsigned)tiles, kDwThreads, kDwSmemBytes, (cudaStream_t)stream>>>(P);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    if (db) {
+        AffineDbParams B;
+        memset(&B, 0, sizeof(B));
+        for (int i = 0; i < pfo; ++i) {
+            B.dy[i] = (const uint16_t *)dy[i];
+            B.db[i] = (float *)db[i];
+        }
+        B.nb = (int32_t)nb;
+        B.bfo = (int32_t)bfo;
+        dim3 grid((unsigned)(bfo / 64), (unsigned)pfo);
+        affine_db_kernel<<<grid, kDbThreads, 0, (cudaStream_t)stream>>>(B);
+        DISTDL_CUDA_CHECK(cudaGetLastError());
+    }
+    return DISTDL_OK;
+}
+
 }  // namespace distdl
 
 extern "C" distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
@@ -746,6 +1026,12 @@ extern "C" distdl_status_t distdl_affine_adj(int64_t nb, int64_t nfi, int64_t nf
                                              const void *const *dy, const void *const *w, void *const *dx,
                                              void *stream) {
     return distdl::affine_impl(nb, nfi, nfo, pfo, pfi, dy, w, nullptr, dx, stream, true, "affine_adj");
+}
+
+extern "C" distdl_status_t distdl_affine_adj_params(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,
+                                                    const void *const *dy, const void *const *x, void *const *dw,
+                                                    void *const *db, void *stream) {
+    return distdl::affine_params_impl(nb, nfi, nfo, pfo, pfi, dy, x, dw, db, stream);
 }
 
 namespace distdl {

@@ -828,6 +828,344 @@ static distdl_status_t conv_impl(const distdl_partition *p, const void *const *i
     return launch_conv<7, true>(P, tt, tiles_y, pl, s);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Parameter gradients of the layer (adjoint convolution algorithm, Section 4 "Sparse layers"):
+//   dw^_k[c,a,b] = sum_{n,i,j} dy_k[n,c,i,j] * (H x)_k[n,c,i+a,j+b],   db^_k[c] = sum dy_k[n,c,i,j],
+//   dw = R_k dw^_k,  db = R_k db^_k      (every worker holds a copy of the kernel).
+// H is fused as in the forward kernel: a block stages the x tile with its ghost rows and columns
+// straight from the neighbouring shards' bulk, and the dy tile beside it.  A work item is one
+// (channel, slice): the tiles slice, slice + S, slice + 2 S, ... of that channel's planes across all
+// workers, so the K*K + 1 running sums stay in registers from tile to tile.  Every thread owns 4 x 8
+// pixels of a tile and keeps each sum as a pair (even pixel column, odd pixel column) for the
+// packed fp32 FMAs.  At the end of an item the block folds its sums (lanes by shuffles, warps in
+// order) and writes one row of K*K + 1 values to the scratch table; a second small kernel adds the
+// S rows of a channel in order.  The assignment of tiles to sums is static, so the result does not
+// change from run to run.
+// ---------------------------------------------------------------------------------------------
+constexpr int kGradRow = 64;   // floats per (channel, slice) row of the scratch table (K*K + 1 <= 50 used)
+
+struct ConvGradParams {
+    ConvParams base;                        // in = padded x shards; out unused
+    const float *dy[kConvMaxWorkers];       // bulk-shaped shards
+    float *partial;                         // [channels][slices][kGradRow]
+    int32_t slices;
+    int32_t tiles_per_plane;                // Ph * tiles_y * Pw * tiles_x
+    int32_t tiles_per_channel;              // batch * tiles_per_plane
+    int32_t tiles_y;
+};
+
+// dy tile: kTileH rows of kTileW floats, zero outside the shard's bulk
+__device__ __forceinline__ void stage_dy_tile(const ConvGradParams &G, const ConvTile &t, float *dt) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rows = min(kTileH, t.bh - t.i0), cols = min(kTileW, t.bw - t.j0);
+    const float *plane = G.dy[t.shard] + (size_t)t.plane * t.bh * t.bw;
+    const bool fast = (t.bw % 4) == 0;
+    const int nv = fast ? cols / 4 : 0;
+    for (int ry = warp; ry < kTileH; ry += kConvThreads / 32) {
+        float *srow = dt + ry * kTileW;
+        if (ry >= rows) {
+            for (int v = lane; v < kTileW / 4; v += 32) *reinterpret_cast<float4 *>(srow + 4 * v) = make_float4(0.f, 0.f, 0.f, 0.f);
+            continue;
+        }
+        const float *grow = plane + (size_t)(t.i0 + ry) * t.bw + t.j0;
+        for (int v = lane; v < nv; v += 32) cp_async16(srow + 4 * v, grow + 4 * v);
+        for (int e = 4 * nv + lane; e < kTileW; e += 32) {
+            if (e < cols) cp_async4(srow + e, grow + e);
+            else srow[e] = 0.f;
+        }
+    }
+}
+
+// Cells of the x tile that stage_tile leaves untouched when the tile is ragged: set to zero, so that
+// the products with the zeros of the dy tile are zeros whatever an earlier tile left there.
+template <int K>
+__device__ __forceinline__ void clear_unstaged_x(const ConvTile &t, float *tile) {
+    using C = ConvCfg<K, false>;
+    const int out_rows = min(kTileH, t.bh - t.i0), out_cols = min(kTileW, t.bw - t.j0);
+    if (out_rows == kTileH && out_cols == kTileW) return;
+    const int need_rows = out_rows + 2 * C::PH;
+    const int staged = ((out_cols + C::PADL + C::PH + 3) / 4) * 4;
+    for (int idx = threadIdx.x; idx < C::ROWS * C::PITCH; idx += kConvThreads) {
+        const int ry = idx / C::PITCH, s = idx - ry * C::PITCH;
+        if (ry >= need_rows || s >= staged) tile[idx] = 0.f;
+    }
+}
+
+template <int K>
+__device__ __forceinline__ void grad_accumulate(const float *xt, const float *dt, uint64_t (&acc)[K][K], uint64_t &accb) {
+    using C = ConvCfg<K, false>;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    constexpr int NP = C::NF / 2;
+    uint64_t D[kRowsPerThread][4];
+#pragma unroll
+    for (int r = 0; r < kRowsPerThread; ++r) {
+        const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(dt + (ty * kRowsPerThread + r) * kTileW + kColsPerThread * tx);
+        const ulonglong2 q0 = src[0], q1 = src[1];
+        D[r][0] = q0.x;
+        D[r][1] = q0.y;
+        D[r][2] = q1.x;
+        D[r][3] = q1.y;
+    }
+    const uint64_t ones = pack2(1.f, 1.f);
+#pragma unroll
+    for (int r = 0; r < kRowsPerThread; ++r)
+#pragma unroll
+        for (int p2 = 0; p2 < 4; ++p2) accb = fma2(D[r][p2], ones, accb);
+    const float *tbase = xt + (ty * kRowsPerThread) * C::PITCH + kColsPerThread * tx;
+#pragma unroll
+    for (int rho = 0; rho < kRowsPerThread + K - 1; ++rho) {
+        // one input row: aligned pairs P[i] = (x[2i], x[2i+1]) and shifted pairs Q[i] = (x[2i+1], x[2i+2])
+        uint64_t Pr[NP], Qr[NP - 1];
+        const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(tbase + rho * C::PITCH);
+#pragma unroll
+        for (int v = 0; v < NP / 2; ++v) {
+            const ulonglong2 q = src[v];
+            Pr[2 * v] = q.x;
+            Pr[2 * v + 1] = q.y;
+        }
+#pragma unroll
+        for (int i = 0; i < NP - 1; ++i) {
+            float a0, a1, b0, b1;
+            unpack2(Pr[i], a0, a1);
+            unpack2(Pr[i + 1], b0, b1);
+            Qr[i] = pack2(a1, b0);
+        }
+#pragma unroll
+        for (int r = 0; r < kRowsPerThread; ++r) {
+            const int a = rho - r;
+            if (a < 0 || a >= K) continue;
+#pragma unroll
+            for (int b = 0; b < K; ++b) {
+#pragma unroll
+                for (int p2 = 0; p2 < 4; ++p2) {
+                    // pixels (2 p2, 2 p2 + 1) of output row r read x columns 2 p2 + b, 2 p2 + b + 1
+                    const uint64_t X = (b & 1) ? Qr[p2 + (b - 1) / 2] : Pr[p2 + b / 2];
+                    acc[a][b] = fma2(D[r][p2], X, acc[a][b]);
+                }
+            }
+        }
+    }
+}
+
+template <int K>
+__global__ void __launch_bounds__(kConvThreads, 3)
+conv_grad_kernel(const __grid_constant__ ConvGradParams G) {
+    using C = ConvCfg<K, false>;
+    extern __shared__ __align__(16) float smem[];        // two x tiles, then two dy tiles
+    float *xts = smem;
+    float *dts = smem + 2 * C::TILE_FLOATS;
+    __shared__ float red[kConvThreads / 32][K * K + 1];
+    const ConvParams &P = G.base;
+    const int items = P.channels * G.slices;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int ch = item / G.slices, sl = item - ch * G.slices;
+        uint64_t acc[K][K];
+        uint64_t accb = 0ull;
+#pragma unroll
+        for (int a = 0; a < K; ++a)
+#pragma unroll
+            for (int b = 0; b < K; ++b) acc[a][b] = 0ull;
+        auto tile_of = [&](int L) {
+            const int n = L / G.tiles_per_plane;
+            return decode_tile(P, (n * P.channels + ch) * G.tiles_per_plane + (L - n * G.tiles_per_plane), G.tiles_y, 0);
+        };
+        auto stage = [&](const ConvTile &t, int b) {
+            if (!t.valid) return;
+            float *xt = xts + b * C::TILE_FLOATS;
+            clear_unstaged_x<K>(t, xt);
+            stage_tile<K, false>(P, t, xt);
+            stage_dy_tile(G, t, dts + b * (kTileH * kTileW));
+        };
+        int L = sl, buf = 0;
+        if (L < G.tiles_per_channel) {
+            ConvTile cur = tile_of(L);
+            stage(cur, 0);
+            cp_async_commit();
+            while (true) {
+                const int next = L + G.slices;
+                const bool has_next = next < G.tiles_per_channel;
+                ConvTile nxt = cur;
+                if (has_next) {
+                    nxt = tile_of(next);
+                    stage(nxt, buf ^ 1);
+                }
+                cp_async_commit();
+                cp_async_wait_group<1>();
+                __syncthreads();
+                if (cur.valid) grad_accumulate<K>(xts + buf * C::TILE_FLOATS, dts + buf * (kTileH * kTileW), acc, accb);
+                __syncthreads();
+                if (!has_next) break;
+                cur = nxt;
+                L = next;
+                buf ^= 1;
+            }
+            cp_async_wait_group<0>();
+        }
+        // fold: pair halves, lanes (butterfly), then the warps in order
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+        for (int a = 0; a < K; ++a)
+#pragma unroll
+            for (int b = 0; b <= K; ++b) {
+                if (b == K && a != 0) continue;
+                float lo, hi;
+                unpack2(b == K ? accb : acc[a][b], lo, hi);
+                float v = lo + hi;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) red[warp][b == K ? K * K : a * K + b] = v;
+            }
+        __syncthreads();
+        if (threadIdx.x <= K * K) {
+            float v = red[0][threadIdx.x];
+#pragma unroll
+            for (int w2 = 1; w2 < kConvThreads / 32; ++w2) v += red[w2][threadIdx.x];
+            G.partial[(size_t)item * kGradRow + threadIdx.x] = v;
+        }
+        __syncthreads();
+    }
+}
+
+// dw[c, :, :] and db[c] = the slices' rows of channel c added in order
+__global__ void conv_grad_finish_kernel(const float *partial, int slices, int taps, float *dw, float *db) {
+    const int ch = blockIdx.x, t = threadIdx.x;
+    if (t > taps) return;
+    const float *row = partial + (size_t)ch * slices * kGradRow + t;
+    float v = row[0];
+    for (int s = 1; s < slices; ++s) v += row[(size_t)s * kGradRow];
+    if (t < taps) dw[(size_t)ch * taps + t] = v;
+    else if (db) db[ch] = v;
+}
+
+template <int K>
+static distdl_status_t grad_config(int *blocks_out) {
+    constexpr int smem = 2 * ConvCfg<K, false>::TILE_FLOATS * 4 + 2 * kTileH * kTileW * 4;
+    static bool configured = false;
+    static int blocks = 0;
+    if (!configured) {
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        int dev = 0, sms = 0, per_sm = 0;
+        DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
+        DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, conv_grad_kernel<K>, kConvThreads, smem));
+        blocks = sms * (per_sm > 0 ? per_sm : 1);
+        configured = true;
+    }
+    *blocks_out = blocks;
+    return DISTDL_OK;
+}
+
+// Geometry shared by the workspace query and the launch: slices per channel and tile counts.
+static distdl_status_t grad_plan(const distdl_partition *p, int32_t kh, int32_t kw, const char *what, ConvGradParams *G,
+                                 int *grid) {
+    if (!p) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL partition", what);
+    if (p->rank != 4 || p->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-4 F32 partition", what);
+    if (p->pshape[0] != 1 || p->pshape[1] != 1)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: only the feature-space dimensions may be partitioned", what);
+    if (kh != kw || (kh != 3 && kh != 5 && kh != 7))
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: kernel %d x %d (supported: 3x3, 5x5, 7x7)", what, kh, kw);
+    if (p->num_workers > kConvMaxWorkers) return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d workers", what, kConvMaxWorkers);
+    const int h = kh / 2;
+    for (int k = 0; k < 4; ++k)
+        for (int32_t c = 0; c < p->pshape[k]; ++c) {
+            const int want = k < 2 ? 0 : h;
+            if (p->hlo[k][c] != want || p->hhi[k][c] != want)
+                return fail(DISTDL_ERR_SHAPE, "%s: halo widths must be 0,0,%d,%d on every side", what, h, h);
+        }
+    ConvParams &P = G->base;
+    int64_t max_bh = 0, max_bw = 0;
+    for (int32_t r = 0; r < p->pshape[2]; ++r) {
+        P.bh[r] = (int32_t)p->size[2][r];
+        max_bh = std::max<int64_t>(max_bh, p->size[2][r]);
+    }
+    for (int32_t c = 0; c < p->pshape[3]; ++c) {
+        P.bw[c] = (int32_t)p->size[3][c];
+        max_bw = std::max<int64_t>(max_bw, p->size[3][c]);
+    }
+    P.ph_workers = p->pshape[2];
+    P.pw_workers = p->pshape[3];
+    P.channels = (int32_t)p->global_shape[1];
+    P.tiles_x = (int32_t)((max_bw + kTileW - 1) / kTileW);
+    const int tiles_y = (int)((max_bh + kTileH - 1) / kTileH);
+    conv_set_divisor(P, 0, (uint32_t)P.tiles_x);
+    conv_set_divisor(P, 1, (uint32_t)P.pw_workers);
+    conv_set_divisor(P, 2, (uint32_t)tiles_y);
+    conv_set_divisor(P, 3, (uint32_t)P.ph_workers);
+    const int64_t per_plane = (int64_t)P.tiles_x * tiles_y * p->num_workers;
+    const int64_t per_channel = per_plane * p->global_shape[0];
+    if (per_channel * P.channels >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
+    int blocks = 0;
+    distdl_status_t st = kh == 3 ? grad_config<3>(&blocks) : kh == 5 ? grad_config<5>(&blocks) : grad_config<7>(&blocks);
+    if (st != DISTDL_OK) return st;
+    // enough slices per channel to give every resident block an item, never more than tiles
+    int64_t slices = (blocks + P.channels - 1) / P.channels;
+    slices = std::max<int64_t>(1, std::min<int64_t>(slices, per_channel));
+    G->slices = (int32_t)slices;
+    G->tiles_per_plane = (int32_t)per_plane;
+    G->tiles_per_channel = (int32_t)per_channel;
+    G->tiles_y = tiles_y;
+    *grid = (int)std::min<int64_t>(blocks, slices * P.channels);
+    return DISTDL_OK;
+}
+
+template <int K>
+static distdl_status_t launch_grad(const ConvGradParams &G, int grid, float *dw, float *db, cudaStream_t s) {
+    constexpr int smem = 2 * ConvCfg<K, false>::TILE_FLOATS * 4 + 2 * kTileH * kTileW * 4;
+    conv_grad_kernel<K><<<grid, kConvThreads, smem, s>>>(G);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    conv_grad_finish_kernel<<<G.base.channels, 64, 0, s>>>(G.partial, G.slices, K * K, dw, db);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+}  // namespace distdl
+
+extern "C" distdl_status_t distdl_conv_adj_params_workspace(const distdl_partition_t *p, int32_t kh, int32_t kw,
+                                                            int64_t *bytes) {
+    using namespace distdl;
+    clear_error();
+    if (!bytes) return fail(DISTDL_ERR_INVALID_ARG, "conv_adj_params_workspace: NULL argument");
+    ConvGradParams G;
+    memset(&G, 0, sizeof(G));
+    int grid = 0;
+    const distdl_status_t st = grad_plan(p, kh, kw, "conv_adj_params_workspace", &G, &grid);
+    if (st != DISTDL_OK) return st;
+    *bytes = (int64_t)G.base.channels * G.slices * kGradRow * (int64_t)sizeof(float);
+    return DISTDL_OK;
+}
+
+extern "C" distdl_status_t distdl_conv_adj_params(const distdl_partition_t *p, const void *const *x,
+                                                  const void *const *dy, int32_t kh, int32_t kw, void *dw, void *db,
+                                                  void *workspace, int64_t workspace_bytes, void *stream) {
+    using namespace distdl;
+    clear_error();
+    const char *what = "conv_adj_params";
+    if (!p || !x || !dy || !dw || !workspace) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    ConvGradParams G;
+    memset(&G, 0, sizeof(G));
+    int grid = 0;
+    const distdl_status_t st = grad_plan(p, kh, kw, what, &G, &grid);
+    if (st != DISTDL_OK) return st;
+    const int64_t need = (int64_t)G.base.channels * G.slices * kGradRow * (int64_t)sizeof(float);
+    if (workspace_bytes < need) return fail(DISTDL_ERR_INVALID_ARG, "%s: workspace of %lld bytes, %lld needed", what,
+                                            (long long)workspace_bytes, (long long)need);
+    if (!aligned16(dw) || !aligned16(workspace) || (db && !aligned16(db)))
+        return fail(DISTDL_ERR_ALIGNMENT, "%s: dw / db / workspace not 16-byte aligned", what);
+    for (int32_t wk = 0; wk < p->num_workers; ++wk) {
+        if (!x[wk] || !dy[wk]) return fail(DISTDL_ERR_INVALID_ARG, "%s: shard pointer %d is NULL", what, wk);
+        if (!aligned16(x[wk]) || !aligned16(dy[wk])) return fail(DISTDL_ERR_ALIGNMENT, "%s: shard %d is not 16-byte aligned", what, wk);
+        G.base.in[wk] = (const float *)x[wk];
+        G.dy[wk] = (const float *)dy[wk];
+    }
+    G.partial = (float *)workspace;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (kh == 3) return launch_grad<3>(G, grid, (float *)dw, (float *)db, s);
+    if (kh == 5) return launch_grad<5>(G, grid, (float *)dw, (float *)db, s);
+    return launch_grad<7>(G, grid, (float *)dw, (float *)db, s);
+}
+
+namespace distdl {
+
 }  // namespace distdl
 
 extern "C" distdl_status_t distdl_conv_fwd(const distdl_partition_t *p, const void *const *x, const void *w,

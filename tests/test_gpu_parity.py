@@ -292,6 +292,56 @@ def test_conv_fwd_and_adj(case):
     assert r < 1e-5
 
 
+@pytest.mark.parametrize("case", CONV_CASES, ids=[str(c) for c in CONV_CASES])
+@pytest.mark.parametrize("integer", [True, False], ids=["int", "normal"])
+def test_conv_param_gradients(case, integer):
+    gshape, pshape, k = case
+    h = k // 2
+    hl = (0, 0, h, h)
+    opart = oracle.Partition(gshape, pshape, hl, hl)
+    obulk = oracle.Partition(gshape, pshape, 0, 0)
+    gpart = distdl.Partition(gshape, pshape, hl, hl)
+    gen = (lambda shp, seed: inputs.integers(shp, seed, -3, 4)) if integer else inputs.normal
+    xg, dyg = gen(gshape, 35), gen(gshape, 36)
+    # ghosts hold garbage: the fused exchange must not read them
+    x = oracle.scatter_global(opart, xg, fill=lambda wk: np.full(opart.padded_shape(wk), 1e30, dtype=np.float32))
+    dy = oracle.scatter_global(obulk, dyg)
+    xs, dys = [dev(a) for a in x], [dev(a) for a in dy]
+    C = gshape[1]
+    dw = torch.full((C, k, k), -5.0, device=DEV)
+    db = torch.full((C,), -5.0, device=DEV)
+    ws = torch.empty(distdl.conv_adj_params_workspace(gpart, k, k), dtype=torch.uint8, device=DEV)
+    for _ in range(2):                                   # twice: the scratch table is reused
+        distdl.conv_adj_params(gpart, xs, dys, (k, k), dw, db, ws)
+    torch.cuda.synchronize()
+    dw_ref, db_ref = oracle.conv_adj_params(opart, x, dy, k, k)
+    if integer:
+        # |terms| <= 9, fewer than 2^20 of them: every partial sum is an exact integer in fp32, any order
+        assert np.array_equal(host(dw), dw_ref) and np.array_equal(host(db), db_ref)
+    else:
+        # fp32 running sums: the longest chain has 16 terms per tile of the channel (a thread's pair half),
+        # then the folds over pair halves, lanes, warps and slices
+        tiles = gshape[0] * sum(-(-obulk.padded_shape(wk)[2] // 32) * -(-obulk.padded_shape(wk)[3] // 128)
+                                for wk in range(opart.num_workers))
+        eps = (16 * tiles + 64) * 2.0 ** -24
+        mag_w, mag_b = oracle.conv_adj_params(opart, [np.abs(a) for a in oracle.scatter_global(opart, xg)],
+                                              [np.abs(a) for a in dy], k, k)
+        assert np.all(np.abs(host(dw).astype(np.float64) - dw_ref) <= eps * mag_w)
+        assert np.all(np.abs(host(db).astype(np.float64) - db_ref) <= eps * mag_b)
+        assert np.linalg.norm(host(dw).astype(np.float64) - dw_ref) <= 1e-5 * np.linalg.norm(mag_w)
+    for wk in range(opart.num_workers):
+        assert same_bits(host(xs[wk]), x[wk])
+    if not integer:
+        # dot test in parameter space, forward through the CUDA layer: <Conv(w, b; x), dy> = <w, dw> + <b, db>
+        w = inputs.normal((C, k, k), 37, 0.1)
+        bias = inputs.normal((C,), 38)
+        ys = [torch.empty(obulk.padded_shape(wk), device=DEV) for wk in range(opart.num_workers)]
+        distdl.conv_fwd(gpart, xs, dev(w), dev(bias), ys)
+        torch.cuda.synchronize()
+        r = oracle.adjoint_test_ratio([host(t) for t in ys], dy, [w, bias], [host(dw), host(db)])
+        assert r < 1e-5
+
+
 # --------------------------------------------------------------------------
 # Affine layer
 # --------------------------------------------------------------------------
@@ -369,6 +419,44 @@ def test_affine_fwd_and_adj(case, integer):
         distdl.device_status()
         r = oracle.adjoint_test_ratio([host(t) for t in y0], dyf, xf, dx)
         assert r < 1e-4
+
+
+@pytest.mark.parametrize("case", AFFINE_CASES, ids=[str(c) for c in AFFINE_CASES])
+@pytest.mark.parametrize("integer", [True, False], ids=["int", "normal"])
+def test_affine_param_gradients(case, integer):
+    nb, nfi, nfo, pfo, pfi = case
+    xs, ws, dys = _affine_inputs(nb, nfi, nfo, pfo, pfi, 45, integer)
+    x_d, dy_d = [_bf16_dev(a) for a in xs], [_bf16_dev(a) for a in dys]
+    dw_d = [torch.full((nfo // pfo, nfi // pfi), -9.0, device=DEV) for _ in range(pfo * pfi)]
+    db_d = [torch.full((nfo // pfo,), -9.0, device=DEV) for _ in range(pfo)]
+    distdl.affine_adj_params(nb, nfi, nfo, pfo, pfi, dy_d, x_d, dw_d, db_d)
+    distdl.device_status()
+    xf = [oracle.bf16_bits_to_f64(a) for a in xs]
+    dyf = [oracle.bf16_bits_to_f64(a) for a in dys]
+    dw_ref, db_ref = oracle.affine_adj_params(dyf, xf, pfo, pfi)
+    dw, db = [host(t) for t in dw_d], [host(t) for t in db_d]
+    if integer:
+        for a, b in zip(dw + db, dw_ref + db_ref):
+            assert np.array_equal(a, b)
+    else:
+        for got, ref in zip(dw, dw_ref):
+            emax, el2 = _rel_errors([got], [ref])
+            assert emax < 2e-2 and el2 < 2e-2
+            assert emax < 1e-4 and el2 < 1e-5
+        emax, el2 = _rel_errors([np.concatenate(db)[None]], [np.concatenate(db_ref)[None]])
+        assert emax < 1e-5 and el2 < 1e-5
+        # dot test in parameter space, forward through the CUDA layer: <Affine(W, b; x), dy> = <W, dW> + <b, db>
+        w_d = [_bf16_dev(a) for a in ws]
+        bias = np.split(inputs.normal((nfo,), 46), pfo)
+        y_d = [torch.empty((nb, nfo // pfo), device=DEV) for _ in range(pfo)]
+        distdl.affine_fwd(nb, nfi, nfo, pfo, pfi, x_d, w_d, [dev(b) for b in bias], y_d)
+        distdl.device_status()
+        wf = [oracle.bf16_bits_to_f64(a) for a in ws]
+        r = oracle.adjoint_test_ratio([host(t) for t in y_d], dyf, wf + bias, dw + db)
+        assert r < 1e-4
+    # db is optional
+    distdl.affine_adj_params(nb, nfi, nfo, pfo, pfi, dy_d, x_d, dw_d, None)
+    distdl.device_status()
 
 
 # --------------------------------------------------------------------------
