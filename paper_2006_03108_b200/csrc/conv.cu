@@ -520,10 +520,15 @@ __device__ __forceinline__ void for_each_patch_cell(const ConvTile &t, F f) {
             for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, r, colS + s);
         q0 += C::PH * W;
     }
-    if (t.i0 + out_rows == t.bh) {
+    // rows / columns of the tile that lie beyond the shard's bulk: all PH of them in the last tile, and
+    // some already in the tile before it when the last one holds fewer than PH rows / columns
+    const int nbot = min(C::PH, max(0, t.i0 + out_rows + C::PH - t.bh));
+    const int nright = min(C::PH, max(0, t.j0 + out_cols + C::PH - t.bw));
+    if (nbot > 0) {
 #pragma unroll
         for (int r = 0; r < C::PH; ++r)
-            for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, rowB + r, colS + s);
+            if (r < nbot)
+                for (int s = threadIdx.x; s < W; s += kConvThreads) f(q0 + r * W + s, rowB + C::PH - nbot + r, colS + s);
         q0 += C::PH * W;
     }
     if (t.j0 == 0) {
@@ -532,35 +537,19 @@ __device__ __forceinline__ void for_each_patch_cell(const ConvTile &t, F f) {
             for (int c = 0; c < C::PH; ++c) f(q0 + ry * C::PH + c, ry, colL + c);
         q0 += C::PH * H;
     }
-    if (t.j0 + out_cols == t.bw) {
+    if (nright > 0) {
         for (int ry = threadIdx.x; ry < H; ry += kConvThreads)
 #pragma unroll
-            for (int c = 0; c < C::PH; ++c) f(q0 + ry * C::PH + c, ry, colR + c);
+            for (int c = 0; c < C::PH; ++c)
+                if (c < nright) f(q0 + ry * C::PH + c, ry, colR + C::PH - nright + c);
     }
 }
 
+// Fetches the halo strips of tile t (cells that belong to neighbouring shards, or zeros outside the
+// tensor) into the side buffer, cell by cell.
 template <int K, bool ADJ>
-__device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const ConvTile &t, float *tile, float *side,
-                                               float *wk, uint32_t bar) {
+__device__ __forceinline__ void stage_halo_strips(const ConvParams &P, const ConvTile &t, float *side) {
     using C = ConvCfg<K, ADJ>;
-    using T = ConvTmaCfg<K, ADJ>;
-    const ConvParams &P = Q.base;
-    if (!t.valid) return;
-    if (threadIdx.x == 0) {
-        fence_proxy_async();     // earlier generic-proxy accesses to this buffer are ordered before the bulk copy
-        mbar_expect_tx(bar, T::BOX_BYTES);
-        // forward: padded coordinates (bulk column j sits at j + PH); adjoint: bulk coordinates
-        const int x = ADJ ? t.j0 - C::PADL : t.j0;
-        const int y = ADJ ? t.i0 - C::PH : t.i0;
-        tma_load_3d(smem_u32(tile), &Q.in_map[t.shard], x, y, t.plane, bar);
-    }
-    // this channel's weights and bias
-    if (threadIdx.x <= K * K) {
-        const int ch = t.plane % P.channels;
-        if (threadIdx.x < K * K) cp_async4(wk + threadIdx.x, P.w + (size_t)ch * K * K + threadIdx.x);
-        else if (P.bias) cp_async4(wk + K * K, P.bias + ch);
-        else wk[K * K] = 0.f;
-    }
     for_each_patch_cell<K, ADJ>(t, [&](int q, int ry, int s) {
         int i = t.i0 - C::PH + ry, rr = t.r;
         bool ok = true;
@@ -598,6 +587,31 @@ __device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const Con
             side[q] = 0.f;
         }
     });
+}
+
+template <int K, bool ADJ>
+__device__ __forceinline__ void stage_tile_tma(const ConvTmaParams &Q, const ConvTile &t, float *tile, float *side,
+                                               float *wk, uint32_t bar) {
+    using C = ConvCfg<K, ADJ>;
+    using T = ConvTmaCfg<K, ADJ>;
+    const ConvParams &P = Q.base;
+    if (!t.valid) return;
+    if (threadIdx.x == 0) {
+        fence_proxy_async();     // earlier generic-proxy accesses to this buffer are ordered before the bulk copy
+        mbar_expect_tx(bar, T::BOX_BYTES);
+        // forward: padded coordinates (bulk column j sits at j + PH); adjoint: bulk coordinates
+        const int x = ADJ ? t.j0 - C::PADL : t.j0;
+        const int y = ADJ ? t.i0 - C::PH : t.i0;
+        tma_load_3d(smem_u32(tile), &Q.in_map[t.shard], x, y, t.plane, bar);
+    }
+    // this channel's weights and bias
+    if (threadIdx.x <= K * K) {
+        const int ch = t.plane % P.channels;
+        if (threadIdx.x < K * K) cp_async4(wk + threadIdx.x, P.w + (size_t)ch * K * K + threadIdx.x);
+        else if (P.bias) cp_async4(wk + K * K, P.bias + ch);
+        else wk[K * K] = 0.f;
+    }
+    stage_halo_strips<K, ADJ>(P, t, side);
 }
 
 template <int K, bool ADJ>
@@ -1026,6 +1040,154 @@ conv_grad_kernel(const __grid_constant__ ConvGradParams G) {
     }
 }
 
+// TMA variant of the parameter-gradient kernel: the x tile body and (when every shard's rows are
+// whole 16-byte units) the dy tile arrive by one bulk tensor copy each -- out-of-range parts of a
+// ragged tile are filled with zeros by the copy -- and only the halo strips are fetched cell by cell.
+struct ConvGradTmaParams {
+    ConvGradParams g;
+    CUtensorMap x_map[kConvTmaMaxWorkers];
+    CUtensorMap dy_map[kConvTmaMaxWorkers];
+};
+
+template <int K, bool DYTMA>
+__global__ void __launch_bounds__(kConvThreads, 3)
+conv_grad_tma_kernel(const __grid_constant__ ConvGradTmaParams Q) {
+    using C = ConvCfg<K, false>;
+    using T = ConvTmaCfg<K, false>;
+    constexpr int DY_FLOATS = kTileH * kTileW;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    float *tiles = reinterpret_cast<float *>(smem_raw + (((raw + 127u) & ~127u) - raw));
+    float *sides = tiles + 2 * T::TILE_STRIDE;
+    float *dts = sides + 2 * T::SIDE_STRIDE;
+    const uint32_t bars = smem_u32(dts + 2 * DY_FLOATS);
+    // the fold at the end of an item reuses the first x tile buffer (idle by then): no static shared memory,
+    // which is what lets three blocks share an SM for K = 5
+    float (*red)[K * K + 1] = reinterpret_cast<float (*)[K * K + 1]>(tiles);
+    const ConvGradParams &G = Q.g;
+    const ConvParams &P = G.base;
+    if (threadIdx.x == 0) {
+        mbar_init(bars, 1);
+        mbar_init(bars + 8, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    uint32_t phase0 = 0, phase1 = 0;
+    bool failed = false;
+    const int items = P.channels * G.slices;
+    for (int item = blockIdx.x; item < items && !failed; item += gridDim.x) {
+        const int ch = item / G.slices, sl = item - ch * G.slices;
+        uint64_t acc[K][K];
+        uint64_t accb = 0ull;
+#pragma unroll
+        for (int a = 0; a < K; ++a)
+#pragma unroll
+            for (int b = 0; b < K; ++b) acc[a][b] = 0ull;
+        auto tile_of = [&](int L) {
+            const int n = L / G.tiles_per_plane;
+            return decode_tile(P, (n * P.channels + ch) * G.tiles_per_plane + (L - n * G.tiles_per_plane), G.tiles_y, 0);
+        };
+        auto stage = [&](const ConvTile &t, int b) {
+            if (!t.valid) return;
+            float *xt = tiles + b * T::TILE_STRIDE, *dt = dts + b * DY_FLOATS;
+            if (threadIdx.x == 0) {
+                fence_proxy_async();
+                mbar_expect_tx(bars + 8 * b, T::BOX_BYTES + (DYTMA ? DY_FLOATS * 4 : 0));
+                tma_load_3d(smem_u32(xt), &Q.x_map[t.shard], t.j0, t.i0, t.plane, bars + 8 * b);
+                if (DYTMA) tma_load_3d(smem_u32(dt), &Q.dy_map[t.shard], t.j0, t.i0, t.plane, bars + 8 * b);
+            }
+            if (!DYTMA) stage_dy_tile(G, t, dt);
+            stage_halo_strips<K, false>(P, t, sides + b * T::SIDE_STRIDE);
+        };
+        int L = sl, buf = 0;
+        if (L < G.tiles_per_channel) {
+            ConvTile cur = tile_of(L);
+            stage(cur, 0);
+            cp_async_commit();
+            while (true) {
+                const int next = L + G.slices;
+                const bool has_next = next < G.tiles_per_channel;
+                ConvTile nxt = cur;
+                if (has_next) {
+                    nxt = tile_of(next);
+                    stage(nxt, buf ^ 1);
+                }
+                cp_async_commit();
+                cp_async_wait_group<1>();
+                bool ok = true;
+                if (cur.valid) {
+                    const uint32_t bar = bars + 8 * buf, parity = buf ? phase1 : phase0;
+                    if (!mbar_try_wait(bar, parity)) {
+                        const uint64_t t0 = global_timer();
+                        while (!mbar_try_wait(bar, parity)) {
+                            if (global_timer() - t0 > kConvWaitLimitNs) {
+                                ok = false;
+                                break;
+                            }
+                        }
+                    }
+                    if (buf) phase1 ^= 1; else phase0 ^= 1;
+                }
+                if (__syncthreads_or(!ok)) {
+                    if (threadIdx.x == 0) {
+                        atomicExch(&g_conv_status, (int)DISTDL_ERR_TIMEOUT);
+                        const uint64_t t0 = global_timer();
+                        while (global_timer() - t0 < 1000000ull) {}
+                    }
+                    failed = true;
+                    break;
+                }
+                float *tl = tiles + buf * T::TILE_STRIDE;
+                if (cur.valid) {
+                    const float *sd = sides + buf * T::SIDE_STRIDE;
+                    for_each_patch_cell<K, false>(cur, [&](int q, int ry, int s2) { tl[ry * C::PITCH + s2] = sd[q]; });
+                    // ragged tile: what the box holds beyond the cells the tile's own outputs read is ghost
+                    // storage of unknown content; it only ever meets the zeros of the dy tile, but 0 * inf
+                    // is not 0 -- clear it
+                    const int out_rows = min(kTileH, cur.bh - cur.i0), out_cols = min(kTileW, cur.bw - cur.j0);
+                    if (out_rows < kTileH || out_cols < kTileW) {
+                        const int need_rows = out_rows + 2 * C::PH, need_cols = out_cols + 2 * C::PH;
+                        for (int idx = threadIdx.x; idx < C::ROWS * C::PITCH; idx += kConvThreads) {
+                            const int ry = idx / C::PITCH, s2 = idx - ry * C::PITCH;
+                            if (ry >= need_rows || s2 >= need_cols) tl[idx] = 0.f;
+                        }
+                    }
+                }
+                __syncthreads();
+                if (cur.valid) grad_accumulate<K>(tl, dts + buf * DY_FLOATS, acc, accb);
+                __syncthreads();
+                if (!has_next) break;
+                cur = nxt;
+                L = next;
+                buf ^= 1;
+            }
+            cp_async_wait_group<0>();
+        }
+        if (failed) break;
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+        for (int a = 0; a < K; ++a)
+#pragma unroll
+            for (int b = 0; b <= K; ++b) {
+                if (b == K && a != 0) continue;
+                float lo, hi;
+                unpack2(b == K ? accb : acc[a][b], lo, hi);
+                float v = lo + hi;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) red[warp][b == K ? K * K : a * K + b] = v;
+            }
+        __syncthreads();
+        if (threadIdx.x <= K * K) {
+            float v = red[0][threadIdx.x];
+#pragma unroll
+            for (int w2 = 1; w2 < kConvThreads / 32; ++w2) v += red[w2][threadIdx.x];
+            G.partial[(size_t)item * kGradRow + threadIdx.x] = v;
+        }
+        __syncthreads();
+    }
+}
+
 // dw[c, :, :] and db[c] = the slices' rows of channel c added in order
 __global__ void conv_grad_finish_kernel(const float *partial, int slices, int taps, float *dw, float *db) {
     const int ch = blockIdx.x, t = threadIdx.x;
@@ -1038,17 +1200,30 @@ __global__ void conv_grad_finish_kernel(const float *partial, int slices, int ta
 }
 
 template <int K>
+static constexpr int grad_smem_bytes(bool tma) {
+    return tma ? 2 * ConvTmaCfg<K, false>::TILE_STRIDE * 4 + 2 * ConvTmaCfg<K, false>::SIDE_STRIDE * 4 + 2 * kTileH * kTileW * 4 + 64 + 128
+               : 2 * ConvCfg<K, false>::TILE_FLOATS * 4 + 2 * kTileH * kTileW * 4;
+}
+
+// Resident blocks on the current device: the same number for the plain and the TMA kernels (the smaller
+// of their occupancies), so that the slicing -- and with it the order of the sums and the size of the
+// scratch table -- does not depend on which of them a call ends up using.
+template <int K>
 static distdl_status_t grad_config(int *blocks_out) {
-    constexpr int smem = 2 * ConvCfg<K, false>::TILE_FLOATS * 4 + 2 * kTileH * kTileW * 4;
     static bool configured = false;
     static int blocks = 0;
     if (!configured) {
-        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        int dev = 0, sms = 0, per_sm = 0;
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(false)));
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_tma_kernel<K, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(true)));
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_tma_kernel<K, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(true)));
+        int dev = 0, sms = 0, a = 0, b = 0, c = 0;
         DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
         DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, conv_grad_kernel<K>, kConvThreads, smem));
-        blocks = sms * (per_sm > 0 ? per_sm : 1);
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, conv_grad_kernel<K>, kConvThreads, grad_smem_bytes<K>(false)));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, conv_grad_tma_kernel<K, true>, kConvThreads, grad_smem_bytes<K>(true)));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c, conv_grad_tma_kernel<K, false>, kConvThreads, grad_smem_bytes<K>(true)));
+        const int per_sm = std::max(1, std::min(a, std::min(b, c)));
+        blocks = sms * per_sm;
         configured = true;
     }
     *blocks_out = blocks;
@@ -1097,8 +1272,9 @@ static distdl_status_t grad_plan(const distdl_partition *p, int32_t kh, int32_t 
     int blocks = 0;
     distdl_status_t st = kh == 3 ? grad_config<3>(&blocks) : kh == 5 ? grad_config<5>(&blocks) : grad_config<7>(&blocks);
     if (st != DISTDL_OK) return st;
-    // enough slices per channel to give every resident block an item, never more than tiles
-    int64_t slices = (blocks + P.channels - 1) / P.channels;
+    // as many slices per channel as give every item a resident block of its own (one wave), never more
+    // than tiles; with more channels than blocks, one slice per channel
+    int64_t slices = blocks / P.channels;
     slices = std::max<int64_t>(1, std::min<int64_t>(slices, per_channel));
     G->slices = (int32_t)slices;
     G->tiles_per_plane = (int32_t)per_plane;
@@ -1109,9 +1285,48 @@ static distdl_status_t grad_plan(const distdl_partition *p, int32_t kh, int32_t 
 }
 
 template <int K>
-static distdl_status_t launch_grad(const ConvGradParams &G, int grid, float *dw, float *db, cudaStream_t s) {
-    constexpr int smem = 2 * ConvCfg<K, false>::TILE_FLOATS * 4 + 2 * kTileH * kTileW * 4;
-    conv_grad_kernel<K><<<grid, kConvThreads, smem, s>>>(G);
+static distdl_status_t launch_grad(const distdl_partition *p, const ConvGradParams &G, int grid, float *dw, float *db,
+                                   cudaStream_t s) {
+    const ConvParams &P = G.base;
+    // TMA for the x tiles: few enough workers for the maps to travel as kernel parameters and padded rows
+    // of whole 16-byte units; for the dy tiles as well when the bulk rows are
+    EncodeTiledFn enc = tensor_map_encoder();
+    bool x_tma = p->num_workers <= kConvTmaMaxWorkers && enc != nullptr, dy_tma = true;
+    for (int32_t c = 0; c < P.pw_workers; ++c) {
+        x_tma = x_tma && ((P.bw[c] + 2 * (K / 2)) % 4) == 0;
+        dy_tma = dy_tma && (P.bw[c] % 4) == 0;
+    }
+    if (x_tma) {
+        using C = ConvCfg<K, false>;
+        ConvGradTmaParams Q;
+        memset(&Q, 0, sizeof(Q));
+        Q.g = G;
+        const cuuint64_t planes = (cuuint64_t)(p->global_shape[0] * p->global_shape[1]);
+        const cuuint32_t estr[3] = {1, 1, 1};
+        for (int32_t wk = 0; wk < p->num_workers; ++wk) {
+            const int r = wk / P.pw_workers, c = wk % P.pw_workers;
+            const cuuint64_t pitch = (cuuint64_t)(P.bw[c] + 2 * C::PH), rows = (cuuint64_t)(P.bh[r] + 2 * C::PH);
+            const cuuint64_t dims[3] = {pitch, rows, planes};
+            const cuuint64_t strides[2] = {pitch * 4, pitch * rows * 4};
+            const cuuint32_t box[3] = {(cuuint32_t)C::PITCH, (cuuint32_t)C::ROWS, 1};
+            if (enc(&Q.x_map[wk], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(P.in[wk]), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return fail(DISTDL_ERR_CUDA, "conv_adj_params: tensor map of x shard %d failed", wk);
+            if (!dy_tma) continue;
+            const cuuint64_t ddims[3] = {(cuuint64_t)P.bw[c], (cuuint64_t)P.bh[r], planes};
+            const cuuint64_t dstrides[2] = {(cuuint64_t)P.bw[c] * 4, (cuuint64_t)P.bw[c] * (cuuint64_t)P.bh[r] * 4};
+            const cuuint32_t dbox[3] = {(cuuint32_t)kTileW, (cuuint32_t)kTileH, 1};
+            if (enc(&Q.dy_map[wk], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(G.dy[wk]), ddims, dstrides, dbox, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return fail(DISTDL_ERR_CUDA, "conv_adj_params: tensor map of dy shard %d failed", wk);
+        }
+        if (dy_tma) conv_grad_tma_kernel<K, true><<<grid, kConvThreads, grad_smem_bytes<K>(true), s>>>(Q);
+        else conv_grad_tma_kernel<K, false><<<grid, kConvThreads, grad_smem_bytes<K>(true), s>>>(Q);
+    } else {
+        conv_grad_kernel<K><<<grid, kConvThreads, grad_smem_bytes<K>(false), s>>>(G);
+    }
     DISTDL_CUDA_CHECK(cudaGetLastError());
     conv_grad_finish_kernel<<<G.base.channels, 64, 0, s>>>(G.partial, G.slices, K * K, dw, db);
     DISTDL_CUDA_CHECK(cudaGetLastError());
@@ -1159,9 +1374,9 @@ extern "C" distdl_status_t distdl_conv_adj_params(const distdl_partition_t *p, c
     }
     G.partial = (float *)workspace;
     cudaStream_t s = (cudaStream_t)stream;
-    if (kh == 3) return launch_grad<3>(G, grid, (float *)dw, (float *)db, s);
-    if (kh == 5) return launch_grad<5>(G, grid, (float *)dw, (float *)db, s);
-    return launch_grad<7>(G, grid, (float *)dw, (float *)db, s);
+    if (kh == 3) return launch_grad<3>(p, G, grid, (float *)dw, (float *)db, s);
+    if (kh == 5) return launch_grad<5>(p, G, grid, (float *)dw, (float *)db, s);
+    return launch_grad<7>(p, G, grid, (float *)dw, (float *)db, s);
 }
 
 namespace distdl {

@@ -231,6 +231,10 @@ CONV_CASES = [
     ((1, 2, 300, 520), (1, 1, 2, 2), 5),     # three tile columns per shard, vertical neighbours, TMA path
     ((1, 1, 200, 1032), (1, 1, 3, 2), 7),
     ((1, 1, 100, 780), (1, 1, 2, 3), 3),
+    ((1, 2, 70, 260), (1, 1, 2, 2), 3),      # padded rows of whole 16-byte units, bulk rows not (K = 3)
+    ((1, 1, 70, 260), (1, 1, 2, 2), 7),      # the same for K = 7; the last tile column holds 2 < 3 columns
+    ((1, 2, 66, 264), (1, 1, 2, 2), 5),      # the last tile row holds 1 < 2 rows: the tile above it reaches into the halo
+    ((1, 1, 68, 260), (1, 1, 2, 2), 7),      # 2 < 3 rows and 2 < 3 columns
 ]
 
 
