@@ -155,7 +155,7 @@ class Workload:
         self.c_ws = torch.empty(d.conv_adj_params_workspace(self.cpart, 5, 5), dtype=torch.uint8, device=dev)
         self.a_dw = [torch.empty(blk, blk, device=dev) for _ in range(self.pf * self.pf)]
         self.a_db = [torch.empty(blk, device=dev) for _ in range(self.pf)]
-        side2 = 4096 if small else 8192
+        side2 = 8192
         self.rep = d.Repartition((side2, side2), (8, 1), (1, 8))
         self.t_src = [u(side2 // 8, side2) for _ in range(8)]
         self.t_dst = [torch.empty(side2, side2 // 8, device=dev) for _ in range(8)]

@@ -18,6 +18,7 @@
 // device status word, releases its tensor memory and returns.
 #include <cuda.h>
 
+#include <algorithm>
 #include <cstring>
 
 #include "common.h"
@@ -612,17 +613,17 @@ affine_kernel_quad(const __grid_constant__ AffineParams P) {
 // thread block owns one 128 x 128 tile of one worker's dW block and contracts over the batch.
 // Both operands are MN-major for the tensor cores (dy_i is [nb, out] row-major: the M index is
 // contiguous; x_j is [nb, in]: the N index is contiguous), staged by TMA as 64 x 64 swizzled atoms.
-// The output (fp32, nfo x nfi) dominates the traffic, so up to three blocks share an SM and the
-// epilogue stages the tile in (swizzled) shared memory and hands it to TMA stores: whole 128-byte
-// lines leave the SM while the next block's loads and MMAs run.
+// The output (fp32, nfo x nfi) dominates the traffic: the epilogue stages the tile in (swizzled)
+// shared memory and hands it to TMA stores, so whole 128-byte lines leave the SM while the loads and
+// MMAs of the next tile run.
 // ------------------------------------------------------------------------------------------
 constexpr int kDwThreads = 192;                              // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
-constexpr int kDwStages = 2;
+constexpr int kDwStages = 4;
 constexpr int kDwOperandBytes = 2 * 64 * kBlockK * 2;        // two 64 x 64 bf16 atoms = 16 KB
 constexpr int kDwStageBytes = 2 * kDwOperandBytes;           // A and B
 constexpr int kDwOutBytes = kTileM * kTileN * 4;             // 64 KB: the fp32 tile as four 128 x 32 boxes
-static_assert(kDwStages * kDwStageBytes == kDwOutBytes, "the epilogue reuses the ring");
-constexpr int kDwSmemBytes = kDwOutBytes + 1024 + 128;
+constexpr int kDwSmemBytes = kDwStages * kDwStageBytes + kDwOutBytes + 1024 + 128;
+constexpr int kDwTmemCols = 2 * kTileN;                      // two accumulators
 
 struct AffineDwParams {
     CUtensorMap dy_map[8];                  // dy_i  [nb, bfo] bf16, box {64 out, 64 batch}
@@ -630,35 +631,64 @@ struct AffineDwParams {
     CUtensorMap dw_map[kMaxMaps - 8];       // dW_ij [bfo, bfi] fp32, box {32 in, 128 out}
     int32_t nb, pfi;
     int32_t tiles_m, tiles_n;               // 128 x 128 tiles per worker block
+    int32_t total_tiles;
 };
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int32_t c0, int32_t c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// barrier 1 of the four epilogue warps, combined with an AND over their predicates
+__device__ __forceinline__ bool epilogue_all(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "barrier.cta.red.and.pred p, 1, 128, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(out) : "r"((uint32_t)pred) : "memory");
+    return out != 0;
+}
 
-__global__ void __launch_bounds__(kDwThreads, 3)
+struct DwTile {
+    int wi, wj, m0, n0;
+};
+__device__ __forceinline__ DwTile dw_tile(const AffineDwParams &P, int tile) {
+    // tile id: column tile fastest, then row tile, then worker j, then worker i
+    DwTile t;
+    int rest = tile;
+    t.n0 = (rest % P.tiles_n) * kTileN;
+    rest /= P.tiles_n;
+    t.m0 = (rest % P.tiles_m) * kTileM;
+    rest /= P.tiles_m;
+    t.wj = rest % P.pfi;
+    t.wi = rest / P.pfi;
+    return t;
+}
+
+// Persistent: one block per SM walks over tiles blockIdx.x, + gridDim.x, ...  The producer runs ahead
+// through a four-stage ring (a whole tile at batch 256), the accumulator alternates between two
+// 128-column halves of tensor memory, and the epilogue of tile t (tensor memory -> swizzled shared
+// memory -> TMA stores) runs while the tensor cores work on tile t + 1.
+__global__ void __launch_bounds__(kDwThreads, 1)
 affine_dw_kernel(const __grid_constant__ AffineDwParams P) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *aligned = smem_raw + (base - raw);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kDwOutBytes);
+    const uint32_t out_base = base + kDwStages * kDwStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kDwStages * kDwStageBytes + kDwOutBytes);
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * kDwStages;
-    const uint32_t bar_acc = bar_empty + 8 * kDwStages;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kDwStages + 1);
+    const uint32_t bar_acc_full = bar_empty + 8 * kDwStages;     // two
+    const uint32_t bar_acc_empty = bar_acc_full + 16;            // two
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kDwStages + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // tile id: column tile fastest, then row tile, then worker j, then worker i
-    int rest = blockIdx.x;
-    const int tn = rest % P.tiles_n;
-    rest /= P.tiles_n;
-    const int tm = rest % P.tiles_m;
-    rest /= P.tiles_m;
-    const int wj = rest % P.pfi, wi = rest / P.pfi;
-    const int m0 = tm * kTileM, n0 = tn * kTileN;
     const int num_kblocks = (P.nb + kBlockK - 1) / kBlockK;       // rows past nb are filled with zeros by TMA
 
     if (threadIdx.x == 0) {
@@ -666,36 +696,44 @@ affine_dw_kernel(const __grid_constant__ AffineDwParams P) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        mbar_init(bar_acc, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, 4);                  // one arrival per epilogue warp
+        }
         *abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kDwTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
-    const uint32_t tmem_acc = *tmem_slot;
+    const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
         if (lane == 0) {
-            const CUtensorMap *amap = &P.dy_map[wi], *bmap = &P.x_map[wj];
             uint32_t s = 0, phase = 0;
-            for (int kb = 0; kb < num_kblocks; ++kb) {
-                if (!mbar_wait(bar_empty + 8 * s, phase ^ 1, abort_flag)) break;
-                const uint32_t full = bar_full + 8 * s, sa = base + s * kDwStageBytes;
-                mbar_expect_tx(full, kDwStageBytes);
-                const int k0 = kb * kBlockK;
-                tma_load_2d(sa, amap, m0, k0, full);                                   // atom: out features m0 .. m0 + 63
-                tma_load_2d(sa + kDwOperandBytes / 2, amap, m0 + 64, k0, full);
-                tma_load_2d(sa + kDwOperandBytes, bmap, n0, k0, full);                 // atom: in features n0 .. n0 + 63
-                tma_load_2d(sa + kDwOperandBytes + kDwOperandBytes / 2, bmap, n0 + 64, k0, full);
-                if (++s == kDwStages) {
-                    s = 0;
-                    phase ^= 1;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+                const DwTile t = dw_tile(P, tile);
+                const CUtensorMap *amap = &P.dy_map[t.wi], *bmap = &P.x_map[t.wj];
+                for (int kb = 0; kb < num_kblocks; ++kb) {
+                    ok = mbar_wait(bar_empty + 8 * s, phase ^ 1, abort_flag);
+                    if (!ok) break;
+                    const uint32_t full = bar_full + 8 * s, sa = base + s * kDwStageBytes;
+                    mbar_expect_tx(full, kDwStageBytes);
+                    const int k0 = kb * kBlockK;
+                    tma_load_2d(sa, amap, t.m0, k0, full);                                 // atom: out features m0 .. m0 + 63
+                    tma_load_2d(sa + kDwOperandBytes / 2, amap, t.m0 + 64, k0, full);
+                    tma_load_2d(sa + kDwOperandBytes, bmap, t.n0, k0, full);               // atom: in features n0 .. n0 + 63
+                    tma_load_2d(sa + kDwOperandBytes + kDwOperandBytes / 2, bmap, t.n0 + 64, k0, full);
+                    if (++s == kDwStages) {
+                        s = 0;
+                        phase ^= 1;
+                    }
                 }
             }
             if (*abort_flag) {
@@ -711,64 +749,86 @@ affine_dw_kernel(const __grid_constant__ AffineDwParams P) {
             const uint32_t idesc = instr_desc(kTileM, kTileN, 1) | (1u << 15);
             uint32_t s = 0, phase = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kblocks; ++kb) {
-                ok = mbar_wait(bar_full + 8 * s, phase, abort_flag);
+            int it = 0;
+            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++it) {
+                const uint32_t buf = (uint32_t)it & 1u;
+                // the epilogue has read this half's previous tile (passes at once the first two times)
+                ok = mbar_wait(bar_acc_empty + 8 * buf, (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag);
                 if (!ok) break;
                 tcgen05_fence_after();
-                const uint32_t sa = base + s * kDwStageBytes;
-                const uint64_t a = smem_desc(sa, kDwOperandBytes / 2, 1024);
-                const uint64_t b = smem_desc(sa + kDwOperandBytes, kDwOperandBytes / 2, 1024);
-                constexpr uint64_t kstep = 2048 >> 4;
-                umma_bf16(tmem_acc, a, b, idesc, kb ? 1u : 0u);
-                umma_bf16(tmem_acc, a + kstep, b + kstep, idesc, 1u);
-                umma_bf16(tmem_acc, a + 2 * kstep, b + 2 * kstep, idesc, 1u);
-                umma_bf16(tmem_acc, a + 3 * kstep, b + 3 * kstep, idesc, 1u);
-                tcgen05_commit(bar_empty + 8 * s);
-                if (++s == kDwStages) {
-                    s = 0;
-                    phase ^= 1;
+                const uint32_t tmem_acc = tmem_base + buf * (uint32_t)kTileN;
+                for (int kb = 0; kb < num_kblocks; ++kb) {
+                    ok = mbar_wait(bar_full + 8 * s, phase, abort_flag);
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint32_t sa = base + s * kDwStageBytes;
+                    const uint64_t a = smem_desc(sa, kDwOperandBytes / 2, 1024);
+                    const uint64_t b = smem_desc(sa + kDwOperandBytes, kDwOperandBytes / 2, 1024);
+                    constexpr uint64_t kstep = 2048 >> 4;
+                    umma_bf16(tmem_acc, a, b, idesc, kb ? 1u : 0u);
+                    umma_bf16(tmem_acc, a + kstep, b + kstep, idesc, 1u);
+                    umma_bf16(tmem_acc, a + 2 * kstep, b + 2 * kstep, idesc, 1u);
+                    umma_bf16(tmem_acc, a + 3 * kstep, b + 3 * kstep, idesc, 1u);
+                    tcgen05_commit(bar_empty + 8 * s);
+                    if (++s == kDwStages) {
+                        s = 0;
+                        phase ^= 1;
+                    }
                 }
+                if (ok) tcgen05_commit(bar_acc_full + 8 * buf);
             }
-            if (ok) tcgen05_commit(bar_acc);
         }
         __syncwarp();
     } else {
-        // epilogue: the accumulator is complete, so every MMA has retired and the ring is free.
-        // Box q (columns 32 q .. 32 q + 31) is a 128 x 32 fp32 array of 128-byte rows with the 16-byte
-        // chunks of row r stored at chunk ^ (r & 7): the layout of a 128-byte-swizzled tensor map.
+        // epilogue.  Box q of the staging buffer (columns 32 q .. 32 q + 31) is a 128 x 32 fp32 array of
+        // 128-byte rows with the 16-byte chunks of row r stored at chunk ^ (r & 7): the layout of a
+        // 128-byte-swizzled tensor map.  Every decision to go on or to give up is taken by the four warps
+        // together, so they always meet at the same barriers.
         const int quarter = warp & 3;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, abort_flag));
-        tcgen05_fence_after();
-        if (ok) {
-            const int row = quarter * 32 + lane;
+        const int row = quarter * 32 + lane;
+        const bool issuer = warp == 2 && lane == 0;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++it) {
+            const uint32_t buf = (uint32_t)it & 1u;
+            // the stores of the previous tile have read the staging buffer
+            if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            const bool mine = mbar_wait(bar_acc_full + 8 * buf, ((uint32_t)it >> 1) & 1u, abort_flag);
+            if (!epilogue_all(mine)) break;
+            tcgen05_fence_after();
+            const uint32_t tmem_acc = tmem_base + buf * (uint32_t)kTileN;
 #pragma unroll 1
             for (int q = 0; q < kTileN / 32; ++q) {
                 uint32_t v[32];
                 tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(32 * q), v);
-                const uint32_t rowaddr = base + (uint32_t)q * (kTileM * 128) + (uint32_t)row * 128;
+                const uint32_t rowaddr = out_base + (uint32_t)q * (kTileM * 128) + (uint32_t)row * 128;
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
                                  ::"r"(rowaddr + (uint32_t)((c ^ (row & 7)) << 4)), "r"(v[4 * c]), "r"(v[4 * c + 1]),
                                    "r"(v[4 * c + 2]), "r"(v[4 * c + 3]) : "memory");
             }
+            // this half of tensor memory may be overwritten by the tile after the next
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
             fence_proxy_async();
-        }
-        // the four epilogue warps meet, then one thread hands the tile to TMA
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ok && warp == 2 && lane == 0) {
-            const CUtensorMap *omap = &P.dw_map[wi * P.pfi + wj];
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (issuer) {
+                const DwTile t = dw_tile(P, tile);
+                const CUtensorMap *omap = &P.dw_map[t.wi * P.pfi + t.wj];
 #pragma unroll
-            for (int q = 0; q < kTileN / 32; ++q) tma_store_2d(omap, base + (uint32_t)q * (kTileM * 128), n0 + 32 * q, m0);
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory read out before the block retires
+                for (int q = 0; q < kTileN / 32; ++q)
+                    tma_store_2d(omap, out_base + (uint32_t)q * (kTileM * 128), t.n0 + 32 * q, t.m0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
         }
+        if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores done before the block retires
     }
     tcgen05_fence_before();
     __syncthreads();
     if (warp == 1) {
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)kTileN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kDwTmemCols) : "memory");
     }
 }
 
@@ -991,12 +1051,18 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
     P.pfi = pfi;
     P.tiles_m = (int32_t)(bfo / kTileM);
     P.tiles_n = (int32_t)(bfi / kTileN);
+    P.total_tiles = (int32_t)tiles;
     static bool configured = false;
+    static int sms = 0;
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemBytes));
+        int dev = 0;
+        DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
+        DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         configured = true;
     }
-    affine_dw_kernel<<<(unsigned)tiles, kDwThreads, kDwSmemBytes, (cudaStream_t)stream>>>(P);
+    const unsigned grid = (unsigned)std::min<int64_t>(tiles, sms > 0 ? sms : 1);
+    affine_dw_kernel<<<grid, kDwThreads, kDwSmemBytes, (cudaStream_t)stream>>>(P);
     DISTDL_CUDA_CHECK(cudaGetLastError());
     if (db) {
         AffineDbParams B;
