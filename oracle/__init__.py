@@ -3,7 +3,7 @@
 TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, deliberately naive
 numpy restatement of what the operators compute (broadcast B, sum-reduce R = B*,
 halo exchange H, adjoint halo exchange H*, the generalized all-to-all with scatter and
-gather as special cases, all-reduce, the distributed depthwise convolution,
+gather as special cases, all-reduce, the distributed depthwise convolution, the 3-D star-stencil layer,
 the distributed pooling layer and the distributed affine layer, each with its adjoint).  Nothing in the product
 package imports it; only the test-suite, the smoke check and the CPU-baseline leg
 of the benchmark may call it.  It shares no code, table or helper with the CUDA
@@ -39,6 +39,9 @@ from .layers import (  # noqa: F401
     conv_adj,
     conv_adj_scatter_then_halo,
     conv_adj_params,
+    stencil3d_fwd,
+    stencil3d_adj,
+    stencil3d_fwd_exchange_then_local,
     affine_fwd,
     affine_adj,
     affine_adj_params,

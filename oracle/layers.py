@@ -148,6 +148,79 @@ def conv_adj_params(part: Partition, x_shards, dy_shards, kh, kw):
 
 
 # --------------------------------------------------------------------------
+# Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers":
+# a sliding-kernel layer on a feature-space partition = halo exchange, then the
+# local kernel; Section 6 names large volumetric data as the target)
+# --------------------------------------------------------------------------
+
+def _star_apply(g, w, flip):
+    """sum over axes d and offsets k = -R..R of w[d][k + R] * g shifted by k along d (zeros outside).
+
+    flip = False: out[i] = sum w[d][k + R] * g[i + k e_d]   (cross-correlation, as for Conv)
+    flip = True:  out[i] = sum w[d][k + R] * g[i - k e_d]   (its transpose)
+    fp64 throughout.
+    """
+    w = np.asarray(w, dtype=np.float64)
+    assert w.ndim == 2 and w.shape[0] == 3 and w.shape[1] % 2 == 1
+    R = w.shape[1] // 2
+    g = np.asarray(g, dtype=np.float64)
+    gp = np.zeros(tuple(n + 2 * R for n in g.shape), dtype=np.float64)
+    gp[R:R + g.shape[0], R:R + g.shape[1], R:R + g.shape[2]] = g
+    out = np.zeros(g.shape, dtype=np.float64)
+    for d in range(3):
+        for k in range(-R, R + 1):
+            off = [R, R, R]
+            off[d] += -k if flip else k
+            out += w[d][k + R] * gp[off[0]:off[0] + g.shape[0], off[1]:off[1] + g.shape[1], off[2]:off[2] + g.shape[2]]
+    return out
+
+
+def stencil3d_fwd(part: Partition, x_shards, w):
+    """y = Stencil(w; H x): the sequential layer written out on the global tensor.
+
+    w[d][k + R], d = 0..2, k = -R..R: one 1-D kernel per dimension (a star);
+    y[i] = sum_d sum_k w[d][k + R] * x[i + k e_d], x = 0 outside the tensor.
+    fp64 accumulation, rounded once to fp32.  Returns bulk-shaped shards.
+    """
+    assert part.rank == 3
+    yg = _star_apply(assemble_global(part, x_shards), w, flip=False).astype(np.float32)
+    return scatter_global(Partition(part.global_shape, part.pshape, 0, 0), yg)
+
+
+def stencil3d_adj(part: Partition, dy_shards, w):
+    """dx = H* [dStencil]* dy as the transpose of stencil3d_fwd on the global tensor.
+
+    dx[i] = sum_d sum_k w[d][k + R] * dy[i - k e_d], dy = 0 outside.  Returned as
+    padded shards of `part` whose ghosts are zero (what H* leaves behind).
+    """
+    assert part.rank == 3
+    ypart = Partition(part.global_shape, part.pshape, 0, 0)
+    dxg = _star_apply(assemble_global(ypart, dy_shards), w, flip=True).astype(np.float32)
+    return scatter_global(part, dxg)
+
+
+def stencil3d_fwd_exchange_then_local(part: Partition, x_shards, w):
+    """The layer taken step by step (cross-check form): x <- H x, then every worker
+    applies the kernel to its own padded shard, producing its bulk-shaped block."""
+    w = np.asarray(w, dtype=np.float64)
+    R = w.shape[1] // 2
+    from .primitives import halo_fwd_sequence
+    out = []
+    for wk, xh in enumerate(halo_fwd_sequence(part, x_shards)):
+        xh = np.asarray(xh, dtype=np.float64)
+        assert all(part.hlo[d][c] == R and part.hhi[d][c] == R for d in range(3) for c in range(part.pshape[d]))
+        b = tuple(n - 2 * R for n in xh.shape)
+        acc = np.zeros(b, dtype=np.float64)
+        for d in range(3):
+            for k in range(-R, R + 1):
+                off = [R, R, R]
+                off[d] += k
+                acc += w[d][k + R] * xh[off[0]:off[0] + b[0], off[1]:off[1] + b[1], off[2]:off[2] + b[2]]
+        out.append(acc.astype(np.float32))
+    return out
+
+
+# --------------------------------------------------------------------------
 # Distributed affine layer (Section 4, "Dense layers")
 # --------------------------------------------------------------------------
 

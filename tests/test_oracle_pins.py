@@ -737,3 +737,79 @@ def test_conv_param_gradients_brute_force_taps_and_dot_test():
     bias = inputs.normal((2,), 78)
     y = oracle.conv_fwd(part, x, w, bias)
     assert oracle.adjoint_test_ratio(y, dy, [w, bias], [dw, db]) < 1e-6
+
+
+# --------------------------------------------------------------------------
+# 3-D star-stencil layer (halo exchange + local sliding kernel on a rank-3 tensor)
+# --------------------------------------------------------------------------
+
+STENCIL_CASES = [
+    # global shape, partition, radius
+    ((6, 7, 8), (1, 1, 1), 2),
+    ((9, 8, 10), (2, 2, 2), 2),
+    ((12, 9, 13), (3, 1, 2), 4),
+    ((5, 6, 7), (1, 2, 3), 1),
+]
+
+
+def _stencil_problem(case, seed):
+    gs, ps, R = case
+    part = Partition(gs, ps, R, R)
+    xg = inputs.normal(gs, seed)
+    w = inputs.normal((3, 2 * R + 1), seed + 1, 0.5)
+    return part, xg, w
+
+
+@pytest.mark.parametrize("case", STENCIL_CASES, ids=[str(c) for c in STENCIL_CASES])
+def test_stencil3d_matches_library_correlation_and_stepwise_form(case):
+    from scipy.ndimage import correlate1d
+    part, xg, w = _stencil_problem(case, 81)
+    x = oracle.scatter_global(part, xg, fill=lambda wk: np.full(part.padded_shape(wk), 5.0))    # garbage ghosts
+    y = oracle.assemble_global(Partition(xg.shape, part.pshape), oracle.stencil3d_fwd(part, x, w))
+    ref = sum(correlate1d(xg.astype(np.float64), w[d].astype(np.float64), axis=d, mode="constant", cval=0.0)
+              for d in range(3))
+    assert np.allclose(y, ref, rtol=0, atol=5e-6)
+    # the distributed algorithm itself: exchange, then the local kernel on every padded shard
+    for a, b in zip(oracle.stencil3d_fwd(part, x, w), oracle.stencil3d_fwd_exchange_then_local(part, x, w)):
+        assert np.allclose(a, b, rtol=0, atol=5e-6)
+
+
+def test_stencil3d_adjoint_is_the_transpose_matrix():
+    gs, ps, R = (3, 4, 5), (1, 2, 2), 1
+    part, ypart = Partition(gs, ps, R, R), Partition(gs, ps)
+    w = inputs.normal((3, 3), 83, 0.5)
+    n = int(np.prod(gs))
+    F = np.zeros((n, n))
+    A = np.zeros((n, n))
+    for e in range(n):
+        u = np.zeros(n, np.float32)
+        u[e] = 1.0
+        ug = u.reshape(gs)
+        F[:, e] = oracle.assemble_global(ypart, oracle.stencil3d_fwd(part, oracle.scatter_global(part, ug), w)).reshape(-1)
+        A[:, e] = oracle.assemble_global(part, oracle.stencil3d_adj(part, oracle.scatter_global(ypart, ug), w)).reshape(-1)
+    assert np.array_equal(A, F.T)
+    # the matrix itself, entry by entry: F[i, j] = sum of w[d][k + R] over (d, k) with j = i + k e_d
+    idx = np.arange(n).reshape(gs)
+    G = np.zeros((n, n))
+    for i in itertools.product(*[range(v) for v in gs]):
+        for d in range(3):
+            for k in (-1, 0, 1):
+                j = list(i)
+                j[d] += k
+                if 0 <= j[d] < gs[d]:
+                    G[idx[i], idx[tuple(j)]] += float(np.float64(w[d][k + 1]))
+    assert np.allclose(F, G.astype(np.float32), rtol=0, atol=1e-7)
+
+
+@pytest.mark.parametrize("case", STENCIL_CASES[1:], ids=[str(c) for c in STENCIL_CASES[1:]])
+def test_stencil3d_dot_test_and_zero_ghosts(case):
+    part, xg, w = _stencil_problem(case, 85)
+    ypart = Partition(xg.shape, part.pshape)
+    x = oracle.scatter_global(part, xg)
+    dy = oracle.scatter_global(ypart, inputs.normal(xg.shape, 87))
+    y, dx = oracle.stencil3d_fwd(part, x, w), oracle.stencil3d_adj(part, dy, w)
+    assert oracle.adjoint_test_ratio(y, dy, x, dx) < 1e-6
+    for wk in range(part.num_workers):
+        mask = np.ones(part.padded_shape(wk), dtype=bool)
+        mask[part.bulk_slices(wk)] = False
+        assert not dx[wk][mask].any()
