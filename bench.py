@@ -159,6 +159,29 @@ class Workload:
         self.rep = d.Repartition((side2, side2), (8, 1), (1, 8))
         self.t_src = [u(side2 // 8, side2) for _ in range(8)]
         self.t_dst = [torch.empty(side2, side2 // 8, device=dev) for _ in range(8)]
+        # fused halo exchange + 25-point star (radius 4) on the step's 512^3 volume (4 x 4 x 4 workers)
+        self.s_w = [[0.05 * (1 + abs(k - 4)) * (-1) ** k for k in range(9)] for _ in range(3)]
+        nw = self.hpart.num_workers
+        if small:
+            self.spart = d.Partition((256, 512, 512), (2, 4, 4), (4,) * 3, (4,) * 3)
+            nw = self.spart.num_workers
+            self.s_x = self.h_x[:nw]
+        else:
+            self.spart, self.s_x = self.hpart, self.h_x
+        self.s_y = [torch.empty(*self.spart.bulk_shape(w), device=dev) for w in range(nw)]
+        self.s_dx = [torch.empty(*self.spart.padded_shape(w), device=dev) for w in range(nw)]
+        cells = 1
+        for v in self.spart.global_shape:
+            cells *= v
+        halo_read = (self.spart.halo_stats(False)[2] - sum(t.numel() - y.numel() for t, y in zip(self.s_dx, self.s_y)) * 4)
+        st_bytes = 8 * cells + halo_read
+        ghost_b = sum(t.numel() - y.numel() for t, y in zip(self.s_dx, self.s_y)) * 4
+        self.extra_ops += [
+            ("stencil3d_fwd", lambda: d.stencil3d_fwd(self.spart, self.s_x, self.s_w, self.s_y), st_bytes, 2 * 27 * cells, 1,
+             "hbm"),
+            ("stencil3d_adj", lambda: d.stencil3d_adj(self.spart, self.s_y, self.s_w, self.s_dx), st_bytes + ghost_b,
+             2 * 27 * cells, 1, "hbm"),
+        ]
         self.extra_ops += [
             ("conv_adj_params", lambda: d.conv_adj_params(self.cpart, self.c_x, self.c_dy, (5, 5), self.c_dw, self.c_db,
                                                           self.c_ws), conv_bytes, 2 * 25 * self._conv_outputs(), 2, "hbm"),
@@ -514,7 +537,8 @@ def main():
             "ops": ops,
             "extra_ops": {"note": "timed separately, not part of value: 3x3 max pooling, stride 2, padding 1 on fp32 "
                                   "16x16x1024x1024 over 4x4 workers (H + local kernel, local adjoint + H*); parameter "
-                                  "gradients of the step's convolution (dw, db) and affine layer (dW, db); generalized "
+                                  "gradients of the step's convolution (dw, db) and affine layer (dW, db); fused halo + radius-4 star stencil "
+                                  "on the step's 512^3 volume (4x4x4 workers); generalized "
                                   "all-to-all of fp32 8192x8192 between 8 row blocks and 8 column blocks",
                           **extra},
             "roofline": roofline,

@@ -260,6 +260,27 @@ distdl_status_t distdl_conv_adj_params(const distdl_partition_t *p, const void *
                                        void *stream);
 
 /* ------------------------------------------------------------------------
+ * Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers": on a feature-space
+ * partition a sliding-kernel layer is the halo exchange followed by the local kernel, its adjoint the
+ * local adjoint followed by H*; Section 6 names large volumetric data as the target).
+ *
+ * p: rank-3 F32 partition, at most 8 workers along a dimension and 64 in all, whose halo widths equal
+ *    `radius` (1..4) on every side of every dimension (else DISTDL_ERR_SHAPE).
+ * w: HOST array [3][2*radius+1]: w[d][k+radius] is the tap at offset k along dimension d.
+ * stencil3d_fwd = H then the local kernel, fused:
+ *    y[i] = sum_d sum_{k=-radius..radius} w[d][k+radius] * x[i + k e_d] over the GLOBAL tensor, zeros outside.
+ *    x[w]: padded shards (only their bulk is read; ghost storage is neither read nor written);
+ *    y[w]: bulk-shaped shards.  6*radius+3 fp32 FMAs per output, z taps first, then y, then x.
+ * stencil3d_adj = local adjoint then H*, fused (gather form):
+ *    dx[i] = sum_d sum_k w[d][k+radius] * dy[i - k e_d] (zeros outside), written to the bulk of the
+ *    padded shards dx[w], whose ghosts are set to zero.  dy[w]: bulk-shaped shards.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_stencil3d_fwd(const distdl_partition_t *p, const void *const *x, const float *w,
+                                     int32_t radius, void *const *y, void *stream);
+distdl_status_t distdl_stencil3d_adj(const distdl_partition_t *p, const void *const *dy, const float *w,
+                                     int32_t radius, void *const *dx, void *stream);
+
+/* ------------------------------------------------------------------------
  * Distributed pooling layer, feature-space partition only (Section 4, "Sparse layers": pooling
  * layers follow the convolution algorithms; Section 3 / Appendix B: for a strided kernel the halo
  * widths differ from worker to worker and owned inputs may go unused, Figs. B2-B4).

@@ -79,6 +79,8 @@ def lib():
     L.distdl_affine_adj_params.argtypes = [c_i64, c_i64, c_i64, c_i32, c_i32, pvp, pvp, pvp, pvp, vp]
     L.distdl_conv_adj_params_workspace.argtypes = [vp, c_i32, c_i32, pi64]
     L.distdl_conv_adj_params.argtypes = [vp, pvp, pvp, c_i32, c_i32, vp, vp, vp, c_i64, vp]
+    L.distdl_stencil3d_fwd.argtypes = [vp, pvp, ctypes.POINTER(ctypes.c_float), c_i32, pvp, vp]
+    L.distdl_stencil3d_adj.argtypes = [vp, pvp, ctypes.POINTER(ctypes.c_float), c_i32, pvp, vp]
     L.distdl_device_status.argtypes = [vp]
     _lib = L
     return L
@@ -262,6 +264,25 @@ def conv_fwd(part, x, w, bias, y, stream=None):
 def conv_adj(part, dy, w, dx, stream=None):
     kh, kw = int(w.shape[-2]), int(w.shape[-1])
     _check(lib().distdl_conv_adj(part.handle, _ptr_array(dy), _ptr(w), kh, kw, _ptr_array(dx), _stream(stream)))
+
+
+def _taps(w):
+    """Host array of the 3 x (2R+1) taps (any nested sequence or numpy array) and the radius."""
+    rows = [[float(v) for v in row] for row in w]
+    if len(rows) != 3 or len(set(len(r) for r in rows)) != 1 or len(rows[0]) % 2 != 1:
+        raise ValueError("taps must have shape [3][2R+1]")
+    n = len(rows[0])
+    return (ctypes.c_float * (3 * n))(*[v for row in rows for v in row]), n // 2
+
+
+def stencil3d_fwd(part, x, w, y, stream=None):
+    arr, radius = _taps(w)
+    _check(lib().distdl_stencil3d_fwd(part.handle, _ptr_array(x), arr, radius, _ptr_array(y), _stream(stream)))
+
+
+def stencil3d_adj(part, dy, w, dx, stream=None):
+    arr, radius = _taps(w)
+    _check(lib().distdl_stencil3d_adj(part.handle, _ptr_array(dy), arr, radius, _ptr_array(dx), _stream(stream)))
 
 
 class Repartition:

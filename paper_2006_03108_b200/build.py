@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdistdl.so")
 
-SOURCES = ["planner.cpp", "partition.cu", "bcast_reduce.cu", "halo.cu", "conv.cu", "pool.cu", "affine.cu"]
+SOURCES = ["planner.cpp", "partition.cu", "bcast_reduce.cu", "halo.cu", "conv.cu", "pool.cu", "stencil3d.cu", "affine.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -790,36 +790,40 @@ affine_dw_kernel(const __grid_constant__ AffineDwParams P) {
         int it = 0;
         for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++it) {
             const uint32_t buf = (uint32_t)it & 1u;
-            // the stores of the previous tile have read the staging buffer
-            if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             const bool mine = mbar_wait(bar_acc_full + 8 * buf, ((uint32_t)it >> 1) & 1u, abort_flag);
             if (!epilogue_all(mine)) break;
             tcgen05_fence_after();
             const uint32_t tmem_acc = tmem_base + buf * (uint32_t)kTileN;
+            const DwTile t = dw_tile(P, tile);
+            const CUtensorMap *omap = &P.dw_map[t.wi * P.pfi + t.wj];
+            // box by box, so that the read-out of one box by its store (which runs at the rate of the SM's
+            // port into the memory system) overlaps the copy of the next box out of tensor memory
 #pragma unroll 1
             for (int q = 0; q < kTileN / 32; ++q) {
+                // at most three stores in flight: the one that read this box for the previous tile is done
+                if (issuer) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                asm volatile("bar.sync 1, 128;" ::: "memory");
                 uint32_t v[32];
                 tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(32 * q), v);
-                const uint32_t rowaddr = out_base + (uint32_t)q * (kTileM * 128) + (uint32_t)row * 128;
+                const uint32_t boxaddr = out_base + (uint32_t)q * (kTileM * 128);
+                const uint32_t rowaddr = boxaddr + (uint32_t)row * 128;
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
                                  ::"r"(rowaddr + (uint32_t)((c ^ (row & 7)) << 4)), "r"(v[4 * c]), "r"(v[4 * c + 1]),
                                    "r"(v[4 * c + 2]), "r"(v[4 * c + 3]) : "memory");
-            }
-            // this half of tensor memory may be overwritten by the tile after the next
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
-            fence_proxy_async();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (issuer) {
-                const DwTile t = dw_tile(P, tile);
-                const CUtensorMap *omap = &P.dw_map[t.wi * P.pfi + t.wj];
-#pragma unroll
-                for (int q = 0; q < kTileN / 32; ++q)
-                    tma_store_2d(omap, out_base + (uint32_t)q * (kTileM * 128), t.n0 + 32 * q, t.m0);
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                if (q == kTileN / 32 - 1) {
+                    // this half of tensor memory may be overwritten by the tile after the next
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                }
+                fence_proxy_async();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (issuer) {
+                    tma_store_2d(omap, boxaddr, t.n0 + 32 * q, t.m0);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
             }
         }
         if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores done before the block retires

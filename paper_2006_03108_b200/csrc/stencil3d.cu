@@ -1,0 +1,337 @@
+// Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers": a sliding-kernel
+// layer on a feature-space partition is the halo exchange H followed by the local kernel; its
+// adjoint is the local adjoint followed by H*).  The kernel is a star: one 1-D kernel of radius R
+// per dimension,
+//   y[i] = sum_d sum_{k=-R..R} w[d][k+R] * x[i + k e_d],     x = 0 outside the tensor,
+// which is the shape of the finite-difference operators of the volumetric problems the paper
+// names as its target.  Both directions are fused with their exchange: a thread block reads the
+// planes, rows and columns it needs straight from the bulk of whichever shard owns them, so no
+// ghost cell is ever written to or read from device memory by the forward pass.  The adjoint is
+// the same star with every 1-D kernel reversed, evaluated in gather form on the bulk-shaped dy,
+// written into the bulk of the padded dx shards whose ghosts are cleared as H* leaves them.
+//
+// Blocking: a block owns 8 rows x 128 columns of one shard and marches through a chunk of planes.
+// A thread owns 4 consecutive columns of one row; the 2R+1 planes around the current one live in
+// its registers (z neighbours), the current plane with R extra rows above / below and R extra
+// columns left / right lives in shared memory (y and x neighbours; a star needs no corners).
+// The values of the next plane -- the thread's own cells R planes ahead, one vector of an extra
+// row, one cell of an extra column -- are fetched one step early, so their latency is covered by
+// the arithmetic of the current plane.  Two plane buffers, one barrier per plane.
+#include <algorithm>
+#include <cstring>
+
+#include "common.h"
+
+namespace distdl {
+
+constexpr int kStMaxWorkers = 64;
+constexpr int kStMaxPerDim = 8;
+constexpr int kStMaxR = 4;
+constexpr int kStRows = 8;            // rows of a tile = warps of a block
+constexpr int kStCols = 128;          // columns of a tile = 32 lanes x 4
+constexpr int kStThreads = 256;
+constexpr int kStChunk = 64;          // planes a block marches through
+constexpr int kStLead = 4;            // shared-memory column of the tile's first column (keeps rows 16-byte aligned)
+constexpr int kStPitch = kStLead + kStCols + 4;   // 136 floats
+
+struct StencilParams {
+    const float *in[kStMaxWorkers];
+    float *out[kStMaxWorkers];
+    int32_t bz[kStMaxPerDim], by[kStMaxPerDim], bx[kStMaxPerDim];   // bulk extents per worker coordinate
+    int32_t pz, py, px;
+    int32_t in_off, out_off;          // ghost width of the input / output layout (R or 0)
+    int32_t tiles_y, tiles_x, chunks_z;
+    int32_t clear_ghosts;             // adjoint: the ghosts of the output shards are set to zero
+    float w[3][2 * kStMaxR + 1];      // taps; [d][k + R], already reversed for the adjoint
+};
+
+// Owner of coordinate c along one dimension, seen from worker coordinate s: the worker itself, or the
+// one below / above (a ghost is never wider than the neighbour's bulk).  Returns false outside the tensor.
+__device__ __forceinline__ bool st_owner(const int32_t *b, int p, int s, int c, int &so, int &co) {
+    so = s;
+    co = c;
+    if (c < 0) {
+        so = s - 1;
+        if (so < 0) return false;
+        co = c + b[so];
+        return co >= 0;
+    }
+    if (c >= b[s]) {
+        so = s + 1;
+        if (so >= p) return false;
+        co = c - b[s];
+        return co < b[so];
+    }
+    return true;
+}
+
+template <int R, bool VEC>
+__global__ void __launch_bounds__(kStThreads, 2)
+stencil3d_kernel(const __grid_constant__ StencilParams P) {
+    __shared__ __align__(16) float plane[2][kStRows + 2 * R][kStPitch];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // block -> (shard, plane chunk, row tile, column tile), column tile fastest
+    int rest = blockIdx.x;
+    const int tx = rest % P.tiles_x;
+    rest /= P.tiles_x;
+    const int ty = rest % P.tiles_y;
+    rest /= P.tiles_y;
+    const int cz = rest % P.chunks_z;
+    const int shard = rest / P.chunks_z;
+    const int sx = shard % P.px, sy = (shard / P.px) % P.py, sz = shard / (P.px * P.py);
+    const int bz = P.bz[sz], by = P.by[sy], bx = P.bx[sx];
+    const int x0 = tx * kStCols, y0 = ty * kStRows, z0 = cz * kStChunk;
+    if (x0 >= bx || y0 >= by || z0 >= bz) return;
+    const int z1 = min(z0 + kStChunk, bz);
+    const int th = min(kStRows, by - y0), tw = min(kStCols, bx - x0);
+    const int io = P.in_off;
+    const int ipx = bx + 2 * io;                       // input row pitch of every shard in this worker column
+
+    const int y = y0 + warp, x = x0 + 4 * lane;
+    const bool row_ok = y < by;
+
+    // this thread's four cells of plane zp (any plane within R of the chunk), zeros outside the tensor
+    auto load_own = [&](int zp) -> float4 {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        int so, zo;
+        if (!row_ok || x >= bx || !st_owner(P.bz, P.pz, sz, zp, so, zo)) return v;
+        const float *src = P.in[(so * P.py + sy) * P.px + sx] +
+                           ((size_t)(zo + io) * (by + 2 * io) + (size_t)(y + io)) * ipx + (x + io);
+        if (VEC) return __ldg(reinterpret_cast<const float4 *>(src));
+        v.x = __ldg(src);
+        if (x + 1 < bx) v.y = __ldg(src + 1);
+        if (x + 2 < bx) v.z = __ldg(src + 2);
+        if (x + 3 < bx) v.w = __ldg(src + 3);
+        return v;
+    };
+    // warps 0 .. 2R-1: this thread's four cells of one extra row of plane zp (a plane of the chunk itself)
+    const int hrow_y = warp < R ? y0 - R + warp : y0 + th + (warp - R);
+    const int hrow_s = warp < R ? warp : R + th + (warp - R);           // its row in the shared-memory plane
+    auto load_hrow = [&](int zp) -> float4 {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        int so, yo;
+        if (warp >= 2 * R || x >= bx || !st_owner(P.by, P.py, sy, hrow_y, so, yo)) return v;
+        const float *src = P.in[(sz * P.py + so) * P.px + sx] +
+                           ((size_t)(zp + io) * (P.by[so] + 2 * io) + (size_t)(yo + io)) * ipx + (x + io);
+        if (VEC) return __ldg(reinterpret_cast<const float4 *>(src));
+        v.x = __ldg(src);
+        if (x + 1 < bx) v.y = __ldg(src + 1);
+        if (x + 2 < bx) v.z = __ldg(src + 2);
+        if (x + 3 < bx) v.w = __ldg(src + 3);
+        return v;
+    };
+    // threads 0 .. 8 * 2R - 1: one cell of an extra column of plane zp
+    const int hc_row = threadIdx.x / (2 * R), hc_c = threadIdx.x % (2 * R);
+    const bool hc_active = (int)threadIdx.x < kStRows * 2 * R && y0 + hc_row < by;
+    const int hc_x = hc_c < R ? x0 - R + hc_c : x0 + tw + (hc_c - R);
+    const int hc_s = kStLead + (hc_x - x0);                               // its column in the shared-memory plane
+    auto load_hcol = [&](int zp) -> float {
+        int so, xo;
+        if (!hc_active || !st_owner(P.bx, P.px, sx, hc_x, so, xo)) return 0.f;
+        const int pitch = P.bx[so] + 2 * io;
+        return __ldg(P.in[(sz * P.py + sy) * P.px + so] +
+                     ((size_t)(zp + io) * (by + 2 * io) + (size_t)(y0 + hc_row + io)) * pitch + (xo + io));
+    };
+
+    // prime: planes z0 - R .. z0 + R, extra row / column of plane z0
+    float4 q[2 * R + 1];
+#pragma unroll
+    for (int i = 0; i <= 2 * R; ++i) q[i] = load_own(z0 - R + i);
+    float4 hrow = load_hrow(z0);
+    float hcol = load_hcol(z0);
+
+    const int oo = P.out_off;
+    const int opy = by + 2 * oo, opx = bx + 2 * oo;
+    float *optr = P.out[shard] + ((size_t)(z0 + oo) * opy + (size_t)(y + oo)) * opx + (x + oo);
+    const size_t oplane = (size_t)opy * opx;
+
+    for (int z = z0; z < z1; ++z) {
+        float(*pl)[kStPitch] = plane[(z - z0) & 1];
+        // current plane into shared memory: own cells, one extra-row vector, one extra-column cell.
+        // Cells beyond the bulk are written by the extra-row / extra-column threads only.
+        if (row_ok) {
+            if (VEC) {
+                if (x < bx) *reinterpret_cast<float4 *>(&pl[R + warp][kStLead + 4 * lane]) = q[R];
+            } else {
+                float *d = &pl[R + warp][kStLead + 4 * lane];
+                if (x < bx) d[0] = q[R].x;
+                if (x + 1 < bx) d[1] = q[R].y;
+                if (x + 2 < bx) d[2] = q[R].z;
+                if (x + 3 < bx) d[3] = q[R].w;
+            }
+        }
+        if (warp < 2 * R) {
+            if (VEC) {
+                if (x < bx) *reinterpret_cast<float4 *>(&pl[hrow_s][kStLead + 4 * lane]) = hrow;
+            } else {
+                float *d = &pl[hrow_s][kStLead + 4 * lane];
+                if (x < bx) d[0] = hrow.x;
+                if (x + 1 < bx) d[1] = hrow.y;
+                if (x + 2 < bx) d[2] = hrow.z;
+                if (x + 3 < bx) d[3] = hrow.w;
+            }
+        }
+        if (hc_active) pl[R + hc_row][hc_s] = hcol;
+        // next plane's values, one step early
+        float4 lead = make_float4(0.f, 0.f, 0.f, 0.f), hrow_n = lead;
+        float hcol_n = 0.f;
+        if (z + 1 < z1) {
+            lead = load_own(z + 1 + R);
+            hrow_n = load_hrow(z + 1);
+            hcol_n = load_hcol(z + 1);
+        }
+        __syncthreads();
+
+        if (row_ok && x < bx) {
+            float o[4] = {0.f, 0.f, 0.f, 0.f};
+            // z neighbours: registers
+#pragma unroll
+            for (int k = 0; k <= 2 * R; ++k) {
+                const float wz = P.w[0][k];
+                o[0] = fmaf(wz, q[k].x, o[0]);
+                o[1] = fmaf(wz, q[k].y, o[1]);
+                o[2] = fmaf(wz, q[k].z, o[2]);
+                o[3] = fmaf(wz, q[k].w, o[3]);
+            }
+            // y neighbours: the rows above and below in shared memory
+#pragma unroll
+            for (int k = 0; k <= 2 * R; ++k) {
+                float4 v;
+                if (k == R) v = q[R];
+                else if (VEC) v = *reinterpret_cast<const float4 *>(&pl[warp + k][kStLead + 4 * lane]);
+                else {
+                    const float *s = &pl[warp + k][kStLead + 4 * lane];
+                    v = make_float4(s[0], s[1], s[2], s[3]);
+                }
+                const float wy = P.w[1][k];
+                o[0] = fmaf(wy, v.x, o[0]);
+                o[1] = fmaf(wy, v.y, o[1]);
+                o[2] = fmaf(wy, v.z, o[2]);
+                o[3] = fmaf(wy, v.w, o[3]);
+            }
+            // x neighbours: the vectors left and right of the own one
+            float xs[12];
+            {
+                const float4 l = *reinterpret_cast<const float4 *>(&pl[R + warp][4 * lane]);
+                const float4 r = *reinterpret_cast<const float4 *>(&pl[R + warp][4 * lane + 8]);
+                xs[0] = l.x; xs[1] = l.y; xs[2] = l.z; xs[3] = l.w;
+                if (VEC) {
+                    xs[4] = q[R].x; xs[5] = q[R].y; xs[6] = q[R].z; xs[7] = q[R].w;
+                } else {
+                    // a ragged last vector: its cells beyond the bulk are extra-column cells, not the thread's own
+                    const float4 c = *reinterpret_cast<const float4 *>(&pl[R + warp][kStLead + 4 * lane]);
+                    xs[4] = c.x; xs[5] = c.y; xs[6] = c.z; xs[7] = c.w;
+                }
+                xs[8] = r.x; xs[9] = r.y; xs[10] = r.z; xs[11] = r.w;
+            }
+#pragma unroll
+            for (int k = 0; k <= 2 * R; ++k) {
+                const float wx = P.w[2][k];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[e] = fmaf(wx, xs[4 + e + k - R], o[e]);
+            }
+            if (VEC) {
+                *reinterpret_cast<float4 *>(optr) = make_float4(o[0], o[1], o[2], o[3]);
+            } else {
+                optr[0] = o[0];
+                if (x + 1 < bx) optr[1] = o[1];
+                if (x + 2 < bx) optr[2] = o[2];
+                if (x + 3 < bx) optr[3] = o[3];
+            }
+        }
+        optr += oplane;
+#pragma unroll
+        for (int i = 0; i < 2 * R; ++i) q[i] = q[i + 1];
+        q[2 * R] = lead;
+        hrow = hrow_n;
+        hcol = hcol_n;
+    }
+
+    if (P.clear_ghosts && oo > 0) {
+        // this block's part of the ghost shell of the output shard: its box of bulk cells, extended
+        // through the ghost layers wherever it touches a face of the shard
+        const int zl = z0 == 0 ? 0 : z0 + oo, zh = z1 == bz ? bz + 2 * oo : z1 + oo;
+        const int yl = y0 == 0 ? 0 : y0 + oo, yh = y0 + th == by ? by + 2 * oo : y0 + th + oo;
+        const int xl = x0 == 0 ? 0 : x0 + oo, xh = x0 + tw == bx ? bx + 2 * oo : x0 + tw + oo;
+        float *ob = P.out[shard];
+        const int ny = yh - yl, nx = xh - xl;
+        for (int pz = zl; pz < zh; ++pz) {
+            const bool zg = pz < oo || pz >= bz + oo;
+            for (int idx = threadIdx.x; idx < ny * nx; idx += kStThreads) {
+                const int py = yl + idx / nx, px = xl + idx % nx;
+                if (zg || py < oo || py >= by + oo || px < oo || px >= bx + oo) ob[((size_t)pz * opy + py) * opx + px] = 0.f;
+            }
+        }
+    }
+}
+
+template <int R>
+static distdl_status_t launch_stencil(const StencilParams &P, unsigned grid, bool vec, cudaStream_t s) {
+    if (vec) stencil3d_kernel<R, true><<<grid, kStThreads, 0, s>>>(P);
+    else stencil3d_kernel<R, false><<<grid, kStThreads, 0, s>>>(P);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+static distdl_status_t stencil_impl(const distdl_partition *p, const void *const *in, const float *w, int32_t radius,
+                                    void *const *out, void *stream, bool adj, const char *what) {
+    clear_error();
+    if (!p || !in || !w || !out) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (p->rank != 3 || p->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-3 F32 partition", what);
+    if (radius < 1 || radius > kStMaxR) return fail(DISTDL_ERR_UNSUPPORTED, "%s: radius %d (supported: 1..%d)", what, radius, kStMaxR);
+    if (p->num_workers > kStMaxWorkers) return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d workers", what, kStMaxWorkers);
+    for (int k = 0; k < 3; ++k) {
+        if (p->pshape[k] > kStMaxPerDim)
+            return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d workers along a dimension", what, kStMaxPerDim);
+        for (int32_t c = 0; c < p->pshape[k]; ++c)
+            if (p->hlo[k][c] != radius || p->hhi[k][c] != radius)
+                return fail(DISTDL_ERR_SHAPE, "%s: halo widths must equal the radius %d on every side", what, radius);
+    }
+    StencilParams P;
+    memset(&P, 0, sizeof(P));
+    int64_t mz = 0, my = 0, mx = 0;
+    for (int32_t c = 0; c < p->pshape[0]; ++c) mz = std::max<int64_t>(mz, P.bz[c] = (int32_t)p->size[0][c]);
+    for (int32_t c = 0; c < p->pshape[1]; ++c) my = std::max<int64_t>(my, P.by[c] = (int32_t)p->size[1][c]);
+    for (int32_t c = 0; c < p->pshape[2]; ++c) mx = std::max<int64_t>(mx, P.bx[c] = (int32_t)p->size[2][c]);
+    P.pz = p->pshape[0];
+    P.py = p->pshape[1];
+    P.px = p->pshape[2];
+    P.in_off = adj ? 0 : radius;
+    P.out_off = adj ? radius : 0;
+    P.clear_ghosts = adj ? 1 : 0;
+    P.tiles_x = (int32_t)((mx + kStCols - 1) / kStCols);
+    P.tiles_y = (int32_t)((my + kStRows - 1) / kStRows);
+    P.chunks_z = (int32_t)((mz + kStChunk - 1) / kStChunk);
+    for (int d = 0; d < 3; ++d)
+        for (int k = 0; k <= 2 * radius; ++k) P.w[d][k] = adj ? w[d * (2 * radius + 1) + (2 * radius - k)] : w[d * (2 * radius + 1) + k];
+    // 16-byte accesses: every row of every layout starts on a 16-byte boundary and holds whole vectors
+    bool vec = (P.in_off % 4) == 0 && (P.out_off % 4) == 0;
+    for (int32_t c = 0; c < p->pshape[2]; ++c) vec = vec && (P.bx[c] % 4) == 0;
+    for (int32_t wk = 0; wk < p->num_workers; ++wk) {
+        if (!in[wk] || !out[wk]) return fail(DISTDL_ERR_INVALID_ARG, "%s: shard pointer %d is NULL", what, wk);
+        if (!aligned16(in[wk]) || !aligned16(out[wk])) return fail(DISTDL_ERR_ALIGNMENT, "%s: shard %d is not 16-byte aligned", what, wk);
+        if (p->shard_elems(wk) >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: shard %d too large", what, wk);
+        P.in[wk] = (const float *)in[wk];
+        P.out[wk] = (float *)out[wk];
+    }
+    const int64_t blocks = (int64_t)p->num_workers * P.chunks_z * P.tiles_y * P.tiles_x;
+    if (blocks >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (radius) {
+        case 1: return launch_stencil<1>(P, (unsigned)blocks, vec, s);
+        case 2: return launch_stencil<2>(P, (unsigned)blocks, vec, s);
+        case 3: return launch_stencil<3>(P, (unsigned)blocks, vec, s);
+        default: return launch_stencil<4>(P, (unsigned)blocks, vec, s);
+    }
+}
+
+}  // namespace distdl
+
+extern "C" distdl_status_t distdl_stencil3d_fwd(const distdl_partition_t *p, const void *const *x, const float *w,
+                                                int32_t radius, void *const *y, void *stream) {
+    return distdl::stencil_impl(p, x, w, radius, y, stream, false, "stencil3d_fwd");
+}
+extern "C" distdl_status_t distdl_stencil3d_adj(const distdl_partition_t *p, const void *const *dy, const float *w,
+                                                int32_t radius, void *const *dx, void *stream) {
+    return distdl::stencil_impl(p, dy, w, radius, dx, stream, true, "stencil3d_adj");
+}

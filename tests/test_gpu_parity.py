@@ -347,6 +347,62 @@ def test_conv_param_gradients(case, integer):
 
 
 # --------------------------------------------------------------------------
+# 3-D star-stencil layer
+# --------------------------------------------------------------------------
+
+STENCIL_CASES = [
+    # global shape, partition, radius
+    ((16, 16, 16), (1, 1, 1), 4),
+    ((40, 36, 48), (2, 2, 2), 4),         # vector path, every kind of neighbour
+    ((20, 19, 150), (2, 2, 2), 2),        # odd row lengths: element-wise path, ragged last vector
+    ((70, 20, 264), (1, 2, 2), 4),        # two column tiles per shard, the second one partly empty
+    ((130, 17, 40), (2, 1, 1), 1),        # two plane chunks per shard
+    ((12, 25, 36), (1, 3, 2), 3),
+    ((14, 40, 512), (3, 2, 2), 4),        # uneven plane split (5, 5, 4), full 128-column tiles
+    ((11, 21, 260), (2, 2, 2), 4),        # shards of 130 columns: a second tile of two columns
+]
+
+
+@pytest.mark.parametrize("case", STENCIL_CASES, ids=[str(c) for c in STENCIL_CASES])
+def test_stencil3d_fwd_and_adj(case):
+    gshape, pshape, R = case
+    opart = oracle.Partition(gshape, pshape, R, R)
+    obulk = oracle.Partition(gshape, pshape, 0, 0)
+    gpart = distdl.Partition(gshape, pshape, (R,) * 3, (R,) * 3)
+    xg = inputs.normal(gshape, 91)
+    w = inputs.normal((3, 2 * R + 1), 92, 0.5)
+    x = oracle.scatter_global(opart, xg, fill=lambda wk: np.full(opart.padded_shape(wk), 1e30, dtype=np.float32))
+    xs = [dev(a) for a in x]
+    ys = [torch.full(obulk.padded_shape(wk), -7.0, device=DEV) for wk in range(opart.num_workers)]
+    distdl.stencil3d_fwd(gpart, xs, w, ys)
+    torch.cuda.synchronize()
+    ref = oracle.stencil3d_fwd(opart, x, w)
+    bound = oracle.stencil3d_fwd(opart, [np.abs(a) for a in oracle.scatter_global(opart, xg)], np.abs(w))
+    # 6R+3 FMA roundings and the oracle's own rounding of its fp64 sum to fp32
+    eps = (6 * R + 3 + 2) * 2.0 ** -24
+    for wk in range(opart.num_workers):
+        assert np.all(np.abs(host(ys[wk]).astype(np.float64) - ref[wk]) <= eps * bound[wk] + 1e-30)
+        assert same_bits(host(xs[wk]), x[wk])            # x, ghosts included, is left untouched
+    # adjoint
+    dy = oracle.scatter_global(obulk, inputs.normal(gshape, 93))
+    dys = [dev(a) for a in dy]
+    dxs = [torch.full(opart.padded_shape(wk), 3.0, device=DEV) for wk in range(opart.num_workers)]
+    distdl.stencil3d_adj(gpart, dys, w, dxs)
+    torch.cuda.synchronize()
+    refa = oracle.stencil3d_adj(opart, dy, w)
+    bounda = oracle.stencil3d_adj(opart, [np.abs(a) for a in dy], np.abs(w))
+    for wk in range(opart.num_workers):
+        got = host(dxs[wk])
+        assert np.all(np.abs(got.astype(np.float64) - refa[wk]) <= eps * bounda[wk] + 1e-30)
+        mask = np.ones(opart.padded_shape(wk), dtype=bool)
+        mask[opart.bulk_slices(wk)] = False
+        assert not got[mask].any()                       # ghosts of dx are zero, as H* leaves them
+    xb = oracle.scatter_global(opart, xg)
+    r = oracle.adjoint_test_ratio([host(t) for t in ys], dy, xb, [host(t) for t in dxs])
+    assert r < 1e-5
+
+
+# --------------------------------------------------------------------------
 # Affine layer
 # --------------------------------------------------------------------------
 
