@@ -944,14 +944,15 @@ __device__ __forceinline__ void grad_accumulate(const float *xt, const float *dt
             unpack2(Pr[i + 1], b0, b1);
             Qr[i] = pack2(a1, b0);
         }
+        // pixel pair outermost, taps innermost: consecutive FMAs go to different running sums
 #pragma unroll
-        for (int r = 0; r < kRowsPerThread; ++r) {
-            const int a = rho - r;
-            if (a < 0 || a >= K) continue;
+        for (int p2 = 0; p2 < 4; ++p2) {
 #pragma unroll
-            for (int b = 0; b < K; ++b) {
+            for (int r = 0; r < kRowsPerThread; ++r) {
+                const int a = rho - r;
+                if (a < 0 || a >= K) continue;
 #pragma unroll
-                for (int p2 = 0; p2 < 4; ++p2) {
+                for (int b = 0; b < K; ++b) {
                     // pixels (2 p2, 2 p2 + 1) of output row r read x columns 2 p2 + b, 2 p2 + b + 1
                     const uint64_t X = (b & 1) ? Qr[p2 + (b - 1) / 2] : Pr[p2 + b / 2];
                     acc[a][b] = fma2(D[r][p2], X, acc[a][b]);

@@ -19,6 +19,7 @@
 // the arithmetic of the current plane.  Two plane buffers, one barrier per plane.
 #include <algorithm>
 #include <cstring>
+#include <type_traits>
 
 #include "common.h"
 
@@ -65,6 +66,17 @@ __device__ __forceinline__ bool st_owner(const int32_t *b, int p, int s, int c, 
     return true;
 }
 
+// Calls f(phase PH, plane z + PH) for PH = 0 .. N-1 as long as the plane is below z1.
+template <int PH, int N, typename F>
+__device__ __forceinline__ void st_phases(F &f, int z, int z1) {
+    if constexpr (PH < N) {
+        if (z + PH < z1) {
+            f(std::integral_constant<int, PH>{}, z + PH);
+            st_phases<PH + 1, N>(f, z, z1);
+        }
+    }
+}
+
 template <int R, bool VEC>
 __global__ void __launch_bounds__(kStThreads, 2)
 stencil3d_kernel(const __grid_constant__ StencilParams P) {
@@ -90,47 +102,73 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
     const int y = y0 + warp, x = x0 + 4 * lane;
     const bool row_ok = y < by;
 
-    // this thread's four cells of plane zp (any plane within R of the chunk), zeros outside the tensor
-    auto load_own = [&](int zp) -> float4 {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        int so, zo;
-        if (!row_ok || x >= bx || !st_owner(P.bz, P.pz, sz, zp, so, zo)) return v;
-        const float *src = P.in[(so * P.py + sy) * P.px + sx] +
-                           ((size_t)(zo + io) * (by + 2 * io) + (size_t)(y + io)) * ipx + (x + io);
+    // Everything that does not change from plane to plane is resolved once: for each kind of load a
+    // base pointer (plane 0 of the owning shard, the thread's row and column; nullptr = zeros) and the
+    // plane stride of that shard, in elements (a shard holds fewer than 2^31 of them).
+    auto load4 = [&](const float *src) -> float4 {
         if (VEC) return __ldg(reinterpret_cast<const float4 *>(src));
-        v.x = __ldg(src);
+        float4 v = make_float4(__ldg(src), 0.f, 0.f, 0.f);
         if (x + 1 < bx) v.y = __ldg(src + 1);
         if (x + 2 < bx) v.z = __ldg(src + 2);
         if (x + 3 < bx) v.w = __ldg(src + 3);
         return v;
     };
+    const uint32_t ipy = (uint32_t)(by + 2 * io);
+    const uint32_t own_stride = ipy * (uint32_t)ipx;                   // the same in the shards below and above
+    const bool own_ok = row_ok && x < bx;
+    const uint32_t own_off = (uint32_t)(y + io) * (uint32_t)ipx + (uint32_t)(x + io);
+    const float *own_mid = own_ok ? P.in[shard] + own_off : nullptr;
+    const float *own_lo = own_ok && sz > 0 ? P.in[shard - P.py * P.px] + own_off : nullptr;
+    const float *own_hi = own_ok && sz + 1 < P.pz ? P.in[shard + P.py * P.px] + own_off : nullptr;
+    const int bz_lo = sz > 0 ? P.bz[sz - 1] : 0, bz_hi = sz + 1 < P.pz ? P.bz[sz + 1] : 0;
+    // this thread's four cells of plane zp (any plane within R of the chunk), zeros outside the tensor
+    auto load_own = [&](int zp) -> float4 {
+        const float *base = own_mid;
+        if (zp < 0) {
+            base = own_lo;
+            zp += bz_lo;
+            if (zp < 0) base = nullptr;
+        } else if (zp >= bz) {
+            base = own_hi;
+            zp -= bz;
+            if (zp >= bz_hi) base = nullptr;
+        }
+        if (!base) return make_float4(0.f, 0.f, 0.f, 0.f);
+        return load4(base + (uint32_t)(zp + io) * own_stride);
+    };
     // warps 0 .. 2R-1: this thread's four cells of one extra row of plane zp (a plane of the chunk itself)
     const int hrow_y = warp < R ? y0 - R + warp : y0 + th + (warp - R);
     const int hrow_s = warp < R ? warp : R + th + (warp - R);           // its row in the shared-memory plane
-    auto load_hrow = [&](int zp) -> float4 {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float *hrow_base = nullptr;
+    uint32_t hrow_stride = 0;
+    {
         int so, yo;
-        if (warp >= 2 * R || x >= bx || !st_owner(P.by, P.py, sy, hrow_y, so, yo)) return v;
-        const float *src = P.in[(sz * P.py + so) * P.px + sx] +
-                           ((size_t)(zp + io) * (P.by[so] + 2 * io) + (size_t)(yo + io)) * ipx + (x + io);
-        if (VEC) return __ldg(reinterpret_cast<const float4 *>(src));
-        v.x = __ldg(src);
-        if (x + 1 < bx) v.y = __ldg(src + 1);
-        if (x + 2 < bx) v.z = __ldg(src + 2);
-        if (x + 3 < bx) v.w = __ldg(src + 3);
-        return v;
+        if (warp < 2 * R && x < bx && st_owner(P.by, P.py, sy, hrow_y, so, yo)) {
+            hrow_stride = (uint32_t)(P.by[so] + 2 * io) * (uint32_t)ipx;
+            hrow_base = P.in[(sz * P.py + so) * P.px + sx] + (uint32_t)(yo + io) * (uint32_t)ipx + (uint32_t)(x + io);
+        }
+    }
+    auto load_hrow = [&](int zp) -> float4 {
+        if (!hrow_base) return make_float4(0.f, 0.f, 0.f, 0.f);
+        return load4(hrow_base + (uint32_t)(zp + io) * hrow_stride);
     };
     // threads 0 .. 8 * 2R - 1: one cell of an extra column of plane zp
     const int hc_row = threadIdx.x / (2 * R), hc_c = threadIdx.x % (2 * R);
     const bool hc_active = (int)threadIdx.x < kStRows * 2 * R && y0 + hc_row < by;
     const int hc_x = hc_c < R ? x0 - R + hc_c : x0 + tw + (hc_c - R);
     const int hc_s = kStLead + (hc_x - x0);                               // its column in the shared-memory plane
-    auto load_hcol = [&](int zp) -> float {
+    const float *hcol_base = nullptr;
+    uint32_t hcol_stride = 0;
+    {
         int so, xo;
-        if (!hc_active || !st_owner(P.bx, P.px, sx, hc_x, so, xo)) return 0.f;
-        const int pitch = P.bx[so] + 2 * io;
-        return __ldg(P.in[(sz * P.py + sy) * P.px + so] +
-                     ((size_t)(zp + io) * (by + 2 * io) + (size_t)(y0 + hc_row + io)) * pitch + (xo + io));
+        if (hc_active && st_owner(P.bx, P.px, sx, hc_x, so, xo)) {
+            const uint32_t pitch = (uint32_t)(P.bx[so] + 2 * io);
+            hcol_stride = ipy * pitch;
+            hcol_base = P.in[(sz * P.py + sy) * P.px + so] + (uint32_t)(y0 + hc_row + io) * pitch + (uint32_t)(xo + io);
+        }
+    }
+    auto load_hcol = [&](int zp) -> float {
+        return hcol_base ? __ldg(hcol_base + (uint32_t)(zp + io) * hcol_stride) : 0.f;
     };
 
     // prime: planes z0 - R .. z0 + R, extra row / column of plane z0
@@ -145,19 +183,25 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
     float *optr = P.out[shard] + ((size_t)(z0 + oo) * opy + (size_t)(y + oo)) * opx + (x + oo);
     const size_t oplane = (size_t)opy * opx;
 
-    for (int z = z0; z < z1; ++z) {
+    // One plane.  The 2R+1 planes of the queue are not shifted: in phase PH the plane at offset j
+    // (0 = R planes behind the current one) sits in q[(PH + j) % N], and the slot of the oldest plane
+    // takes the newly fetched one, which makes it offset 2R of phase PH + 1.
+    constexpr int N = 2 * R + 1;
+    auto step = [&](auto phase, int z) {
+        constexpr int PH = decltype(phase)::value;
+        const float4 ctr = q[(PH + R) % N];
         float(*pl)[kStPitch] = plane[(z - z0) & 1];
         // current plane into shared memory: own cells, one extra-row vector, one extra-column cell.
         // Cells beyond the bulk are written by the extra-row / extra-column threads only.
         if (row_ok) {
             if (VEC) {
-                if (x < bx) *reinterpret_cast<float4 *>(&pl[R + warp][kStLead + 4 * lane]) = q[R];
+                if (x < bx) *reinterpret_cast<float4 *>(&pl[R + warp][kStLead + 4 * lane]) = ctr;
             } else {
                 float *d = &pl[R + warp][kStLead + 4 * lane];
-                if (x < bx) d[0] = q[R].x;
-                if (x + 1 < bx) d[1] = q[R].y;
-                if (x + 2 < bx) d[2] = q[R].z;
-                if (x + 3 < bx) d[3] = q[R].w;
+                if (x < bx) d[0] = ctr.x;
+                if (x + 1 < bx) d[1] = ctr.y;
+                if (x + 2 < bx) d[2] = ctr.z;
+                if (x + 3 < bx) d[3] = ctr.w;
             }
         }
         if (warp < 2 * R) {
@@ -188,16 +232,17 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
 #pragma unroll
             for (int k = 0; k <= 2 * R; ++k) {
                 const float wz = P.w[0][k];
-                o[0] = fmaf(wz, q[k].x, o[0]);
-                o[1] = fmaf(wz, q[k].y, o[1]);
-                o[2] = fmaf(wz, q[k].z, o[2]);
-                o[3] = fmaf(wz, q[k].w, o[3]);
+                const float4 v = q[(PH + k) % N];
+                o[0] = fmaf(wz, v.x, o[0]);
+                o[1] = fmaf(wz, v.y, o[1]);
+                o[2] = fmaf(wz, v.z, o[2]);
+                o[3] = fmaf(wz, v.w, o[3]);
             }
             // y neighbours: the rows above and below in shared memory
 #pragma unroll
             for (int k = 0; k <= 2 * R; ++k) {
                 float4 v;
-                if (k == R) v = q[R];
+                if (k == R) v = ctr;
                 else if (VEC) v = *reinterpret_cast<const float4 *>(&pl[warp + k][kStLead + 4 * lane]);
                 else {
                     const float *s = &pl[warp + k][kStLead + 4 * lane];
@@ -216,7 +261,7 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
                 const float4 r = *reinterpret_cast<const float4 *>(&pl[R + warp][4 * lane + 8]);
                 xs[0] = l.x; xs[1] = l.y; xs[2] = l.z; xs[3] = l.w;
                 if (VEC) {
-                    xs[4] = q[R].x; xs[5] = q[R].y; xs[6] = q[R].z; xs[7] = q[R].w;
+                    xs[4] = ctr.x; xs[5] = ctr.y; xs[6] = ctr.z; xs[7] = ctr.w;
                 } else {
                     // a ragged last vector: its cells beyond the bulk are extra-column cells, not the thread's own
                     const float4 c = *reinterpret_cast<const float4 *>(&pl[R + warp][kStLead + 4 * lane]);
@@ -240,12 +285,11 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
             }
         }
         optr += oplane;
-#pragma unroll
-        for (int i = 0; i < 2 * R; ++i) q[i] = q[i + 1];
-        q[2 * R] = lead;
+        q[PH % N] = lead;
         hrow = hrow_n;
         hcol = hcol_n;
-    }
+    };
+    for (int z = z0; z < z1; z += N) st_phases<0, N>(step, z, z1);
 
     if (P.clear_ghosts && oo > 0) {
         // this block's part of the ghost shell of the output shard: its box of bulk cells, extended
@@ -255,11 +299,32 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
         const int xl = x0 == 0 ? 0 : x0 + oo, xh = x0 + tw == bx ? bx + 2 * oo : x0 + tw + oo;
         float *ob = P.out[shard];
         const int ny = yh - yl, nx = xh - xl;
+        // whole planes of the ghost layers below / above
         for (int pz = zl; pz < zh; ++pz) {
-            const bool zg = pz < oo || pz >= bz + oo;
-            for (int idx = threadIdx.x; idx < ny * nx; idx += kStThreads) {
-                const int py = yl + idx / nx, px = xl + idx % nx;
-                if (zg || py < oo || py >= by + oo || px < oo || px >= bx + oo) ob[((size_t)pz * opy + py) * opx + px] = 0.f;
+            if (pz >= oo && pz < bz + oo) continue;
+            for (int idx = threadIdx.x; idx < ny * nx; idx += kStThreads)
+                ob[((size_t)pz * opy + (yl + idx / nx)) * opx + (xl + idx % nx)] = 0.f;
+        }
+        // planes of the bulk: ghost rows over the whole width, then ghost columns beside the bulk rows
+        const int gy_lo = y0 == 0 ? oo : 0, gy = gy_lo + (y0 + th == by ? oo : 0);
+        const int gx_lo = x0 == 0 ? oo : 0, gx = gx_lo + (x0 + tw == bx ? oo : 0);
+        const int per_plane = gy * nx + th * gx;
+        if (per_plane > 0) {
+            const int total = (z1 - z0) * per_plane;
+            for (int idx = threadIdx.x; idx < total; idx += kStThreads) {
+                const int pz = z0 + oo + idx / per_plane;
+                int e = idx % per_plane, py, px;
+                if (e < gy * nx) {
+                    const int r = e / nx;
+                    py = r < gy_lo ? r : by + oo + (r - gy_lo);
+                    px = xl + e % nx;
+                } else {
+                    e -= gy * nx;
+                    const int c = e % gx;
+                    py = y0 + oo + e / gx;
+                    px = c < gx_lo ? c : bx + oo + (c - gx_lo);
+                }
+                ob[((size_t)pz * opy + py) * opx + px] = 0.f;
             }
         }
     }
