@@ -182,6 +182,7 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
     const int opy = by + 2 * oo, opx = bx + 2 * oo;
     float *optr = P.out[shard] + ((size_t)(z0 + oo) * opy + (size_t)(y + oo)) * opx + (x + oo);
     const size_t oplane = (size_t)opy * opx;
+    const bool clear_x = P.clear_ghosts && oo > 0;
 
     // One plane.  The 2R+1 planes of the queue are not shifted: in phase PH the plane at offset j
     // (0 = R planes behind the current one) sits in q[(PH + j) % N], and the slot of the oldest plane
@@ -283,6 +284,20 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
                 if (x + 2 < bx) optr[2] = o[2];
                 if (x + 3 < bx) optr[3] = o[3];
             }
+            // adjoint: the ghost columns beside this row are cleared by the threads that write the row's
+            // ends, so that they land in the same lines of memory as the row itself
+            if (clear_x) {
+                if (x == 0) {
+                    if (VEC && R == 4) *reinterpret_cast<float4 *>(optr - 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+                    else
+                        for (int c = 1; c <= oo; ++c) optr[-c] = 0.f;
+                }
+                if (x + 4 >= bx) {
+                    if (VEC && R == 4) *reinterpret_cast<float4 *>(optr + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+                    else
+                        for (int c = 0; c < oo; ++c) optr[bx - x + c] = 0.f;
+                }
+            }
         }
         optr += oplane;
         q[PH % N] = lead;
@@ -305,26 +320,17 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
             for (int idx = threadIdx.x; idx < ny * nx; idx += kStThreads)
                 ob[((size_t)pz * opy + (yl + idx / nx)) * opx + (xl + idx % nx)] = 0.f;
         }
-        // planes of the bulk: ghost rows over the whole width, then ghost columns beside the bulk rows
+        // planes of the bulk: ghost rows over the whole width (the ghost columns beside bulk rows were
+        // cleared together with those rows)
         const int gy_lo = y0 == 0 ? oo : 0, gy = gy_lo + (y0 + th == by ? oo : 0);
-        const int gx_lo = x0 == 0 ? oo : 0, gx = gx_lo + (x0 + tw == bx ? oo : 0);
-        const int per_plane = gy * nx + th * gx;
+        const int per_plane = gy * nx;
         if (per_plane > 0) {
             const int total = (z1 - z0) * per_plane;
             for (int idx = threadIdx.x; idx < total; idx += kStThreads) {
                 const int pz = z0 + oo + idx / per_plane;
-                int e = idx % per_plane, py, px;
-                if (e < gy * nx) {
-                    const int r = e / nx;
-                    py = r < gy_lo ? r : by + oo + (r - gy_lo);
-                    px = xl + e % nx;
-                } else {
-                    e -= gy * nx;
-                    const int c = e % gx;
-                    py = y0 + oo + e / gx;
-                    px = c < gx_lo ? c : bx + oo + (c - gx_lo);
-                }
-                ob[((size_t)pz * opy + py) * opx + px] = 0.f;
+                const int e = idx % per_plane, r = e / nx;
+                const int py = r < gy_lo ? r : by + oo + (r - gy_lo);
+                ob[((size_t)pz * opy + py) * opx + (xl + e % nx)] = 0.f;
             }
         }
     }
