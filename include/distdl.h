@@ -44,7 +44,7 @@ typedef enum {
     DISTDL_ERR_NOMEM = 7
 } distdl_status_t;
 
-typedef enum { DISTDL_F32 = 0, DISTDL_BF16 = 1 } distdl_dtype_t;
+typedef enum { DISTDL_F32 = 0, DISTDL_BF16 = 1, DISTDL_F64 = 2 } distdl_dtype_t;
 
 #define DISTDL_MAX_RANK 5
 #define DISTDL_MAX_WORKERS 256
@@ -122,7 +122,8 @@ distdl_status_t distdl_halo_widths_1d(int64_t n, int32_t p, int32_t kernel, int3
  * n = elements per realisation (n = 0 is a no-op), 1 <= k.  In broadcast a dst[i] equal to
  * src is the in-place form (identity copy, skipped); any other overlap between buffers is not
  * detected and gives undefined results.  In sum-reduce dst may equal src[0] only.
- * F32 and BF16 are supported by the copies; the sums support F32 (BF16: UNSUPPORTED).
+ * F32, BF16 and F64, for the copies and for the sums: every addition is the exact sum of its two
+ * operands rounded once to the type, to nearest even (fp32 / fp64 IEEE addition; bfloat16: add.rn.bf16).
  * ---------------------------------------------------------------------- */
 distdl_status_t distdl_broadcast_fwd(const void *src, void *const *dst, int32_t k, int64_t n,
                                      distdl_dtype_t t, void *stream);
@@ -143,7 +144,7 @@ distdl_status_t distdl_sumreduce_adj(const void *dy, void *const *dx, int32_t k,
  * halo_adj: every bulk cell that some neighbour holds ghost copies of <- itself plus those
  *   copies, summed in the nested order of H* (dimension d-1 undone first, so the sum is
  *   grouped by dimension 0 outermost; within a dimension: own, low neighbour, high neighbour);
- *   then every ghost cell <- 0.  F32 only.
+ *   then every ghost cell <- 0.  Additions in the partition's type (F32, BF16 or F64), each rounded once.
  * shards[w] = device pointer of worker w's padded shard, w < P (host array).
  * Shards must not overlap one another.
  * ---------------------------------------------------------------------- */
@@ -193,12 +194,12 @@ distdl_status_t distdl_halo_fwd_noalloc(int32_t rank, const int64_t *global_shap
  *   repartition_fwd: dst[Pdst] <- src[Psrc]   (contiguous row-major blocks, bit copies)
  *   repartition_adj: dx[Psrc] <- dy[Pdst]     (every copy is a move, so the adjoint is the
  *                                              inverse: the all-to-all back)
- * Outputs may overlap neither each other nor any input (DISTDL_ERR_INVALID_ARG).  F32 and BF16.
+ * Outputs may overlap neither each other nor any input (DISTDL_ERR_INVALID_ARG).  F32, BF16 and F64.
  * repartition_shard_shape: extents of one worker's block (destination != 0: in the destination
  * partition); `shape` has rank entries.
  *
  * allreduce: A = B R on k buffers of n elements in place: every buffer ends up holding
- * ((b[0] + b[1]) + ...) + b[k-1] (F32, fixed order); self-adjoint.  Two launches.
+ * ((b[0] + b[1]) + ...) + b[k-1] (fixed order, in the arithmetic of `t`); self-adjoint.  Two launches.
  * ---------------------------------------------------------------------- */
 typedef struct distdl_repartition distdl_repartition_t; /* opaque, immutable after create */
 distdl_status_t distdl_repartition_create(int32_t rank, const int64_t *global_shape,

@@ -33,6 +33,8 @@ from .primitives import (  # noqa: F401
     repartition_fwd,
     repartition_adj,
     allreduce,
+    round_to_bf16_bits,
+    bf16_add,
 )
 from .layers import (  # noqa: F401
     conv_fwd,

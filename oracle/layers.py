@@ -14,6 +14,7 @@ import numpy as np
 
 from .partition import Partition
 from .primitives import (
+    bf16_bits_to_f64,
     assemble_global,
     scatter_global,
     halo_adj_sequence,
@@ -223,12 +224,6 @@ def stencil3d_fwd_exchange_then_local(part: Partition, x_shards, w):
 # --------------------------------------------------------------------------
 # Distributed affine layer (Section 4, "Dense layers")
 # --------------------------------------------------------------------------
-
-def bf16_bits_to_f64(bits):
-    """Widen bfloat16 bit patterns (uint16) exactly to fp64."""
-    u = np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
-    return u.view(np.float32).astype(np.float64)
-
 
 def affine_fwd(x_parts, w_parts, pfo, pfi, bias_parts=None):
     """Forward affine algorithm on a P_fo x P_fi worker grid.

@@ -20,16 +20,50 @@ def broadcast_fwd(src, k):
     return [np.array(src, copy=True) for _ in range(k)]
 
 
-def sumreduce_fwd(parts):
+def round_to_bf16_bits(x):
+    """fp64 values -> bfloat16 bit patterns (uint16), one rounding to nearest, ties to even.
+
+    bfloat16 has 8 significant bits and the exponent range of fp32: the spacing of
+    representable values at |x| in [2^(e-1), 2^e) is 2^(e-8), and never finer than
+    2^-133 (subnormals).  The value is divided by its spacing, rounded to the nearest
+    integer with ties to even (numpy.rint), and scaled back; the result is exactly
+    representable in fp32, whose upper 16 bits are the answer.  Values beyond the
+    largest finite bfloat16 are not handled (the operators here never produce them).
+    """
+    x = np.asarray(x, dtype=np.float64)
+    _, e = np.frexp(x)                                  # |x| = m * 2^e with m in [0.5, 1)
+    q = np.maximum(e - 8, -133).astype(np.int64)
+    r = np.ldexp(np.rint(np.ldexp(x, -q)), q)
+    return (r.astype(np.float32).view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f64(bits):
+    """bfloat16 bit patterns (uint16) -> the same values in fp64 (exact)."""
+    u = np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+def bf16_add(a_bits, b_bits):
+    """a + b in bfloat16 arithmetic on bit patterns: the exact sum, rounded once.
+
+    The sum of two bfloat16 values is exact in fp64 unless their exponents differ by
+    more than 44, in which case the fp64 sum already rounds to the larger operand, as
+    the bfloat16 result does.
+    """
+    return round_to_bf16_bits(bf16_bits_to_f64(a_bits) + bf16_bits_to_f64(b_bits))
+
+
+def sumreduce_fwd(parts, add=None):
     """R_{{k}->a} = B*: sum of the k realisations (adjoint-of-broadcast equation).
 
     The sum is taken in worker order 0, 1, ..., k-1 in the arithmetic of the
     inputs: acc = y_0; acc = acc + y_i.  Starting from y_0 makes k = 1 an exact
-    copy.
+    copy.  `add` replaces the addition of the arrays' own type (bf16_add for
+    bfloat16 bit patterns).
     """
     acc = np.array(parts[0], copy=True)
     for i in range(1, len(parts)):
-        acc = acc + parts[i]
+        acc = acc + parts[i] if add is None else add(acc, parts[i])
     return acc
 
 
@@ -199,8 +233,8 @@ def halo_fwd_sequence(part: Partition, shards):
 # Adjoint halo exchange H* (Section 3, the H* equation; Appendix B.2)
 # --------------------------------------------------------------------------
 
-def halo_adj_sequence(part: Partition, shards):
-    """H* as the paper's reversed operator sequence.
+def halo_adj_sequence(part: Partition, shards, add=None):
+    """H* as the paper's reversed operator sequence (`add`: see sumreduce_fwd).
 
     Ghosts on the tensor's own boundary are cleared (the adjoint of writing a
     zero).  Then for dimension k = d-1 down to 0 and every worker: the ghost
@@ -249,7 +283,7 @@ def halo_adj_sequence(part: Partition, shards):
                 assert width <= b[k], "halo reaches beyond the adjacent worker"
                 dst = _slab(part, w, k, mine, True)
                 src = _slab(part, n, k, theirs, True)
-                y[w][dst] = y[w][dst] + y[n][src]
+                y[w][dst] = y[w][dst] + y[n][src] if add is None else add(y[w][dst], y[n][src])
                 y[n][src] = 0
     return y
 
@@ -312,7 +346,7 @@ def repartition_adj(src_part: Partition, dst_part: Partition, dy_shards):
     return scatter_global(src_part, assemble_global(dst_part, dy_shards))
 
 
-def allreduce(parts):
+def allreduce(parts, add=None):
     """All-reduce = broadcast after sum-reduce (self-adjoint): every worker ends up with
     the fixed-order sum of all k realisations."""
-    return broadcast_fwd(sumreduce_fwd(parts), len(parts))
+    return broadcast_fwd(sumreduce_fwd(parts, add), len(parts))

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libdistdl.so")
 
 F32 = 0
 BF16 = 1
+F64 = 2
 MAX_RANK = 5
 
 STATUS_NAMES = {
@@ -122,6 +123,8 @@ def _dtype_code(t):
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
+    if t.dtype == torch.float64:
+        return F64
     raise TypeError("unsupported dtype %s" % t.dtype)
 
 

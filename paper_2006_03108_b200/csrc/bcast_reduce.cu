@@ -60,19 +60,47 @@ broadcast_kernel(const uint4 *__restrict__ src, const __grid_constant__ FanPoint
     }
 }
 
-__device__ __forceinline__ uint4 add_f32x4(uint4 a, uint4 b) {
+// One addition per element of a 16-byte vector, each the exact sum rounded once to the type.
+// DT: 0 = four fp32, 1 = eight bfloat16, 2 = two fp64.
+__device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ unsigned short add_bf16(unsigned short a, unsigned short b) {
+    unsigned short r;
+    asm("add.rn.bf16 %0, %1, %2;" : "=h"(r) : "h"(a), "h"(b));
+    return r;
+}
+template <int DT>
+__device__ __forceinline__ uint4 add_vec(uint4 a, uint4 b) {
     uint4 r;
-    r.x = __float_as_uint(__fadd_rn(__uint_as_float(a.x), __uint_as_float(b.x)));
-    r.y = __float_as_uint(__fadd_rn(__uint_as_float(a.y), __uint_as_float(b.y)));
-    r.z = __float_as_uint(__fadd_rn(__uint_as_float(a.z), __uint_as_float(b.z)));
-    r.w = __float_as_uint(__fadd_rn(__uint_as_float(a.w), __uint_as_float(b.w)));
+    if (DT == 0) {
+        r.x = __float_as_uint(__fadd_rn(__uint_as_float(a.x), __uint_as_float(b.x)));
+        r.y = __float_as_uint(__fadd_rn(__uint_as_float(a.y), __uint_as_float(b.y)));
+        r.z = __float_as_uint(__fadd_rn(__uint_as_float(a.z), __uint_as_float(b.z)));
+        r.w = __float_as_uint(__fadd_rn(__uint_as_float(a.w), __uint_as_float(b.w)));
+    } else if (DT == 1) {
+        r.x = add_bf16x2(a.x, b.x);
+        r.y = add_bf16x2(a.y, b.y);
+        r.z = add_bf16x2(a.z, b.z);
+        r.w = add_bf16x2(a.w, b.w);
+    } else {
+        const double lo = __dadd_rn(__hiloint2double((int)a.y, (int)a.x), __hiloint2double((int)b.y, (int)b.x));
+        const double hi = __dadd_rn(__hiloint2double((int)a.w, (int)a.z), __hiloint2double((int)b.w, (int)b.z));
+        r.x = (uint32_t)__double2loint(lo);
+        r.y = (uint32_t)__double2hiint(lo);
+        r.z = (uint32_t)__double2loint(hi);
+        r.w = (uint32_t)__double2hiint(hi);
+    }
     return r;
 }
 
-// dst[i] = ((src[0][i] + src[1][i]) + ...) + src[k-1][i]   (fp32, left fold in source order)
-template <int K>
+// dst[i] = ((src[0][i] + src[1][i]) + ...) + src[k-1][i]   (left fold in source order, in the type's arithmetic)
+// nvec 16-byte vectors, then `tail` trailing elements.
+template <int K, int DT>
 __global__ void __launch_bounds__(kStreamThreads)
-sumreduce_kernel(const __grid_constant__ FanPointers src, float *__restrict__ dst, int k_runtime, size_t nvec, int tail) {
+sumreduce_kernel(const __grid_constant__ FanPointers src, void *__restrict__ dst, int k_runtime, size_t nvec, int tail) {
     const int k = K > 0 ? K : k_runtime;
     const size_t stride = (size_t)gridDim.x * kStreamThreads;
     for (size_t i = (size_t)blockIdx.x * kStreamThreads + threadIdx.x; i < nvec; i += stride) {
@@ -83,14 +111,26 @@ sumreduce_kernel(const __grid_constant__ FanPointers src, float *__restrict__ ds
         uint4 acc = v[0];
 #pragma unroll
         for (int j = 1; j < (K > 0 ? K : kMaxFan); ++j)
-            if (j < k) acc = add_f32x4(acc, v[j]);
+            if (j < k) acc = add_vec<DT>(acc, v[j]);
         st_stream(reinterpret_cast<uint4 *>(dst) + i, acc);
     }
     if (blockIdx.x == 0 && (int)threadIdx.x < tail) {
-        const size_t e = nvec * 4 + threadIdx.x;
-        float acc = reinterpret_cast<const float *>(src.p[0])[e];
-        for (int j = 1; j < k; ++j) acc = __fadd_rn(acc, reinterpret_cast<const float *>(src.p[j])[e]);
-        dst[e] = acc;
+        if (DT == 0) {
+            const size_t e = nvec * 4 + threadIdx.x;
+            float acc = reinterpret_cast<const float *>(src.p[0])[e];
+            for (int j = 1; j < k; ++j) acc = __fadd_rn(acc, reinterpret_cast<const float *>(src.p[j])[e]);
+            reinterpret_cast<float *>(dst)[e] = acc;
+        } else if (DT == 1) {
+            const size_t e = nvec * 8 + threadIdx.x;
+            unsigned short acc = reinterpret_cast<const unsigned short *>(src.p[0])[e];
+            for (int j = 1; j < k; ++j) acc = add_bf16(acc, reinterpret_cast<const unsigned short *>(src.p[j])[e]);
+            reinterpret_cast<unsigned short *>(dst)[e] = acc;
+        } else {
+            const size_t e = nvec * 2 + threadIdx.x;
+            double acc = reinterpret_cast<const double *>(src.p[0])[e];
+            for (int j = 1; j < k; ++j) acc = __dadd_rn(acc, reinterpret_cast<const double *>(src.p[j])[e]);
+            reinterpret_cast<double *>(dst)[e] = acc;
+        }
     }
 }
 
@@ -154,7 +194,7 @@ static distdl_status_t broadcast_impl(const void *src, void *const *dst, int32_t
     clear_error();
     if (!src || !dst) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
     if (k < 1 || n < 0) return fail(DISTDL_ERR_INVALID_ARG, "%s: k = %d, n = %lld", what, k, (long long)n);
-    if (t != DISTDL_F32 && t != DISTDL_BF16) return fail(DISTDL_ERR_INVALID_ARG, "%s: bad dtype", what);
+    if (!valid_dtype(t)) return fail(DISTDL_ERR_INVALID_ARG, "%s: bad dtype", what);
     if (!aligned16(src)) return fail(DISTDL_ERR_ALIGNMENT, "%s: src is not 16-byte aligned", what);
     for (int32_t j = 0; j < k; ++j) {
         if (!dst[j]) return fail(DISTDL_ERR_INVALID_ARG, "%s: destination %d is NULL", what, j);
@@ -199,8 +239,11 @@ static distdl_status_t broadcast_impl(const void *src, void *const *dst, int32_t
 }
 
 template <int K>
-static void launch_sum(const FanPointers &fp, float *dst, int k, size_t nvec, int tail, int grid, cudaStream_t s) {
-    sumreduce_kernel<K><<<grid, kStreamThreads, 0, s>>>(fp, dst, k, nvec, tail);
+static void launch_sum(const FanPointers &fp, void *dst, int k, size_t nvec, int tail, int grid, distdl_dtype_t t,
+                       cudaStream_t s) {
+    if (t == DISTDL_F32) sumreduce_kernel<K, 0><<<grid, kStreamThreads, 0, s>>>(fp, dst, k, nvec, tail);
+    else if (t == DISTDL_BF16) sumreduce_kernel<K, 1><<<grid, kStreamThreads, 0, s>>>(fp, dst, k, nvec, tail);
+    else sumreduce_kernel<K, 2><<<grid, kStreamThreads, 0, s>>>(fp, dst, k, nvec, tail);
 }
 
 static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t k, int64_t n, distdl_dtype_t t,
@@ -208,8 +251,7 @@ static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t
     clear_error();
     if (!src || !dst) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
     if (k < 1 || n < 0) return fail(DISTDL_ERR_INVALID_ARG, "%s: k = %d, n = %lld", what, k, (long long)n);
-    if (t == DISTDL_BF16) return fail(DISTDL_ERR_UNSUPPORTED, "%s: BF16 sums are not implemented", what);
-    if (t != DISTDL_F32) return fail(DISTDL_ERR_INVALID_ARG, "%s: bad dtype", what);
+    if (!valid_dtype(t)) return fail(DISTDL_ERR_INVALID_ARG, "%s: bad dtype", what);
     if (!aligned16(dst)) return fail(DISTDL_ERR_ALIGNMENT, "%s: dst is not 16-byte aligned", what);
     for (int32_t j = 0; j < k; ++j) {
         if (!src[j]) return fail(DISTDL_ERR_INVALID_ARG, "%s: source %d is NULL", what, j);
@@ -217,8 +259,9 @@ static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t
         if (j > 0 && src[j] == dst) return fail(DISTDL_ERR_INVALID_ARG, "%s: dst may alias source 0 only", what);
     }
     if (n == 0) return DISTDL_OK;
-    const size_t nvec = (size_t)n / 4;
-    const int tail = (int)(n % 4);
+    const int per = 16 / elem_size(t);
+    const size_t nvec = (size_t)n / per;
+    const int tail = (int)(n % per);
     const int grid = stream_grid(nvec, 1);
     // sources in groups of kMaxFan; later groups continue the fold from dst, which keeps the order
     int32_t done = 0;
@@ -230,11 +273,11 @@ static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t
         for (int r = filled; r < kMaxFan; ++r) fp.p[r] = nullptr;
         cudaStream_t s = (cudaStream_t)stream;
         switch (filled) {
-            case 1: launch_sum<1>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
-            case 2: launch_sum<2>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
-            case 4: launch_sum<4>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
-            case 8: launch_sum<8>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
-            default: launch_sum<0>(fp, (float *)dst, filled, nvec, tail, grid, s); break;
+            case 1: launch_sum<1>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 2: launch_sum<2>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 4: launch_sum<4>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 8: launch_sum<8>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            default: launch_sum<0>(fp, dst, filled, nvec, tail, grid, t, s); break;
         }
         DISTDL_CUDA_CHECK(cudaGetLastError());
     }

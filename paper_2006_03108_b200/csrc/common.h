@@ -24,7 +24,8 @@ void clear_error();
     } while (0)
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline int elem_size(distdl_dtype_t t) { return t == DISTDL_F32 ? 4 : 2; }
+inline int elem_size(distdl_dtype_t t) { return t == DISTDL_F32 ? 4 : (t == DISTDL_F64 ? 8 : 2); }
+inline bool valid_dtype(distdl_dtype_t t) { return t == DISTDL_F32 || t == DISTDL_BF16 || t == DISTDL_F64; }
 
 // ---------------------------------------------------------------------------------------------
 // Device-side plan tables of the halo kernels.

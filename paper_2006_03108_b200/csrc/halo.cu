@@ -18,16 +18,49 @@ struct ShardPointers {
 
 constexpr int kHaloThreads = 256;
 
+// Element and 16-byte vector types of the sums, one addition per element, each the exact sum rounded
+// once to the type (fp32 / fp64 IEEE addition, add.rn.bf16).
+struct bf16x1 {
+    unsigned short v;
+};
+struct bf16x8 {
+    uint4 v;
+};
+__device__ __forceinline__ uint32_t halo_add_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
 __device__ __forceinline__ float4 vadd(float4 a, float4 b) {
     return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
 }
 __device__ __forceinline__ float vadd(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ double2 vadd(double2 a, double2 b) { return make_double2(__dadd_rn(a.x, b.x), __dadd_rn(a.y, b.y)); }
+__device__ __forceinline__ double vadd(double a, double b) { return __dadd_rn(a, b); }
+__device__ __forceinline__ bf16x8 vadd(bf16x8 a, bf16x8 b) {
+    bf16x8 r;
+    r.v.x = halo_add_bf16x2(a.v.x, b.v.x);
+    r.v.y = halo_add_bf16x2(a.v.y, b.v.y);
+    r.v.z = halo_add_bf16x2(a.v.z, b.v.z);
+    r.v.w = halo_add_bf16x2(a.v.w, b.v.w);
+    return r;
+}
+__device__ __forceinline__ bf16x1 vadd(bf16x1 a, bf16x1 b) {
+    bf16x1 r;
+    asm("add.rn.bf16 %0, %1, %2;" : "=h"(r.v) : "h"(a.v), "h"(b.v));
+    return r;
+}
 
 template <typename T> __device__ __forceinline__ T zero_of();
 template <> __device__ __forceinline__ float4 zero_of<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 template <> __device__ __forceinline__ float zero_of<float>() { return 0.f; }
 template <> __device__ __forceinline__ uint4 zero_of<uint4>() { return make_uint4(0, 0, 0, 0); }
 template <> __device__ __forceinline__ unsigned short zero_of<unsigned short>() { return 0; }
+template <> __device__ __forceinline__ unsigned long long zero_of<unsigned long long>() { return 0ull; }
+template <> __device__ __forceinline__ double2 zero_of<double2>() { return make_double2(0.0, 0.0); }
+template <> __device__ __forceinline__ double zero_of<double>() { return 0.0; }
+template <> __device__ __forceinline__ bf16x8 zero_of<bf16x8>() { return bf16x8{make_uint4(0, 0, 0, 0)}; }
+template <> __device__ __forceinline__ bf16x1 zero_of<bf16x1>() { return bf16x1{0}; }
 
 // Coordinates of flattened unit n inside the box (innermost dimension last).
 __device__ __forceinline__ void decompose(const HaloBox &box, uint32_t n, uint32_t *coord) {
@@ -102,6 +135,10 @@ __device__ __forceinline__ void stores_after(const float4 &v) {
     asm volatile("" ::"f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 __device__ __forceinline__ void stores_after(const float &v) { asm volatile("" ::"f"(v) : "memory"); }
+__device__ __forceinline__ void stores_after(const double2 &v) { asm volatile("" ::"d"(v.x), "d"(v.y) : "memory"); }
+__device__ __forceinline__ void stores_after(const double &v) { asm volatile("" ::"d"(v) : "memory"); }
+__device__ __forceinline__ void stores_after(const bf16x8 &v) { asm volatile("" ::"r"(v.v.x), "r"(v.v.y), "r"(v.v.z), "r"(v.v.w) : "memory"); }
+__device__ __forceinline__ void stores_after(const bf16x1 &v) { asm volatile("" ::"h"(v.v) : "memory"); }
 
 template <typename T, int NSRC>
 __device__ __forceinline__ void run_sum_tile_balanced(const HaloBox &box, const HaloSource *src,
@@ -230,10 +267,17 @@ halo_box_kernel(const HaloBox *__restrict__ boxes, const HaloSource *__restrict_
     if (!SUMS || nsrc <= 1) {
         if (s_box.vec) run_copy_tile<uint4>(s_box, s_src, nsrc, sh, first, count);
         else if (elem_bytes == 4) run_copy_tile<float>(s_box, s_src, nsrc, sh, first, count);
+        else if (elem_bytes == 8) run_copy_tile<unsigned long long>(s_box, s_src, nsrc, sh, first, count);
         else run_copy_tile<unsigned short>(s_box, s_src, nsrc, sh, first, count);
-    } else {
+    } else if (elem_bytes == 4) {
         if (s_box.vec) run_sum_tile<float4>(s_box, s_src, nsrc, sh, first, count);
         else run_sum_tile<float>(s_box, s_src, nsrc, sh, first, count);
+    } else if (elem_bytes == 8) {
+        if (s_box.vec) run_sum_tile<double2>(s_box, s_src, nsrc, sh, first, count);
+        else run_sum_tile<double>(s_box, s_src, nsrc, sh, first, count);
+    } else {
+        if (s_box.vec) run_sum_tile<bf16x8>(s_box, s_src, nsrc, sh, first, count);
+        else run_sum_tile<bf16x1>(s_box, s_src, nsrc, sh, first, count);
     }
 }
 
@@ -241,7 +285,6 @@ static distdl_status_t launch(const distdl_partition *p, const HaloPlanDevice &p
                               void *stream, bool adjoint, const char *what) {
     clear_error();
     if (!p || !shards) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
-    if (adjoint && p->dtype != DISTDL_F32) return fail(DISTDL_ERR_UNSUPPORTED, "%s: F32 only", what);
     if (!p->device_block) return fail(DISTDL_ERR_CUDA, "%s: the partition was created without a CUDA device", what);
     ShardPointers sh;
     for (int32_t w = 0; w < p->num_workers; ++w) {

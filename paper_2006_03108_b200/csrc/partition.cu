@@ -61,7 +61,7 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
     if (rank < 1 || rank > DISTDL_MAX_RANK)
         return fail(DISTDL_ERR_INVALID_ARG, "partition_create: rank %d outside 1..%d", rank, DISTDL_MAX_RANK);
     if (!global_shape || !partition_shape) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: NULL shape");
-    if (dtype != DISTDL_F32 && dtype != DISTDL_BF16) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: bad dtype");
+    if (!valid_dtype(dtype)) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: bad dtype");
     int64_t workers = 1;
     for (int k = 0; k < rank; ++k) {
         if (partition_shape[k] < 1) return fail(DISTDL_ERR_SHAPE, "partition_create: partition_shape[%d] < 1", k);
@@ -209,7 +209,7 @@ extern "C" distdl_status_t distdl_repartition_create(int32_t rank, const int64_t
     if (!global_shape || !src_partition_shape || !dst_partition_shape || !out)
         return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: NULL argument");
     if (rank < 1 || rank > DISTDL_MAX_RANK) return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: rank %d", rank);
-    if (dtype != DISTDL_F32 && dtype != DISTDL_BF16) return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: bad dtype");
+    if (!valid_dtype(dtype)) return fail(DISTDL_ERR_INVALID_ARG, "repartition_create: bad dtype");
     distdl_repartition *r = new distdl_repartition();
     r->rank = rank;
     r->dtype = dtype;

@@ -215,6 +215,75 @@ def test_halo_bf16_copies():
 
 
 # --------------------------------------------------------------------------
+# bfloat16 and fp64 variants of B, R, H, H*, all-reduce
+# --------------------------------------------------------------------------
+
+def _bits_dev(bits):
+    return dev(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+
+
+def _bits_host(t):
+    return host(t.view(torch.int16)).view(np.uint16)
+
+
+@pytest.mark.parametrize("n", [1, 7, 8, 1001, (1 << 20) + 3])
+@pytest.mark.parametrize("k", [1, 2, 3, 8, 19])
+def test_sumreduce_and_broadcast_bf16_fp64_bit_exact(n, k):
+    parts = [inputs.uniform_pm1((n,), 500 * k + i) * np.float32(10.0 ** (i % 5)) for i in range(k)]
+    # fp64
+    p64 = [p.astype(np.float64) * (1.0 + 2.0 ** -30 * (i + 1)) for i, p in enumerate(parts)]
+    dst = torch.empty(n, dtype=torch.float64, device=DEV)
+    distdl.sumreduce_fwd([dev(p) for p in p64], dst)
+    copies = [torch.empty(n, dtype=torch.float64, device=DEV) for _ in range(k)]
+    distdl.broadcast_fwd(dev(p64[0]), copies)
+    # bfloat16
+    pbf = [inputs.f32_to_bf16_bits(p) for p in parts]
+    dstb = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    distdl.sumreduce_fwd([_bits_dev(p) for p in pbf], dstb)
+    ar = [_bits_dev(p) for p in pbf]
+    distdl.allreduce(ar)
+    torch.cuda.synchronize()
+    assert same_bits(host(dst), oracle.sumreduce_fwd(p64))
+    assert all(same_bits(host(c), p64[0]) for c in copies)
+    refb = oracle.sumreduce_fwd(pbf, add=oracle.bf16_add)
+    assert same_bits(_bits_host(dstb), refb)
+    assert all(same_bits(_bits_host(t), refb) for t in ar)
+
+
+HALO_DTYPE_CASES = [HALO_CASES[i] for i in (0, 5, 7, 9, 10, 12, 14, 15)]
+
+
+@pytest.mark.parametrize("case", HALO_DTYPE_CASES, ids=[str(c[0]) + str(c[1]) for c in HALO_DTYPE_CASES])
+def test_halo_fwd_and_adj_bf16_fp64_bit_exact(case):
+    gshape, pshape, hlo, hhi = case
+    opart = oracle.Partition(gshape, pshape, hlo, hhi)
+    rank = len(gshape)
+    for code in (distdl.F64, distdl.BF16):
+        gpart = distdl.Partition(gshape, pshape, _w(hlo, rank), _w(hhi, rank), dtype=code)
+        x32, y32 = random_shards(opart, 21), []
+        for w in range(opart.num_workers):      # values of very different magnitude: the order of the sums shows in the bits
+            a = inputs.uniform_pm1(opart.padded_shape(w), 2200 + w)
+            y32.append((a * np.float32(10.0) ** inputs.integers(opart.padded_shape(w), 2300 + w, -3, 4)).astype(np.float32))
+        if code == distdl.F64:
+            x = [a.astype(np.float64) * (1.0 + 2.0 ** -33) for a in x32]
+            y = [a.astype(np.float64) * (1.0 + 2.0 ** -33) for a in y32]
+            xs, ys = [dev(a) for a in x], [dev(a) for a in y]
+            add, back = None, host
+        else:
+            x = [inputs.f32_to_bf16_bits(a) for a in x32]
+            y = [inputs.f32_to_bf16_bits(a) for a in y32]
+            xs, ys = [_bits_dev(a) for a in x], [_bits_dev(a) for a in y]
+            add, back = oracle.bf16_add, _bits_host
+        distdl.halo_fwd(gpart, xs)
+        distdl.halo_adj(gpart, ys)
+        torch.cuda.synchronize()
+        for a, b in zip(xs, oracle.halo_fwd_sequence(opart, x)):
+            assert same_bits(back(a), b)
+        for a, b in zip(ys, oracle.halo_adj_sequence(opart, y, add=add)):
+            assert same_bits(back(a), b)
+
+
+# --------------------------------------------------------------------------
 # Convolution layer
 # --------------------------------------------------------------------------
 

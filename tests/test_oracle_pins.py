@@ -813,3 +813,73 @@ def test_stencil3d_dot_test_and_zero_ghosts(case):
         mask = np.ones(part.padded_shape(wk), dtype=bool)
         mask[part.bulk_slices(wk)] = False
         assert not dx[wk][mask].any()
+
+
+# --------------------------------------------------------------------------
+# bfloat16 and fp64 arithmetic of the sums (R, H*, all-reduce)
+# --------------------------------------------------------------------------
+
+def test_bf16_rounding_against_library_conversion_and_ties():
+    import torch
+    rng = np.random.Generator(np.random.Philox(97))
+    vals = np.concatenate([
+        rng.standard_normal(20000).astype(np.float32),
+        (rng.standard_normal(2000) * 1e-39).astype(np.float32),          # bfloat16 subnormals
+        np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8), 0.0, -0.0, 2.0 ** -133, 1.5 * 2.0 ** -133,
+                  2.5 * 2.0 ** -133, 255.5, 256.5], dtype=np.float32)])
+    ref = torch.from_numpy(vals).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = oracle.round_to_bf16_bits(vals.astype(np.float64))
+    assert np.array_equal(got, ref)
+    assert got[22000:22003].tolist() == [0x3F80, 0x3F82, 0xBF80]           # ties go to the even mantissa
+    assert np.array_equal(oracle.bf16_bits_to_f64(got), oracle.bf16_bits_to_f64(ref))
+
+
+def test_bf16_add_is_the_exact_sum_rounded_once():
+    import torch
+    rng = np.random.Generator(np.random.Philox(98))
+    a = inputs.f32_to_bf16_bits((rng.standard_normal(50000) * 10.0 ** rng.integers(-6, 6, 50000)).astype(np.float32))
+    b = inputs.f32_to_bf16_bits((rng.standard_normal(50000) * 10.0 ** rng.integers(-6, 6, 50000)).astype(np.float32))
+    ta = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    tb = torch.from_numpy(b.view(np.int16)).view(torch.bfloat16)
+    ref = (ta + tb).view(torch.int16).numpy().view(np.uint16)              # library bfloat16 addition
+    assert np.array_equal(oracle.bf16_add(a, b), ref)
+    # brute force on a few pairs: the nearest bfloat16 to the exact rational sum
+    from fractions import Fraction
+    for i in range(40):
+        exact = Fraction(float(oracle.bf16_bits_to_f64(a[i:i + 1])[0])) + Fraction(float(oracle.bf16_bits_to_f64(b[i:i + 1])[0]))
+        got = int(oracle.bf16_add(a[i:i + 1], b[i:i + 1])[0])
+        gv = Fraction(float(oracle.bf16_bits_to_f64(np.array([got], np.uint16))[0]))
+        for nb in (got - 1, got + 1):                                      # neighbours in the bit pattern order
+            nv = Fraction(float(oracle.bf16_bits_to_f64(np.array([nb & 0xFFFF], np.uint16))[0]))
+            assert abs(gv - exact) <= abs(nv - exact)
+
+
+def test_sums_in_bf16_and_fp64_follow_the_fold_order():
+    import torch
+    k, n = 5, 3000
+    parts32 = [inputs.uniform_pm1((n,), 300 + i) for i in range(k)]
+    # bfloat16: left fold with library additions
+    bits = [inputs.f32_to_bf16_bits(p) for p in parts32]
+    acc = torch.from_numpy(bits[0].view(np.int16)).view(torch.bfloat16)
+    for b in bits[1:]:
+        acc = acc + torch.from_numpy(b.view(np.int16)).view(torch.bfloat16)
+    assert np.array_equal(oracle.sumreduce_fwd(bits, add=oracle.bf16_add), acc.view(torch.int16).numpy().view(np.uint16))
+    assert all(np.array_equal(o, oracle.sumreduce_fwd(bits, add=oracle.bf16_add)) for o in oracle.allreduce(bits, add=oracle.bf16_add))
+    # fp64: a plain Python left fold
+    parts64 = [p.astype(np.float64) * (1.0 + 2.0 ** -40 * i) for i, p in enumerate(parts32)]
+    ref = [float(parts64[0][e]) for e in range(n)]
+    for p in parts64[1:]:
+        ref = [r + float(p[e]) for e, r in enumerate(ref)]
+    assert oracle.sumreduce_fwd(parts64).tolist() == ref
+
+
+def test_halo_adjoint_in_bf16_and_fp64_on_integer_data():
+    # small integers: every sum is exact in all three types, so they must agree cell by cell
+    part = Partition((9, 10), (2, 3), 2, 1)
+    y32 = [inputs.integers(part.padded_shape(w), 400 + w) for w in range(part.num_workers)]
+    ref = oracle.halo_adj_sequence(part, y32)
+    got64 = oracle.halo_adj_sequence(part, [a.astype(np.float64) for a in y32])
+    gotbf = oracle.halo_adj_sequence(part, [inputs.f32_to_bf16_bits(a) for a in y32], add=oracle.bf16_add)
+    for a, b, c in zip(ref, got64, gotbf):
+        assert np.array_equal(a.astype(np.float64), b)
+        assert np.array_equal(a.astype(np.float64), oracle.bf16_bits_to_f64(c))
