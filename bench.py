@@ -563,13 +563,13 @@ def main():
 # capture ended) or that changed since its counters were taken.
 NCU_TRAFFIC = {
     "broadcast_fwd": None,
-    "sumreduce_fwd": 4 * (134223104 + 5289728),
-    "halo_fwd": 203052544 + 117629440,
-    "halo_adj": 262138112 + 167800064,
-    "conv_fwd": 4 * (277898496 + 221322496),
-    "conv_adj": 4 * (269446656 + 227919872),
-    "affine_fwd": 138432256 + 4193024,
-    "affine_adj": 138448640 + 4337152,
+    "sumreduce_fwd": 4 * (134224128 + 5519616),
+    "halo_fwd": 203430912 + 116587264,
+    "halo_adj": 261940992 + 166233344,
+    "conv_fwd": 4 * (277958400 + 220996352),
+    "conv_adj": 4 * (269584384 + 227286784),
+    "affine_fwd": 138450176 + 3624704,
+    "affine_adj": 138434816 + 3114240,
 }
 
 if __name__ == "__main__":
