@@ -1,6 +1,8 @@
 """GPU parity at the full sizes of the benchmark configurations, in the launch configuration that
-bench.py times.  B, R, H, H* and the affine layer are compared in full; the convolution on sampled
-(n, c) planes, which the oracle computes one by one."""
+bench.py times.  B, R, H, H*, the all-to-all and the affine layer are compared in full; the convolution
+and the pooling layer on sampled (n, c) planes, the star stencil on sampled boxes, the parameter gradients on
+sampled channels / worker blocks, which the oracle computes one by one; properties that hold at any size
+(zero ghosts, dot test) over everything."""
 
 import numpy as np
 import pytest
@@ -163,3 +165,130 @@ def test_pool_full_size_on_sampled_planes():
     total_dx = sum(float(t.double().sum()) for t in dxs)
     total_dy = sum(float(t.double().sum()) for t in dys)
     assert abs(total_dx - total_dy) <= 1e-6 * sum(float(t.double().abs().sum()) for t in dys)
+
+
+def test_stencil3d_full_size_on_sampled_boxes():
+    # the configuration bench.py times: 512^3 on 4 x 4 x 4 workers, radius 4
+    gs, ps, R = (512,) * 3, (4,) * 3, 4
+    gpart = distdl.Partition(gs, ps, (R,) * 3, (R,) * 3)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(11)
+    xs = [torch.randn(136, 136, 136, device=DEV, generator=g) for _ in range(64)]
+    dys = [torch.randn(128, 128, 128, device=DEV, generator=g) for _ in range(64)]
+    w = inputs.normal((3, 9), 7001, 0.5)
+    ys = [torch.empty(128, 128, 128, device=DEV) for _ in range(64)]
+    dxs = [torch.full((136, 136, 136), 7.0, device=DEV) for _ in range(64)]
+    distdl.stencil3d_fwd(gpart, xs, w, ys)
+    distdl.stencil3d_adj(gpart, dys, w, dxs)
+    torch.cuda.synchronize()
+
+    def gather(shards, off, lo, hi):
+        """Global box [lo, hi) put together from the bulks of the device shards (bulk offset `off` inside a shard)."""
+        out = np.zeros(tuple(b - a for a, b in zip(lo, hi)), dtype=np.float32)
+        for s in range(64):
+            c = (s // 16, (s // 4) % 4, s % 4)
+            a = [max(lo[k], 128 * c[k]) for k in range(3)]
+            b = [min(hi[k], 128 * c[k] + 128) for k in range(3)]
+            if any(a[k] >= b[k] for k in range(3)):
+                continue
+            src = tuple(slice(a[k] - 128 * c[k] + off, b[k] - 128 * c[k] + off) for k in range(3))
+            dst = tuple(slice(a[k] - lo[k], b[k] - lo[k]) for k in range(3))
+            out[dst] = host(shards[s][src])
+        return out
+
+    eps = (6 * R + 5) * 2.0 ** -24
+    # boxes at a corner of the tensor, where eight shards meet, across a face, and at the far corner
+    for lo in [(0, 0, 0), (120, 120, 120), (250, 380, 120), (492, 492, 492)]:
+        hi = tuple(v + 20 for v in lo)
+        elo = tuple(max(v - R, 0) for v in lo)
+        ehi = tuple(min(v + R, 512) for v in hi)
+        one = oracle.Partition(tuple(b - a for a, b in zip(elo, ehi)), (1, 1, 1), R, R)
+        inner = tuple(slice(l - e, l - e + 20) for l, e in zip(lo, elo))
+        for shards_in, off_in, got_shards, off_out, fn in ((xs, R, ys, 0, oracle.stencil3d_fwd), (dys, 0, dxs, R, oracle.stencil3d_adj)):
+            sub = gather(shards_in, off_in, elo, ehi)
+            if fn is oracle.stencil3d_fwd:
+                ref = fn(one, oracle.scatter_global(one, sub), w)[0][inner]
+                mag = fn(one, oracle.scatter_global(one, np.abs(sub)), np.abs(w))[0][inner]
+            else:
+                ref = fn(one, [sub], w)[0][one.bulk_slices(0)][inner]
+                mag = fn(one, [np.abs(sub)], np.abs(w))[0][one.bulk_slices(0)][inner]
+            # the extended box is cut R cells beyond the sampled one (or at the tensor's own boundary, where the
+            # oracle's zero padding is the right one), so the sampled cells see exactly their global neighbours
+            got = gather(got_shards, off_out, lo, hi)
+            assert np.all(np.abs(got.astype(np.float64) - ref) <= eps * mag + 1e-30)
+    # properties at full size: x untouched is checked in the small tests; ghosts of every dx shard are zero
+    for t in dxs:
+        assert float(t[:R].abs().max()) == 0.0 and float(t[-R:].abs().max()) == 0.0
+        assert float(t[:, :R].abs().max()) == 0.0 and float(t[:, -R:].abs().max()) == 0.0
+        assert float(t[:, :, :R].abs().max()) == 0.0 and float(t[:, :, -R:].abs().max()) == 0.0
+    # dot test over the whole volume, fp64 on the device (x's ghost storage does not take part)
+    lhs = sum(float((a.double() * b.double()).sum()) for a, b in zip(ys, dys))
+    rhs = sum(float((a[R:-R, R:-R, R:-R].double() * b[R:-R, R:-R, R:-R].double()).sum()) for a, b in zip(xs, dxs))
+    ny = sum(float((a.double() ** 2).sum()) for a in ys) ** 0.5
+    ndy = sum(float((a.double() ** 2).sum()) for a in dys) ** 0.5
+    assert abs(lhs - rhs) <= 1e-5 * ny * ndy
+
+
+def test_parameter_gradients_full_size():
+    # convolution: dw, db of two channels of the 16 x 16 x 1024 x 1024 case, each over all 16 batch entries
+    gs, ps = (16, 16, 1024, 1024), (1, 1, 4, 4)
+    gpart = distdl.Partition(gs, ps, (0, 0, 2, 2), (0, 0, 2, 2))
+    g = torch.Generator(device=DEV)
+    g.manual_seed(13)
+    xs = [torch.randn(16, 16, 260, 260, device=DEV, generator=g) for _ in range(16)]
+    dys = [torch.randn(16, 16, 256, 256, device=DEV, generator=g) for _ in range(16)]
+    dw, db = torch.empty(16, 5, 5, device=DEV), torch.empty(16, device=DEV)
+    ws = torch.empty(distdl.conv_adj_params_workspace(gpart, 5, 5), dtype=torch.uint8, device=DEV)
+    distdl.conv_adj_params(gpart, xs, dys, (5, 5), dw, db, ws)
+    distdl.device_status()
+    sub = (16, 1, 1024, 1024)
+    op = oracle.Partition(sub, ps, (0, 0, 2, 2), (0, 0, 2, 2))
+    for c in (0, 11):
+        x1 = [host(t[:, c:c + 1]) for t in xs]
+        dy1 = [host(t[:, c:c + 1]) for t in dys]
+        dw_ref, db_ref = oracle.conv_adj_params(op, x1, dy1, 5, 5)
+        # 16.8 M terms per tap; a running sum has 16 terms per tile of the channel (4096 tiles), then the folds
+        mag_w, mag_b = oracle.conv_adj_params(op, [np.abs(a) for a in oracle.halo_fwd_sequence(op, x1)],
+                                              [np.abs(a) for a in dy1], 5, 5)
+        eps = (16 * 4096 + 64) * 2.0 ** -24
+        assert np.all(np.abs(host(dw[c:c + 1]).astype(np.float64) - dw_ref) <= eps * mag_w)
+        assert np.all(np.abs(host(db[c:c + 1]).astype(np.float64) - db_ref) <= eps * mag_b)
+        assert np.linalg.norm(host(dw[c:c + 1]).astype(np.float64) - dw_ref) <= 1e-5 * np.linalg.norm(mag_w)
+    del xs, dys
+
+    # affine: dW blocks of three workers and every db of the 256 x 8192 x 8192 case
+    nb, nf, pf = 256, 8192, 4
+    blk = nf // pf
+    xb = inputs.f32_to_bf16_bits(inputs.normal((nb, nf), 6100))
+    dyb = inputs.f32_to_bf16_bits(inputs.normal((nb, nf), 6102))
+    bf = lambda a: dev(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+    xp, dyp = np.split(xb, pf, axis=1), np.split(dyb, pf, axis=1)
+    dW = [torch.empty(blk, blk, device=DEV) for _ in range(pf * pf)]
+    dB = [torch.empty(blk, device=DEV) for _ in range(pf)]
+    distdl.affine_adj_params(nb, nf, nf, pf, pf, [bf(a) for a in dyp], [bf(a) for a in xp], dW, dB)
+    distdl.device_status()
+    f64 = oracle.bf16_bits_to_f64
+    for i, j in ((0, 0), (2, 3), (3, 1)):
+        ref, dbref = oracle.affine_adj_params([f64(dyp[i])], [f64(xp[j])], 1, 1)
+        got = host(dW[i * pf + j]).astype(np.float64)
+        assert np.max(np.abs(got - ref[0])) / np.max(np.abs(ref[0])) < 1e-4
+        assert np.linalg.norm(got - ref[0]) / np.linalg.norm(ref[0]) < 1e-5
+        assert np.max(np.abs(host(dB[i]).astype(np.float64) - dbref[0])) <= 1e-5 * np.max(np.abs(dbref[0]))
+
+
+def test_repartition_full_size():
+    # the all-to-all bench.py times: fp32 8192 x 8192, 8 row blocks -> 8 column blocks and back
+    n = 8192
+    rep = distdl.Repartition((n, n), (8, 1), (1, 8))
+    rows = [inputs.uniform_pm1((n // 8, n), 8000 + i) for i in range(8)]
+    src = [dev(a) for a in rows]
+    dst = [torch.empty(n, n // 8, device=DEV) for _ in range(8)]
+    distdl.repartition_fwd(rep, src, dst)
+    back = [torch.empty(n // 8, n, device=DEV) for _ in range(8)]
+    distdl.repartition_adj(rep, dst, back)
+    torch.cuda.synchronize()
+    ref = oracle.repartition_fwd(oracle.Partition((n, n), (8, 1)), oracle.Partition((n, n), (1, 8)), rows)
+    for a, b in zip(dst, ref):
+        assert host(a).tobytes() == b.tobytes()
+    for a, b in zip(back, rows):
+        assert host(a).tobytes() == b.tobytes()

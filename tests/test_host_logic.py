@@ -136,3 +136,42 @@ def test_operator_argument_validation_without_a_device():
     assert lib.distdl_conv_fwd(p4.handle, arr, vp(0x50000), None, 3, 3, arr, None) == 2    # widths do not match 3x3
     assert lib.distdl_conv_fwd(p4.handle, arr, vp(0x50000), None, 4, 4, arr, None) == 4    # even kernel
     assert lib.distdl_last_error().decode() != ""
+
+
+def test_validation_of_the_gradient_stencil_and_dtype_entry_points():
+    lib = distdl.lib()
+    vp = ctypes.c_void_p
+    arr = (vp * 16)(*[0x10000 * (i + 1) for i in range(16)])
+    # affine parameter gradients
+    assert lib.distdl_affine_adj_params(16, 100, 128, 1, 1, arr, arr, arr, None, None) == 4   # block not a multiple of 128
+    assert lib.distdl_affine_adj_params(16, 256, 256, 3, 1, arr, arr, arr, None, None) == 2   # not divisible by the grid
+    assert lib.distdl_affine_adj_params(16, 256, 256, 1, 1, None, arr, arr, None, None) == 1  # NULL argument
+    odd = (vp * 1)(0x10004)
+    assert lib.distdl_affine_adj_params(16, 128, 128, 1, 1, odd, arr, arr, None, None) == 3   # alignment
+    # convolution parameter gradients: the geometry is checked before anything touches a device
+    p2 = distdl.Partition((8, 8), (2, 2), (1, 1), (1, 1))
+    p4 = distdl.Partition((1, 2, 16, 16), (1, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2))
+    n = ctypes.c_int64(0)
+    assert lib.distdl_conv_adj_params_workspace(p2.handle, 3, 3, ctypes.byref(n)) == 2          # not rank 4
+    assert lib.distdl_conv_adj_params_workspace(p4.handle, 3, 3, ctypes.byref(n)) == 2          # widths do not match 3x3
+    assert lib.distdl_conv_adj_params_workspace(p4.handle, 4, 4, ctypes.byref(n)) == 4          # even kernel
+    assert lib.distdl_conv_adj_params_workspace(p4.handle, 5, 5, None) == 1
+    assert lib.distdl_conv_adj_params(p4.handle, arr, arr, 5, 5, vp(0x50000), None, None, 0, None) == 1   # no workspace
+    # star stencil
+    taps = (ctypes.c_float * 27)(*([0.5] * 27))
+    p3 = distdl.Partition((8, 8, 8), (2, 1, 1), (2, 2, 2), (2, 2, 2))
+    assert lib.distdl_stencil3d_fwd(p2.handle, arr, taps, 1, arr, None) == 2                    # not rank 3
+    assert lib.distdl_stencil3d_fwd(p3.handle, arr, taps, 5, arr, None) == 4                    # radius beyond 4
+    assert lib.distdl_stencil3d_fwd(p3.handle, arr, taps, 1, arr, None) == 2                    # halo width is not the radius
+    assert lib.distdl_stencil3d_adj(p3.handle, arr, None, 2, arr, None) == 1
+    odd8 = (vp * 2)(0x10008, 0x20000)
+    assert lib.distdl_stencil3d_fwd(p3.handle, odd8, taps, 2, arr, None) == 3                   # alignment
+    with pytest.raises(ValueError):
+        distdl.stencil3d_fwd(p3, [], [[1.0, 2.0]] * 3, [])                                      # even tap count
+    # element types
+    assert lib.distdl_sumreduce_fwd(arr, vp(0x90000), 2, 8, 7, None) == 1                       # unknown dtype
+    assert lib.distdl_broadcast_fwd(vp(0x90000), arr, 2, 8, 7, None) == 1
+    p64 = distdl.Partition((9, 9), (2, 2), (1, 1), (1, 1), dtype=distdl.F64)
+    assert p64.halo_stats(False)[2] == 2 * distdl.Partition((9, 9), (2, 2), (1, 1), (1, 1)).halo_stats(False)[2]
+    r64 = distdl.Repartition((12, 8), (3, 1), (1, 2), distdl.F64)
+    assert r64.shard_shape(0) == (4, 8) and r64.shard_shape(1, destination=True) == (12, 4)
