@@ -10,16 +10,17 @@
 // the same star with every 1-D kernel reversed, evaluated in gather form on the bulk-shaped dy,
 // written into the bulk of the padded dx shards whose ghosts are cleared as H* leaves them.
 //
-// Blocking: a block owns 8 rows x 128 columns of one shard and marches through a chunk of planes.
-// A thread owns 4 consecutive columns of one row; the 2R+1 planes around the current one live in
-// its registers (z neighbours), the current plane with R extra rows above / below and R extra
-// columns left / right lives in shared memory (y and x neighbours; a star needs no corners).
-// The values of the next plane -- the thread's own cells R planes ahead, one vector of an extra
-// row, one cell of an extra column -- are fetched one step early, so their latency is covered by
-// the arithmetic of the current plane.  Two plane buffers, one barrier per plane.
+// Blocking: a block (four warps) owns 8 rows x 128 columns of one shard and marches through a chunk
+// of planes.  A thread owns 4 consecutive columns of two consecutive rows; the 2R+1 planes around the
+// current one live in its registers (z neighbours), the current plane with R extra rows above /
+// below and R extra columns left / right lives in shared memory (y and x neighbours; a star needs
+// no corners).  The two rows of a thread share their y neighbours: 2R + 2 plane rows, two of them its
+// own, serve both, which halves the shared-memory reads per output.  The values of the next plane --
+// the thread's own cells R planes ahead, its vectors of the extra rows, one cell of an extra column
+// -- are fetched one step early, so their latency is covered by the arithmetic of the current plane.
+// Two plane buffers, one barrier per plane.
 #include <algorithm>
 #include <cstring>
-#include <type_traits>
 
 #include "common.h"
 
@@ -28,9 +29,10 @@ namespace distdl {
 constexpr int kStMaxWorkers = 64;
 constexpr int kStMaxPerDim = 8;
 constexpr int kStMaxR = 4;
-constexpr int kStRows = 8;            // rows of a tile = warps of a block
+constexpr int kStRpt = 2;             // consecutive rows per thread
+constexpr int kStThreads = 128;
+constexpr int kStRows = kStRpt * (kStThreads / 32);   // rows of a tile: 8
 constexpr int kStCols = 128;          // columns of a tile = 32 lanes x 4
-constexpr int kStThreads = 256;
 constexpr int kStChunk = 64;          // planes a block marches through
 constexpr int kStLead = 4;            // shared-memory column of the tile's first column (keeps rows 16-byte aligned)
 constexpr int kStPitch = kStLead + kStCols + 4;   // 136 floats
@@ -66,21 +68,13 @@ __device__ __forceinline__ bool st_owner(const int32_t *b, int p, int s, int c, 
     return true;
 }
 
-// Calls f(phase PH, plane z + PH) for PH = 0 .. N-1 as long as the plane is below z1.
-template <int PH, int N, typename F>
-__device__ __forceinline__ void st_phases(F &f, int z, int z1) {
-    if constexpr (PH < N) {
-        if (z + PH < z1) {
-            f(std::integral_constant<int, PH>{}, z + PH);
-            st_phases<PH + 1, N>(f, z, z1);
-        }
-    }
-}
-
 template <int R, bool VEC>
-__global__ void __launch_bounds__(kStThreads, 2)
+__global__ void __launch_bounds__(kStThreads, 3)
 stencil3d_kernel(const __grid_constant__ StencilParams P) {
     __shared__ __align__(16) float plane[2][kStRows + 2 * R][kStPitch];
+    constexpr int N = 2 * R + 1;
+    constexpr int kWarps = kStThreads / 32;
+    constexpr int HR = (2 * R + kWarps - 1) / kWarps;     // extra rows a warp fetches per plane
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // block -> (shard, plane chunk, row tile, column tile), column tile fastest
     int rest = blockIdx.x;
@@ -99,8 +93,12 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
     const int io = P.in_off;
     const int ipx = bx + 2 * io;                       // input row pitch of every shard in this worker column
 
-    const int y = y0 + warp, x = x0 + 4 * lane;
-    const bool row_ok = y < by;
+    const int rw = kStRpt * warp;                      // first of this warp's rows inside the tile
+    const int x = x0 + 4 * lane;
+    const bool col_ok = x < bx;
+    bool row_ok[kStRpt];
+#pragma unroll
+    for (int r = 0; r < kStRpt; ++r) row_ok[r] = y0 + rw + r < by;
 
     // Everything that does not change from plane to plane is resolved once: for each kind of load a
     // base pointer (plane 0 of the owning shard, the thread's row and column; nullptr = zeros) and the
@@ -115,14 +113,13 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
     };
     const uint32_t ipy = (uint32_t)(by + 2 * io);
     const uint32_t own_stride = ipy * (uint32_t)ipx;                   // the same in the shards below and above
-    const bool own_ok = row_ok && x < bx;
-    const uint32_t own_off = (uint32_t)(y + io) * (uint32_t)ipx + (uint32_t)(x + io);
-    const float *own_mid = own_ok ? P.in[shard] + own_off : nullptr;
-    const float *own_lo = own_ok && sz > 0 ? P.in[shard - P.py * P.px] + own_off : nullptr;
-    const float *own_hi = own_ok && sz + 1 < P.pz ? P.in[shard + P.py * P.px] + own_off : nullptr;
+    const uint32_t own_off = (uint32_t)(y0 + rw + io) * (uint32_t)ipx + (uint32_t)(x + io);   // row 0 of the thread
+    const float *own_mid = col_ok ? P.in[shard] + own_off : nullptr;
+    const float *own_lo = col_ok && sz > 0 ? P.in[shard - P.py * P.px] + own_off : nullptr;
+    const float *own_hi = col_ok && sz + 1 < P.pz ? P.in[shard + P.py * P.px] + own_off : nullptr;
     const int bz_lo = sz > 0 ? P.bz[sz - 1] : 0, bz_hi = sz + 1 < P.pz ? P.bz[sz + 1] : 0;
-    // this thread's four cells of plane zp (any plane within R of the chunk), zeros outside the tensor
-    auto load_own = [&](int zp) -> float4 {
+    // this thread's cells of plane zp (any plane within R of the chunk), zeros outside the tensor
+    auto load_own = [&](int zp, float4 (&v)[kStRpt]) {
         const float *base = own_mid;
         if (zp < 0) {
             base = own_lo;
@@ -133,24 +130,33 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
             zp -= bz;
             if (zp >= bz_hi) base = nullptr;
         }
-        if (!base) return make_float4(0.f, 0.f, 0.f, 0.f);
-        return load4(base + (uint32_t)(zp + io) * own_stride);
+#pragma unroll
+        for (int r = 0; r < kStRpt; ++r) {
+            v[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (base && row_ok[r]) v[r] = load4(base + (uint32_t)(zp + io) * own_stride + (uint32_t)(r * ipx));
+        }
     };
-    // warps 0 .. 2R-1: this thread's four cells of one extra row of plane zp (a plane of the chunk itself)
-    const int hrow_y = warp < R ? y0 - R + warp : y0 + th + (warp - R);
-    const int hrow_s = warp < R ? warp : R + th + (warp - R);           // its row in the shared-memory plane
-    const float *hrow_base = nullptr;
-    uint32_t hrow_stride = 0;
-    {
+    // extra rows of the current plane: row h of the 2R (R above the tile, R below) goes to warp h % kWarps
+    const float *hrow_base[HR];
+    uint32_t hrow_stride[HR];
+    int hrow_s[HR];
+#pragma unroll
+    for (int i = 0; i < HR; ++i) {
+        const int h = warp + kWarps * i;
+        hrow_base[i] = nullptr;
+        hrow_stride[i] = 0;
+        hrow_s[i] = h < R ? h : R + th + (h - R);                      // its row in the shared-memory plane
+        const int hy = h < R ? y0 - R + h : y0 + th + (h - R);
         int so, yo;
-        if (warp < 2 * R && x < bx && st_owner(P.by, P.py, sy, hrow_y, so, yo)) {
-            hrow_stride = (uint32_t)(P.by[so] + 2 * io) * (uint32_t)ipx;
-            hrow_base = P.in[(sz * P.py + so) * P.px + sx] + (uint32_t)(yo + io) * (uint32_t)ipx + (uint32_t)(x + io);
+        if (h < 2 * R && col_ok && st_owner(P.by, P.py, sy, hy, so, yo)) {
+            hrow_stride[i] = (uint32_t)(P.by[so] + 2 * io) * (uint32_t)ipx;
+            hrow_base[i] = P.in[(sz * P.py + so) * P.px + sx] + (uint32_t)(yo + io) * (uint32_t)ipx + (uint32_t)(x + io);
         }
     }
-    auto load_hrow = [&](int zp) -> float4 {
-        if (!hrow_base) return make_float4(0.f, 0.f, 0.f, 0.f);
-        return load4(hrow_base + (uint32_t)(zp + io) * hrow_stride);
+    auto load_hrow = [&](int zp, float4 (&v)[HR]) {
+#pragma unroll
+        for (int i = 0; i < HR; ++i)
+            v[i] = hrow_base[i] ? load4(hrow_base[i] + (uint32_t)(zp + io) * hrow_stride[i]) : make_float4(0.f, 0.f, 0.f, 0.f);
     };
     // threads 0 .. 8 * 2R - 1: one cell of an extra column of plane zp
     const int hc_row = threadIdx.x / (2 * R), hc_c = threadIdx.x % (2 * R);
@@ -171,140 +177,168 @@ stencil3d_kernel(const __grid_constant__ StencilParams P) {
         return hcol_base ? __ldg(hcol_base + (uint32_t)(zp + io) * hcol_stride) : 0.f;
     };
 
-    // prime: planes z0 - R .. z0 + R, extra row / column of plane z0
-    float4 q[2 * R + 1];
+    // prime: planes z0 - R .. z0 + R, extra rows / column of plane z0
+    float4 q[N][kStRpt];
 #pragma unroll
-    for (int i = 0; i <= 2 * R; ++i) q[i] = load_own(z0 - R + i);
-    float4 hrow = load_hrow(z0);
+    for (int i = 0; i < N; ++i) load_own(z0 - R + i, q[i]);
+    float4 hrow[HR];
+    load_hrow(z0, hrow);
     float hcol = load_hcol(z0);
 
     const int oo = P.out_off;
     const int opy = by + 2 * oo, opx = bx + 2 * oo;
-    float *optr = P.out[shard] + ((size_t)(z0 + oo) * opy + (size_t)(y + oo)) * opx + (x + oo);
+    float *optr = P.out[shard] + ((size_t)(z0 + oo) * opy + (size_t)(y0 + rw + oo)) * opx + (x + oo);
     const size_t oplane = (size_t)opy * opx;
     const bool clear_x = P.clear_ghosts && oo > 0;
 
-    // One plane.  The 2R+1 planes of the queue are not shifted: in phase PH the plane at offset j
-    // (0 = R planes behind the current one) sits in q[(PH + j) % N], and the slot of the oldest plane
-    // takes the newly fetched one, which makes it offset 2R of phase PH + 1.
-    constexpr int N = 2 * R + 1;
-    auto step = [&](auto phase, int z) {
-        constexpr int PH = decltype(phase)::value;
-        const float4 ctr = q[(PH + R) % N];
-        float(*pl)[kStPitch] = plane[(z - z0) & 1];
-        // current plane into shared memory: own cells, one extra-row vector, one extra-column cell.
-        // Cells beyond the bulk are written by the extra-row / extra-column threads only.
-        if (row_ok) {
-            if (VEC) {
-                if (x < bx) *reinterpret_cast<float4 *>(&pl[R + warp][kStLead + 4 * lane]) = ctr;
-            } else {
-                float *d = &pl[R + warp][kStLead + 4 * lane];
-                if (x < bx) d[0] = ctr.x;
-                if (x + 1 < bx) d[1] = ctr.y;
-                if (x + 2 < bx) d[2] = ctr.z;
-                if (x + 3 < bx) d[3] = ctr.w;
-            }
+    auto put4 = [&](float *d, const float4 &v) {      // own / extra-row cells into the shared-memory plane
+        if (VEC) {
+            *reinterpret_cast<float4 *>(d) = v;
+        } else {
+            d[0] = v.x;
+            if (x + 1 < bx) d[1] = v.y;
+            if (x + 2 < bx) d[2] = v.z;
+            if (x + 3 < bx) d[3] = v.w;
         }
-        if (warp < 2 * R) {
-            if (VEC) {
-                if (x < bx) *reinterpret_cast<float4 *>(&pl[hrow_s][kStLead + 4 * lane]) = hrow;
-            } else {
-                float *d = &pl[hrow_s][kStLead + 4 * lane];
-                if (x < bx) d[0] = hrow.x;
-                if (x + 1 < bx) d[1] = hrow.y;
-                if (x + 2 < bx) d[2] = hrow.z;
-                if (x + 3 < bx) d[3] = hrow.w;
-            }
+    };
+
+    // One plane per turn; q[j] is the plane j - R away from the current one.  The queue is shifted by
+    // register moves at the end of a turn: rotating it at compile time instead needs 2R+1 copies of the
+    // loop body, which no longer fit the instruction cache (measured: 13 % slower).
+    for (int z = z0; z < z1; ++z) {
+        float(*pl)[kStPitch] = plane[(z - z0) & 1];
+        // current plane into shared memory: own cells, the extra-row vectors, one extra-column cell.
+        // Cells beyond the bulk are written by the extra-row / extra-column threads only.
+        if (col_ok) {
+#pragma unroll
+            for (int r = 0; r < kStRpt; ++r)
+                if (row_ok[r]) put4(&pl[R + rw + r][kStLead + 4 * lane], q[R][r]);
+#pragma unroll
+            for (int i = 0; i < HR; ++i)
+                if (warp + kWarps * i < 2 * R) put4(&pl[hrow_s[i]][kStLead + 4 * lane], hrow[i]);
         }
         if (hc_active) pl[R + hc_row][hc_s] = hcol;
         // next plane's values, one step early
-        float4 lead = make_float4(0.f, 0.f, 0.f, 0.f), hrow_n = lead;
+        float4 lead[kStRpt], hrow_n[HR];
         float hcol_n = 0.f;
         if (z + 1 < z1) {
-            lead = load_own(z + 1 + R);
-            hrow_n = load_hrow(z + 1);
+            load_own(z + 1 + R, lead);
+            load_hrow(z + 1, hrow_n);
             hcol_n = load_hcol(z + 1);
+        } else {
+#pragma unroll
+            for (int r = 0; r < kStRpt; ++r) lead[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < HR; ++i) hrow_n[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         __syncthreads();
 
-        if (row_ok && x < bx) {
-            float o[4] = {0.f, 0.f, 0.f, 0.f};
+        if (col_ok && row_ok[0]) {
+            float o[kStRpt][4];
+#pragma unroll
+            for (int r = 0; r < kStRpt; ++r)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[r][e] = 0.f;
             // z neighbours: registers
 #pragma unroll
-            for (int k = 0; k <= 2 * R; ++k) {
+            for (int k = 0; k < N; ++k) {
                 const float wz = P.w[0][k];
-                const float4 v = q[(PH + k) % N];
-                o[0] = fmaf(wz, v.x, o[0]);
-                o[1] = fmaf(wz, v.y, o[1]);
-                o[2] = fmaf(wz, v.z, o[2]);
-                o[3] = fmaf(wz, v.w, o[3]);
-            }
-            // y neighbours: the rows above and below in shared memory
 #pragma unroll
-            for (int k = 0; k <= 2 * R; ++k) {
+                for (int r = 0; r < kStRpt; ++r) {
+                    const float4 v = q[k][r];
+                    o[r][0] = fmaf(wz, v.x, o[r][0]);
+                    o[r][1] = fmaf(wz, v.y, o[r][1]);
+                    o[r][2] = fmaf(wz, v.z, o[r][2]);
+                    o[r][3] = fmaf(wz, v.w, o[r][3]);
+                }
+            }
+            // y neighbours: the rows rw .. rw + 2R + RPT - 1 of the plane, each read once and used by every
+            // row of the thread it is a neighbour of (tap k of row r is plane row rw + r + k)
+#pragma unroll
+            for (int j = 0; j < N + kStRpt - 1; ++j) {
                 float4 v;
-                if (k == R) v = ctr;
-                else if (VEC) v = *reinterpret_cast<const float4 *>(&pl[warp + k][kStLead + 4 * lane]);
+                // the thread's own rows come from its registers -- unless such a row lies beyond the bulk (a ragged
+                // last tile): then that plane row holds an extra row fetched from the shard below
+                const bool own = j >= R && j < R + kStRpt && row_ok[j >= R && j < R + kStRpt ? j - R : 0];
+                if (own) v = q[R][j >= R && j < R + kStRpt ? j - R : 0];
+                else if (VEC) v = *reinterpret_cast<const float4 *>(&pl[rw + j][kStLead + 4 * lane]);
                 else {
-                    const float *s = &pl[warp + k][kStLead + 4 * lane];
+                    const float *s = &pl[rw + j][kStLead + 4 * lane];
                     v = make_float4(s[0], s[1], s[2], s[3]);
                 }
-                const float wy = P.w[1][k];
-                o[0] = fmaf(wy, v.x, o[0]);
-                o[1] = fmaf(wy, v.y, o[1]);
-                o[2] = fmaf(wy, v.z, o[2]);
-                o[3] = fmaf(wy, v.w, o[3]);
+#pragma unroll
+                for (int r = 0; r < kStRpt; ++r) {
+                    const int k = j - r;
+                    if (k < 0 || k >= N) continue;
+                    const float wy = P.w[1][k];
+                    o[r][0] = fmaf(wy, v.x, o[r][0]);
+                    o[r][1] = fmaf(wy, v.y, o[r][1]);
+                    o[r][2] = fmaf(wy, v.z, o[r][2]);
+                    o[r][3] = fmaf(wy, v.w, o[r][3]);
+                }
             }
             // x neighbours: the vectors left and right of the own one
-            float xs[12];
-            {
-                const float4 l = *reinterpret_cast<const float4 *>(&pl[R + warp][4 * lane]);
-                const float4 r = *reinterpret_cast<const float4 *>(&pl[R + warp][4 * lane + 8]);
+#pragma unroll
+            for (int r = 0; r < kStRpt; ++r) {
+                float xs[12];
+                const float4 l = *reinterpret_cast<const float4 *>(&pl[R + rw + r][4 * lane]);
+                const float4 rt = *reinterpret_cast<const float4 *>(&pl[R + rw + r][4 * lane + 8]);
                 xs[0] = l.x; xs[1] = l.y; xs[2] = l.z; xs[3] = l.w;
                 if (VEC) {
-                    xs[4] = ctr.x; xs[5] = ctr.y; xs[6] = ctr.z; xs[7] = ctr.w;
+                    const float4 c = q[R][r];
+                    xs[4] = c.x; xs[5] = c.y; xs[6] = c.z; xs[7] = c.w;
                 } else {
                     // a ragged last vector: its cells beyond the bulk are extra-column cells, not the thread's own
-                    const float4 c = *reinterpret_cast<const float4 *>(&pl[R + warp][kStLead + 4 * lane]);
+                    const float4 c = *reinterpret_cast<const float4 *>(&pl[R + rw + r][kStLead + 4 * lane]);
                     xs[4] = c.x; xs[5] = c.y; xs[6] = c.z; xs[7] = c.w;
                 }
-                xs[8] = r.x; xs[9] = r.y; xs[10] = r.z; xs[11] = r.w;
-            }
+                xs[8] = rt.x; xs[9] = rt.y; xs[10] = rt.z; xs[11] = rt.w;
 #pragma unroll
-            for (int k = 0; k <= 2 * R; ++k) {
-                const float wx = P.w[2][k];
+                for (int k = 0; k < N; ++k) {
+                    const float wx = P.w[2][k];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) o[e] = fmaf(wx, xs[4 + e + k - R], o[e]);
-            }
-            if (VEC) {
-                *reinterpret_cast<float4 *>(optr) = make_float4(o[0], o[1], o[2], o[3]);
-            } else {
-                optr[0] = o[0];
-                if (x + 1 < bx) optr[1] = o[1];
-                if (x + 2 < bx) optr[2] = o[2];
-                if (x + 3 < bx) optr[3] = o[3];
-            }
-            // adjoint: the ghost columns beside this row are cleared by the threads that write the row's
-            // ends, so that they land in the same lines of memory as the row itself
-            if (clear_x) {
-                if (x == 0) {
-                    if (VEC && R == 4) *reinterpret_cast<float4 *>(optr - 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-                    else
-                        for (int c = 1; c <= oo; ++c) optr[-c] = 0.f;
+                    for (int e = 0; e < 4; ++e) o[r][e] = fmaf(wx, xs[4 + e + k - R], o[r][e]);
                 }
-                if (x + 4 >= bx) {
-                    if (VEC && R == 4) *reinterpret_cast<float4 *>(optr + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-                    else
-                        for (int c = 0; c < oo; ++c) optr[bx - x + c] = 0.f;
+            }
+#pragma unroll
+            for (int r = 0; r < kStRpt; ++r) {
+                if (!row_ok[r]) continue;
+                float *op = optr + (size_t)r * opx;
+                if (VEC) {
+                    *reinterpret_cast<float4 *>(op) = make_float4(o[r][0], o[r][1], o[r][2], o[r][3]);
+                } else {
+                    op[0] = o[r][0];
+                    if (x + 1 < bx) op[1] = o[r][1];
+                    if (x + 2 < bx) op[2] = o[r][2];
+                    if (x + 3 < bx) op[3] = o[r][3];
+                }
+                // adjoint: the ghost columns beside this row are cleared by the threads that write the row's
+                // ends, so that they land in the same lines of memory as the row itself
+                if (clear_x) {
+                    if (x == 0) {
+                        if (VEC && R == 4) *reinterpret_cast<float4 *>(op - 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+                        else
+                            for (int c = 1; c <= oo; ++c) op[-c] = 0.f;
+                    }
+                    if (x + 4 >= bx) {
+                        if (VEC && R == 4) *reinterpret_cast<float4 *>(op + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+                        else
+                            for (int c = 0; c < oo; ++c) op[bx - x + c] = 0.f;
+                    }
                 }
             }
         }
         optr += oplane;
-        q[PH % N] = lead;
-        hrow = hrow_n;
+#pragma unroll
+        for (int i = 0; i + 1 < N; ++i)
+#pragma unroll
+            for (int r = 0; r < kStRpt; ++r) q[i][r] = q[i + 1][r];
+#pragma unroll
+        for (int r = 0; r < kStRpt; ++r) q[N - 1][r] = lead[r];
+#pragma unroll
+        for (int i = 0; i < HR; ++i) hrow[i] = hrow_n[i];
         hcol = hcol_n;
-    };
-    for (int z = z0; z < z1; z += N) st_phases<0, N>(step, z, z1);
+    }
 
     if (P.clear_ghosts && oo > 0) {
         // this block's part of the ghost shell of the output shard: its box of bulk cells, extended
