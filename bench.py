@@ -100,6 +100,8 @@ class Workload:
         d = distdl
         el = self.b_src.numel() * 4
         conv_bytes = conv_algorithmic_bytes(self.cpart)
+        # the adjoint also clears the ghost cells of the padded dx shards (as H* does): one more write per ghost cell
+        conv_ghost_bytes = 4 * sum(a.numel() - b.numel() for a, b in zip(self.c_dx, self.c_dy))
         aff_flops = 2 * self.nb * self.nf * self.nf
         aff_bytes = self.nf * self.nf * 2 + self.nb * self.nf * 2 + self.nb * self.nf * 4
         # name, call, algorithmic bytes, flops, kernel launches, bound
@@ -110,7 +112,7 @@ class Workload:
             ("halo_adj", lambda: d.halo_adj(self.hpart, self.h_y), self.hpart.halo_stats(True)[2], 0, 1, "hbm"),
             ("conv_fwd", lambda: d.conv_fwd(self.cpart, self.c_x, self.c_w, None, self.c_y), conv_bytes,
              2 * 25 * self._conv_outputs(), 1, "hbm"),
-            ("conv_adj", lambda: d.conv_adj(self.cpart, self.c_dy, self.c_w, self.c_dx), conv_bytes,
+            ("conv_adj", lambda: d.conv_adj(self.cpart, self.c_dy, self.c_w, self.c_dx), conv_bytes + conv_ghost_bytes,
              2 * 25 * self._conv_outputs(), 1, "hbm"),
             ("affine_fwd", lambda: d.affine_fwd(self.nb, self.nf, self.nf, self.pf, self.pf, self.a_x, self.a_w,
                                                 None, self.a_y), aff_bytes, aff_flops, 1, "tensor"),

@@ -82,6 +82,18 @@ distdl_status_t distdl_partition_create_general(int32_t rank, const int64_t *glo
                                                 const int32_t *const *halo_lo,
                                                 const int32_t *const *halo_hi,
                                                 distdl_dtype_t dtype, distdl_partition_t **out);
+/* The same as distdl_partition_create with periodic[k] != 0 marking dimensions that wrap around: the
+ * first and the last worker along such a dimension are neighbours (a worker alone along it is its own
+ * neighbour), and the ghosts on that boundary of the tensor receive the cells from the other end
+ * instead of zeros; H* adds them back there.  The paper's exchange stops at the tensor's boundary;
+ * this is the same operator sequence with one more pair of neighbours per periodic dimension.
+ * periodic == NULL: no dimension is periodic.  The fused layers (conv, pool, stencil3d) do not take
+ * periodic partitions (DISTDL_ERR_UNSUPPORTED). */
+distdl_status_t distdl_partition_create_periodic(int32_t rank, const int64_t *global_shape,
+                                                 const int32_t *partition_shape,
+                                                 const int32_t *halo_lo, const int32_t *halo_hi,
+                                                 const int32_t *periodic, distdl_dtype_t dtype,
+                                                 distdl_partition_t **out);
 void distdl_partition_destroy(distdl_partition_t *p); /* NULL is allowed */
 int32_t distdl_partition_num_workers(const distdl_partition_t *p); /* -1 if p is NULL */
 

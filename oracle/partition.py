@@ -79,17 +79,24 @@ class Partition:
                      dimension k is c (Section 3: every side of every dimension
                      may have its own thickness).  An int, or a per-dimension
                      int, means "the same width for every worker".
+    periodic[k]      True: dimension k wraps around (not in the paper, whose
+                     exchange stops at the tensor's boundary; the same operator
+                     sequence with the first and last worker as neighbours).
 
     Worker ids are the row-major index of the partition coordinate, last
     dimension fastest (Appendix B.2: in a 2 x 2 partition workers 0,1 are the
     top row and 2,3 the bottom row).
     """
 
-    def __init__(self, global_shape, pshape, hlo=0, hhi=0):
+    def __init__(self, global_shape, pshape, hlo=0, hhi=0, periodic=None):
         self.global_shape = tuple(int(v) for v in global_shape)
         self.pshape = tuple(int(v) for v in pshape)
         self.rank = len(self.global_shape)
         assert len(self.pshape) == self.rank
+        # periodic[k]: dimension k wraps around (the first and the last worker are neighbours, and the
+        # ghosts on the tensor's boundary hold the cells from the other end instead of zeros)
+        self.periodic = tuple(bool(v) for v in periodic) if periodic is not None else (False,) * self.rank
+        assert len(self.periodic) == self.rank
         self.start, self.size = [], []
         for k in range(self.rank):
             s, z = balanced_split(self.global_shape[k], self.pshape[k])

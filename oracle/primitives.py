@@ -130,20 +130,27 @@ def halo_fwd_definition(part: Partition, shards):
     g = assemble_global(part, shards)
     out = []
     for w in range(part.num_workers):
-        a = np.zeros(part.padded_shape(w), dtype=shards[w].dtype)
         st = part.bulk_start(w)
         lo, _ = part.widths(w)
         pshape = part.padded_shape(w)
-        # global index of padded-local index l is st - lo + l
-        src, dst = [], []
+        # global index of padded-local index l is st - lo + l; taken modulo the extent in a periodic
+        # dimension, otherwise cells outside the tensor stay zero
+        a = g
+        keep = []
         for k in range(part.rank):
-            g0 = st[k] - lo[k]
-            g1 = g0 + pshape[k]
-            c0 = max(g0, 0)
-            c1 = min(g1, part.global_shape[k])
-            src.append(slice(c0, max(c0, c1)))
-            dst.append(slice(c0 - g0, max(c0, c1) - g0))
-        a[tuple(dst)] = g[tuple(src)]
+            idx = np.arange(st[k] - lo[k], st[k] - lo[k] + pshape[k])
+            n = part.global_shape[k]
+            if part.periodic[k]:
+                keep.append(np.ones(pshape[k], dtype=bool))
+                idx = idx % n
+            else:
+                keep.append((idx >= 0) & (idx < n))
+                idx = np.clip(idx, 0, n - 1)
+            a = np.take(a, idx, axis=k)
+        mask = keep[0]
+        for k in range(1, part.rank):
+            mask = np.multiply.outer(mask, keep[k])
+        a = np.where(mask, a, np.zeros((), dtype=a.dtype)).astype(shards[w].dtype)
         a[part.bulk_slices(w)] = shards[w][part.bulk_slices(w)]
         out.append(a)
     return out
@@ -170,7 +177,9 @@ def _neighbour(part, w, k, step):
     c = list(part.coords(w))
     c[k] += step
     if c[k] < 0 or c[k] >= part.pshape[k]:
-        return None
+        if not part.periodic[k]:
+            return None
+        c[k] %= part.pshape[k]           # across the seam; the worker itself when it is alone along k
     return part.worker(c)
 
 

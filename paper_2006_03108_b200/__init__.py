@@ -51,6 +51,7 @@ def lib():
     L.distdl_last_error.argtypes = []
     L.distdl_partition_create.argtypes = [c_i32, pi64, pi32, pi32, pi32, c_i32, pvp]
     L.distdl_partition_create_general.argtypes = [c_i32, pi64, pi32, ppi32, ppi32, c_i32, pvp]
+    L.distdl_partition_create_periodic.argtypes = [c_i32, pi64, pi32, pi32, pi32, pi32, c_i32, pvp]
     L.distdl_partition_destroy.argtypes = [vp]
     L.distdl_partition_destroy.restype = None
     L.distdl_partition_num_workers.argtypes = [vp]
@@ -131,7 +132,7 @@ def _dtype_code(t):
 class Partition:
     """Handle of a distdl_partition_t (see distdl_partition_create in include/distdl.h)."""
 
-    def __init__(self, global_shape, partition_shape, halo_lo=None, halo_hi=None, dtype=F32):
+    def __init__(self, global_shape, partition_shape, halo_lo=None, halo_hi=None, dtype=F32, periodic=None):
         L = lib()
         rank = len(global_shape)
         if len(partition_shape) != rank:
@@ -146,7 +147,14 @@ class Partition:
         def general(h):
             return h is not None and any(isinstance(v, (list, tuple)) for v in h)
 
-        if general(halo_lo) or general(halo_hi):
+        if periodic is not None and any(periodic):
+            if general(halo_lo) or general(halo_hi):
+                raise ValueError("periodic partitions take one halo width per side and dimension")
+            lo = None if halo_lo is None else (ctypes.c_int32 * rank)(*[int(v) for v in halo_lo])
+            hi = None if halo_hi is None else (ctypes.c_int32 * rank)(*[int(v) for v in halo_hi])
+            per = (ctypes.c_int32 * rank)(*[1 if v else 0 for v in periodic])
+            _check(L.distdl_partition_create_periodic(rank, gs, ps, lo, hi, per, dtype, ctypes.byref(self._h)))
+        elif general(halo_lo) or general(halo_hi):
             keep = []
 
             def rows(h):

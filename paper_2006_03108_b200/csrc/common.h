@@ -101,6 +101,12 @@ struct distdl_partition {
     int device = 0;
     int64_t global_shape[DISTDL_MAX_RANK] = {0};
     int32_t pshape[DISTDL_MAX_RANK] = {0};
+    bool periodic[DISTDL_MAX_RANK] = {false, false, false, false, false};   // dimension wraps around
+    bool any_periodic() const {
+        for (int k = 0; k < rank; ++k)
+            if (periodic[k]) return true;
+        return false;
+    }
     // per dimension, per worker coordinate along that dimension
     std::vector<int64_t> start[DISTDL_MAX_RANK];
     std::vector<int64_t> size[DISTDL_MAX_RANK];

@@ -766,6 +766,7 @@ static distdl_status_t conv_impl(const distdl_partition *p, const void *const *i
     clear_error();
     if (!p || !in || !w || !out) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
     if (p->rank != 4 || p->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-4 F32 partition", what);
+    if (p->any_periodic()) return fail(DISTDL_ERR_UNSUPPORTED, "%s: periodic partitions are not supported by the fused layers", what);
     if (p->pshape[0] != 1 || p->pshape[1] != 1)
         return fail(DISTDL_ERR_UNSUPPORTED, "%s: only the feature-space dimensions may be partitioned", what);
     if (kh != kw || (kh != 3 && kh != 5 && kh != 7))
@@ -1236,6 +1237,7 @@ static distdl_status_t grad_plan(const distdl_partition *p, int32_t kh, int32_t 
                                  int *grid) {
     if (!p) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL partition", what);
     if (p->rank != 4 || p->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-4 F32 partition", what);
+    if (p->any_periodic()) return fail(DISTDL_ERR_UNSUPPORTED, "%s: periodic partitions are not supported by the fused layers", what);
     if (p->pshape[0] != 1 || p->pshape[1] != 1)
         return fail(DISTDL_ERR_UNSUPPORTED, "%s: only the feature-space dimensions may be partitioned", what);
     if (kh != kw || (kh != 3 && kh != 5 && kh != 7))

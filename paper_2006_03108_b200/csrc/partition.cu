@@ -55,7 +55,7 @@ distdl_status_t distdl::upload_plan_pair(const HaloPlanHost &a, const HaloPlanHo
 static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
                                    const int32_t *const *hlo, const int32_t *const *hhi,
                                    const int32_t *ulo, const int32_t *uhi, distdl_dtype_t dtype,
-                                   distdl_partition_t **out, bool upload = true) {
+                                   distdl_partition_t **out, bool upload = true, const int32_t *periodic = nullptr) {
     clear_error();
     if (!out) return fail(DISTDL_ERR_INVALID_ARG, "partition_create: out is NULL");
     if (rank < 1 || rank > DISTDL_MAX_RANK)
@@ -79,6 +79,7 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
     for (int k = 0; k < rank; ++k) {
         p->global_shape[k] = global_shape[k];
         p->pshape[k] = partition_shape[k];
+        p->periodic[k] = periodic && periodic[k] != 0;
         const int32_t pk = partition_shape[k];
         const int64_t q = global_shape[k] / pk, r = global_shape[k] % pk;
         int64_t at = 0;
@@ -96,7 +97,12 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
             p->hlo[k].push_back(lo);
             p->hhi[k].push_back(hi);
         }
-        // a ghost may only hold cells of the directly adjacent worker
+        // a ghost may only hold cells of the directly adjacent worker (around the seam too, when the
+        // dimension is periodic)
+        if (p->periodic[k] && (p->hlo[k][0] > p->size[k][pk - 1] || p->hhi[k][pk - 1] > p->size[k][0])) {
+            delete p;
+            return fail(DISTDL_ERR_SHAPE, "partition_create: a halo across the periodic seam of dimension %d is wider than its neighbour's bulk", k);
+        }
         for (int32_t c = 0; c < pk; ++c) {
             if (c > 0 && p->hlo[k][c] > p->size[k][c - 1]) {
                 delete p;
@@ -147,6 +153,13 @@ extern "C" distdl_status_t distdl_partition_create_general(int32_t rank, const i
     static const int32_t *const none[DISTDL_MAX_RANK] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     return create_impl(rank, global_shape, partition_shape, halo_lo ? halo_lo : none, halo_hi ? halo_hi : none,
                        nullptr, nullptr, dtype, out);
+}
+
+extern "C" distdl_status_t distdl_partition_create_periodic(int32_t rank, const int64_t *global_shape,
+                                                            const int32_t *partition_shape, const int32_t *halo_lo,
+                                                            const int32_t *halo_hi, const int32_t *periodic,
+                                                            distdl_dtype_t dtype, distdl_partition_t **out) {
+    return create_impl(rank, global_shape, partition_shape, nullptr, nullptr, halo_lo, halo_hi, dtype, out, true, periodic);
 }
 
 namespace distdl {

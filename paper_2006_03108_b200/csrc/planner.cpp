@@ -319,7 +319,7 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
             for (int k = 0; k < d; ++k) {
                 if (delta[k] != 0) centre = false;
                 const int32_t nc = c[k] + delta[k];
-                if (nc < 0 || nc >= p->pshape[k]) has_neighbour = false;
+                if ((nc < 0 || nc >= p->pshape[k]) && !p->periodic[k]) has_neighbour = false;
             }
             if (centre) continue;
             Region dst;
@@ -329,7 +329,9 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
                 const int64_t hl = p->hlo[k][c[k]], b = p->size[k][c[k]], hh = p->hhi[k][c[k]];
                 dst.start[k] = delta[k] < 0 ? 0 : (delta[k] == 0 ? hl : hl + b);
                 dst.extent[k] = delta[k] < 0 ? hl : (delta[k] == 0 ? b : hh);
-                nc[k] = c[k] + delta[k];
+                // a periodic dimension wraps around: the neighbour across the seam (the worker itself when
+                // it is alone along that dimension)
+                nc[k] = (c[k] + delta[k] + p->pshape[k]) % p->pshape[k];
             }
             std::vector<PendingSource> srcs;
             if (has_neighbour) {
@@ -363,8 +365,10 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
         std::vector<Seg> segs[DISTDL_MAX_RANK];
         for (int k = 0; k < d; ++k) {
             const int64_t b = p->size[k][c[k]];
-            const int64_t wl = c[k] > 0 ? p->hhi[k][c[k] - 1] : 0;                  // low neighbour's high ghost
-            const int64_t wh = c[k] + 1 < p->pshape[k] ? p->hlo[k][c[k] + 1] : 0;   // high neighbour's low ghost
+            const int32_t pk = p->pshape[k];
+            const bool has_lo = c[k] > 0 || p->periodic[k], has_hi = c[k] + 1 < pk || p->periodic[k];
+            const int64_t wl = has_lo ? p->hhi[k][(c[k] + pk - 1) % pk] : 0;   // low neighbour's high ghost
+            const int64_t wh = has_hi ? p->hlo[k][(c[k] + 1) % pk] : 0;        // high neighbour's low ghost
             int64_t cuts[4] = {0, wl, b - wh, b};
             std::sort(cuts, cuts + 4);
             for (int i = 0; i < 3; ++i) {
@@ -399,15 +403,20 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
                     int32_t nc[DISTDL_MAX_RANK];
                     bool self = true;
                     for (int k = 0; k < d; ++k) {
-                        nc[k] = c[k] + options[k][o[k]];
+                        nc[k] = (c[k] + options[k][o[k]] + p->pshape[k]) % p->pshape[k];   // wraps in a periodic dimension
                         if (options[k][o[k]] != 0) self = false;
                     }
                     s.r.shard = p->worker_of(nc);
                     s.clear_after = self ? 0 : 1;
                     for (int k = 0; k < d; ++k) {
-                        // same global index, expressed in the neighbour's padded-local index
-                        const int64_t g = p->start[k][c[k]] + segs[k][pick[k]].s0;
-                        s.r.start[k] = g - p->start[k][nc[k]] + p->hlo[k][nc[k]];
+                        // the same cell in the neighbour's padded-local index: offset s0 of this bulk is the
+                        // low neighbour's high ghost cell s0 (right after its bulk), or lies b - s0 cells
+                        // before the start of the high neighbour's bulk
+                        const int64_t s0 = segs[k][pick[k]].s0, b = p->size[k][c[k]];
+                        const int opt = options[k][o[k]];
+                        s.r.start[k] = opt == 0 ? p->hlo[k][c[k]] + s0
+                                     : opt < 0 ? p->hlo[k][nc[k]] + p->size[k][nc[k]] + s0
+                                               : p->hlo[k][nc[k]] - (b - s0);
                         s.r.extent[k] = dst.extent[k];
                     }
                     // levels folded after this term: trailing active dimensions at their last option

@@ -319,6 +319,7 @@ static distdl_status_t pool_impl(const distdl_partition *p, const void *const *i
     clear_error();
     if (!p || !in || !out) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
     if (p->rank != 4 || p->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-4 F32 partition", what);
+    if (p->any_periodic()) return fail(DISTDL_ERR_UNSUPPORTED, "%s: periodic partitions are not supported by the fused layers", what);
     if (p->pshape[0] != 1 || p->pshape[1] != 1)
         return fail(DISTDL_ERR_UNSUPPORTED, "%s: only the feature-space dimensions may be partitioned", what);
     if (p->num_workers > kPoolMaxWorkers) return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d workers", what, kPoolMaxWorkers);

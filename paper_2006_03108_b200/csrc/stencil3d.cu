@@ -383,6 +383,7 @@ static distdl_status_t stencil_impl(const distdl_partition *p, const void *const
     clear_error();
     if (!p || !in || !w || !out) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
     if (p->rank != 3 || p->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-3 F32 partition", what);
+    if (p->any_periodic()) return fail(DISTDL_ERR_UNSUPPORTED, "%s: periodic partitions are not supported by the fused layers", what);
     if (radius < 1 || radius > kStMaxR) return fail(DISTDL_ERR_UNSUPPORTED, "%s: radius %d (supported: 1..%d)", what, radius, kStMaxR);
     if (p->num_workers > kStMaxWorkers) return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d workers", what, kStMaxWorkers);
     for (int k = 0; k < 3; ++k) {

@@ -283,6 +283,40 @@ def test_halo_fwd_and_adj_bf16_fp64_bit_exact(case):
             assert same_bits(back(a), b)
 
 
+PERIODIC_HALO_CASES = [
+    # global shape, partition, halo lo, halo hi, periodic
+    ((7,), (1,), (2,), (3,), (True,)),
+    ((9,), (2,), (2,), (1,), (True,)),
+    ((6, 8), (2, 2), (1, 1), (2, 2), (True, False)),
+    ((12, 16), (1, 3), (2, 1), (1, 2), (True, True)),
+    ((8, 10, 12), (2, 1, 2), (1, 1, 1), (1, 1, 1), (False, True, True)),
+    ((70, 66, 72), (2, 2, 2), (4, 4, 4), (4, 4, 4), (True, True, True)),      # 16-byte paths, several tiles
+]
+
+
+@pytest.mark.parametrize("case", PERIODIC_HALO_CASES, ids=[str(c[0]) + str(c[1]) + str(c[4]) for c in PERIODIC_HALO_CASES])
+def test_periodic_halo_fwd_and_adj_bit_exact(case):
+    gs, ps, hlo, hhi, per = case
+    opart = oracle.Partition(gs, ps, hlo, hhi, per)
+    gpart = distdl.Partition(gs, ps, hlo, hhi, periodic=per)
+    x = random_shards(opart, 31)
+    xs = [dev(a) for a in x]
+    distdl.halo_fwd(gpart, xs)
+    y = []
+    for w in range(opart.num_workers):
+        a = inputs.uniform_pm1(opart.padded_shape(w), 3200 + w)
+        y.append((a * np.float32(10.0) ** inputs.integers(opart.padded_shape(w), 3300 + w, -3, 4)).astype(np.float32))
+    ys = [dev(a) for a in y]
+    distdl.halo_adj(gpart, ys)
+    torch.cuda.synchronize()
+    for a, b in zip(xs, oracle.halo_fwd_sequence(opart, x)):
+        assert same_bits(host(a), b)
+    for a, b in zip(ys, oracle.halo_adj_sequence(opart, y)):
+        assert same_bits(host(a), b)
+    r = oracle.adjoint_test_ratio([host(t) for t in xs], y, x, [host(t) for t in ys])
+    assert r < 1e-5
+
+
 # --------------------------------------------------------------------------
 # Convolution layer
 # --------------------------------------------------------------------------

@@ -175,3 +175,30 @@ def test_validation_of_the_gradient_stencil_and_dtype_entry_points():
     assert p64.halo_stats(False)[2] == 2 * distdl.Partition((9, 9), (2, 2), (1, 1), (1, 1)).halo_stats(False)[2]
     r64 = distdl.Repartition((12, 8), (3, 1), (1, 2), distdl.F64)
     assert r64.shard_shape(0) == (4, 8) and r64.shard_shape(1, destination=True) == (12, 4)
+
+
+def test_periodic_partition_geometry_and_refusals():
+    lib = distdl.lib()
+    vp = ctypes.c_void_p
+    # 8 x 8 on 2 x 2 workers, width 1: 20 ghost cells per shard; all of them have an owner when both
+    # dimensions wrap (20 reads + 20 writes of 4 bytes per shard), only 9 of them (a row, a column, a corner) otherwise
+    per = distdl.Partition((8, 8), (2, 2), (1, 1), (1, 1), periodic=(True, True))
+    flat = distdl.Partition((8, 8), (2, 2), (1, 1), (1, 1))
+    assert per.halo_stats(False)[2] == 4 * (20 + 20) * 4
+    assert flat.halo_stats(False)[2] == 4 * (20 + 9) * 4
+    # adjoint: every ghost read and cleared (8 B), every bulk cell in reach of a face read and written (8 B):
+    # all 12 cells of the bulk's rim with both dimensions periodic, 7 of them (one row, one column) otherwise
+    assert per.halo_stats(True)[2] == 4 * (20 * 8 + 12 * 8)
+    assert flat.halo_stats(True)[2] == 4 * (20 * 4 + 9 * 4 + 7 * 8)
+    # the ghost-width rule holds across the seam as well
+    assert _status(distdl.Partition, (6,), (2,), (4,), (0,), periodic=(True,)) == 2
+    # a worker alone along a periodic dimension is its own neighbour
+    one = distdl.Partition((7,), (1,), (2,), (3,), periodic=(True,))
+    assert one.halo_stats(False)[2] == (5 + 5) * 4 and one.halo_stats(True)[0] >= 1
+    # fused layers take no periodic partitions
+    arr = (vp * 16)(*[0x10000 * (i + 1) for i in range(16)])
+    p4 = distdl.Partition((1, 2, 16, 16), (1, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2), periodic=(False, False, True, True))
+    assert lib.distdl_conv_fwd(p4.handle, arr, vp(0x50000), None, 5, 5, arr, None) == 4
+    p3 = distdl.Partition((8, 8, 8), (2, 1, 1), (2, 2, 2), (2, 2, 2), periodic=(True, False, False))
+    taps = (ctypes.c_float * 15)(*([0.5] * 15))
+    assert lib.distdl_stencil3d_fwd(p3.handle, arr, taps, 2, arr, None) == 4

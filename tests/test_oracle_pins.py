@@ -883,3 +883,50 @@ def test_halo_adjoint_in_bf16_and_fp64_on_integer_data():
     for a, b, c in zip(ref, got64, gotbf):
         assert np.array_equal(a.astype(np.float64), b)
         assert np.array_equal(a.astype(np.float64), oracle.bf16_bits_to_f64(c))
+
+
+# --------------------------------------------------------------------------
+# Periodic dimensions of the halo exchange
+# --------------------------------------------------------------------------
+
+PERIODIC_CASES = [
+    # global shape, partition, hlo, hhi, periodic
+    ((7,), (1,), 2, 3, (True,)),                       # one worker: its own neighbour on both sides
+    ((9,), (2,), 2, 1, (True,)),                       # two workers: the same neighbour low and high
+    ((10,), (3,), [[1, 2, 0]], [[2, 0, 1]], (True,)),
+    ((6, 8), (2, 2), 1, 2, (True, False)),
+    ((6, 8), (1, 3), (2, 1), (1, 2), (True, True)),
+    ((4, 5, 6), (2, 1, 2), 1, 1, (False, True, True)),
+]
+
+
+@pytest.mark.parametrize("case", PERIODIC_CASES, ids=[str(c[0]) + str(c[1]) + str(c[4]) for c in PERIODIC_CASES])
+def test_periodic_halo_matches_wrapped_padding_and_has_transpose_adjoint(case):
+    gs, ps, hlo, hhi, per = case
+    part = Partition(gs, ps, hlo, hhi, per)
+    x = _random_shards(part, 9)                      # garbage in the ghosts
+    a = oracle.halo_fwd_definition(part, x)
+    b = oracle.halo_fwd_sequence(part, x)
+    g = oracle.assemble_global(part, x)
+    # library pin: a window of the global tensor padded by wrapping (periodic dimensions) or with zeros
+    mlo = [max(part.hlo[k]) for k in range(part.rank)]
+    mhi = [max(part.hhi[k]) for k in range(part.rank)]
+    gp = g
+    for k in range(part.rank):
+        width = [(0, 0)] * part.rank
+        width[k] = (mlo[k], mhi[k])
+        gp = np.pad(gp, width, mode="wrap") if per[k] else np.pad(gp, width)
+    for w in range(part.num_workers):
+        assert a[w].tobytes() == b[w].tobytes()
+        lo, _ = part.widths(w)
+        st, pshape = part.bulk_start(w), part.padded_shape(w)
+        win = tuple(slice(st[k] - lo[k] + mlo[k], st[k] - lo[k] + mlo[k] + pshape[k]) for k in range(part.rank))
+        assert np.array_equal(a[w], gp[win])
+    # operator matrices: 0/1 entries, one per ghost row; the adjoint sequence is the exact transpose
+    M = _operator_matrix(part, oracle.halo_fwd_sequence)
+    assert set(np.unique(M)) <= {0.0, 1.0} and np.all(M.sum(axis=1) <= 1)
+    if all(per):
+        assert np.all(M.sum(axis=1) == 1)                  # no zero padding anywhere
+    assert np.array_equal(_operator_matrix(part, oracle.halo_adj_sequence), M.T)
+    y = _random_shards(part, 10)
+    assert oracle.adjoint_test_ratio(b, y, x, oracle.halo_adj_sequence(part, y)) < 1e-6
