@@ -212,24 +212,58 @@ class Workload:
 
     # ---- end-to-end variant: inputs come from pinned host memory, results go back to it ----
     def e2e_setup(self):
+        """Pinned host copies of every input and output, per operator, and the three streams of the pipeline."""
         torch = self.torch
-        ins = [self.b_src] + self.r_src + self.h_x + self.h_y + self.c_x + self.c_dy + [self.c_w] + \
-            self.a_x + self.a_w + self.a_dy
-        outs = self.b_dst + [self.r_dst] + self.h_x + self.h_y + self.c_y + self.c_dx + self.a_y + self.a_dx
-        self.e2e_in = [(t, torch.empty(t.shape, dtype=t.dtype, pin_memory=True)) for t in ins]
-        self.e2e_out = [(t, torch.empty(t.shape, dtype=t.dtype, pin_memory=True)) for t in outs]
-        for t, h in self.e2e_in:
-            h.copy_(t)
+        per_op = [
+            ([self.b_src], self.b_dst),
+            (self.r_src, [self.r_dst]),
+            (self.h_x, self.h_x),
+            (self.h_y, self.h_y),
+            (self.c_x + [self.c_w], self.c_y),
+            (self.c_dy, self.c_dx),
+            (self.a_x + self.a_w, self.a_y),
+            (self.a_dy, self.a_dx),
+        ]
+        pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        self.e2e_ops = [([(t, pin(t)) for t in ins], [(t, pin(t)) for t in outs]) for ins, outs in per_op]
+        for ins, _ in self.e2e_ops:
+            for t, h in ins:
+                h.copy_(t)
         torch.cuda.synchronize()
-        self.h2d_bytes = sum(t.numel() * t.element_size() for t, _ in self.e2e_in)
-        self.d2h_bytes = sum(t.numel() * t.element_size() for t, _ in self.e2e_out)
+        self.h2d_bytes = sum(t.numel() * t.element_size() for ins, _ in self.e2e_ops for t, _ in ins)
+        self.d2h_bytes = sum(t.numel() * t.element_size() for _, outs in self.e2e_ops for t, _ in outs)
+        self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        self.e2e_done = None
 
     def e2e_step(self):
-        for t, h in self.e2e_in:
-            t.copy_(h, non_blocking=True)
-        self.step()
-        for t, h in self.e2e_out:
-            h.copy_(t, non_blocking=True)
+        """One step through the public calls with host buffers on both ends: the inputs of every operator come
+        from pinned host memory and its results go back to it.  Three streams: uploads, the operators, downloads;
+        the upload of the next operator's inputs and the download of the previous one's results run while an
+        operator computes, so both directions of the host link are busy.  A step starts its uploads only when
+        the previous step's downloads are done (some buffers are input and output at once)."""
+        torch = self.torch
+        main = torch.cuda.current_stream()
+        if self.e2e_done is not None:
+            self.s_in.wait_event(self.e2e_done)
+        else:
+            self.s_in.wait_stream(main)
+        for (ins, outs), op in zip(self.e2e_ops, self.ops):
+            with torch.cuda.stream(self.s_in):
+                for t, h in ins:
+                    t.copy_(h, non_blocking=True)
+                up = torch.cuda.Event()
+                up.record()
+            main.wait_event(up)
+            op[1]()
+            ran = torch.cuda.Event()
+            ran.record(main)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(ran)
+                for t, h in outs:
+                    h.copy_(t, non_blocking=True)
+        self.e2e_done = torch.cuda.Event()
+        self.e2e_done.record(self.s_out)
+        main.wait_event(self.e2e_done)      # the step is over when its last result has reached the host
 
 
 # ----------------------------------------------------------------------------------------------
