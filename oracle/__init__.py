@@ -41,6 +41,8 @@ from .layers import (  # noqa: F401
     conv_adj,
     conv_adj_scatter_then_halo,
     conv_adj_params,
+    convg_fwd,
+    convg_adj,
     stencil3d_fwd,
     stencil3d_adj,
     stencil3d_fwd_exchange_then_local,

@@ -149,6 +149,95 @@ def conv_adj_params(part: Partition, x_shards, dy_shards, kh, kw):
 
 
 # --------------------------------------------------------------------------
+# Generalized distributed convolution: channels partitioned as well
+# (Section 4, "Sparse layers": forward / adjoint convolution algorithms with
+# P_x = 1 x P_ci x P_0 x P_1, P_y = 1 x P_co x P_0 x P_1, weights on P_co x P_ci,
+# work partition 1 x P_co x P_ci x P_0 x P_1)
+# --------------------------------------------------------------------------
+
+def _channel_blocks(n, p):
+    from .partition import balanced_split
+    return balanced_split(n, p)
+
+
+def convg_fwd(xpart: Partition, nco, pco, x_shards, w_blocks, bias_blocks=None):
+    """Forward convolution algorithm, step by step.
+
+    xpart: partition 1 x P_ci x P_0 x P_1 of x [N, n_ci, H, W] with ghost widths
+    (0, 0, ph, pw); worker (j, r, c) has id (j * P_0 + r) * P_1 + c.
+    w_blocks[i * P_ci + j]: [n_co/P_co, n_ci/P_ci, kh, kw] (the block of worker (i, j)
+    of P_r); bias_blocks[i]: [n_co/P_co] or None, present on the j = 0 subpartition only.
+      x <- H x;  w^ <- B w, b^ <- B b (to every spatial worker);  x^ <- B x (to the
+      P_co copies of the work partition);  y^_{ijs} <- Conv(w^_{ij}, b^_i if j = 0; x^_{js});
+      y_{is} <- R over j = 0..P_ci-1 in order.
+    Local convolutions and the fold in fp64, rounded once to fp32.  Returns the
+    bulk-shaped shards of y on 1 x P_co x P_0 x P_1, id (i * P_0 + r) * P_1 + c.
+    """
+    from .primitives import halo_fwd_sequence
+    assert xpart.rank == 4 and xpart.pshape[0] == 1
+    _, pci, p0, p1 = xpart.pshape
+    kh, kw = np.asarray(w_blocks[0]).shape[2:]
+    ph, pw = kh // 2, kw // 2
+    xh = halo_fwd_sequence(xpart, x_shards)
+    xhat = [broadcast_fwd(np.asarray(a, dtype=np.float64), pco) for a in xh]        # copies for i = 0..P_co-1
+    y = []
+    for i in range(pco):
+        for r in range(p0):
+            for c in range(p1):
+                partial = []
+                for j in range(pci):
+                    x = xhat[(j * p0 + r) * p1 + c][i]
+                    w = np.asarray(w_blocks[i * pci + j], dtype=np.float64)
+                    N, cib, hp, wp = x.shape
+                    cob = w.shape[0]
+                    assert w.shape[1] == cib
+                    hb, wb = hp - 2 * ph, wp - 2 * pw
+                    acc = np.zeros((N, cob, hb, wb), dtype=np.float64)
+                    for a in range(kh):
+                        for b in range(kw):
+                            # sum over the block's input channels, in channel order
+                            acc += np.einsum("oc,nchw->nohw", w[:, :, a, b], x[:, :, a:a + hb, b:b + wb])
+                    if bias_blocks is not None and j == 0:
+                        acc += np.asarray(bias_blocks[i], dtype=np.float64)[None, :, None, None]
+                    partial.append(acc)
+                y.append(sumreduce_fwd(partial).astype(np.float32))
+    return y
+
+
+def convg_adj(xpart: Partition, nco, pco, dy_shards, w_blocks):
+    """Adjoint convolution algorithm, dx output, step by step.
+
+      dy^_{ijs} <- B dy_{is} (to the P_ci copies);  dx^_{ijs} <- [dConv]*(dy^_{ijs}) with
+      w^_{ij}: the local adjoint scatters into the whole padded input shard;
+      dx_{js} <- R over i = 0..P_co-1 in order;  dx <- H* dx.
+    fp64 up to the end of R, rounded to fp32 before H* (whose sums are then fp32, as in
+    the halo oracle).  Returns padded shards of xpart with zero ghosts.
+    """
+    assert xpart.rank == 4 and xpart.pshape[0] == 1
+    _, pci, p0, p1 = xpart.pshape
+    kh, kw = np.asarray(w_blocks[0]).shape[2:]
+    local = []
+    for j in range(pci):
+        for r in range(p0):
+            for c in range(p1):
+                wk = (j * p0 + r) * p1 + c
+                partial = []
+                for i in range(pco):
+                    dy = np.asarray(dy_shards[(i * p0 + r) * p1 + c], dtype=np.float64)
+                    w = np.asarray(w_blocks[i * pci + j], dtype=np.float64)
+                    N, cob, hb, wb = dy.shape
+                    dx = np.zeros((N, w.shape[1], hb + kh - 1, wb + kw - 1), dtype=np.float64)
+                    for a in range(kh):
+                        for b in range(kw):
+                            dx[:, :, a:a + hb, b:b + wb] += np.einsum("oc,nohw->nchw", w[:, :, a, b], dy)
+                    partial.append(dx)
+                got = sumreduce_fwd(partial).astype(np.float32)
+                assert got.shape == xpart.padded_shape(wk)
+                local.append(got)
+    return halo_adj_sequence(xpart, local)
+
+
+# --------------------------------------------------------------------------
 # Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers":
 # a sliding-kernel layer on a feature-space partition = halo exchange, then the
 # local kernel; Section 6 names large volumetric data as the target)

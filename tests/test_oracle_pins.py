@@ -930,3 +930,70 @@ def test_periodic_halo_matches_wrapped_padding_and_has_transpose_adjoint(case):
     assert np.array_equal(_operator_matrix(part, oracle.halo_adj_sequence), M.T)
     y = _random_shards(part, 10)
     assert oracle.adjoint_test_ratio(b, y, x, oracle.halo_adj_sequence(part, y)) < 1e-6
+
+
+# --------------------------------------------------------------------------
+# Generalized convolution: channel partitions P_co x P_ci besides the feature space
+# --------------------------------------------------------------------------
+
+CONVG_CASES = [
+    # N, n_ci, n_co, H, W, P_ci, P_co, P_0, P_1, k
+    (2, 4, 6, 9, 10, 2, 3, 2, 2, 3),
+    (1, 5, 3, 8, 7, 2, 2, 1, 2, 5),        # uneven channel blocks (3 + 2, 2 + 1)
+    (1, 3, 4, 6, 6, 1, 1, 1, 1, 3),
+    (2, 2, 2, 12, 9, 2, 1, 3, 1, 5),
+]
+
+
+def _convg_problem(case, seed):
+    N, nci, nco, H, W, pci, pco, p0, p1, k = case
+    h = k // 2
+    xpart = Partition((N, nci, H, W), (1, pci, p0, p1), (0, 0, h, h), (0, 0, h, h))
+    ypart = Partition((N, nco, H, W), (1, pco, p0, p1))
+    xg = inputs.normal((N, nci, H, W), seed)
+    wg = inputs.normal((nco, nci, k, k), seed + 1, 0.2)
+    bg = inputs.normal((nco,), seed + 2)
+    cs_i, cz_i = oracle.balanced_split(nco, pco)
+    cs_j, cz_j = oracle.balanced_split(nci, pci)
+    wb = [wg[cs_i[i]:cs_i[i] + cz_i[i], cs_j[j]:cs_j[j] + cz_j[j]] for i in range(pco) for j in range(pci)]
+    bb = [bg[cs_i[i]:cs_i[i] + cz_i[i]] for i in range(pco)]
+    return xpart, ypart, xg, wg, bg, wb, bb
+
+
+@pytest.mark.parametrize("case", CONVG_CASES, ids=[str(c) for c in CONVG_CASES])
+def test_generalized_conv_matches_the_sequential_layer_and_its_autograd(case):
+    import torch
+    xpart, ypart, xg, wg, bg, wb, bb = _convg_problem(case, 101)
+    nco, pco, k = case[2], case[6], case[9]
+    x = oracle.scatter_global(xpart, xg, fill=lambda wk: np.full(xpart.padded_shape(wk), 3.0))     # garbage ghosts
+    y = oracle.assemble_global(ypart, oracle.convg_fwd(xpart, nco, pco, x, wb, bb))
+    X = torch.tensor(xg, dtype=torch.float64, requires_grad=True)
+    Y = torch.nn.functional.conv2d(X, torch.tensor(wg, dtype=torch.float64), torch.tensor(bg, dtype=torch.float64), padding=k // 2)
+    assert np.allclose(y, Y.detach().numpy(), rtol=1e-6, atol=1e-5)
+    dyg = inputs.normal(Y.shape, 105)
+    Y.backward(torch.tensor(dyg, dtype=torch.float64))
+    dx = oracle.convg_adj(xpart, nco, pco, oracle.scatter_global(ypart, dyg), wb)
+    assert np.allclose(oracle.assemble_global(xpart, dx), X.grad.numpy(), rtol=1e-6, atol=1e-5)
+    for wk in range(xpart.num_workers):
+        mask = np.ones(xpart.padded_shape(wk), dtype=bool)
+        mask[xpart.bulk_slices(wk)] = False
+        assert not dx[wk][mask].any()
+    # dot test of the pair (no bias)
+    y0 = oracle.convg_fwd(xpart, nco, pco, oracle.scatter_global(xpart, xg), wb)
+    assert oracle.adjoint_test_ratio(y0, oracle.scatter_global(ypart, dyg), oracle.scatter_global(xpart, xg), dx) < 1e-6
+
+
+def test_generalized_conv_reduces_to_the_depthwise_layer_on_diagonal_weights():
+    # weights that couple channel c only to itself: the layer is the depthwise one, which is pinned separately
+    N, C, H, W, k = 1, 4, 10, 8, 5
+    xpart = Partition((N, C, H, W), (1, 2, 2, 1), (0, 0, 2, 2), (0, 0, 2, 2))
+    dpart = Partition((N, C, H, W), (1, 1, 2, 1), (0, 0, 2, 2), (0, 0, 2, 2))
+    xg = inputs.normal((N, C, H, W), 111)
+    wd = inputs.normal((C, k, k), 112, 0.2)
+    wg = np.zeros((C, C, k, k), np.float32)
+    for c in range(C):
+        wg[c, c] = wd[c]
+    wb = [wg[2 * i:2 * i + 2, 2 * j:2 * j + 2] for i in range(2) for j in range(2)]
+    y = oracle.assemble_global(Partition((N, C, H, W), (1, 2, 2, 1)), oracle.convg_fwd(xpart, C, 2, oracle.scatter_global(xpart, xg), wb))
+    yd = oracle.assemble_global(Partition((N, C, H, W), (1, 1, 2, 1)), oracle.conv_fwd(dpart, oracle.scatter_global(dpart, xg), wd))
+    assert np.allclose(y, yd, rtol=0, atol=2e-6)
