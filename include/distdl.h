@@ -273,6 +273,33 @@ distdl_status_t distdl_conv_adj_params(const distdl_partition_t *p, const void *
                                        void *stream);
 
 /* ------------------------------------------------------------------------
+ * Generalized convolution layer: channels partitioned as well (Section 4, "Sparse layers": the forward /
+ * adjoint convolution algorithms with x on 1 x P_ci x P_0 x P_1, y on 1 x P_co x P_0 x P_1, the weights on
+ * P_co x P_ci and the work partition 1 x P_co x P_ci x P_0 x P_1).
+ *
+ * px: rank-4 NCHW F32 partition of x, shape 1 x P_ci x P_0 x P_1, halo widths (0, 0, (kh-1)/2, (kw-1)/2) on
+ *     every side; worker (j, r, c) has id (j*P_0 + r)*P_1 + c.  nco output channels are split evenly over pco
+ *     blocks; y / dy live on 1 x pco x P_0 x P_1, worker (i, r, c) has id (i*P_0 + r)*P_1 + c.
+ *     P_ci, pco <= 8; at most 64 shards per tensor; kh = kw in {3, 5, 7}, stride 1, centred.
+ * w[i*P_ci + j]: F32 [nco_i, nci_j, kh, kw], the block of worker (i, j) of the weight partition.
+ * bias[i]: F32 [nco_i], or bias == NULL (the bias lives on the j = 0 subpartition: added once).
+ * convg_fwd: x <- H x; x^ <- B x (to the pco copies of the work partition); y^_{ijs} <- Conv(w_ij, b_i on j = 0;
+ *     x^_js); y_is <- R over j = 0..P_ci-1 in order -- fused: y[n,o,p] = b[o] + sum over input channels c
+ *     (block after block, channel after channel) and taps of w[o,c,a,b] * x[n,c,p + (a,b) - pad] on the
+ *     GLOBAL tensor, zeros outside.  x[.]: padded shards (bulk read only); y[.]: bulk-shaped shards.
+ * convg_adj: dy^ <- B dy; dx^_{ijs} <- [dConv]*(dy^_{ijs}); dx_js <- R over i in order; dx <- H* dx -- fused in
+ *     gather form: dx[n,c,p] = sum over output channels o and taps of w[o,c,a,b] * dy[n,o,p - (a,b) + pad];
+ *     dy[.]: bulk-shaped shards; dx[.]: padded shards whose ghosts are set to zero.
+ * (dw, db of this layer are not computed.)
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_convg_fwd(const distdl_partition_t *px, int64_t nco, int32_t pco,
+                                 const void *const *x, const void *const *w, const void *const *bias,
+                                 int32_t kh, int32_t kw, void *const *y, void *stream);
+distdl_status_t distdl_convg_adj(const distdl_partition_t *px, int64_t nco, int32_t pco,
+                                 const void *const *dy, const void *const *w, int32_t kh, int32_t kw,
+                                 void *const *dx, void *stream);
+
+/* ------------------------------------------------------------------------
  * Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers": on a feature-space
  * partition a sliding-kernel layer is the halo exchange followed by the local kernel, its adjoint the
  * local adjoint followed by H*; Section 6 names large volumetric data as the target).

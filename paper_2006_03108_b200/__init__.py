@@ -83,6 +83,8 @@ def lib():
     L.distdl_conv_adj_params.argtypes = [vp, pvp, pvp, c_i32, c_i32, vp, vp, vp, c_i64, vp]
     L.distdl_stencil3d_fwd.argtypes = [vp, pvp, ctypes.POINTER(ctypes.c_float), c_i32, pvp, vp]
     L.distdl_stencil3d_adj.argtypes = [vp, pvp, ctypes.POINTER(ctypes.c_float), c_i32, pvp, vp]
+    L.distdl_convg_fwd.argtypes = [vp, c_i64, c_i32, pvp, pvp, pvp, c_i32, c_i32, pvp, vp]
+    L.distdl_convg_adj.argtypes = [vp, c_i64, c_i32, pvp, pvp, c_i32, c_i32, pvp, vp]
     L.distdl_device_status.argtypes = [vp]
     _lib = L
     return L
@@ -294,6 +296,20 @@ def stencil3d_fwd(part, x, w, y, stream=None):
 def stencil3d_adj(part, dy, w, dx, stream=None):
     arr, radius = _taps(w)
     _check(lib().distdl_stencil3d_adj(part.handle, _ptr_array(dy), arr, radius, _ptr_array(dx), _stream(stream)))
+
+
+def convg_fwd(px, nco, pco, x, w, bias, y, stream=None):
+    """Channel-partitioned convolution layer; w: list of blocks [nco_i, nci_j, kh, kw] in order i * P_ci + j."""
+    kh, kw = int(w[0].shape[-2]), int(w[0].shape[-1])
+    b = None if bias is None else _ptr_array(bias)
+    _check(lib().distdl_convg_fwd(px.handle, nco, pco, _ptr_array(x), _ptr_array(w), b, kh, kw, _ptr_array(y),
+                                  _stream(stream)))
+
+
+def convg_adj(px, nco, pco, dy, w, dx, stream=None):
+    kh, kw = int(w[0].shape[-2]), int(w[0].shape[-1])
+    _check(lib().distdl_convg_adj(px.handle, nco, pco, _ptr_array(dy), _ptr_array(w), kh, kw, _ptr_array(dx),
+                                  _stream(stream)))
 
 
 class Repartition:

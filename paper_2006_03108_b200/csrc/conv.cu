@@ -8,6 +8,7 @@
 // any atomics, and it leaves the ghosts of dx zero as H* does.
 #include <algorithm>
 #include <cstring>
+#include <vector>
 
 #include "common.h"
 #include "tma.h"
@@ -158,8 +159,10 @@ struct ConvCfg {
 };
 
 // Issues the asynchronous copies (and the direct zero stores) that fill `tile` for output tile t.
+// wofs: first entry of P.in of the group of Ph x Pw shards the tile belongs to (the channel-partitioned
+// layer keeps one such group per block of input channels).
 template <int K, bool ADJ>
-__device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &t, float *tile) {
+__device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &t, float *tile, int wofs = 0) {
     using C = ConvCfg<K, ADJ>;
     if (!t.valid) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -194,7 +197,7 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
         }
         const int rbh = P.bh[rr];
         const int pitch_c = t.bw + 2 * C::IOFF;
-        const float *grow = P.in[rr * P.pw_workers + t.c] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_c +
+        const float *grow = P.in[wofs + rr * P.pw_workers + t.c] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_c +
                             (size_t)(i + C::IOFF) * pitch_c + C::IOFF + first_col;
         for (int v = v_lo + lane; v < v_hi; v += 32) cp_async16(srow + 4 * v, grow + 4 * v);
         // edge columns: left of v_lo and right of v_hi, element by element (neighbour columns or zero)
@@ -218,7 +221,7 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
             }
             if (ok) {
                 const int pitch_n = P.bw[cc] + 2 * C::IOFF;
-                cp_async4(srow + s, P.in[rr * P.pw_workers + cc] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_n +
+                cp_async4(srow + s, P.in[wofs + rr * P.pw_workers + cc] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_n +
                                         (size_t)(i + C::IOFF) * pitch_n + C::IOFF + j);
             } else {
                 srow[s] = 0.f;
@@ -844,6 +847,337 @@ static distdl_status_t conv_impl(const distdl_partition *p, const void *const *i
 }
 
 // ---------------------------------------------------------------------------------------------
+// Generalized convolution layer: channels partitioned as well (Section 4, "Sparse layers": forward /
+// adjoint convolution algorithms with x on 1 x P_ci x P_0 x P_1, y on 1 x P_co x P_0 x P_1, weights on
+// P_co x P_ci and the work partition 1 x P_co x P_ci x P_0 x P_1).
+//   forward:  x <- H x;  x^ <- B x (to the P_co copies);  y^_{ijs} <- Conv(w_{ij}, b_i on j = 0; x^_{js});
+//             y_{is} <- R over j, in order.
+//   adjoint:  dy^ <- B dy (to the P_ci copies);  dx^_{ijs} <- [dConv]*(dy^_{ijs});  dx_{js} <- R over i, in
+//             order;  dx <- H* dx  (gather form: a correlation of dy with the rotated kernels).
+// With every shard in one memory the broadcasts are implicit and the sum-reduce is the running sum of
+// the block that owns an output tile: it walks through the blocks of the reduced channel partition in
+// worker order and through the channels of a block in channel order, so the order of the sum is fixed.
+// H / H* are fused as in the depthwise kernels (tiles staged with their ghost rows and columns from
+// the neighbouring shards' bulk).  A block owns 32 x 128 pixels of kCob output channels; a thread
+// 4 x 8 pixels of them, as packed pairs of neighbouring pixels.
+// ---------------------------------------------------------------------------------------------
+constexpr int kCob = 2;                 // output channels per block
+constexpr int kMaxChanBlocks = 8;       // P_co, P_ci
+constexpr int kMaxGroups = 128;         // groups of kCob output channels
+
+struct ConvGParams {
+    ConvParams base;                        // in = shards of the input tensor, out = shards of the output tensor
+    const float *w[kMaxChanBlocks * kMaxChanBlocks];   // weight blocks, worker order i * P_ci + j
+    const float *bias[kMaxChanBlocks];      // forward only; per block of output channels, may be null
+    int32_t cnt_out[kMaxChanBlocks], cnt_in[kMaxChanBlocks];   // channels per block of the output / input partition
+    int32_t p_out, p_in, pci;               // blocks of the output / input channel partition; P_ci
+    int32_t groups;                         // groups of up to kCob output channels, all blocks together
+    uint8_t grp_block[kMaxGroups], grp_first[kMaxGroups], grp_count[kMaxGroups];
+    int32_t tiles_y, total_tiles;
+    int32_t ooff;                           // ghost width of the output layout
+};
+
+template <int K, bool ADJ>
+__global__ void __launch_bounds__(kConvThreads, 3)
+convg_kernel(const __grid_constant__ ConvGParams G) {
+    using C = ConvCfg<K, ADJ>;
+    constexpr int XO = C::PADL - C::PH;                         // tile column of the first input of output column 0
+    constexpr int NF2 = ((XO + kColsPerThread + K - 1 + 3) / 4) * 4;   // floats of a thread's (aligned) window
+    constexpr int NP = NF2 / 2;
+    static_assert(kTileW - kColsPerThread + NF2 <= C::PITCH, "window beyond the tile row");
+    extern __shared__ __align__(16) float smem[];               // two x tiles, then two weight tables
+    float *tiles = smem;
+    uint64_t *wtab = reinterpret_cast<uint64_t *>(smem + 2 * C::TILE_FLOATS);   // [2][kCob * K * K] (w, w) pairs
+    const ConvParams &P = G.base;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int spatial = P.ph_workers * P.pw_workers;
+
+    for (int tile = blockIdx.x; tile < G.total_tiles; tile += gridDim.x) {
+        ConvTile t = decode_tile(P, tile, G.tiles_y, 0);
+        if (!t.valid) continue;                                  // the same for every thread of the block
+        const int n = t.plane / G.groups, g = t.plane - n * G.groups;
+        const int ob = G.grp_block[g], o0 = G.grp_first[g], oc = G.grp_count[g];
+
+        uint64_t acc[kCob][kRowsPerThread][4];
+#pragma unroll
+        for (int o = 0; o < kCob; ++o) {
+            float b = 0.f;
+            if (!ADJ && G.bias[ob] && o < oc) b = __ldg(G.bias[ob] + o0 + o);
+#pragma unroll
+            for (int r = 0; r < kRowsPerThread; ++r)
+#pragma unroll
+                for (int p2 = 0; p2 < 4; ++p2) acc[o][r][p2] = pack2(b, b);
+        }
+
+        // the channels of the reduced partition: block after block, channel after channel
+        auto stage = [&](int ib, int cl, int buf) {
+            ConvTile ti = t;
+            ti.plane = n * G.cnt_in[ib] + cl;
+            stage_tile<K, ADJ>(P, ti, tiles + buf * C::TILE_FLOATS, ib * spatial);
+            // weights of (output channel o0 + o, this input channel), as (w, w) pairs; adjoint: rotated
+            if ((int)threadIdx.x < kCob * K * K) {
+                const int o = threadIdx.x / (K * K), tap = threadIdx.x - o * (K * K);
+                float w = 0.f;
+                if (o < oc) {
+                    const float *blk = ADJ ? G.w[ib * G.pci + ob] : G.w[ob * G.pci + ib];
+                    const int s_out = ADJ ? K * K : G.cnt_in[ib] * K * K, s_in = ADJ ? G.cnt_out[ob] * K * K : K * K;
+                    w = __ldg(blk + (size_t)(o0 + o) * s_out + (size_t)cl * s_in + (ADJ ? K * K - 1 - tap : tap));
+                }
+                reinterpret_cast<float2 *>(wtab + buf * (kCob * K * K))[threadIdx.x] = make_float2(w, w);
+            }
+        };
+        int ib = 0, cl = 0, buf = 0;
+        stage(0, 0, 0);
+        cp_async_commit();
+        while (true) {
+            int nib = ib, ncl = cl + 1;
+            if (ncl == G.cnt_in[ib]) {
+                ncl = 0;
+                ++nib;
+            }
+            const bool has_next = nib < G.p_in;
+            if (has_next) stage(nib, ncl, buf ^ 1);
+            cp_async_commit();
+            cp_async_wait_group<1>();
+            __syncthreads();
+            {
+                const float *tbase = tiles + buf * C::TILE_FLOATS + (ty * kRowsPerThread) * C::PITCH + kColsPerThread * tx;
+                const uint64_t *wp = wtab + buf * (kCob * K * K);
+#pragma unroll
+                for (int rho = 0; rho < kRowsPerThread + K - 1; ++rho) {
+                    uint64_t Pr[NP], Qr[NP - 1];
+                    const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(tbase + rho * C::PITCH);
+#pragma unroll
+                    for (int v = 0; v < NP / 2; ++v) {
+                        const ulonglong2 q = src[v];
+                        Pr[2 * v] = q.x;
+                        Pr[2 * v + 1] = q.y;
+                    }
+#pragma unroll
+                    for (int i = 0; i < NP - 1; ++i) {
+                        float a0, a1, b0, b1;
+                        unpack2(Pr[i], a0, a1);
+                        unpack2(Pr[i + 1], b0, b1);
+                        Qr[i] = pack2(a1, b0);
+                    }
+#pragma unroll
+                    for (int r = 0; r < kRowsPerThread; ++r) {
+                        const int a = rho - r;
+                        if (a < 0 || a >= K) continue;
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+#pragma unroll
+                            for (int o = 0; o < kCob; ++o) {
+                                const uint64_t w2 = wp[o * K * K + a * K + b];
+#pragma unroll
+                                for (int p2 = 0; p2 < 4; ++p2) {
+                                    // outputs (2 p2, 2 p2 + 1) read window floats XO + 2 p2 + b, + 1
+                                    constexpr int dummy = 0;
+                                    (void)dummy;
+                                    const int j0 = XO + b;
+                                    const uint64_t X = (j0 & 1) ? Qr[p2 + (j0 - 1) / 2] : Pr[p2 + j0 / 2];
+                                    acc[o][r][p2] = fma2(w2, X, acc[o][r][p2]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            if (!has_next) break;
+            ib = nib;
+            cl = ncl;
+            buf ^= 1;
+        }
+        cp_async_wait_group<0>();
+
+        // store: output channel o0 + o of block ob, rows i0 + 4 ty .., columns j0 + 8 tx ..
+        const int oo = G.ooff;
+        const uint32_t pitch_o = (uint32_t)(t.bw + 2 * oo), rows_o = (uint32_t)(t.bh + 2 * oo);
+        const int jo = t.j0 + kColsPerThread * tx;
+#pragma unroll
+        for (int o = 0; o < kCob; ++o) {
+            if (o >= oc) continue;
+            float *oplane = P.out[ob * spatial + t.shard] +
+                            ((size_t)n * G.cnt_out[ob] + (size_t)(o0 + o)) * rows_o * pitch_o;
+#pragma unroll
+            for (int r = 0; r < kRowsPerThread; ++r) {
+                const int io = t.i0 + ty * kRowsPerThread + r;
+                if (io >= t.bh || jo >= t.bw) continue;
+                float v[8];
+#pragma unroll
+                for (int p2 = 0; p2 < 4; ++p2) unpack2(acc[o][r][p2], v[2 * p2], v[2 * p2 + 1]);
+                float *dst = oplane + ((size_t)(io + oo) * pitch_o + (size_t)(jo + oo));
+                if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+                    *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4 *>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (jo + q < t.bw) dst[q] = v[q];
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Clears the ghost frame of every plane of the padded output shards (what H* leaves behind).
+struct GhostFrameParams {
+    float *shard[kConvMaxWorkers];
+    int32_t planes[kConvMaxWorkers], bh[kConvMaxWorkers], bw[kConvMaxWorkers];
+    int32_t h;
+};
+__global__ void clear_ghost_frame_kernel(const __grid_constant__ GhostFrameParams Q) {
+    const int s = blockIdx.y;
+    const int bh = Q.bh[s], bw = Q.bw[s], h = Q.h;
+    const int pw = bw + 2 * h, ph = bh + 2 * h;
+    const int frame = ph * pw - bh * bw;                  // ghost cells per plane
+    const long long total = (long long)Q.planes[s] * frame;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
+        const int plane = (int)(idx / frame);
+        int e = (int)(idx - (long long)plane * frame), row, col;
+        if (e < h * pw) {                                 // rows above the bulk
+            row = e / pw;
+            col = e - row * pw;
+        } else if (e < 2 * h * pw) {                      // rows below
+            e -= h * pw;
+            row = h + bh + e / pw;
+            col = e % pw;
+        } else {                                          // columns beside the bulk rows
+            e -= 2 * h * pw;
+            row = h + e / (2 * h);
+            const int c = e % (2 * h);
+            col = c < h ? c : bw + c;
+        }
+        Q.shard[s][((size_t)plane * ph + row) * pw + col] = 0.f;
+    }
+}
+
+template <int K, bool ADJ>
+static distdl_status_t launch_convg(const ConvGParams &G, cudaStream_t s) {
+    constexpr int smem = 2 * ConvCfg<K, ADJ>::TILE_FLOATS * 4 + 2 * kCob * K * K * 8;
+    static bool configured = false;
+    static int blocks = 0;
+    if (!configured) {
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        int dev = 0, sms = 0, per_sm = 0;
+        DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
+        DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, convg_kernel<K, ADJ>, kConvThreads, smem));
+        blocks = sms * (per_sm > 0 ? per_sm : 1);
+        configured = true;
+    }
+    const int grid = G.total_tiles < blocks ? G.total_tiles : blocks;
+    convg_kernel<K, ADJ><<<grid, kConvThreads, smem, s>>>(G);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+// px: partition of the tensor with n_ci channels (x, dx); the other tensor (y, dy) has n_co channels on pco
+// blocks and the same spatial partition.  Forward: in = x (padded), out = y (bulk-shaped); adjoint: in = dy
+// (bulk-shaped), out = dx (padded, ghosts cleared).
+static distdl_status_t convg_impl(const distdl_partition *px, int64_t nco, int32_t pco, const void *const *in,
+                                  const void *const *w, const void *const *bias, int32_t kh, int32_t kw,
+                                  void *const *out, void *stream, bool adj, const char *what) {
+    clear_error();
+    if (!px || !in || !w || !out) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    if (px->rank != 4 || px->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-4 F32 partition", what);
+    if (px->any_periodic()) return fail(DISTDL_ERR_UNSUPPORTED, "%s: periodic partitions are not supported by the fused layers", what);
+    if (px->pshape[0] != 1) return fail(DISTDL_ERR_UNSUPPORTED, "%s: the batch dimension may not be partitioned", what);
+    if (kh != kw || (kh != 3 && kh != 5 && kh != 7))
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: kernel %d x %d (supported: 3x3, 5x5, 7x7)", what, kh, kw);
+    const int32_t pci = px->pshape[1], ph = px->pshape[2], pw = px->pshape[3];
+    if (pco < 1 || nco < pco) return fail(DISTDL_ERR_SHAPE, "%s: %lld output channels on %d blocks", what, (long long)nco, pco);
+    if (pci > kMaxChanBlocks || pco > kMaxChanBlocks)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d blocks of a channel partition", what, kMaxChanBlocks);
+    if ((int64_t)std::max(pci, pco) * ph * pw > kConvMaxWorkers)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d shards of one tensor", what, kConvMaxWorkers);
+    const int h = kh / 2;
+    for (int k = 0; k < 4; ++k)
+        for (int32_t c = 0; c < px->pshape[k]; ++c) {
+            const int want = k < 2 ? 0 : h;
+            if (px->hlo[k][c] != want || px->hhi[k][c] != want)
+                return fail(DISTDL_ERR_SHAPE, "%s: halo widths must be 0,0,%d,%d on every side", what, h, h);
+        }
+    ConvGParams G;
+    memset(&G, 0, sizeof(G));
+    ConvParams &P = G.base;
+    int64_t max_bh = 0, max_bw = 0;
+    for (int32_t r = 0; r < ph; ++r) max_bh = std::max<int64_t>(max_bh, P.bh[r] = (int32_t)px->size[2][r]);
+    for (int32_t c = 0; c < pw; ++c) max_bw = std::max<int64_t>(max_bw, P.bw[c] = (int32_t)px->size[3][c]);
+    P.ph_workers = ph;
+    P.pw_workers = pw;
+    P.tiles_x = (int32_t)((max_bw + kTileW - 1) / kTileW);
+    G.tiles_y = (int32_t)((max_bh + kTileH - 1) / kTileH);
+    conv_set_divisor(P, 0, (uint32_t)P.tiles_x);
+    conv_set_divisor(P, 1, (uint32_t)pw);
+    conv_set_divisor(P, 2, (uint32_t)G.tiles_y);
+    conv_set_divisor(P, 3, (uint32_t)ph);
+    // channel blocks: the evenly split n_ci (from the partition) and n_co
+    std::vector<int64_t> co_start, co_size;
+    split_evenly(nco, pco, co_start, co_size);
+    const int32_t p_out = adj ? pci : pco, p_in = adj ? pco : pci;
+    for (int32_t b = 0; b < pci; ++b) (adj ? G.cnt_out : G.cnt_in)[b] = (int32_t)px->size[1][b];
+    for (int32_t b = 0; b < pco; ++b) (adj ? G.cnt_in : G.cnt_out)[b] = (int32_t)co_size[b];
+    G.p_out = p_out;
+    G.p_in = p_in;
+    G.pci = pci;
+    int groups = 0;
+    for (int32_t b = 0; b < p_out; ++b)
+        for (int32_t f = 0; f < G.cnt_out[b]; f += kCob) {
+            if (groups == kMaxGroups || f > 255) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many output channels", what);
+            G.grp_block[groups] = (uint8_t)b;
+            G.grp_first[groups] = (uint8_t)f;
+            G.grp_count[groups] = (uint8_t)std::min<int32_t>(kCob, G.cnt_out[b] - f);
+            ++groups;
+        }
+    G.groups = groups;
+    G.ooff = adj ? h : 0;
+    const int64_t total = (int64_t)P.tiles_x * G.tiles_y * ph * pw * px->global_shape[0] * groups;
+    if (total >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
+    G.total_tiles = (int32_t)total;
+    const int spatial = ph * pw;
+    for (int32_t k = 0; k < p_in * spatial; ++k) {
+        if (!in[k]) return fail(DISTDL_ERR_INVALID_ARG, "%s: input shard %d is NULL", what, k);
+        if (!aligned16(in[k])) return fail(DISTDL_ERR_ALIGNMENT, "%s: input shard %d is not 16-byte aligned", what, k);
+        P.in[k] = (const float *)in[k];
+    }
+    for (int32_t k = 0; k < p_out * spatial; ++k) {
+        if (!out[k]) return fail(DISTDL_ERR_INVALID_ARG, "%s: output shard %d is NULL", what, k);
+        if (!aligned16(out[k])) return fail(DISTDL_ERR_ALIGNMENT, "%s: output shard %d is not 16-byte aligned", what, k);
+        P.out[k] = (float *)out[k];
+    }
+    for (int32_t k = 0; k < pco * pci; ++k) {
+        if (!w[k]) return fail(DISTDL_ERR_INVALID_ARG, "%s: weight block %d is NULL", what, k);
+        G.w[k] = (const float *)w[k];
+    }
+    if (!adj && bias)
+        for (int32_t b = 0; b < pco; ++b) G.bias[b] = (const float *)bias[b];
+    cudaStream_t s = (cudaStream_t)stream;
+    distdl_status_t st;
+    if (!adj) st = kh == 3 ? launch_convg<3, false>(G, s) : kh == 5 ? launch_convg<5, false>(G, s) : launch_convg<7, false>(G, s);
+    else st = kh == 3 ? launch_convg<3, true>(G, s) : kh == 5 ? launch_convg<5, true>(G, s) : launch_convg<7, true>(G, s);
+    if (st != DISTDL_OK || !adj) return st;
+    // adjoint: the ghosts of dx are zero, as H* leaves them
+    GhostFrameParams Q;
+    memset(&Q, 0, sizeof(Q));
+    Q.h = h;
+    for (int32_t b = 0; b < pci; ++b)
+        for (int32_t r = 0; r < ph; ++r)
+            for (int32_t c = 0; c < pw; ++c) {
+                const int k = (b * ph + r) * pw + c;
+                Q.shard[k] = (float *)out[k];
+                Q.planes[k] = (int32_t)(px->global_shape[0] * px->size[1][b]);
+                Q.bh[k] = P.bh[r];
+                Q.bw[k] = P.bw[c];
+            }
+    clear_ghost_frame_kernel<<<dim3(64, (unsigned)(pci * spatial)), 256, 0, s>>>(Q);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Parameter gradients of the layer (adjoint convolution algorithm, Section 4 "Sparse layers"):
 //   dw^_k[c,a,b] = sum_{n,i,j} dy_k[n,c,i,j] * (H x)_k[n,c,i+a,j+b],   db^_k[c] = sum dy_k[n,c,i,j],
 //   dw = R_k dw^_k,  db = R_k db^_k      (every worker holds a copy of the kernel).
@@ -1337,6 +1671,16 @@ static distdl_status_t launch_grad(const distdl_partition *p, const ConvGradPara
 }
 
 }  // namespace distdl
+
+extern "C" distdl_status_t distdl_convg_fwd(const distdl_partition_t *px, int64_t nco, int32_t pco, const void *const *x,
+                                            const void *const *w, const void *const *bias, int32_t kh, int32_t kw,
+                                            void *const *y, void *stream) {
+    return distdl::convg_impl(px, nco, pco, x, w, bias, kh, kw, y, stream, false, "convg_fwd");
+}
+extern "C" distdl_status_t distdl_convg_adj(const distdl_partition_t *px, int64_t nco, int32_t pco, const void *const *dy,
+                                            const void *const *w, int32_t kh, int32_t kw, void *const *dx, void *stream) {
+    return distdl::convg_impl(px, nco, pco, dy, w, nullptr, kh, kw, dx, stream, true, "convg_adj");
+}
 
 extern "C" distdl_status_t distdl_conv_adj_params_workspace(const distdl_partition_t *p, int32_t kh, int32_t kw,
                                                             int64_t *bytes) {

@@ -450,6 +450,71 @@ def test_conv_param_gradients(case, integer):
 
 
 # --------------------------------------------------------------------------
+# Generalized convolution layer (channel partitions)
+# --------------------------------------------------------------------------
+
+CONVG_CASES = [
+    # N, n_ci, n_co, H, W, P_ci, P_co, P_0, P_1, k
+    (2, 4, 6, 9, 10, 2, 3, 2, 2, 3),
+    (1, 5, 3, 8, 7, 2, 2, 1, 2, 5),          # uneven channel blocks, odd channel counts (a group of one)
+    (1, 3, 4, 40, 150, 1, 1, 1, 1, 5),       # two tile rows and columns in one shard
+    (2, 3, 5, 70, 264, 3, 2, 2, 2, 5),       # 16-byte aligned rows, ragged tiles
+    (1, 2, 2, 66, 260, 2, 1, 2, 2, 7),       # short last tile row and column
+    (1, 4, 4, 34, 131, 2, 2, 1, 1, 3),
+]
+
+
+@pytest.mark.parametrize("case", CONVG_CASES, ids=[str(c) for c in CONVG_CASES])
+@pytest.mark.parametrize("integer", [True, False], ids=["int", "normal"])
+def test_generalized_conv_fwd_and_adj(case, integer):
+    N, nci, nco, H, W, pci, pco, p0, p1, k = case
+    h = k // 2
+    xpart = oracle.Partition((N, nci, H, W), (1, pci, p0, p1), (0, 0, h, h), (0, 0, h, h))
+    ypart = oracle.Partition((N, nco, H, W), (1, pco, p0, p1))
+    gpart = distdl.Partition((N, nci, H, W), (1, pci, p0, p1), (0, 0, h, h), (0, 0, h, h))
+    gen = (lambda shp, seed, std=1.0: inputs.integers(shp, seed, -2, 3)) if integer else inputs.normal
+    xg, wg, bg = gen((N, nci, H, W), 61), gen((nco, nci, k, k), 62, 0.2), gen((nco,), 63)
+    dyg = gen((N, nco, H, W), 64)
+    cs_i, cz_i = oracle.balanced_split(nco, pco)
+    cs_j, cz_j = oracle.balanced_split(nci, pci)
+    wb = [np.ascontiguousarray(wg[cs_i[i]:cs_i[i] + cz_i[i], cs_j[j]:cs_j[j] + cz_j[j]]) for i in range(pco) for j in range(pci)]
+    bb = [np.ascontiguousarray(bg[cs_i[i]:cs_i[i] + cz_i[i]]) for i in range(pco)]
+    x = oracle.scatter_global(xpart, xg, fill=lambda wk: np.full(xpart.padded_shape(wk), 1e30, dtype=np.float32))
+    dy = oracle.scatter_global(ypart, dyg)
+    xs, dys = [dev(a) for a in x], [dev(a) for a in dy]
+    wd = [dev(a) for a in wb]
+    ys = [torch.full(ypart.padded_shape(wk), -7.0, device=DEV) for wk in range(ypart.num_workers)]
+    dxs = [torch.full(xpart.padded_shape(wk), 3.0, device=DEV) for wk in range(xpart.num_workers)]
+    distdl.convg_fwd(gpart, nco, pco, xs, wd, [dev(b) for b in bb], ys)
+    distdl.convg_adj(gpart, nco, pco, dys, wd, dxs)
+    torch.cuda.synchronize()
+    xz = oracle.scatter_global(xpart, xg)
+    yref = oracle.convg_fwd(xpart, nco, pco, xz, wb, bb)
+    dxref = oracle.convg_adj(xpart, nco, pco, dy, wb)
+    for wk in range(xpart.num_workers):
+        assert same_bits(host(xs[wk]), x[wk])            # x, ghosts included, is left untouched
+        mask = np.ones(xpart.padded_shape(wk), dtype=bool)
+        mask[xpart.bulk_slices(wk)] = False
+        assert not host(dxs[wk])[mask].any()             # ghosts of dx are zero, as H* leaves them
+    if integer:
+        # small integers: every product and partial sum is exact in fp32, any order
+        for a, b in zip(ys + dxs, yref + dxref):
+            assert np.array_equal(host(a), b)
+        return
+    # n_ci * K * K (adjoint: n_co * K * K) FMA roundings and the oracle's own rounding of its fp64 sum to fp32
+    ymag = oracle.convg_fwd(xpart, nco, pco, [np.abs(a) for a in xz], [np.abs(a) for a in wb], [np.abs(b) for b in bb])
+    dxmag = oracle.convg_adj(xpart, nco, pco, [np.abs(a) for a in dy], [np.abs(a) for a in wb])
+    for got, ref, mag, terms in ((ys, yref, ymag, nci * k * k + 1), (dxs, dxref, dxmag, nco * k * k)):
+        for a, b, m in zip(got, ref, mag):
+            assert np.all(np.abs(host(a).astype(np.float64) - b) <= (terms + 2) * 2.0 ** -24 * m + 1e-30)
+    y0 = [torch.empty_like(t) for t in ys]
+    distdl.convg_fwd(gpart, nco, pco, xs, wd, None, y0)
+    torch.cuda.synchronize()
+    r = oracle.adjoint_test_ratio([host(t) for t in y0], dy, xz, [host(t) for t in dxs])
+    assert r < 1e-5
+
+
+# --------------------------------------------------------------------------
 # 3-D star-stencil layer
 # --------------------------------------------------------------------------
 
