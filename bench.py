@@ -184,6 +184,19 @@ class Workload:
             ("stencil3d_adj", lambda: d.stencil3d_adj(self.spart, self.s_y, self.s_w, self.s_dx), st_bytes + ghost_b,
              2 * 27 * cells, 1, "hbm"),
         ]
+        # generalized convolution: 16 -> 16 channels, 5 x 5, channel partitions 2 x 2, feature space 2 x 2
+        gN = 1 if small else 4
+        self.gpart = d.Partition((gN, 16, 1024, 1024), (1, 2, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2))
+        self.g_x = [n(*self.gpart.padded_shape(w)) for w in range(8)]
+        self.g_y = [torch.empty(gN, 8, 512, 512, device=dev) for _ in range(8)]
+        self.g_dx = [torch.empty(*self.gpart.padded_shape(w), device=dev) for w in range(8)]
+        self.g_w = [n(8, 8, 5, 5) * 0.05 for _ in range(4)]
+        g_flops = 2 * 25 * 16 * 16 * gN * 1024 * 1024
+        g_bytes = 2 * gN * 16 * 1024 * 1024 * 4
+        self.extra_ops += [
+            ("convg_fwd", lambda: d.convg_fwd(self.gpart, 16, 2, self.g_x, self.g_w, None, self.g_y), g_bytes, g_flops, 1, "alu"),
+            ("convg_adj", lambda: d.convg_adj(self.gpart, 16, 2, self.g_y, self.g_w, self.g_dx), g_bytes, g_flops, 2, "alu"),
+        ]
         self.extra_ops += [
             ("conv_adj_params", lambda: d.conv_adj_params(self.cpart, self.c_x, self.c_dy, (5, 5), self.c_dw, self.c_db,
                                                           self.c_ws), conv_bytes, 2 * 25 * self._conv_outputs(), 2, "hbm"),
@@ -545,9 +558,13 @@ def main():
                 entry["frac_tensor"] = round(flops / ms / 1e9 / peaks["bf16_sustained"], 4)
             ops[name] = entry
         extra = {}
-        for (name, _, nbytes, _, _, bound), ms in zip(wl.extra_ops, extra_ms):
+        for (name, _, nbytes, flops, _, bound), ms in zip(wl.extra_ops, extra_ms):
             extra[name] = {"ms": round(ms, 5), "gbs": round(nbytes / ms / 1e6, 1), "bound": bound,
                            "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm"], 4)}
+            if bound == "alu":
+                # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock (packed pairs issue at half rate)
+                extra[name]["tflops"] = round(flops / ms / 1e9, 2)
+                extra[name]["frac_alu"] = round(flops / ms / 1e9 / FP32_PEAK_TFLOPS, 4)
         # dominant kernel = the launch with the largest share of the step
         top = max(range(nops), key=lambda i: per_op_ms[i])
         tname, _, tbytes, _, _, tbound = wl.ops[top]
@@ -574,7 +591,8 @@ def main():
             "extra_ops": {"note": "timed separately, not part of value: 3x3 max pooling, stride 2, padding 1 on fp32 "
                                   "16x16x1024x1024 over 4x4 workers (H + local kernel, local adjoint + H*); parameter "
                                   "gradients of the step's convolution (dw, db) and affine layer (dW, db); fused halo + radius-4 star stencil "
-                                  "on the step's 512^3 volume (4x4x4 workers); generalized "
+                                  "on the step's 512^3 volume (4x4x4 workers); generalized convolution 16 -> 16 channels, 5x5, fp32 "
+                                  "4x16x1024x1024 on channel partitions 2x2 and 2x2 feature-space workers; generalized "
                                   "all-to-all of fp32 8192x8192 between 8 row blocks and 8 column blocks",
                           **extra},
             "roofline": roofline,
@@ -597,6 +615,8 @@ def main():
 # the quarter-size case are scaled by 4: traffic grows with the number of planes / rows); None for a
 # kernel whose counters were not meaningful (the broadcast's output was still in L2 when the short
 # capture ended) or that changed since its counters were taken.
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.4
+
 NCU_TRAFFIC = {
     "broadcast_fwd": None,
     "sumreduce_fwd": 4 * (134224128 + 5519616),

@@ -551,7 +551,7 @@ __device__ __forceinline__ void for_each_patch_cell(const ConvTile &t, F f) {
 // Fetches the halo strips of tile t (cells that belong to neighbouring shards, or zeros outside the
 // tensor) into the side buffer, cell by cell.
 template <int K, bool ADJ>
-__device__ __forceinline__ void stage_halo_strips(const ConvParams &P, const ConvTile &t, float *side) {
+__device__ __forceinline__ void stage_halo_strips(const ConvParams &P, const ConvTile &t, float *side, int wofs = 0) {
     using C = ConvCfg<K, ADJ>;
     for_each_patch_cell<K, ADJ>(t, [&](int q, int ry, int s) {
         int i = t.i0 - C::PH + ry, rr = t.r;
@@ -585,7 +585,7 @@ __device__ __forceinline__ void stage_halo_strips(const ConvParams &P, const Con
             const uint32_t pitch_n = (uint32_t)(P.bw[cc] + 2 * C::IOFF);
             const uint32_t off = ((uint32_t)t.plane * (uint32_t)(P.bh[rr] + 2 * C::IOFF) + (uint32_t)(i + C::IOFF)) * pitch_n +
                                  (uint32_t)(C::IOFF + j);
-            cp_async4(side + q, P.in[rr * P.pw_workers + cc] + off);
+            cp_async4(side + q, P.in[wofs + rr * P.pw_workers + cc] + off);
         } else {
             side[q] = 0.f;
         }
@@ -877,19 +877,132 @@ struct ConvGParams {
     int32_t ooff;                           // ghost width of the output layout
 };
 
+// One input channel's contribution to the block's kCob x 32 x 128 outputs: per thread 4 x 8 pixels of kCob
+// channels as packed pairs.  wp: K * K * kCob (w, w) pairs of this input channel, [tap][channel].
 template <int K, bool ADJ>
-__global__ void __launch_bounds__(kConvThreads, 3)
-convg_kernel(const __grid_constant__ ConvGParams G) {
+__device__ __forceinline__ void convg_accumulate(const float *tile, const uint64_t *wp, uint64_t (&acc)[kCob][kRowsPerThread][4]) {
     using C = ConvCfg<K, ADJ>;
     constexpr int XO = C::PADL - C::PH;                         // tile column of the first input of output column 0
     constexpr int NF2 = ((XO + kColsPerThread + K - 1 + 3) / 4) * 4;   // floats of a thread's (aligned) window
     constexpr int NP = NF2 / 2;
     static_assert(kTileW - kColsPerThread + NF2 <= C::PITCH, "window beyond the tile row");
-    extern __shared__ __align__(16) float smem[];               // two x tiles, then two weight tables
-    float *tiles = smem;
-    uint64_t *wtab = reinterpret_cast<uint64_t *>(smem + 2 * C::TILE_FLOATS);   // [2][kCob * K * K] (w, w) pairs
+    static_assert(kCob % 2 == 0, "weight pairs are read two channels at a time");
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const float *tbase = tile + (ty * kRowsPerThread) * C::PITCH + kColsPerThread * tx;
+#pragma unroll
+    for (int rho = 0; rho < kRowsPerThread + K - 1; ++rho) {
+        uint64_t Pr[NP], Qr[NP - 1];
+        const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(tbase + rho * C::PITCH);
+#pragma unroll
+        for (int v = 0; v < NP / 2; ++v) {
+            const ulonglong2 q = src[v];
+            Pr[2 * v] = q.x;
+            Pr[2 * v + 1] = q.y;
+        }
+#pragma unroll
+        for (int i = 0; i < NP - 1; ++i) {
+            float a0, a1, b0, b1;
+            unpack2(Pr[i], a0, a1);
+            unpack2(Pr[i + 1], b0, b1);
+            Qr[i] = pack2(a1, b0);
+        }
+#pragma unroll
+        for (int r = 0; r < kRowsPerThread; ++r) {
+            const int a = rho - r;
+            if (a < 0 || a >= K) continue;
+#pragma unroll
+            for (int b = 0; b < K; ++b) {
+                // the pairs of all kCob channels of one tap sit side by side: one 16-byte read for two channels
+                uint64_t w2[kCob];
+#pragma unroll
+                for (int o = 0; o < kCob; o += 2) {
+                    const ulonglong2 q = *reinterpret_cast<const ulonglong2 *>(wp + (a * K + b) * kCob + o);
+                    w2[o] = q.x;
+                    w2[o + 1] = q.y;
+                }
+                // outputs (2 p2, 2 p2 + 1) read window floats XO + 2 p2 + b, + 1
+                const int j0 = XO + b;
+#pragma unroll
+                for (int p2 = 0; p2 < 4; ++p2) {
+                    const uint64_t X = (j0 & 1) ? Qr[p2 + (j0 - 1) / 2] : Pr[p2 + j0 / 2];
+#pragma unroll
+                    for (int o = 0; o < kCob; ++o) acc[o][r][p2] = fma2(w2[o], X, acc[o][r][p2]);
+                }
+            }
+        }
+    }
+}
+
+// (w, w) pairs of input channel (ib, cl) for the output channels of group (ob, o0, oc); layout [tap][channel]
+template <int K, bool ADJ>
+__device__ __forceinline__ void convg_stage_weights(const ConvGParams &G, int ob, int o0, int oc, int ib, int cl, uint64_t *dst) {
+    if ((int)threadIdx.x < kCob * K * K) {
+        const int tap = threadIdx.x / kCob, o = threadIdx.x - tap * kCob;
+        float w = 0.f;
+        if (o < oc) {
+            const float *blk = ADJ ? G.w[ib * G.pci + ob] : G.w[ob * G.pci + ib];
+            const int s_out = ADJ ? K * K : G.cnt_in[ib] * K * K, s_in = ADJ ? G.cnt_out[ob] * K * K : K * K;
+            w = __ldg(blk + (size_t)(o0 + o) * s_out + (size_t)cl * s_in + (ADJ ? K * K - 1 - tap : tap));   // adjoint: rotated
+        }
+        reinterpret_cast<float2 *>(dst)[threadIdx.x] = make_float2(w, w);
+    }
+}
+
+template <int K, bool ADJ>
+__device__ __forceinline__ void convg_store(const ConvGParams &G, const ConvTile &t, int n, int ob, int o0, int oc,
+                                            const uint64_t (&acc)[kCob][kRowsPerThread][4]) {
     const ConvParams &P = G.base;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int spatial = P.ph_workers * P.pw_workers;
+    const int oo = G.ooff;
+    const uint32_t pitch_o = (uint32_t)(t.bw + 2 * oo), rows_o = (uint32_t)(t.bh + 2 * oo);
+    const int jo = t.j0 + kColsPerThread * tx;
+#pragma unroll
+    for (int o = 0; o < kCob; ++o) {
+        if (o >= oc) continue;
+        float *oplane = P.out[ob * spatial + t.shard] + ((size_t)n * G.cnt_out[ob] + (size_t)(o0 + o)) * rows_o * pitch_o;
+#pragma unroll
+        for (int r = 0; r < kRowsPerThread; ++r) {
+            const int io = t.i0 + ty * kRowsPerThread + r;
+            if (io >= t.bh || jo >= t.bw) continue;
+            float v[8];
+#pragma unroll
+            for (int p2 = 0; p2 < 4; ++p2) unpack2(acc[o][r][p2], v[2 * p2], v[2 * p2 + 1]);
+            float *dst = oplane + ((size_t)(io + oo) * pitch_o + (size_t)(jo + oo));
+            if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+                *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4 *>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (jo + q < t.bw) dst[q] = v[q];
+            }
+        }
+    }
+}
+
+template <int K, bool ADJ>
+__device__ __forceinline__ void convg_init(const ConvGParams &G, int ob, int o0, int oc, uint64_t (&acc)[kCob][kRowsPerThread][4]) {
+#pragma unroll
+    for (int o = 0; o < kCob; ++o) {
+        float b = 0.f;
+        if (!ADJ && G.bias[ob] && o < oc) b = __ldg(G.bias[ob] + o0 + o);
+#pragma unroll
+        for (int r = 0; r < kRowsPerThread; ++r)
+#pragma unroll
+            for (int p2 = 0; p2 < 4; ++p2) acc[o][r][p2] = pack2(b, b);
+    }
+}
+
+// General variant: tiles staged by per-thread asynchronous copies (any row pitch, any number of shards).
+template <int K, bool ADJ>
+__global__ void __launch_bounds__(kConvThreads, 3)
+convg_kernel(const __grid_constant__ ConvGParams G) {
+    using C = ConvCfg<K, ADJ>;
+    extern __shared__ __align__(16) float smem[];               // two x tiles, then two weight tables
+    float *tiles = smem;
+    uint64_t *wtab = reinterpret_cast<uint64_t *>(smem + 2 * C::TILE_FLOATS);   // [2][K * K][kCob] (w, w) pairs
+    const ConvParams &P = G.base;
     const int spatial = P.ph_workers * P.pw_workers;
 
     for (int tile = blockIdx.x; tile < G.total_tiles; tile += gridDim.x) {
@@ -897,34 +1010,14 @@ convg_kernel(const __grid_constant__ ConvGParams G) {
         if (!t.valid) continue;                                  // the same for every thread of the block
         const int n = t.plane / G.groups, g = t.plane - n * G.groups;
         const int ob = G.grp_block[g], o0 = G.grp_first[g], oc = G.grp_count[g];
-
         uint64_t acc[kCob][kRowsPerThread][4];
-#pragma unroll
-        for (int o = 0; o < kCob; ++o) {
-            float b = 0.f;
-            if (!ADJ && G.bias[ob] && o < oc) b = __ldg(G.bias[ob] + o0 + o);
-#pragma unroll
-            for (int r = 0; r < kRowsPerThread; ++r)
-#pragma unroll
-                for (int p2 = 0; p2 < 4; ++p2) acc[o][r][p2] = pack2(b, b);
-        }
-
+        convg_init<K, ADJ>(G, ob, o0, oc, acc);
         // the channels of the reduced partition: block after block, channel after channel
         auto stage = [&](int ib, int cl, int buf) {
             ConvTile ti = t;
             ti.plane = n * G.cnt_in[ib] + cl;
             stage_tile<K, ADJ>(P, ti, tiles + buf * C::TILE_FLOATS, ib * spatial);
-            // weights of (output channel o0 + o, this input channel), as (w, w) pairs; adjoint: rotated
-            if ((int)threadIdx.x < kCob * K * K) {
-                const int o = threadIdx.x / (K * K), tap = threadIdx.x - o * (K * K);
-                float w = 0.f;
-                if (o < oc) {
-                    const float *blk = ADJ ? G.w[ib * G.pci + ob] : G.w[ob * G.pci + ib];
-                    const int s_out = ADJ ? K * K : G.cnt_in[ib] * K * K, s_in = ADJ ? G.cnt_out[ob] * K * K : K * K;
-                    w = __ldg(blk + (size_t)(o0 + o) * s_out + (size_t)cl * s_in + (ADJ ? K * K - 1 - tap : tap));
-                }
-                reinterpret_cast<float2 *>(wtab + buf * (kCob * K * K))[threadIdx.x] = make_float2(w, w);
-            }
+            convg_stage_weights<K, ADJ>(G, ob, o0, oc, ib, cl, wtab + buf * (kCob * K * K));
         };
         int ib = 0, cl = 0, buf = 0;
         stage(0, 0, 0);
@@ -940,49 +1033,7 @@ convg_kernel(const __grid_constant__ ConvGParams G) {
             cp_async_commit();
             cp_async_wait_group<1>();
             __syncthreads();
-            {
-                const float *tbase = tiles + buf * C::TILE_FLOATS + (ty * kRowsPerThread) * C::PITCH + kColsPerThread * tx;
-                const uint64_t *wp = wtab + buf * (kCob * K * K);
-#pragma unroll
-                for (int rho = 0; rho < kRowsPerThread + K - 1; ++rho) {
-                    uint64_t Pr[NP], Qr[NP - 1];
-                    const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(tbase + rho * C::PITCH);
-#pragma unroll
-                    for (int v = 0; v < NP / 2; ++v) {
-                        const ulonglong2 q = src[v];
-                        Pr[2 * v] = q.x;
-                        Pr[2 * v + 1] = q.y;
-                    }
-#pragma unroll
-                    for (int i = 0; i < NP - 1; ++i) {
-                        float a0, a1, b0, b1;
-                        unpack2(Pr[i], a0, a1);
-                        unpack2(Pr[i + 1], b0, b1);
-                        Qr[i] = pack2(a1, b0);
-                    }
-#pragma unroll
-                    for (int r = 0; r < kRowsPerThread; ++r) {
-                        const int a = rho - r;
-                        if (a < 0 || a >= K) continue;
-#pragma unroll
-                        for (int b = 0; b < K; ++b) {
-#pragma unroll
-                            for (int o = 0; o < kCob; ++o) {
-                                const uint64_t w2 = wp[o * K * K + a * K + b];
-#pragma unroll
-                                for (int p2 = 0; p2 < 4; ++p2) {
-                                    // outputs (2 p2, 2 p2 + 1) read window floats XO + 2 p2 + b, + 1
-                                    constexpr int dummy = 0;
-                                    (void)dummy;
-                                    const int j0 = XO + b;
-                                    const uint64_t X = (j0 & 1) ? Qr[p2 + (j0 - 1) / 2] : Pr[p2 + j0 / 2];
-                                    acc[o][r][p2] = fma2(w2, X, acc[o][r][p2]);
-                                }
-                            }
-                        }
-                    }
-                }
-            }
+            convg_accumulate<K, ADJ>(tiles + buf * C::TILE_FLOATS, wtab + buf * (kCob * K * K), acc);
             __syncthreads();
             if (!has_next) break;
             ib = nib;
@@ -990,34 +1041,115 @@ convg_kernel(const __grid_constant__ ConvGParams G) {
             buf ^= 1;
         }
         cp_async_wait_group<0>();
+        convg_store<K, ADJ>(G, t, n, ob, o0, oc, acc);
+        __syncthreads();
+    }
+}
 
-        // store: output channel o0 + o of block ob, rows i0 + 4 ty .., columns j0 + 8 tx ..
-        const int oo = G.ooff;
-        const uint32_t pitch_o = (uint32_t)(t.bw + 2 * oo), rows_o = (uint32_t)(t.bh + 2 * oo);
-        const int jo = t.j0 + kColsPerThread * tx;
-#pragma unroll
-        for (int o = 0; o < kCob; ++o) {
-            if (o >= oc) continue;
-            float *oplane = P.out[ob * spatial + t.shard] +
-                            ((size_t)n * G.cnt_out[ob] + (size_t)(o0 + o)) * rows_o * pitch_o;
-#pragma unroll
-            for (int r = 0; r < kRowsPerThread; ++r) {
-                const int io = t.i0 + ty * kRowsPerThread + r;
-                if (io >= t.bh || jo >= t.bw) continue;
-                float v[8];
-#pragma unroll
-                for (int p2 = 0; p2 < 4; ++p2) unpack2(acc[o][r][p2], v[2 * p2], v[2 * p2 + 1]);
-                float *dst = oplane + ((size_t)(io + oo) * pitch_o + (size_t)(jo + oo));
-                if (jo + 7 < t.bw && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
-                    *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-                    *reinterpret_cast<float4 *>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        if (jo + q < t.bw) dst[q] = v[q];
-                }
+// TMA variant (at most kConvGTmaShards input shards, rows of whole 16-byte units): the tile body of every
+// input channel arrives by one bulk tensor copy, the halo strips cell by cell into a side buffer.
+constexpr int kConvGTmaShards = 32;
+struct ConvGTmaParams {
+    ConvGParams g;
+    CUtensorMap in_map[kConvGTmaShards];
+};
+
+template <int K, bool ADJ>
+__global__ void __launch_bounds__(kConvThreads, 3)
+convg_tma_kernel(const __grid_constant__ ConvGTmaParams Q) {
+    using C = ConvCfg<K, ADJ>;
+    using T = ConvTmaCfg<K, ADJ>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    float *tiles = reinterpret_cast<float *>(smem_raw + (((raw + 127u) & ~127u) - raw));
+    float *sides = tiles + 2 * T::TILE_STRIDE;
+    uint64_t *wtab = reinterpret_cast<uint64_t *>(sides + 2 * T::SIDE_STRIDE);          // [2][K * K][kCob]
+    const uint32_t bars = smem_u32(wtab + 2 * kCob * K * K);
+    const ConvGParams &G = Q.g;
+    const ConvParams &P = G.base;
+    const int spatial = P.ph_workers * P.pw_workers;
+    if (threadIdx.x == 0) {
+        mbar_init(bars, 1);
+        mbar_init(bars + 8, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    uint32_t phase0 = 0, phase1 = 0;
+    bool failed = false;
+
+    for (int tile = blockIdx.x; tile < G.total_tiles && !failed; tile += gridDim.x) {
+        ConvTile t = decode_tile(P, tile, G.tiles_y, 0);
+        if (!t.valid) continue;
+        const int n = t.plane / G.groups, g = t.plane - n * G.groups;
+        const int ob = G.grp_block[g], o0 = G.grp_first[g], oc = G.grp_count[g];
+        uint64_t acc[kCob][kRowsPerThread][4];
+        convg_init<K, ADJ>(G, ob, o0, oc, acc);
+        auto stage = [&](int ib, int cl, int buf) {
+            ConvTile ti = t;
+            ti.plane = n * G.cnt_in[ib] + cl;
+            if (threadIdx.x == 0) {
+                fence_proxy_async();
+                mbar_expect_tx(bars + 8 * buf, T::BOX_BYTES);
+                // forward: padded coordinates (bulk column j sits at j + PH); adjoint: bulk coordinates
+                const int x = ADJ ? t.j0 - C::PADL : t.j0;
+                const int y = ADJ ? t.i0 - C::PH : t.i0;
+                tma_load_3d(smem_u32(tiles + buf * T::TILE_STRIDE), &Q.in_map[ib * spatial + t.shard], x, y, ti.plane, bars + 8 * buf);
             }
+            stage_halo_strips<K, ADJ>(P, ti, sides + buf * T::SIDE_STRIDE, ib * spatial);
+            convg_stage_weights<K, ADJ>(G, ob, o0, oc, ib, cl, wtab + buf * (kCob * K * K));
+        };
+        int ib = 0, cl = 0, buf = 0;
+        stage(0, 0, 0);
+        cp_async_commit();
+        while (true) {
+            int nib = ib, ncl = cl + 1;
+            if (ncl == G.cnt_in[ib]) {
+                ncl = 0;
+                ++nib;
+            }
+            const bool has_next = nib < G.p_in;
+            if (has_next) stage(nib, ncl, buf ^ 1);
+            cp_async_commit();
+            cp_async_wait_group<1>();
+            bool ok = true;
+            {
+                const uint32_t bar = bars + 8 * buf, parity = buf ? phase1 : phase0;
+                if (!mbar_try_wait(bar, parity)) {
+                    const uint64_t t0 = global_timer();
+                    while (!mbar_try_wait(bar, parity)) {
+                        if (global_timer() - t0 > kConvWaitLimitNs) {
+                            ok = false;
+                            break;
+                        }
+                    }
+                }
+                if (buf) phase1 ^= 1; else phase0 ^= 1;
+            }
+            if (__syncthreads_or(!ok)) {
+                if (threadIdx.x == 0) {
+                    atomicExch(&g_conv_status, (int)DISTDL_ERR_TIMEOUT);
+                    const uint64_t t0 = global_timer();
+                    while (global_timer() - t0 < 1000000ull) {}
+                }
+                failed = true;
+                break;
+            }
+            float *tl = tiles + buf * T::TILE_STRIDE;
+            {
+                const float *sd = sides + buf * T::SIDE_STRIDE;
+                for_each_patch_cell<K, ADJ>(t, [&](int q, int ry, int s2) { tl[ry * C::PITCH + s2] = sd[q]; });
+            }
+            __syncthreads();
+            convg_accumulate<K, ADJ>(tl, wtab + buf * (kCob * K * K), acc);
+            __syncthreads();
+            if (!has_next) break;
+            ib = nib;
+            cl = ncl;
+            buf ^= 1;
         }
+        cp_async_wait_group<0>();
+        if (failed) break;
+        convg_store<K, ADJ>(G, t, n, ob, o0, oc, acc);
         __syncthreads();
     }
 }
@@ -1055,21 +1187,52 @@ __global__ void clear_ghost_frame_kernel(const __grid_constant__ GhostFrameParam
 }
 
 template <int K, bool ADJ>
-static distdl_status_t launch_convg(const ConvGParams &G, cudaStream_t s) {
-    constexpr int smem = 2 * ConvCfg<K, ADJ>::TILE_FLOATS * 4 + 2 * kCob * K * K * 8;
+static distdl_status_t launch_convg(const ConvGParams &G, int in_shards, const int64_t *in_planes, cudaStream_t s) {
+    using C = ConvCfg<K, ADJ>;
+    using T = ConvTmaCfg<K, ADJ>;
+    constexpr int smem_plain = 2 * C::TILE_FLOATS * 4 + 2 * kCob * K * K * 8;
+    constexpr int smem_tma = 2 * T::TILE_STRIDE * 4 + 2 * T::SIDE_STRIDE * 4 + 2 * kCob * K * K * 8 + 64 + 128;
     static bool configured = false;
-    static int blocks = 0;
+    static int blocks_plain = 0, blocks_tma = 0;
     if (!configured) {
-        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        int dev = 0, sms = 0, per_sm = 0;
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_plain));
+        DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_tma_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_tma));
+        int dev = 0, sms = 0, a = 0, b = 0;
         DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
         DISTDL_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, convg_kernel<K, ADJ>, kConvThreads, smem));
-        blocks = sms * (per_sm > 0 ? per_sm : 1);
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, convg_kernel<K, ADJ>, kConvThreads, smem_plain));
+        DISTDL_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, convg_tma_kernel<K, ADJ>, kConvThreads, smem_tma));
+        blocks_plain = sms * std::max(a, 1);
+        blocks_tma = sms * std::max(b, 1);
         configured = true;
     }
-    const int grid = G.total_tiles < blocks ? G.total_tiles : blocks;
-    convg_kernel<K, ADJ><<<grid, kConvThreads, smem, s>>>(G);
+    const ConvParams &P = G.base;
+    EncodeTiledFn enc = tensor_map_encoder();
+    bool tma = enc != nullptr && in_shards <= kConvGTmaShards;
+    for (int32_t c = 0; c < P.pw_workers; ++c) tma = tma && ((P.bw[c] + 2 * C::IOFF) % 4) == 0;
+    if (tma) {
+        ConvGTmaParams Q;
+        memset(&Q, 0, sizeof(Q));
+        Q.g = G;
+        const int spatial = P.ph_workers * P.pw_workers;
+        const cuuint32_t estr[3] = {1, 1, 1};
+        for (int k = 0; k < in_shards; ++k) {
+            const int r = (k % spatial) / P.pw_workers, c = k % P.pw_workers;
+            const cuuint64_t pitch = (cuuint64_t)(P.bw[c] + 2 * C::IOFF), rows = (cuuint64_t)(P.bh[r] + 2 * C::IOFF);
+            const cuuint64_t dims[3] = {pitch, rows, (cuuint64_t)in_planes[k / spatial]};
+            const cuuint64_t strides[2] = {pitch * 4, pitch * rows * 4};
+            const cuuint32_t box[3] = {(cuuint32_t)C::PITCH, (cuuint32_t)C::ROWS, 1};
+            if (enc(&Q.in_map[k], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(P.in[k]), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return fail(DISTDL_ERR_CUDA, "convg: tensor map of input shard %d failed", k);
+        }
+        const int grid = G.total_tiles < blocks_tma ? G.total_tiles : blocks_tma;
+        convg_tma_kernel<K, ADJ><<<grid, kConvThreads, smem_tma, s>>>(Q);
+    } else {
+        const int grid = G.total_tiles < blocks_plain ? G.total_tiles : blocks_plain;
+        convg_kernel<K, ADJ><<<grid, kConvThreads, smem_plain, s>>>(G);
+    }
     DISTDL_CUDA_CHECK(cudaGetLastError());
     return DISTDL_OK;
 }
@@ -1156,8 +1319,13 @@ static distdl_status_t convg_impl(const distdl_partition *px, int64_t nco, int32
         for (int32_t b = 0; b < pco; ++b) G.bias[b] = (const float *)bias[b];
     cudaStream_t s = (cudaStream_t)stream;
     distdl_status_t st;
-    if (!adj) st = kh == 3 ? launch_convg<3, false>(G, s) : kh == 5 ? launch_convg<5, false>(G, s) : launch_convg<7, false>(G, s);
-    else st = kh == 3 ? launch_convg<3, true>(G, s) : kh == 5 ? launch_convg<5, true>(G, s) : launch_convg<7, true>(G, s);
+    int64_t in_planes[kMaxChanBlocks];
+    for (int32_t b = 0; b < p_in; ++b) in_planes[b] = px->global_shape[0] * G.cnt_in[b];
+    const int ins = p_in * spatial;
+    if (!adj) st = kh == 3 ? launch_convg<3, false>(G, ins, in_planes, s) : kh == 5 ? launch_convg<5, false>(G, ins, in_planes, s)
+                                                                        : launch_convg<7, false>(G, ins, in_planes, s);
+    else st = kh == 3 ? launch_convg<3, true>(G, ins, in_planes, s) : kh == 5 ? launch_convg<5, true>(G, ins, in_planes, s)
+                                                                     : launch_convg<7, true>(G, ins, in_planes, s);
     if (st != DISTDL_OK || !adj) return st;
     // adjoint: the ghosts of dx are zero, as H* leaves them
     GhostFrameParams Q;
