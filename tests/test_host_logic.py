@@ -202,3 +202,19 @@ def test_periodic_partition_geometry_and_refusals():
     p3 = distdl.Partition((8, 8, 8), (2, 1, 1), (2, 2, 2), (2, 2, 2), periodic=(True, False, False))
     taps = (ctypes.c_float * 15)(*([0.5] * 15))
     assert lib.distdl_stencil3d_fwd(p3.handle, arr, taps, 2, arr, None) == 4
+
+
+def test_validation_of_the_generalized_convolution():
+    lib = distdl.lib()
+    vp = ctypes.c_void_p
+    arr = (vp * 64)(*[0x10000 * (i + 1) for i in range(64)])
+    px = distdl.Partition((1, 4, 16, 16), (1, 2, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2))
+    assert lib.distdl_convg_fwd(px.handle, 6, 2, arr, arr, None, 3, 3, arr, None) == 2          # widths do not match 3x3
+    assert lib.distdl_convg_fwd(px.handle, 6, 2, arr, arr, None, 4, 4, arr, None) == 4          # even kernel
+    assert lib.distdl_convg_fwd(px.handle, 1, 2, arr, arr, None, 5, 5, arr, None) == 2          # fewer channels than blocks
+    assert lib.distdl_convg_fwd(px.handle, 18, 9, arr, arr, None, 5, 5, arr, None) == 4         # more than 8 channel blocks
+    assert lib.distdl_convg_adj(px.handle, 6, 2, None, arr, 5, 5, arr, None) == 1
+    pb = distdl.Partition((2, 4, 16, 16), (2, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2))
+    assert lib.distdl_convg_fwd(pb.handle, 6, 2, arr, arr, None, 5, 5, arr, None) == 4          # batch partitioned
+    odd = (vp * 8)(*[0x10004 + 0x10000 * i for i in range(8)])
+    assert lib.distdl_convg_fwd(px.handle, 6, 2, odd, arr, None, 5, 5, arr, None) == 3          # alignment
