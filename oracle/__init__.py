@@ -43,6 +43,7 @@ from .layers import (  # noqa: F401
     conv_adj_params,
     convg_fwd,
     convg_adj,
+    convg_adj_params,
     stencil3d_fwd,
     stencil3d_adj,
     stencil3d_fwd_exchange_then_local,

@@ -237,6 +237,41 @@ def convg_adj(xpart: Partition, nco, pco, dy_shards, w_blocks):
     return halo_adj_sequence(xpart, local)
 
 
+def convg_adj_params(xpart: Partition, nco, pco, x_shards, dy_shards, kh, kw):
+    """Parameter part of the adjoint convolution algorithm with channel partitions: (dw blocks, db blocks).
+
+      x <- H x (the exchanged input of the forward pass);  dy^_{ijs} <- B dy_{is};
+      dw^_{ijs}[o,c,a,b] = sum_{n,p} dy^_{ijs}[n,o,p] * x^_{js}[n,c,p + (a,b)]   (padded-local indices),
+      db^_{ijs}[o]       = sum_{n,p} dy^_{ijs}[n,o,p]                            (j = 0 only);
+      dw_{ij} <- R over the feature-space workers s in order,  db_i <- R over s (from the j = 0 workers).
+    fp64 throughout, rounded once to fp32.  Returns (dw, db): dw[i * P_ci + j] of shape
+    [nco_i, nci_j, kh, kw], db[i] of shape [nco_i].
+    """
+    from .primitives import halo_fwd_sequence
+    assert xpart.rank == 4 and xpart.pshape[0] == 1
+    _, pci, p0, p1 = xpart.pshape
+    xh = halo_fwd_sequence(xpart, x_shards)
+    dw, db = [], []
+    for i in range(pco):
+        for j in range(pci):
+            per_worker = []
+            for r in range(p0):
+                for c in range(p1):
+                    x = np.asarray(xh[(j * p0 + r) * p1 + c], dtype=np.float64)
+                    dy = np.asarray(dy_shards[(i * p0 + r) * p1 + c], dtype=np.float64)
+                    N, cob, hb, wb = dy.shape
+                    g = np.zeros((cob, x.shape[1], kh, kw), dtype=np.float64)
+                    for a in range(kh):
+                        for b in range(kw):
+                            g[:, :, a, b] = np.einsum("nohw,nchw->oc", dy, x[:, :, a:a + hb, b:b + wb])
+                    per_worker.append(g)
+            dw.append(sumreduce_fwd(per_worker).astype(np.float32))
+        sums = [np.asarray(dy_shards[(i * p0 + r) * p1 + c], dtype=np.float64).sum(axis=(0, 2, 3))
+                for r in range(p0) for c in range(p1)]
+        db.append(sumreduce_fwd(sums).astype(np.float32))
+    return dw, db
+
+
 # --------------------------------------------------------------------------
 # Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers":
 # a sliding-kernel layer on a feature-space partition = halo exchange, then the

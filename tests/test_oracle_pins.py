@@ -997,3 +997,28 @@ def test_generalized_conv_reduces_to_the_depthwise_layer_on_diagonal_weights():
     y = oracle.assemble_global(Partition((N, C, H, W), (1, 2, 2, 1)), oracle.convg_fwd(xpart, C, 2, oracle.scatter_global(xpart, xg), wb))
     yd = oracle.assemble_global(Partition((N, C, H, W), (1, 1, 2, 1)), oracle.conv_fwd(dpart, oracle.scatter_global(dpart, xg), wd))
     assert np.allclose(y, yd, rtol=0, atol=2e-6)
+
+
+@pytest.mark.parametrize("case", CONVG_CASES, ids=[str(c) for c in CONVG_CASES])
+def test_generalized_conv_param_gradients_against_autograd_and_dot_test(case):
+    import torch
+    xpart, ypart, xg, wg, bg, wb, bb = _convg_problem(case, 121)
+    N, nci, nco, H, W, pci, pco, p0, p1, k = case
+    dyg = inputs.normal((N, nco, H, W), 125)
+    x = oracle.scatter_global(xpart, xg, fill=lambda wk: np.full(xpart.padded_shape(wk), 4.0))     # garbage ghosts
+    dy = oracle.scatter_global(ypart, dyg)
+    dw, db = oracle.convg_adj_params(xpart, nco, pco, x, dy, k, k)
+    Wt = torch.tensor(wg, dtype=torch.float64, requires_grad=True)
+    Bt = torch.tensor(bg, dtype=torch.float64, requires_grad=True)
+    Y = torch.nn.functional.conv2d(torch.tensor(xg, dtype=torch.float64), Wt, Bt, padding=k // 2)
+    Y.backward(torch.tensor(dyg, dtype=torch.float64))
+    cs_i, cz_i = oracle.balanced_split(nco, pco)
+    cs_j, cz_j = oracle.balanced_split(nci, pci)
+    for i in range(pco):
+        for j in range(pci):
+            ref = Wt.grad.numpy()[cs_i[i]:cs_i[i] + cz_i[i], cs_j[j]:cs_j[j] + cz_j[j]]
+            assert np.allclose(dw[i * pci + j], ref, rtol=1e-6, atol=1e-5)
+        assert np.allclose(db[i], Bt.grad.numpy()[cs_i[i]:cs_i[i] + cz_i[i]], rtol=1e-6, atol=1e-5)
+    # parameter-space dot test through the (separately pinned) forward oracle: <Conv(w, b; x), dy> = <w, dw> + <b, db>
+    y = oracle.convg_fwd(xpart, nco, pco, x, wb, bb)
+    assert oracle.adjoint_test_ratio(y, dy, list(wb) + list(bb), list(dw) + list(db)) < 1e-6
