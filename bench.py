@@ -191,11 +191,15 @@ class Workload:
         self.g_y = [torch.empty(gN, 8, 512, 512, device=dev) for _ in range(8)]
         self.g_dx = [torch.empty(*self.gpart.padded_shape(w), device=dev) for w in range(8)]
         self.g_w = [n(8, 8, 5, 5) * 0.05 for _ in range(4)]
+        self.g_dw = [torch.empty(8, 8, 5, 5, device=dev) for _ in range(4)]
+        self.g_ws = torch.empty(d.convg_adj_params_workspace(self.gpart, 16, 2, 5, 5), dtype=torch.uint8, device=dev)
         g_flops = 2 * 25 * 16 * 16 * gN * 1024 * 1024
         g_bytes = 2 * gN * 16 * 1024 * 1024 * 4
         self.extra_ops += [
             ("convg_fwd", lambda: d.convg_fwd(self.gpart, 16, 2, self.g_x, self.g_w, None, self.g_y), g_bytes, g_flops, 1, "alu"),
             ("convg_adj", lambda: d.convg_adj(self.gpart, 16, 2, self.g_y, self.g_w, self.g_dx), g_bytes, g_flops, 2, "alu"),
+            ("convg_adj_params", lambda: d.convg_adj_params(self.gpart, 16, 2, self.g_x, self.g_y, (5, 5), self.g_dw, None,
+                                                            self.g_ws), g_bytes, g_flops, 2, "alu"),
         ]
         self.extra_ops += [
             ("conv_adj_params", lambda: d.conv_adj_params(self.cpart, self.c_x, self.c_dy, (5, 5), self.c_dw, self.c_db,

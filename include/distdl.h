@@ -290,7 +290,13 @@ distdl_status_t distdl_conv_adj_params(const distdl_partition_t *p, const void *
  * convg_adj: dy^ <- B dy; dx^_{ijs} <- [dConv]*(dy^_{ijs}); dx_js <- R over i in order; dx <- H* dx -- fused in
  *     gather form: dx[n,c,p] = sum over output channels o and taps of w[o,c,a,b] * dy[n,o,p - (a,b) + pad];
  *     dy[.]: bulk-shaped shards; dx[.]: padded shards whose ghosts are set to zero.
- * (dw, db of this layer are not computed.)
+ * convg_adj_params: the parameter part of the adjoint algorithm: dw^_{ijs}, db^_{ijs} <- [dConv]*(dy^_{ijs}) with the
+ *     exchanged x^_{js} of the forward pass, then dw_ij <- R over the feature-space workers s, db_i <- R over s
+ *     (from the j = 0 workers): dw[i*P_ci + j] F32 [nco_i, nci_j, kh, kw] with
+ *     dw[o,c,a,b] = sum_{n,p} dy[n,o,p] * x[n,c,p + (a,b) - pad] on the GLOBAL tensors; db[i] F32 [nco_i] (db may be
+ *     NULL).  x[.]: padded shards (bulk read only, the exchange is fused); dy[.]: bulk-shaped shards.  Sums in
+ *     fp32 in a fixed order (running sums over a static set of tiles, lanes, warps, then the slices of a
+ *     channel pair in order).  workspace: device scratch of the size convg_adj_params_workspace reports.
  * ---------------------------------------------------------------------- */
 distdl_status_t distdl_convg_fwd(const distdl_partition_t *px, int64_t nco, int32_t pco,
                                  const void *const *x, const void *const *w, const void *const *bias,
@@ -298,6 +304,12 @@ distdl_status_t distdl_convg_fwd(const distdl_partition_t *px, int64_t nco, int3
 distdl_status_t distdl_convg_adj(const distdl_partition_t *px, int64_t nco, int32_t pco,
                                  const void *const *dy, const void *const *w, int32_t kh, int32_t kw,
                                  void *const *dx, void *stream);
+distdl_status_t distdl_convg_adj_params_workspace(const distdl_partition_t *px, int64_t nco, int32_t pco,
+                                                  int32_t kh, int32_t kw, int64_t *bytes);
+distdl_status_t distdl_convg_adj_params(const distdl_partition_t *px, int64_t nco, int32_t pco,
+                                        const void *const *x, const void *const *dy, int32_t kh,
+                                        int32_t kw, void *const *dw, void *const *db, void *workspace,
+                                        int64_t workspace_bytes, void *stream);
 
 /* ------------------------------------------------------------------------
  * Distributed star-stencil layer on a rank-3 tensor (Section 4, "Sparse layers": on a feature-space

@@ -85,6 +85,8 @@ def lib():
     L.distdl_stencil3d_adj.argtypes = [vp, pvp, ctypes.POINTER(ctypes.c_float), c_i32, pvp, vp]
     L.distdl_convg_fwd.argtypes = [vp, c_i64, c_i32, pvp, pvp, pvp, c_i32, c_i32, pvp, vp]
     L.distdl_convg_adj.argtypes = [vp, c_i64, c_i32, pvp, pvp, c_i32, c_i32, pvp, vp]
+    L.distdl_convg_adj_params_workspace.argtypes = [vp, c_i64, c_i32, c_i32, c_i32, pi64]
+    L.distdl_convg_adj_params.argtypes = [vp, c_i64, c_i32, pvp, pvp, c_i32, c_i32, pvp, pvp, vp, c_i64, vp]
     L.distdl_device_status.argtypes = [vp]
     _lib = L
     return L
@@ -310,6 +312,20 @@ def convg_adj(px, nco, pco, dy, w, dx, stream=None):
     kh, kw = int(w[0].shape[-2]), int(w[0].shape[-1])
     _check(lib().distdl_convg_adj(px.handle, nco, pco, _ptr_array(dy), _ptr_array(w), kh, kw, _ptr_array(dx),
                                   _stream(stream)))
+
+
+def convg_adj_params_workspace(px, nco, pco, kh, kw):
+    n = ctypes.c_int64(0)
+    _check(lib().distdl_convg_adj_params_workspace(px.handle, nco, pco, kh, kw, ctypes.byref(n)))
+    return n.value
+
+
+def convg_adj_params(px, nco, pco, x, dy, kernel, dw, db, workspace, stream=None):
+    """dw: list of blocks [nco_i, nci_j, kh, kw] in order i * P_ci + j; db: list of [nco_i] or None."""
+    b = None if db is None else _ptr_array(db)
+    _check(lib().distdl_convg_adj_params(px.handle, nco, pco, _ptr_array(x), _ptr_array(dy), kernel[0], kernel[1],
+                                         _ptr_array(dw), b, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 class Repartition:

@@ -1369,13 +1369,46 @@ struct ConvGradParams {
     int32_t tiles_per_plane;                // Ph * tiles_y * Pw * tiles_x
     int32_t tiles_per_channel;              // batch * tiles_per_plane
     int32_t tiles_y;
+    // Which planes an item reads.  pairs == 0 (depthwise layer): item channel ch, plane n * channels + ch of x
+    // and of dy.  pairs = n_co * n_ci (generalized layer): item (o, c) reads input channel c of x and output
+    // channel o of dy, each found in the group of Ph x Pw shards of its channel block.
+    int32_t pairs, spatial, n_x;
+    int32_t x_blocks, y_blocks;
+    int32_t x_start[8], x_cnt[8], y_start[8], y_cnt[8];
 };
 
+// plane of batch entry n = n * mult + base, in the shards [wofs, wofs + Ph * Pw)
+struct GradItem {
+    int x_wofs, x_base, x_mult, dy_wofs, dy_base, dy_mult;
+};
+__device__ __forceinline__ GradItem grad_item(const ConvGradParams &G, int q) {
+    GradItem it;
+    if (G.pairs == 0) {
+        it.x_wofs = it.dy_wofs = 0;
+        it.x_base = it.dy_base = q;
+        it.x_mult = it.dy_mult = G.base.channels;
+        return it;
+    }
+    const int o = q / G.n_x, c = q - o * G.n_x;
+    int jb = 0, ib = 0;
+    for (int b = 1; b < G.x_blocks; ++b)
+        if (c >= G.x_start[b]) jb = b;
+    for (int b = 1; b < G.y_blocks; ++b)
+        if (o >= G.y_start[b]) ib = b;
+    it.x_wofs = jb * G.spatial;
+    it.x_base = c - G.x_start[jb];
+    it.x_mult = G.x_cnt[jb];
+    it.dy_wofs = ib * G.spatial;
+    it.dy_base = o - G.y_start[ib];
+    it.dy_mult = G.y_cnt[ib];
+    return it;
+}
+
 // dy tile: kTileH rows of kTileW floats, zero outside the shard's bulk
-__device__ __forceinline__ void stage_dy_tile(const ConvGradParams &G, const ConvTile &t, float *dt) {
+__device__ __forceinline__ void stage_dy_tile(const float *shard, int dy_plane, const ConvTile &t, float *dt) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = min(kTileH, t.bh - t.i0), cols = min(kTileW, t.bw - t.j0);
-    const float *plane = G.dy[t.shard] + (size_t)t.plane * t.bh * t.bw;
+    const float *plane = shard + (size_t)dy_plane * t.bh * t.bw;
     const bool fast = (t.bw % 4) == 0;
     const int nv = fast ? cols / 4 : 0;
     for (int ry = warp; ry < kTileH; ry += kConvThreads / 32) {
@@ -1474,7 +1507,7 @@ conv_grad_kernel(const __grid_constant__ ConvGradParams G) {
     float *dts = smem + 2 * C::TILE_FLOATS;
     __shared__ float red[kConvThreads / 32][K * K + 1];
     const ConvParams &P = G.base;
-    const int items = P.channels * G.slices;
+    const int items = (G.pairs ? G.pairs : P.channels) * G.slices;
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int ch = item / G.slices, sl = item - ch * G.slices;
         uint64_t acc[K][K];
@@ -1483,16 +1516,21 @@ conv_grad_kernel(const __grid_constant__ ConvGradParams G) {
         for (int a = 0; a < K; ++a)
 #pragma unroll
             for (int b = 0; b < K; ++b) acc[a][b] = 0ull;
+        const GradItem it = grad_item(G, ch);
+        // tile L of the item: its place (batch entry, shard, rows, columns); .plane = the plane of x, dyp = that of dy
+        int dyp = 0;
         auto tile_of = [&](int L) {
-            const int n = L / G.tiles_per_plane;
-            return decode_tile(P, (n * P.channels + ch) * G.tiles_per_plane + (L - n * G.tiles_per_plane), G.tiles_y, 0);
+            ConvTile t = decode_tile(P, L, G.tiles_y, 0);          // decodes the batch entry into .plane
+            dyp = t.plane * it.dy_mult + it.dy_base;
+            t.plane = t.plane * it.x_mult + it.x_base;
+            return t;
         };
         auto stage = [&](const ConvTile &t, int b) {
             if (!t.valid) return;
             float *xt = xts + b * C::TILE_FLOATS;
             clear_unstaged_x<K>(t, xt);
-            stage_tile<K, false>(P, t, xt);
-            stage_dy_tile(G, t, dts + b * (kTileH * kTileW));
+            stage_tile<K, false>(P, t, xt, it.x_wofs);
+            stage_dy_tile(G.dy[it.dy_wofs + t.shard], dyp, t, dts + b * (kTileH * kTileW));
         };
         int L = sl, buf = 0;
         if (L < G.tiles_per_channel) {
@@ -1578,7 +1616,7 @@ conv_grad_tma_kernel(const __grid_constant__ ConvGradTmaParams Q) {
     __syncthreads();
     uint32_t phase0 = 0, phase1 = 0;
     bool failed = false;
-    const int items = P.channels * G.slices;
+    const int items = (G.pairs ? G.pairs : P.channels) * G.slices;
     for (int item = blockIdx.x; item < items && !failed; item += gridDim.x) {
         const int ch = item / G.slices, sl = item - ch * G.slices;
         uint64_t acc[K][K];
@@ -1587,9 +1625,14 @@ conv_grad_tma_kernel(const __grid_constant__ ConvGradTmaParams Q) {
         for (int a = 0; a < K; ++a)
 #pragma unroll
             for (int b = 0; b < K; ++b) acc[a][b] = 0ull;
+        const GradItem it = grad_item(G, ch);
+        // tile L of the item: its place (batch entry, shard, rows, columns); .plane = the plane of x, dyp = that of dy
+        int dyp = 0;
         auto tile_of = [&](int L) {
-            const int n = L / G.tiles_per_plane;
-            return decode_tile(P, (n * P.channels + ch) * G.tiles_per_plane + (L - n * G.tiles_per_plane), G.tiles_y, 0);
+            ConvTile t = decode_tile(P, L, G.tiles_y, 0);          // decodes the batch entry into .plane
+            dyp = t.plane * it.dy_mult + it.dy_base;
+            t.plane = t.plane * it.x_mult + it.x_base;
+            return t;
         };
         auto stage = [&](const ConvTile &t, int b) {
             if (!t.valid) return;
@@ -1597,11 +1640,11 @@ conv_grad_tma_kernel(const __grid_constant__ ConvGradTmaParams Q) {
             if (threadIdx.x == 0) {
                 fence_proxy_async();
                 mbar_expect_tx(bars + 8 * b, T::BOX_BYTES + (DYTMA ? DY_FLOATS * 4 : 0));
-                tma_load_3d(smem_u32(xt), &Q.x_map[t.shard], t.j0, t.i0, t.plane, bars + 8 * b);
-                if (DYTMA) tma_load_3d(smem_u32(dt), &Q.dy_map[t.shard], t.j0, t.i0, t.plane, bars + 8 * b);
+                tma_load_3d(smem_u32(xt), &Q.x_map[it.x_wofs + t.shard], t.j0, t.i0, t.plane, bars + 8 * b);
+                if (DYTMA) tma_load_3d(smem_u32(dt), &Q.dy_map[it.dy_wofs + t.shard], t.j0, t.i0, dyp, bars + 8 * b);
             }
-            if (!DYTMA) stage_dy_tile(G, t, dt);
-            stage_halo_strips<K, false>(P, t, sides + b * T::SIDE_STRIDE);
+            if (!DYTMA) stage_dy_tile(G.dy[it.dy_wofs + t.shard], dyp, t, dt);
+            stage_halo_strips<K, false>(P, t, sides + b * T::SIDE_STRIDE, it.x_wofs);
         };
         int L = sl, buf = 0;
         if (L < G.tiles_per_channel) {
@@ -1703,6 +1746,24 @@ __global__ void conv_grad_finish_kernel(const float *partial, int slices, int ta
     else if (db) db[ch] = v;
 }
 
+// Generalized layer: item q = (o, c); the slices' rows added in order go to tap t of dw block (i, j) at
+// [o_local][c_local], the last entry of the c = 0 items to db_i[o_local].
+struct ConvGGradOut {
+    float *dw[64];
+    float *db[8];
+};
+__global__ void convg_grad_finish_kernel(const __grid_constant__ ConvGradParams G, const __grid_constant__ ConvGGradOut O, int taps) {
+    const int q = blockIdx.x, t = threadIdx.x;
+    if (t > taps) return;
+    const float *row = G.partial + (size_t)q * G.slices * kGradRow + t;
+    float v = row[0];
+    for (int s = 1; s < G.slices; ++s) v += row[(size_t)s * kGradRow];
+    const GradItem it = grad_item(G, q);
+    const int ib = it.dy_wofs / G.spatial, jb = it.x_wofs / G.spatial;
+    if (t < taps) O.dw[ib * G.x_blocks + jb][((size_t)it.dy_base * it.x_mult + it.x_base) * taps + t] = v;
+    else if (O.db[ib] && q % G.n_x == 0) O.db[ib][it.dy_base] = v;
+}
+
 template <int K>
 static constexpr int grad_smem_bytes(bool tma) {
     return tma ? 2 * ConvTmaCfg<K, false>::TILE_STRIDE * 4 + 2 * ConvTmaCfg<K, false>::SIDE_STRIDE * 4 + 2 * kTileH * kTileW * 4 + 64 + 128
@@ -1791,12 +1852,15 @@ static distdl_status_t grad_plan(const distdl_partition *p, int32_t kh, int32_t 
 
 template <int K>
 static distdl_status_t launch_grad(const distdl_partition *p, const ConvGradParams &G, int grid, float *dw, float *db,
-                                   cudaStream_t s) {
+                                   cudaStream_t s, const ConvGGradOut *gout = nullptr) {
     const ConvParams &P = G.base;
+    // shards of x and of dy: one group of Ph x Pw for the depthwise layer, one per channel block otherwise
+    const int spatial = P.ph_workers * P.pw_workers;
+    const int nx = G.pairs ? G.x_blocks * spatial : p->num_workers, ny = G.pairs ? G.y_blocks * spatial : p->num_workers;
     // TMA for the x tiles: few enough workers for the maps to travel as kernel parameters and padded rows
     // of whole 16-byte units; for the dy tiles as well when the bulk rows are
     EncodeTiledFn enc = tensor_map_encoder();
-    bool x_tma = p->num_workers <= kConvTmaMaxWorkers && enc != nullptr, dy_tma = true;
+    bool x_tma = nx <= kConvTmaMaxWorkers && ny <= kConvTmaMaxWorkers && enc != nullptr, dy_tma = true;
     for (int32_t c = 0; c < P.pw_workers; ++c) {
         x_tma = x_tma && ((P.bw[c] + 2 * (K / 2)) % 4) == 0;
         dy_tma = dy_tma && (P.bw[c] % 4) == 0;
@@ -1806,19 +1870,22 @@ static distdl_status_t launch_grad(const distdl_partition *p, const ConvGradPara
         ConvGradTmaParams Q;
         memset(&Q, 0, sizeof(Q));
         Q.g = G;
-        const cuuint64_t planes = (cuuint64_t)(p->global_shape[0] * p->global_shape[1]);
         const cuuint32_t estr[3] = {1, 1, 1};
-        for (int32_t wk = 0; wk < p->num_workers; ++wk) {
-            const int r = wk / P.pw_workers, c = wk % P.pw_workers;
+        for (int32_t wk = 0; wk < std::max(nx, ny); ++wk) {
+            const int r = (wk % spatial) / P.pw_workers, c = wk % P.pw_workers;
+            const cuuint64_t batch = (cuuint64_t)p->global_shape[0];
+            const cuuint64_t xplanes = batch * (cuuint64_t)(G.pairs ? G.x_cnt[std::min(wk / spatial, 7)] : p->global_shape[1]);
+            const cuuint64_t planes = batch * (cuuint64_t)(G.pairs ? G.y_cnt[std::min(wk / spatial, 7)] : p->global_shape[1]);
             const cuuint64_t pitch = (cuuint64_t)(P.bw[c] + 2 * C::PH), rows = (cuuint64_t)(P.bh[r] + 2 * C::PH);
-            const cuuint64_t dims[3] = {pitch, rows, planes};
+            const cuuint64_t dims[3] = {pitch, rows, xplanes};
             const cuuint64_t strides[2] = {pitch * 4, pitch * rows * 4};
             const cuuint32_t box[3] = {(cuuint32_t)C::PITCH, (cuuint32_t)C::ROWS, 1};
-            if (enc(&Q.x_map[wk], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(P.in[wk]), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-                return fail(DISTDL_ERR_CUDA, "conv_adj_params: tensor map of x shard %d failed", wk);
-            if (!dy_tma) continue;
+            if (wk < nx)
+                if (enc(&Q.x_map[wk], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(P.in[wk]), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                    return fail(DISTDL_ERR_CUDA, "conv_adj_params: tensor map of x shard %d failed", wk);
+            if (!dy_tma || wk >= ny) continue;
             const cuuint64_t ddims[3] = {(cuuint64_t)P.bw[c], (cuuint64_t)P.bh[r], planes};
             const cuuint64_t dstrides[2] = {(cuuint64_t)P.bw[c] * 4, (cuuint64_t)P.bw[c] * (cuuint64_t)P.bh[r] * 4};
             const cuuint32_t dbox[3] = {(cuuint32_t)kTileW, (cuuint32_t)kTileH, 1};
@@ -1833,8 +1900,76 @@ static distdl_status_t launch_grad(const distdl_partition *p, const ConvGradPara
         conv_grad_kernel<K><<<grid, kConvThreads, grad_smem_bytes<K>(false), s>>>(G);
     }
     DISTDL_CUDA_CHECK(cudaGetLastError());
-    conv_grad_finish_kernel<<<G.base.channels, 64, 0, s>>>(G.partial, G.slices, K * K, dw, db);
+    if (G.pairs) convg_grad_finish_kernel<<<G.pairs, 64, 0, s>>>(G, *gout, K * K);
+    else conv_grad_finish_kernel<<<G.base.channels, 64, 0, s>>>(G.partial, G.slices, K * K, dw, db);
     DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
+}
+
+// Parameter gradients of the generalized layer: geometry, slices and the channel tables of the items.
+static distdl_status_t convg_grad_plan(const distdl_partition *px, int64_t nco, int32_t pco, int32_t kh, int32_t kw,
+                                       const char *what, ConvGradParams *G, int *grid) {
+    if (!px) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL partition", what);
+    if (px->rank != 4 || px->dtype != DISTDL_F32) return fail(DISTDL_ERR_SHAPE, "%s: needs a rank-4 F32 partition", what);
+    if (px->any_periodic()) return fail(DISTDL_ERR_UNSUPPORTED, "%s: periodic partitions are not supported by the fused layers", what);
+    if (px->pshape[0] != 1) return fail(DISTDL_ERR_UNSUPPORTED, "%s: the batch dimension may not be partitioned", what);
+    if (kh != kw || (kh != 3 && kh != 5 && kh != 7))
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: kernel %d x %d (supported: 3x3, 5x5, 7x7)", what, kh, kw);
+    const int32_t pci = px->pshape[1], ph = px->pshape[2], pw = px->pshape[3];
+    if (pco < 1 || nco < pco) return fail(DISTDL_ERR_SHAPE, "%s: %lld output channels on %d blocks", what, (long long)nco, pco);
+    if (pci > 8 || pco > 8) return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than 8 blocks of a channel partition", what);
+    if ((int64_t)std::max(pci, pco) * ph * pw > kConvMaxWorkers)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d shards of one tensor", what, kConvMaxWorkers);
+    const int h = kh / 2;
+    for (int k = 0; k < 4; ++k)
+        for (int32_t c = 0; c < px->pshape[k]; ++c) {
+            const int want = k < 2 ? 0 : h;
+            if (px->hlo[k][c] != want || px->hhi[k][c] != want)
+                return fail(DISTDL_ERR_SHAPE, "%s: halo widths must be 0,0,%d,%d on every side", what, h, h);
+        }
+    ConvParams &P = G->base;
+    int64_t max_bh = 0, max_bw = 0;
+    for (int32_t r = 0; r < ph; ++r) max_bh = std::max<int64_t>(max_bh, P.bh[r] = (int32_t)px->size[2][r]);
+    for (int32_t c = 0; c < pw; ++c) max_bw = std::max<int64_t>(max_bw, P.bw[c] = (int32_t)px->size[3][c]);
+    P.ph_workers = ph;
+    P.pw_workers = pw;
+    P.channels = (int32_t)px->global_shape[1];
+    P.tiles_x = (int32_t)((max_bw + kTileW - 1) / kTileW);
+    const int tiles_y = (int)((max_bh + kTileH - 1) / kTileH);
+    conv_set_divisor(P, 0, (uint32_t)P.tiles_x);
+    conv_set_divisor(P, 1, (uint32_t)pw);
+    conv_set_divisor(P, 2, (uint32_t)tiles_y);
+    conv_set_divisor(P, 3, (uint32_t)ph);
+    const int64_t per_plane = (int64_t)P.tiles_x * tiles_y * ph * pw;
+    const int64_t per_item = per_plane * px->global_shape[0];
+    const int64_t pairs = nco * px->global_shape[1];
+    if (per_item >= ((int64_t)1 << 31) || pairs > 65536) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles or channel pairs", what);
+    int blocks = 0;
+    distdl_status_t st = kh == 3 ? grad_config<3>(&blocks) : kh == 5 ? grad_config<5>(&blocks) : grad_config<7>(&blocks);
+    if (st != DISTDL_OK) return st;
+    // about four items per resident block, handed out round-robin; never more slices than tiles
+    int64_t slices = (4 * (int64_t)blocks + pairs - 1) / pairs;
+    slices = std::max<int64_t>(1, std::min<int64_t>(slices, per_item));
+    G->slices = (int32_t)slices;
+    G->tiles_per_plane = (int32_t)per_plane;
+    G->tiles_per_channel = (int32_t)per_item;
+    G->tiles_y = tiles_y;
+    G->pairs = (int32_t)pairs;
+    G->spatial = ph * pw;
+    G->n_x = (int32_t)px->global_shape[1];
+    G->x_blocks = pci;
+    G->y_blocks = pco;
+    std::vector<int64_t> co_start, co_size;
+    split_evenly(nco, pco, co_start, co_size);
+    for (int32_t b = 0; b < pci; ++b) {
+        G->x_start[b] = (int32_t)px->start[1][b];
+        G->x_cnt[b] = (int32_t)px->size[1][b];
+    }
+    for (int32_t b = 0; b < pco; ++b) {
+        G->y_start[b] = (int32_t)co_start[b];
+        G->y_cnt[b] = (int32_t)co_size[b];
+    }
+    *grid = (int)std::min<int64_t>(blocks, slices * pairs);
     return DISTDL_OK;
 }
 
@@ -1848,6 +1983,62 @@ extern "C" distdl_status_t distdl_convg_fwd(const distdl_partition_t *px, int64_
 extern "C" distdl_status_t distdl_convg_adj(const distdl_partition_t *px, int64_t nco, int32_t pco, const void *const *dy,
                                             const void *const *w, int32_t kh, int32_t kw, void *const *dx, void *stream) {
     return distdl::convg_impl(px, nco, pco, dy, w, nullptr, kh, kw, dx, stream, true, "convg_adj");
+}
+
+extern "C" distdl_status_t distdl_convg_adj_params_workspace(const distdl_partition_t *px, int64_t nco, int32_t pco,
+                                                             int32_t kh, int32_t kw, int64_t *bytes) {
+    using namespace distdl;
+    clear_error();
+    if (!bytes) return fail(DISTDL_ERR_INVALID_ARG, "convg_adj_params_workspace: NULL argument");
+    ConvGradParams G;
+    memset(&G, 0, sizeof(G));
+    int grid = 0;
+    const distdl_status_t st = convg_grad_plan(px, nco, pco, kh, kw, "convg_adj_params_workspace", &G, &grid);
+    if (st != DISTDL_OK) return st;
+    *bytes = (int64_t)G.pairs * G.slices * kGradRow * (int64_t)sizeof(float);
+    return DISTDL_OK;
+}
+
+extern "C" distdl_status_t distdl_convg_adj_params(const distdl_partition_t *px, int64_t nco, int32_t pco,
+                                                   const void *const *x, const void *const *dy, int32_t kh, int32_t kw,
+                                                   void *const *dw, void *const *db, void *workspace,
+                                                   int64_t workspace_bytes, void *stream) {
+    using namespace distdl;
+    clear_error();
+    const char *what = "convg_adj_params";
+    if (!px || !x || !dy || !dw || !workspace) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    ConvGradParams G;
+    memset(&G, 0, sizeof(G));
+    int grid = 0;
+    const distdl_status_t st = convg_grad_plan(px, nco, pco, kh, kw, what, &G, &grid);
+    if (st != DISTDL_OK) return st;
+    const int64_t need = (int64_t)G.pairs * G.slices * kGradRow * (int64_t)sizeof(float);
+    if (workspace_bytes < need) return fail(DISTDL_ERR_INVALID_ARG, "%s: workspace of %lld bytes, %lld needed", what,
+                                            (long long)workspace_bytes, (long long)need);
+    if (!aligned16(workspace)) return fail(DISTDL_ERR_ALIGNMENT, "%s: workspace not 16-byte aligned", what);
+    for (int32_t k = 0; k < G.x_blocks * G.spatial; ++k) {
+        if (!x[k]) return fail(DISTDL_ERR_INVALID_ARG, "%s: x shard %d is NULL", what, k);
+        if (!aligned16(x[k])) return fail(DISTDL_ERR_ALIGNMENT, "%s: x shard %d is not 16-byte aligned", what, k);
+        G.base.in[k] = (const float *)x[k];
+    }
+    for (int32_t k = 0; k < G.y_blocks * G.spatial; ++k) {
+        if (!dy[k]) return fail(DISTDL_ERR_INVALID_ARG, "%s: dy shard %d is NULL", what, k);
+        if (!aligned16(dy[k])) return fail(DISTDL_ERR_ALIGNMENT, "%s: dy shard %d is not 16-byte aligned", what, k);
+        G.dy[k] = (const float *)dy[k];
+    }
+    ConvGGradOut O;
+    memset(&O, 0, sizeof(O));
+    for (int32_t k = 0; k < G.x_blocks * G.y_blocks; ++k) {
+        if (!dw[k]) return fail(DISTDL_ERR_INVALID_ARG, "%s: dw block %d is NULL", what, k);
+        O.dw[k] = (float *)dw[k];
+    }
+    if (db)
+        for (int32_t b = 0; b < G.y_blocks; ++b) O.db[b] = (float *)db[b];
+    G.partial = (float *)workspace;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (kh == 3) return launch_grad<3>(px, G, grid, nullptr, nullptr, s, &O);
+    if (kh == 5) return launch_grad<5>(px, G, grid, nullptr, nullptr, s, &O);
+    return launch_grad<7>(px, G, grid, nullptr, nullptr, s, &O);
 }
 
 extern "C" distdl_status_t distdl_conv_adj_params_workspace(const distdl_partition_t *p, int32_t kh, int32_t kw,

@@ -514,6 +514,51 @@ def test_generalized_conv_fwd_and_adj(case, integer):
     assert r < 1e-5
 
 
+@pytest.mark.parametrize("case", CONVG_CASES, ids=[str(c) for c in CONVG_CASES])
+@pytest.mark.parametrize("integer", [True, False], ids=["int", "normal"])
+def test_generalized_conv_param_gradients(case, integer):
+    N, nci, nco, H, W, pci, pco, p0, p1, k = case
+    h = k // 2
+    xpart = oracle.Partition((N, nci, H, W), (1, pci, p0, p1), (0, 0, h, h), (0, 0, h, h))
+    ypart = oracle.Partition((N, nco, H, W), (1, pco, p0, p1))
+    gpart = distdl.Partition((N, nci, H, W), (1, pci, p0, p1), (0, 0, h, h), (0, 0, h, h))
+    gen = (lambda shp, seed: inputs.integers(shp, seed, -2, 3)) if integer else inputs.normal
+    xg, dyg = gen((N, nci, H, W), 71), gen((N, nco, H, W), 72)
+    x = oracle.scatter_global(xpart, xg, fill=lambda wk: np.full(xpart.padded_shape(wk), 1e30, dtype=np.float32))
+    dy = oracle.scatter_global(ypart, dyg)
+    xs, dys = [dev(a) for a in x], [dev(a) for a in dy]
+    _, cz_i = oracle.balanced_split(nco, pco)
+    _, cz_j = oracle.balanced_split(nci, pci)
+    dw = [torch.full((cz_i[i], cz_j[j], k, k), -5.0, device=DEV) for i in range(pco) for j in range(pci)]
+    db = [torch.full((cz_i[i],), -5.0, device=DEV) for i in range(pco)]
+    ws = torch.empty(distdl.convg_adj_params_workspace(gpart, nco, pco, k, k), dtype=torch.uint8, device=DEV)
+    for _ in range(2):                                   # twice: the scratch table is reused
+        distdl.convg_adj_params(gpart, nco, pco, xs, dys, (k, k), dw, db, ws)
+    distdl.device_status()
+    xz = oracle.scatter_global(xpart, xg)
+    dw_ref, db_ref = oracle.convg_adj_params(xpart, nco, pco, xz, dy, k, k)
+    if integer:
+        for a, b in zip(dw + db, dw_ref + db_ref):
+            assert np.array_equal(host(a), b)
+        return
+    tiles = N * sum(-(-ypart.padded_shape(wk)[2] // 32) * -(-ypart.padded_shape(wk)[3] // 128) for wk in range(p0 * p1))
+    eps = (16 * tiles + 64) * 2.0 ** -24
+    mag_w, mag_b = oracle.convg_adj_params(xpart, nco, pco, [np.abs(a) for a in xz], [np.abs(a) for a in dy], k, k)
+    for a, b, m in zip(dw + db, dw_ref + db_ref, mag_w + mag_b):
+        assert np.all(np.abs(host(a).astype(np.float64) - b) <= eps * m)
+    # parameter-space dot test through the CUDA forward: <Conv(w, b; x), dy> = <w, dw> + <b, db>
+    cs_i, _ = oracle.balanced_split(nco, pco)
+    cs_j, _ = oracle.balanced_split(nci, pci)
+    wg, bg = inputs.normal((nco, nci, k, k), 73, 0.2), inputs.normal((nco,), 74)
+    wb = [np.ascontiguousarray(wg[cs_i[i]:cs_i[i] + cz_i[i], cs_j[j]:cs_j[j] + cz_j[j]]) for i in range(pco) for j in range(pci)]
+    bb = [np.ascontiguousarray(bg[cs_i[i]:cs_i[i] + cz_i[i]]) for i in range(pco)]
+    ys = [torch.empty(ypart.padded_shape(wk), device=DEV) for wk in range(ypart.num_workers)]
+    distdl.convg_fwd(gpart, nco, pco, xs, [dev(a) for a in wb], [dev(b) for b in bb], ys)
+    distdl.device_status()
+    r = oracle.adjoint_test_ratio([host(t) for t in ys], dy, wb + bb, [host(t) for t in dw + db])
+    assert r < 1e-5
+
+
 # --------------------------------------------------------------------------
 # 3-D star-stencil layer
 # --------------------------------------------------------------------------
