@@ -21,8 +21,10 @@
  *   - A shard is one contiguous row-major array of the padded shape
  *     bulk[k] + halo_lo[k] + halo_hi[k]; the bulk (the part the worker owns,
  *     Section 3 "Halo exchange") starts at index halo_lo[k] in each dimension.
- *   - The library allocates device memory only inside distdl_partition_create*
- *     (a few KB of plan tables, freed by distdl_partition_destroy).
+ *   - The library allocates device memory only inside distdl_partition_create* and
+ *     distdl_repartition_create (plan tables of a few KB to a few hundred KB, freed by the
+ *     matching destroy call).  The calls that need scratch (the *_adj_params of the
+ *     convolution layers) take it from the caller.
  */
 #ifndef DISTDL_H
 #define DISTDL_H
