@@ -461,6 +461,9 @@ CONVG_CASES = [
     (2, 3, 5, 70, 264, 3, 2, 2, 2, 5),       # 16-byte aligned rows, ragged tiles
     (1, 2, 2, 66, 260, 2, 1, 2, 2, 7),       # short last tile row and column
     (1, 4, 4, 34, 131, 2, 2, 1, 1, 3),
+    (1, 2, 3, 40, 264, 1, 2, 1, 2, 7),       # 7 x 7: bulk rows of whole 16-byte units (bulk copies in the adjoint)
+    (1, 3, 2, 34, 260, 1, 1, 1, 2, 3),       # 3 x 3: padded rows of whole 16-byte units (bulk copies in the forward)
+    (2, 2, 2, 33, 264, 2, 2, 2, 2, 3),       # 3 x 3: bulk copies in the adjoint, short last tile row
 ]
 
 
