@@ -1,6 +1,7 @@
 """GPU parity at the full sizes of the benchmark configurations, in the launch configuration that
 bench.py times.  B, R, H, H*, the all-to-all and the affine layer are compared in full; the convolution
-and the pooling layer on sampled (n, c) planes, the star stencil on sampled boxes, the parameter gradients on
+and the pooling layer on sampled (n, c) planes, the star stencil and the generalized convolution on sampled boxes,
+the parameter gradients on
 sampled channels / worker blocks, which the oracle computes one by one; properties that hold at any size
 (zero ghosts, dot test) over everything."""
 
@@ -292,3 +293,81 @@ def test_repartition_full_size():
         assert host(a).tobytes() == b.tobytes()
     for a, b in zip(back, rows):
         assert host(a).tobytes() == b.tobytes()
+
+
+def test_generalized_conv_full_size_on_samples():
+    # the configuration bench.py times: 16 -> 16 channels, 5 x 5, fp32 4 x 16 x 1024 x 1024, channel partitions 2 x 2,
+    # feature space 2 x 2
+    N, C, S, k, h = 4, 16, 1024, 5, 2
+    gpart = distdl.Partition((N, C, S, S), (1, 2, 2, 2), (0, 0, h, h), (0, 0, h, h))
+    g = torch.Generator(device=DEV)
+    g.manual_seed(17)
+    xs = [torch.randn(N, 8, 516, 516, device=DEV, generator=g) for _ in range(8)]
+    dys = [torch.randn(N, 8, 512, 512, device=DEV, generator=g) for _ in range(8)]
+    wb = [inputs.normal((8, 8, k, k), 9000 + q, 0.05) for q in range(4)]
+    wd = [dev(a) for a in wb]
+    ys = [torch.empty(N, 8, 512, 512, device=DEV) for _ in range(8)]
+    dxs = [torch.full((N, 8, 516, 516), 7.0, device=DEV) for _ in range(8)]
+    dws = [torch.empty(8, 8, k, k, device=DEV) for _ in range(4)]
+    dbs = [torch.empty(8, device=DEV) for _ in range(2)]
+    ws = torch.empty(distdl.convg_adj_params_workspace(gpart, C, 2, k, k), dtype=torch.uint8, device=DEV)
+    distdl.convg_fwd(gpart, C, 2, xs, wd, None, ys)
+    distdl.convg_adj(gpart, C, 2, dys, wd, dxs)
+    distdl.convg_adj_params(gpart, C, 2, xs, dys, (k, k), dws, dbs, ws)
+    distdl.device_status()
+
+    def gather(shards, off, n, lo, hi):
+        """[16, rows, cols] of batch entry n over the global box [lo, hi) from the bulks of the eight shards."""
+        out = np.zeros((C, hi[0] - lo[0], hi[1] - lo[1]), dtype=np.float32)
+        for b in range(2):
+            for r in range(2):
+                for c in range(2):
+                    a = [max(lo[0], 512 * r), max(lo[1], 512 * c)]
+                    e = [min(hi[0], 512 * r + 512), min(hi[1], 512 * c + 512)]
+                    if a[0] >= e[0] or a[1] >= e[1]:
+                        continue
+                    t = shards[(b * 2 + r) * 2 + c]
+                    out[8 * b:8 * b + 8, a[0] - lo[0]:e[0] - lo[0], a[1] - lo[1]:e[1] - lo[1]] = host(
+                        t[n, :, a[0] - 512 * r + off:e[0] - 512 * r + off, a[1] - 512 * c + off:e[1] - 512 * c + off])
+        return out
+
+    # boxes where the four feature-space shards meet, at a corner of the tensor, and inside a shard
+    for n, lo in ((2, (500, 490)), (0, (0, 0)), (3, (984, 960)), (1, (130, 700))):
+        hi = (lo[0] + 40, lo[1] + 64)
+        elo = tuple(max(v - h, 0) for v in lo)
+        ehi = tuple(min(v + h, S) for v in hi)
+        shape = (1, C, ehi[0] - elo[0], ehi[1] - elo[1])
+        sub = oracle.Partition(shape, (1, 2, 1, 1), (0, 0, h, h), (0, 0, h, h))
+        suby = oracle.Partition(shape, (1, 2, 1, 1))
+        inner = (slice(None), slice(lo[0] - elo[0], lo[0] - elo[0] + 40), slice(lo[1] - elo[1], lo[1] - elo[1] + 64))
+        xbox = gather(xs, h, n, elo, ehi)[None]
+        yref = oracle.assemble_global(suby, oracle.convg_fwd(sub, C, 2, oracle.scatter_global(sub, xbox), wb))[0][inner]
+        ymag = oracle.assemble_global(suby, oracle.convg_fwd(sub, C, 2, oracle.scatter_global(sub, np.abs(xbox)),
+                                                              [np.abs(a) for a in wb]))[0][inner]
+        got = gather(ys, 0, n, lo, hi)
+        assert np.all(np.abs(got.astype(np.float64) - yref) <= (C * k * k + 2) * 2.0 ** -24 * ymag + 1e-30)
+        dybox = gather(dys, 0, n, elo, ehi)[None]
+        dxref = oracle.assemble_global(sub, oracle.convg_adj(sub, C, 2, oracle.scatter_global(suby, dybox), wb))[0][inner]
+        dxmag = oracle.assemble_global(sub, oracle.convg_adj(sub, C, 2, oracle.scatter_global(suby, np.abs(dybox)),
+                                                             [np.abs(a) for a in wb]))[0][inner]
+        gotx = gather(dxs, h, n, lo, hi)
+        # the adjoint oracle rounds to fp32 before its halo sums: two more roundings at the box's own cut edges
+        assert np.all(np.abs(gotx.astype(np.float64) - dxref) <= (C * k * k + 6) * 2.0 ** -24 * dxmag + 1e-30)
+    for t in dxs:                                         # ghosts of dx are zero
+        assert float(t[:, :, :h].abs().max()) == 0.0 and float(t[:, :, -h:].abs().max()) == 0.0
+        assert float(t[:, :, :, :h].abs().max()) == 0.0 and float(t[:, :, :, -h:].abs().max()) == 0.0
+    # parameter gradients of sampled channel pairs (o, c): the oracle on those two channels alone
+    one = oracle.Partition((N, 1, S, S), (1, 1, 2, 2), (0, 0, h, h), (0, 0, h, h))
+    for o, c in ((0, 0), (5, 12), (11, 3), (15, 15)):
+        x1 = [host(xs[((c // 8) * 2 + r) * 2 + q][:, c % 8:c % 8 + 1]) for r in range(2) for q in range(2)]
+        dy1 = [host(dys[((o // 8) * 2 + r) * 2 + q][:, o % 8:o % 8 + 1]) for r in range(2) for q in range(2)]
+        dw_ref, db_ref = oracle.convg_adj_params(one, 1, 1, x1, dy1, k, k)
+        xh = oracle.halo_fwd_sequence(one, x1)
+        mag, _ = oracle.convg_adj_params(one, 1, 1, [np.abs(a) for a in xh], [np.abs(a) for a in dy1], k, k)
+        got = host(dws[(o // 8) * 2 + c // 8][o % 8, c % 8]).astype(np.float64)
+        tiles = N * 4 * 16 * 4
+        assert np.all(np.abs(got - dw_ref[0][0, 0]) <= (16 * tiles + 64) * 2.0 ** -24 * mag[0][0, 0])
+        assert np.linalg.norm(got - dw_ref[0][0, 0]) <= 1e-5 * np.linalg.norm(mag[0][0, 0])
+        if c == 0:
+            sum_abs = float(sum(np.abs(a.astype(np.float64)).sum() for a in dy1))
+            assert abs(float(host(dbs[o // 8])[o % 8]) - float(db_ref[0][0])) <= (16 * tiles + 64) * 2.0 ** -24 * sum_abs
