@@ -534,6 +534,50 @@ def main():
         torch.cuda.synchronize()
         extra_ms.append((xe[0].elapsed_time(xe[reps]) - b0[0].elapsed_time(b0[reps])) / reps)
 
+    # ---- the small 2-D configuration (256 x 256 on 2 x 2 workers, halo 1): launch-bound, so H + H* are timed as
+    # separate calls and as replays of a CUDA graph that holds 50 such pairs ----
+    small_cfg = None
+    if True:
+        import paper_2006_03108_b200 as distdl
+        p1 = distdl.Partition((256, 256), (2, 2), (1, 1), (1, 1))
+        sx = [torch.rand(*p1.padded_shape(w), device=dev) for w in range(4)]
+        pairs = 50
+
+        def run_pairs():
+            for _ in range(pairs):
+                distdl.halo_fwd(p1, sx)
+                distdl.halo_adj(p1, sx)
+
+        run_pairs()
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        run_pairs()
+        c1.record()
+        torch.cuda.synchronize()
+        eager_us = c0.elapsed_time(c1) * 1e3 / pairs
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            run_pairs()
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                run_pairs()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        c0.record()
+        for _ in range(5):
+            graph.replay()
+        c1.record()
+        torch.cuda.synchronize()
+        graph_us = c0.elapsed_time(c1) * 1e3 / (5 * pairs)
+        nb = p1.halo_stats(False)[2] + p1.halo_stats(True)[2]
+        small_cfg = {"workload": "H + H* on fp32 256x256, 2x2 workers, halo 1 (32,896 algorithmic bytes per pair)",
+                     "us_per_pair_separate_calls": round(eager_us, 2), "us_per_pair_cuda_graph": round(graph_us, 2),
+                     "gbs_cuda_graph": round(nb / graph_us / 1e3, 2), "bound": "launch latency"}
+
     # ---- end to end: inputs from pinned host memory, results back to the host, every step ----
     wl.e2e_setup()
     wl.e2e_step()
@@ -599,6 +643,7 @@ def main():
                                   "4x16x1024x1024 on channel partitions 2x2 and 2x2 feature-space workers; generalized "
                                   "all-to-all of fp32 8192x8192 between 8 row blocks and 8 column blocks",
                           **extra},
+            "small_config": small_cfg,
             "roofline": roofline,
             "clocks": clocks,
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes,

@@ -214,6 +214,38 @@ def test_halo_bf16_copies():
         assert same_bits(host(xs[w].view(torch.int16)).view(np.uint16), ref[w])
 
 
+def test_operator_calls_replay_from_a_cuda_graph():
+    """The calls only enqueue kernels on the given stream, so a captured sequence replays with the same bits."""
+    case = ((70, 66, 72), (2, 2, 2), 4, 4)
+    opart, gpart = make_partitions(case)
+    x, y = random_shards(opart, 41), random_shards(opart, 42)
+    xs, ys = [dev(a) for a in x], [dev(a) for a in y]
+    srcs = [dev(inputs.uniform_pm1((5000,), 4300 + i)) for i in range(3)]
+    red = torch.empty(5000, device=DEV)
+    # first calls outside the capture (one-time set-up of kernel attributes happens on first use)
+    distdl.halo_fwd(gpart, [t.clone() for t in xs])
+    distdl.halo_adj(gpart, [t.clone() for t in ys])
+    distdl.sumreduce_fwd(srcs, red)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            distdl.halo_fwd(gpart, xs)
+            distdl.halo_adj(gpart, ys)
+            distdl.sumreduce_fwd(srcs, red)
+    for t, a in zip(xs + ys, x + y):                 # capture does not run anything: restore and replay
+        t.copy_(dev(a))
+    red.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(xs, oracle.halo_fwd_sequence(opart, x)):
+        assert same_bits(host(a), b)
+    for a, b in zip(ys, oracle.halo_adj_sequence(opart, y)):
+        assert same_bits(host(a), b)
+    assert same_bits(host(red), oracle.sumreduce_fwd([host(t) for t in srcs]))
+
+
 # --------------------------------------------------------------------------
 # bfloat16 and fp64 variants of B, R, H, H*, all-reduce
 # --------------------------------------------------------------------------
