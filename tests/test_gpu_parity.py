@@ -921,3 +921,86 @@ def test_allreduce_bit_exact(k):
     torch.cuda.synchronize()
     for got, ref in zip(bufs, oracle.allreduce(parts)):
         assert same_bits(host(got), ref)
+
+
+# --------------------------------------------------------------------------
+# Seeded sweep over random small geometries (uneven splits, thin shards, ragged tiles)
+# --------------------------------------------------------------------------
+
+def _random_geometry(rng, rank, max_extent, max_workers, max_halo):
+    while True:
+        ps = [int(rng.integers(1, max_workers + 1)) for _ in range(rank)]
+        if int(np.prod(ps)) > 32:
+            continue
+        gs = [int(rng.integers(p * (max_halo + 1), max(p * (max_halo + 1) + 1, max_extent))) for p in ps]
+        return tuple(gs), tuple(ps)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_halo_geometries(seed):
+    rng = np.random.Generator(np.random.Philox(7000 + seed))
+    rank = int(rng.integers(1, 5))
+    gs, ps = _random_geometry(rng, rank, 40 if rank < 3 else 18, 4, 3)
+    per = tuple(bool(rng.integers(0, 2)) for _ in range(rank)) if seed % 3 == 0 else None
+    if per is None:
+        # per-worker widths, each no wider than the neighbour's bulk
+        sizes = [oracle.balanced_split(gs[k], ps[k])[1] for k in range(rank)]
+        hlo = [[int(rng.integers(0, min(3, sizes[k][c - 1]) + 1)) if c > 0 else int(rng.integers(0, 4)) for c in range(ps[k])]
+               for k in range(rank)]
+        hhi = [[int(rng.integers(0, min(3, sizes[k][c + 1]) + 1)) if c + 1 < ps[k] else int(rng.integers(0, 4))
+                for c in range(ps[k])] for k in range(rank)]
+        opart = oracle.Partition(gs, ps, hlo, hhi)
+        gpart = distdl.Partition(gs, ps, hlo, hhi)
+    else:
+        h = tuple(int(rng.integers(0, 4)) for _ in range(rank))
+        opart = oracle.Partition(gs, ps, h, h, per)
+        gpart = distdl.Partition(gs, ps, h, h, periodic=per)
+    x, y = random_shards(opart, 50 + seed), random_shards(opart, 80 + seed)
+    xs, ys = [dev(a) for a in x], [dev(a) for a in y]
+    distdl.halo_fwd(gpart, xs)
+    distdl.halo_adj(gpart, ys)
+    torch.cuda.synchronize()
+    for a, b in zip(xs, oracle.halo_fwd_sequence(opart, x)):
+        assert same_bits(host(a), b)
+    for a, b in zip(ys, oracle.halo_adj_sequence(opart, y)):
+        assert same_bits(host(a), b)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_stencil_and_repartition_geometries(seed):
+    rng = np.random.Generator(np.random.Philox(7100 + seed))
+    R = int(rng.integers(1, 5))
+    ps = tuple(int(rng.integers(1, 4)) for _ in range(3))
+    gs = tuple(int(rng.integers(p * R, p * R + 40)) for p in ps)
+    opart, obulk = oracle.Partition(gs, ps, R, R), oracle.Partition(gs, ps)
+    gpart = distdl.Partition(gs, ps, (R,) * 3, (R,) * 3)
+    w = inputs.normal((3, 2 * R + 1), 7200 + seed, 0.5)
+    xg = inputs.normal(gs, 7300 + seed)
+    x = oracle.scatter_global(opart, xg, fill=lambda wk: np.full(opart.padded_shape(wk), 1e30, dtype=np.float32))
+    ys = [torch.empty(obulk.padded_shape(k), device=DEV) for k in range(opart.num_workers)]
+    distdl.stencil3d_fwd(gpart, [dev(a) for a in x], w, ys)
+    dy = oracle.scatter_global(obulk, inputs.normal(gs, 7400 + seed))
+    dxs = [torch.full(opart.padded_shape(k), 5.0, device=DEV) for k in range(opart.num_workers)]
+    distdl.stencil3d_adj(gpart, [dev(a) for a in dy], w, dxs)
+    torch.cuda.synchronize()
+    xz = oracle.scatter_global(opart, xg)
+    eps = (6 * R + 5) * 2.0 ** -24
+    for got, ref, mag in ((ys, oracle.stencil3d_fwd(opart, xz, w), oracle.stencil3d_fwd(opart, [np.abs(a) for a in xz], np.abs(w))),
+                          (dxs, oracle.stencil3d_adj(opart, dy, w), oracle.stencil3d_adj(opart, [np.abs(a) for a in dy], np.abs(w)))):
+        for a, b, m in zip(got, ref, mag):
+            assert np.all(np.abs(host(a).astype(np.float64) - b) <= eps * m + 1e-30)
+    # the same tensor from this partition to another random one and back
+    ps2 = tuple(int(rng.integers(1, 4)) for _ in range(3))
+    if all(g >= p for g, p in zip(gs, ps2)):
+        rep = distdl.Repartition(gs, ps, ps2)
+        odst = oracle.Partition(gs, ps2)
+        src = oracle.scatter_global(obulk, xg)
+        dst = [torch.empty(odst.padded_shape(k), device=DEV) for k in range(odst.num_workers)]
+        back = [torch.empty(obulk.padded_shape(k), device=DEV) for k in range(obulk.num_workers)]
+        distdl.repartition_fwd(rep, [dev(a) for a in src], dst)
+        distdl.repartition_adj(rep, dst, back)
+        torch.cuda.synchronize()
+        for a, b in zip(dst, oracle.repartition_fwd(obulk, odst, src)):
+            assert same_bits(host(a), b)
+        for a, b in zip(back, src):
+            assert same_bits(host(a), b)
