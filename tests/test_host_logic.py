@@ -218,3 +218,18 @@ def test_validation_of_the_generalized_convolution():
     assert lib.distdl_convg_fwd(pb.handle, 6, 2, arr, arr, None, 5, 5, arr, None) == 4          # batch partitioned
     odd = (vp * 8)(*[0x10004 + 0x10000 * i for i in range(8)])
     assert lib.distdl_convg_fwd(px.handle, 6, 2, odd, arr, None, 5, 5, arr, None) == 3          # alignment
+
+
+def test_header_compiles_as_c_and_the_library_links_from_c(tmp_path):
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    exe = str(tmp_path / "host_check")
+    libdir = os.path.dirname(distdl.LIB_PATH)
+    subprocess.check_call([gcc, "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           os.path.join(ROOT, "tests", "c_abi", "host_check.c"), "-o", exe,
+                           "-L", libdir, "-ldistdl", "-Wl,-rpath," + libdir])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.strip().endswith("ok"), out.stdout + out.stderr
