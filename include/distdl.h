@@ -378,8 +378,9 @@ distdl_status_t distdl_pool_adj(const distdl_partition_t *p, const void *const *
  * dy[i] BF16 [nb, nfo/Pfo]      dx[j] F32 [nb, nfi/Pfi]
  * The contraction runs on the tensor cores with fp32 accumulation; the sums of R continue in the
  * same fp32 accumulator in the stated order.  nfi % Pfi == 0, nfo % Pfo == 0 (else
- * DISTDL_ERR_SHAPE); the per-worker block sizes nfi/Pfi and nfo/Pfo must be multiples of 128,
- * Pfo, Pfi <= 8 and Pfo * Pfi <= 16 (else DISTDL_ERR_UNSUPPORTED); nb >= 1 is arbitrary.
+ * DISTDL_ERR_SHAPE); the per-worker block sizes nfi/Pfi and nfo/Pfo must be multiples of 8 (rows of
+ * whole 16-byte units; tiles that reach past a block are filled with zeros on the way in and clipped
+ * on the way out), Pfo, Pfi <= 8 and Pfo * Pfi <= 16 (else DISTDL_ERR_UNSUPPORTED); nb >= 1 is arbitrary.
  * A launch whose device-side waits ran out reports through distdl_device_status().
  * ---------------------------------------------------------------------- */
 distdl_status_t distdl_affine_fwd(int64_t nb, int64_t nfi, int64_t nfo, int32_t pfo, int32_t pfi,

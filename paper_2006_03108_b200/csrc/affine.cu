@@ -185,10 +185,11 @@ affine_kernel(const __grid_constant__ AffineParams P) {
     const int row_tiles = (P.nb + rows_per_tile - 1) / rows_per_tile;
     const int m0 = (tile % row_tiles) * rows_per_tile + (int)rank * kTileM;   // this block's first row
     const int ntile = tile / row_tiles;
-    const int tiles_per_block = P.blk_out / kTileN;
+    const int tiles_per_block = (P.blk_out + kTileN - 1) / kTileN;   // the last tile of a block may be partly empty
     const int oblk = ntile / tiles_per_block;                  // output block (i forward, j adjoint)
     const int n0 = (ntile % tiles_per_block) * kTileN;         // first output column inside the block
-    const int kblocks_per_worker = P.blk_red / kBlockK;
+    // the last k-block of a worker may reach past its block: TMA fills both operands with zeros there
+    const int kblocks_per_worker = (P.blk_red + kBlockK - 1) / kBlockK;
     const int num_kblocks = P.nred * kblocks_per_worker;
 
     if (threadIdx.x == 0) {
@@ -339,6 +340,7 @@ affine_kernel(const __grid_constant__ AffineParams P) {
                 if (row < P.nb) {
 #pragma unroll
                     for (int q = 0; q < 32; q += 4) {
+                        if (n0 + c + q >= P.blk_out) continue;      // columns past the block (whole float4s: blocks are multiples of 8)
                         float4 o;
                         o.x = __uint_as_float(v[q + 0]);
                         o.y = __uint_as_float(v[q + 1]);
@@ -442,7 +444,7 @@ affine_kernel_quad(const __grid_constant__ AffineParams P) {
     const int tiles_per_block = P.blk_out / kQuadN;
     const int oblk = ntile / tiles_per_block;
     const int n0 = (ntile % tiles_per_block) * kQuadN;
-    const int kblocks_per_worker = P.blk_red / kBlockK;
+    const int kblocks_per_worker = (P.blk_red + kBlockK - 1) / kBlockK;
     const int workers = P.nred / 2;                  // workers summed by this pair
     const int r0 = (int)khalf * workers;             // first of them
     const int num_kblocks = workers * kblocks_per_worker;
@@ -632,6 +634,7 @@ struct AffineDwParams {
     int32_t nb, pfi;
     int32_t tiles_m, tiles_n;               // 128 x 128 tiles per worker block
     int32_t total_tiles;
+    int32_t bfi;                            // columns of a dW block
 };
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int32_t c0, int32_t c1) {
@@ -821,7 +824,9 @@ affine_dw_kernel(const __grid_constant__ AffineDwParams P) {
                 fence_proxy_async();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (issuer) {
-                    tma_store_2d(omap, boxaddr, t.n0 + 32 * q, t.m0);
+                    // a box that starts past the last column of the block has nothing to store (boxes that
+                    // only reach past it are clipped by the copy); its group is committed empty
+                    if (t.n0 + 32 * q < P.bfi) tma_store_2d(omap, boxaddr, t.n0 + 32 * q, t.m0);
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
@@ -854,11 +859,13 @@ __global__ void __launch_bounds__(kDbThreads) affine_db_kernel(const AffineDbPar
     const int b0 = warp * chunk, b1 = min(P.nb, b0 + chunk);
     const uint16_t *src = P.dy[i] + col;
     float s0 = 0.f, s1 = 0.f;
+    if (col < P.bfo) {
 #pragma unroll 8
-    for (int b = b0; b < b1; ++b) {
-        const uint32_t two = *reinterpret_cast<const uint32_t *>(src + (size_t)b * P.bfo);
-        s0 += __uint_as_float(two << 16);
-        s1 += __uint_as_float(two & 0xffff0000u);
+        for (int b = b0; b < b1; ++b) {
+            const uint32_t two = *reinterpret_cast<const uint32_t *>(src + (size_t)b * P.bfo);
+            s0 += __uint_as_float(two << 16);
+            s1 += __uint_as_float(two & 0xffff0000u);
+        }
     }
     part[warp][2 * lane] = s0;
     part[warp][2 * lane + 1] = s1;
@@ -867,7 +874,7 @@ __global__ void __launch_bounds__(kDbThreads) affine_db_kernel(const AffineDbPar
         float v = part[0][threadIdx.x];
 #pragma unroll
         for (int w = 1; w < kDbThreads / 32; ++w) v += part[w][threadIdx.x];
-        P.db[i][blockIdx.x * 64 + threadIdx.x] = v;
+        if (blockIdx.x * 64 + (int)threadIdx.x < P.bfo) P.db[i][blockIdx.x * 64 + threadIdx.x] = v;
     }
 }
 
@@ -898,8 +905,8 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
         return fail(DISTDL_ERR_INVALID_ARG, "%s: non-positive size", what);
     if (nfi % pfi || nfo % pfo) return fail(DISTDL_ERR_SHAPE, "%s: features not divisible by the worker grid", what);
     const int64_t bfi = nfi / pfi, bfo = nfo / pfo;
-    if (bfi % kTileN || bfo % kTileN)
-        return fail(DISTDL_ERR_UNSUPPORTED, "%s: per-worker feature blocks must be multiples of %d", what, kTileN);
+    if (bfi % 8 || bfo % 8)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: per-worker feature blocks must be multiples of 8 (rows of whole 16-byte units)", what);
     if (pfo > 8 || pfi > 8 || pfo * pfi > kMaxMaps - 8)
         return fail(DISTDL_ERR_UNSUPPORTED, "%s: worker grid larger than 8 per side or %d workers", what, kMaxMaps - 8);
     if (nb > (1 << 20)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: batch too large", what);
@@ -958,7 +965,8 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel_quad, cudaFuncAttributeMaxDynamicSharedMemorySize, kQuadSmemBytes));
         configured = true;
     }
-    const int64_t ntiles = (adjoint ? nfi : nfo) / kTileN;
+    const int64_t blk_out = adjoint ? bfi : bfo;
+    const int64_t ntiles = (adjoint ? pfi : pfo) * ((blk_out + kTileN - 1) / kTileN);
     if (quad) {
         const int64_t row_pairs = (nb + 2 * kTileM - 1) / (2 * kTileM);
         const int64_t qtiles = (adjoint ? nfi : nfo) / kQuadN;
@@ -1022,8 +1030,8 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
     if (nb < 1 || nfi < 1 || nfo < 1 || pfo < 1 || pfi < 1) return fail(DISTDL_ERR_INVALID_ARG, "%s: non-positive size", what);
     if (nfi % pfi || nfo % pfo) return fail(DISTDL_ERR_SHAPE, "%s: features not divisible by the worker grid", what);
     const int64_t bfi = nfi / pfi, bfo = nfo / pfo;
-    if (bfi % kTileN || bfo % kTileM)
-        return fail(DISTDL_ERR_UNSUPPORTED, "%s: per-worker feature blocks must be multiples of %d", what, kTileN);
+    if (bfi % 8 || bfo % 8)
+        return fail(DISTDL_ERR_UNSUPPORTED, "%s: per-worker feature blocks must be multiples of 8 (rows of whole 16-byte units)", what);
     if (pfo > 8 || pfi > 8 || pfo * pfi > kMaxMaps - 8)
         return fail(DISTDL_ERR_UNSUPPORTED, "%s: worker grid larger than 8 per side or %d workers", what, kMaxMaps - 8);
     if (nb > (1 << 20)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: batch too large", what);
@@ -1040,7 +1048,8 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
         if (!aligned16(dw[i])) return fail(DISTDL_ERR_ALIGNMENT, "%s: dW block %d not 16-byte aligned", what, i);
     }
     if (!encode_fn()) return fail(DISTDL_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", what);
-    const int64_t tiles = (bfo / kTileM) * (bfi / kTileN) * pfo * pfi;
+    // tiles past the end of a block are partly empty: loads are zero-filled and stores clipped by TMA
+    const int64_t tiles = ((bfo + kTileM - 1) / kTileM) * ((bfi + kTileN - 1) / kTileN) * pfo * pfi;
     if (tiles >= ((int64_t)1 << 31)) return fail(DISTDL_ERR_UNSUPPORTED, "%s: too many tiles", what);
 
     AffineDwParams P;
@@ -1053,9 +1062,10 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
         if (!make_map_f32(&P.dw_map[i], dw[i], bfo, bfi, 32, kTileM)) return fail(DISTDL_ERR_CUDA, "%s: tensor map of dW block %d failed", what, i);
     P.nb = (int32_t)nb;
     P.pfi = pfi;
-    P.tiles_m = (int32_t)(bfo / kTileM);
-    P.tiles_n = (int32_t)(bfi / kTileN);
+    P.tiles_m = (int32_t)((bfo + kTileM - 1) / kTileM);
+    P.tiles_n = (int32_t)((bfi + kTileN - 1) / kTileN);
     P.total_tiles = (int32_t)tiles;
+    P.bfi = (int32_t)bfi;
     static bool configured = false;
     static int sms = 0;
     if (!configured) {
@@ -1077,7 +1087,7 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
         }
         B.nb = (int32_t)nb;
         B.bfo = (int32_t)bfo;
-        dim3 grid((unsigned)(bfo / 64), (unsigned)pfo);
+        dim3 grid((unsigned)((bfo + 63) / 64), (unsigned)pfo);
         affine_db_kernel<<<grid, kDbThreads, 0, (cudaStream_t)stream>>>(B);
         DISTDL_CUDA_CHECK(cudaGetLastError());
     }

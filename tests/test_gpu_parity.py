@@ -664,6 +664,9 @@ AFFINE_CASES = [
     (300, 768, 256, 2, 1),
     (300, 1024, 1024, 2, 4),     # 256-column tiles, reduction split between two pairs (both directions)
     (520, 512, 768, 3, 2),       # forward splits the reduction, adjoint (three workers) does not
+    (40, 200, 136, 1, 1),        # blocks that are not multiples of the 128 / 64 tile sizes (multiples of 8)
+    (300, 400, 528, 2, 2),       # ... with pairs of blocks: blocks of 200 and 264 features
+    (150, 72, 1032, 3, 1),       # a reduction shorter than two k-blocks; 344-feature output blocks
 ]
 
 

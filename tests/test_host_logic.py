@@ -129,7 +129,7 @@ def test_operator_argument_validation_without_a_device():
     lib = distdl.lib()
     vp = ctypes.c_void_p
     arr = (vp * 4)(0x10000, 0x20000, 0x30000, 0x40000)
-    assert lib.distdl_affine_fwd(16, 100, 128, 1, 1, arr, arr, None, arr, None) == 4   # block not a multiple of 128
+    assert lib.distdl_affine_fwd(16, 100, 128, 1, 1, arr, arr, None, arr, None) == 4   # block not a multiple of 8
     assert lib.distdl_affine_fwd(16, 256, 256, 3, 1, arr, arr, None, arr, None) == 2   # not divisible by the grid
     assert lib.distdl_conv_fwd(part.handle, arr, vp(0x50000), None, 3, 3, arr, None) == 2  # not a rank-4 partition
     p4 = distdl.Partition((1, 2, 16, 16), (1, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2))
@@ -143,7 +143,7 @@ def test_validation_of_the_gradient_stencil_and_dtype_entry_points():
     vp = ctypes.c_void_p
     arr = (vp * 16)(*[0x10000 * (i + 1) for i in range(16)])
     # affine parameter gradients
-    assert lib.distdl_affine_adj_params(16, 100, 128, 1, 1, arr, arr, arr, None, None) == 4   # block not a multiple of 128
+    assert lib.distdl_affine_adj_params(16, 100, 128, 1, 1, arr, arr, arr, None, None) == 4   # block not a multiple of 8
     assert lib.distdl_affine_adj_params(16, 256, 256, 3, 1, arr, arr, arr, None, None) == 2   # not divisible by the grid
     assert lib.distdl_affine_adj_params(16, 256, 256, 1, 1, None, arr, arr, None, None) == 1  # NULL argument
     odd = (vp * 1)(0x10004)
