@@ -956,7 +956,11 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
     P.nred = adjoint ? pfo : pfi;
     P.adjoint = adjoint ? 1 : 0;
 
-    static bool configured = false;
+    // one-time set-up per device (kernel attributes, occupancy): a process may drive several GPUs
+    static bool configured_on[kMaxDevicesPerProcess] = {false};
+    int cur_dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
+    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                AffineCfg<false>::SMEM_BYTES));
@@ -1066,8 +1070,13 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
     P.tiles_n = (int32_t)((bfi + kTileN - 1) / kTileN);
     P.total_tiles = (int32_t)tiles;
     P.bfi = (int32_t)bfi;
-    static bool configured = false;
-    static int sms = 0;
+    // one-time set-up per device (kernel attributes, occupancy): a process may drive several GPUs
+    static bool configured_on[kMaxDevicesPerProcess] = {false};
+    int cur_dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
+    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    static int sms_on[kMaxDevicesPerProcess] = {0};
+    int &sms = sms_on[cur_dev % kMaxDevicesPerProcess];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemBytes));
         int dev = 0;

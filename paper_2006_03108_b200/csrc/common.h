@@ -23,6 +23,8 @@ void clear_error();
                                   cudaGetErrorString(e__));                              \
     } while (0)
 
+constexpr int kMaxDevicesPerProcess = 64;   // per-device one-time set-up flags are kept for this many devices
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int elem_size(distdl_dtype_t t) { return t == DISTDL_F32 ? 4 : (t == DISTDL_F64 ? 8 : 2); }
 inline bool valid_dtype(distdl_dtype_t t) { return t == DISTDL_F32 || t == DISTDL_BF16 || t == DISTDL_F64; }

@@ -712,8 +712,13 @@ static constexpr int conv_smem_bytes() {
 template <int K, bool ADJ>
 static distdl_status_t launch_conv(const ConvParams &P, int total_tiles, int tiles_y, int planes, cudaStream_t s) {
     constexpr int smem = conv_smem_bytes<K, ADJ>();
-    static bool configured = false;
-    static int blocks = 0;
+    // one-time set-up per device (kernel attributes, occupancy): a process may drive several GPUs
+    static bool configured_on[kMaxDevicesPerProcess] = {false};
+    int cur_dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
+    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    static int blocks_on[kMaxDevicesPerProcess] = {0};
+    int &blocks = blocks_on[cur_dev % kMaxDevicesPerProcess];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_depthwise_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         int dev = 0, sms = 0, per_sm = 0;
@@ -747,8 +752,13 @@ static distdl_status_t launch_conv_tma(const distdl_partition *p, ConvTmaParams 
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return fail(DISTDL_ERR_CUDA, "conv: tensor map of shard %d failed", wk);
     }
-    static bool configured = false;
-    static int blocks = 0;
+    // one-time set-up per device (kernel attributes, occupancy): a process may drive several GPUs
+    static bool configured_on[kMaxDevicesPerProcess] = {false};
+    int cur_dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
+    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    static int blocks_on[kMaxDevicesPerProcess] = {0};
+    int &blocks = blocks_on[cur_dev % kMaxDevicesPerProcess];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_tma_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES));
         int dev = 0, sms = 0, per_sm = 0;
@@ -1192,8 +1202,13 @@ static distdl_status_t launch_convg(const ConvGParams &G, int in_shards, const i
     using T = ConvTmaCfg<K, ADJ>;
     constexpr int smem_plain = 2 * C::TILE_FLOATS * 4 + 2 * kCob * K * K * 8;
     constexpr int smem_tma = 2 * T::TILE_STRIDE * 4 + 2 * T::SIDE_STRIDE * 4 + 2 * kCob * K * K * 8 + 64 + 128;
-    static bool configured = false;
-    static int blocks_plain = 0, blocks_tma = 0;
+    // one-time set-up per device (kernel attributes, occupancy): a process may drive several GPUs
+    static bool configured_on[kMaxDevicesPerProcess] = {false};
+    int cur_dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
+    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    static int blocks_plain_on[kMaxDevicesPerProcess] = {0}, blocks_tma_on[kMaxDevicesPerProcess] = {0};
+    int &blocks_plain = blocks_plain_on[cur_dev % kMaxDevicesPerProcess], &blocks_tma = blocks_tma_on[cur_dev % kMaxDevicesPerProcess];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_plain));
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_tma_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_tma));
@@ -1775,8 +1790,13 @@ static constexpr int grad_smem_bytes(bool tma) {
 // scratch table -- does not depend on which of them a call ends up using.
 template <int K>
 static distdl_status_t grad_config(int *blocks_out) {
-    static bool configured = false;
-    static int blocks = 0;
+    // one-time set-up per device (kernel attributes, occupancy): a process may drive several GPUs
+    static bool configured_on[kMaxDevicesPerProcess] = {false};
+    int cur_dev = 0;
+    DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
+    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    static int blocks_on[kMaxDevicesPerProcess] = {0};
+    int &blocks = blocks_on[cur_dev % kMaxDevicesPerProcess];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(false)));
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_tma_kernel<K, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(true)));
