@@ -668,13 +668,13 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.4
 
 NCU_TRAFFIC = {
     "broadcast_fwd": None,
-    "sumreduce_fwd": 4 * (134224128 + 5519616),
-    "halo_fwd": 203430912 + 116587264,
-    "halo_adj": 261940992 + 166233344,
-    "conv_fwd": 4 * (277958400 + 220996352),
-    "conv_adj": 4 * (269584384 + 227286784),
-    "affine_fwd": 138450176 + 3624704,
-    "affine_adj": 138434816 + 3114240,
+    "sumreduce_fwd": 4 * (134225152 + 5290496),
+    "halo_fwd": 204656128 + 117036544,
+    "halo_adj": 261646336 + 164815616,
+    "conv_fwd": 4 * (278041088 + 221260288),
+    "conv_adj": 4 * (269701888 + 228404480),
+    "affine_fwd": 138435072 + 3728128,
+    "affine_adj": 138447104 + 3240448,
 }
 
 if __name__ == "__main__":
