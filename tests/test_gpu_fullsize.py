@@ -35,6 +35,44 @@ def test_broadcast_and_sumreduce_full_size():
     assert host(out).tobytes() == oracle.sumreduce_fwd(parts).tobytes()
 
 
+def _long_vector(n, seed):
+    """n fp32 values on the device: a seeded block of 2^24 values repeated, plus the number of the repeat
+    (exact in fp32), so that no two positions 2^24 k apart, and none 2^31 or 2^32 apart, hold the same value."""
+    blk = 1 << 24
+    block = dev(inputs.uniform_pm1((blk,), seed))
+    x = torch.empty(n, device=DEV)
+    for seg in range((n + blk - 1) // blk):
+        lo, hi = seg * blk, min(n, (seg + 1) * blk)
+        torch.add(block[: hi - lo], float(seg), out=x[lo:hi])
+    return x
+
+
+def test_broadcast_and_sumreduce_beyond_2_to_31_elements():
+    """Element counts above 2^31 (and byte counts above 2^33) with a ragged tail: the copies are compared
+    in full as bit patterns on the device, the fold against the oracle on windows at the start, around
+    element 2^31 and at the end, and against the single correctly rounded fp32 sum everywhere."""
+    n = (1 << 31) + (1 << 20) + 3
+    windows = [(0, 1 << 16), ((1 << 31) - (1 << 16), (1 << 31) + (1 << 16)), (n - (1 << 16) - 3, n)]
+    x = _long_vector(n, 2101)
+    dst = [torch.empty(n, device=DEV) for _ in range(2)]
+    distdl.broadcast_fwd(x, dst)
+    torch.cuda.synchronize()
+    for d in dst:
+        assert torch.equal(d.view(torch.int32), x.view(torch.int32))
+        for lo, hi in windows:
+            assert host(d[lo:hi]).tobytes() == host(x[lo:hi]).tobytes()
+    del dst
+    y = _long_vector(n, 2102)
+    out = torch.empty(n, device=DEV)
+    distdl.sumreduce_fwd([x, y], out)
+    torch.cuda.synchronize()
+    for lo, hi in windows:
+        ref = oracle.sumreduce_fwd([host(x[lo:hi]), host(y[lo:hi])])
+        assert host(out[lo:hi]).tobytes() == ref.tobytes()
+    y.add_(x)                        # fp32 addition of two values has one correctly rounded result
+    assert torch.equal(out.view(torch.int32), y.view(torch.int32))
+
+
 def test_halo_3d_full_size():
     gs, ps, h = (512,) * 3, (4,) * 3, 4
     opart = oracle.Partition(gs, ps, h, h)
