@@ -73,6 +73,40 @@ def test_broadcast_and_sumreduce_beyond_2_to_31_elements():
     assert torch.equal(out.view(torch.int32), y.view(torch.int32))
 
 
+def test_halo_on_shards_just_below_2_to_31_elements():
+    """Two padded shards of 32770 x 65530 cells (2,147,418,100 each, 8.6 GB: cell offsets up to 2^31, byte
+    offsets above 2^33), one interface between them.  The rows next to the interface are compared with
+    the oracle run on those rows alone (a problem with one bulk row per worker has the same exchange);
+    everything else by what H and H* leave behind: exterior ghosts zero, the rest of the bulk untouched."""
+    R, C = 32770, 65530
+    gs, ps = (2 * (R - 2), C - 2), (2, 1)
+    gpart = distdl.Partition(gs, ps, (1, 1), (1, 1))
+    mini = oracle.Partition((2, C - 2), ps, 1, 1)
+    rows = [slice(R - 3, R), slice(0, 3)]           # worker 0: its last three rows; worker 1: its first three
+
+    def check(call, seq, seed, adjoint):
+        x = [_long_vector(R * C, seed + w).view(R, C) for w in range(2)]
+        small = [host(x[w][rows[w]]) for w in range(2)]
+        call(gpart, x)
+        torch.cuda.synchronize()
+        ref = seq(mini, small)
+        # the mini problem's own exterior row (row 0 of worker 0, row 2 of worker 1) is a bulk row here
+        assert host(x[0][R - 2:R]).tobytes() == ref[0][1:3].tobytes()
+        assert host(x[1][0:2]).tobytes() == ref[1][0:2].tobytes()
+        for w in range(2):
+            keep = _long_vector(R * C, seed + w).view(R, C)
+            inner = slice(1, R - 2) if w == 0 else slice(2, R - 1)      # bulk rows away from the interface
+            assert torch.equal(x[w][inner, 1:C - 1].view(torch.int32), keep[inner, 1:C - 1].view(torch.int32))
+            del keep
+            assert not x[w][:, 0].any() and not x[w][:, C - 1].any()
+            assert not x[w][0 if w == 0 else R - 1].any()
+            if adjoint:
+                assert not x[w][R - 1 if w == 0 else 0].any()
+
+    check(distdl.halo_fwd, oracle.halo_fwd_sequence, 2201, False)
+    check(distdl.halo_adj, oracle.halo_adj_sequence, 2211, True)
+
+
 def test_halo_3d_full_size():
     gs, ps, h = (512,) * 3, (4,) * 3, 4
     opart = oracle.Partition(gs, ps, h, h)
