@@ -172,6 +172,49 @@ def test_conv_full_size_on_sampled_planes():
         assert float(t[:, :, :, :2].abs().max()) == 0.0 and float(t[:, :, :, -2:].abs().max()) == 0.0
 
 
+def test_conv_on_shards_just_below_2_to_31_elements():
+    """Four padded shards of 1982 x 16 planes of 260 x 260 cells (2,143,731,200 cells, 8.6 GB each): the
+    last planes start at cell offsets just below 2^31.  Sampled planes against the oracle, as above."""
+    N, C = 1982, 16
+    gs, ps = (N, C, 512, 512), (1, 1, 2, 2)
+    gpart = distdl.Partition(gs, ps, (0, 0, 2, 2), (0, 0, 2, 2))
+    g = torch.Generator(device=DEV)
+    g.manual_seed(6)
+    w = inputs.normal((C, 5, 5), 5002, 0.1)
+    planes = [(0, 0), (1000, 7), (N - 1, 0), (N - 1, C - 1)]
+    sub = (1, 1, 512, 512)
+    op = oracle.Partition(sub, ps, (0, 0, 2, 2), (0, 0, 2, 2))
+
+    xs = [torch.randn(N, C, 260, 260, device=DEV, generator=g) for _ in range(4)]
+    ys = [torch.empty(N, C, 256, 256, device=DEV) for _ in range(4)]
+    distdl.conv_fwd(gpart, xs, dev(w), None, ys)
+    distdl.device_status()
+    for n, c in planes:
+        x1 = [host(t[n:n + 1, c:c + 1]) for t in xs]
+        yref = oracle.conv_fwd(op, x1, w[c:c + 1])
+        ybound = oracle.conv_fwd(op, [np.abs(a) for a in x1], np.abs(w[c:c + 1]))
+        for k in range(4):
+            got = host(ys[k][n:n + 1, c:c + 1]).astype(np.float64)
+            assert np.all(np.abs(got - yref[k]) <= 27 * 2.0 ** -24 * ybound[k] + 1e-30)
+    del xs, ys
+    torch.cuda.empty_cache()
+
+    dys = [torch.randn(N, C, 256, 256, device=DEV, generator=g) for _ in range(4)]
+    dxs = [torch.full((N, C, 260, 260), 7.0, device=DEV) for _ in range(4)]
+    distdl.conv_adj(gpart, dys, dev(w), dxs)
+    distdl.device_status()
+    for n, c in planes:
+        dy1 = [host(t[n:n + 1, c:c + 1]) for t in dys]
+        dxref = oracle.conv_adj(op, dy1, w[c:c + 1])
+        dxbound = oracle.conv_adj(op, [np.abs(a) for a in dy1], np.abs(w[c:c + 1]))
+        for k in range(4):
+            gotx = host(dxs[k][n:n + 1, c:c + 1])
+            assert np.all(np.abs(gotx.astype(np.float64) - dxref[k]) <= 27 * 2.0 ** -24 * dxbound[k] + 1e-30)
+    for t in dxs:
+        assert float(t[:, :, :2, :].abs().max()) == 0.0 and float(t[:, :, -2:, :].abs().max()) == 0.0
+        assert float(t[:, :, :, :2].abs().max()) == 0.0 and float(t[:, :, :, -2:].abs().max()) == 0.0
+
+
 def test_affine_full_size():
     nb, nf, pf = 256, 8192, 4
     blk = nf // pf
