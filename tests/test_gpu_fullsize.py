@@ -283,17 +283,18 @@ def test_pool_full_size_on_sampled_planes():
     assert abs(total_dx - total_dy) <= 1e-6 * sum(float(t.double().abs().sum()) for t in dys)
 
 
-def test_stencil3d_full_size_on_sampled_boxes():
-    # the configuration bench.py times: 512^3 on 4 x 4 x 4 workers, radius 4
-    gs, ps, R = (512,) * 3, (4,) * 3, 4
+def _stencil3d_on_sampled_boxes(gs, ps, R, boxes, seed, dot_test):
+    P = ps[0] * ps[1] * ps[2]
+    bk = tuple(g // q for g, q in zip(gs, ps))                     # bulk extents (the splits are even)
+    pad = tuple(v + 2 * R for v in bk)
     gpart = distdl.Partition(gs, ps, (R,) * 3, (R,) * 3)
     g = torch.Generator(device=DEV)
-    g.manual_seed(11)
-    xs = [torch.randn(136, 136, 136, device=DEV, generator=g) for _ in range(64)]
-    dys = [torch.randn(128, 128, 128, device=DEV, generator=g) for _ in range(64)]
-    w = inputs.normal((3, 9), 7001, 0.5)
-    ys = [torch.empty(128, 128, 128, device=DEV) for _ in range(64)]
-    dxs = [torch.full((136, 136, 136), 7.0, device=DEV) for _ in range(64)]
+    g.manual_seed(seed)
+    xs = [torch.randn(*pad, device=DEV, generator=g) for _ in range(P)]
+    dys = [torch.randn(*bk, device=DEV, generator=g) for _ in range(P)]
+    w = inputs.normal((3, 2 * R + 1), 7001, 0.5)
+    ys = [torch.empty(*bk, device=DEV) for _ in range(P)]
+    dxs = [torch.full(pad, 7.0, device=DEV) for _ in range(P)]
     distdl.stencil3d_fwd(gpart, xs, w, ys)
     distdl.stencil3d_adj(gpart, dys, w, dxs)
     torch.cuda.synchronize()
@@ -301,23 +302,22 @@ def test_stencil3d_full_size_on_sampled_boxes():
     def gather(shards, off, lo, hi):
         """Global box [lo, hi) put together from the bulks of the device shards (bulk offset `off` inside a shard)."""
         out = np.zeros(tuple(b - a for a, b in zip(lo, hi)), dtype=np.float32)
-        for s in range(64):
-            c = (s // 16, (s // 4) % 4, s % 4)
-            a = [max(lo[k], 128 * c[k]) for k in range(3)]
-            b = [min(hi[k], 128 * c[k] + 128) for k in range(3)]
+        for s in range(P):
+            c = (s // (ps[1] * ps[2]), (s // ps[2]) % ps[1], s % ps[2])
+            a = [max(lo[k], bk[k] * c[k]) for k in range(3)]
+            b = [min(hi[k], bk[k] * c[k] + bk[k]) for k in range(3)]
             if any(a[k] >= b[k] for k in range(3)):
                 continue
-            src = tuple(slice(a[k] - 128 * c[k] + off, b[k] - 128 * c[k] + off) for k in range(3))
+            src = tuple(slice(a[k] - bk[k] * c[k] + off, b[k] - bk[k] * c[k] + off) for k in range(3))
             dst = tuple(slice(a[k] - lo[k], b[k] - lo[k]) for k in range(3))
             out[dst] = host(shards[s][src])
         return out
 
     eps = (6 * R + 5) * 2.0 ** -24
-    # boxes at a corner of the tensor, where eight shards meet, across a face, and at the far corner
-    for lo in [(0, 0, 0), (120, 120, 120), (250, 380, 120), (492, 492, 492)]:
+    for lo in boxes:
         hi = tuple(v + 20 for v in lo)
         elo = tuple(max(v - R, 0) for v in lo)
-        ehi = tuple(min(v + R, 512) for v in hi)
+        ehi = tuple(min(v + R, n) for v, n in zip(hi, gs))
         one = oracle.Partition(tuple(b - a for a, b in zip(elo, ehi)), (1, 1, 1), R, R)
         inner = tuple(slice(l - e, l - e + 20) for l, e in zip(lo, elo))
         for shards_in, off_in, got_shards, off_out, fn in ((xs, R, ys, 0, oracle.stencil3d_fwd), (dys, 0, dxs, R, oracle.stencil3d_adj)):
@@ -337,12 +337,27 @@ def test_stencil3d_full_size_on_sampled_boxes():
         assert float(t[:R].abs().max()) == 0.0 and float(t[-R:].abs().max()) == 0.0
         assert float(t[:, :R].abs().max()) == 0.0 and float(t[:, -R:].abs().max()) == 0.0
         assert float(t[:, :, :R].abs().max()) == 0.0 and float(t[:, :, -R:].abs().max()) == 0.0
-    # dot test over the whole volume, fp64 on the device (x's ghost storage does not take part)
-    lhs = sum(float((a.double() * b.double()).sum()) for a, b in zip(ys, dys))
-    rhs = sum(float((a[R:-R, R:-R, R:-R].double() * b[R:-R, R:-R, R:-R].double()).sum()) for a, b in zip(xs, dxs))
-    ny = sum(float((a.double() ** 2).sum()) for a in ys) ** 0.5
-    ndy = sum(float((a.double() ** 2).sum()) for a in dys) ** 0.5
-    assert abs(lhs - rhs) <= 1e-5 * ny * ndy
+    if dot_test:
+        # dot test over the whole volume, fp64 on the device (x's ghost storage does not take part)
+        lhs = sum(float((a.double() * b.double()).sum()) for a, b in zip(ys, dys))
+        rhs = sum(float((a[R:-R, R:-R, R:-R].double() * b[R:-R, R:-R, R:-R].double()).sum()) for a, b in zip(xs, dxs))
+        ny = sum(float((a.double() ** 2).sum()) for a in ys) ** 0.5
+        ndy = sum(float((a.double() ** 2).sum()) for a in dys) ** 0.5
+        assert abs(lhs - rhs) <= 1e-5 * ny * ndy
+
+
+def test_stencil3d_full_size_on_sampled_boxes():
+    # the configuration bench.py times: 512^3 on 4 x 4 x 4 workers, radius 4; boxes at a corner of the
+    # tensor, where eight shards meet, across a face, and at the far corner
+    _stencil3d_on_sampled_boxes((512,) * 3, (4,) * 3, 4, [(0, 0, 0), (120, 120, 120), (250, 380, 120), (492, 492, 492)],
+                                11, True)
+
+
+def test_stencil3d_on_shards_just_below_2_to_31_elements():
+    # two padded shards of 1288^3 = 2,136,719,872 cells (8.5 GB each); boxes at the first cells, across the
+    # interface between the two workers (the last planes of worker 0, the first of worker 1) and at the far corner
+    _stencil3d_on_sampled_boxes((2560, 1280, 1280), (2, 1, 1), 4,
+                                [(0, 0, 0), (1270, 600, 1260), (1270, 1260, 1260), (2540, 1260, 1260)], 12, False)
 
 
 def test_parameter_gradients_full_size():
