@@ -241,20 +241,22 @@ def test_affine_full_size():
     assert oracle.adjoint_test_ratio([host(t) for t in y], dyf, xf, [host(t) for t in dx]) < 1e-4
 
 
-def test_pool_full_size_on_sampled_planes():
-    # the configuration bench.py times: 3 x 3 max pooling, stride 2, padding 1, ghost widths (1, 0) per worker
-    gs, ps, k, s, pad = (16, 16, 1024, 1024), (1, 1, 4, 4), (3, 3), (2, 2), ((1, 1), (1, 1))
-    sub = (1, 1, 1024, 1024)
+def _pool_on_sampled_planes(N, C, image, ps, planes, seed):
+    # 3 x 3 max pooling, stride 2, padding 1: ghost widths (1, 0) per worker
+    gs, k, s, pad = (N, C) + image, (3, 3), (2, 2), ((1, 1), (1, 1))
+    sub = (1, 1) + image
+    P = ps[2] * ps[3]
     opart, geo = oracle.pool_partition(sub, ps, k, s, pad)
     gpart = distdl.Partition(gs, ps, [list(h) for h in opart.hlo], [list(h) for h in opart.hhi])
+    oshape = (N, C, image[0] // 2 // ps[2], image[1] // 2 // ps[3])
     g = torch.Generator(device=DEV)
-    g.manual_seed(7)
-    xs = [torch.randn(*gpart.padded_shape(w), device=DEV, generator=g) for w in range(16)]
-    ys = [torch.empty(16, 16, 128, 128, device=DEV) for _ in range(16)]
-    args = [torch.full((16, 16, 128, 128), -1, dtype=torch.int32, device=DEV) for _ in range(16)]
-    dys = [torch.randn(16, 16, 128, 128, device=DEV, generator=g) for _ in range(16)]
-    dxs = [torch.full(tuple(gpart.padded_shape(w)), 7.0, device=DEV) for w in range(16)]
-    x_before = {(n, c): [host(t[n:n + 1, c:c + 1]) for t in xs] for n, c in [(0, 0), (5, 11), (15, 15)]}
+    g.manual_seed(seed)
+    xs = [torch.randn(*gpart.padded_shape(w), device=DEV, generator=g) for w in range(P)]
+    ys = [torch.empty(oshape, device=DEV) for _ in range(P)]
+    args = [torch.full(oshape, -1, dtype=torch.int32, device=DEV) for _ in range(P)]
+    dys = [torch.randn(oshape, device=DEV, generator=g) for _ in range(P)]
+    dxs = [torch.full(tuple(gpart.padded_shape(w)), 7.0, device=DEV) for w in range(P)]
+    x_before = {(n, c): [host(t[n:n + 1, c:c + 1]) for t in xs] for n, c in planes}
     distdl.pool_fwd(gpart, xs, k, s, pad, distdl.POOL_MAX, ys, args)
     distdl.pool_adj(gpart, dys, args, k, s, pad, distdl.POOL_MAX, dxs)
     torch.cuda.synchronize()
@@ -262,7 +264,7 @@ def test_pool_full_size_on_sampled_planes():
         yref, aref = oracle.pool_fwd(opart, geo, x1, k, s, pad, "max")
         dy1 = [host(t[n:n + 1, c:c + 1]) for t in dys]
         dxref = oracle.pool_adj(opart, geo, dy1, k, s, pad, "max", aref)
-        for w in range(16):
+        for w in range(P):
             assert host(ys[w][n:n + 1, c:c + 1]).tobytes() == yref[w].tobytes()
             assert np.array_equal(host(args[w][n:n + 1, c:c + 1]), aref[w])
             got = host(dxs[w][n:n + 1, c:c + 1])
@@ -270,7 +272,7 @@ def test_pool_full_size_on_sampled_planes():
             assert np.max(np.abs(got - dxref[w])) <= 8 * 2.0 ** -24 * 4 * float(np.max(np.abs(dy1[w])))
     # properties at full size: every recorded position is a window position, ghosts of dx are zero,
     # and the adjoint routes all of dy (sum preserved up to fp32 rounding)
-    for w in range(16):
+    for w in range(P):
         assert int(args[w].min()) >= 0 and int(args[w].max()) <= 8
         lo, hi = opart.widths(w)
         t = dxs[w]
@@ -278,9 +280,19 @@ def test_pool_full_size_on_sampled_planes():
             assert float(t[:, :, :lo[2], :].abs().max()) == 0.0
         if lo[3]:
             assert float(t[:, :, :, :lo[3]].abs().max()) == 0.0
-    total_dx = sum(float(t.double().sum()) for t in dxs)
-    total_dy = sum(float(t.double().sum()) for t in dys)
-    assert abs(total_dx - total_dy) <= 1e-6 * sum(float(t.double().abs().sum()) for t in dys)
+    total_dx = sum(float(t.sum(dtype=torch.float64)) for t in dxs)
+    total_dy = sum(float(t.sum(dtype=torch.float64)) for t in dys)
+    assert abs(total_dx - total_dy) <= 1e-6 * sum(float(t.abs().sum(dtype=torch.float64)) for t in dys)
+
+
+def test_pool_full_size_on_sampled_planes():
+    # the configuration bench.py times
+    _pool_on_sampled_planes(16, 16, (1024, 1024), (1, 1, 4, 4), [(0, 0), (5, 11), (15, 15)], 7)
+
+
+def test_pool_on_shards_just_below_2_to_31_elements():
+    # four padded shards of 2031 x 16 planes of 257 x 257 cells: 2,146,328,304 cells (8.6 GB) each
+    _pool_on_sampled_planes(2031, 16, (512, 512), (1, 1, 2, 2), [(0, 0), (1017, 5), (2030, 0), (2030, 15)], 8)
 
 
 def _stencil3d_on_sampled_boxes(gs, ps, R, boxes, seed, dot_test):
@@ -423,6 +435,34 @@ def test_repartition_full_size():
         assert host(a).tobytes() == b.tobytes()
     for a, b in zip(back, rows):
         assert host(a).tobytes() == b.tobytes()
+
+
+def test_repartition_on_shards_just_below_2_to_31_elements():
+    """Two row blocks <-> two column blocks of a 46340 x 92672 matrix: every shard holds 2,147,210,240
+    cells (8.6 GB).  The sixteen rows and columns around the point where all four shards meet are compared
+    with the oracle on that window alone (its even split falls on the same lines); every cell with the
+    plain definition, a re-slicing of the matrix, on the device."""
+    nr, nc = 46340, 92672
+    rep = distdl.Repartition((nr, nc), (2, 1), (1, 2))
+    src = [_long_vector(nr // 2 * nc, 8100 + i).view(nr // 2, nc) for i in range(2)]
+    dst = [torch.empty(nr, nc // 2, device=DEV) for _ in range(2)]
+    distdl.repartition_fwd(rep, src, dst)
+    torch.cuda.synchronize()
+    h = 8
+    win = [host(src[0][-h:, nc // 2 - h:nc // 2 + h]), host(src[1][:h, nc // 2 - h:nc // 2 + h])]
+    ref = oracle.repartition_fwd(oracle.Partition((2 * h, 2 * h), (2, 1)), oracle.Partition((2 * h, 2 * h), (1, 2)), win)
+    assert host(dst[0][nr // 2 - h:nr // 2 + h, -h:]).tobytes() == ref[0].tobytes()
+    assert host(dst[1][nr // 2 - h:nr // 2 + h, :h]).tobytes() == ref[1].tobytes()
+    for j in range(2):
+        for i in range(2):
+            a = dst[j][i * (nr // 2):(i + 1) * (nr // 2)]
+            b = src[i][:, j * (nc // 2):(j + 1) * (nc // 2)]
+            assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    back = [torch.empty(nr // 2, nc, device=DEV) for _ in range(2)]
+    distdl.repartition_adj(rep, dst, back)
+    torch.cuda.synchronize()
+    for a, b in zip(back, src):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
 
 
 def test_generalized_conv_full_size_on_samples():
