@@ -241,6 +241,42 @@ def test_affine_full_size():
     assert oracle.adjoint_test_ratio([host(t) for t in y], dyf, xf, [host(t) for t in dx]) < 1e-4
 
 
+def test_affine_on_the_largest_batch():
+    """nb = 2^20 rows (the most the layer accepts), 4096 x 4096 weights on 2 x 2 workers: every output block
+    holds 2^31 values (8.6 GB).  Rows of the batch are independent, so windows of rows at the start, the middle
+    and the end are compared with the oracle run on those rows."""
+    nb, nf, pf = 1 << 20, 4096, 2
+    blk = nf // pf
+    wb = inputs.f32_to_bf16_bits(inputs.normal((nf, nf), 6011, nf ** -0.5))
+    bf = lambda a: dev(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+    ws = [b for row in np.split(wb, pf, axis=0) for b in np.split(row, pf, axis=1)]
+    w_d = [bf(a) for a in ws]
+    g = torch.Generator(device=DEV)
+    g.manual_seed(13)
+    xs = [torch.randn(nb, blk, device=DEV, generator=g).to(torch.bfloat16) for _ in range(pf)]
+    dys = [torch.randn(nb, blk, device=DEV, generator=g).to(torch.bfloat16) for _ in range(pf)]
+    y = [torch.full((nb, blk), float("nan"), device=DEV) for _ in range(pf)]
+    dx = [torch.full((nb, blk), float("nan"), device=DEV) for _ in range(pf)]
+    distdl.affine_fwd(nb, nf, nf, pf, pf, xs, w_d, None, y)
+    distdl.affine_adj(nb, nf, nf, pf, pf, dys, w_d, dx)
+    distdl.device_status()
+    f64 = oracle.bf16_bits_to_f64
+    bits = lambda t: host(t.view(torch.int16)).view(np.uint16)
+    wf = [f64(a) for a in ws]
+    for lo, hi in [(0, 128), (nb // 2 - 64, nb // 2 + 64), (nb - 128, nb)]:
+        xf = [f64(bits(t[lo:hi])) for t in xs]
+        dyf = [f64(bits(t[lo:hi])) for t in dys]
+        yref, dxref = oracle.affine_fwd(xf, wf, pf, pf), oracle.affine_adj(dyf, wf, pf, pf)
+        for got, ref in ((y, yref), (dx, dxref)):
+            gg = np.concatenate([host(t[lo:hi]).astype(np.float64) for t in got], axis=1)
+            r = np.concatenate([a.astype(np.float64) for a in ref], axis=1)
+            assert np.max(np.abs(gg - r)) / np.max(np.abs(r)) < 2e-2
+            assert np.linalg.norm(gg - r) / np.linalg.norm(r) < 1e-4
+    # every one of the 2^31 values of a block was written (the blocks were filled with NaN)
+    for t in y + dx:
+        assert bool(torch.isfinite(t).all())
+
+
 def _pool_on_sampled_planes(N, C, image, ps, planes, seed):
     # 3 x 3 max pooling, stride 2, padding 1: ghost widths (1, 0) per worker
     gs, k, s, pad = (N, C) + image, (3, 3), (2, 2), ((1, 1), (1, 1))
