@@ -20,6 +20,14 @@ dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
 host = lambda t: t.cpu().numpy()
 
 
+def _need_free_gb(gb):
+    """The largest-size cases hold tens of GB on the device; they are skipped where that much is not free."""
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < gb * (1 << 30):
+        pytest.skip("needs %d GB of free device memory, %.0f GB are free" % (gb, free / (1 << 30)))
+
+
 def test_broadcast_and_sumreduce_full_size():
     k, shape = 8, (4096, 4096)
     x = inputs.uniform_pm1(shape, 2001)
@@ -51,6 +59,7 @@ def test_broadcast_and_sumreduce_beyond_2_to_31_elements():
     """Element counts above 2^31 (and byte counts above 2^33) with a ragged tail: the copies are compared
     in full as bit patterns on the device, the fold against the oracle on windows at the start, around
     element 2^31 and at the end, and against the single correctly rounded fp32 sum everywhere."""
+    _need_free_gb(40)
     n = (1 << 31) + (1 << 20) + 3
     windows = [(0, 1 << 16), ((1 << 31) - (1 << 16), (1 << 31) + (1 << 16)), (n - (1 << 16) - 3, n)]
     x = _long_vector(n, 2101)
@@ -78,6 +87,7 @@ def test_halo_on_shards_just_below_2_to_31_elements():
     offsets above 2^33), one interface between them.  The rows next to the interface are compared with
     the oracle run on those rows alone (a problem with one bulk row per worker has the same exchange);
     everything else by what H and H* leave behind: exterior ghosts zero, the rest of the bulk untouched."""
+    _need_free_gb(40)
     R, C = 32770, 65530
     gs, ps = (2 * (R - 2), C - 2), (2, 1)
     gpart = distdl.Partition(gs, ps, (1, 1), (1, 1))
@@ -175,6 +185,7 @@ def test_conv_full_size_on_sampled_planes():
 def test_conv_on_shards_just_below_2_to_31_elements():
     """Four padded shards of 1982 x 16 planes of 260 x 260 cells (2,143,731,200 cells, 8.6 GB each): the
     last planes start at cell offsets just below 2^31.  Sampled planes against the oracle, as above."""
+    _need_free_gb(80)
     N, C = 1982, 16
     gs, ps = (N, C, 512, 512), (1, 1, 2, 2)
     gpart = distdl.Partition(gs, ps, (0, 0, 2, 2), (0, 0, 2, 2))
@@ -245,6 +256,7 @@ def test_affine_on_the_largest_batch():
     """nb = 2^20 rows (the most the layer accepts), 4096 x 4096 weights on 2 x 2 workers: every output block
     holds 2^31 values (8.6 GB).  Rows of the batch are independent, so windows of rows at the start, the middle
     and the end are compared with the oracle run on those rows."""
+    _need_free_gb(70)
     nb, nf, pf = 1 << 20, 4096, 2
     blk = nf // pf
     wb = inputs.f32_to_bf16_bits(inputs.normal((nf, nf), 6011, nf ** -0.5))
@@ -328,6 +340,7 @@ def test_pool_full_size_on_sampled_planes():
 
 def test_pool_on_shards_just_below_2_to_31_elements():
     # four padded shards of 2031 x 16 planes of 257 x 257 cells: 2,146,328,304 cells (8.6 GB) each
+    _need_free_gb(120)
     _pool_on_sampled_planes(2031, 16, (512, 512), (1, 1, 2, 2), [(0, 0), (1017, 5), (2030, 0), (2030, 15)], 8)
 
 
@@ -404,6 +417,7 @@ def test_stencil3d_full_size_on_sampled_boxes():
 def test_stencil3d_on_shards_just_below_2_to_31_elements():
     # two padded shards of 1288^3 = 2,136,719,872 cells (8.5 GB each); boxes at the first cells, across the
     # interface between the two workers (the last planes of worker 0, the first of worker 1) and at the far corner
+    _need_free_gb(80)
     _stencil3d_on_sampled_boxes((2560, 1280, 1280), (2, 1, 1), 4,
                                 [(0, 0, 0), (1270, 600, 1260), (1270, 1260, 1260), (2540, 1260, 1260)], 12, False)
 
@@ -478,6 +492,7 @@ def test_repartition_on_shards_just_below_2_to_31_elements():
     cells (8.6 GB).  The sixteen rows and columns around the point where all four shards meet are compared
     with the oracle on that window alone (its even split falls on the same lines); every cell with the
     plain definition, a re-slicing of the matrix, on the device."""
+    _need_free_gb(70)
     nr, nc = 46340, 92672
     rep = distdl.Repartition((nr, nc), (2, 1), (1, 2))
     src = [_long_vector(nr // 2 * nc, 8100 + i).view(nr // 2, nc) for i in range(2)]
