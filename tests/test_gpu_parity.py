@@ -370,6 +370,9 @@ CONV_CASES = [
     ((1, 1, 70, 260), (1, 1, 2, 2), 7),      # the same for K = 7; the last tile column holds 2 < 3 columns
     ((1, 2, 66, 264), (1, 1, 2, 2), 5),      # the last tile row holds 1 < 2 rows: the tile above it reaches into the halo
     ((1, 1, 68, 260), (1, 1, 2, 2), 7),      # 2 < 3 rows and 2 < 3 columns
+    ((1, 2, 70, 272), (1, 1, 2, 2), 5),      # bulk widths of whole groups of eight columns (136), two tile columns of 128 + 8
+    ((1, 2, 70, 272), (1, 1, 2, 2), 3),      # the same for the adjoint of K = 3 (rows 8-byte aligned)
+    ((1, 1, 70, 528), (1, 1, 2, 2), 7),      # and of K = 7 (264 columns per worker)
 ]
 
 
