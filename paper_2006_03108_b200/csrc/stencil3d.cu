@@ -69,7 +69,7 @@ __device__ __forceinline__ bool st_owner(const int32_t *b, int p, int s, int c, 
 }
 
 template <int R, bool VEC>
-__global__ void __launch_bounds__(kStThreads, 3)
+__global__ void __launch_bounds__(kStThreads, 4)
 stencil3d_kernel(const __grid_constant__ StencilParams P) {
     __shared__ __align__(16) float plane[2][kStRows + 2 * R][kStPitch];
     constexpr int N = 2 * R + 1;
