@@ -1064,8 +1064,9 @@ struct ConvGTmaParams {
     CUtensorMap in_map[kConvGTmaShards];
 };
 
+// Four blocks per SM where the register tile allows it without spills (5 x 5), three otherwise.
 template <int K, bool ADJ>
-__global__ void __launch_bounds__(kConvThreads, 3)
+__global__ void __launch_bounds__(kConvThreads, K == 5 ? 4 : 3)
 convg_tma_kernel(const __grid_constant__ ConvGTmaParams Q) {
     using C = ConvCfg<K, ADJ>;
     using T = ConvTmaCfg<K, ADJ>;
