@@ -88,7 +88,7 @@ __device__ __forceinline__ uint32_t dot_stride(const uint32_t *coord, const uint
 // Copy / clear tile (H, and the ghost clears of H*): T = uint4 (16 bytes), float, unsigned short.
 // Each thread keeps kCopyBatch independent loads in flight.
 // ---------------------------------------------------------------------------------------------
-constexpr int kCopyBatch = 4;
+constexpr int kCopyBatch = 8;
 
 template <typename T>
 __device__ __forceinline__ void run_copy_tile(const HaloBox &box, const HaloSource *src, int nsrc,
