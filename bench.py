@@ -669,7 +669,7 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.4
 NCU_TRAFFIC = {
     "broadcast_fwd": None,
     "sumreduce_fwd": 4 * (134225152 + 5290496),
-    "halo_fwd": 204656128 + 117036544,
+    "halo_fwd": 203393024 + 116994304,
     "halo_adj": 261646336 + 164815616,
     "conv_fwd": 4 * (278041088 + 221260288),
     "conv_adj": 4 * (269701888 + 228404480),
