@@ -670,7 +670,7 @@ NCU_TRAFFIC = {
     "broadcast_fwd": None,
     "sumreduce_fwd": 4 * (134225152 + 5290496),
     "halo_fwd": 203393024 + 116994304,
-    "halo_adj": 261646336 + 164815616,
+    "halo_adj": 261256448 + 164833792,
     "conv_fwd": 4 * (278041088 + 221260288),
     "conv_adj": 4 * (269701888 + 228404480),
     "affine_fwd": 138435072 + 3728128,

@@ -143,7 +143,7 @@ __device__ __forceinline__ void stores_after(const bf16x1 &v) { asm volatile("" 
 template <typename T, int NSRC>
 __device__ __forceinline__ void run_sum_tile_balanced(const HaloBox &box, const HaloSource *src,
                                                       const ShardPointers &sh, uint32_t first, uint32_t count) {
-    constexpr int U = NSRC >= 8 ? 1 : (NSRC == 4 ? 2 : 4);   // units per thread per batch
+    constexpr int U = NSRC >= 8 ? 1 : (NSRC == 4 ? 2 : 8);   // units per thread per batch
     const int nd = box.ndim;
     T *base[NSRC];
 #pragma unroll
