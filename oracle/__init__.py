@@ -3,7 +3,7 @@
 TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, deliberately naive
 numpy restatement of what the operators compute (broadcast B, sum-reduce R = B*,
 halo exchange H, adjoint halo exchange H*, the generalized all-to-all with scatter and
-gather as special cases, all-reduce, the distributed depthwise convolution, the 3-D star-stencil layer,
+gather as special cases, all-reduce, the broadcast / sum-reduce along partition dimensions, the distributed depthwise convolution, the 3-D star-stencil layer,
 the distributed pooling layer and the distributed affine layer, each with its adjoint).  Nothing in the product
 package imports it; only the test-suite, the smoke check and the CPU-baseline leg
 of the benchmark may call it.  It shares no code, table or helper with the CUDA
@@ -33,6 +33,8 @@ from .primitives import (  # noqa: F401
     repartition_fwd,
     repartition_adj,
     allreduce,
+    partition_broadcast_fwd,
+    partition_broadcast_adj,
     round_to_bf16_bits,
     bf16_add,
 )

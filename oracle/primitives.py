@@ -359,3 +359,57 @@ def allreduce(parts, add=None):
     """All-reduce = broadcast after sum-reduce (self-adjoint): every worker ends up with
     the fixed-order sum of all k realisations."""
     return broadcast_fwd(sumreduce_fwd(parts, add), len(parts))
+
+
+# --------------------------------------------------------------------------
+# Partition broadcast / sum-reduce along partition dimensions
+# (Section 4, "Sparse layers": the forward and adjoint convolution algorithms and the two
+# footnotes on broadcasting along partitions; "Dense layers": the affine algorithms)
+# --------------------------------------------------------------------------
+
+def _partition_sources(src_pshape, dst_pshape):
+    """For every worker of the destination partition (row-major id) the worker of the source
+    partition whose realisation it receives.
+
+    The rule is NumPy's broadcasting rule applied to the two partition shapes, from source to
+    destination only: along a partition dimension where the source has one worker and the
+    destination has several, that one worker's realisation goes to all of them; along every other
+    dimension both partitions have the same number of workers and coordinates correspond.
+    """
+    src_pshape, dst_pshape = tuple(int(v) for v in src_pshape), tuple(int(v) for v in dst_pshape)
+    assert len(src_pshape) == len(dst_pshape)
+    for a, b in zip(src_pshape, dst_pshape):
+        assert a == b or a == 1, "a partition dimension broadcasts only from one worker"
+    out = []
+    for w in range(int(np.prod(dst_pshape))):
+        coords, rest = [], w
+        for p in reversed(dst_pshape):
+            coords.append(rest % p)
+            rest //= p
+        coords.reverse()
+        src = 0
+        for k, c in enumerate(coords):
+            src = src * src_pshape[k] + (c if src_pshape[k] > 1 else 0)
+        out.append(src)
+    return out
+
+
+def partition_broadcast_fwd(src_pshape, dst_pshape, shards):
+    """B_{{P_x} -> {P_w}}: every worker of the destination partition gets a copy of the realisation
+    held by its source worker (x^ <- B x in the forward algorithms; dy^ <- B dy in the adjoint ones)."""
+    src_of = _partition_sources(src_pshape, dst_pshape)
+    assert len(shards) == int(np.prod(src_pshape))
+    return [np.array(shards[j], copy=True) for j in src_of]
+
+
+def partition_broadcast_adj(src_pshape, dst_pshape, dy_shards, add=None):
+    """R_{{P_w} -> {P_x}} = B*: every worker of the smaller partition gets the sum of the realisations
+    of the workers that its own realisation was (or would be) broadcast to, taken in the order of
+    their worker ids, in the arithmetic of the inputs (y <- R y^ in the forward algorithms; dx <- R dx^
+    in the adjoint ones)."""
+    src_of = _partition_sources(src_pshape, dst_pshape)
+    assert len(dy_shards) == len(src_of)
+    out = []
+    for j in range(int(np.prod(src_pshape))):
+        out.append(sumreduce_fwd([dy_shards[w] for w in range(len(src_of)) if src_of[w] == j], add))
+    return out

@@ -653,6 +653,86 @@ def test_allreduce_is_symmetric_and_gives_every_worker_the_sum():
 
 
 # --------------------------------------------------------------------------
+# Broadcast / sum-reduce along partition dimensions (Section 4: the B and R of the layer algorithms)
+# --------------------------------------------------------------------------
+
+PARTITION_BROADCAST_CASES = [
+    # source partition, destination partition, elements of every source realisation
+    ((1,), (4,), [5]),
+    ((1, 3), (2, 3), [2, 3, 1]),                       # the affine layer's x: 1 x P_fi -> P_fo x P_fi
+    ((2, 1), (2, 3), [2, 3]),                          # its y: P_fo x 1 <- P_fo x P_fi
+    ((1, 1, 2, 2, 1), (1, 3, 2, 2, 1), [1, 2, 3, 2]),  # the convolution's x: 1 x 1 x P_ci x P_0 x P_1 -> 1 x P_co x P_ci x P_0 x P_1
+    ((1, 2, 1, 2), (1, 2, 3, 2), [2, 1, 1, 3]),        # its y: 1 x P_co x 1 x P_0 <- 1 x P_co x P_ci x P_0
+    ((2, 2), (2, 2), [1, 2, 3, 4]),                    # equal partitions: the identity
+]
+
+
+def _pb_matrix(src_p, dst_p, sizes, adjoint):
+    """The operator as a dense matrix, one column per unit vector, through the oracle."""
+    src_of = oracle.primitives._partition_sources(src_p, dst_p)
+    in_sizes = [sizes[j] for j in src_of] if adjoint else sizes
+    total = sum(in_sizes)
+    cols = []
+    for e in range(total):
+        u = np.zeros(total, np.float32)
+        u[e] = 1
+        parts, at = [], 0
+        for n in in_sizes:
+            parts.append(u[at:at + n])
+            at += n
+        out = (oracle.partition_broadcast_adj(src_p, dst_p, parts) if adjoint
+               else oracle.partition_broadcast_fwd(src_p, dst_p, parts))
+        cols.append(np.concatenate(out))
+    return np.stack(cols, axis=1)
+
+
+@pytest.mark.parametrize("case", PARTITION_BROADCAST_CASES, ids=[str(c[0]) + "->" + str(c[1]) for c in PARTITION_BROADCAST_CASES])
+def test_partition_broadcast_is_the_stacked_identity_matrix_and_its_adjoint_the_transpose(case):
+    src_p, dst_p, sizes = case
+    B = _pb_matrix(src_p, dst_p, sizes, False)
+    # built by hand, without the oracle: destination worker w (row-major coordinates) copies source worker j, whose
+    # coordinates are w's where the source partition has several workers and 0 where it has one
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    blocks = []
+    for w in np.ndindex(*dst_p):
+        j = int(np.ravel_multi_index([c if p > 1 else 0 for c, p in zip(w, src_p)], src_p))
+        blk = np.zeros((sizes[j], offs[-1]), np.float32)
+        blk[:, offs[j]:offs[j + 1]] = np.eye(sizes[j], dtype=np.float32)
+        blocks.append(blk)
+    assert np.array_equal(B, np.concatenate(blocks, axis=0))
+    assert np.array_equal(_pb_matrix(src_p, dst_p, sizes, True), B.T)
+    copies = int(np.prod(dst_p)) // int(np.prod(src_p))
+    assert np.array_equal(B.T @ B, copies * np.eye(offs[-1], dtype=np.float32))       # R B = k I
+
+
+def test_partition_broadcast_special_cases_order_of_the_sum_and_dot_test():
+    x = inputs.uniform_pm1((1000,), 5)
+    out = oracle.partition_broadcast_fwd((1,), (5,), [x])                   # one source worker: the plain broadcast
+    assert all(a.tobytes() == b.tobytes() for a, b in zip(out, oracle.broadcast_fwd(x, 5)))
+    ys = [inputs.uniform_pm1((1000,), 60 + i) for i in range(5)]
+    assert oracle.partition_broadcast_adj((1,), (5,), ys)[0].tobytes() == oracle.sumreduce_fwd(ys).tobytes()
+    # order of the sum: in a 1 x 2 -> 3 x 2 partition pair source worker 1 gets (y1 + y3) + y5
+    big, one = np.float32(2.0 ** 24), np.float32(1.0)
+    ys = [np.zeros(1, np.float32), np.array([big]), np.zeros(1, np.float32), np.array([one]), np.zeros(1, np.float32),
+          np.array([one])]
+    got = oracle.partition_broadcast_adj((1, 2), (3, 2), ys)
+    assert got[1][0] == big                                                 # (2^24 + 1) + 1 stays 2^24 in fp32 ...
+    ys[1], ys[5] = ys[5], ys[1]
+    assert oracle.partition_broadcast_adj((1, 2), (3, 2), ys)[1][0] == big + np.float32(2.0)   # ... (1 + 1) + 2^24 does not
+    # bfloat16 sums through the same hook as the other folds
+    b = [oracle.round_to_bf16_bits(inputs.uniform_pm1((64,), 70 + i).astype(np.float64)) for i in range(4)]
+    ref = oracle.sumreduce_fwd([b[0], b[2]], add=oracle.bf16_add)
+    assert np.array_equal(oracle.partition_broadcast_adj((1, 2), (2, 2), b, add=oracle.bf16_add)[0], ref)
+    # adjoint test on random data
+    src_p, dst_p, sizes = (1, 3), (4, 3), [50, 70, 30]
+    xs = [inputs.uniform_pm1((n,), 80 + i) for i, n in enumerate(sizes)]
+    ys = [inputs.uniform_pm1((sizes[w % 3],), 90 + w) for w in range(12)]
+    r = oracle.adjoint_test_ratio(oracle.partition_broadcast_fwd(src_p, dst_p, xs), ys, xs,
+                                  oracle.partition_broadcast_adj(src_p, dst_p, ys))
+    assert r < 1e-6
+
+
+# --------------------------------------------------------------------------
 # Parameter gradients of the two layers (adjoint algorithms of Section 4: dW, db / dw, db)
 # --------------------------------------------------------------------------
 
