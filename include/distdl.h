@@ -149,6 +149,37 @@ distdl_status_t distdl_sumreduce_adj(const void *dy, void *const *dx, int32_t k,
                                      distdl_dtype_t t, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Broadcast and sum-reduce along partition dimensions (Section 4, "Sparse layers": the broadcasts
+ * B_{P_x -> P_w} and reductions R_{P_w -> P_y} of the forward and adjoint convolution algorithms and
+ * the two footnotes on broadcasting along partitions; "Dense layers": the same operators in the
+ * affine algorithms).
+ *
+ * Two Cartesian worker partitions of the same rank: along every dimension the destination has as
+ * many workers as the source, or the source has exactly one (NumPy's broadcasting rule on the two
+ * partition shapes, from source to destination only).  Worker ids are row-major in both.  The
+ * destination worker with coordinates c copies the source worker whose coordinates are c where
+ * the source partition has several workers and 0 where it has one.
+ *   partition_broadcast_fwd: dst[w] <- src[source of w]  for every w < Pdst (bit copies)
+ *   partition_broadcast_adj: dx[j] <- sum of dy[w] over the destination workers w whose source is
+ *       j, in ascending w, starting from the first (one addition per element and term, rounded
+ *       once to the type): the sum-reduce R = B*, e.g. y <- R y^ with the roles of the two
+ *       partitions as here (the smaller one receives).
+ * elems[j]: elements of source worker j's realisation (its copies have the same size), j < Psrc.
+ * src / dx: Psrc device pointers; dst / dy: Pdst device pointers (host arrays); all 16-byte
+ * aligned.  A dst[w] equal to its source is left alone (the in-place form of the broadcast); dx[j]
+ * may alias the first of its terms only.  rank 1..DISTDL_MAX_RANK, Pdst <= DISTDL_MAX_WORKERS.
+ * Errors: DISTDL_ERR_SHAPE for partition shapes that do not broadcast, else as broadcast_fwd.
+ * ---------------------------------------------------------------------- */
+distdl_status_t distdl_partition_broadcast_fwd(int32_t rank, const int32_t *src_partition_shape,
+                                               const int32_t *dst_partition_shape, const int64_t *elems,
+                                               const void *const *src, void *const *dst, distdl_dtype_t t,
+                                               void *stream);
+distdl_status_t distdl_partition_broadcast_adj(int32_t rank, const int32_t *src_partition_shape,
+                                               const int32_t *dst_partition_shape, const int64_t *elems,
+                                               const void *const *dy, void *const *dx, distdl_dtype_t t,
+                                               void *stream);
+
+/* ------------------------------------------------------------------------
  * Halo exchange H and its adjoint H* (Section 3, "Halo exchange": the H and H* operator
  * sequences; Appendix B.2), in place on the P padded shards.
  *
@@ -164,6 +195,12 @@ distdl_status_t distdl_sumreduce_adj(const void *dy, void *const *dx, int32_t k,
  * ---------------------------------------------------------------------- */
 distdl_status_t distdl_halo_fwd(const distdl_partition_t *p, void *const *shards, void *stream);
 distdl_status_t distdl_halo_adj(const distdl_partition_t *p, void *const *shards, void *stream);
+/* 1 if H (adjoint = 0) or H* (adjoint != 0) of this partition runs through the row plan -- every ghost
+ * width and bulk extent of the innermost dimension is a whole number of 16-byte units, so ghost rows are
+ * moved end to end as aligned vectors; for H* also: every bulk is at least as wide as the ghosts its two
+ * neighbours hold of it together, and at most two of the outer dimensions have neighbours -- 0 if it runs
+ * through the general box plan, -1 for a NULL partition.  Same results, bit for bit, either way. */
+int32_t         distdl_partition_uses_row_plan(const distdl_partition_t *p, int32_t adjoint);
 
 /* ------------------------------------------------------------------------
  * distdl_halo_fwd_noalloc: the halo exchange H for callers that must not allocate device memory.
@@ -184,7 +221,10 @@ distdl_status_t distdl_halo_adj(const distdl_partition_t *p, void *const *shards
  * the 1 MiB array, else DISTDL_ERR_UNSUPPORTED with the sizes in the message -- e.g. 64 workers
  * in 3-D with 128^3 shards need about 0.36 MiB, 256 workers in 3-D do not fit.
  * The first call on a device looks up the device address of the array (one cudaGetSymbolAddress
- * with that device current); make that first call outside any stream capture.
+ * with that device current).  No call may be made on a stream that is being captured: the tables
+ * are copied from host memory that is freed on return, so the call answers DISTDL_ERR_UNSUPPORTED
+ * there and records nothing.  Like any copy from pageable host memory, the table copies may also
+ * keep the host waiting until earlier work on `stream` has drained.
  * All calls share the one array: the tables of the previous call stay in it and are overwritten,
  * entry by entry as far as the new plan reaches, before the kernel of this call reads them.  Two
  * calls whose work overlaps on the GPU (different streams, no ordering between them) race on the

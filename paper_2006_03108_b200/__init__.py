@@ -57,11 +57,14 @@ def lib():
     L.distdl_partition_num_workers.argtypes = [vp]
     L.distdl_partition_shard_extents.argtypes = [vp, c_i32, pi64, pi64, pi64, pi32, pi32]
     L.distdl_partition_halo_stats.argtypes = [vp, c_i32, pi64, pi64, pi64]
+    L.distdl_partition_uses_row_plan.argtypes = [vp, c_i32]
     L.distdl_halo_widths_1d.argtypes = [c_i64, c_i32, c_i32, c_i32, c_i32, c_i32, c_i32, pi32, pi32, pi32, pi32]
     L.distdl_broadcast_fwd.argtypes = [vp, pvp, c_i32, c_i64, c_i32, vp]
     L.distdl_sumreduce_adj.argtypes = [vp, pvp, c_i32, c_i64, c_i32, vp]
     L.distdl_sumreduce_fwd.argtypes = [pvp, vp, c_i32, c_i64, c_i32, vp]
     L.distdl_broadcast_adj.argtypes = [pvp, vp, c_i32, c_i64, c_i32, vp]
+    L.distdl_partition_broadcast_fwd.argtypes = [c_i32, pi32, pi32, pi64, pvp, pvp, c_i32, vp]
+    L.distdl_partition_broadcast_adj.argtypes = [c_i32, pi32, pi32, pi64, pvp, pvp, c_i32, vp]
     L.distdl_halo_fwd.argtypes = [vp, pvp, vp]
     L.distdl_halo_adj.argtypes = [vp, pvp, vp]
     L.distdl_halo_fwd_noalloc.argtypes = [c_i32, pi64, pi32, pi32, pi32, c_i32, pvp, vp]
@@ -88,6 +91,8 @@ def lib():
     L.distdl_convg_adj_params_workspace.argtypes = [vp, c_i64, c_i32, c_i32, c_i32, pi64]
     L.distdl_convg_adj_params.argtypes = [vp, c_i64, c_i32, pvp, pvp, c_i32, c_i32, pvp, pvp, vp, c_i64, vp]
     L.distdl_device_status.argtypes = [vp]
+    L.distdl_selftest_wait_timeout.argtypes = [c_i64, vp]
+    L.distdl_selftest_row_plan.argtypes = [vp, c_i32, pi32, c_i32, pi32, c_i32, pi32]
     _lib = L
     return L
 
@@ -207,6 +212,10 @@ class Partition:
                                                  ctypes.byref(b), ctypes.byref(c)))
         return a.value, b.value, c.value
 
+    def uses_row_plan(self, adjoint=False):
+        """True if H (or H*) of this partition runs through the row plan (rows of whole 16-byte units)."""
+        return lib().distdl_partition_uses_row_plan(self._h, 1 if adjoint else 0) == 1
+
     def close(self):
         if self._h:
             lib().distdl_partition_destroy(self._h)
@@ -248,6 +257,30 @@ def sumreduce_fwd(srcs, dst, stream=None):
 def broadcast_adj(dys, dx, stream=None):
     _check(lib().distdl_broadcast_adj(_ptr_array(dys), _ptr(dx), len(dys), dx.numel(), _dtype_code(dx),
                                       _stream(stream)))
+
+
+def _partition_pair(src_pshape, dst_pshape, small):
+    rank = len(src_pshape)
+    if len(dst_pshape) != rank:
+        raise ValueError("partition shapes differ in rank")
+    sp = (ctypes.c_int32 * rank)(*[int(v) for v in src_pshape])
+    dp = (ctypes.c_int32 * rank)(*[int(v) for v in dst_pshape])
+    el = (ctypes.c_int64 * len(small))(*[t.numel() for t in small])
+    return rank, sp, dp, el
+
+
+def partition_broadcast_fwd(src_pshape, dst_pshape, src, dst, stream=None):
+    """dst[w] <- src[source of w]: broadcast along the partition dimensions where src_pshape is 1."""
+    rank, sp, dp, el = _partition_pair(src_pshape, dst_pshape, src)
+    _check(lib().distdl_partition_broadcast_fwd(rank, sp, dp, el, _ptr_array(src), _ptr_array(dst), _dtype_code(src[0]),
+                                                _stream(stream)))
+
+
+def partition_broadcast_adj(src_pshape, dst_pshape, dy, dx, stream=None):
+    """dx[j] <- sum, in worker order, of the dy[w] whose source is j: the sum-reduce back to the smaller partition."""
+    rank, sp, dp, el = _partition_pair(src_pshape, dst_pshape, dx)
+    _check(lib().distdl_partition_broadcast_adj(rank, sp, dp, el, _ptr_array(dy), _ptr_array(dx), _dtype_code(dx[0]),
+                                                _stream(stream)))
 
 
 def halo_fwd(part, shards, stream=None):
@@ -427,3 +460,18 @@ def conv_adj_params(part, x, dy, kernel, dw, db, workspace, stream=None):
 def device_status(stream=None):
     """Synchronises the stream and raises DistdlError(DISTDL_ERR_TIMEOUT) if an affine kernel gave up."""
     _check(lib().distdl_device_status(_stream(stream)))
+
+
+def selftest_wait_timeout(limit_cycles, stream=None):
+    """Runs the bounded wait of the tensor-core kernels on a barrier nobody signals (include/distdl_selftest.h);
+    the following device_status() raises DistdlError(DISTDL_ERR_TIMEOUT) once."""
+    _check(lib().distdl_selftest_wait_timeout(int(limit_cycles), _stream(stream)))
+
+
+def selftest_row_plan(part, adjoint=False):
+    """(header words, list of 16-word records) of a partition's row plan (include/distdl_selftest.h)."""
+    hdr = (ctypes.c_int32 * 64)()
+    rec = (ctypes.c_int32 * (16 * 64))()
+    n = ctypes.c_int32(0)
+    _check(lib().distdl_selftest_row_plan(part.handle, 1 if adjoint else 0, hdr, 64, rec, 16 * 64, ctypes.byref(n)))
+    return list(hdr), [list(rec[16 * i:16 * i + 16]) for i in range(n.value)]

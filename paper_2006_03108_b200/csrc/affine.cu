@@ -55,7 +55,8 @@ struct AffineParams {
 // the pipeline when it sits on the critical path of every k-block), and the clock is only looked
 // at once in a while.
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles) {
     long long t0 = 0;
     for (unsigned spins = 0;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -63,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitCycles) {
+            if (now - t0 > limit_cycles) {
                 *abort_flag = 1;
                 atomicExch(&g_affine_status, (int)DISTDL_ERR_TIMEOUT);
                 return false;
@@ -1125,6 +1126,31 @@ extern "C" distdl_status_t distdl_affine_adj_params(int64_t nb, int64_t nfi, int
 
 namespace distdl {
 int conv_take_status();   // conv.cu
+
+// Self-test of the bounded wait: one thread waits, through the same mbar_wait as the kernels above, on a
+// barrier that nobody arrives at.  The wait gives up after `limit_cycles`, records DISTDL_ERR_TIMEOUT in the
+// status word and the kernel returns by itself.
+__global__ void selftest_wait_kernel(long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+        mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_cycles);
+    }
+}
+}
+
+extern "C" distdl_status_t distdl_selftest_wait_timeout(int64_t limit_cycles, void *stream) {
+    using namespace distdl;
+    clear_error();
+    // the limit of the self-test stays short: at most about a tenth of a second of SM clock cycles
+    if (limit_cycles < 1 || limit_cycles > 200000000ll)
+        return fail(DISTDL_ERR_INVALID_ARG, "selftest_wait_timeout: limit outside 1 .. 2e8 cycles");
+    selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((long long)limit_cycles);
+    DISTDL_CUDA_CHECK(cudaGetLastError());
+    return DISTDL_OK;
 }
 
 extern "C" distdl_status_t distdl_device_status(void *stream) {

@@ -5,6 +5,7 @@
 // once, several independent loads in flight per thread; 16-byte accesses, and 32-byte ones in the
 // broadcast when every pointer allows them.
 #include <algorithm>
+#include <vector>
 
 #include "common.h"
 
@@ -284,7 +285,82 @@ static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t
     return DISTDL_OK;
 }
 
+// Broadcast / sum-reduce along partition dimensions (Section 4, the B and R of the layer algorithms): the
+// destination partition repeats the source partition along the dimensions where the source has one worker.
+// For every worker of the destination partition (row-major id) the worker of the source partition it copies.
+static distdl_status_t partition_sources(int32_t rank, const int32_t *src_p, const int32_t *dst_p, std::vector<int32_t> *src_of,
+                                         int32_t *num_src, const char *what) {
+    if (!src_p || !dst_p) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL partition shape", what);
+    if (rank < 1 || rank > DISTDL_MAX_RANK) return fail(DISTDL_ERR_INVALID_ARG, "%s: rank %d outside 1..%d", what, rank, DISTDL_MAX_RANK);
+    int64_t ns = 1, nd = 1;
+    for (int k = 0; k < rank; ++k) {
+        if (src_p[k] < 1 || dst_p[k] < 1) return fail(DISTDL_ERR_SHAPE, "%s: partition dimension %d is not positive", what, k);
+        if (src_p[k] != dst_p[k] && src_p[k] != 1)
+            return fail(DISTDL_ERR_SHAPE, "%s: partition dimension %d has %d source and %d destination workers (equal, or one source worker)",
+                        what, k, src_p[k], dst_p[k]);
+        ns *= src_p[k];
+        nd *= dst_p[k];
+        if (nd > DISTDL_MAX_WORKERS) return fail(DISTDL_ERR_UNSUPPORTED, "%s: more than %d workers", what, DISTDL_MAX_WORKERS);
+    }
+    src_of->resize((size_t)nd);
+    for (int64_t w = 0; w < nd; ++w) {
+        int32_t c[DISTDL_MAX_RANK];
+        int64_t rest = w;
+        for (int k = rank - 1; k >= 0; --k) {
+            c[k] = (int32_t)(rest % dst_p[k]);
+            rest /= dst_p[k];
+        }
+        int32_t j = 0;
+        for (int k = 0; k < rank; ++k) j = j * src_p[k] + (src_p[k] > 1 ? c[k] : 0);
+        (*src_of)[(size_t)w] = j;
+    }
+    *num_src = (int32_t)ns;
+    return DISTDL_OK;
+}
+
+static distdl_status_t partition_broadcast_impl(int32_t rank, const int32_t *src_p, const int32_t *dst_p, const int64_t *elems,
+                                                const void *const *small, const void *const *big, distdl_dtype_t t,
+                                                void *stream, bool adjoint, const char *what) {
+    clear_error();
+    if (!elems || !small || !big) return fail(DISTDL_ERR_INVALID_ARG, "%s: NULL argument", what);
+    std::vector<int32_t> src_of;
+    int32_t ns = 0;
+    distdl_status_t st = partition_sources(rank, src_p, dst_p, &src_of, &ns, what);
+    if (st != DISTDL_OK) return st;
+    for (int32_t j = 0; j < ns; ++j) {
+        if (elems[j] < 0) return fail(DISTDL_ERR_INVALID_ARG, "%s: negative element count for source worker %d", what, j);
+        if (!small[j]) return fail(DISTDL_ERR_INVALID_ARG, "%s: buffer of source-partition worker %d is NULL", what, j);
+    }
+    for (size_t w = 0; w < src_of.size(); ++w)
+        if (!big[w]) return fail(DISTDL_ERR_INVALID_ARG, "%s: buffer of destination-partition worker %zu is NULL", what, w);
+    std::vector<void *> group;
+    for (int32_t j = 0; j < ns; ++j) {
+        group.clear();
+        for (size_t w = 0; w < src_of.size(); ++w)
+            if (src_of[w] == j) group.push_back(const_cast<void *>(big[w]));      // ascending worker id: the order of the sum
+        st = adjoint ? sumreduce_impl(group.data(), const_cast<void *>(small[j]), (int32_t)group.size(), elems[j], t, stream, what)
+                     : broadcast_impl(small[j], group.data(), (int32_t)group.size(), elems[j], t, stream, what);
+        if (st != DISTDL_OK) return st;
+    }
+    return DISTDL_OK;
+}
+
 }  // namespace distdl
+
+extern "C" distdl_status_t distdl_partition_broadcast_fwd(int32_t rank, const int32_t *src_partition_shape,
+                                                          const int32_t *dst_partition_shape, const int64_t *elems,
+                                                          const void *const *src, void *const *dst, distdl_dtype_t t,
+                                                          void *stream) {
+    return distdl::partition_broadcast_impl(rank, src_partition_shape, dst_partition_shape, elems, src,
+                                            reinterpret_cast<const void *const *>(dst), t, stream, false, "partition_broadcast_fwd");
+}
+extern "C" distdl_status_t distdl_partition_broadcast_adj(int32_t rank, const int32_t *src_partition_shape,
+                                                          const int32_t *dst_partition_shape, const int64_t *elems,
+                                                          const void *const *dy, void *const *dx, distdl_dtype_t t,
+                                                          void *stream) {
+    return distdl::partition_broadcast_impl(rank, src_partition_shape, dst_partition_shape, elems,
+                                            reinterpret_cast<const void *const *>(dx), dy, t, stream, true, "partition_broadcast_adj");
+}
 
 extern "C" distdl_status_t distdl_broadcast_fwd(const void *src, void *const *dst, int32_t k, int64_t n,
                                                 distdl_dtype_t t, void *stream) {

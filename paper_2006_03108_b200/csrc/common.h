@@ -93,6 +93,62 @@ struct HaloPlanDevice {
     int32_t num_tiles = 0;
 };
 
+// ---------------------------------------------------------------------------------------------
+// Row plan of the halo kernels: used when every ghost width and bulk extent of the innermost
+// dimension is a whole number of 16-byte units, so that all ghost cells can be moved as aligned
+// vectors.  The geometry of a Cartesian partition is separable: where a ghost cell's value lives
+// follows, dimension by dimension, from the worker's coordinate along that dimension alone.  The
+// plan is therefore one small record per (dimension, worker coordinate); the kernels derive
+// everything else (which rows are ghost rows, their source rows in the neighbours) from it.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxFastCoords = 64;    // sum over the dimensions of the workers along each
+
+struct FastDim {
+    int32_t n, hlo, b;                // padded extent, low ghost width, bulk extent (innermost dimension: in units)
+    int32_t lo_c, hi_c;               // coordinate of the low / high neighbour along this dimension, -1: none
+    int32_t lo_shift, hi_shift;       // index in that neighbour's padded range minus the own index of the same cell
+    int32_t rlo, rhi;                 // bulk cells at the low / high end that the neighbour there holds ghost copies of
+    // x / e == umulhi(x, magic) >> shift for x < 2^31 (magic 0: e <= 1, the quotient is x), for the extents
+    // e = n, b, g = n - b (ghost cells), bi = b - rlo - rhi (bulk cells out of every neighbour's reach), rr = rlo + rhi
+    uint32_t magic_n, magic_b, magic_g, magic_bi, magic_rr;
+    uint32_t shifts;                  // shift of n | b << 6 | g << 12 | bi << 18 | rr << 24
+    int32_t pad_;
+};
+static_assert(sizeof(FastDim) == 64, "FastDim layout");
+
+__host__ __device__ inline uint32_t fast_shift_n(const FastDim &f) { return f.shifts & 63u; }
+__host__ __device__ inline uint32_t fast_shift_b(const FastDim &f) { return (f.shifts >> 6) & 63u; }
+__host__ __device__ inline uint32_t fast_shift_g(const FastDim &f) { return (f.shifts >> 12) & 63u; }
+__host__ __device__ inline uint32_t fast_shift_bi(const FastDim &f) { return (f.shifts >> 18) & 63u; }
+__host__ __device__ inline uint32_t fast_shift_rr(const FastDim &f) { return (f.shifts >> 24) & 63u; }
+
+// Block counts of one kernel launch: blocks are dealt out in groups holding a fixed number of blocks of each kind.
+struct FastHeader {
+    int32_t rank;                     // dimensions (the innermost one in 16-byte units)
+    int32_t num_workers;
+    int32_t pshape[kMaxBoxDims];
+    int32_t dim_base[kMaxBoxDims];    // index of (dimension k, coordinate 0) in the record table
+    int32_t wstride[kMaxBoxDims];     // worker-id stride of a step along dimension k
+    int32_t num_records;
+    int32_t num_lines;                // workers / pshape[rank - 1]
+    // kind 0: ghost rows (H: filled; H*: the ones outside the tensor cleared), per worker
+    // kind 1: row ends of bulk rows, per line of workers along the innermost dimension (H: all bulk rows; H*: the bulk
+    //         rows out of reach in every outer dimension)
+    // kind 2 (H* only): bulk rows within a neighbour's reach in some outer dimension, per worker
+    int32_t rows_per_tile[3];
+    int32_t tiles_per_owner[3];       // per worker (kinds 0, 2) or per line (kind 1)
+    int32_t group[3];                 // blocks of each kind per group
+    int32_t num_groups;
+};
+
+struct FastPlanHost {
+    bool usable = false;              // H runs through the row plan
+    bool adj_usable = false;          // H* too (needs bulks at least as wide as the two neighbours' reach together)
+    FastHeader hdr;                   // H
+    FastHeader adj_hdr;               // H*
+    std::vector<FastDim> dims;
+};
+
 }  // namespace distdl
 
 // The opaque partition object of the C ABI.
@@ -117,6 +173,8 @@ struct distdl_partition {
 
     distdl::HaloPlanHost fwd_host, adj_host;
     distdl::HaloPlanDevice fwd_dev, adj_dev;
+    distdl::FastPlanHost fast;      // row plan (see FastDim); fast.usable says whether the geometry allows it
+    distdl::FastDim *fast_dims_dev = nullptr;
     void *device_block = nullptr;   // one allocation holding all device tables
 
     void coords(int32_t worker, int32_t *c) const {
@@ -163,9 +221,12 @@ void split_evenly(int64_t n, int32_t p, std::vector<int64_t> &start, std::vector
 // One device allocation holding the tables of two plans; host-only when there is no CUDA device
 // (*block stays nullptr).  Synchronous copies on the current device.
 distdl_status_t upload_plan_pair(const HaloPlanHost &a, const HaloPlanHost &b, HaloPlanDevice *da, HaloPlanDevice *db,
-                                 void **block, int *device, const char *what);
+                                 void **block, int *device, const char *what, const void *extra = nullptr,
+                                 size_t extra_bytes = 0, void **extra_dev = nullptr);
 // Builds the forward (H) and adjoint (H*) box/tile lists of a partition (host only).
 distdl_status_t build_halo_plans(distdl_partition *p);
+// Fills p->fast (row plan) where the geometry allows it.
+void build_fast_plan(distdl_partition *p);
 // Geometry and halo plans only, no device memory.
 distdl_status_t partition_create_host_only(int32_t rank, const int64_t *global_shape, const int32_t *partition_shape,
                                            const int32_t *halo_lo, const int32_t *halo_hi, distdl_dtype_t dtype,

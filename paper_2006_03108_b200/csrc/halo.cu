@@ -281,6 +281,586 @@ halo_box_kernel(const HaloBox *__restrict__ boxes, const HaloSource *__restrict_
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Row plan kernels (see FastDim): H and H* for partitions whose innermost dimension is made of
+// whole 16-byte units.  Kinds of block, dealt out interleaved:
+//
+//  * ghost-row blocks: a range of one worker's *ghost rows* -- rows of the padded array whose index
+//    is a ghost index in some outer dimension.  Such a row is ghost from end to end, and consecutive
+//    ghost rows are contiguous in memory, so the block writes whole runs of memory; each row is
+//    fetched as (low ghost columns | bulk columns | high ghost columns) from up to three neighbours.
+//    H* only clears the ghost rows (or parts of rows) that lie outside the tensor here; the others are
+//    cleared by the thread that adds them to their bulk cell.
+//  * line blocks: a range of bulk rows of all the workers that sit next to each other along the
+//    innermost dimension.  There the ghosts are a few units at both ends of every row.  The ghost
+//    units at the end of row r and at the start of row r + 1 are adjacent in memory, and so are the
+//    bulk units that the two neighbours want from (H) or add to (H*) those rows; loads are issued in
+//    the order of the source rows and stores in the order of the destination rows, with shared
+//    memory in between, so that a warp touches each 128-byte line once per direction.
+//  * receiving-row blocks (H* only): bulk rows that a neighbour in some outer dimension holds ghost
+//    copies of.  Every unit of such a row is the nested sum of two, four or eight terms.
+// ---------------------------------------------------------------------------------------------
+constexpr int kFastThreads = 256;
+constexpr int kFastMaxRows = 256;      // row records per block
+constexpr int kFastMaxSlots = 1024;    // staged units per line block (16 KB)
+
+struct FastRowRec {
+    uint32_t dst_off;      // unit offset of the row inside the worker's array
+    int32_t shard[3];      // source worker of the low ghost / bulk / high ghost columns, -1: zeros
+    uint32_t off[3];       // unit offset of the source row plus the column shift
+};
+
+__device__ __forceinline__ uint32_t fast_div(uint32_t x, uint32_t magic, uint32_t shift) {
+    return magic ? (__umulhi(x, magic) >> shift) : x;
+}
+
+// Which kind of block this is, and its index among the blocks of that kind.
+__device__ __forceinline__ int fast_block_kind(const FastHeader &H, uint32_t *tile_id) {
+    const uint32_t per_group = (uint32_t)(H.group[0] + H.group[1] + H.group[2]);
+    const uint32_t group = blockIdx.x / per_group;
+    uint32_t in_group = blockIdx.x - group * per_group;
+    int kind = 0;
+    if (in_group >= (uint32_t)H.group[0]) {
+        in_group -= (uint32_t)H.group[0];
+        kind = 1;
+        if (in_group >= (uint32_t)H.group[1]) {
+            in_group -= (uint32_t)H.group[1];
+            kind = 2;
+        }
+    }
+    *tile_id = group * (uint32_t)H.group[kind] + in_group;
+    return kind;
+}
+
+__device__ __forceinline__ void fast_load_records(const FastHeader &H, const FastDim *dims_g, FastDim *dims) {
+    for (int i = threadIdx.x; i < H.num_records * (int)(sizeof(FastDim) / 4); i += kFastThreads)
+        reinterpret_cast<uint32_t *>(dims)[i] = __ldg(reinterpret_cast<const uint32_t *>(dims_g) + i);
+    __syncthreads();
+}
+
+// Coordinates of worker w and its record in every dimension.
+__device__ __forceinline__ void fast_worker(const FastHeader &H, const FastDim *dims, uint32_t w, int *c, const FastDim **e) {
+#pragma unroll
+    for (int k = 0; k < kMaxBoxDims; ++k) {
+        c[k] = 0;
+        e[k] = dims;
+        if (k < H.rank) {
+            c[k] = (int)(w / (uint32_t)H.wstride[k]);
+            w -= (uint32_t)c[k] * (uint32_t)H.wstride[k];
+            e[k] = dims + H.dim_base[k] + c[k];
+        }
+    }
+}
+
+// Ghost-row block of worker s: rows [row0, ...) of its ghost rows.  CLEAR_ONLY: only the units without a
+// source (outside the tensor) are written, with zeros.
+template <bool CLEAR_ONLY>
+__device__ __forceinline__ void fast_ghost_rows(const FastHeader &H, const FastDim *dims, const ShardPointers &sh,
+                                                unsigned char *scratch, uint32_t s, uint32_t t) {
+    const int d = H.rank;
+    int c[kMaxBoxDims];
+    const FastDim *e[kMaxBoxDims];
+    fast_worker(H, dims, s, c, e);
+    if (CLEAR_ONLY) {
+        bool complete = true;       // a worker with neighbours on every side has no ghost outside the tensor
+#pragma unroll
+        for (int k = 0; k < kMaxBoxDims; ++k)
+            if (k < d && ((e[k]->hlo > 0 && e[k]->lo_c < 0) || (e[k]->n - e[k]->hlo - e[k]->b > 0 && e[k]->hi_c < 0))) complete = false;
+        if (complete) return;
+    }
+    // class j holds the rows whose index is a bulk index in the dimensions before j, a ghost index in dimension j
+    // and anything after it
+    uint32_t cls_rows[kMaxBoxDims];
+    uint32_t total_rows = 0;
+#pragma unroll
+    for (int j = 0; j < kMaxBoxDims - 1; ++j) {
+        cls_rows[j] = 0;
+        if (j < d - 1) {
+            uint32_t r = (uint32_t)(e[j]->n - e[j]->b);
+#pragma unroll
+            for (int k = 0; k < kMaxBoxDims - 1; ++k)
+                if (k < d - 1 && k != j) r *= (uint32_t)(k < j ? e[k]->b : e[k]->n);
+            cls_rows[j] = r;
+            total_rows += r;
+        }
+    }
+    const uint32_t row0 = t * (uint32_t)H.rows_per_tile[0];
+    if (row0 >= total_rows) return;
+    const uint32_t nrows = min((uint32_t)H.rows_per_tile[0], total_rows - row0);
+    const FastDim *ex = e[d - 1];
+    const uint32_t nx = (uint32_t)ex->n;
+    FastRowRec *recs = reinterpret_cast<FastRowRec *>(scratch);
+    static_assert(sizeof(FastRowRec) * kFastMaxRows <= kFastMaxSlots * 16, "row records fit the scratch array");
+    for (uint32_t rl = threadIdx.x; rl < nrows; rl += kFastThreads) {
+        uint32_t idx = row0 + rl;
+        int j = 0;
+#pragma unroll
+        for (int q = 0; q < kMaxBoxDims - 2; ++q)
+            if (j == q && q < d - 2 && idx >= cls_rows[q]) {
+                idx -= cls_rows[q];
+                ++j;
+            }
+        // coordinates of the row inside its class, innermost outer dimension first
+        uint32_t dst_lin = 0, src_lin = 0, dst_pitch = 1, src_pitch = 1;
+        int outer_w = 0;
+        bool zero = false;
+#pragma unroll
+        for (int k = kMaxBoxDims - 2; k >= 0; --k) {
+            if (k < d - 1) {
+                const FastDim &f = *e[k];
+                uint32_t coord;
+                if (k == 0) {
+                    coord = idx;
+                } else {
+                    const uint32_t ext = k > j ? (uint32_t)f.n : (k == j ? (uint32_t)(f.n - f.b) : (uint32_t)f.b);
+                    const uint32_t mg = k > j ? f.magic_n : (k == j ? f.magic_g : f.magic_b);
+                    const uint32_t sf = k > j ? fast_shift_n(f) : (k == j ? fast_shift_g(f) : fast_shift_b(f));
+                    const uint32_t q = fast_div(idx, mg, sf);
+                    coord = idx - q * ext;
+                    idx = q;
+                }
+                const int i = k > j ? (int)coord : (k == j ? ((int)coord < f.hlo ? (int)coord : (int)coord + f.b) : f.hlo + (int)coord);
+                int nc = c[k], si = i;
+                if (i < f.hlo) {
+                    nc = f.lo_c;
+                    si = i + f.lo_shift;
+                } else if (i >= f.hlo + f.b) {
+                    nc = f.hi_c;
+                    si = i + f.hi_shift;
+                }
+                dst_lin += (uint32_t)i * dst_pitch;
+                dst_pitch *= (uint32_t)f.n;
+                if (nc < 0) {
+                    zero = true;
+                } else {
+                    src_lin += (uint32_t)si * src_pitch;
+                    src_pitch *= (uint32_t)dims[H.dim_base[k] + nc].n;
+                    outer_w += nc * H.wstride[k];
+                }
+            }
+        }
+        FastRowRec r;
+        r.dst_off = dst_lin * nx;
+#pragma unroll
+        for (int reg = 0; reg < 3; ++reg) {
+            const int ncx = reg == 0 ? ex->lo_c : (reg == 1 ? c[d - 1] : ex->hi_c);
+            const int shift = reg == 0 ? ex->lo_shift : (reg == 1 ? 0 : ex->hi_shift);
+            r.shard[reg] = -1;
+            r.off[reg] = 0;
+            if (!zero && ncx >= 0) {
+                r.shard[reg] = outer_w + ncx * H.wstride[d - 1];
+                r.off[reg] = src_lin * (uint32_t)dims[H.dim_base[d - 1] + ncx].n + (uint32_t)shift;
+            }
+        }
+        recs[rl] = r;
+    }
+    __syncthreads();
+    uint4 *dst = reinterpret_cast<uint4 *>(sh.p[s]);
+    const uint32_t count = nrows * nx;
+    const uint32_t xlo = (uint32_t)ex->hlo, xhi = (uint32_t)(ex->hlo + ex->b);
+    const uint32_t shx = fast_shift_n(*ex);
+    constexpr int U = 4;
+    for (uint32_t base = threadIdx.x; base < count; base += kFastThreads * U) {
+        uint4 v[U];
+        uint32_t doff[U];
+        bool wr[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kFastThreads;
+            wr[u] = false;
+            v[u] = make_uint4(0, 0, 0, 0);
+            doff[u] = 0;
+            if (i < count) {
+                const uint32_t rl = fast_div(i, ex->magic_n, shx);
+                const uint32_t col = i - rl * nx;
+                const FastRowRec &r = recs[rl];
+                const int reg = col < xlo ? 0 : (col < xhi ? 1 : 2);
+                const int src = r.shard[reg];
+                doff[u] = r.dst_off + col;
+                if (CLEAR_ONLY) {
+                    wr[u] = src < 0;
+                } else {
+                    wr[u] = true;
+                    if (src >= 0) v[u] = __ldg(reinterpret_cast<const uint4 *>(sh.p[src]) + (r.off[reg] + col));
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (wr[u]) dst[doff[u]] = v[u];
+    }
+}
+
+// Unit offsets of bulk rows [row0, row0 + nrows) of a line of workers (the same in all of them up to the row
+// pitch): `inner` restricts the rows to those out of every outer neighbour's reach.
+__device__ __forceinline__ void fast_line_rows(const FastHeader &H, const FastDim *const *e, bool inner, uint32_t row0,
+                                               uint32_t nrows, uint32_t *rowlin) {
+    const int d = H.rank;
+    for (uint32_t rl = threadIdx.x; rl < nrows; rl += kFastThreads) {
+        uint32_t idx = row0 + rl, lin = 0, pitch = 1;
+#pragma unroll
+        for (int k = kMaxBoxDims - 2; k >= 0; --k) {
+            if (k < d - 1) {
+                const FastDim &f = *e[k];
+                uint32_t coord = idx;
+                if (k > 0) {
+                    const uint32_t ext = inner ? (uint32_t)(f.b - f.rlo - f.rhi) : (uint32_t)f.b;
+                    const uint32_t q = inner ? fast_div(idx, f.magic_bi, fast_shift_bi(f)) : fast_div(idx, f.magic_b, fast_shift_b(f));
+                    coord = idx - q * ext;
+                    idx = q;
+                }
+                lin += ((uint32_t)f.hlo + (inner ? (uint32_t)f.rlo : 0u) + coord) * pitch;
+                pitch *= (uint32_t)f.n;
+            }
+        }
+        rowlin[rl] = lin;
+    }
+}
+
+__global__ void __launch_bounds__(kFastThreads)
+halo_fast_fwd_kernel(const __grid_constant__ FastHeader H, const FastDim *__restrict__ dims_g,
+                     const __grid_constant__ ShardPointers sh) {
+    __shared__ FastDim dims[kMaxFastCoords];
+    __shared__ __align__(16) unsigned char scratch[kFastMaxSlots * 16];
+    fast_load_records(H, dims_g, dims);
+    const int d = H.rank;
+    uint32_t tile_id;
+    const int kind = fast_block_kind(H, &tile_id);
+    if (kind == 0) {
+        const uint32_t s = tile_id / (uint32_t)H.tiles_per_owner[0];
+        if (s < (uint32_t)H.num_workers) fast_ghost_rows<false>(H, dims, sh, scratch, s, tile_id - s * (uint32_t)H.tiles_per_owner[0]);
+        return;
+    }
+    // ---------------------------------------------------------------------- line block
+    const uint32_t line = tile_id / (uint32_t)H.tiles_per_owner[1];
+    if (line >= (uint32_t)H.num_lines) return;
+    const uint32_t t = tile_id - line * (uint32_t)H.tiles_per_owner[1];
+    const int px = H.pshape[d - 1];
+    const uint32_t first_worker = line * (uint32_t)px;        // the innermost dimension has worker stride 1
+    int c[kMaxBoxDims];
+    const FastDim *e[kMaxBoxDims];
+    fast_worker(H, dims, first_worker, c, e);
+    uint32_t total_rows = 1;
+#pragma unroll
+    for (int k = 0; k < kMaxBoxDims - 1; ++k)
+        if (k < d - 1) total_rows *= (uint32_t)e[k]->b;
+    const uint32_t row0 = t * (uint32_t)H.rows_per_tile[1];
+    if (row0 >= total_rows) return;
+    const uint32_t nrows = min((uint32_t)H.rows_per_tile[1], total_rows - row0);
+    // per worker of the line: cumulative counts of ghost units (stores) and of wanted bulk units (loads)
+    __shared__ uint32_t cum_g[kMaxFastCoords + 1], cum_p[kMaxFastCoords + 1];
+    __shared__ uint32_t rowlin[128];
+    const FastDim *xd = dims + H.dim_base[d - 1];
+    if (threadIdx.x == 0) {
+        uint32_t g = 0, pc = 0;
+        for (int a = 0; a < px; ++a) {
+            cum_g[a] = g;
+            cum_p[a] = pc;
+            g += (uint32_t)(xd[a].n - xd[a].b);
+            pc += (uint32_t)(xd[a].rlo + xd[a].rhi);      // what the two neighbours' ghosts hold of this worker's rows
+        }
+        cum_g[px] = g;
+        cum_p[px] = pc;
+    }
+    fast_line_rows(H, e, false, row0, nrows, rowlin);
+    __syncthreads();
+    uint4 *slots = reinterpret_cast<uint4 *>(scratch);
+    const uint32_t GC = cum_g[px], PC = cum_p[px];
+    // loads, in the order (worker, row, wanted unit): the last units of row r and the first units of
+    // row r + 1 are neighbours in memory and in this order
+    for (uint32_t q = threadIdx.x; q < nrows * PC; q += kFastThreads) {
+        int a = 0;
+        while (q >= nrows * cum_p[a + 1]) ++a;
+        const uint32_t qa = q - nrows * cum_p[a];
+        const FastDim &f = xd[a];
+        const uint32_t pc = (uint32_t)(f.rlo + f.rhi);
+        const uint32_t rl = qa / pc, piece = qa - rl * pc;
+        uint32_t col, slot;
+        if (piece < (uint32_t)f.rlo) {      // first bulk units -> high ghost of the low neighbour
+            const FastDim &g = xd[f.lo_c];
+            col = (uint32_t)f.hlo + piece;
+            slot = nrows * cum_g[f.lo_c] + rl * (uint32_t)(g.n - g.b) + (uint32_t)g.hlo + piece;
+        } else {                            // last bulk units -> low ghost of the high neighbour
+            const FastDim &g = xd[f.hi_c];
+            const uint32_t u = piece - (uint32_t)f.rlo;
+            col = (uint32_t)(f.hlo + f.b - f.rhi) + u;
+            slot = nrows * cum_g[f.hi_c] + rl * (uint32_t)(g.n - g.b) + u;
+        }
+        slots[slot] = __ldg(reinterpret_cast<const uint4 *>(sh.p[first_worker + a]) + (rowlin[rl] * (uint32_t)f.n + col));
+    }
+    __syncthreads();
+    // stores, in the order (worker, row, ghost unit): the high ghost of row r is followed by the low ghost of row r + 1
+    for (uint32_t q = threadIdx.x; q < nrows * GC; q += kFastThreads) {
+        int a = 0;
+        while (q >= nrows * cum_g[a + 1]) ++a;
+        const uint32_t qa = q - nrows * cum_g[a];
+        const FastDim &f = xd[a];
+        const uint32_t gc = (uint32_t)(f.n - f.b);
+        const uint32_t rl = qa / gc, g = qa - rl * gc;
+        const bool low = g < (uint32_t)f.hlo;
+        const bool has = low ? f.lo_c >= 0 : f.hi_c >= 0;
+        const uint32_t col = low ? g : g + (uint32_t)f.b;
+        uint4 *dst = reinterpret_cast<uint4 *>(sh.p[first_worker + a]) + (rowlin[rl] * (uint32_t)f.n + col);
+        *dst = has ? slots[nrows * cum_g[a] + qa] : make_uint4(0, 0, 0, 0);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// H* through the row plan.  T: 16-byte vector of the element type (float4, double2, bf16x8).
+// ---------------------------------------------------------------------------------------------
+struct FastSumRec {
+    uint32_t nterms;       // rows added together: 1 << (outer dimensions in which the row is within a neighbour's reach)
+    int32_t shard[4];      // worker of every row, without the coordinate along the innermost dimension; [0] is the row itself
+    uint32_t lin[4];       // linear index of the row in that worker's array (multiply by its row pitch)
+};
+
+template <typename T, int N>
+__device__ __forceinline__ void fast_sum_unit(T *const *ptr) {
+    T v[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) v[j] = *ptr[j];
+    // fixed tree: neighbouring terms first (innermost dimension), own value before the neighbour's at every level
+#pragma unroll
+    for (int width = 1; width < N; width *= 2)
+#pragma unroll
+        for (int j = 0; j < N; j += 2 * width) v[j] = vadd(v[j], v[j + width]);
+    stores_after(v[0]);
+    *ptr[0] = v[0];
+#pragma unroll
+    for (int j = 1; j < N; ++j) *ptr[j] = zero_of<T>();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kFastThreads)
+halo_fast_adj_kernel(const __grid_constant__ FastHeader H, const FastDim *__restrict__ dims_g,
+                     const __grid_constant__ ShardPointers sh) {
+    __shared__ FastDim dims[kMaxFastCoords];
+    __shared__ __align__(16) unsigned char scratch[kFastMaxSlots * 16];
+    fast_load_records(H, dims_g, dims);
+    const int d = H.rank;
+    uint32_t tile_id;
+    const int kind = fast_block_kind(H, &tile_id);
+    if (kind == 0) {
+        // ghost rows outside the tensor: cleared; the others are cleared by whoever adds them to a bulk cell
+        const uint32_t s = tile_id / (uint32_t)H.tiles_per_owner[0];
+        if (s < (uint32_t)H.num_workers) fast_ghost_rows<true>(H, dims, sh, scratch, s, tile_id - s * (uint32_t)H.tiles_per_owner[0]);
+        return;
+    }
+    if (kind == 2) {
+        // ------------------------------------------------------------------ receiving rows
+        const uint32_t s = tile_id / (uint32_t)H.tiles_per_owner[2];
+        if (s >= (uint32_t)H.num_workers) return;
+        const uint32_t t = tile_id - s * (uint32_t)H.tiles_per_owner[2];
+        int c[kMaxBoxDims];
+        const FastDim *e[kMaxBoxDims];
+        fast_worker(H, dims, s, c, e);
+        // class j: out of reach in the dimensions before j, within reach in dimension j, any bulk index after it
+        uint32_t cls_rows[kMaxBoxDims];
+        uint32_t total_rows = 0;
+#pragma unroll
+        for (int j = 0; j < kMaxBoxDims - 1; ++j) {
+            cls_rows[j] = 0;
+            if (j < d - 1) {
+                uint32_t r = (uint32_t)(e[j]->rlo + e[j]->rhi);
+#pragma unroll
+                for (int k = 0; k < kMaxBoxDims - 1; ++k)
+                    if (k < d - 1 && k != j) r *= (uint32_t)(k < j ? e[k]->b - e[k]->rlo - e[k]->rhi : e[k]->b);
+                cls_rows[j] = r;
+                total_rows += r;
+            }
+        }
+        const uint32_t row0 = t * (uint32_t)H.rows_per_tile[2];
+        if (row0 >= total_rows) return;
+        const uint32_t nrows = min((uint32_t)H.rows_per_tile[2], total_rows - row0);
+        FastSumRec *recs = reinterpret_cast<FastSumRec *>(scratch);
+        static_assert(sizeof(FastSumRec) * kFastMaxRows <= kFastMaxSlots * 16, "row records fit the scratch array");
+        for (uint32_t rl = threadIdx.x; rl < nrows; rl += kFastThreads) {
+            uint32_t idx = row0 + rl;
+            int j = 0;
+#pragma unroll
+            for (int q = 0; q < kMaxBoxDims - 2; ++q)
+                if (j == q && q < d - 2 && idx >= cls_rows[q]) {
+                    idx -= cls_rows[q];
+                    ++j;
+                }
+            FastSumRec r;
+            r.nterms = 1;
+            r.shard[0] = 0;
+            r.lin[0] = 0;
+            uint32_t pitch[4] = {1, 1, 1, 1};
+            // innermost outer dimension first: a dimension within reach doubles the rows, the new ones (the
+            // neighbour's ghost rows) after the old ones, so the outermost dimension ends up as the slowest index
+            // of the list, as the nested sum wants it
+#pragma unroll
+            for (int k = kMaxBoxDims - 2; k >= 0; --k) {
+                if (k < d - 1) {
+                    const FastDim &f = *e[k];
+                    const uint32_t inner = (uint32_t)(f.b - f.rlo - f.rhi), rr = (uint32_t)(f.rlo + f.rhi);
+                    uint32_t coord = idx;
+                    if (k > 0) {
+                        const uint32_t ext = k > j ? (uint32_t)f.b : (k == j ? rr : inner);
+                        const uint32_t q = k > j ? fast_div(idx, f.magic_b, fast_shift_b(f))
+                                                 : (k == j ? fast_div(idx, f.magic_rr, fast_shift_rr(f)) : fast_div(idx, f.magic_bi, fast_shift_bi(f)));
+                        coord = idx - q * ext;
+                        idx = q;
+                    }
+                    // position inside the bulk
+                    const uint32_t pos = k > j ? coord : (k == j ? (coord < (uint32_t)f.rlo ? coord : coord + inner) : (uint32_t)f.rlo + coord);
+                    const int i = f.hlo + (int)pos;
+                    int nc = -1, si = 0;
+                    if (pos < (uint32_t)f.rlo) {
+                        nc = f.lo_c;
+                        si = i + f.lo_shift;
+                    } else if (pos >= (uint32_t)(f.b - f.rhi)) {
+                        nc = f.hi_c;
+                        si = i + f.hi_shift;
+                    }
+                    const uint32_t old = r.nterms;
+                    if (nc >= 0 && old <= 2) {
+                        const uint32_t npitch = (uint32_t)dims[H.dim_base[k] + nc].n;
+#pragma unroll
+                        for (uint32_t q = 0; q < 2; ++q)
+                            if (q < old) {
+                                r.shard[old + q] = r.shard[q] + nc * H.wstride[k];
+                                r.lin[old + q] = r.lin[q] + (uint32_t)si * pitch[q];
+                                pitch[old + q] = pitch[q] * npitch;
+                            }
+                        r.nterms = 2 * old;
+                    }
+#pragma unroll
+                    for (uint32_t q = 0; q < 2; ++q)
+                        if (q < old) {
+                            r.shard[q] += c[k] * H.wstride[k];
+                            r.lin[q] += (uint32_t)i * pitch[q];
+                            pitch[q] *= (uint32_t)f.n;
+                        }
+                }
+            }
+            recs[rl] = r;
+        }
+        __syncthreads();
+        const FastDim *ex = e[d - 1];
+        const uint32_t nx = (uint32_t)ex->n;
+        const uint32_t count = nrows * nx;
+        const uint32_t shx = fast_shift_n(*ex);
+        const int cx = c[d - 1];
+        for (uint32_t i = threadIdx.x; i < count; i += kFastThreads) {
+            const uint32_t rl = fast_div(i, ex->magic_n, shx);
+            const uint32_t col = i - rl * nx;
+            const FastSumRec &r = recs[rl];
+            if (col < (uint32_t)ex->hlo || col >= (uint32_t)(ex->hlo + ex->b)) {
+                // a ghost unit at the end of a bulk row: its neighbour along the row clears it, unless there is none
+                const bool none = col < (uint32_t)ex->hlo ? ex->lo_c < 0 : ex->hi_c < 0;
+                if (none) reinterpret_cast<T *>(sh.p[s])[r.lin[0] * nx + col] = zero_of<T>();
+                continue;
+            }
+            const uint32_t pos = col - (uint32_t)ex->hlo;
+            int ncx = -1, shift = 0;
+            if (pos < (uint32_t)ex->rlo) {
+                ncx = ex->lo_c;
+                shift = ex->lo_shift;
+            } else if (pos >= (uint32_t)(ex->b - ex->rhi)) {
+                ncx = ex->hi_c;
+                shift = ex->hi_shift;
+            }
+            T *ptr[8];
+            const uint32_t nt = r.nterms;
+            const uint32_t nnx = ncx >= 0 ? (uint32_t)dims[H.dim_base[d - 1] + ncx].n : 0u;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if ((uint32_t)q < nt) {
+                    T *own = reinterpret_cast<T *>(sh.p[r.shard[q] + cx]) + (r.lin[q] * nx + col);
+                    if (ncx >= 0) {
+                        ptr[2 * q] = own;
+                        ptr[2 * q + 1] = reinterpret_cast<T *>(sh.p[r.shard[q] + ncx]) + (r.lin[q] * nnx + (uint32_t)((int)col + shift));
+                    } else {
+                        ptr[q] = own;
+                    }
+                }
+            }
+            const uint32_t terms = ncx >= 0 ? 2 * nt : nt;
+            if (terms == 2) fast_sum_unit<T, 2>(ptr);
+            else if (terms == 4) fast_sum_unit<T, 4>(ptr);
+            else if (terms == 8) fast_sum_unit<T, 8>(ptr);
+        }
+        return;
+    }
+    // ---------------------------------------------------------------------- line block: both ends of the bulk rows that
+    // are out of reach in every outer dimension, for all workers of the line
+    const uint32_t line = tile_id / (uint32_t)H.tiles_per_owner[1];
+    if (line >= (uint32_t)H.num_lines) return;
+    const uint32_t t = tile_id - line * (uint32_t)H.tiles_per_owner[1];
+    const int px = H.pshape[d - 1];
+    const uint32_t first_worker = line * (uint32_t)px;
+    int c[kMaxBoxDims];
+    const FastDim *e[kMaxBoxDims];
+    fast_worker(H, dims, first_worker, c, e);
+    uint32_t total_rows = 1;
+#pragma unroll
+    for (int k = 0; k < kMaxBoxDims - 1; ++k)
+        if (k < d - 1) total_rows *= (uint32_t)(e[k]->b - e[k]->rlo - e[k]->rhi);
+    const uint32_t row0 = t * (uint32_t)H.rows_per_tile[1];
+    if (row0 >= total_rows) return;
+    const uint32_t nrows = min((uint32_t)H.rows_per_tile[1], total_rows - row0);
+    __shared__ uint32_t cum_e[kMaxFastCoords + 1];
+    __shared__ uint32_t rowlin[128];
+    const FastDim *xd = dims + H.dim_base[d - 1];
+    if (threadIdx.x == 0) {
+        uint32_t n = 0;
+        for (int a = 0; a < px; ++a) {
+            cum_e[a] = n;
+            n += (uint32_t)(xd[a].n - xd[a].b + xd[a].rlo + xd[a].rhi);     // low ghost, low receiving, high receiving, high ghost
+        }
+        cum_e[px] = n;
+    }
+    fast_line_rows(H, e, true, row0, nrows, rowlin);
+    __syncthreads();
+    T *slots = reinterpret_cast<T *>(scratch);
+    const uint32_t EC = cum_e[px];
+    // pass 1: every unit of the row ends into shared memory, in memory order per worker
+    for (uint32_t q = threadIdx.x; q < nrows * EC; q += kFastThreads) {
+        int a = 0;
+        while (q >= nrows * cum_e[a + 1]) ++a;
+        const uint32_t qa = q - nrows * cum_e[a];
+        const FastDim &f = xd[a];
+        const uint32_t ec = (uint32_t)(f.n - f.b + f.rlo + f.rhi), lo_end = (uint32_t)(f.hlo + f.rlo);
+        const uint32_t rl = qa / ec, u = qa - rl * ec;
+        const uint32_t col = u < lo_end ? u : u - lo_end + (uint32_t)(f.hlo + f.b - f.rhi);
+        const bool ghost = col < (uint32_t)f.hlo || col >= (uint32_t)(f.hlo + f.b);
+        const bool outside = ghost && (col < (uint32_t)f.hlo ? f.lo_c < 0 : f.hi_c < 0);      // never read: only cleared
+        if (!outside) slots[q] = reinterpret_cast<const T *>(sh.p[first_worker + a])[rowlin[rl] * (uint32_t)f.n + col];
+    }
+    __syncthreads();
+    // pass 2: ghosts <- 0, receiving units <- own value + the neighbour's ghost copy, same order
+    for (uint32_t q = threadIdx.x; q < nrows * EC; q += kFastThreads) {
+        int a = 0;
+        while (q >= nrows * cum_e[a + 1]) ++a;
+        const uint32_t qa = q - nrows * cum_e[a];
+        const FastDim &f = xd[a];
+        const uint32_t ec = (uint32_t)(f.n - f.b + f.rlo + f.rhi), lo_end = (uint32_t)(f.hlo + f.rlo);
+        const uint32_t rl = qa / ec, u = qa - rl * ec;
+        const uint32_t col = u < lo_end ? u : u - lo_end + (uint32_t)(f.hlo + f.b - f.rhi);
+        T v = zero_of<T>();
+        if (col >= (uint32_t)f.hlo && col < (uint32_t)(f.hlo + f.b)) {
+            v = slots[q];
+            if (u < lo_end) {
+                if (f.lo_c >= 0) {      // the low neighbour's high ghost unit of the same cell: the last units of its row ends
+                    const FastDim &g = xd[f.lo_c];
+                    const uint32_t gec = (uint32_t)(g.n - g.b + g.rlo + g.rhi);
+                    const uint32_t gu = (uint32_t)(g.hlo + g.rlo + g.rhi) + (u - (uint32_t)f.hlo);
+                    v = vadd(v, slots[nrows * cum_e[f.lo_c] + rl * gec + gu]);
+                }
+            } else if (f.hi_c >= 0) {   // the high neighbour's low ghost unit: the first units of its row
+                const FastDim &g = xd[f.hi_c];
+                const uint32_t gec = (uint32_t)(g.n - g.b + g.rlo + g.rhi);
+                v = vadd(v, slots[nrows * cum_e[f.hi_c] + rl * gec + (u - lo_end)]);
+            }
+        }
+        reinterpret_cast<T *>(sh.p[first_worker + a])[rowlin[rl] * (uint32_t)f.n + col] = v;
+    }
+}
+
 static distdl_status_t launch(const distdl_partition *p, const HaloPlanDevice &plan, void *const *shards,
                               void *stream, bool adjoint, const char *what) {
     clear_error();
@@ -304,6 +884,23 @@ static distdl_status_t launch(const distdl_partition *p, const HaloPlanDevice &p
     }
     for (int32_t w = p->num_workers; w < DISTDL_MAX_WORKERS; ++w) sh.p[w] = nullptr;
     if (plan.num_tiles == 0) return DISTDL_OK;
+    if (!adjoint && p->fast.usable && p->fast_dims_dev) {
+        const FastHeader &h = p->fast.hdr;
+        halo_fast_fwd_kernel<<<(unsigned)h.num_groups * (unsigned)(h.group[0] + h.group[1] + h.group[2]), kFastThreads, 0,
+                               (cudaStream_t)stream>>>(h, p->fast_dims_dev, sh);
+        DISTDL_CUDA_CHECK(cudaGetLastError());
+        return DISTDL_OK;
+    }
+    if (adjoint && p->fast.adj_usable && p->fast_dims_dev) {
+        const FastHeader &h = p->fast.adj_hdr;
+        const unsigned grid = (unsigned)h.num_groups * (unsigned)(h.group[0] + h.group[1] + h.group[2]);
+        cudaStream_t st = (cudaStream_t)stream;
+        if (p->dtype == DISTDL_F32) halo_fast_adj_kernel<float4><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
+        else if (p->dtype == DISTDL_F64) halo_fast_adj_kernel<double2><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
+        else halo_fast_adj_kernel<bf16x8><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
+        DISTDL_CUDA_CHECK(cudaGetLastError());
+        return DISTDL_OK;
+    }
     if (adjoint)
         halo_box_kernel<true><<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(
             plan.boxes, plan.sources, plan.tiles, elem_size(p->dtype), sh);
@@ -343,6 +940,15 @@ static distdl_status_t halo_fwd_noalloc_impl(int32_t rank, const int64_t *global
     const char *what = "halo_fwd_noalloc";
     clear_error();
     if (!shards) return fail(DISTDL_ERR_INVALID_ARG, "%s: shards is NULL", what);
+    // The plan tables below are copied from host memory that is freed when this call returns: a captured
+    // copy would read it again at every replay.  So the call refuses a stream that is being captured.
+    {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        DISTDL_CUDA_CHECK(cudaStreamIsCapturing((cudaStream_t)stream, &cap));
+        if (cap != cudaStreamCaptureStatusNone)
+            return fail(DISTDL_ERR_UNSUPPORTED, "%s: the stream is being captured; this call copies its plan tables from "
+                        "temporary host memory and cannot be recorded in a graph (use distdl_partition_create + distdl_halo_fwd)", what);
+    }
     distdl_partition *p = nullptr;
     distdl_status_t st = partition_create_host_only(rank, global_shape, partition_shape, halo_lo, halo_hi, dtype, &p);
     if (st != DISTDL_OK) return st;

@@ -7,7 +7,8 @@
 using namespace distdl;
 
 distdl_status_t distdl::upload_plan_pair(const HaloPlanHost &a, const HaloPlanHost &b, HaloPlanDevice *da, HaloPlanDevice *db,
-                                 void **block, int *device, const char *what) {
+                                 void **block, int *device, const char *what, const void *extra, size_t extra_bytes,
+                                 void **extra_dev) {
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) {
         cudaGetLastError();
@@ -23,7 +24,8 @@ distdl_status_t distdl::upload_plan_pair(const HaloPlanHost &a, const HaloPlanHo
     size_t fbz, fsz, ftz, abz, asz, atz;
     bytes_of(a, &fbz, &fsz, &ftz);
     bytes_of(b, &abz, &asz, &atz);
-    const size_t total = fbz + fsz + ftz + abz + asz + atz + 256;
+    const size_t ebz = (extra_bytes + 255) & ~(size_t)255;
+    const size_t total = fbz + fsz + ftz + abz + asz + atz + ebz + 256;
     cudaError_t e = cudaMalloc(block, total);
     if (e != cudaSuccess) {
         *block = nullptr;
@@ -44,6 +46,7 @@ distdl_status_t distdl::upload_plan_pair(const HaloPlanHost &a, const HaloPlanHo
     db->sources = (HaloSource *)put(b.sources.data(), b.sources.size() * sizeof(HaloSource), asz);
     db->tiles = (HaloTile *)put(b.tiles.data(), b.tiles.size() * sizeof(HaloTile), atz);
     db->num_tiles = (int32_t)b.tiles.size();
+    if (extra_dev) *extra_dev = extra_bytes ? put(extra, extra_bytes, ebz) : nullptr;
     if (e != cudaSuccess) {
         cudaFree(*block);
         *block = nullptr;
@@ -124,11 +127,15 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
         delete p;
         return st;
     }
+    build_fast_plan(p);
     // Upload.  Without a CUDA device the object stays host-only: geometry queries work, operator
     // calls report DISTDL_ERR_CUDA.
     if (upload) {
+        void *fast_dev = nullptr;
         st = upload_plan_pair(p->fwd_host, p->adj_host, &p->fwd_dev, &p->adj_dev, &p->device_block, &p->device,
-                              "partition_create");
+                              "partition_create", p->fast.usable ? p->fast.dims.data() : nullptr,
+                              p->fast.usable ? p->fast.dims.size() * sizeof(FastDim) : 0, &fast_dev);
+        p->fast_dims_dev = static_cast<FastDim *>(fast_dev);
         if (st != DISTDL_OK) {
             delete p;
             return st;
@@ -209,6 +216,28 @@ extern "C" distdl_status_t distdl_partition_halo_stats(const distdl_partition_t 
     if (tiles) *tiles = (int64_t)h.tiles.size();
     if (bytes) *bytes = h.algorithmic_bytes;
     return DISTDL_OK;
+}
+
+// Copies the row plan (header and per-coordinate records, as 32-bit words) to the caller: lets a host-side
+// test replay the kernels' index arithmetic.
+extern "C" distdl_status_t distdl_selftest_row_plan(const distdl_partition_t *p, int32_t adjoint, int32_t *header,
+                                                    int32_t header_words, int32_t *records, int32_t record_words,
+                                                    int32_t *num_records) {
+    clear_error();
+    if (!p || !header || !records || !num_records) return fail(DISTDL_ERR_INVALID_ARG, "selftest_row_plan: NULL argument");
+    if (adjoint ? !p->fast.adj_usable : !p->fast.usable)
+        return fail(DISTDL_ERR_UNSUPPORTED, "selftest_row_plan: this partition has no row plan for %s", adjoint ? "H*" : "H");
+    const size_t hw = sizeof(FastHeader) / 4, rw = p->fast.dims.size() * (sizeof(FastDim) / 4);
+    if ((size_t)header_words < hw || (size_t)record_words < rw)
+        return fail(DISTDL_ERR_INVALID_ARG, "selftest_row_plan: need %zu header words and %zu record words", hw, rw);
+    memcpy(header, adjoint ? &p->fast.adj_hdr : &p->fast.hdr, hw * 4);
+    memcpy(records, p->fast.dims.data(), rw * 4);
+    *num_records = (int32_t)p->fast.dims.size();
+    return DISTDL_OK;
+}
+
+extern "C" int32_t distdl_partition_uses_row_plan(const distdl_partition_t *p, int32_t adjoint) {
+    return p ? ((adjoint ? p->fast.adj_usable : p->fast.usable) ? 1 : 0) : -1;
 }
 
 // ---------------------------------------------------------------------------------------------

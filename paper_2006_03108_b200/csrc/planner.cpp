@@ -510,6 +510,165 @@ distdl_status_t build_repartition_plans(distdl_repartition *r) {
     return DISTDL_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Row plan: one record per (dimension, worker coordinate), see FastDim.
+// ---------------------------------------------------------------------------------------------
+static void magic_of(int64_t e, uint32_t *magic, uint32_t *shift) {
+    // exact division of any x < 2^31 by e >= 2: x / e == umulhi(x, magic) >> shift with s = ceil(log2 e),
+    // magic = ceil(2^(31+s) / e) < 2^32, shift = s - 1; e <= 1: magic 0 (the quotient is x itself)
+    *magic = 0;
+    *shift = 0;
+    if (e < 2) return;
+    int sft = 0;
+    while (((int64_t)1 << sft) < e) ++sft;
+    const unsigned __int128 num = (unsigned __int128)1 << (31 + sft);
+    *magic = (uint32_t)((num + (uint64_t)e - 1) / (uint64_t)e);
+    *shift = (uint32_t)(sft - 1);
+}
+
+// Deals `total[i]` blocks of kind i out in groups: the rarest kind present gets one block per group.
+static bool fast_groups(const int64_t total[3], FastHeader *h) {
+    int64_t least = 0;
+    for (int i = 0; i < 3; ++i)
+        if (total[i] > 0 && (least == 0 || total[i] < least)) least = total[i];
+    if (least == 0) return false;
+    int64_t groups = 0, per_group = 0;
+    for (int i = 0; i < 3; ++i) {
+        h->group[i] = total[i] > 0 ? (int32_t)std::min<int64_t>(64, total[i] / least) : 0;
+        if (h->group[i]) groups = std::max(groups, (total[i] + h->group[i] - 1) / h->group[i]);
+        per_group += h->group[i];
+    }
+    if (groups * per_group >= ((int64_t)1 << 31)) return false;
+    h->num_groups = (int32_t)groups;
+    return true;
+}
+
+void build_fast_plan(distdl_partition *p) {
+    FastPlanHost &f = p->fast;
+    f.usable = f.adj_usable = false;
+    f.dims.clear();
+    memset(&f.hdr, 0, sizeof(f.hdr));
+    memset(&f.adj_hdr, 0, sizeof(f.adj_hdr));
+    const int d = p->rank;
+    const int esize = elem_size(p->dtype);
+    const int64_t per = 16 / esize;
+    int64_t coords = 0;
+    for (int k = 0; k < d; ++k) coords += p->pshape[k];
+    if (coords > kMaxFastCoords) return;
+    // the innermost dimension in whole 16-byte units, for every worker coordinate along it
+    for (int32_t c = 0; c < p->pshape[d - 1]; ++c)
+        if (p->hlo[d - 1][c] % per || p->hhi[d - 1][c] % per || p->size[d - 1][c] % per) return;
+    FastHeader &h = f.hdr;
+    h.rank = d;
+    h.num_workers = p->num_workers;
+    int32_t stride = 1;
+    for (int k = d - 1; k >= 0; --k) {
+        h.wstride[k] = stride;
+        stride *= p->pshape[k];
+    }
+    int64_t any_ghost = 0;
+    bool wide_enough = true;          // every bulk at least as wide as its two neighbours' reach together
+    int dims_with_reach = 0;
+    for (int k = 0; k < d; ++k) {
+        h.pshape[k] = p->pshape[k];
+        h.dim_base[k] = (int32_t)f.dims.size();
+        const int64_t unit = k == d - 1 ? per : 1;
+        const int32_t pk = p->pshape[k];
+        bool reach = false;
+        for (int32_t c = 0; c < pk; ++c) {
+            FastDim e;
+            memset(&e, 0, sizeof(e));
+            e.hlo = (int32_t)(p->hlo[k][c] / unit);
+            e.b = (int32_t)(p->size[k][c] / unit);
+            e.n = (int32_t)(p->padded_extent(k, c) / unit);
+            any_ghost += e.n - e.b;
+            const bool has_lo = c > 0 || p->periodic[k], has_hi = c + 1 < pk || p->periodic[k];
+            e.lo_c = has_lo ? (c + pk - 1) % pk : -1;
+            e.hi_c = has_hi ? (c + 1) % pk : -1;
+            if (has_lo) {
+                e.lo_shift = (int32_t)((p->hlo[k][e.lo_c] + p->size[k][e.lo_c] - p->hlo[k][c]) / unit);
+                e.rlo = (int32_t)(p->hhi[k][e.lo_c] / unit);
+            }
+            if (has_hi) {
+                e.hi_shift = (int32_t)((p->hlo[k][e.hi_c] - p->hlo[k][c] - p->size[k][c]) / unit);
+                e.rhi = (int32_t)(p->hlo[k][e.hi_c] / unit);
+            }
+            if (e.rlo + e.rhi > e.b) wide_enough = false;
+            reach = reach || e.rlo + e.rhi > 0;
+            uint32_t sn, sb, sg, sbi, srr;
+            magic_of(e.n, &e.magic_n, &sn);
+            magic_of(e.b, &e.magic_b, &sb);
+            magic_of(e.n - e.b, &e.magic_g, &sg);
+            magic_of(e.b - e.rlo - e.rhi, &e.magic_bi, &sbi);
+            magic_of(e.rlo + e.rhi, &e.magic_rr, &srr);
+            e.shifts = sn | (sb << 6) | (sg << 12) | (sbi << 18) | (srr << 24);
+            f.dims.push_back(e);
+        }
+        if (reach && k < d - 1) ++dims_with_reach;
+    }
+    h.num_records = (int32_t)f.dims.size();
+    h.num_lines = p->num_workers / p->pshape[d - 1];
+    if (any_ghost == 0) return;     // nothing to exchange: the box plan (empty) handles it
+    // block sizes from the largest worker
+    int64_t nx_max = 1, ghost_rows_max = 0, bulk_rows_max = 0, reach_rows_max = 0, inner_rows_max = 0;
+    int64_t gc = 0, ec = 0;         // per row of a line: ghost units, and units of the row ends that H* rewrites
+    for (int32_t c = 0; c < p->pshape[d - 1]; ++c) {
+        const FastDim &e = f.dims[h.dim_base[d - 1] + c];
+        nx_max = std::max<int64_t>(nx_max, e.n);
+        gc += e.n - e.b;
+        ec += e.n - e.b + e.rlo + e.rhi;
+    }
+    for (int32_t w = 0; w < p->num_workers; ++w) {
+        int32_t c[DISTDL_MAX_RANK];
+        p->coords(w, c);
+        int64_t all = 1, bulk = 1, inner = 1;
+        for (int k = 0; k + 1 < d; ++k) {
+            const FastDim &e = f.dims[h.dim_base[k] + c[k]];
+            all *= e.n;
+            bulk *= e.b;
+            inner *= std::max(0, e.b - e.rlo - e.rhi);
+        }
+        ghost_rows_max = std::max(ghost_rows_max, all - bulk);   // rows with a ghost index in some outer dimension
+        bulk_rows_max = std::max(bulk_rows_max, bulk);
+        reach_rows_max = std::max(reach_rows_max, bulk - inner);
+        inner_rows_max = std::max(inner_rows_max, inner);
+    }
+    if (ghost_rows_max >= ((int64_t)1 << 31) || bulk_rows_max >= ((int64_t)1 << 31)) return;
+    if (gc > 1024) return;          // staging of one row's ghost units for all workers of a line: 16 KB at most
+    const int32_t rows_s = (int32_t)std::min<int64_t>(256, std::max<int64_t>(1, 2048 / nx_max));
+    auto tiles = [](int64_t rows, int32_t per_tile) { return (int32_t)((rows + per_tile - 1) / per_tile); };
+    // ---- H
+    h.rows_per_tile[0] = rows_s;
+    h.tiles_per_owner[0] = tiles(ghost_rows_max, rows_s);
+    if (gc > 0) {
+        h.rows_per_tile[1] = (int32_t)std::min<int64_t>(128, std::max<int64_t>(1, 512 / gc));
+        h.tiles_per_owner[1] = tiles(bulk_rows_max, h.rows_per_tile[1]);
+    }
+    {
+        const int64_t total[3] = {(int64_t)h.tiles_per_owner[0] * p->num_workers, (int64_t)h.tiles_per_owner[1] * h.num_lines, 0};
+        f.usable = fast_groups(total, &h);
+    }
+    // ---- H*: at most two outer dimensions with neighbours (four rows summed into one, eight terms with the row ends)
+    if (!f.usable || !wide_enough || dims_with_reach > 2 || ec > 1024) return;
+    FastHeader &a = f.adj_hdr;
+    a = h;
+    memset(a.rows_per_tile, 0, sizeof(a.rows_per_tile));
+    memset(a.tiles_per_owner, 0, sizeof(a.tiles_per_owner));
+    a.rows_per_tile[0] = rows_s;
+    a.tiles_per_owner[0] = tiles(ghost_rows_max, rows_s);
+    if (ec > 0) {
+        a.rows_per_tile[1] = (int32_t)std::min<int64_t>(128, std::max<int64_t>(1, 512 / ec));
+        a.tiles_per_owner[1] = tiles(inner_rows_max, a.rows_per_tile[1]);
+    }
+    a.rows_per_tile[2] = rows_s;
+    a.tiles_per_owner[2] = tiles(reach_rows_max, rows_s);
+    {
+        const int64_t total[3] = {(int64_t)a.tiles_per_owner[0] * p->num_workers, (int64_t)a.tiles_per_owner[1] * a.num_lines,
+                                  (int64_t)a.tiles_per_owner[2] * p->num_workers};
+        f.adj_usable = fast_groups(total, &a);
+    }
+}
+
 void split_evenly(int64_t n, int32_t p, std::vector<int64_t> &start, std::vector<int64_t> &size) {
     balanced_split(n, p, start, size);
 }

@@ -136,6 +136,54 @@ def test_reduce_after_broadcast_and_dot_test():
 
 
 # --------------------------------------------------------------------------
+# Broadcast / sum-reduce along partition dimensions
+# --------------------------------------------------------------------------
+
+PARTITION_BROADCAST_CASES = [
+    # source partition, destination partition, elements per source worker, dtype
+    ((1, 4), (4, 4), [256 * 2048] * 4, "f32"),                       # the affine layer's x: 1 x P_fi -> P_fo x P_fi
+    ((4, 1), (4, 4), [70001, 3, 4099, 1 << 16], "f32"),              # its y^ -> y: P_fo x P_fi -> P_fo x 1, ragged sizes
+    ((1, 1, 2, 2, 2), (1, 3, 2, 2, 2), [5000 + 7 * i for i in range(8)], "f32"),   # the convolution's x: ... -> 1 x P_co x P_ci x P_0 x P_1
+    ((1, 2, 1, 2, 2), (1, 2, 3, 2, 2), [4096] * 8, "bf16"),          # its y: 1 x P_co x 1 x P_0 x P_1 <- 1 x P_co x P_ci x P_0 x P_1
+    ((1,), (20,), [33333], "f64"),                                   # more copies than one launch takes
+    ((3,), (3,), [100, 200, 300], "f32"),                            # equal partitions
+]
+
+
+@pytest.mark.parametrize("case", PARTITION_BROADCAST_CASES, ids=[str(c[0]) + "->" + str(c[1]) for c in PARTITION_BROADCAST_CASES])
+def test_partition_broadcast_and_sumreduce_bit_exact(case):
+    src_p, dst_p, sizes, dtype = case
+    src_of = oracle.primitives._partition_sources(src_p, dst_p)
+    scaled = lambda n, seed: (inputs.uniform_pm1((n,), seed) * np.float32(10.0) ** inputs.integers((n,), seed + 1, -3, 4)).astype(np.float32)
+    x32 = [scaled(n, 5000 + 2 * j) for j, n in enumerate(sizes)]
+    y32 = [scaled(sizes[j], 6000 + 2 * w) for w, j in enumerate(src_of)]
+    if dtype == "bf16":
+        x, y = [inputs.f32_to_bf16_bits(a) for a in x32], [inputs.f32_to_bf16_bits(a) for a in y32]
+        up, back, add = _bits_dev, _bits_host, oracle.bf16_add
+        empty = lambda n: torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    elif dtype == "f64":
+        x, y = [a.astype(np.float64) * (1.0 + 2.0 ** -33) for a in x32], [a.astype(np.float64) * (1.0 + 2.0 ** -33) for a in y32]
+        up, back, add = dev, host, None
+        empty = lambda n: torch.empty(n, dtype=torch.float64, device=DEV)
+    else:
+        x, y, up, back, add = x32, y32, dev, host, None
+        empty = lambda n: torch.empty(n, device=DEV)
+    xs, ys = [up(a) for a in x], [up(a) for a in y]
+    out = [empty(sizes[j]) for j in src_of]
+    distdl.partition_broadcast_fwd(src_p, dst_p, xs, out)
+    dx = [empty(n) for n in sizes]
+    distdl.partition_broadcast_adj(src_p, dst_p, ys, dx)
+    torch.cuda.synchronize()
+    for got, ref in zip(out, oracle.partition_broadcast_fwd(src_p, dst_p, x)):
+        assert same_bits(back(got), ref)
+    for got, ref in zip(dx, oracle.partition_broadcast_adj(src_p, dst_p, y, add=add)):
+        assert same_bits(back(got), ref)
+    if dtype == "f32":
+        r = oracle.adjoint_test_ratio([host(t) for t in out], y, x, [host(t) for t in dx])
+        assert r < 1e-5
+
+
+# --------------------------------------------------------------------------
 # Halo exchange
 # --------------------------------------------------------------------------
 
@@ -158,6 +206,29 @@ HALO_CASES = [
     ((67, 61, 68), (3, 2, 2), (2, 4, 4), (3, 4, 4)),          # uneven split, mixed alignment
     ((2, 3, 40, 44), (1, 1, 2, 2), (0, 0, 2, 2), (0, 0, 2, 2)),
 ]
+
+# Geometries whose innermost dimension is made of whole 16-byte units (fp32: multiples of 4): these run through
+# the row plan (ghost rows written end to end, the ghosts at the row ends staged through shared memory).
+ROW_PLAN_CASES = [
+    ((40,), (2,), 4, 4),                                      # rank 1: row ends only
+    ((12, 16), (3, 1), (1, 4), (1, 4)),                       # one worker along the rows: both row ends are cleared
+    ((13, 48), (3, 2), (1, 4), (2, 8)),                       # uneven rows, different widths per side
+    ((9, 7, 64), (2, 3, 4), [[1, 2], [0, 1, 2], [4, 0, 8, 4]], [[2, 0], [1, 1, 0], [4, 8, 0, 4]]),   # per-worker widths
+    ((10, 10, 72), (3, 2, 3), (1, 2, 4), (2, 1, 4)),          # uneven outer splits
+    ((3, 3, 6, 16), (1, 1, 2, 2), (0, 0, 1, 4), (0, 0, 1, 4)),
+    ((4, 5, 6, 4, 16), (2, 1, 2, 1, 2), (1, 0, 1, 1, 4), (0, 1, 1, 0, 4)),
+    ((150, 40, 136), (2, 2, 2), (3, 2, 8), (1, 4, 4)),        # several blocks per worker, two units per ghost
+    ((64, 48), (4, 4), (2, 0), (2, 0)),                       # no ghosts along the rows: row blocks only
+    ((8, 8, 1040), (2, 2, 2), (1, 1, 260), (1, 1, 260)),      # ghosts half as wide as the bulk
+]
+HALO_CASES += ROW_PLAN_CASES
+
+
+def test_row_plan_is_used_where_the_geometry_allows_it():
+    for case in ROW_PLAN_CASES + [((70, 66, 72), (2, 2, 2), 4, 4)]:
+        assert make_partitions(case)[1].uses_row_plan(), case
+    for case in [((11,), (3,), 2, 2), ((67, 61, 68), (3, 2, 2), (2, 4, 4), (3, 4, 4)), ((256, 256), (2, 2), 1, 1)]:
+        assert not make_partitions(case)[1].uses_row_plan(), case
 
 
 @pytest.mark.parametrize("case", HALO_CASES, ids=[str(c[0]) + str(c[1]) for c in HALO_CASES])
@@ -182,6 +253,24 @@ def test_halo_fwd_and_adj_bit_exact(case):
     # the adjoint (dot-product) test on the GPU results, fp64 inner products over every cell
     r = oracle.adjoint_test_ratio([host(t) for t in xs], y, x, [host(t) for t in ys])
     assert r < 1e-5
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """A wait that nothing ends: the kernel gives up after its limit (here about a millisecond of SM cycles),
+    returns by itself and leaves DISTDL_ERR_TIMEOUT in the status word, once; the context stays usable."""
+    distdl.device_status()
+    distdl.selftest_wait_timeout(2_000_000)
+    with pytest.raises(distdl.DistdlError) as err:
+        distdl.device_status()
+    assert err.value.status == 6 and "wait" in str(err.value)
+    distdl.device_status()                                   # reported once, then clear again
+    x = inputs.uniform_pm1((4097,), 77)
+    out = [torch.empty(4097, device=DEV) for _ in range(2)]
+    distdl.broadcast_fwd(dev(x), out)                        # ordinary work still runs
+    torch.cuda.synchronize()
+    assert all(same_bits(host(o), x) for o in out)
+    with pytest.raises(distdl.DistdlError):
+        distdl.selftest_wait_timeout(10 ** 12)               # limits of seconds are refused
 
 
 def test_halo_adj_order_sensitive_values():
@@ -323,6 +412,9 @@ PERIODIC_HALO_CASES = [
     ((12, 16), (1, 3), (2, 1), (1, 2), (True, True)),
     ((8, 10, 12), (2, 1, 2), (1, 1, 1), (1, 1, 1), (False, True, True)),
     ((70, 66, 72), (2, 2, 2), (4, 4, 4), (4, 4, 4), (True, True, True)),      # 16-byte paths, several tiles
+    ((16,), (1,), (4,), (8,), (True,)),                                       # a worker that is its own neighbour
+    ((12, 32), (1, 2), (2, 4), (1, 8), (True, True)),                         # the same neighbour on both sides
+    ((6, 10, 48), (2, 1, 3), (1, 2, 4), (2, 1, 4), (True, False, True)),
 ]
 
 
@@ -970,6 +1062,50 @@ def test_random_halo_geometries(seed):
         assert same_bits(host(a), b)
     for a, b in zip(ys, oracle.halo_adj_sequence(opart, y)):
         assert same_bits(host(a), b)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_row_plan_geometries(seed):
+    """Random geometries with rows of whole 16-byte units, in all three element types."""
+    rng = np.random.Generator(np.random.Philox(7500 + seed))
+    rank = int(rng.integers(1, 5))
+    code, per_unit = [(distdl.F32, 4), (distdl.F64, 2), (distdl.BF16, 8)][seed % 3]
+    gs, ps = _random_geometry(rng, rank, 30 if rank < 3 else 14, 4, 3)
+    gs, ps = list(gs), list(ps)
+    gs[-1] = ps[-1] * per_unit * int(rng.integers(1, 4))                  # equal blocks of whole units along the rows
+    periodic = tuple(bool(rng.integers(0, 2)) for _ in range(rank)) if seed % 2 == 0 else None
+    if periodic is None:
+        sizes = [oracle.balanced_split(gs[k], ps[k])[1] for k in range(rank)]
+        step = [1] * (rank - 1) + [per_unit]
+        hlo = [[step[k] * int(rng.integers(0, min(3, sizes[k][c - 1] // step[k]) + 1)) if c > 0
+                else step[k] * int(rng.integers(0, 3)) for c in range(ps[k])] for k in range(rank)]
+        hhi = [[step[k] * int(rng.integers(0, min(3, sizes[k][c + 1] // step[k]) + 1)) if c + 1 < ps[k]
+                else step[k] * int(rng.integers(0, 3)) for c in range(ps[k])] for k in range(rank)]
+        opart = oracle.Partition(gs, ps, hlo, hhi)
+        gpart = distdl.Partition(gs, ps, hlo, hhi, dtype=code)
+    else:
+        h = tuple(int(rng.integers(0, 3)) for _ in range(rank - 1)) + (per_unit * int(rng.integers(0, 2)),)
+        opart = oracle.Partition(gs, ps, h, h, periodic)
+        gpart = distdl.Partition(gs, ps, h, h, dtype=code, periodic=periodic)
+    x32, y32 = random_shards(opart, 150 + seed), random_shards(opart, 180 + seed)
+    if code == distdl.F32:
+        x, y, add, back = x32, y32, None, host
+        xs, ys = [dev(a) for a in x], [dev(a) for a in y]
+    elif code == distdl.F64:
+        x = [a.astype(np.float64) * (1.0 + 2.0 ** -33) for a in x32]
+        y = [a.astype(np.float64) * (1.0 + 2.0 ** -33) for a in y32]
+        xs, ys, add, back = [dev(a) for a in x], [dev(a) for a in y], None, host
+    else:
+        x = [inputs.f32_to_bf16_bits(a) for a in x32]
+        y = [inputs.f32_to_bf16_bits(a) for a in y32]
+        xs, ys, add, back = [_bits_dev(a) for a in x], [_bits_dev(a) for a in y], oracle.bf16_add, _bits_host
+    distdl.halo_fwd(gpart, xs)
+    distdl.halo_adj(gpart, ys)
+    torch.cuda.synchronize()
+    for a, b in zip(xs, oracle.halo_fwd_sequence(opart, x)):
+        assert same_bits(back(a), b)
+    for a, b in zip(ys, oracle.halo_adj_sequence(opart, y, add=add)):
+        assert same_bits(back(a), b)
 
 
 @pytest.mark.parametrize("seed", range(8))

@@ -16,9 +16,15 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "distdl.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(distdl_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for header in sorted(os.listdir(inc)):
+        if not header.endswith(".h"):
+            continue
+        text = open(os.path.join(inc, header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names.update(re.findall(r"\b(distdl_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol():
@@ -233,3 +239,50 @@ def test_header_compiles_as_c_and_the_library_links_from_c(tmp_path):
                            "-L", libdir, "-ldistdl", "-Wl,-rpath," + libdir])
     out = subprocess.run([exe], capture_output=True, text=True)
     assert out.returncode == 0 and out.stdout.strip().endswith("ok"), out.stdout + out.stderr
+
+
+@pytest.mark.parametrize("gs,ps,lo,hi", [
+    ((512, 512, 512), (4, 4, 4), (4, 4, 4), (4, 4, 4)),
+    ((256, 256), (2, 2), (1, 1), (1, 1)),
+    ((70, 66, 72), (2, 3, 2), (4, 2, 3), (1, 4, 2)),
+    ((37, 45), (3, 2), (2, 1), (1, 3)),
+    ((9, 40), (4, 1), (2, 3), (2, 0)),            # shards as thin as their neighbours' ghosts
+    ((16, 16, 1024, 1024), (1, 1, 4, 4), (0, 0, 2, 2), (0, 0, 2, 2)),
+])
+def test_bench_byte_counts_from_oracle_geometry_match_the_planner(gs, ps, lo, hi):
+    """bench.py counts the algorithmic bytes of H, H* and the convolution from partition geometry alone (the
+    oracle's Partition, or its own extents-only stand-in); the library's planner counts them from its box lists."""
+    import bench
+    gp = distdl.Partition(gs, ps, lo, hi)
+    want = (gp.halo_stats(False)[2], gp.halo_stats(True)[2])
+    assert bench.halo_algorithmic_bytes(oracle.Partition(gs, ps, lo, hi)) == want
+    assert bench.halo_algorithmic_bytes(bench._Geometry(gs, ps, lo, hi)) == want
+    if len(gs) == 4:
+        a = bench.conv_algorithmic_bytes(oracle.Partition(gs, ps, lo, hi))
+        assert a == bench.conv_algorithmic_bytes(bench._Geometry(gs, ps, lo, hi)) == 2172796928
+
+
+def test_bench_reference_arm_does_not_load_the_cuda_library():
+    """`bench.py --impl reference` and the CPU-baseline leg time the oracle alone."""
+    import subprocess, sys
+    code = ("import sys, bench; b, s, per = bench.oracle_sample_step(bench.ORACLE_LEVELS[2]); "
+            "import paper_2006_03108_b200 as d; assert d._lib is None, 'library was loaded'; "
+            "assert b > 0 and s > 0; print('ok')")
+    r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0 and r.stdout.strip() == "ok", r.stderr
+
+
+def test_partition_broadcast_rejects_shapes_that_do_not_broadcast():
+    lib = distdl.lib()
+    one = ctypes.c_void_p(256)
+    ptrs = (ctypes.c_void_p * 8)(*[256] * 8)
+    elems = (ctypes.c_int64 * 8)(*[4] * 8)
+
+    def call(src_p, dst_p):
+        r = len(src_p)
+        return lib.distdl_partition_broadcast_fwd(r, (ctypes.c_int32 * r)(*src_p), (ctypes.c_int32 * r)(*dst_p), elems,
+                                                  ptrs, ptrs, distdl.F32, None)
+    assert call((2, 2), (4, 2)) == 2 and b"dimension 0" in lib.distdl_last_error()       # DISTDL_ERR_SHAPE
+    assert call((2, 1), (1, 2)) == 2
+    assert call((1,), (512,)) == 4                                                        # DISTDL_ERR_UNSUPPORTED
+    assert lib.distdl_partition_broadcast_fwd(1, None, None, elems, ptrs, ptrs, distdl.F32, None) == 1

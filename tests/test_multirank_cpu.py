@@ -1,7 +1,8 @@
 """World-size-2 check (gloo, CPU) of the host logic that bench.py uses when it runs N replicas:
 every rank times its own replica, the slowest rank decides, and the reported value is N times the
-per-replica work divided by that time.  No data-path collective exists, so this is all there is to
-cover."""
+per-replica work divided by that time.  The two functions of bench.py that do this (reduce_max_ms,
+aggregate_value) are called here as they stand.  No data-path collective exists, so this is all there
+is to cover."""
 
 import os
 import socket
@@ -23,15 +24,17 @@ def _free_port():
 def _worker(rank, world, port, out):
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    if root not in sys.path:
+        sys.path.insert(0, root)
+    import bench
     dist.init_process_group("gloo", rank=rank, world_size=world)
     # each rank "measures" a different time for the same per-replica work
-    elapsed_ms = torch.tensor([10.0 + 5.0 * rank], dtype=torch.float64)
     dist.barrier()
-    dist.all_reduce(elapsed_ms, op=dist.ReduceOp.MAX)
-    bytes_per_replica = 6_000_000_000
-    value = world * bytes_per_replica / (elapsed_ms.item() * 1e-3) / 1e9
+    elapsed_ms = bench.reduce_max_ms(10.0 + 5.0 * rank, world, dist, torch, torch.device("cpu"))
+    value = bench.aggregate_value(6_000_000_000, world, elapsed_ms)
     if rank == 0:
-        out.put((elapsed_ms.item(), value))
+        out.put((elapsed_ms, value))
     dist.destroy_process_group()
 
 
