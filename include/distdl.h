@@ -195,11 +195,12 @@ distdl_status_t distdl_partition_broadcast_adj(int32_t rank, const int32_t *src_
  * ---------------------------------------------------------------------- */
 distdl_status_t distdl_halo_fwd(const distdl_partition_t *p, void *const *shards, void *stream);
 distdl_status_t distdl_halo_adj(const distdl_partition_t *p, void *const *shards, void *stream);
-/* 1 if H (adjoint = 0) or H* (adjoint != 0) of this partition runs through the row plan -- every ghost
- * width and bulk extent of the innermost dimension is a whole number of 16-byte units, so ghost rows are
- * moved end to end as aligned vectors; for H* also: every bulk is at least as wide as the ghosts its two
- * neighbours hold of it together, and at most two of the outer dimensions have neighbours -- 0 if it runs
- * through the general box plan, -1 for a NULL partition.  Same results, bit for bit, either way. */
+/* 1 if H (adjoint = 0) of this partition runs through the row plan -- every ghost width and bulk extent of
+ * the innermost dimension is a whole number of 16-byte units, so ghost rows are moved end to end as aligned
+ * vectors and the ghosts at the row ends are staged through shared memory -- or (adjoint != 0) if H* hands
+ * the row ends to it: besides the above, every bulk is at least as wide as the ghosts its two neighbours
+ * hold of it together, and the innermost dimension has neighbours.  0 if the general box plan does all the
+ * work, -1 for a NULL partition.  Same results, bit for bit, either way. */
 int32_t         distdl_partition_uses_row_plan(const distdl_partition_t *p, int32_t adjoint);
 
 /* ------------------------------------------------------------------------

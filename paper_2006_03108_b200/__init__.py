@@ -213,7 +213,8 @@ class Partition:
         return a.value, b.value, c.value
 
     def uses_row_plan(self, adjoint=False):
-        """True if H (or H*) of this partition runs through the row plan (rows of whole 16-byte units)."""
+        """True if H of this partition runs through the row plan (rows of whole 16-byte units), or, with adjoint, if
+        H* hands the row ends to it."""
         return lib().distdl_partition_uses_row_plan(self._h, 1 if adjoint else 0) == 1
 
     def close(self):
@@ -469,7 +470,8 @@ def selftest_wait_timeout(limit_cycles, stream=None):
 
 
 def selftest_row_plan(part, adjoint=False):
-    """(header words, list of 16-word records) of a partition's row plan (include/distdl_selftest.h)."""
+    """(header words, list of 16-word records) of a partition's row plan (include/distdl_selftest.h): of H, or of
+    the row ends of H*."""
     hdr = (ctypes.c_int32 * 64)()
     rec = (ctypes.c_int32 * (16 * 64))()
     n = ctypes.c_int32(0)

@@ -131,21 +131,20 @@ struct FastHeader {
     int32_t wstride[kMaxBoxDims];     // worker-id stride of a step along dimension k
     int32_t num_records;
     int32_t num_lines;                // workers / pshape[rank - 1]
-    // kind 0: ghost rows (H: filled; H*: the ones outside the tensor cleared), per worker
+    // kind 0: ghost rows, per worker (H only)
     // kind 1: row ends of bulk rows, per line of workers along the innermost dimension (H: all bulk rows; H*: the bulk
-    //         rows out of reach in every outer dimension)
-    // kind 2 (H* only): bulk rows within a neighbour's reach in some outer dimension, per worker
-    int32_t rows_per_tile[3];
-    int32_t tiles_per_owner[3];       // per worker (kinds 0, 2) or per line (kind 1)
-    int32_t group[3];                 // blocks of each kind per group
+    //         rows out of every outer neighbour's reach)
+    int32_t rows_per_tile[2];
+    int32_t tiles_per_owner[2];       // per worker (kind 0) or per line (kind 1)
+    int32_t group[2];                 // blocks of each kind per group
     int32_t num_groups;
 };
 
 struct FastPlanHost {
     bool usable = false;              // H runs through the row plan
-    bool adj_usable = false;          // H* too (needs bulks at least as wide as the two neighbours' reach together)
+    bool adj_usable = false;          // the row ends of H* too (needs bulks at least as wide as the two neighbours' reach together)
     FastHeader hdr;                   // H
-    FastHeader adj_hdr;               // H*
+    FastHeader adj_hdr;               // H*: line blocks only
     std::vector<FastDim> dims;
 };
 
@@ -173,6 +172,9 @@ struct distdl_partition {
 
     distdl::HaloPlanHost fwd_host, adj_host;
     distdl::HaloPlanDevice fwd_dev, adj_dev;
+    // H* without the row ends that the row plan handles (built when fast.adj_usable)
+    distdl::HaloPlanHost adj_rest_host;
+    distdl::HaloPlanDevice adj_rest_dev;
     distdl::FastPlanHost fast;      // row plan (see FastDim); fast.usable says whether the geometry allows it
     distdl::FastDim *fast_dims_dev = nullptr;
     void *device_block = nullptr;   // one allocation holding all device tables

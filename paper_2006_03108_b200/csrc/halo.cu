@@ -8,6 +8,9 @@
 // same nested sum the d reversed phases would produce -- own value, low neighbour, high
 // neighbour within a dimension; dimension 0 outermost -- so the result is bit-identical to the
 // phase-by-phase order.  Each ghost cell is read by exactly one thread, which also clears it.
+#include <cstdlib>
+#include <cstring>
+
 #include "common.h"
 
 namespace distdl {
@@ -283,23 +286,19 @@ halo_box_kernel(const HaloBox *__restrict__ boxes, const HaloSource *__restrict_
 
 
 // ---------------------------------------------------------------------------------------------
-// Row plan kernels (see FastDim): H and H* for partitions whose innermost dimension is made of
-// whole 16-byte units.  Kinds of block, dealt out interleaved:
+// Row plan kernels (see FastDim): H, and the row ends of H*, for partitions whose innermost
+// dimension is made of whole 16-byte units.  Kinds of block, dealt out interleaved:
 //
 //  * ghost-row blocks: a range of one worker's *ghost rows* -- rows of the padded array whose index
 //    is a ghost index in some outer dimension.  Such a row is ghost from end to end, and consecutive
 //    ghost rows are contiguous in memory, so the block writes whole runs of memory; each row is
 //    fetched as (low ghost columns | bulk columns | high ghost columns) from up to three neighbours.
-//    H* only clears the ghost rows (or parts of rows) that lie outside the tensor here; the others are
-//    cleared by the thread that adds them to their bulk cell.
 //  * line blocks: a range of bulk rows of all the workers that sit next to each other along the
 //    innermost dimension.  There the ghosts are a few units at both ends of every row.  The ghost
 //    units at the end of row r and at the start of row r + 1 are adjacent in memory, and so are the
 //    bulk units that the two neighbours want from (H) or add to (H*) those rows; loads are issued in
 //    the order of the source rows and stores in the order of the destination rows, with shared
 //    memory in between, so that a warp touches each 128-byte line once per direction.
-//  * receiving-row blocks (H* only): bulk rows that a neighbour in some outer dimension holds ghost
-//    copies of.  Every unit of such a row is the nested sum of two, four or eight terms.
 // ---------------------------------------------------------------------------------------------
 constexpr int kFastThreads = 256;
 constexpr int kFastMaxRows = 256;      // row records per block
@@ -317,17 +316,13 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t x, uint32_t magic, uint32_
 
 // Which kind of block this is, and its index among the blocks of that kind.
 __device__ __forceinline__ int fast_block_kind(const FastHeader &H, uint32_t *tile_id) {
-    const uint32_t per_group = (uint32_t)(H.group[0] + H.group[1] + H.group[2]);
+    const uint32_t per_group = (uint32_t)(H.group[0] + H.group[1]);
     const uint32_t group = blockIdx.x / per_group;
     uint32_t in_group = blockIdx.x - group * per_group;
     int kind = 0;
     if (in_group >= (uint32_t)H.group[0]) {
         in_group -= (uint32_t)H.group[0];
         kind = 1;
-        if (in_group >= (uint32_t)H.group[1]) {
-            in_group -= (uint32_t)H.group[1];
-            kind = 2;
-        }
     }
     *tile_id = group * (uint32_t)H.group[kind] + in_group;
     return kind;
@@ -353,22 +348,13 @@ __device__ __forceinline__ void fast_worker(const FastHeader &H, const FastDim *
     }
 }
 
-// Ghost-row block of worker s: rows [row0, ...) of its ghost rows.  CLEAR_ONLY: only the units without a
-// source (outside the tensor) are written, with zeros.
-template <bool CLEAR_ONLY>
+// Ghost-row block of worker s: rows [row0, ...) of its ghost rows.
 __device__ __forceinline__ void fast_ghost_rows(const FastHeader &H, const FastDim *dims, const ShardPointers &sh,
                                                 unsigned char *scratch, uint32_t s, uint32_t t) {
     const int d = H.rank;
     int c[kMaxBoxDims];
     const FastDim *e[kMaxBoxDims];
     fast_worker(H, dims, s, c, e);
-    if (CLEAR_ONLY) {
-        bool complete = true;       // a worker with neighbours on every side has no ghost outside the tensor
-#pragma unroll
-        for (int k = 0; k < kMaxBoxDims; ++k)
-            if (k < d && ((e[k]->hlo > 0 && e[k]->lo_c < 0) || (e[k]->n - e[k]->hlo - e[k]->b > 0 && e[k]->hi_c < 0))) complete = false;
-        if (complete) return;
-    }
     // class j holds the rows whose index is a bulk index in the dimensions before j, a ghost index in dimension j
     // and anything after it
     uint32_t cls_rows[kMaxBoxDims];
@@ -478,12 +464,8 @@ __device__ __forceinline__ void fast_ghost_rows(const FastHeader &H, const FastD
                 const int reg = col < xlo ? 0 : (col < xhi ? 1 : 2);
                 const int src = r.shard[reg];
                 doff[u] = r.dst_off + col;
-                if (CLEAR_ONLY) {
-                    wr[u] = src < 0;
-                } else {
-                    wr[u] = true;
-                    if (src >= 0) v[u] = __ldg(reinterpret_cast<const uint4 *>(sh.p[src]) + (r.off[reg] + col));
-                }
+                wr[u] = true;
+                if (src >= 0) v[u] = __ldg(reinterpret_cast<const uint4 *>(sh.p[src]) + (r.off[reg] + col));
             }
         }
 #pragma unroll
@@ -529,7 +511,7 @@ halo_fast_fwd_kernel(const __grid_constant__ FastHeader H, const FastDim *__rest
     const int kind = fast_block_kind(H, &tile_id);
     if (kind == 0) {
         const uint32_t s = tile_id / (uint32_t)H.tiles_per_owner[0];
-        if (s < (uint32_t)H.num_workers) fast_ghost_rows<false>(H, dims, sh, scratch, s, tile_id - s * (uint32_t)H.tiles_per_owner[0]);
+        if (s < (uint32_t)H.num_workers) fast_ghost_rows(H, dims, sh, scratch, s, tile_id - s * (uint32_t)H.tiles_per_owner[0]);
         return;
     }
     // ---------------------------------------------------------------------- line block
@@ -607,187 +589,27 @@ halo_fast_fwd_kernel(const __grid_constant__ FastHeader H, const FastDim *__rest
 }
 
 // ---------------------------------------------------------------------------------------------
-// H* through the row plan.  T: 16-byte vector of the element type (float4, double2, bf16x8).
+// H* at the row ends.  T: 16-byte vector of the element type (float4, double2, bf16x8).
+//
+// The box plan is at its best where rows are long; where a partition is split along the innermost
+// dimension, most of its boxes are columns a few units wide.  For those H* runs in two launches that
+// touch disjoint cells: the box kernel on a plan without the row-end columns of the bulk rows that no
+// outer neighbour reaches, and this kernel on exactly those.  There a bulk unit near a row end receives
+// from one ghost unit of the neighbour along the row, and every unit involved -- low ghost, low
+// receiving, high receiving, high ghost of every worker of the line -- is read once and written once,
+// in memory order, with the neighbour's ghost value taken from shared memory.
 // ---------------------------------------------------------------------------------------------
-struct FastSumRec {
-    uint32_t nterms;       // rows added together: 1 << (outer dimensions in which the row is within a neighbour's reach)
-    int32_t shard[4];      // worker of every row, without the coordinate along the innermost dimension; [0] is the row itself
-    uint32_t lin[4];       // linear index of the row in that worker's array (multiply by its row pitch)
-};
-
-template <typename T, int N>
-__device__ __forceinline__ void fast_sum_unit(T *const *ptr) {
-    T v[N];
-#pragma unroll
-    for (int j = 0; j < N; ++j) v[j] = *ptr[j];
-    // fixed tree: neighbouring terms first (innermost dimension), own value before the neighbour's at every level
-#pragma unroll
-    for (int width = 1; width < N; width *= 2)
-#pragma unroll
-        for (int j = 0; j < N; j += 2 * width) v[j] = vadd(v[j], v[j + width]);
-    stores_after(v[0]);
-    *ptr[0] = v[0];
-#pragma unroll
-    for (int j = 1; j < N; ++j) *ptr[j] = zero_of<T>();
-}
-
 template <typename T>
 __global__ void __launch_bounds__(kFastThreads)
-halo_fast_adj_kernel(const __grid_constant__ FastHeader H, const FastDim *__restrict__ dims_g,
-                     const __grid_constant__ ShardPointers sh) {
+halo_fast_adj_lines_kernel(const __grid_constant__ FastHeader H, const FastDim *__restrict__ dims_g,
+                           const __grid_constant__ ShardPointers sh) {
     __shared__ FastDim dims[kMaxFastCoords];
     __shared__ __align__(16) unsigned char scratch[kFastMaxSlots * 16];
     fast_load_records(H, dims_g, dims);
     const int d = H.rank;
     uint32_t tile_id;
-    const int kind = fast_block_kind(H, &tile_id);
-    if (kind == 0) {
-        // ghost rows outside the tensor: cleared; the others are cleared by whoever adds them to a bulk cell
-        const uint32_t s = tile_id / (uint32_t)H.tiles_per_owner[0];
-        if (s < (uint32_t)H.num_workers) fast_ghost_rows<true>(H, dims, sh, scratch, s, tile_id - s * (uint32_t)H.tiles_per_owner[0]);
-        return;
-    }
-    if (kind == 2) {
-        // ------------------------------------------------------------------ receiving rows
-        const uint32_t s = tile_id / (uint32_t)H.tiles_per_owner[2];
-        if (s >= (uint32_t)H.num_workers) return;
-        const uint32_t t = tile_id - s * (uint32_t)H.tiles_per_owner[2];
-        int c[kMaxBoxDims];
-        const FastDim *e[kMaxBoxDims];
-        fast_worker(H, dims, s, c, e);
-        // class j: out of reach in the dimensions before j, within reach in dimension j, any bulk index after it
-        uint32_t cls_rows[kMaxBoxDims];
-        uint32_t total_rows = 0;
-#pragma unroll
-        for (int j = 0; j < kMaxBoxDims - 1; ++j) {
-            cls_rows[j] = 0;
-            if (j < d - 1) {
-                uint32_t r = (uint32_t)(e[j]->rlo + e[j]->rhi);
-#pragma unroll
-                for (int k = 0; k < kMaxBoxDims - 1; ++k)
-                    if (k < d - 1 && k != j) r *= (uint32_t)(k < j ? e[k]->b - e[k]->rlo - e[k]->rhi : e[k]->b);
-                cls_rows[j] = r;
-                total_rows += r;
-            }
-        }
-        const uint32_t row0 = t * (uint32_t)H.rows_per_tile[2];
-        if (row0 >= total_rows) return;
-        const uint32_t nrows = min((uint32_t)H.rows_per_tile[2], total_rows - row0);
-        FastSumRec *recs = reinterpret_cast<FastSumRec *>(scratch);
-        static_assert(sizeof(FastSumRec) * kFastMaxRows <= kFastMaxSlots * 16, "row records fit the scratch array");
-        for (uint32_t rl = threadIdx.x; rl < nrows; rl += kFastThreads) {
-            uint32_t idx = row0 + rl;
-            int j = 0;
-#pragma unroll
-            for (int q = 0; q < kMaxBoxDims - 2; ++q)
-                if (j == q && q < d - 2 && idx >= cls_rows[q]) {
-                    idx -= cls_rows[q];
-                    ++j;
-                }
-            FastSumRec r;
-            r.nterms = 1;
-            r.shard[0] = 0;
-            r.lin[0] = 0;
-            uint32_t pitch[4] = {1, 1, 1, 1};
-            // innermost outer dimension first: a dimension within reach doubles the rows, the new ones (the
-            // neighbour's ghost rows) after the old ones, so the outermost dimension ends up as the slowest index
-            // of the list, as the nested sum wants it
-#pragma unroll
-            for (int k = kMaxBoxDims - 2; k >= 0; --k) {
-                if (k < d - 1) {
-                    const FastDim &f = *e[k];
-                    const uint32_t inner = (uint32_t)(f.b - f.rlo - f.rhi), rr = (uint32_t)(f.rlo + f.rhi);
-                    uint32_t coord = idx;
-                    if (k > 0) {
-                        const uint32_t ext = k > j ? (uint32_t)f.b : (k == j ? rr : inner);
-                        const uint32_t q = k > j ? fast_div(idx, f.magic_b, fast_shift_b(f))
-                                                 : (k == j ? fast_div(idx, f.magic_rr, fast_shift_rr(f)) : fast_div(idx, f.magic_bi, fast_shift_bi(f)));
-                        coord = idx - q * ext;
-                        idx = q;
-                    }
-                    // position inside the bulk
-                    const uint32_t pos = k > j ? coord : (k == j ? (coord < (uint32_t)f.rlo ? coord : coord + inner) : (uint32_t)f.rlo + coord);
-                    const int i = f.hlo + (int)pos;
-                    int nc = -1, si = 0;
-                    if (pos < (uint32_t)f.rlo) {
-                        nc = f.lo_c;
-                        si = i + f.lo_shift;
-                    } else if (pos >= (uint32_t)(f.b - f.rhi)) {
-                        nc = f.hi_c;
-                        si = i + f.hi_shift;
-                    }
-                    const uint32_t old = r.nterms;
-                    if (nc >= 0 && old <= 2) {
-                        const uint32_t npitch = (uint32_t)dims[H.dim_base[k] + nc].n;
-#pragma unroll
-                        for (uint32_t q = 0; q < 2; ++q)
-                            if (q < old) {
-                                r.shard[old + q] = r.shard[q] + nc * H.wstride[k];
-                                r.lin[old + q] = r.lin[q] + (uint32_t)si * pitch[q];
-                                pitch[old + q] = pitch[q] * npitch;
-                            }
-                        r.nterms = 2 * old;
-                    }
-#pragma unroll
-                    for (uint32_t q = 0; q < 2; ++q)
-                        if (q < old) {
-                            r.shard[q] += c[k] * H.wstride[k];
-                            r.lin[q] += (uint32_t)i * pitch[q];
-                            pitch[q] *= (uint32_t)f.n;
-                        }
-                }
-            }
-            recs[rl] = r;
-        }
-        __syncthreads();
-        const FastDim *ex = e[d - 1];
-        const uint32_t nx = (uint32_t)ex->n;
-        const uint32_t count = nrows * nx;
-        const uint32_t shx = fast_shift_n(*ex);
-        const int cx = c[d - 1];
-        for (uint32_t i = threadIdx.x; i < count; i += kFastThreads) {
-            const uint32_t rl = fast_div(i, ex->magic_n, shx);
-            const uint32_t col = i - rl * nx;
-            const FastSumRec &r = recs[rl];
-            if (col < (uint32_t)ex->hlo || col >= (uint32_t)(ex->hlo + ex->b)) {
-                // a ghost unit at the end of a bulk row: its neighbour along the row clears it, unless there is none
-                const bool none = col < (uint32_t)ex->hlo ? ex->lo_c < 0 : ex->hi_c < 0;
-                if (none) reinterpret_cast<T *>(sh.p[s])[r.lin[0] * nx + col] = zero_of<T>();
-                continue;
-            }
-            const uint32_t pos = col - (uint32_t)ex->hlo;
-            int ncx = -1, shift = 0;
-            if (pos < (uint32_t)ex->rlo) {
-                ncx = ex->lo_c;
-                shift = ex->lo_shift;
-            } else if (pos >= (uint32_t)(ex->b - ex->rhi)) {
-                ncx = ex->hi_c;
-                shift = ex->hi_shift;
-            }
-            T *ptr[8];
-            const uint32_t nt = r.nterms;
-            const uint32_t nnx = ncx >= 0 ? (uint32_t)dims[H.dim_base[d - 1] + ncx].n : 0u;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if ((uint32_t)q < nt) {
-                    T *own = reinterpret_cast<T *>(sh.p[r.shard[q] + cx]) + (r.lin[q] * nx + col);
-                    if (ncx >= 0) {
-                        ptr[2 * q] = own;
-                        ptr[2 * q + 1] = reinterpret_cast<T *>(sh.p[r.shard[q] + ncx]) + (r.lin[q] * nnx + (uint32_t)((int)col + shift));
-                    } else {
-                        ptr[q] = own;
-                    }
-                }
-            }
-            const uint32_t terms = ncx >= 0 ? 2 * nt : nt;
-            if (terms == 2) fast_sum_unit<T, 2>(ptr);
-            else if (terms == 4) fast_sum_unit<T, 4>(ptr);
-            else if (terms == 8) fast_sum_unit<T, 8>(ptr);
-        }
-        return;
-    }
-    // ---------------------------------------------------------------------- line block: both ends of the bulk rows that
-    // are out of reach in every outer dimension, for all workers of the line
+    if (fast_block_kind(H, &tile_id) != 1) return;
+    // both ends of the bulk rows that are out of reach in every outer dimension, for all workers of the line
     const uint32_t line = tile_id / (uint32_t)H.tiles_per_owner[1];
     if (line >= (uint32_t)H.num_lines) return;
     const uint32_t t = tile_id - line * (uint32_t)H.tiles_per_owner[1];
@@ -884,20 +706,40 @@ static distdl_status_t launch(const distdl_partition *p, const HaloPlanDevice &p
     }
     for (int32_t w = p->num_workers; w < DISTDL_MAX_WORKERS; ++w) sh.p[w] = nullptr;
     if (plan.num_tiles == 0) return DISTDL_OK;
+    // DISTDL_HALO_PLAN=box in the environment sends every call through the general box plan (for comparisons)
+    static const bool box_only = [] {
+        const char *v = getenv("DISTDL_HALO_PLAN");
+        return v && strcmp(v, "box") == 0;
+    }();
+    if (box_only) {
+        if (adjoint)
+            halo_box_kernel<true><<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(
+                plan.boxes, plan.sources, plan.tiles, elem_size(p->dtype), sh);
+        else
+            halo_box_kernel<false><<<plan.num_tiles, kHaloThreads, 0, (cudaStream_t)stream>>>(
+                plan.boxes, plan.sources, plan.tiles, elem_size(p->dtype), sh);
+        DISTDL_CUDA_CHECK(cudaGetLastError());
+        return DISTDL_OK;
+    }
     if (!adjoint && p->fast.usable && p->fast_dims_dev) {
         const FastHeader &h = p->fast.hdr;
-        halo_fast_fwd_kernel<<<(unsigned)h.num_groups * (unsigned)(h.group[0] + h.group[1] + h.group[2]), kFastThreads, 0,
+        halo_fast_fwd_kernel<<<(unsigned)h.num_groups * (unsigned)(h.group[0] + h.group[1]), kFastThreads, 0,
                                (cudaStream_t)stream>>>(h, p->fast_dims_dev, sh);
         DISTDL_CUDA_CHECK(cudaGetLastError());
         return DISTDL_OK;
     }
     if (adjoint && p->fast.adj_usable && p->fast_dims_dev) {
-        const FastHeader &h = p->fast.adj_hdr;
-        const unsigned grid = (unsigned)h.num_groups * (unsigned)(h.group[0] + h.group[1] + h.group[2]);
         cudaStream_t st = (cudaStream_t)stream;
-        if (p->dtype == DISTDL_F32) halo_fast_adj_kernel<float4><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
-        else if (p->dtype == DISTDL_F64) halo_fast_adj_kernel<double2><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
-        else halo_fast_adj_kernel<bf16x8><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
+        const HaloPlanDevice &rest = p->adj_rest_dev;      // everything but the row ends of the rows out of outer reach
+        if (rest.num_tiles > 0) {
+            halo_box_kernel<true><<<rest.num_tiles, kHaloThreads, 0, st>>>(rest.boxes, rest.sources, rest.tiles, elem_size(p->dtype), sh);
+            DISTDL_CUDA_CHECK(cudaGetLastError());
+        }
+        const FastHeader &h = p->fast.adj_hdr;
+        const unsigned grid = (unsigned)h.num_groups * (unsigned)(h.group[0] + h.group[1]);
+        if (p->dtype == DISTDL_F32) halo_fast_adj_lines_kernel<float4><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
+        else if (p->dtype == DISTDL_F64) halo_fast_adj_lines_kernel<double2><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
+        else halo_fast_adj_lines_kernel<bf16x8><<<grid, kFastThreads, 0, st>>>(h, p->fast_dims_dev, sh);
         DISTDL_CUDA_CHECK(cudaGetLastError());
         return DISTDL_OK;
     }

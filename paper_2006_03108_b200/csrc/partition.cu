@@ -122,20 +122,42 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
             delete p;
             return fail(DISTDL_ERR_UNSUPPORTED, "partition_create: shard too large");
         }
+    build_fast_plan(p);
     distdl_status_t st = build_halo_plans(p);
     if (st != DISTDL_OK) {
         delete p;
         return st;
     }
-    build_fast_plan(p);
     // Upload.  Without a CUDA device the object stays host-only: geometry queries work, operator
     // calls report DISTDL_ERR_CUDA.
     if (upload) {
-        void *fast_dev = nullptr;
+        // one more blob behind the two box plans: the row plan's records and the box plan of the rest of H*
+        std::vector<unsigned char> blob;
+        size_t at_boxes = 0, at_sources = 0, at_tiles = 0;
+        auto append = [&blob](const void *src, size_t n) {
+            const size_t at = blob.size();
+            blob.resize(at + ((n + 255) & ~(size_t)255));
+            if (n) memcpy(blob.data() + at, src, n);
+            return at;
+        };
+        if (p->fast.usable) {
+            append(p->fast.dims.data(), p->fast.dims.size() * sizeof(FastDim));
+            const HaloPlanHost &r = p->adj_rest_host;
+            at_boxes = append(r.boxes.data(), r.boxes.size() * sizeof(HaloBox));
+            at_sources = append(r.sources.data(), r.sources.size() * sizeof(HaloSource));
+            at_tiles = append(r.tiles.data(), r.tiles.size() * sizeof(HaloTile));
+        }
+        void *blob_dev = nullptr;
         st = upload_plan_pair(p->fwd_host, p->adj_host, &p->fwd_dev, &p->adj_dev, &p->device_block, &p->device,
-                              "partition_create", p->fast.usable ? p->fast.dims.data() : nullptr,
-                              p->fast.usable ? p->fast.dims.size() * sizeof(FastDim) : 0, &fast_dev);
-        p->fast_dims_dev = static_cast<FastDim *>(fast_dev);
+                              "partition_create", blob.data(), blob.size(), &blob_dev);
+        if (st == DISTDL_OK && blob_dev) {
+            unsigned char *base = static_cast<unsigned char *>(blob_dev);
+            p->fast_dims_dev = reinterpret_cast<FastDim *>(base);
+            p->adj_rest_dev.boxes = reinterpret_cast<HaloBox *>(base + at_boxes);
+            p->adj_rest_dev.sources = reinterpret_cast<HaloSource *>(base + at_sources);
+            p->adj_rest_dev.tiles = reinterpret_cast<HaloTile *>(base + at_tiles);
+            p->adj_rest_dev.num_tiles = (int32_t)p->adj_rest_host.tiles.size();
+        }
         if (st != DISTDL_OK) {
             delete p;
             return st;
@@ -226,7 +248,7 @@ extern "C" distdl_status_t distdl_selftest_row_plan(const distdl_partition_t *p,
     clear_error();
     if (!p || !header || !records || !num_records) return fail(DISTDL_ERR_INVALID_ARG, "selftest_row_plan: NULL argument");
     if (adjoint ? !p->fast.adj_usable : !p->fast.usable)
-        return fail(DISTDL_ERR_UNSUPPORTED, "selftest_row_plan: this partition has no row plan for %s", adjoint ? "H*" : "H");
+        return fail(DISTDL_ERR_UNSUPPORTED, "selftest_row_plan: this partition has no row plan for %s", adjoint ? "the row ends of H*" : "H");
     const size_t hw = sizeof(FastHeader) / 4, rw = p->fast.dims.size() * (sizeof(FastDim) / 4);
     if ((size_t)header_words < hw || (size_t)record_words < rw)
         return fail(DISTDL_ERR_INVALID_ARG, "selftest_row_plan: need %zu header words and %zu record words", hw, rw);

@@ -309,6 +309,19 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
     Builder fb(p, &p->fwd_host, esize);
     // exterior-ghost clear boxes are shared by the adjoint plan
     Builder ab(p, &p->adj_host, esize);
+    // H* without the part that the row plan takes (p->fast.adj_usable): the row ends -- ghost cells and receiving bulk
+    // cells along the innermost dimension -- of the bulk rows that no neighbour in an outer dimension reaches
+    const bool split_adj = p->fast.adj_usable;
+    Builder rb(p, &p->adj_rest_host, esize);
+    // reach of the low / high neighbour into the bulk of the workers with coordinate c along dimension k
+    auto reach_lo = [&](int k, int32_t c) -> int64_t {
+        const int32_t pk = p->pshape[k];
+        return (c > 0 || p->periodic[k]) ? p->hhi[k][(c + pk - 1) % pk] : 0;
+    };
+    auto reach_hi = [&](int k, int32_t c) -> int64_t {
+        const int32_t pk = p->pshape[k];
+        return (c + 1 < pk || p->periodic[k]) ? p->hlo[k][(c + 1) % pk] : 0;
+    };
     for (int32_t w = 0; w < p->num_workers; ++w) {
         int32_t c[DISTDL_MAX_RANK];
         p->coords(w, c);
@@ -351,6 +364,31 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
             } else {
                 if (!fb.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
                 if (!ab.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
+                if (split_adj) {
+                    bool row_end = delta[d - 1] != 0;
+                    for (int k = 0; k + 1 < d; ++k) row_end = row_end && delta[k] == 0;
+                    if (!row_end) {
+                        if (!rb.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
+                    } else {
+                        // ghosts at the row ends of the bulk rows: only the rows within some outer neighbour's reach stay
+                        // here, as one slab per outer dimension and side (out of reach before it, any bulk index after it)
+                        for (int j = 0; j + 1 < d; ++j) {
+                            for (int side = 0; side < 2; ++side) {
+                                Region r = dst;
+                                const int64_t hl = p->hlo[j][c[j]], b = p->size[j][c[j]];
+                                const int64_t wl = reach_lo(j, c[j]), wh = reach_hi(j, c[j]);
+                                r.start[j] = side == 0 ? hl : hl + b - wh;
+                                r.extent[j] = side == 0 ? wl : wh;
+                                for (int k = 0; k < j; ++k) {
+                                    const int64_t kl = reach_lo(k, c[k]), kh = reach_hi(k, c[k]);
+                                    r.start[k] = p->hlo[k][c[k]] + kl;
+                                    r.extent[k] = p->size[k][c[k]] - kl - kh;
+                                }
+                                if (!rb.add(r, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
+                            }
+                        }
+                    }
+                }
             }
         } while (next_delta(delta, d));
     }
@@ -437,6 +475,10 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
                 if ((int)srcs.size() > kMaxSources)
                     return fail(DISTDL_ERR_UNSUPPORTED, "halo plan: a bulk cell receives from more than %d ghosts", kMaxSources);
                 if (!ab.add(dst, srcs, levels)) return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint box out of range");
+                // the row plan takes the boxes that receive along the innermost dimension only
+                const bool row_end_only = levels == 1 && active[0] == d - 1;
+                if (split_adj && !row_end_only && !rb.add(dst, srcs, levels))
+                    return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint box out of range");
             }
             int k = d - 1;
             for (; k >= 0; --k) {
@@ -447,6 +489,7 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
         }
     }
     if (!ab.destinations_disjoint()) return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint boxes overlap");
+    if (split_adj && !rb.destinations_disjoint()) return fail(DISTDL_ERR_SHAPE, "halo plan: adjoint boxes overlap");
     return DISTDL_OK;
 }
 
@@ -527,13 +570,13 @@ static void magic_of(int64_t e, uint32_t *magic, uint32_t *shift) {
 }
 
 // Deals `total[i]` blocks of kind i out in groups: the rarest kind present gets one block per group.
-static bool fast_groups(const int64_t total[3], FastHeader *h) {
+static bool fast_groups(const int64_t total[2], FastHeader *h) {
     int64_t least = 0;
-    for (int i = 0; i < 3; ++i)
+    for (int i = 0; i < 2; ++i)
         if (total[i] > 0 && (least == 0 || total[i] < least)) least = total[i];
     if (least == 0) return false;
     int64_t groups = 0, per_group = 0;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 2; ++i) {
         h->group[i] = total[i] > 0 ? (int32_t)std::min<int64_t>(64, total[i] / least) : 0;
         if (h->group[i]) groups = std::max(groups, (total[i] + h->group[i] - 1) / h->group[i]);
         per_group += h->group[i];
@@ -568,13 +611,11 @@ void build_fast_plan(distdl_partition *p) {
     }
     int64_t any_ghost = 0;
     bool wide_enough = true;          // every bulk at least as wide as its two neighbours' reach together
-    int dims_with_reach = 0;
     for (int k = 0; k < d; ++k) {
         h.pshape[k] = p->pshape[k];
         h.dim_base[k] = (int32_t)f.dims.size();
         const int64_t unit = k == d - 1 ? per : 1;
         const int32_t pk = p->pshape[k];
-        bool reach = false;
         for (int32_t c = 0; c < pk; ++c) {
             FastDim e;
             memset(&e, 0, sizeof(e));
@@ -594,7 +635,6 @@ void build_fast_plan(distdl_partition *p) {
                 e.rhi = (int32_t)(p->hlo[k][e.hi_c] / unit);
             }
             if (e.rlo + e.rhi > e.b) wide_enough = false;
-            reach = reach || e.rlo + e.rhi > 0;
             uint32_t sn, sb, sg, sbi, srr;
             magic_of(e.n, &e.magic_n, &sn);
             magic_of(e.b, &e.magic_b, &sb);
@@ -604,13 +644,12 @@ void build_fast_plan(distdl_partition *p) {
             e.shifts = sn | (sb << 6) | (sg << 12) | (sbi << 18) | (srr << 24);
             f.dims.push_back(e);
         }
-        if (reach && k < d - 1) ++dims_with_reach;
     }
     h.num_records = (int32_t)f.dims.size();
     h.num_lines = p->num_workers / p->pshape[d - 1];
     if (any_ghost == 0) return;     // nothing to exchange: the box plan (empty) handles it
     // block sizes from the largest worker
-    int64_t nx_max = 1, ghost_rows_max = 0, bulk_rows_max = 0, reach_rows_max = 0, inner_rows_max = 0;
+    int64_t nx_max = 1, ghost_rows_max = 0, bulk_rows_max = 0, inner_rows_max = 0;
     int64_t gc = 0, ec = 0;         // per row of a line: ghost units, and units of the row ends that H* rewrites
     for (int32_t c = 0; c < p->pshape[d - 1]; ++c) {
         const FastDim &e = f.dims[h.dim_base[d - 1] + c];
@@ -630,7 +669,6 @@ void build_fast_plan(distdl_partition *p) {
         }
         ghost_rows_max = std::max(ghost_rows_max, all - bulk);   // rows with a ghost index in some outer dimension
         bulk_rows_max = std::max(bulk_rows_max, bulk);
-        reach_rows_max = std::max(reach_rows_max, bulk - inner);
         inner_rows_max = std::max(inner_rows_max, inner);
     }
     if (ghost_rows_max >= ((int64_t)1 << 31) || bulk_rows_max >= ((int64_t)1 << 31)) return;
@@ -645,26 +683,20 @@ void build_fast_plan(distdl_partition *p) {
         h.tiles_per_owner[1] = tiles(bulk_rows_max, h.rows_per_tile[1]);
     }
     {
-        const int64_t total[3] = {(int64_t)h.tiles_per_owner[0] * p->num_workers, (int64_t)h.tiles_per_owner[1] * h.num_lines, 0};
+        const int64_t total[2] = {(int64_t)h.tiles_per_owner[0] * p->num_workers, (int64_t)h.tiles_per_owner[1] * h.num_lines};
         f.usable = fast_groups(total, &h);
     }
-    // ---- H*: at most two outer dimensions with neighbours (four rows summed into one, eight terms with the row ends)
-    if (!f.usable || !wide_enough || dims_with_reach > 2 || ec > 1024) return;
+    // ---- row ends of H*: every bulk at least as wide as its two neighbours' reach together, some reach along the rows,
+    // and some rows out of every outer neighbour's reach
+    if (!f.usable || !wide_enough || ec == gc || ec > 1024 || inner_rows_max == 0) return;
     FastHeader &a = f.adj_hdr;
     a = h;
     memset(a.rows_per_tile, 0, sizeof(a.rows_per_tile));
     memset(a.tiles_per_owner, 0, sizeof(a.tiles_per_owner));
-    a.rows_per_tile[0] = rows_s;
-    a.tiles_per_owner[0] = tiles(ghost_rows_max, rows_s);
-    if (ec > 0) {
-        a.rows_per_tile[1] = (int32_t)std::min<int64_t>(128, std::max<int64_t>(1, 512 / ec));
-        a.tiles_per_owner[1] = tiles(inner_rows_max, a.rows_per_tile[1]);
-    }
-    a.rows_per_tile[2] = rows_s;
-    a.tiles_per_owner[2] = tiles(reach_rows_max, rows_s);
+    a.rows_per_tile[1] = (int32_t)std::min<int64_t>(128, std::max<int64_t>(1, 512 / ec));
+    a.tiles_per_owner[1] = tiles(inner_rows_max, a.rows_per_tile[1]);
     {
-        const int64_t total[3] = {(int64_t)a.tiles_per_owner[0] * p->num_workers, (int64_t)a.tiles_per_owner[1] * a.num_lines,
-                                  (int64_t)a.tiles_per_owner[2] * p->num_workers};
+        const int64_t total[2] = {0, (int64_t)a.tiles_per_owner[1] * a.num_lines};
         f.adj_usable = fast_groups(total, &a);
     }
 }

@@ -1,10 +1,10 @@
-"""Host-side replay of the row plan of H and H* (CPU, no kernel launched).
+"""Host-side replay of the row plan of H and of the row ends of H* (CPU, no kernel launched).
 
 The row-plan kernels derive every address from one small record per (dimension, worker coordinate).  This test
 fetches those records from the library (include/distdl_selftest.h), replays the kernels' index arithmetic block
-by block in Python -- the same row classes, divisions by multiply-and-shift, neighbour lookups, term lists and
-staging slots -- checks that every unit it touches lies inside its worker's array, that no unit is written
-twice, and that the result equals the oracle's H / H* bit for bit.
+by block in Python -- the same row classes, divisions by multiply-and-shift, neighbour lookups and staging
+slots -- checks that every unit it touches lies inside its worker's array, that the units handled are exactly
+the ones the kernel is responsible for, each once, and that their values equal the oracle's H / H* bit for bit.
 """
 
 import numpy as np
@@ -29,8 +29,8 @@ class Header:
         self.rank, self.nw = h[0], h[1]
         self.pshape, self.base, self.wstride = h[2:7], h[7:12], h[12:17]
         self.nrec, self.nlines = h[17], h[18]
-        self.rows, self.tiles, self.group = h[19:22], h[22:25], h[25:28]
-        self.ngroups = h[28]
+        self.rows, self.tiles, self.group = h[19:21], h[21:23], h[23:25]
+        self.ngroups = h[25]
 
 
 def fdiv(x, magic, shift, e):
@@ -48,9 +48,6 @@ def blocks(H):
         if ing >= H.group[0]:
             ing -= H.group[0]
             kind = 1
-            if ing >= H.group[1]:
-                ing -= H.group[1]
-                kind = 2
         yield kind, group * H.group[kind] + ing
 
 
@@ -62,7 +59,7 @@ def worker(H, dims, w):
     return c, [dims[H.base[k] + c[k]] for k in range(H.rank)]
 
 
-def ghost_rows(H, dims, src, out, written, s, t, clear_only):
+def ghost_rows(H, dims, src, out, written, s, t):
     d = H.rank
     c, e = worker(H, dims, s)
     cls = []
@@ -120,7 +117,7 @@ def ghost_rows(H, dims, src, out, written, s, t, clear_only):
             if zero or ncx < 0:
                 out[s][doff] = 0
                 written[s][doff] += 1
-            elif not clear_only:
+            else:
                 w = outer_w + ncx * H.wstride[d - 1]
                 soff = src_lin * dims[H.base[d - 1] + ncx].n + shift + col
                 assert 0 <= w < H.nw and 0 <= soff < len(src[w])
@@ -155,7 +152,7 @@ def replay_forward(hdr, recs, units):
         if kind == 0:
             s, t = divmod(tile, H.tiles[0])
             if s < H.nw:
-                ghost_rows(H, dims, units, out, written, s, t, False)
+                ghost_rows(H, dims, units, out, written, s, t)
             continue
         assert kind == 1
         line, t = divmod(tile, H.tiles[1])
@@ -216,111 +213,14 @@ def replay_forward(hdr, recs, units):
     return out, written
 
 
-def replay_adjoint(hdr, recs, units, add):
-    """In place, like the kernel: every read sees the value before this operator or a cleared ghost, never a sum."""
+def replay_adjoint_row_ends(hdr, recs, units, add):
+    """The launch that handles the row ends of H*: in place, every unit read once and written once."""
     H, dims = Header(hdr), [Rec(r) for r in recs]
     d = H.rank
     mem = [u.copy() for u in units]
-    touched = [np.zeros(len(u), dtype=np.int32) for u in units]     # reads and writes by the summing threads
-
-    def fold(ptrs):
-        vals = [mem[w][o].copy() for w, o in ptrs]
-        for w, o in ptrs:
-            assert 0 <= w < H.nw and 0 <= o < len(mem[w])
-            touched[w][o] += 1
-        width = 1
-        while width < len(vals):
-            for j in range(0, len(vals), 2 * width):
-                vals[j] = add(vals[j], vals[j + width])
-            width *= 2
-        mem[ptrs[0][0]][ptrs[0][1]] = vals[0]
-        for w, o in ptrs[1:]:
-            mem[w][o] = 0
-
+    touched = [np.zeros(len(u), dtype=np.int32) for u in units]
     for kind, tile in blocks(H):
-        if kind == 0:
-            s, t = divmod(tile, H.tiles[0])
-            if s < H.nw:
-                ghost_rows(H, dims, mem, mem, touched, s, t, True)
-            continue
-        if kind == 2:
-            s, t = divmod(tile, H.tiles[2])
-            if s >= H.nw:
-                continue
-            c, e = worker(H, dims, s)
-            cls = []
-            for j in range(d - 1):
-                r = e[j].rlo + e[j].rhi
-                for k in range(d - 1):
-                    if k != j:
-                        r *= (e[k].b - e[k].rlo - e[k].rhi) if k < j else e[k].b
-                cls.append(r)
-            total, row0 = sum(cls), t * H.rows[2]
-            if row0 >= total:
-                continue
-            nrows = min(H.rows[2], total - row0)
-            ex, nx, cx = e[d - 1], e[d - 1].n, c[d - 1]
-            for rl in range(nrows):
-                idx, j = row0 + rl, 0
-                while j < d - 2 and idx >= cls[j]:
-                    idx -= cls[j]
-                    j += 1
-                shard, lin, pitch = [0], [0], [1]
-                for k in range(d - 2, -1, -1):
-                    f = e[k]
-                    inner, rr = f.b - f.rlo - f.rhi, f.rlo + f.rhi
-                    coord = idx
-                    if k > 0:
-                        if k > j:
-                            ext, q = f.b, fdiv(idx, f.magic_b, f.shift_b, f.b)
-                        elif k == j:
-                            ext, q = rr, fdiv(idx, f.magic_rr, f.shift_rr, rr)
-                        else:
-                            ext, q = inner, fdiv(idx, f.magic_bi, f.shift_bi, inner)
-                        coord, idx = idx - q * ext, q
-                    pos = coord if k > j else ((coord if coord < f.rlo else coord + inner) if k == j else f.rlo + coord)
-                    assert 0 <= pos < f.b
-                    i = f.hlo + pos
-                    nc, si = -1, 0
-                    if pos < f.rlo:
-                        nc, si = f.lo_c, i + f.lo_shift
-                    elif pos >= f.b - f.rhi:
-                        nc, si = f.hi_c, i + f.hi_shift
-                    old = len(shard)
-                    if nc >= 0:
-                        assert old <= 2
-                        npitch = dims[H.base[k] + nc].n
-                        for q in range(old):
-                            shard.append(shard[q] + nc * H.wstride[k])
-                            lin.append(lin[q] + si * pitch[q])
-                            pitch.append(pitch[q] * npitch)
-                    for q in range(old):
-                        shard[q] += c[k] * H.wstride[k]
-                        lin[q] += i * pitch[q]
-                        pitch[q] *= f.n
-                assert len(shard) in (2, 4)
-                for col in range(nx):
-                    if col < ex.hlo or col >= ex.hlo + ex.b:
-                        none = ex.lo_c < 0 if col < ex.hlo else ex.hi_c < 0
-                        if none:
-                            off = lin[0] * nx + col
-                            assert 0 <= off < len(mem[s]) and shard[0] + cx == s
-                            mem[s][off] = 0
-                            touched[s][off] += 1
-                        continue
-                    pos = col - ex.hlo
-                    ncx, shift = -1, 0
-                    if pos < ex.rlo:
-                        ncx, shift = ex.lo_c, ex.lo_shift
-                    elif pos >= ex.b - ex.rhi:
-                        ncx, shift = ex.hi_c, ex.hi_shift
-                    ptrs = []
-                    for q in range(len(shard)):
-                        ptrs.append((shard[q] + cx, lin[q] * nx + col))
-                        if ncx >= 0:
-                            ptrs.append((shard[q] + ncx, lin[q] * dims[H.base[d - 1] + ncx].n + col + shift))
-                    fold(ptrs)
-            continue
+        assert kind == 1
         line, t = divmod(tile, H.tiles[1])
         if line >= H.nlines:
             continue
@@ -332,6 +232,7 @@ def replay_adjoint(hdr, recs, units, add):
         if row0 >= total:
             continue
         nrows = min(H.rows[1], total - row0)
+        assert nrows <= 128
         xd = dims[H.base[d - 1]:H.base[d - 1] + px]
         cum_e = [0]
         for a in range(px):
@@ -432,31 +333,56 @@ def test_row_plan_replay_of_the_forward_kernel_matches_the_oracle(case):
         assert np.array_equal(written[k], ghost.reshape(-1, per_unit).all(axis=1).astype(np.int32))
 
 
+def _row_end_units(opart, k, per_unit):
+    """The 16-byte units of worker k that the row-end launch of H* owns: in the bulk rows out of every outer
+    neighbour's reach, the ghost units at both ends and the bulk units within reach of the neighbours along the row."""
+    rank = opart.rank
+    c = opart.coords(k)
+    lo, hi = opart.widths(k)
+    b = opart.bulk_shape(k)
+
+    def reach(dim):
+        p, per = opart.pshape[dim], opart.periodic[dim]
+        rl = opart.hhi[dim][(c[dim] - 1) % p] if (c[dim] > 0 or per) else 0
+        rh = opart.hlo[dim][(c[dim] + 1) % p] if (c[dim] + 1 < p or per) else 0
+        return rl, rh
+    mask = np.zeros(opart.padded_shape(k), dtype=bool)
+    rows = tuple(slice(lo[dim] + reach(dim)[0], lo[dim] + b[dim] - reach(dim)[1]) for dim in range(rank - 1))
+    rl, rh = reach(rank - 1)
+    x = rank - 1
+    mask[rows + (slice(0, lo[x] + rl),)] = True
+    mask[rows + (slice(lo[x] + b[x] - rh, lo[x] + b[x] + hi[x]),)] = True
+    return mask.reshape(-1, per_unit).all(axis=1)
+
+
 @pytest.mark.parametrize("case", CASES, ids=[str(c[0]) + str(c[1]) for c in CASES])
-def test_row_plan_replay_of_the_adjoint_kernel_matches_the_oracle(case):
+def test_row_plan_replay_of_the_row_ends_of_the_adjoint_matches_the_oracle(case):
     opart, gpart, x, per_unit = _make(case)
-    if case[0] == (9, 7, 64):
-        # a bulk of 2 cells whose neighbours reach 1 and 2 cells into it: the box plan runs H*
+    if case[0] in ((9, 7, 64), (12, 16), (64, 48), (6, 10, 48)):
+        # a bulk of 2 cells whose neighbours reach 1 and 2 cells into it; one worker along the rows; no ghosts along
+        # the rows; no row out of reach of the (periodic) neighbours in dimension 0: the box plan does all of H*
         assert not gpart.uses_row_plan(adjoint=True)
         return
     assert gpart.uses_row_plan(adjoint=True)
     hdr, recs = distdl.selftest_row_plan(gpart, adjoint=True)
+    assert Header(hdr).group[0] == 0
     if case[5] == np.uint16:
         add = lambda a, b: oracle.bf16_add(a, b)
         ref = oracle.halo_adj_sequence(opart, x, add=oracle.bf16_add)
     else:
         add = lambda a, b: a + b
         ref = oracle.halo_adj_sequence(opart, x)
-    got, touched = replay_adjoint(hdr, recs, [a.reshape(-1, per_unit) for a in x], add)
+    got, touched = replay_adjoint_row_ends(hdr, recs, [a.reshape(-1, per_unit) for a in x], add)
     for k in range(opart.num_workers):
-        assert got[k].reshape(x[k].shape).tobytes() == ref[k].tobytes(), "worker %d" % k
-        assert touched[k].max() <= 1                     # no unit is handled by two threads
+        own = _row_end_units(opart, k, per_unit)
+        assert np.array_equal(touched[k], own.astype(np.int32)), "worker %d: units handled" % k
+        want = ref[k].reshape(-1, per_unit)
+        assert got[k][own].tobytes() == want[own].tobytes(), "worker %d: values" % k
+        assert got[k][~own].tobytes() == x[k].reshape(-1, per_unit)[~own].tobytes()      # nothing else is touched
 
 
 def test_geometries_outside_the_row_plan():
     for gs, ps, lo, hi in [((11,), (3,), (2,), (2,)), ((67, 61, 68), (3, 2, 2), (2, 4, 4), (3, 4, 4)), ((256, 256), (2, 2), (1, 1), (1, 1))]:
         assert not distdl.Partition(gs, ps, lo, hi).uses_row_plan()
-    thin = distdl.Partition((6, 16), (3, 1), (2, 4), (2, 4))      # the middle worker's bulk is thinner than the two reaches
+    thin = distdl.Partition((6, 32), (3, 2), (2, 4), (2, 4))      # the middle worker's bulk is thinner than the two reaches
     assert thin.uses_row_plan() and not thin.uses_row_plan(adjoint=True)
-    many = distdl.Partition((4, 4, 4, 8), (2, 2, 2, 2), (1, 1, 1, 4), (1, 1, 1, 4))   # neighbours in three outer dimensions
-    assert many.uses_row_plan() and not many.uses_row_plan(adjoint=True)
