@@ -960,16 +960,17 @@ def main():
 
 
 # DRAM bytes (read + write) per launch from the committed ncu summaries under profiles/ (one launch of
-# `bench.py --profile-op <op>`; full size where the summary says so, else the quarter-size case scaled
-# by 4: traffic grows with the number of planes / rows); None for a kernel whose counters were not
-# meaningful or that changed since its counters were taken.
+# `bench.py --profile-op <op>`: full size for H, H*, the affine layer and -- with --profile-full and the two DRAM
+# byte counters alone -- the convolution; the quarter-size case scaled by 4 for R, whose traffic grows with the
+# number of rows); None for a kernel whose counters were not meaningful (the broadcast's output was still in L2
+# when the short capture ended) or that changed since its counters were taken.
 NCU_TRAFFIC = {
     "broadcast_fwd": None,
     "sumreduce_fwd": 4 * (134225152 + 5290496),
-    "halo_fwd": None,
-    "halo_adj": None,
-    "conv_fwd": 4 * (278041088 + 221260288),
-    "conv_adj": 4 * (269701888 + 228404480),
+    "halo_fwd": 194266368 + 124569856,
+    "halo_adj": (107870464 + 72062976) + (139435264 + 39406592),      # box kernel + row-end kernel
+    "conv_fwd": 1173479680 + 1030533632,
+    "conv_adj": 1178607872 + 1071105024,
     "affine_fwd": 138435072 + 3728128,
     "affine_adj": 138447104 + 3240448,
 }

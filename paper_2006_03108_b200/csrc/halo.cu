@@ -446,7 +446,7 @@ __device__ __forceinline__ void fast_ghost_rows(const FastHeader &H, const FastD
     const uint32_t count = nrows * nx;
     const uint32_t xlo = (uint32_t)ex->hlo, xhi = (uint32_t)(ex->hlo + ex->b);
     const uint32_t shx = fast_shift_n(*ex);
-    constexpr int U = 4;
+    constexpr int U = 8;
     for (uint32_t base = threadIdx.x; base < count; base += kFastThreads * U) {
         uint4 v[U];
         uint32_t doff[U];

@@ -673,7 +673,7 @@ void build_fast_plan(distdl_partition *p) {
     }
     if (ghost_rows_max >= ((int64_t)1 << 31) || bulk_rows_max >= ((int64_t)1 << 31)) return;
     if (gc > 1024) return;          // staging of one row's ghost units for all workers of a line: 16 KB at most
-    const int32_t rows_s = (int32_t)std::min<int64_t>(256, std::max<int64_t>(1, 2048 / nx_max));
+    const int32_t rows_s = (int32_t)std::min<int64_t>(256, std::max<int64_t>(1, 4096 / nx_max));
     auto tiles = [](int64_t rows, int32_t per_tile) { return (int32_t)((rows + per_tile - 1) / per_tile); };
     // ---- H
     h.rows_per_tile[0] = rows_s;
