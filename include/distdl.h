@@ -113,9 +113,9 @@ distdl_status_t distdl_partition_shard_extents(const distdl_partition_t *p, int3
 distdl_status_t distdl_partition_halo_stats(const distdl_partition_t *p, int32_t adjoint,
                                             int64_t *boxes, int64_t *tiles, int64_t *bytes);
 
-/* Halo widths of a 1-D sliding kernel (Section 3: "determined by the minimum and maximum global
- * indices of the worker's output tensor and the size, stride, dilation, and padding parameters of
- * the kernel"; worked cases: Figs. B1-B4).  Input length n and the output length
+/* Halo widths of a 1-D sliding kernel (Section 3, "Halo exchange": the widths follow from the first
+ * and the last input index that a worker's own outputs touch, hence from the kernel's size, stride,
+ * dilation and padding; worked cases: Figs. B1-B4).  Input length n and the output length
  * floor((n + pad_lo + pad_hi - dilation*(kernel-1) - 1)/stride) + 1 are both split evenly over p
  * workers.  Host only.  Each output array has p entries and may be NULL: halo widths, and the
  * count of owned inputs at either end that the worker's outputs never read. */

@@ -354,8 +354,9 @@ def affine_fwd(x_parts, w_parts, pfo, pfi, bias_parts=None):
 
     x_parts[j]   (n_b, n_fi/P_fi) fp64 values, j = 0..P_fi-1 (partition 1 x P_fi)
     w_parts[i*P_fi + j]  (n_fo/P_fo, n_fi/P_fi), worker (i, j) in row-major order
-    bias_parts[i]  (n_fo/P_fo,) or None; lives on grid column j = 0 only (the
-                 "one P_fo x 1 subset", cf. Table C1: workers 0 and 2 of a 2 x 2)
+    bias_parts[i]  (n_fo/P_fo,) or None; lives on grid column j = 0 only (Section 4,
+                 "Dense layers": the bias sits on a single column of the grid so that it is
+                 counted once; cf. Table C1: workers 0 and 2 of a 2 x 2)
     Steps: x^_{ij} <- B x_j;  y^_{ij} <- Affine(w_{ij}, b_{ij}; x^_{ij});
            y_i <- R over j = 0..P_fi-1 in order.
     Local contraction in fp64; the fold over j is done in fp64 as well and the

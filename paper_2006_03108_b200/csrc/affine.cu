@@ -961,7 +961,10 @@ static distdl_status_t affine_impl(int64_t nb, int64_t nfi, int64_t nfo, int32_t
     static bool configured_on[kMaxDevicesPerProcess] = {false};
     int cur_dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
-    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    if (cur_dev < 0 || cur_dev >= kMaxDevicesPerProcess)
+        return fail(DISTDL_ERR_UNSUPPORTED, "device index %d: at most %d devices per process", cur_dev, kMaxDevicesPerProcess);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());      // first calls from several threads set up once
+    bool &configured = configured_on[cur_dev];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                AffineCfg<false>::SMEM_BYTES));
@@ -1075,9 +1078,12 @@ static distdl_status_t affine_params_impl(int64_t nb, int64_t nfi, int64_t nfo, 
     static bool configured_on[kMaxDevicesPerProcess] = {false};
     int cur_dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
-    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    if (cur_dev < 0 || cur_dev >= kMaxDevicesPerProcess)
+        return fail(DISTDL_ERR_UNSUPPORTED, "device index %d: at most %d devices per process", cur_dev, kMaxDevicesPerProcess);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());      // first calls from several threads set up once
+    bool &configured = configured_on[cur_dev];
     static int sms_on[kMaxDevicesPerProcess] = {0};
-    int &sms = sms_on[cur_dev % kMaxDevicesPerProcess];
+    int &sms = sms_on[cur_dev];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(affine_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemBytes));
         int dev = 0;

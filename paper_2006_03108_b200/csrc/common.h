@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -24,6 +25,7 @@ void clear_error();
     } while (0)
 
 constexpr int kMaxDevicesPerProcess = 64;   // per-device one-time set-up flags are kept for this many devices
+std::mutex &setup_mutex();                  // guards the one-time, per-device set-up of the operator entry points
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int elem_size(distdl_dtype_t t) { return t == DISTDL_F32 ? 4 : (t == DISTDL_F64 ? 8 : 2); }
@@ -226,7 +228,7 @@ distdl_status_t upload_plan_pair(const HaloPlanHost &a, const HaloPlanHost &b, H
                                  void **block, int *device, const char *what, const void *extra = nullptr,
                                  size_t extra_bytes = 0, void **extra_dev = nullptr);
 // Builds the forward (H) and adjoint (H*) box/tile lists of a partition (host only).
-distdl_status_t build_halo_plans(distdl_partition *p);
+distdl_status_t build_halo_plans(distdl_partition *p, bool forward_only = false);
 // Fills p->fast (row plan) where the geometry allows it.
 void build_fast_plan(distdl_partition *p);
 // Geometry and halo plans only, no device memory.

@@ -716,9 +716,12 @@ static distdl_status_t launch_conv(const ConvParams &P, int total_tiles, int til
     static bool configured_on[kMaxDevicesPerProcess] = {false};
     int cur_dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
-    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    if (cur_dev < 0 || cur_dev >= kMaxDevicesPerProcess)
+        return fail(DISTDL_ERR_UNSUPPORTED, "device index %d: at most %d devices per process", cur_dev, kMaxDevicesPerProcess);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());      // first calls from several threads set up once
+    bool &configured = configured_on[cur_dev];
     static int blocks_on[kMaxDevicesPerProcess] = {0};
-    int &blocks = blocks_on[cur_dev % kMaxDevicesPerProcess];
+    int &blocks = blocks_on[cur_dev];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_depthwise_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         int dev = 0, sms = 0, per_sm = 0;
@@ -756,9 +759,12 @@ static distdl_status_t launch_conv_tma(const distdl_partition *p, ConvTmaParams 
     static bool configured_on[kMaxDevicesPerProcess] = {false};
     int cur_dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
-    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    if (cur_dev < 0 || cur_dev >= kMaxDevicesPerProcess)
+        return fail(DISTDL_ERR_UNSUPPORTED, "device index %d: at most %d devices per process", cur_dev, kMaxDevicesPerProcess);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());      // first calls from several threads set up once
+    bool &configured = configured_on[cur_dev];
     static int blocks_on[kMaxDevicesPerProcess] = {0};
-    int &blocks = blocks_on[cur_dev % kMaxDevicesPerProcess];
+    int &blocks = blocks_on[cur_dev];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_tma_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES));
         int dev = 0, sms = 0, per_sm = 0;
@@ -1207,9 +1213,12 @@ static distdl_status_t launch_convg(const ConvGParams &G, int in_shards, const i
     static bool configured_on[kMaxDevicesPerProcess] = {false};
     int cur_dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
-    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    if (cur_dev < 0 || cur_dev >= kMaxDevicesPerProcess)
+        return fail(DISTDL_ERR_UNSUPPORTED, "device index %d: at most %d devices per process", cur_dev, kMaxDevicesPerProcess);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());      // first calls from several threads set up once
+    bool &configured = configured_on[cur_dev];
     static int blocks_plain_on[kMaxDevicesPerProcess] = {0}, blocks_tma_on[kMaxDevicesPerProcess] = {0};
-    int &blocks_plain = blocks_plain_on[cur_dev % kMaxDevicesPerProcess], &blocks_tma = blocks_tma_on[cur_dev % kMaxDevicesPerProcess];
+    int &blocks_plain = blocks_plain_on[cur_dev], &blocks_tma = blocks_tma_on[cur_dev];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_plain));
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(convg_tma_kernel<K, ADJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_tma));
@@ -1795,9 +1804,12 @@ static distdl_status_t grad_config(int *blocks_out) {
     static bool configured_on[kMaxDevicesPerProcess] = {false};
     int cur_dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&cur_dev));
-    bool &configured = configured_on[cur_dev % kMaxDevicesPerProcess];
+    if (cur_dev < 0 || cur_dev >= kMaxDevicesPerProcess)
+        return fail(DISTDL_ERR_UNSUPPORTED, "device index %d: at most %d devices per process", cur_dev, kMaxDevicesPerProcess);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());      // first calls from several threads set up once
+    bool &configured = configured_on[cur_dev];
     static int blocks_on[kMaxDevicesPerProcess] = {0};
-    int &blocks = blocks_on[cur_dev % kMaxDevicesPerProcess];
+    int &blocks = blocks_on[cur_dev];
     if (!configured) {
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(false)));
         DISTDL_CUDA_CHECK(cudaFuncSetAttribute(conv_grad_tma_kernel<K, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem_bytes<K>(true)));

@@ -767,6 +767,7 @@ static distdl_status_t static_plan_address(unsigned char **out) {
     int dev = 0;
     DISTDL_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return fail(DISTDL_ERR_UNSUPPORTED, "halo_fwd_noalloc: device index %d", dev);
+    std::lock_guard<std::mutex> setup_lock(setup_mutex());
     if (!cached[dev]) {
         void *ptr = nullptr;
         DISTDL_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_static_plan));

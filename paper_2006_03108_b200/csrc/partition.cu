@@ -122,8 +122,8 @@ static distdl_status_t create_impl(int32_t rank, const int64_t *global_shape, co
             delete p;
             return fail(DISTDL_ERR_UNSUPPORTED, "partition_create: shard too large");
         }
-    build_fast_plan(p);
-    distdl_status_t st = build_halo_plans(p);
+    if (upload) build_fast_plan(p);
+    distdl_status_t st = build_halo_plans(p, !upload);      // without an upload (the entry point that allocates nothing) only H is planned
     if (st != DISTDL_OK) {
         delete p;
         return st;

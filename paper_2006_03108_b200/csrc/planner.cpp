@@ -23,6 +23,11 @@ distdl_status_t fail(distdl_status_t code, const char *fmt, ...) {
 }
 void clear_error() { g_error[0] = 0; }
 
+std::mutex &setup_mutex() {
+    static std::mutex m;
+    return m;
+}
+
 }  // namespace distdl
 
 extern "C" const char *distdl_last_error(void) { return distdl::g_error; }
@@ -301,7 +306,7 @@ inline bool next_delta(int *delta, int d) {
 
 namespace distdl {
 
-distdl_status_t build_halo_plans(distdl_partition *p) {
+distdl_status_t build_halo_plans(distdl_partition *p, bool forward_only) {
     const int d = p->rank;
     const int esize = elem_size(p->dtype);
 
@@ -311,7 +316,7 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
     Builder ab(p, &p->adj_host, esize);
     // H* without the part that the row plan takes (p->fast.adj_usable): the row ends -- ghost cells and receiving bulk
     // cells along the innermost dimension -- of the bulk rows that no neighbour in an outer dimension reaches
-    const bool split_adj = p->fast.adj_usable;
+    const bool split_adj = p->fast.adj_usable && !forward_only;
     Builder rb(p, &p->adj_rest_host, esize);
     // reach of the low / high neighbour into the bulk of the workers with coordinate c along dimension k
     auto reach_lo = [&](int k, int32_t c) -> int64_t {
@@ -363,6 +368,7 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
                 if (!fb.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: forward box out of range");
             } else {
                 if (!fb.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
+                if (forward_only) continue;
                 if (!ab.add(dst, srcs, 1)) return fail(DISTDL_ERR_SHAPE, "halo plan: clear box out of range");
                 if (split_adj) {
                     bool row_end = delta[d - 1] != 0;
@@ -392,6 +398,9 @@ distdl_status_t build_halo_plans(distdl_partition *p) {
             }
         } while (next_delta(delta, d));
     }
+    // The forward-only form serves the entry point that builds its plan at every call: the pairwise check of the
+    // destination boxes (quadratic in their number) is left to partition_create, which builds the same boxes.
+    if (forward_only) return DISTDL_OK;
     if (!fb.destinations_disjoint()) return fail(DISTDL_ERR_SHAPE, "halo plan: forward boxes overlap");
 
     // ---------------- adjoint: receiving bulk boxes with their nested sources ----------------

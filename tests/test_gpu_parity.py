@@ -492,11 +492,17 @@ def test_conv_fwd_and_adj(case):
     torch.cuda.synchronize()
     ref = oracle.conv_fwd(opart, x, w, bias)
     bound = _abs_bound(opart, x, w)
-    # K*K FMA roundings, one add of the kernel's two partial sums, the oracle's own rounding to fp32
-    eps = (k * k + 2) * 2.0 ** -24
+    # First-order worst case: K*K FMA roundings, one add of the kernel's two partial sums, the oracle's own rounding
+    # to fp32: (K*K + 2) * 2^-24 relative to sum |w||x|.  Asserted: the smaller of that and 1e-6, the relative error
+    # the operator is specified to (the largest ratio seen over these cases is 2.6e-7 forward, 2.0e-7 adjoint).
+    eps = min((k * k + 2) * 2.0 ** -24, 1e-6)
+    worst_fwd = 0.0
     for wk in range(opart.num_workers):
         got = host(ys[wk])
-        assert np.all(np.abs(got.astype(np.float64) - ref[wk]) <= eps * (bound[wk] + np.abs(bias)[None, :, None, None]) + 1e-30)
+        scale = bound[wk] + np.abs(bias)[None, :, None, None]
+        err = np.abs(got.astype(np.float64) - ref[wk])
+        assert np.all(err <= eps * scale + 1e-30)
+        worst_fwd = max(worst_fwd, float(np.max(err / (scale + 1e-30))))
         assert same_bits(host(xs[wk]), x[wk])            # x, ghosts included, is left untouched
     num = np.sqrt(sum(float(np.sum((host(a).astype(np.float64) - b) ** 2)) for a, b in zip(ys, ref)))
     den = np.sqrt(sum(float(np.sum(b.astype(np.float64) ** 2)) for b in ref))
@@ -511,9 +517,12 @@ def test_conv_fwd_and_adj(case):
     torch.cuda.synchronize()
     refa = oracle.conv_adj(opart, dy, w)
     bounda = oracle.conv_adj(opart, [np.abs(a) for a in dy], np.abs(w))
+    worst_adj = 0.0
     for wk in range(opart.num_workers):
         got = host(dxs[wk])
-        assert np.all(np.abs(got.astype(np.float64) - refa[wk]) <= eps * bounda[wk] + 1e-30)
+        err = np.abs(got.astype(np.float64) - refa[wk])
+        assert np.all(err <= eps * bounda[wk] + 1e-30)
+        worst_adj = max(worst_adj, float(np.max(err / (bounda[wk] + 1e-30))))
         mask = np.ones(opart.padded_shape(wk), dtype=bool)
         mask[opart.bulk_slices(wk)] = False
         assert not got[mask].any()                       # ghosts of dx are zero, as H* leaves them
@@ -524,6 +533,9 @@ def test_conv_fwd_and_adj(case):
     xb = oracle.scatter_global(opart, xg)                # zero ghosts: the inner product is over the bulk
     r = oracle.adjoint_test_ratio([host(t) for t in y0], dy, xb, [host(t) for t in dxs])
     assert r < 1e-5
+    # achieved figures, next to the bounds above (shown with pytest -s / -rP)
+    print("conv %s: max |err| / sum|w||x| forward %.3g, adjoint %.3g (bound %.3g); 2-norm forward %.3g; dot test %.3g"
+          % (case, worst_fwd, worst_adj, eps, num / den, r))
 
 
 @pytest.mark.parametrize("case", CONV_CASES, ids=[str(c) for c in CONV_CASES])
@@ -734,9 +746,12 @@ def test_stencil3d_fwd_and_adj(case):
     torch.cuda.synchronize()
     refa = oracle.stencil3d_adj(opart, dy, w)
     bounda = oracle.stencil3d_adj(opart, [np.abs(a) for a in dy], np.abs(w))
+    worst_adj = 0.0
     for wk in range(opart.num_workers):
         got = host(dxs[wk])
-        assert np.all(np.abs(got.astype(np.float64) - refa[wk]) <= eps * bounda[wk] + 1e-30)
+        err = np.abs(got.astype(np.float64) - refa[wk])
+        assert np.all(err <= eps * bounda[wk] + 1e-30)
+        worst_adj = max(worst_adj, float(np.max(err / (bounda[wk] + 1e-30))))
         mask = np.ones(opart.padded_shape(wk), dtype=bool)
         mask[opart.bulk_slices(wk)] = False
         assert not got[mask].any()                       # ghosts of dx are zero, as H* leaves them
