@@ -117,6 +117,61 @@ def test_halo_on_shards_just_below_2_to_31_elements():
     check(distdl.halo_adj, oracle.halo_adj_sequence, 2211, True)
 
 
+def test_halo_row_plan_on_shards_just_below_2_to_31_elements():
+    """The row plan at its largest: two padded shards of 32760 x 65544 cells (2,147,221,440 each; unit offsets up to
+    2^29, byte offsets above 2^33) side by side along the rows, ghost width 4 along the rows and 2 across them.  Ghost
+    rows and the row ends next to the tensor's boundary must come out zero, the row ends at the interface must hold
+    the neighbour's bulk columns (H) or be added into them (H*), the rest of the bulk must be untouched; windows of
+    rows at the top, around cell 2^31 / 2 and at the bottom are also compared with the oracle run on those rows."""
+    _need_free_gb(45)
+    R, C, hr, hc = 32760, 65544, 2, 4
+    gs, ps = (R - 2 * hr, 2 * (C - 2 * hc)), (1, 2)
+    gpart = distdl.Partition(gs, ps, (hr, hc), (hr, hc))
+    assert gpart.uses_row_plan() and gpart.uses_row_plan(adjoint=True)
+    windows = [2, 16380, R - 5]                      # first bulk row of each three-row window
+    mini = oracle.Partition((3, gs[1]), ps, (hr, hc), (hr, hc))
+
+    def window(t, r0):                                # three bulk rows with two rows of (zero) ghost above and below
+        out = np.zeros((7, C), dtype=np.float32)
+        out[2:5] = host(t[r0:r0 + 3])
+        return out
+
+    for adjoint, seed in ((False, 2301), (True, 2311)):
+        x = [_long_vector(R * C, seed + w).view(R, C) for w in range(2)]
+        before = [[window(x[w], r0) for w in range(2)] for r0 in windows]
+        if adjoint:
+            distdl.halo_adj(gpart, x)
+        else:
+            distdl.halo_fwd(gpart, x)
+        torch.cuda.synchronize()
+        for r0, small in zip(windows, before):
+            ref = (oracle.halo_adj_sequence if adjoint else oracle.halo_fwd_sequence)(mini, small)
+            for w in range(2):
+                assert host(x[w][r0:r0 + 3]).tobytes() == ref[w][2:5].tobytes(), "window at row %d, worker %d" % (r0, w)
+        for w in range(2):
+            keep = _long_vector(R * C, seed + w).view(R, C)
+            # ghost rows, and the row ends on the tensor's boundary
+            assert not x[w][:hr].any() and not x[w][R - hr:].any()
+            assert not (x[w][:, :hc] if w == 0 else x[w][:, C - hc:]).any()
+            inner = (slice(hr, R - hr), slice(2 * hc, C - 2 * hc))       # bulk cells away from both row ends
+            assert torch.equal(x[w][inner].view(torch.int32), keep[inner].view(torch.int32))
+            other = _long_vector(R * C, seed + 1 - w).view(R, C)
+            rows = slice(hr, R - hr)
+            mine = (slice(C - hc, C) if w == 0 else slice(0, hc))        # this worker's ghost columns at the interface
+            theirs = (slice(hc, 2 * hc) if w == 0 else slice(C - 2 * hc, C - hc))   # the neighbour's bulk columns they mirror
+            if adjoint:
+                assert not x[w][rows, mine].any()
+                recv = (slice(C - 2 * hc, C - hc) if w == 0 else slice(hc, 2 * hc))      # own bulk columns that receive
+                from_ghost = (slice(0, hc) if w == 0 else slice(C - hc, C))              # the neighbour's ghost columns
+                assert torch.equal(x[w][rows, recv], keep[rows, recv] + other[rows, from_ghost])
+            else:
+                assert torch.equal(x[w][rows, mine].view(torch.int32), other[rows, theirs].view(torch.int32))
+                edge = (slice(C - 2 * hc, C - hc) if w == 0 else slice(hc, 2 * hc))
+                assert torch.equal(x[w][rows, edge].view(torch.int32), keep[rows, edge].view(torch.int32))
+            del keep, other
+        del x
+
+
 def test_halo_3d_full_size():
     gs, ps, h = (512,) * 3, (4,) * 3, 4
     opart = oracle.Partition(gs, ps, h, h)
