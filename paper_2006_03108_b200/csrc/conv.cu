@@ -140,6 +140,15 @@ __device__ __forceinline__ ConvTile decode_tile(const ConvParams &P, int tile, i
     return t;
 }
 
+// Tile that a persistent block takes in turn `it` when its strided walk has reached id `walk`.  With an even grid a
+// block would see only even or only odd ids, i.e. only left or only right tiles of a two-tile-wide shard, and the
+// adjoint's extra pass over the last padded columns would always fall to the same blocks (and, with blocks dealt out
+// to the SMs in order, to the same SMs).  In odd turns the two blocks of a pair of neighbouring ids swap their tiles.
+__device__ __forceinline__ int conv_walk_tile(int walk, int it, int total) {
+    if ((gridDim.x & 1u) == 0 && (it & 1) && (walk ^ 1) < total) return walk ^ 1;
+    return walk;
+}
+
 // K: kernel extent (odd).  ADJ: false = forward (padded x -> bulk-shaped y), true = adjoint
 // (bulk-shaped dy -> padded dx, rotated kernel, ghosts of dx cleared).
 //
@@ -238,7 +247,8 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
 // sets of partial sums are added once at the end.
 // wk2: K*K weights as (w, w) pairs (already rotated for the adjoint), then the bias.
 template <int K, bool ADJ>
-__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile, const float *wk2) {
+__device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile &t, const float *tile, const float *wk2,
+                                             int extra_warp = 0) {
     using C = ConvCfg<K, ADJ>;
     if (!t.valid) return;
     const float b0 = ADJ ? 0.f : wk2[2 * K * K];
@@ -261,10 +271,11 @@ __device__ __forceinline__ void compute_tile(const ConvParams &P, const ConvTile
                 for (int q = c0 + threadIdx.x; q < c1; q += kConvThreads) oplane[(t.bh + C::PH + r) * pitch_o + q] = 0.f;
         if (last_tile_x) {
             // padded columns bw .. bw + 2 PH - 1: the outputs bw - PH .. bw - 1, then the right ghost.
-            // One thread per tile row (a single warp), so the other warps go straight to the main pass.
+            // One thread per tile row (a single warp, extra_warp: the caller rotates it from tile to tile so that the
+            // four schedulers of an SM share this work), so the other warps go straight to the main pass.
             const int out_rows = min(kTileH, t.bh - t.i0);
-            if ((int)threadIdx.x < out_rows) {
-                const int row = threadIdx.x;
+            if ((int)(threadIdx.x >> 5) == extra_warp && (int)(threadIdx.x & 31) < out_rows) {
+                const int row = threadIdx.x & 31;
                 const int first = t.bw - 2 * C::PH - (t.j0 - C::PADL);     // tile column of the window's first input
                 float acc[C::PH];
 #pragma unroll
@@ -447,15 +458,17 @@ conv_depthwise_kernel(const __grid_constant__ ConvParams P, int total_tiles, int
     int buf = 0;
     int tile = blockIdx.x;
     if (tile >= total_tiles) return;
-    ConvTile cur = decode_tile(P, tile, tiles_y, planes);
+    int turn = 0;
+    ConvTile cur = decode_tile(P, conv_walk_tile(tile, turn, total_tiles), tiles_y, planes);
     stage_tile<K, ADJ>(P, cur, smem);
     cp_async_commit();
     while (true) {
         const int next = tile + gridDim.x;
         const bool has_next = next < total_tiles;
         ConvTile nxt = cur;
+        ++turn;
         if (has_next) {
-            nxt = decode_tile(P, next, tiles_y, planes);
+            nxt = decode_tile(P, conv_walk_tile(next, turn, total_tiles), tiles_y, planes);
             stage_tile<K, ADJ>(P, nxt, smem + (buf ^ 1) * C::TILE_FLOATS);
         }
         cp_async_commit();
@@ -639,15 +652,17 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
     if (tile >= Q.total_tiles) return;
     int buf = 0;
     uint32_t phase0 = 0, phase1 = 0;          // parity of the next completion of each buffer's barrier
-    ConvTile cur = decode_tile(Q.base, tile, Q.tiles_y, Q.planes);
+    int turn = 0;
+    ConvTile cur = decode_tile(Q.base, conv_walk_tile(tile, turn, Q.total_tiles), Q.tiles_y, Q.planes);
     stage_tile_tma<K, ADJ>(Q, cur, tiles, sides, wks, bars);
     cp_async_commit();
     while (true) {
         const int next = tile + gridDim.x;
         const bool has_next = next < Q.total_tiles;
         ConvTile nxt = cur;
+        ++turn;
         if (has_next) {
-            nxt = decode_tile(Q.base, next, Q.tiles_y, Q.planes);
+            nxt = decode_tile(Q.base, conv_walk_tile(next, turn, Q.total_tiles), Q.tiles_y, Q.planes);
             stage_tile_tma<K, ADJ>(Q, nxt, tiles + (buf ^ 1) * T::TILE_STRIDE, sides + (buf ^ 1) * T::SIDE_STRIDE,
                                    wks + (buf ^ 1) * T::WK_STRIDE, bars + 8 * (buf ^ 1));
         }
@@ -684,7 +699,7 @@ conv_tma_kernel(const __grid_constant__ ConvTmaParams Q) {
             fill_weight_pairs<K, ADJ>(wraw + 64, wraw, wraw[K * K]);
         }
         __syncthreads();
-        compute_tile<K, ADJ>(Q.base, cur, tl, wraw + 64);
+        compute_tile<K, ADJ>(Q.base, cur, tl, wraw + 64, (turn >> 1) & 3);
         __syncthreads();
         if (!has_next) break;
         cur = nxt;
