@@ -467,16 +467,21 @@ class Workload:
         """One step through the public calls with host buffers on both ends: the inputs of every operator come
         from pinned host memory and its results go back to it.  Three streams: uploads, the operators, downloads;
         the upload of the next operator's inputs and the download of the previous one's results run while an
-        operator computes, so both directions of the host link are busy.  A step starts its uploads only when
-        the previous step's downloads are done (some buffers are input and output at once)."""
+        operator computes, so both directions of the host link are busy.  The upload of an operator's inputs waits
+        for the previous step's download of the same operator's results (some buffers are input and output at
+        once) and for the previous step's last operator (the convolution weights are read by two of them), not for
+        the whole previous step, so the uploads of a step overlap the downloads of the one before."""
         torch = self.torch
         main = torch.cuda.current_stream()
-        if self.e2e_done is not None:
-            self.s_in.wait_event(self.e2e_done)
-        else:
+        if self.e2e_done is None:
             self.s_in.wait_stream(main)
-        for ins, outs, op in self.e2e_ops:
+            self.e2e_down = [None] * len(self.e2e_ops)
+        else:
+            self.s_in.wait_event(self.e2e_ran)
+        for k, (ins, outs, op) in enumerate(self.e2e_ops):
             with torch.cuda.stream(self.s_in):
+                if self.e2e_down[k] is not None:
+                    self.s_in.wait_event(self.e2e_down[k])
                 for t, h in ins:
                     t.copy_(h, non_blocking=True)
                 up = torch.cuda.Event()
@@ -489,8 +494,11 @@ class Workload:
                 self.s_out.wait_event(ran)
                 for t, h in outs:
                     h.copy_(t, non_blocking=True)
-        self.e2e_done = torch.cuda.Event()
-        self.e2e_done.record(self.s_out)
+                down = torch.cuda.Event()
+                down.record()
+            self.e2e_down[k] = down
+        self.e2e_ran = ran
+        self.e2e_done = down
         main.wait_event(self.e2e_done)      # the step is over when its last result has reached the host
 
 
@@ -722,7 +730,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra-ops", action="store_true")
     ap.add_argument("--profile-op", default=None,
