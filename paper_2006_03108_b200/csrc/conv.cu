@@ -101,6 +101,10 @@ __device__ __forceinline__ void cp_async4(float *smem, const float *gmem) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(gmem) : "memory");
 }
+__device__ __forceinline__ void cp_async8(float *smem, const float *gmem) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gmem) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -178,12 +182,11 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
     const int need_cols = min(kTileW, t.bw - t.j0) + C::PADL + C::PH;
     const int nvec_row = (need_cols + 3) / 4;
     const int need_rows = min(kTileH, t.bh - t.i0) + 2 * C::PH;
-    // vectors [v_lo, v_hi) of a row lie inside this worker column's bulk and are 16-byte aligned
-    const bool fast = ((t.bw + 2 * C::IOFF) % 4) == 0;   // row pitch keeps every row 16-byte aligned
+    // vectors [v_lo, v_hi) of a row lie inside this worker column's bulk; whether they can be copied 16 or 8 bytes
+    // at a time depends on where the row starts in memory (a pitch of 4 k + 2 floats alternates between the two)
     const int first_col = t.j0 - C::PADL;                               // bulk column of tile column 0
-    int v_lo = first_col < 0 ? (-first_col + 3) / 4 : 0;
-    int v_hi = min(nvec_row, (t.bw - first_col) / 4);
-    if (!fast) v_lo = v_hi = 0;
+    const int v_lo_in = first_col < 0 ? (-first_col + 3) / 4 : 0;
+    const int v_hi_in = max(v_lo_in, min(nvec_row, (t.bw - first_col) / 4));
     for (int ry = warp; ry < need_rows; ry += kConvThreads / 32) {
         // which worker row owns bulk row i (warp-uniform), or none: outside the tensor
         int i = t.i0 - C::PH + ry, rr = t.r;
@@ -208,7 +211,15 @@ __device__ __forceinline__ void stage_tile(const ConvParams &P, const ConvTile &
         const int pitch_c = t.bw + 2 * C::IOFF;
         const float *grow = P.in[wofs + rr * P.pw_workers + t.c] + (size_t)t.plane * (rbh + 2 * C::IOFF) * pitch_c +
                             (size_t)(i + C::IOFF) * pitch_c + C::IOFF + first_col;
-        for (int v = v_lo + lane; v < v_hi; v += 32) cp_async16(srow + 4 * v, grow + 4 * v);
+        const uint32_t mis = (uint32_t)reinterpret_cast<uintptr_t>(grow) & 15u;
+        int v_lo = v_lo_in, v_hi = v_hi_in;
+        if (mis == 0) {
+            for (int v = v_lo + lane; v < v_hi; v += 32) cp_async16(srow + 4 * v, grow + 4 * v);
+        } else if (mis == 8) {
+            for (int u = 2 * v_lo + lane; u < 2 * v_hi; u += 32) cp_async8(srow + 2 * u, grow + 2 * u);
+        } else {
+            v_lo = v_hi = 0;            // element by element below
+        }
         // edge columns: left of v_lo and right of v_hi, element by element (neighbour columns or zero)
         const int n_left = 4 * v_lo, n_right = 4 * (nvec_row - v_hi);
         for (int e = lane; e < n_left + n_right; e += 32) {
