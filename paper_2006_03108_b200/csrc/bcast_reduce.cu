@@ -276,7 +276,11 @@ static distdl_status_t sumreduce_impl(const void *const *src, void *dst, int32_t
         switch (filled) {
             case 1: launch_sum<1>(fp, dst, filled, nvec, tail, grid, t, s); break;
             case 2: launch_sum<2>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 3: launch_sum<3>(fp, dst, filled, nvec, tail, grid, t, s); break;
             case 4: launch_sum<4>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 5: launch_sum<5>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 6: launch_sum<6>(fp, dst, filled, nvec, tail, grid, t, s); break;
+            case 7: launch_sum<7>(fp, dst, filled, nvec, tail, grid, t, s); break;
             case 8: launch_sum<8>(fp, dst, filled, nvec, tail, grid, t, s); break;
             default: launch_sum<0>(fp, dst, filled, nvec, tail, grid, t, s); break;
         }
