@@ -465,6 +465,9 @@ CONV_CASES = [
     ((1, 2, 70, 272), (1, 1, 2, 2), 5),      # bulk widths of whole groups of eight columns (136), two tile columns of 128 + 8
     ((1, 2, 70, 272), (1, 1, 2, 2), 3),      # the same for the adjoint of K = 3 (rows 8-byte aligned)
     ((1, 1, 70, 528), (1, 1, 2, 2), 7),      # and of K = 7 (264 columns per worker)
+    ((1, 41, 160, 384), (1, 1, 1, 3), 5),    # 615 tiles: more than the persistent grid holds (4 x 148 blocks), so blocks take a
+                                             # second turn with swapped neighbours, and the odd last tile has no partner
+    ((1, 41, 160, 384), (1, 1, 1, 3), 3),    # the same through the kernel without bulk tensor copies (forward)
 ]
 
 
