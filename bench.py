@@ -977,8 +977,8 @@ NCU_TRAFFIC = {
     "sumreduce_fwd": 4 * (134225152 + 5290496),
     "halo_fwd": 194266368 + 124569856,
     "halo_adj": (107870464 + 72062976) + (139435264 + 39406592),      # box kernel + row-end kernel
-    "conv_fwd": 1173479680 + 1030533632,
-    "conv_adj": 1178607872 + 1071105024,
+    "conv_fwd": 1137867008 + 1029683968,
+    "conv_adj": 1099090944 + 1063217152,
     "affine_fwd": 138435072 + 3728128,
     "affine_adj": 138447104 + 3240448,
 }
